@@ -1,0 +1,345 @@
+#!/usr/bin/env python
+"""Benchmark of the fused preprocessing path.
+
+A step is one pass of the path over one ragged batch: 256 images, H and W uniform in
+[240, 500], smooth-noise content, resize 256 / crop 224 / normalise, fp16 NCHW output.
+`value` is images/s with the packed batch already in device memory (one kernel launch per
+step); `e2e` is images/s from separate decoded host images: pack into pinned memory, copy
+in, kernel, copy the result out.  Prints one JSON line (rank 0).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--workload mixed|320x240|1080p|sweep] [--batch N]
+"""
+from __future__ import annotations
+
+import argparse
+import ctypes
+import hashlib
+import json
+import os
+import sys
+import threading
+import time
+from pathlib import Path
+
+import numpy as np
+
+ROOT = Path(__file__).resolve().parent
+if str(ROOT) not in sys.path:
+    sys.path.insert(0, str(ROOT))
+
+from paper_2411_19114_b200 import accounting  # noqa: E402
+from paper_2411_19114_b200 import workloads as wl  # noqa: E402
+
+METRIC = "preprocessed images/sec"
+UNIT = "images/s"
+FALLBACK_HBM_GBS = 6650.0
+
+# DRAM bytes (read + write) per launch of the kernel on the default workload, from one
+# ncu capture, valid only for the kernel sources with this digest (else reported as null).
+NCU_TRAFFIC = {"csrc_sha1": None, "bytes_per_launch": None}
+
+
+def csrc_digest() -> str:
+    h = hashlib.sha1()
+    for p in sorted((ROOT / "paper_2411_19114_b200" / "csrc").glob("*")):
+        if p.suffix in (".cu", ".cpp", ".h", ".cuh"):
+            h.update(p.read_bytes())
+    return h.hexdigest()
+
+
+def make_workload(name: str, batch: int | None, rank: int):
+    """(images, out dtype name, description).  Every rank draws its own batch."""
+    shift = 1000 * rank
+    if name == "mixed":
+        n = batch or 256
+        return wl.mixed_smooth(n, seed=2 + shift), "f16", \
+            f"{n} mixed-size images, H,W~U[240,500], smooth noise, fp16 out (ragged batch)"
+    if name == "320x240":
+        n = batch or 64
+        return wl.uniform_320x240(n, seed=1 + shift), "f32", \
+            f"{n} images 320x240, uniform bytes, fp32 out"
+    if name == "1080p":
+        n = batch or 64
+        return wl.hires_1080p(n, seed=4 + shift), "f32", \
+            f"{n} images 1920x1080, smooth noise, fp32 out"
+    if name == "sweep":
+        n = batch or 2048
+        return wl.sweep_500x375(n, seed=5 + shift), "f16", \
+            f"{n} images 500x375, uniform bytes, fp16 out"
+    raise SystemExit(f"unknown workload {name}")
+
+
+def measured_peak() -> tuple[float, str]:
+    p = ROOT / "MEASURED_PEAKS.json"
+    try:
+        return float(json.loads(p.read_text())["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (no MEASURED_PEAKS.json)"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU through NVML while a region runs."""
+
+    REASONS = {
+        0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
+        0x4: "sw_power_cap", 0x80: "hw_power_brake", 0x2: "applications_clocks_setting",
+        0x100: "display_clock_setting", 0x10: "sync_boost",
+    }
+
+    def __init__(self, index: int, period_s: float = 0.01):
+        self.index, self.period = index, period_s
+        self.sm, self.bits, self.max_mhz = [], 0, None
+        self._stop = threading.Event()
+        self._thread = None
+        self.error = None
+
+    def _run(self):
+        try:
+            import pynvml as nv
+
+            nv.nvmlInit()
+            uuid = None
+            try:
+                import torch
+
+                uuid = "GPU-" + str(torch.cuda.get_device_properties(self.index).uuid)
+            except Exception:
+                pass
+            try:
+                dev = nv.nvmlDeviceGetHandleByUUID(uuid.encode() if uuid else b"")
+            except Exception:
+                dev = nv.nvmlDeviceGetHandleByIndex(self.index)
+            self.max_mhz = int(nv.nvmlDeviceGetMaxClockInfo(dev, nv.NVML_CLOCK_SM))
+            while not self._stop.is_set():
+                self.sm.append(int(nv.nvmlDeviceGetClockInfo(dev, nv.NVML_CLOCK_SM)))
+                try:
+                    self.bits |= int(nv.nvmlDeviceGetCurrentClocksEventReasons(dev))
+                except Exception:
+                    self.bits |= int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(dev))
+                self._stop.wait(self.period)
+        except Exception as exc:  # NVML missing: report, do not invent numbers
+            self.error = repr(exc)
+
+    def __enter__(self):
+        self._thread = threading.Thread(target=self._run, daemon=True)
+        self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        self._thread.join(timeout=5)
+
+    def summary(self) -> dict:
+        if not self.sm:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [],
+                    "error": self.error or "no samples"}
+        reasons = [name for bit, name in self.REASONS.items() if self.bits & bit]
+        return {"sm_mhz": float(np.median(self.sm)), "sm_max_mhz": self.max_mhz,
+                "reasons": reasons, "samples": len(self.sm)}
+
+
+def cpu_threads() -> int:
+    return max(1, len(os.sched_getaffinity(0)))
+
+
+def time_oracle(images, out_kind_name: str, budget_s: float, max_passes: int):
+    """The oracle as it stands, all host threads, whole batch per pass."""
+    import oracle
+
+    kind = oracle.OUT_F16 if out_kind_name == "f16" else oracle.OUT_F32
+    packed, offsets, h, w = oracle.pack(images)
+    threads = min(cpu_threads(), len(images))
+    times = []
+    t_end = time.perf_counter() + budget_s
+    while len(times) < max_passes:
+        t0 = time.perf_counter()
+        oracle.preprocess_packed(packed, offsets, h, w, wl.OUT_SIZE, wl.RESIZE_SHORT, wl.MEAN,
+                                 wl.STD, kind, nthreads=threads)
+        times.append(time.perf_counter() - t0)
+        if time.perf_counter() > t_end:
+            break
+    return times, threads
+
+
+def run_reference(args, rank: int, world: int) -> None:
+    """The reference arm: the CPU oracle on the host cores (rank 0 only)."""
+    if rank != 0:
+        return
+    images, dtype, desc = make_workload(args.workload, args.batch, 0)
+    n = len(images)
+    warm, _ = time_oracle(images, dtype, 0.0, max(1, min(args.warmup, 1)))
+    times, threads = time_oracle(images, dtype, 60.0, max(1, args.steps))
+    total = float(sum(times))
+    value = n * len(times) / total
+    sample = f"whole batch of {n} images per step, {len(times)} steps (time budget 60 s)"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": len(times), "warmup": len(warm), "ms_per_step": 1e3 * total / len(times),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": {"workload": desc, "resize_short": wl.RESIZE_SHORT,
+                                        "out_size": wl.OUT_SIZE},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def run_ours(args, rank: int, world: int, local_rank: int) -> None:
+    import torch
+
+    from paper_2411_19114_b200 import binding as pb
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device (the CUDA path has no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.init_process_group("nccl", device_id=dev)
+    pb.lib()
+
+    images, dtype, desc = make_workload(args.workload, args.batch, rank)
+    n = len(images)
+    out_dtype = pb.F16 if dtype == "f16" else pb.F32
+    tdt = torch.float16 if dtype == "f16" else torch.float32
+    C, S = wl.OUT_SIZE, wl.RESIZE_SHORT
+
+    packed, table = pb.preba_pack(images)
+    acct = accounting.batch_bytes(table, C, S, 2 if dtype == "f16" else 4)
+    l2 = torch.cuda.get_device_properties(dev).L2_cache_size
+    step_bytes = packed.nbytes + acct["output_bytes"]
+    sets = max(2, min(64, -(-4 * l2 // step_bytes)))
+    pix = [torch.from_numpy(packed).to(dev) for _ in range(sets)]
+    outs = [torch.empty((n, 3, C, C), dtype=tdt, device=dev) for _ in range(sets)]
+    tab = torch.from_numpy(table.view(np.uint8)).to(dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    stream = torch.cuda.current_stream()
+
+    calls = [pb.PreparedPreprocess(pix[i], tab, n, outs[i], C, S, wl.MEAN, wl.STD, out_dtype,
+                                   stream=stream, status=status) for i in range(sets)]
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident throughput: one launch per step -------------------------------------
+    for i in range(max(args.warmup, 3)):
+        calls[i % sets]()
+    barrier()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local_rank) as clocks:
+        barrier()
+        start.record(stream)
+        for i in range(args.steps):
+            calls[i % sets]()
+        stop.record(stream)
+        barrier()
+    elapsed_ms = start.elapsed_time(stop)
+    assert int(status.item()) == 0, "kernel reported an error status"
+
+    # ---- end to end from host images ----------------------------------------------------------
+    e2e_steps = max(3, min(args.e2e_steps, args.steps))
+    sizes = pb.preba_query(table["h"], table["w"], C, out_dtype)
+    nbuf = 2
+    ph = [torch.empty(sizes.packed_bytes, dtype=torch.uint8).pin_memory() for _ in range(nbuf)]
+    oh = [torch.empty((n, 3, C, C), dtype=tdt).pin_memory() for _ in range(nbuf)]
+    th = [np.zeros(n, dtype=pb.TABLE_DTYPE) for _ in range(nbuf)]
+    dtab = [torch.empty(n * 16, dtype=torch.uint8, device=dev) for _ in range(nbuf)]
+    done = [torch.cuda.Event() for _ in range(nbuf)]
+
+    def e2e_step(i):
+        b = i % nbuf
+        done[b].synchronize()                       # the set's previous copies have finished
+        pb.preba_pack(images, ph[b].numpy(), th[b])
+        pb.preba_preprocess_host(ph[b], th[b], n, oh[b], pix[b], dtab[b], outs[b], C, S, wl.MEAN,
+                                 wl.STD, out_dtype, stream=stream, dev_status=status)
+        done[b].record(stream)
+
+    for i in range(2):
+        e2e_step(i)
+    barrier()
+    e_start, e_stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_pack = 0.0
+    e_start.record(stream)
+    for i in range(e2e_steps):
+        t0 = time.perf_counter()
+        e2e_step(i)
+        t_pack += time.perf_counter() - t0
+    e_stop.record(stream)
+    barrier()
+    e2e_ms = e_start.elapsed_time(e_stop)
+    assert int(status.item()) == 0
+
+    if dist is not None:
+        t = torch.tensor([elapsed_ms, e2e_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms, e2e_ms = (float(v) for v in t.tolist())
+
+    if rank == 0:
+        peak, peak_src = measured_peak()
+        per_launch_s = elapsed_ms * 1e-3 / args.steps
+        achieved = acct["total"] / per_launch_s / 1e9
+        traffic = NCU_TRAFFIC["bytes_per_launch"] \
+            if NCU_TRAFFIC["csrc_sha1"] == csrc_digest() and args.workload == "mixed" \
+            and not args.batch else None
+        cpu_times, threads = time_oracle(images, dtype, 12.0, 50)
+        cpu_value = n * len(cpu_times) / float(sum(cpu_times))
+        line = {
+            "metric": METRIC, "value": world * n * args.steps / (elapsed_ms * 1e-3), "unit": UNIT,
+            "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+            "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": desc, "resize_short": S, "out_size": C, "out_dtype": dtype,
+                       "images_per_step_per_gpu": n, "parallelism": f"dp{world} (independent batches)",
+                       "l2": f"rotating {sets} input/output buffer sets "
+                             f"({sets * step_bytes / 1e6:.0f} MB) > L2 ({l2 / 1e6:.0f} MB)"},
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                         "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src,
+                         "algorithmic_bytes_per_launch": acct["total"],
+                         "input_sector_bytes": acct["input_sector_bytes"],
+                         "output_bytes": acct["output_bytes"],
+                         "kernel_us": per_launch_s * 1e6},
+            "cpu_baseline": {"value": cpu_value, "unit": UNIT, "cores": threads, "kind": "oracle",
+                             "sample": f"whole batch of {n} images, {len(cpu_times)} passes"},
+            "e2e": {"value": world * n * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT,
+                    "h2d_bytes_per_step": int(sizes.packed_bytes + sizes.table_bytes),
+                    "d2h_bytes_per_step": int(sizes.out_bytes), "steps": e2e_steps,
+                    "ms_per_step": e2e_ms / e2e_steps,
+                    "host_ms_per_step": 1e3 * t_pack / e2e_steps,
+                    "includes": "preba_pack into pinned memory + H2D + kernel + D2H"},
+            "gpu_launches": args.steps,
+            "clocks": clocks.summary(),
+        }
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20000)
+    ap.add_argument("--warmup", type=int, default=200)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="mixed", choices=["mixed", "320x240", "1080p", "sweep"])
+    ap.add_argument("--batch", type=int, default=None)
+    ap.add_argument("--e2e-steps", type=int, default=20)
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+    else:
+        run_ours(args, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()

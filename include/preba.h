@@ -1,0 +1,167 @@
+/*
+ * preba.h — C ABI of the fused vision-preprocessing library for B200 (sm_100a).
+ *
+ * The path is the per-query image preprocessing that runs in front of the model
+ * (paper Sec. 2.3 item 1, Fig. 4; Table 1 rows "Resize", "Crop", "Normalize"):
+ * every decoded uint8 RGB image of a ragged batch is resized (shorter side to
+ * `resize_short`, bilinear, half-pixel centres, edge clamp, no antialias),
+ * center-cropped to `out_size` x `out_size`, converted to float with
+ * out = (v/255 - mean_c)/std_c, and written as plane c, row k, column j of a
+ * dense [n, 3, out_size, out_size] tensor.  As in the paper's pipelined
+ * compute unit (Sec. 4.2), the stages are chained on chip: one kernel launch
+ * per batch, no intermediate image in device memory.
+ *
+ * Conventions for every entry point
+ *   - Plain C.  Returns PREBA_OK (0) or a negative PREBA_ERR_* code; nothing
+ *     is thrown, printed or allocated, and no call synchronises the device.
+ *   - Pointers are marked HOST or DEVICE.  The caller owns every buffer; the
+ *     library borrows HOST arguments for the duration of the call and DEVICE
+ *     buffers until the stream has passed the work the call enqueued.
+ *   - Calls keep no state between them and may be made concurrently from
+ *     several threads, each on its own stream.
+ */
+#ifndef PREBA_H_
+#define PREBA_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define PREBA_PACK_ALIGN 128u     /* every image offset, and the packed size, is a multiple */
+#define PREBA_MAX_DIM 32768u      /* largest accepted image height or width */
+#define PREBA_MAX_RESIZE 16384u   /* largest accepted resize_short (and so out_size) */
+
+#define PREBA_OK 0
+#define PREBA_ERR_INVALID_ARG (-1)      /* NULL, zero or out-of-range argument, misaligned buffer */
+#define PREBA_ERR_BUFFER_TOO_SMALL (-2) /* a capacity is below what preba_query reports */
+#define PREBA_ERR_BAD_TABLE (-3)        /* a table entry is misaligned, out of range or past the pixels */
+#define PREBA_ERR_CUDA (-4)             /* a CUDA runtime call failed; see preba_last_cuda_error */
+#define PREBA_ERR_TIMEOUT (-5)          /* only in the device status word: a bounded wait ran out */
+
+typedef enum { PREBA_F32 = 0, PREBA_F16 = 1 } preba_dtype_t;
+
+/* One image of the packed batch: `offset` is in bytes from the start of the
+ * pixel buffer and a multiple of PREBA_PACK_ALIGN; the image is h rows of w
+ * RGB pixels, 3 bytes per pixel, row pitch exactly 3*w bytes. */
+typedef struct {
+  uint64_t offset;
+  uint32_t h;
+  uint32_t w;
+} preba_img_t;
+
+typedef struct {
+  uint64_t packed_bytes; /* size of the packed pixel buffer */
+  uint64_t table_bytes;  /* n * sizeof(preba_img_t) */
+  uint64_t out_bytes;    /* n * 3 * out_size^2 * sizeof(out element) */
+  uint32_t align;        /* PREBA_PACK_ALIGN */
+  uint32_t reserved;
+} preba_sizes_t;
+
+/* A batch resident in device memory. */
+typedef struct {
+  const uint8_t* pixels;         /* DEVICE, base aligned to 16 bytes, packed as preba_pack lays out */
+  uint64_t pixels_bytes;         /* bytes readable at `pixels` (>= sizes.packed_bytes) */
+  const preba_img_t* table;      /* DEVICE, n entries */
+  const preba_img_t* table_host; /* HOST copy of the table for checking before launch, or NULL */
+  uint32_t n;                    /* images in the batch, >= 1 */
+  uint32_t reserved;
+  void* out;                     /* DEVICE, [n,3,out_size,out_size] contiguous, 16-byte aligned */
+  uint64_t out_bytes;            /* bytes writable at `out` (>= sizes.out_bytes) */
+  int32_t* status;               /* DEVICE word or NULL: the kernel stores the first PREBA_ERR_*
+                                    it meets (bad table entry, wait that ran out); caller zeroes it */
+} preba_batch_t;
+
+/* A batch resident in host memory, with the device buffers the call stages it through. */
+typedef struct {
+  const uint8_t* packed_host;    /* HOST (pinned for an asynchronous copy), packed_bytes bytes */
+  uint64_t packed_bytes;
+  const preba_img_t* table_host; /* HOST, n entries */
+  uint32_t n;
+  uint32_t reserved;
+  void* out_host;                /* HOST (pinned for an asynchronous copy), out_bytes bytes */
+  uint64_t out_bytes;
+  uint8_t* dev_pixels;           /* DEVICE staging, >= packed_bytes, 16-byte aligned */
+  preba_img_t* dev_table;        /* DEVICE staging, n entries */
+  void* dev_out;                 /* DEVICE staging, >= out_bytes, 16-byte aligned */
+  int32_t* dev_status;           /* DEVICE word or NULL, as preba_batch_t.status */
+} preba_host_batch_t;
+
+/*
+ * preba_query — sizes of the buffers a batch needs (host arithmetic only).
+ * The packed layout is the problem statement's, not the paper's (which handles
+ * each single-input request on its own, Sec. 5 "Input query modeling"): images
+ * are concatenated in order, each starting at the running byte count rounded
+ * up to PREBA_PACK_ALIGN, and the total is rounded up as well.
+ *   h, w      HOST, n entries each, every value in [1, PREBA_MAX_DIM]
+ *   out_size  side of the square crop, >= 1
+ *   out_dtype PREBA_F32 or PREBA_F16
+ *   sizes     HOST, written on success
+ * Errors: PREBA_ERR_INVALID_ARG.
+ */
+int preba_query(const uint32_t* h, const uint32_t* w, uint32_t n, uint32_t out_size,
+                int out_dtype, preba_sizes_t* sizes);
+
+/*
+ * preba_pack — step 0 of the path: builds the packed pixel buffer and the
+ * {offset, h, w} table from n separate decoded images (each HWC uint8, row
+ * pitch 3*w).  Padding bytes between images and at the tail are written as 0,
+ * so the result is a pure function of the inputs.
+ *   images    HOST array of n HOST pointers
+ *   packed    HOST, `capacity` bytes; must hold sizes.packed_bytes
+ *   table     HOST, n entries, written
+ * Errors: PREBA_ERR_INVALID_ARG, PREBA_ERR_BUFFER_TOO_SMALL.
+ */
+int preba_pack(const uint8_t* const* images, const uint32_t* h, const uint32_t* w, uint32_t n,
+               uint8_t* packed, uint64_t capacity, preba_img_t* table);
+
+/*
+ * preba_preprocess — the transform (Resize -> Crop -> Normalize of Table 1,
+ * fused as the paper's compute unit chains them, Sec. 4.2), on a device-resident
+ * batch.  Enqueues exactly one kernel on `stream` and returns.
+ *   out_size      crop side C, 1 <= C <= resize_short
+ *   resize_short  target length S of the shorter side, <= PREBA_MAX_RESIZE;
+ *                 the longer side becomes floor(S*long/short)
+ *   mean, std     HOST, 3 floats each, copied at call time; std finite, non-zero
+ *   out_dtype     PREBA_F32 or PREBA_F16 (round to nearest even)
+ *   stream        a cudaStream_t (NULL = the default stream)
+ * Per image: crop origin floor((R - C)/2) on each axis; output index j samples
+ * source coordinate ((j + origin) + 1/2) * in/R - 1/2, clamped to [0, in-1];
+ * taps and weights come from exact integer arithmetic, interpolation and the
+ * normalising multiply-add run in fp32, with no rounding to uint8 in between.
+ * If `table_host` is given, entries are checked before launch
+ * (PREBA_ERR_BAD_TABLE).  The kernel checks each entry again on the device: a
+ * bad entry is skipped, its output left untouched, and PREBA_ERR_BAD_TABLE is
+ * stored in `status`.
+ * Errors: PREBA_ERR_INVALID_ARG, PREBA_ERR_BUFFER_TOO_SMALL,
+ * PREBA_ERR_BAD_TABLE, PREBA_ERR_CUDA.
+ */
+int preba_preprocess(const preba_batch_t* batch, uint32_t out_size, uint32_t resize_short,
+                     const float mean[3], const float std[3], int out_dtype, void* stream);
+
+/*
+ * preba_preprocess_host — the same transform for a batch held in host memory
+ * (the request path of the paper's server: inputs arrive in host memory and
+ * results return to it, Sec. 4.2 "Implication of adding DPU").  Enqueues on
+ * `stream`: copy of the packed pixels and the table to the device staging
+ * buffers, the kernel, and the copy of the result to `out_host`; then returns.
+ * The host buffers must stay valid and unchanged until the stream has passed
+ * these operations; use pinned memory for the copies to be asynchronous.
+ * The table is always checked on the host first.
+ * Errors: as preba_preprocess.
+ */
+int preba_preprocess_host(const preba_host_batch_t* batch, uint32_t out_size,
+                          uint32_t resize_short, const float mean[3], const float std[3],
+                          int out_dtype, void* stream);
+
+/* Text for a PREBA_* code (static storage, never NULL). */
+const char* preba_strerror(int code);
+
+/* The cudaError_t value behind the calling thread's last PREBA_ERR_CUDA, else 0. */
+int preba_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PREBA_H_ */

@@ -1,0 +1,266 @@
+"""ctypes binding of ``libpreba.so`` — argument marshalling only.
+
+Function names and meanings are those of ``include/preba.h``.  Device memory and
+streams come from PyTorch; nothing here computes any part of the transform.  If
+the library has not been built the first call raises: there is no fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+
+import numpy as np
+
+_LIB_PATH = Path(__file__).resolve().parent / "libpreba.so"
+
+PACK_ALIGN = 128
+F32, F16 = 0, 1
+
+OK = 0
+ERR_INVALID_ARG = -1
+ERR_BUFFER_TOO_SMALL = -2
+ERR_BAD_TABLE = -3
+ERR_CUDA = -4
+ERR_TIMEOUT = -5
+
+EXPORTS = ("preba_query", "preba_pack", "preba_preprocess", "preba_preprocess_host",
+           "preba_strerror", "preba_last_cuda_error")
+
+
+class PrebaImg(ctypes.Structure):
+    _fields_ = [("offset", ctypes.c_uint64), ("h", ctypes.c_uint32), ("w", ctypes.c_uint32)]
+
+
+class PrebaSizes(ctypes.Structure):
+    _fields_ = [("packed_bytes", ctypes.c_uint64), ("table_bytes", ctypes.c_uint64),
+                ("out_bytes", ctypes.c_uint64), ("align", ctypes.c_uint32),
+                ("reserved", ctypes.c_uint32)]
+
+
+class PrebaBatch(ctypes.Structure):
+    _fields_ = [("pixels", ctypes.c_void_p), ("pixels_bytes", ctypes.c_uint64),
+                ("table", ctypes.c_void_p), ("table_host", ctypes.c_void_p),
+                ("n", ctypes.c_uint32), ("reserved", ctypes.c_uint32),
+                ("out", ctypes.c_void_p), ("out_bytes", ctypes.c_uint64),
+                ("status", ctypes.c_void_p)]
+
+
+class PrebaHostBatch(ctypes.Structure):
+    _fields_ = [("packed_host", ctypes.c_void_p), ("packed_bytes", ctypes.c_uint64),
+                ("table_host", ctypes.c_void_p), ("n", ctypes.c_uint32),
+                ("reserved", ctypes.c_uint32), ("out_host", ctypes.c_void_p),
+                ("out_bytes", ctypes.c_uint64), ("dev_pixels", ctypes.c_void_p),
+                ("dev_table", ctypes.c_void_p), ("dev_out", ctypes.c_void_p),
+                ("dev_status", ctypes.c_void_p)]
+
+
+TABLE_DTYPE = np.dtype([("offset", "<u8"), ("h", "<u4"), ("w", "<u4")])
+
+
+class PrebaError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        text = lib().preba_strerror(code).decode()
+        extra = f" (cudaError {lib().preba_last_cuda_error()})" if code == ERR_CUDA else ""
+        super().__init__(f"{where}: {text} [{code}]{extra}")
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded library; raises if it is missing."""
+    global _lib
+    if _lib is None:
+        if not _LIB_PATH.exists():
+            raise RuntimeError(
+                f"{_LIB_PATH} is missing: build it with "
+                "`python -m paper_2411_19114_b200.build` (there is no CPU fallback)")
+        L = ctypes.CDLL(str(_LIB_PATH))
+        u32p = ctypes.POINTER(ctypes.c_uint32)
+        f32p = ctypes.POINTER(ctypes.c_float)
+        L.preba_query.argtypes = [u32p, u32p, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_int,
+                                  ctypes.POINTER(PrebaSizes)]
+        L.preba_pack.argtypes = [ctypes.POINTER(ctypes.c_void_p), u32p, u32p, ctypes.c_uint32,
+                                 ctypes.c_void_p, ctypes.c_uint64, ctypes.c_void_p]
+        L.preba_preprocess.argtypes = [ctypes.POINTER(PrebaBatch), ctypes.c_uint32,
+                                       ctypes.c_uint32, f32p, f32p, ctypes.c_int, ctypes.c_void_p]
+        L.preba_preprocess_host.argtypes = [ctypes.POINTER(PrebaHostBatch), ctypes.c_uint32,
+                                            ctypes.c_uint32, f32p, f32p, ctypes.c_int,
+                                            ctypes.c_void_p]
+        L.preba_strerror.argtypes = [ctypes.c_int]
+        L.preba_strerror.restype = ctypes.c_char_p
+        L.preba_last_cuda_error.argtypes = []
+        for name in ("preba_query", "preba_pack", "preba_preprocess", "preba_preprocess_host",
+                     "preba_last_cuda_error"):
+            getattr(L, name).restype = ctypes.c_int
+        _lib = L
+    return _lib
+
+
+def _u32(a) -> np.ndarray:
+    return np.ascontiguousarray(np.asarray(a, dtype=np.uint32))
+
+
+def _f3(v):
+    a = np.ascontiguousarray(np.asarray(v, dtype=np.float32))
+    if a.shape != (3,):
+        raise ValueError("mean/std must have 3 entries")
+    return a
+
+
+def _p(a: np.ndarray, ctype):
+    return a.ctypes.data_as(ctypes.POINTER(ctype))
+
+
+def preba_strerror(code: int) -> str:
+    return lib().preba_strerror(code).decode()
+
+
+def preba_query(h, w, out_size: int, out_dtype: int) -> PrebaSizes:
+    h, w = _u32(h), _u32(w)
+    sizes = PrebaSizes()
+    rc = lib().preba_query(_p(h, ctypes.c_uint32), _p(w, ctypes.c_uint32), len(h), out_size,
+                           out_dtype, ctypes.byref(sizes))
+    if rc != OK:
+        raise PrebaError(rc, "preba_query")
+    return sizes
+
+
+def preba_pack(images, packed: np.ndarray | None = None, table: np.ndarray | None = None):
+    """Pack a list of HWC uint8 arrays.  ``packed``/``table`` may be caller-provided
+    (e.g. views of pinned memory); returns (packed, table)."""
+    imgs = [np.ascontiguousarray(im, dtype=np.uint8) for im in images]
+    n = len(imgs)
+    for im in imgs:
+        if im.ndim != 3 or im.shape[2] != 3:
+            raise ValueError("images must be HWC with 3 channels")
+    h = _u32([im.shape[0] for im in imgs])
+    w = _u32([im.shape[1] for im in imgs])
+    if packed is None:
+        total = preba_query(h, w, 1, F32).packed_bytes
+        packed = np.empty(total, dtype=np.uint8)
+    if table is None:
+        table = np.zeros(n, dtype=TABLE_DTYPE)
+    if packed.dtype != np.uint8 or not packed.flags.c_contiguous:
+        raise ValueError("packed must be a contiguous uint8 array")
+    if table.dtype != TABLE_DTYPE or len(table) < n or not table.flags.c_contiguous:
+        raise ValueError("table must be a contiguous TABLE_DTYPE array with n entries")
+    ptrs = (ctypes.c_void_p * n)(*[im.ctypes.data for im in imgs])
+    rc = lib().preba_pack(ptrs, _p(h, ctypes.c_uint32), _p(w, ctypes.c_uint32), n,
+                          packed.ctypes.data, packed.nbytes, table.ctypes.data)
+    if rc != OK:
+        raise PrebaError(rc, "preba_pack")
+    return packed, table
+
+
+def preba_preprocess(pixels, table, n: int, out, out_size: int, resize_short: int, mean, std,
+                     out_dtype: int, stream=None, table_host: np.ndarray | None = None,
+                     status=None, pixels_bytes: int | None = None,
+                     out_bytes: int | None = None) -> None:
+    """``pixels``, ``table``, ``out`` and ``status`` are CUDA tensors (or raw device
+    addresses); ``stream`` is a torch stream, a raw cudaStream_t or None for torch's
+    current stream."""
+    import torch
+
+    def addr(t):
+        return int(t) if isinstance(t, int) else t.data_ptr()
+
+    def nbytes(t, given):
+        if given is not None:
+            return given
+        return t.numel() * t.element_size()
+
+    if stream is None:
+        stream = torch.cuda.current_stream().cuda_stream
+    elif hasattr(stream, "cuda_stream"):
+        stream = stream.cuda_stream
+    batch = PrebaBatch()
+    batch.pixels = addr(pixels)
+    batch.pixels_bytes = nbytes(pixels, pixels_bytes)
+    batch.table = addr(table)
+    batch.table_host = table_host.ctypes.data if table_host is not None else None
+    batch.n = n
+    batch.out = addr(out)
+    batch.out_bytes = nbytes(out, out_bytes)
+    batch.status = addr(status) if status is not None else None
+    m, s = _f3(mean), _f3(std)
+    rc = lib().preba_preprocess(ctypes.byref(batch), out_size, resize_short,
+                                _p(m, ctypes.c_float), _p(s, ctypes.c_float), out_dtype,
+                                ctypes.c_void_p(stream))
+    if rc != OK:
+        raise PrebaError(rc, "preba_preprocess")
+
+
+class PreparedPreprocess:
+    """The arguments of one ``preba_preprocess`` call, marshalled once; calling the object
+    makes the foreign call and nothing else (for loops that launch back to back)."""
+
+    def __init__(self, pixels, table, n: int, out, out_size: int, resize_short: int, mean, std,
+                 out_dtype: int, stream=None, table_host: np.ndarray | None = None, status=None):
+        import torch
+
+        if stream is None:
+            stream = torch.cuda.current_stream().cuda_stream
+        elif hasattr(stream, "cuda_stream"):
+            stream = stream.cuda_stream
+        self._keep = (pixels, table, out, status, table_host)
+        b = PrebaBatch()
+        b.pixels = pixels.data_ptr()
+        b.pixels_bytes = pixels.numel() * pixels.element_size()
+        b.table = table.data_ptr()
+        b.table_host = table_host.ctypes.data if table_host is not None else None
+        b.n = n
+        b.out = out.data_ptr()
+        b.out_bytes = out.numel() * out.element_size()
+        b.status = status.data_ptr() if status is not None else None
+        self._batch = b
+        self._mean, self._std = _f3(mean), _f3(std)
+        self._args = (ctypes.byref(b), out_size, resize_short, _p(self._mean, ctypes.c_float),
+                      _p(self._std, ctypes.c_float), out_dtype, ctypes.c_void_p(stream))
+        self._fn = lib().preba_preprocess
+
+    def __call__(self) -> None:
+        rc = self._fn(*self._args)
+        if rc != OK:
+            raise PrebaError(rc, "preba_preprocess")
+
+
+def preba_preprocess_host(packed_host, table_host: np.ndarray, n: int, out_host, dev_pixels,
+                          dev_table, dev_out, out_size: int, resize_short: int, mean, std,
+                          out_dtype: int, stream=None, dev_status=None) -> None:
+    """``packed_host``/``out_host`` are (pinned) CPU tensors or numpy arrays; ``dev_*`` are
+    CUDA tensors used as staging."""
+    import torch
+
+    def haddr(t):
+        return t.ctypes.data if isinstance(t, np.ndarray) else t.data_ptr()
+
+    def hbytes(t):
+        return t.nbytes if isinstance(t, np.ndarray) else t.numel() * t.element_size()
+
+    if stream is None:
+        stream = torch.cuda.current_stream().cuda_stream
+    elif hasattr(stream, "cuda_stream"):
+        stream = stream.cuda_stream
+    b = PrebaHostBatch()
+    b.packed_host = haddr(packed_host)
+    b.packed_bytes = hbytes(packed_host)
+    b.table_host = table_host.ctypes.data
+    b.n = n
+    b.out_host = haddr(out_host)
+    b.out_bytes = hbytes(out_host)
+    if dev_pixels.numel() * dev_pixels.element_size() < b.packed_bytes:
+        raise PrebaError(ERR_BUFFER_TOO_SMALL, "preba_preprocess_host (dev_pixels)")
+    if dev_out.numel() * dev_out.element_size() < b.out_bytes:
+        raise PrebaError(ERR_BUFFER_TOO_SMALL, "preba_preprocess_host (dev_out)")
+    b.dev_pixels = dev_pixels.data_ptr()
+    b.dev_table = dev_table.data_ptr()
+    b.dev_out = dev_out.data_ptr()
+    b.dev_status = dev_status.data_ptr() if dev_status is not None else None
+    m, s = _f3(mean), _f3(std)
+    rc = lib().preba_preprocess_host(ctypes.byref(b), out_size, resize_short,
+                                     _p(m, ctypes.c_float), _p(s, ctypes.c_float), out_dtype,
+                                     ctypes.c_void_p(stream))
+    if rc != OK:
+        raise PrebaError(rc, "preba_preprocess_host")

@@ -1,0 +1,17 @@
+// Shared between the host-only and the CUDA translation units of the library.
+#ifndef PREBA_INTERNAL_H_
+#define PREBA_INTERNAL_H_
+
+#include <stdint.h>
+
+#include "preba.h"
+
+namespace preba {
+
+bool dtype_ok(int out_dtype);
+bool dims_ok(uint32_t h, uint32_t w);
+uint64_t align_up(uint64_t v, uint64_t a);
+
+}  // namespace preba
+
+#endif  // PREBA_INTERNAL_H_

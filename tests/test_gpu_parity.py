@@ -1,0 +1,178 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same
+seeded inputs.  fp32 output: max abs error <= 1e-5; fp16 output: <= 1 binary16 ulp of the
+once-rounded double result, or within 1e-5 of the double result (helpers.fp16_report)."""
+from __future__ import annotations
+
+import numpy as np
+import pytest
+
+from paper_2411_19114_b200 import binding as pb
+from paper_2411_19114_b200 import workloads as wl
+
+from helpers import MEAN, STD, assert_parity, oracle_f64, run_gpu
+
+pytestmark = pytest.mark.gpu
+
+DTYPES = [pb.F32, pb.F16]
+
+
+def uniform(seed, h, w):
+    return wl.uniform_image(np.random.default_rng(seed), h, w)
+
+
+# ---- small cases that still span several slabs and a ragged tail --------------------------------
+
+SHAPES = [
+    (1, 1), (1, 9), (9, 1), (2, 2), (7, 7), (224, 224), (256, 256), (240, 320), (320, 240),
+    (375, 500), (500, 375), (257, 255), (255, 257), (256, 341), (333, 471), (240, 500), (500, 240),
+    (100, 3000), (3000, 100), (64, 64), (31, 517), (1080, 1920),
+]
+
+
+@pytest.mark.parametrize("dt", DTYPES)
+def test_single_images_of_many_shapes(dt):
+    for i, (h, w) in enumerate(SHAPES):
+        img = uniform(300 + i, h, w)
+        got = run_gpu([img], 224, 256, out_dtype=dt)
+        assert_parity(got, oracle_f64([img], 224, 256), dt)
+
+
+@pytest.mark.parametrize("dt", DTYPES)
+@pytest.mark.parametrize("c,s", [(1, 1), (1, 7), (7, 7), (8, 8), (9, 17), (33, 40), (224, 224),
+                                 (225, 225), (300, 301), (64, 256)])
+def test_other_crop_and_resize_sizes(dt, c, s):
+    imgs = [uniform(400 + i, h, w) for i, (h, w) in enumerate([(37, 53), (53, 37), (8, 8), (90, 400)])]
+    got = run_gpu(imgs, c, s, out_dtype=dt)
+    assert_parity(got, oracle_f64(imgs, c, s), dt)
+
+
+@pytest.mark.parametrize("dt", DTYPES)
+def test_ragged_batch_with_odd_strides(dt):
+    # widths whose row pitch 3*w is not a multiple of 16, images that end at the buffer end
+    sizes = [(241, 243), (250, 499), (499, 250), (300, 301), (263, 487), (1, 1), (240, 240),
+             (311, 313), (500, 500), (247, 331)]
+    imgs = [uniform(500 + i, h, w) for i, (h, w) in enumerate(sizes)]
+    got = run_gpu(imgs, 224, 256, out_dtype=dt)
+    assert_parity(got, oracle_f64(imgs, 224, 256), dt)
+
+
+def test_other_normalisation_constants_and_constant_images():
+    imgs = [np.full((260, 300, 3), v, dtype=np.uint8) for v in (0, 1, 128, 255)]
+    mean, std = (0.1, 0.5, 0.9), (1.0, 0.05, 2.5)
+    got = run_gpu(imgs, 224, 256, mean, std, pb.F32)
+    want = oracle_f64(imgs, 224, 256, mean, std)
+    assert_parity(got, want, pb.F32)
+    # a constant image gives one value per plane
+    for i in range(4):
+        for ch in range(3):
+            assert np.unique(got[i, ch]).size == 1
+
+
+def test_extreme_downscale_and_upscale():
+    imgs = [uniform(600, 4000, 3000), uniform(601, 20, 4000), uniform(602, 3, 2)]
+    for dt in DTYPES:
+        got = run_gpu(imgs, 224, 256, out_dtype=dt)
+        assert_parity(got, oracle_f64(imgs, 224, 256), dt)
+
+
+# ---- the workloads at full size -------------------------------------------------------------------
+
+def test_workload_uniform_320x240_fp32_full():
+    imgs = wl.uniform_320x240()
+    got = run_gpu(imgs, wl.OUT_SIZE, wl.RESIZE_SHORT, out_dtype=pb.F32)
+    rep = assert_parity(got, oracle_f64(imgs, wl.OUT_SIZE, wl.RESIZE_SHORT), pb.F32)
+    print("320x240 fp32:", rep)
+
+
+def test_workload_mixed_smooth_fp16_full():
+    imgs = wl.mixed_smooth()
+    got = run_gpu(imgs, wl.OUT_SIZE, wl.RESIZE_SHORT, out_dtype=pb.F16)
+    rep = assert_parity(got, oracle_f64(imgs, wl.OUT_SIZE, wl.RESIZE_SHORT), pb.F16)
+    print("mixed fp16:", rep)
+
+
+def test_workload_hires_1080p_fp32_full():
+    imgs = wl.hires_1080p()
+    got = run_gpu(imgs, wl.OUT_SIZE, wl.RESIZE_SHORT, out_dtype=pb.F32)
+    rep = assert_parity(got, oracle_f64(imgs, wl.OUT_SIZE, wl.RESIZE_SHORT), pb.F32)
+    print("1080p fp32:", rep)
+
+
+def test_workload_sweep_500x375_fp16_full_batch_sampled_images():
+    imgs = wl.sweep_500x375(2048)
+    got = run_gpu(imgs, wl.OUT_SIZE, wl.RESIZE_SHORT, out_dtype=pb.F16)
+    rng = np.random.default_rng(7)
+    pick = sorted(set([0, 1, 2047, 1024]) | set(int(v) for v in rng.integers(0, 2048, size=60)))
+    want = oracle_f64([imgs[i] for i in pick], wl.OUT_SIZE, wl.RESIZE_SHORT)
+    rep = assert_parity(got[pick], want, pb.F16)
+    print("sweep fp16:", rep)
+    # prefixes of the batch give the same bits as the full batch (batch-size sweep)
+    for n in (1, 8, 32):
+        sub = run_gpu(imgs[:n], wl.OUT_SIZE, wl.RESIZE_SHORT, out_dtype=pb.F16)
+        assert np.array_equal(sub.view(np.uint16), got[:n].view(np.uint16))
+
+
+# ---- robustness ---------------------------------------------------------------------------------------
+
+def test_output_is_independent_of_batch_position():
+    a, b, c = uniform(700, 300, 420), uniform(701, 480, 250), uniform(702, 256, 256)
+    alone = run_gpu([a], 224, 256, out_dtype=pb.F16)[0]
+    for batch, idx in (([a, b, c], 0), ([b, a, c], 1), ([c, b, a], 2)):
+        got = run_gpu(batch, 224, 256, out_dtype=pb.F16)[idx]
+        assert np.array_equal(got.view(np.uint16), alone.view(np.uint16))
+
+
+def test_streams_give_the_same_bits_as_a_serial_run():
+    import torch
+
+    batches = [wl.server_batch_500x375(s, 8) for s in range(3)]
+    serial = [run_gpu(b, 224, 256, out_dtype=pb.F16) for b in batches]
+    streams = [torch.cuda.Stream() for _ in batches]
+    for b, st, want in zip(batches, streams, serial):
+        got = run_gpu(b, 224, 256, out_dtype=pb.F16, stream=st)
+        assert np.array_equal(got.view(np.uint16), want.view(np.uint16))
+
+
+def test_device_side_table_check_skips_bad_entries():
+    import torch
+
+    imgs = [uniform(800, 64, 64), uniform(801, 64, 64)]
+    packed, table = pb.preba_pack(imgs)
+    bad = table.copy()
+    bad[1]["offset"] = 1 << 30          # far past the pixel buffer
+    dev = torch.device("cuda:0")
+    pix = torch.from_numpy(packed).to(dev)
+    tab = torch.from_numpy(bad.view(np.uint8)).to(dev)
+    out = torch.full((2, 3, 32, 32), 7.0, dtype=torch.float32, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    pb.preba_preprocess(pix, tab, 2, out, 32, 48, MEAN, STD, pb.F32, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == pb.ERR_BAD_TABLE
+    assert torch.all(out[1] == 7.0)     # untouched
+    want = oracle_f64(imgs[:1], 32, 48)
+    assert_parity(out[:1].cpu().numpy(), want, pb.F32)
+    # the host-side check catches the same entry before launch
+    with pytest.raises(pb.PrebaError) as e:
+        pb.preba_preprocess(pix, tab, 2, out, 32, 48, MEAN, STD, pb.F32, table_host=bad)
+    assert e.value.code == pb.ERR_BAD_TABLE
+
+
+def test_host_buffer_entry_point_matches_device_entry_point():
+    import torch
+
+    imgs = wl.mixed_smooth(12, seed=9)
+    packed, table = pb.preba_pack(imgs)
+    n = len(imgs)
+    dev = torch.device("cuda:0")
+    ph = torch.from_numpy(packed).pin_memory()
+    oh = torch.zeros((n, 3, 224, 224), dtype=torch.float16).pin_memory()
+    dp = torch.empty(packed.nbytes, dtype=torch.uint8, device=dev)
+    dtab = torch.empty(n * 16, dtype=torch.uint8, device=dev)
+    dout = torch.empty((n, 3, 224, 224), dtype=torch.float16, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    pb.preba_preprocess_host(ph, table, n, oh, dp, dtab, dout, 224, 256, MEAN, STD, pb.F16,
+                             dev_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    want = run_gpu(imgs, 224, 256, out_dtype=pb.F16)
+    assert np.array_equal(oh.numpy().view(np.uint16), want.view(np.uint16))
