@@ -288,7 +288,7 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
         traffic = NCU_TRAFFIC["bytes_per_launch"] \
             if NCU_TRAFFIC["csrc_sha1"] == csrc_digest() and args.workload == "mixed" \
             and not args.batch else None
-        cpu_times, threads = time_oracle(images, dtype, 12.0, 50)
+        cpu_times, threads = time_oracle(images, dtype, args.cpu_budget, 50)
         cpu_value = n * len(cpu_times) / float(sum(cpu_times))
         line = {
             "metric": METRIC, "value": world * n * args.steps / (elapsed_ms * 1e-3), "unit": UNIT,
@@ -331,6 +331,8 @@ def main() -> None:
     ap.add_argument("--workload", default="mixed", choices=["mixed", "320x240", "1080p", "sweep"])
     ap.add_argument("--batch", type=int, default=None)
     ap.add_argument("--e2e-steps", type=int, default=20)
+    ap.add_argument("--cpu-budget", type=float, default=12.0,
+                    help="seconds of wall time given to the CPU-baseline leg")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
