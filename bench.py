@@ -236,8 +236,10 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
     with ClockSampler(local_rank) as clocks:
         barrier()
         start.record(stream)
+        t_host = time.perf_counter()
         for i in range(args.steps):
             calls[i % sets]()
+        t_host = time.perf_counter() - t_host
         stop.record(stream)
         barrier()
     elapsed_ms = start.elapsed_time(stop)
@@ -304,7 +306,8 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
                          "algorithmic_bytes_per_launch": acct["total"],
                          "input_sector_bytes": acct["input_sector_bytes"],
                          "output_bytes": acct["output_bytes"],
-                         "kernel_us": per_launch_s * 1e6},
+                         "kernel_us": per_launch_s * 1e6,
+                         "host_launch_us": 1e6 * t_host / args.steps},
             "cpu_baseline": {"value": cpu_value, "unit": UNIT, "cores": threads, "kind": "oracle",
                              "sample": f"whole batch of {n} images, {len(cpu_times)} passes"},
             "e2e": {"value": world * n * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT,

@@ -1,20 +1,21 @@
 // Fused resize -> center crop -> normalise -> HWC->NCHW for a ragged batch (sm_100a).
 //
-// One launch per batch.  The grid is persistent: each CTA walks over tiles, a tile being a
-// slab of output rows (times a block of up to 256 output columns) of one image.  Inside a
-// CTA one producer warp reads the image's {offset, h, w} from the device table, derives
-// the sampling grid in exact integers, and streams the tapped source rows into a ring of
-// shared-memory stages with bulk asynchronous copies (one per row, 16-byte aligned,
-// completion counted on an mbarrier).  Four consumer warps follow the ring: per staged
-// row every thread interpolates horizontally for its two output columns, keeps the
-// previous row's result in registers, and emits an output row whenever both of its source
-// rows have passed -- vertical interpolation, normalising multiply-add, conversion and a
-// vectorised planar store.  The ring keeps filling across tile boundaries, so the copies
-// of the next tile are in flight while the current one is computed; nothing but the
-// input bytes and the output tensor touches device memory.
+// One launch per batch, persistent grid.  Every warp works on its own: it claims a task
+// (a slab of output rows of one image, up to 224 output columns wide), reads the image's
+// {offset, h, w} from the device table, derives the sampling grid in exact integers and
+// streams the tapped source rows into its private shared-memory ring with bulk asynchronous
+// copies (one per row, 16-byte aligned, completion counted on an mbarrier).  While a group
+// of rows is in flight the warp computes on the previous one: per staged row each lane
+// interpolates horizontally for its seven output columns and keeps the previous row's
+// result in registers; whenever both source rows of an output row have passed, it
+// interpolates vertically, applies the normalising multiply-add, converts and stores
+// planar output.  The copy stream runs ahead across task boundaries, so a warp's next task
+// is already arriving while it finishes the current one.  Nothing but the input bytes and
+// the output tensor touches device memory; warps never wait for one another.
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
+#include <atomic>
 #include <cmath>
 
 #include "preba.h"
@@ -22,18 +23,35 @@
 
 namespace preba {
 
-constexpr int kConsumerWarps = 4;
-constexpr int kConsumerThreads = kConsumerWarps * 32;
-constexpr int kThreads = kConsumerThreads + 32;  // + one producer warp
-constexpr uint32_t kTileCols = 2 * kConsumerThreads;  // two output columns per consumer thread
-constexpr uint32_t kMaxSlabRows = 32;                 // one producer lane per output row
-constexpr uint32_t kMaxList = 2 * kMaxSlabRows;       // distinct source rows of a slab
-constexpr int kStages = 4;
-constexpr uint32_t kStageBytes = 6144;
-constexpr uint32_t kMaxRowsPerStage = 8;
-constexpr uint32_t kSpinLimit = 1u << 20;  // bounded waits: give up, report, leave
+#ifndef PREBA_WARPS_PER_CTA
+#define PREBA_WARPS_PER_CTA 4
+#endif
+#ifndef PREBA_CTAS_PER_SM
+#define PREBA_CTAS_PER_SM 4
+#endif
+#ifndef PREBA_SLAB_ROWS
+#define PREBA_SLAB_ROWS 16
+#endif
+#ifndef PREBA_GROUP_BYTES
+#define PREBA_GROUP_BYTES 4608
+#endif
 
-enum TileKind : uint32_t { kEnd = 0, kStream = 1, kGather = 2, kSkip = 3 };
+constexpr int kWarpsPerCta = PREBA_WARPS_PER_CTA;
+constexpr int kThreads = 32 * kWarpsPerCta;
+constexpr int kCtasPerSm = PREBA_CTAS_PER_SM;
+constexpr uint32_t kLaneCols = 7;                  // output columns per lane
+constexpr uint32_t kTaskCols = 32 * kLaneCols;     // 224 output columns per task
+constexpr uint32_t kSlabRows = PREBA_SLAB_ROWS;    // output rows per task (one lane per row)
+constexpr uint32_t kMaxList = 2 * 32;              // distinct source rows of a slab
+constexpr uint32_t kGroups = 2;                    // ring: one group computed, one in flight
+constexpr uint32_t kGroupBytes = PREBA_GROUP_BYTES;
+constexpr uint32_t kGroupRows = 4;                 // rows per group at most
+constexpr uint32_t kMetaBufs = 3;                  // the copy stream is at most two tasks ahead
+constexpr uint32_t kSpinLimit = 1u << 20;          // bounded waits: give up, report, leave
+static_assert(kSlabRows >= 1 && kSlabRows <= 32, "one lane per output row of a slab");
+static_assert(kGroupBytes % 16 == 0, "bulk copies need 16-byte aligned destinations");
+
+enum TaskKind : uint32_t { kEnd = 0, kStream = 1, kGather = 2, kSkip = 3 };
 
 struct Params {
   const uint8_t* pixels;
@@ -41,34 +59,39 @@ struct Params {
   const preba_img_t* table;
   void* out;
   int32_t* status;
+  uint32_t* sched;      // two zeroed words for dynamic task claims, or NULL for static turns
   uint32_t n;
-  uint32_t C;          // crop side
-  uint32_t S;          // resized shorter side
-  uint32_t slab_rows;  // output rows per tile, <= kMaxSlabRows
-  uint32_t slabs;      // slabs per image
-  uint32_t col_blocks; // column blocks per image
-  uint32_t tiles;      // n * slabs * col_blocks
-  float a[3];          // 1 / (255 * std_c)
-  float b[3];          // -mean_c / std_c
+  uint32_t C;           // crop side
+  uint32_t S;           // resized shorter side
+  uint32_t slabs;       // slabs per image
+  uint32_t col_blocks;  // column blocks per image
+  uint32_t tasks;       // n * slabs * col_blocks
+  float a[3];           // 1 / (255 * std_c)
+  float b[3];           // -mean_c / std_c
 };
 
-// What the producer tells the consumers about a tile.
-struct TileMeta {
+// A task as its warp sees it, in the warp's shared memory.
+struct TaskMeta {
   uint32_t kind;
   uint32_t img, k0, rows_out, col0;
-  uint32_t w, rw, left;  // x axis: input width, resized width, crop origin
-  uint32_t xmin;         // first source column staged
-  uint32_t stride;       // bytes between staged rows of a stage
-  uint32_t rows_per_stage;
-  uint32_t n_list;       // distinct source rows of the slab, ascending
-  uint64_t src;          // byte offset of the image in the pixel buffer
-  uint32_t info[kMaxList];    // per listed row: low byte = byte skew of the staged row,
-                              // next byte = output rows completed by this row
-  uint32_t lam[kMaxSlabRows]; // per output row: weight of the lower source row (float bits);
-                              // sign bit set when both taps are the same row
-  uint32_t row[kMaxList];     // per listed row: source row index
-  uint32_t y0[kMaxSlabRows];  // per output row: tap rows (direct path)
-  uint32_t y1[kMaxSlabRows];
+  uint32_t w, h, rw, rh;  // input size, resized size
+  uint32_t xmin;          // first source column staged
+  uint32_t stride;        // bytes between staged rows of a group
+  uint32_t rows_per_group;
+  uint32_t n_list;        // distinct source rows of the slab, ascending
+  uint32_t pad;
+  uint64_t src;           // byte offset of the image in the pixel buffer
+  uint32_t info[kMaxList];  // per listed row: low byte = byte skew of the staged row,
+                            // next byte = output rows completed by this row
+  uint32_t lam[32];         // per output row: weight of the lower source row (float bits);
+                            // sign bit set when both taps are the same row
+  uint32_t row[kMaxList];   // per listed row: source row index
+};
+
+struct __align__(16) WarpShared {
+  uint8_t ring[kGroups][kGroupBytes];
+  TaskMeta meta[kMetaBufs];
+  uint64_t full[kGroups];
 };
 
 // Taps and weight of one crop-window index along one axis: the source coordinate
@@ -162,6 +185,11 @@ __device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uin
       : "memory");
 }
 
+// Orders this thread's earlier shared-memory reads before later asynchronous-copy writes.
+__device__ __forceinline__ void fence_async_shared() {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
 __device__ __forceinline__ uint32_t lds32(uint32_t addr) {
   uint32_t v;
   asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
@@ -176,10 +204,10 @@ __device__ __forceinline__ float byte_biased(uint32_t x) {
   return __uint_as_float(__byte_perm(x, 0x4B000000u, 0x7440 + idx));
 }
 
-// Horizontal interpolation of one staged row at byte offset `off` (pixel x0, then x0+1).
-__device__ __forceinline__ void hlerp_row(uint32_t row_addr, uint32_t off, float lam, float h[3]) {
-  const uint32_t addr = row_addr + (off & ~3u);
-  const uint32_t sh = (off & 3u) * 8u;
+// Horizontal interpolation of one staged row at byte offset x (pixel x0, then x0 + 1).
+__device__ __forceinline__ void hlerp_row(uint32_t row_addr, uint32_t x, float lam, float h[3]) {
+  const uint32_t addr = row_addr + (x & ~3u);
+  const uint32_t sh = x << 3;  // the funnel shift takes it modulo 32
   const uint32_t w0 = lds32(addr), w1 = lds32(addr + 4), w2 = lds32(addr + 8);
   const uint32_t lo = __funnelshift_r(w0, w1, sh);  // R0 G0 B0 R1
   const uint32_t hi = __funnelshift_r(w1, w2, sh);  // G1 B1 .. ..
@@ -205,303 +233,389 @@ struct Pack<__half> {
   static __device__ __forceinline__ __half one(float x) { return __float2half_rn(x); }
 };
 
-// Vertical interpolation, normalisation and store of one output row for two columns.
-template <typename OutT>
-__device__ __forceinline__ void emit_row(OutT* __restrict__ dst, size_t plane, float ly,
-                                         const float hpA[3], const float hcA[3],
-                                         const float hpB[3], const float hcB[3],
-                                         const Params& p, bool pair_ok, bool validA, bool validB) {
-#pragma unroll
-  for (int ch = 0; ch < 3; ++ch) {
-    const float vA = fmaf(ly, hcA[ch] - hpA[ch], hpA[ch]);
-    const float vB = fmaf(ly, hcB[ch] - hpB[ch], hpB[ch]);
-    const float oA = fmaf(vA, p.a[ch], p.b[ch]);
-    const float oB = fmaf(vB, p.a[ch], p.b[ch]);
-    OutT* q = dst + ch * plane;
-    if (pair_ok) {
-      *reinterpret_cast<typename Pack<OutT>::Vec*>(q) = Pack<OutT>::pair(oA, oB);
-    } else {
-      if (validA) q[0] = Pack<OutT>::one(oA);
-      if (validB) q[1] = Pack<OutT>::one(oB);
-    }
-  }
+// Columns of a lane inside a task: three adjacent pairs 64 columns apart, then one single.
+__device__ __forceinline__ uint32_t lane_col(uint32_t lane, uint32_t m) {
+  return m < 6 ? 2 * lane + 64 * (m >> 1) + (m & 1) : 192 + lane;
 }
 
-struct __align__(16) Shared {
-  uint8_t ring[kStages][kStageBytes];
-  TileMeta meta[2];
-  uint64_t full[kStages];
-  uint64_t empty[kStages];
-  uint64_t meta_full[2];
-  uint64_t meta_empty[2];
+// What a lane keeps for the task it computes on.
+struct Lane {
+  uint32_t off[kLaneCols];  // byte offset of the first tap in a staged row (before its skew)
+  float lam[kLaneCols];     // weight of the second tap
+  uint32_t valid;           // bit m: column m exists
+  bool pairs;               // adjacent columns may be stored as one vector
 };
 
-// ---- producer warp ---------------------------------------------------------------------------------
-
-__device__ __forceinline__ void produce(const Params& p, Shared& sm, uint32_t lane) {
-  const uint32_t C = p.C;
-  uint32_t fills = 0;  // stages filled so far by this CTA
-  bool failed = false;
-  for (uint32_t it = 0; !failed; ++it) {
-    const uint32_t mb = it & 1;
-    TileMeta& m = sm.meta[mb];
-    if (it >= 2 && !mbar_wait(smem_addr(&sm.meta_empty[mb]), ((it >> 1) - 1) & 1)) {
-      failed = true;
-      break;
-    }
-    const uint64_t tile = static_cast<uint64_t>(blockIdx.x) + static_cast<uint64_t>(it) * gridDim.x;
-    if (tile >= p.tiles) {
-      if (lane == 0) m.kind = kEnd;
-      __syncwarp();
-      if (lane == 0) mbar_arrive(smem_addr(&sm.meta_full[mb]));
-      break;
-    }
-    const uint32_t per_img = p.slabs * p.col_blocks;
-    const uint32_t img = static_cast<uint32_t>(tile / per_img);
-    const uint32_t rest = static_cast<uint32_t>(tile - static_cast<uint64_t>(img) * per_img);
-    const uint32_t slab = rest / p.col_blocks;
-    const uint32_t cb = rest - slab * p.col_blocks;
-    const preba_img_t e = p.table[img];
-    const bool ok = entry_ok(e, p.pixels_bytes);
-    uint32_t kind = kSkip;
-    uint32_t n_list = 0, rps = 0, stride = 0, xmin = 0, copy_px = 0;
-    if (ok) {
-      uint32_t rh, rw;
-      if (e.h <= e.w) {
-        rh = p.S;
-        rw = static_cast<uint32_t>(static_cast<uint64_t>(p.S) * e.w / e.h);
-      } else {
-        rw = p.S;
-        rh = static_cast<uint32_t>(static_cast<uint64_t>(p.S) * e.h / e.w);
-      }
-      const uint32_t top = (rh - C) / 2, left = (rw - C) / 2;
-      const uint32_t k0 = slab * p.slab_rows;
-      const uint32_t rows_out = min(p.slab_rows, C - k0);
-      const uint32_t col0 = cb * kTileCols;
-      const uint32_t cols = min(kTileCols, C - col0);
-      const Tap tf = axis_tap(e.w, rw, left, col0);
-      const Tap tl = axis_tap(e.w, rw, left, col0 + cols - 1);
-      xmin = tf.i0;
-      copy_px = tl.i1 - xmin + 1;
-      // a consumer reads 12 bytes from the word holding its first tap, which may be the
-      // last staged pixel: leave room for one more pixel and the word overshoot
-      stride = (15 + 3 * copy_px + 3 + 12 + 15) & ~15u;
-      rps = min(kMaxRowsPerStage, kStageBytes / stride);
-      const uint64_t end16 = (e.offset + 3ull * e.h * e.w + 15) & ~15ull;
-      kind = (rps >= 1 && end16 <= p.pixels_bytes) ? kStream : kGather;
-
-      // rows of the slab: taps, then the ascending list of distinct source rows
-      const bool active = lane < rows_out;
-      Tap ty = {0, 0, 0.f};
-      if (active) ty = axis_tap(e.h, rh, top, k0 + lane);
-      const uint32_t y1_prev = __shfl_up_sync(0xffffffffu, ty.i1, 1);
-      const bool new0 = active && (lane == 0 || ty.i0 > y1_prev);
-      const bool new1 = active && ty.i1 != ty.i0 && (lane == 0 || ty.i1 > y1_prev);
-      const uint32_t cnt = (new0 ? 1u : 0u) + (new1 ? 1u : 0u);
-      uint32_t incl = cnt;
+// Vertical interpolation, normalisation and store of one output row (seven columns).
+template <typename OutT>
+__device__ __forceinline__ void emit_row(OutT* __restrict__ img_out, uint32_t idx, uint32_t plane,
+                                         uint32_t lane, float ly, const float (&hp)[kLaneCols][3],
+                                         const float (&hc)[kLaneCols][3], const Params& p,
+                                         const Lane& ln) {
 #pragma unroll
-      for (int d = 1; d < 32; d <<= 1) {
-        const uint32_t v = __shfl_up_sync(0xffffffffu, incl, d);
-        if (lane >= static_cast<uint32_t>(d)) incl += v;
-      }
-      n_list = __shfl_sync(0xffffffffu, incl, 31);
-      const uint32_t excl = incl - cnt;
-      if (new0) m.row[excl] = ty.i0;
-      if (new1) m.row[excl + (new0 ? 1u : 0u)] = ty.i1;
-      m.info[lane] = 0;
-      m.info[lane + 32] = 0;
-      __syncwarp();
-      // the row that completes output row `lane` is the last one listed so far
-      const uint32_t key = active ? incl - 1 : 0x80000000u + lane;
-      const uint32_t peers = __match_any_sync(0xffffffffu, key);
-      if (active && lane == static_cast<uint32_t>(__ffs(peers) - 1))
-        m.info[key] = static_cast<uint32_t>(__popc(peers)) << 8;
-      if (active) {
-        m.lam[lane] = __float_as_uint(ty.lam) | (ty.i1 == ty.i0 ? 0x80000000u : 0u);
-        m.y0[lane] = ty.i0;
-        m.y1[lane] = ty.i1;
-      }
-      __syncwarp();
-      for (uint32_t i = lane; i < n_list; i += 32)
-        m.info[i] |= (3u * (m.row[i] * e.w + xmin)) & 15u;
-      if (lane == 0) {
-        m.img = img;
-        m.k0 = k0;
-        m.rows_out = rows_out;
-        m.col0 = col0;
-        m.w = e.w;
-        m.rw = rw;
-        m.left = left;
-        m.xmin = xmin;
-        m.stride = stride;
-        m.rows_per_stage = rps;
-        m.n_list = n_list;
-        m.src = e.offset;
-      }
-    } else if (lane == 0) {
-      report(p.status, PREBA_ERR_BAD_TABLE);
+  for (int ch = 0; ch < 3; ++ch) {
+    float o[kLaneCols];
+#pragma unroll
+    for (int m = 0; m < static_cast<int>(kLaneCols); ++m) {
+      const float v = fmaf(ly, hc[m][ch] - hp[m][ch], hp[m][ch]);
+      o[m] = fmaf(v, p.a[ch], p.b[ch]);
     }
-    if (lane == 0) m.kind = kind;
-    __syncwarp();
-    if (lane == 0) mbar_arrive(smem_addr(&sm.meta_full[mb]));
-
-    if (kind == kStream) {
-      const uint8_t* img_base = p.pixels + e.offset;
-      const uint32_t pitch = 3 * e.w;
-      for (uint32_t base = 0; base < n_list; base += rps) {
-        const uint32_t stage = fills % kStages;
-        if (fills >= kStages &&
-            !mbar_wait(smem_addr(&sm.empty[stage]), ((fills / kStages) - 1) & 1)) {
-          failed = true;
-          break;
-        }
-        const uint32_t cnt = min(rps, n_list - base);
-        const uint32_t bar = smem_addr(&sm.full[stage]);
-        if (lane < cnt) {
-          const uint8_t* src = img_base + static_cast<size_t>(m.row[base + lane]) * pitch + 3 * xmin;
-          const uintptr_t s = reinterpret_cast<uintptr_t>(src);
-          const uintptr_t s0 = s & ~static_cast<uintptr_t>(15);
-          const uint32_t bytes =
-              static_cast<uint32_t>(((s + 3 * copy_px + 15) & ~static_cast<uintptr_t>(15)) - s0);
-          mbar_arrive_expect_tx(bar, bytes);
-          bulk_copy_g2s(smem_addr(&sm.ring[stage][lane * stride]),
-                        reinterpret_cast<const void*>(s0), bytes, bar);
-        } else {
-          mbar_arrive(bar);
-        }
-        ++fills;
+    OutT* q = img_out + (idx + ch * plane);  // column 2*lane of this row and plane
+#pragma unroll
+    for (int pr = 0; pr < 3; ++pr) {
+      OutT* qq = q + 64 * pr;
+      if (ln.pairs && ((ln.valid >> (2 * pr + 1)) & 1u)) {
+        *reinterpret_cast<typename Pack<OutT>::Vec*>(qq) = Pack<OutT>::pair(o[2 * pr], o[2 * pr + 1]);
+      } else {
+        if ((ln.valid >> (2 * pr)) & 1u) qq[0] = Pack<OutT>::one(o[2 * pr]);
+        if ((ln.valid >> (2 * pr + 1)) & 1u) qq[1] = Pack<OutT>::one(o[2 * pr + 1]);
       }
     }
-  }
-  if (failed) {
-    if (lane == 0) report(p.status, PREBA_ERR_TIMEOUT);
-    // copies already issued may still be landing in this CTA's shared memory: wait for
-    // them (bounded) before the CTA can retire
-    const uint32_t first = fills > kStages ? fills - kStages : 0;
-    for (uint32_t f = first; f < fills; ++f)
-      (void)mbar_wait(smem_addr(&sm.full[f % kStages]), (f / kStages) & 1);
+    if ((ln.valid >> 6) & 1u) q[192 - lane] = Pack<OutT>::one(o[6]);
   }
 }
 
-// ---- consumer warps -----------------------------------------------------------------------------------
+// ---- task preparation: geometry of a slab into the warp's meta buffer --------------------------
+
+struct Issue {          // the copy stream's view of the task it is issuing
+  const uint8_t* base;  // image base + 3 * xmin
+  uint32_t pitch;       // 3 * w
+  uint32_t copy_bytes;  // tapped bytes of a row
+  uint32_t stride;
+  uint32_t rpg;         // rows per group
+  uint32_t n_list;
+  uint32_t buf;         // meta buffer of the task
+};
+
+// Fills `m` for task `task`; returns its kind.  All lanes take part.
+__device__ __forceinline__ uint32_t prepare(const Params& p, uint32_t task, TaskMeta& m,
+                                            uint32_t lane, Issue& is) {
+  const uint32_t C = p.C;
+  const uint32_t per_img = p.slabs * p.col_blocks;
+  const uint32_t img = task / per_img;
+  const uint32_t rest = task - img * per_img;
+  const uint32_t slab = rest / p.col_blocks;
+  const uint32_t cb = rest - slab * p.col_blocks;
+  const preba_img_t e = p.table[img];
+  uint32_t kind = kSkip;
+  if (entry_ok(e, p.pixels_bytes)) {
+    uint32_t rh, rw;
+    if (e.h <= e.w) {
+      rh = p.S;
+      rw = static_cast<uint32_t>(static_cast<uint64_t>(p.S) * e.w / e.h);
+    } else {
+      rw = p.S;
+      rh = static_cast<uint32_t>(static_cast<uint64_t>(p.S) * e.h / e.w);
+    }
+    const uint32_t top = (rh - C) / 2, left = (rw - C) / 2;
+    const uint32_t k0 = slab * kSlabRows;
+    const uint32_t rows_out = min(kSlabRows, C - k0);
+    const uint32_t col0 = cb * kTaskCols;
+    const uint32_t cols = min(kTaskCols, C - col0);
+    const Tap tf = axis_tap(e.w, rw, left, col0);
+    const Tap tl = axis_tap(e.w, rw, left, col0 + cols - 1);
+    const uint32_t xmin = tf.i0;
+    const uint32_t copy_px = tl.i1 - xmin + 1;
+    // a lane reads 12 bytes from the word holding its first tap, which may be the last
+    // staged pixel: leave room for one more pixel and the word overshoot
+    const uint32_t stride = (15 + 3 * copy_px + 3 + 12 + 15) & ~15u;
+    const uint32_t rpg = min(kGroupRows, kGroupBytes / stride);
+    const uint64_t end16 = (e.offset + 3ull * e.h * e.w + 15) & ~15ull;
+    kind = (rpg >= 1 && end16 <= p.pixels_bytes) ? kStream : kGather;
+
+    // rows of the slab: taps, then the ascending list of distinct source rows
+    const bool active = lane < rows_out;
+    Tap ty = {0, 0, 0.f};
+    if (active) ty = axis_tap(e.h, rh, top, k0 + lane);
+    const uint32_t y1_prev = __shfl_up_sync(0xffffffffu, ty.i1, 1);
+    const bool new0 = active && (lane == 0 || ty.i0 > y1_prev);
+    const bool new1 = active && ty.i1 != ty.i0 && (lane == 0 || ty.i1 > y1_prev);
+    const uint32_t cnt = (new0 ? 1u : 0u) + (new1 ? 1u : 0u);
+    uint32_t incl = cnt;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const uint32_t v = __shfl_up_sync(0xffffffffu, incl, d);
+      if (lane >= static_cast<uint32_t>(d)) incl += v;
+    }
+    const uint32_t n_list = __shfl_sync(0xffffffffu, incl, 31);
+    const uint32_t excl = incl - cnt;
+    if (new0) m.row[excl] = ty.i0;
+    if (new1) m.row[excl + (new0 ? 1u : 0u)] = ty.i1;
+    m.info[lane] = 0;
+    m.info[lane + 32] = 0;
+    __syncwarp();
+    // the row that completes output row `lane` is the last one listed so far
+    const uint32_t key = active ? incl - 1 : 0x80000000u + lane;
+    const uint32_t peers = __match_any_sync(0xffffffffu, key);
+    if (active && lane == static_cast<uint32_t>(__ffs(peers) - 1))
+      m.info[key] = static_cast<uint32_t>(__popc(peers)) << 8;
+    if (active) m.lam[lane] = __float_as_uint(ty.lam) | (ty.i1 == ty.i0 ? 0x80000000u : 0u);
+    __syncwarp();
+    for (uint32_t i = lane; i < n_list; i += 32)
+      m.info[i] |= (3u * (m.row[i] * e.w + xmin)) & 15u;
+    if (lane == 0) {
+      m.img = img;
+      m.k0 = k0;
+      m.rows_out = rows_out;
+      m.col0 = col0;
+      m.w = e.w;
+      m.h = e.h;
+      m.rw = rw;
+      m.rh = rh;
+      m.xmin = xmin;
+      m.stride = stride;
+      m.rows_per_group = rpg;
+      m.n_list = n_list;
+      m.src = e.offset;
+    }
+    is.base = p.pixels + e.offset + 3 * xmin;
+    is.pitch = 3 * e.w;
+    is.copy_bytes = 3 * copy_px;
+    is.stride = stride;
+    is.rpg = rpg;
+    is.n_list = kind == kStream ? n_list : 0;
+  } else {
+    if (lane == 0) report(p.status, PREBA_ERR_BAD_TABLE);
+    is.n_list = 0;
+  }
+  if (lane == 0) m.kind = kind;
+  __syncwarp();
+  return kind;
+}
+
+// ---- the warp program ---------------------------------------------------------------------------------
 
 template <typename OutT>
-__device__ __forceinline__ void consume(const Params& p, Shared& sm, uint32_t tid, uint32_t lane) {
+__device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint32_t lane,
+                                          uint32_t gwarp, uint32_t nwarps) {
   const uint32_t C = p.C;
-  const size_t plane = static_cast<size_t>(C) * C;
-  const bool even = (C & 1u) == 0;
-  uint32_t drains = 0;  // stages consumed so far by this CTA
-  for (uint32_t it = 0;; ++it) {
-    const uint32_t mb = it & 1;
-    if (!mbar_wait(smem_addr(&sm.meta_full[mb]), (it >> 1) & 1)) {
-      if (lane == 0) report(p.status, PREBA_ERR_TIMEOUT);
-      return;
-    }
-    const TileMeta& m = sm.meta[mb];
-    const uint32_t kind = m.kind;
-    if (kind == kEnd) return;
-    if (kind != kSkip) {
-      const uint32_t w = m.w, rw = m.rw, left = m.left;
-      const uint32_t rows_out = m.rows_out;
-      const uint32_t jA = m.col0 + 2 * tid;
-      const bool validA = jA < C, validB = jA + 1 < C;
-      const bool pair_ok = even && validB;
-      const Tap tA = axis_tap(w, rw, left, validA ? jA : m.col0);
-      const Tap tB = axis_tap(w, rw, left, validB ? jA + 1 : (validA ? jA : m.col0));
-      OutT* dst = static_cast<OutT*>(p.out) +
-                  (static_cast<size_t>(m.img) * 3 * C + m.k0) * C + jA;
-      if (kind == kStream) {
-        const uint32_t n_list = m.n_list, rps = m.rows_per_stage, stride = m.stride;
-        const uint32_t offA = 3 * (tA.i0 - m.xmin), offB = 3 * (tB.i0 - m.xmin);
-        float hpA[3] = {0.f, 0.f, 0.f}, hcA[3] = {0.f, 0.f, 0.f};
-        float hpB[3] = {0.f, 0.f, 0.f}, hcB[3] = {0.f, 0.f, 0.f};
-        uint32_t t_out = 0;
-        for (uint32_t base = 0; base < n_list; base += rps) {
-          const uint32_t stage = drains % kStages;
-          if (!mbar_wait(smem_addr(&sm.full[stage]), (drains / kStages) & 1)) {
-            if (lane == 0) report(p.status, PREBA_ERR_TIMEOUT);
-            return;
+  const uint32_t plane = C * C;
+
+  // task claims: a warp's first task is its own index; later ones come from the shared
+  // counter (dynamic) or every nwarps-th task (static)
+  uint32_t next_task = gwarp;
+  uint32_t turn = 0;
+
+  // copy stream
+  Issue is;
+  is.n_list = 0;
+  is.rpg = 1;
+  is.buf = 0;
+  uint32_t is_row = 0;       // next listed row of the issuing task to copy
+  uint32_t prepared = 0;     // tasks prepared (meta buffers written)
+  uint32_t issued = 0;       // groups issued
+  bool ended = false;        // no task left to prepare
+
+  // compute stream
+  uint32_t finished = 0;     // tasks computed
+  uint32_t consumed = 0;     // groups computed
+  bool need_task = true;
+  bool failed = false;
+  Lane ln;
+  float hA[kLaneCols][3], hB[kLaneCols][3];
+  uint32_t par = 0;          // which of hA/hB holds the latest row
+  uint32_t c_row = 0, c_nlist = 0, c_rpg = 1, c_stride = 0, t_out = 0, out_idx = 0;
+  uint32_t c_kind = kEnd;
+  const TaskMeta* cm = &ws.meta[0];
+  OutT* img_out = static_cast<OutT*>(p.out);
+#pragma unroll
+  for (int m = 0; m < static_cast<int>(kLaneCols); ++m) {
+    ln.off[m] = 0;
+    ln.lam[m] = 0.f;
+#pragma unroll
+    for (int ch = 0; ch < 3; ++ch) hA[m][ch] = hB[m][ch] = 0.f;
+  }
+  ln.valid = 0;
+  ln.pairs = false;
+
+  for (;;) {
+    // -- advance the copy stream: at most kGroups groups and kMetaBufs - 1 tasks ahead -------
+    for (;;) {
+      if (is_row < is.n_list) {
+        if (issued >= consumed + kGroups) break;
+        const uint32_t slot = issued % kGroups;
+        const uint32_t cnt = min(is.rpg, is.n_list - is_row);
+        const uint32_t bar = smem_addr(&ws.full[slot]);
+        if (lane < kGroupRows) {
+          if (lane < cnt) {
+            const uint8_t* src = is.base +
+                static_cast<size_t>(ws.meta[is.buf].row[is_row + lane]) * is.pitch;
+            const uintptr_t s = reinterpret_cast<uintptr_t>(src);
+            const uintptr_t s0 = s & ~static_cast<uintptr_t>(15);
+            const uint32_t bytes = static_cast<uint32_t>(
+                ((s + is.copy_bytes + 15) & ~static_cast<uintptr_t>(15)) - s0);
+            fence_async_shared();
+            mbar_arrive_expect_tx(bar, bytes);
+            bulk_copy_g2s(smem_addr(&ws.ring[slot][lane * is.stride]),
+                          reinterpret_cast<const void*>(s0), bytes, bar);
+          } else {
+            mbar_arrive(bar);
           }
-          const uint32_t cnt = min(rps, n_list - base);
-          uint32_t row_addr = smem_addr(&sm.ring[stage][0]);
-          for (uint32_t r = 0; r < cnt; ++r, row_addr += stride) {
-            const uint32_t info = m.info[base + r];
-            const uint32_t skew = info & 0xffu;
+        }
+        is_row += cnt;
+        ++issued;
+      } else {
+        if (ended || prepared - finished >= kMetaBufs) break;
+        uint32_t task = next_task;
+        if (p.sched) {
+          uint32_t got = 0;
+          if (lane == 0) got = atomicAdd(&p.sched[0], 1u);
+          next_task = nwarps + __shfl_sync(0xffffffffu, got, 0);
+        } else {
+          ++turn;
+          const uint64_t t = static_cast<uint64_t>(gwarp) + static_cast<uint64_t>(turn) * nwarps;
+          next_task = t < p.tasks ? static_cast<uint32_t>(t) : p.tasks;
+        }
+        const uint32_t buf = prepared % kMetaBufs;
+        if (task >= p.tasks) {
+          if (lane == 0) ws.meta[buf].kind = kEnd;
+          __syncwarp();
+          ended = true;
+          is.n_list = 0;
+        } else {
+          (void)prepare(p, task, ws.meta[buf], lane, is);
+        }
+        is.buf = buf;
+        is_row = 0;
+        ++prepared;
+      }
+    }
+
+    // -- compute stream: start the next task, or one group of the current one ------------------
+    if (need_task) {
+      if (finished == prepared) break;  // only after the end marker was consumed
+      cm = &ws.meta[finished % kMetaBufs];
+      c_kind = cm->kind;
+      if (c_kind == kEnd) break;
+      if (c_kind == kSkip) {
+        ++finished;
+        continue;
+      }
+      const uint32_t w = cm->w, rw = cm->rw, left = (rw - C) / 2, col0 = cm->col0;
+      const uint32_t xmin = cm->xmin;
+      ln.valid = 0;
+#pragma unroll
+      for (int m = 0; m < static_cast<int>(kLaneCols); ++m) {
+        const uint32_t j = col0 + lane_col(lane, m);
+        if (j < C) ln.valid |= 1u << m;
+        const Tap t = axis_tap(w, rw, left, j < C ? j : C - 1);
+        ln.off[m] = 3 * (t.i0 - xmin);
+        ln.lam[m] = t.lam;
+      }
+      ln.pairs = (C & 1u) == 0;
+      img_out = static_cast<OutT*>(p.out) + static_cast<size_t>(cm->img) * 3 * plane;
+      out_idx = cm->k0 * C + col0 + 2 * lane;
+      c_nlist = cm->n_list;
+      c_rpg = cm->rows_per_group;
+      c_stride = cm->stride;
+      c_row = 0;
+      t_out = 0;
+      need_task = false;
+      if (c_kind == kGather) {
+        // direct path: taps straight from global memory (footprint too wide for the ring)
+        const uint8_t* __restrict__ src = p.pixels + cm->src;
+        const size_t pitch = 3 * static_cast<size_t>(w);
+        const uint32_t h = cm->h, rh = cm->rh, top = (rh - C) / 2;
+        for (uint32_t t = 0; t < cm->rows_out; ++t, out_idx += C) {
+          const Tap ty = axis_tap(h, rh, top, cm->k0 + t);
+          const uint8_t* r0 = src + ty.i0 * pitch + 3 * xmin;
+          const uint8_t* r1 = src + ty.i1 * pitch + 3 * xmin;
+#pragma unroll
+          for (int m = 0; m < static_cast<int>(kLaneCols); ++m) {
 #pragma unroll
             for (int ch = 0; ch < 3; ++ch) {
-              hpA[ch] = hcA[ch];
-              hpB[ch] = hcB[ch];
-            }
-            hlerp_row(row_addr, offA + skew, tA.lam, hcA);
-            hlerp_row(row_addr, offB + skew, tB.lam, hcB);
-            for (uint32_t e = info >> 8; e > 0; --e, ++t_out) {
-              const uint32_t lbits = m.lam[t_out];
-              float ly = __uint_as_float(lbits);
-              if (lbits >> 31) {  // both taps are this row
-#pragma unroll
-                for (int ch = 0; ch < 3; ++ch) {
-                  hpA[ch] = hcA[ch];
-                  hpB[ch] = hcB[ch];
-                }
-                ly = 0.f;
-              }
-              emit_row<OutT>(dst, plane, ly, hpA, hcA, hpB, hcB, p, pair_ok, validA, validB);
-              dst += C;
+              // the right neighbour is read only where it carries weight (it exists then)
+              const uint32_t nb = ln.lam[m] > 0.f ? 3u : 0u;
+              float a = __ldg(r0 + ln.off[m] + ch), b = __ldg(r0 + ln.off[m] + nb + ch);
+              hA[m][ch] = fmaf(ln.lam[m], b - a, a);
+              a = __ldg(r1 + ln.off[m] + ch), b = __ldg(r1 + ln.off[m] + nb + ch);
+              hB[m][ch] = fmaf(ln.lam[m], b - a, a);
             }
           }
-          __syncwarp();
-          if (lane == 0) mbar_arrive(smem_addr(&sm.empty[stage]));
-          ++drains;
+          emit_row<OutT>(img_out, out_idx, plane, lane, ty.lam, hA, hB, p, ln);
         }
-      } else {  // direct path: taps straight from global memory
-        const uint8_t* __restrict__ src = p.pixels + m.src;
-        const size_t pitch = 3 * static_cast<size_t>(w);
-        const uint32_t cA0 = 3 * tA.i0, cA1 = 3 * tA.i1, cB0 = 3 * tB.i0, cB1 = 3 * tB.i1;
-        for (uint32_t t = 0; t < rows_out; ++t, dst += C) {
-          const uint8_t* r0 = src + m.y0[t] * pitch;
-          const uint8_t* r1 = src + m.y1[t] * pitch;
-          const float ly = __uint_as_float(m.lam[t] & 0x7fffffffu);
-          float h0A[3], h1A[3], h0B[3], h1B[3];
+        ++finished;
+        need_task = true;
+      }
+      continue;
+    }
+
+    // one group of staged rows
+    {
+      const uint32_t slot = consumed % kGroups;
+      if (!mbar_wait(smem_addr(&ws.full[slot]), (consumed / kGroups) & 1)) {
+        failed = true;
+        break;
+      }
+      const uint32_t cnt = min(c_rpg, c_nlist - c_row);
+      uint32_t row_addr = smem_addr(&ws.ring[slot][0]);
+      for (uint32_t r = 0; r < cnt; ++r, row_addr += c_stride) {
+        const uint32_t info = cm->info[c_row + r];
+        const uint32_t skew = info & 0xffu;
+        uint32_t e = info >> 8;
+        if (par == 0) {
 #pragma unroll
-          for (int ch = 0; ch < 3; ++ch) {
-            float a = __ldg(r0 + cA0 + ch), b = __ldg(r0 + cA1 + ch);
-            h0A[ch] = fmaf(tA.lam, b - a, a);
-            a = __ldg(r1 + cA0 + ch), b = __ldg(r1 + cA1 + ch);
-            h1A[ch] = fmaf(tA.lam, b - a, a);
-            a = __ldg(r0 + cB0 + ch), b = __ldg(r0 + cB1 + ch);
-            h0B[ch] = fmaf(tB.lam, b - a, a);
-            a = __ldg(r1 + cB0 + ch), b = __ldg(r1 + cB1 + ch);
-            h1B[ch] = fmaf(tB.lam, b - a, a);
+          for (int m = 0; m < static_cast<int>(kLaneCols); ++m)
+            hlerp_row(row_addr, ln.off[m] + skew, ln.lam[m], hA[m]);
+          for (; e > 0; --e, ++t_out, out_idx += C) {
+            const uint32_t lbits = cm->lam[t_out];
+            if (lbits >> 31)  // both taps are this row
+              emit_row<OutT>(img_out, out_idx, plane, lane, 0.f, hA, hA, p, ln);
+            else
+              emit_row<OutT>(img_out, out_idx, plane, lane, __uint_as_float(lbits), hB, hA, p, ln);
           }
-          emit_row<OutT>(dst, plane, ly, h0A, h1A, h0B, h1B, p, pair_ok, validA, validB);
+        } else {
+#pragma unroll
+          for (int m = 0; m < static_cast<int>(kLaneCols); ++m)
+            hlerp_row(row_addr, ln.off[m] + skew, ln.lam[m], hB[m]);
+          for (; e > 0; --e, ++t_out, out_idx += C) {
+            const uint32_t lbits = cm->lam[t_out];
+            if (lbits >> 31)
+              emit_row<OutT>(img_out, out_idx, plane, lane, 0.f, hB, hB, p, ln);
+            else
+              emit_row<OutT>(img_out, out_idx, plane, lane, __uint_as_float(lbits), hA, hB, p, ln);
+          }
         }
+        par ^= 1u;
+      }
+      c_row += cnt;
+      ++consumed;
+      __syncwarp();  // every lane is done with the slot before the stream refills it
+      if (c_row >= c_nlist) {
+        ++finished;
+        need_task = true;
       }
     }
-    __syncwarp();
-    if (lane == 0) mbar_arrive(smem_addr(&sm.meta_empty[mb]));
+  }
+
+  if (failed) {
+    if (lane == 0) report(p.status, PREBA_ERR_TIMEOUT);
+    // copies already issued may still be landing in this warp's ring: wait for them
+    // (bounded) before the CTA can retire
+    for (uint32_t q = consumed; q < issued; ++q)
+      (void)mbar_wait(smem_addr(&ws.full[q % kGroups]), (q / kGroups) & 1);
+  }
+  // the last warp out leaves the claim counters at zero for the next launch
+  if (p.sched && lane == 0) {
+    __threadfence();
+    if (atomicAdd(&p.sched[1], 1u) == nwarps - 1) {
+      p.sched[0] = 0;
+      p.sched[1] = 0;
+    }
   }
 }
 
 template <typename OutT>
-__global__ void __launch_bounds__(kThreads) preba_fused_kernel(const Params p) {
-  __shared__ Shared sm;
-  const uint32_t tid = threadIdx.x, lane = tid & 31;
-  if (tid == 0) {
-    for (int s = 0; s < kStages; ++s) {
-      mbar_init(smem_addr(&sm.full[s]), 32);               // every producer lane arrives
-      mbar_init(smem_addr(&sm.empty[s]), kConsumerWarps);  // one arrival per consumer warp
-    }
-    for (int b = 0; b < 2; ++b) {
-      mbar_init(smem_addr(&sm.meta_full[b]), 1);
-      mbar_init(smem_addr(&sm.meta_empty[b]), kConsumerWarps);
-    }
+__global__ void __launch_bounds__(kThreads, kCtasPerSm) preba_fused_kernel(const Params p) {
+  __shared__ WarpShared sm[kWarpsPerCta];
+  const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  WarpShared& ws = sm[warp];
+  if (lane == 0) {
+    for (uint32_t g = 0; g < kGroups; ++g) mbar_init(smem_addr(&ws.full[g]), kGroupRows);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  __syncthreads();
-  if (tid >= kConsumerThreads)
-    produce(p, sm, lane);
-  else
-    consume<OutT>(p, sm, tid, lane);
+  __syncwarp();
+  warp_main<OutT>(p, ws, lane, blockIdx.x * kWarpsPerCta + warp, gridDim.x * kWarpsPerCta);
 }
 
 thread_local int g_last_cuda_error = 0;
@@ -523,9 +637,9 @@ int check_args(const uint8_t* pixels, uint64_t pixels_bytes, const void* table, 
                         (out_dtype == PREBA_F16 ? 2u : 4u);
   if (out_bytes < need) return PREBA_ERR_BUFFER_TOO_SMALL;
   if (pixels_bytes == 0) return PREBA_ERR_BUFFER_TOO_SMALL;
-  const uint64_t tiles = static_cast<uint64_t>(n) * ((out_size + 7) / 8) *
-                         ((out_size + kTileCols - 1) / kTileCols);
-  if (tiles > 0x7fffffffull) return PREBA_ERR_INVALID_ARG;
+  const uint64_t tasks = static_cast<uint64_t>(n) * ((out_size + kSlabRows - 1) / kSlabRows) *
+                         ((out_size + kTaskCols - 1) / kTaskCols);
+  if (tasks > 0x7fffffffull) return PREBA_ERR_INVALID_ARG;
   return PREBA_OK;
 }
 
@@ -540,27 +654,40 @@ int check_table(const preba_img_t* t, uint32_t n, uint64_t pixels_bytes) {
 }
 
 // Resident CTAs of the fused kernel on the current device (grid of a persistent launch).
+// The answer depends on the device and the kernel only; it is computed once per device and
+// output type and kept (a benign race: concurrent first calls store the same value).
 int resident_ctas(int out_dtype, cudaError_t* err) {
-  int dev = 0, sms = 0, per_sm = 0;
+  constexpr int kMaxDevices = 64;
+  static std::atomic<int> cache[2][kMaxDevices];
+  int dev = 0;
   *err = cudaGetDevice(&dev);
   if (*err != cudaSuccess) return 0;
+  const int kind = out_dtype == PREBA_F16 ? 1 : 0;
+  if (dev >= 0 && dev < kMaxDevices) {
+    const int known = cache[kind][dev].load(std::memory_order_relaxed);
+    if (known > 0) return known;
+  }
+  int sms = 0, per_sm = 0;
   *err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   if (*err != cudaSuccess) return 0;
-  if (out_dtype == PREBA_F16)
+  if (kind == 1)
     *err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, preba_fused_kernel<__half>,
                                                          kThreads, 0);
   else
     *err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, preba_fused_kernel<float>,
                                                          kThreads, 0);
   if (*err != cudaSuccess) return 0;
-  return sms * (per_sm > 0 ? per_sm : 1);
+  const int resident = sms * (per_sm > 0 ? per_sm : 1);
+  if (dev >= 0 && dev < kMaxDevices) cache[kind][dev].store(resident, std::memory_order_relaxed);
+  return resident;
 }
 
 int launch(const Params& p, int out_dtype, cudaStream_t stream) {
   cudaError_t err = cudaSuccess;
   const int resident = resident_ctas(out_dtype, &err);
   if (err == cudaSuccess) {
-    const uint32_t blocks = p.tiles < static_cast<uint32_t>(resident) ? p.tiles : resident;
+    const uint32_t want = (p.tasks + kWarpsPerCta - 1) / kWarpsPerCta;
+    const uint32_t blocks = want < static_cast<uint32_t>(resident) ? want : resident;
     if (out_dtype == PREBA_F16)
       preba_fused_kernel<__half><<<blocks, kThreads, 0, stream>>>(p);
     else
@@ -586,10 +713,10 @@ Params make_params(const uint8_t* pixels, uint64_t pixels_bytes, const preba_img
   p.n = n;
   p.C = out_size;
   p.S = resize_short;
-  p.slab_rows = 16;
-  p.slabs = (out_size + p.slab_rows - 1) / p.slab_rows;
-  p.col_blocks = (out_size + kTileCols - 1) / kTileCols;
-  p.tiles = static_cast<uint32_t>(static_cast<uint64_t>(n) * p.slabs * p.col_blocks);
+  p.sched = nullptr;
+  p.slabs = (out_size + kSlabRows - 1) / kSlabRows;
+  p.col_blocks = (out_size + kTaskCols - 1) / kTaskCols;
+  p.tasks = static_cast<uint32_t>(static_cast<uint64_t>(n) * p.slabs * p.col_blocks);
   for (int c = 0; c < 3; ++c) {
     const double sd = static_cast<double>(std[c]);
     p.a[c] = static_cast<float>(1.0 / (255.0 * sd));
