@@ -96,34 +96,69 @@ struct __align__(16) WarpShared {
 
 // Taps and weight of one crop-window index along one axis: the source coordinate
 // ((origin + j) + 1/2) * in / r - 1/2, clamped to [0, in - 1], as num / den with
-// num = (2X + 1) * in - r and den = 2r.
+// num = (2X + 1) * in - r and den = 2r.  i0 = floor(num / den) and the remainder are exact
+// integers; the weight is the remainder over den in fp32.
 struct Tap {
   uint32_t i0;
   uint32_t i1;
   float lam;
 };
 
-__device__ __forceinline__ Tap axis_tap(uint32_t in, uint32_t r, uint32_t origin, uint32_t j) {
-  const uint64_t X = static_cast<uint64_t>(origin) + j;
-  const uint64_t den = 2ull * r;
-  const uint64_t pos = (2 * X + 1) * in;  // < 2^46
-  uint64_t num = pos > r ? pos - r : 0;
-  const uint64_t hi = static_cast<uint64_t>(in - 1) * den;
-  num = num < hi ? num : hi;
-  uint64_t q, rem;
-  if ((num | den) >> 32) {
-    q = num / den;
-    rem = num - q * den;
-  } else {
-    const uint32_t n32 = static_cast<uint32_t>(num), d32 = static_cast<uint32_t>(den);
-    const uint32_t q32 = n32 / d32;
-    q = q32;
-    rem = n32 - q32 * d32;
-  }
+struct Axis {
+  uint32_t in;      // source length
+  uint32_t r;       // resized length
+  uint32_t origin;  // crop origin on the resized axis
+  uint32_t den;     // 2r
+  uint32_t hi;      // (in - 1) * den when it fits 32 bits
+  float rden;       // 1 / den
+  bool small;       // every numerator fits 32 bits and den is exact in fp32
+};
+
+__device__ __forceinline__ Axis make_axis(uint32_t in, uint32_t r, uint32_t origin, uint32_t c) {
+  Axis a;
+  a.in = in;
+  a.r = r;
+  a.origin = origin;
+  a.den = 2 * r;  // r <= 2^29
+  const uint64_t top = (2ull * (origin + c) + 1) * in;  // above every numerator of the crop
+  a.small = top < (1ull << 32) && a.den < (1u << 24);
+  // the clamp at the far end: (in - 1) * den, or "never" when that exceeds every numerator
+  const uint64_t hi = static_cast<uint64_t>(in - 1) * a.den;
+  a.hi = hi < (1ull << 32) ? static_cast<uint32_t>(hi) : 0xffffffffu;
+  a.rden = 1.0f / static_cast<float>(a.den);
+  return a;
+}
+
+__device__ __forceinline__ Tap axis_tap(const Axis& a, uint32_t j) {
   Tap t;
-  t.i0 = static_cast<uint32_t>(q);
-  t.i1 = t.i0 + 1 < in ? t.i0 + 1 : in - 1;
-  t.lam = static_cast<float>(rem) / static_cast<float>(den);
+  if (a.small) {
+    // quotient from an fp32 estimate (relative error < 2^-21, so off by at most one),
+    // made exact by the integer remainder
+    const uint32_t pos = (2 * (a.origin + j) + 1) * a.in;
+    uint32_t num = pos > a.r ? pos - a.r : 0;
+    num = min(num, a.hi);
+    uint32_t q = __float2uint_rz(__uint2float_rz(num) * a.rden);
+    int32_t rem = static_cast<int32_t>(num - q * a.den);
+    if (rem < 0) {
+      --q;
+      rem += static_cast<int32_t>(a.den);
+    } else if (rem >= static_cast<int32_t>(a.den)) {
+      ++q;
+      rem -= static_cast<int32_t>(a.den);
+    }
+    t.i0 = q;
+    t.lam = static_cast<float>(rem) * a.rden;
+  } else {
+    const uint64_t den = 2ull * a.r;
+    const uint64_t pos = (2 * (static_cast<uint64_t>(a.origin) + j) + 1) * a.in;  // < 2^46
+    uint64_t num = pos > a.r ? pos - a.r : 0;
+    const uint64_t hi = static_cast<uint64_t>(a.in - 1) * den;
+    num = num < hi ? num : hi;
+    const uint64_t q = num / den;
+    t.i0 = static_cast<uint32_t>(q);
+    t.lam = static_cast<float>(num - q * den) / static_cast<float>(den);
+  }
+  t.i1 = t.i0 + 1 < a.in ? t.i0 + 1 : a.in - 1;
   return t;
 }
 
@@ -204,9 +239,10 @@ __device__ __forceinline__ float byte_biased(uint32_t x) {
   return __uint_as_float(__byte_perm(x, 0x4B000000u, 0x7440 + idx));
 }
 
-// Horizontal interpolation of one staged row at byte offset x (pixel x0, then x0 + 1).
-__device__ __forceinline__ void hlerp_row(uint32_t row_addr, uint32_t x, float lam, float h[3]) {
-  const uint32_t addr = row_addr + (x & ~3u);
+// Horizontal interpolation at shared-memory byte address x (pixel x0, then x0 + 1); x is
+// unaligned: three aligned words are read and shifted.
+__device__ __forceinline__ void hlerp_row(uint32_t x, float lam, float h[3]) {
+  const uint32_t addr = x & ~3u;
   const uint32_t sh = x << 3;  // the funnel shift takes it modulo 32
   const uint32_t w0 = lds32(addr), w1 = lds32(addr + 4), w2 = lds32(addr + 8);
   const uint32_t lo = __funnelshift_r(w0, w1, sh);  // R0 G0 B0 R1
@@ -243,35 +279,37 @@ struct Lane {
   uint32_t off[kLaneCols];  // byte offset of the first tap in a staged row (before its skew)
   float lam[kLaneCols];     // weight of the second tap
   uint32_t valid;           // bit m: column m exists
-  bool pairs;               // adjacent columns may be stored as one vector
 };
 
 // Vertical interpolation, normalisation and store of one output row (seven columns).
-template <typename OutT>
-__device__ __forceinline__ void emit_row(OutT* __restrict__ img_out, uint32_t idx, uint32_t plane,
-                                         uint32_t lane, float ly, const float (&hp)[kLaneCols][3],
-                                         const float (&hc)[kLaneCols][3], const Params& p,
-                                         const Lane& ln) {
+// q points at this row's column 2 * lane in plane 0.  FULL: every column of every lane
+// exists and rows start on even element indices, so pairs go out as one vector each.
+template <typename OutT, bool FULL>
+__device__ __forceinline__ void emit_row(OutT* __restrict__ q, uint32_t plane, uint32_t lane,
+                                         float ly, const float (&hp)[kLaneCols][3],
+                                         const float (&hc)[kLaneCols][3], const float (&na)[3],
+                                         const float (&nb)[3], uint32_t valid) {
 #pragma unroll
-  for (int ch = 0; ch < 3; ++ch) {
+  for (int ch = 0; ch < 3; ++ch, q += plane) {
     float o[kLaneCols];
 #pragma unroll
     for (int m = 0; m < static_cast<int>(kLaneCols); ++m) {
       const float v = fmaf(ly, hc[m][ch] - hp[m][ch], hp[m][ch]);
-      o[m] = fmaf(v, p.a[ch], p.b[ch]);
+      o[m] = fmaf(v, na[ch], nb[ch]);
     }
-    OutT* q = img_out + (idx + ch * plane);  // column 2*lane of this row and plane
+    OutT* single = q + 192 - lane;  // column 192 + lane
+    if (FULL) {
 #pragma unroll
-    for (int pr = 0; pr < 3; ++pr) {
-      OutT* qq = q + 64 * pr;
-      if (ln.pairs && ((ln.valid >> (2 * pr + 1)) & 1u)) {
-        *reinterpret_cast<typename Pack<OutT>::Vec*>(qq) = Pack<OutT>::pair(o[2 * pr], o[2 * pr + 1]);
-      } else {
-        if ((ln.valid >> (2 * pr)) & 1u) qq[0] = Pack<OutT>::one(o[2 * pr]);
-        if ((ln.valid >> (2 * pr + 1)) & 1u) qq[1] = Pack<OutT>::one(o[2 * pr + 1]);
-      }
+      for (int pr = 0; pr < 3; ++pr)
+        *reinterpret_cast<typename Pack<OutT>::Vec*>(q + 64 * pr) =
+            Pack<OutT>::pair(o[2 * pr], o[2 * pr + 1]);
+      *single = Pack<OutT>::one(o[6]);
+    } else {
+#pragma unroll
+      for (int m = 0; m < 6; ++m)
+        if ((valid >> m) & 1u) q[64 * (m >> 1) + (m & 1)] = Pack<OutT>::one(o[m]);
+      if ((valid >> 6) & 1u) *single = Pack<OutT>::one(o[6]);
     }
-    if ((ln.valid >> 6) & 1u) q[192 - lane] = Pack<OutT>::one(o[6]);
   }
 }
 
@@ -312,8 +350,9 @@ __device__ __forceinline__ uint32_t prepare(const Params& p, uint32_t task, Task
     const uint32_t rows_out = min(kSlabRows, C - k0);
     const uint32_t col0 = cb * kTaskCols;
     const uint32_t cols = min(kTaskCols, C - col0);
-    const Tap tf = axis_tap(e.w, rw, left, col0);
-    const Tap tl = axis_tap(e.w, rw, left, col0 + cols - 1);
+    const Axis ax = make_axis(e.w, rw, left, C);
+    const Tap tf = axis_tap(ax, col0);
+    const Tap tl = axis_tap(ax, col0 + cols - 1);
     const uint32_t xmin = tf.i0;
     const uint32_t copy_px = tl.i1 - xmin + 1;
     // a lane reads 12 bytes from the word holding its first tap, which may be the last
@@ -325,8 +364,9 @@ __device__ __forceinline__ uint32_t prepare(const Params& p, uint32_t task, Task
 
     // rows of the slab: taps, then the ascending list of distinct source rows
     const bool active = lane < rows_out;
+    const Axis ay = make_axis(e.h, rh, top, C);
     Tap ty = {0, 0, 0.f};
-    if (active) ty = axis_tap(e.h, rh, top, k0 + lane);
+    if (active) ty = axis_tap(ay, k0 + lane);
     const uint32_t y1_prev = __shfl_up_sync(0xffffffffu, ty.i1, 1);
     const bool new0 = active && (lane == 0 || ty.i0 > y1_prev);
     const bool new1 = active && ty.i1 != ty.i0 && (lane == 0 || ty.i1 > y1_prev);
@@ -390,6 +430,8 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
                                           uint32_t gwarp, uint32_t nwarps) {
   const uint32_t C = p.C;
   const uint32_t plane = C * C;
+  const float na[3] = {p.a[0], p.a[1], p.a[2]};
+  const float nb[3] = {p.b[0], p.b[1], p.b[2]};
 
   // task claims: a warp's first task is its own index; later ones come from the shared
   // counter (dynamic) or every nwarps-th task (static)
@@ -398,6 +440,8 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
 
   // copy stream
   Issue is;
+  is.base = p.pixels;
+  is.pitch = is.copy_bytes = is.stride = 0;
   is.n_list = 0;
   is.rpg = 1;
   is.buf = 0;
@@ -413,11 +457,11 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
   bool failed = false;
   Lane ln;
   float hA[kLaneCols][3], hB[kLaneCols][3];
-  uint32_t par = 0;          // which of hA/hB holds the latest row
-  uint32_t c_row = 0, c_nlist = 0, c_rpg = 1, c_stride = 0, t_out = 0, out_idx = 0;
-  uint32_t c_kind = kEnd;
+  uint32_t par = 0;          // which of hA/hB receives the next row
+  uint32_t c_row = 0, c_nlist = 0, c_rpg = 1, c_stride = 0, t_out = 0;
+  bool full = false;
   const TaskMeta* cm = &ws.meta[0];
-  OutT* img_out = static_cast<OutT*>(p.out);
+  OutT* q_out = static_cast<OutT*>(p.out);  // column 2 * lane of the next output row, plane 0
 #pragma unroll
   for (int m = 0; m < static_cast<int>(kLaneCols); ++m) {
     ln.off[m] = 0;
@@ -426,7 +470,6 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
     for (int ch = 0; ch < 3; ++ch) hA[m][ch] = hB[m][ch] = 0.f;
   }
   ln.valid = 0;
-  ln.pairs = false;
 
   for (;;) {
     // -- advance the copy stream: at most kGroups groups and kMetaBufs - 1 tasks ahead -------
@@ -456,7 +499,7 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
         ++issued;
       } else {
         if (ended || prepared - finished >= kMetaBufs) break;
-        uint32_t task = next_task;
+        const uint32_t task = next_task;
         if (p.sched) {
           uint32_t got = 0;
           if (lane == 0) got = atomicAdd(&p.sched[0], 1u);
@@ -483,56 +526,57 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
 
     // -- compute stream: start the next task, or one group of the current one ------------------
     if (need_task) {
-      if (finished == prepared) break;  // only after the end marker was consumed
+      if (finished == prepared) break;
       cm = &ws.meta[finished % kMetaBufs];
-      c_kind = cm->kind;
-      if (c_kind == kEnd) break;
-      if (c_kind == kSkip) {
+      const uint32_t kind = cm->kind;
+      if (kind == kEnd) break;
+      if (kind == kSkip) {
         ++finished;
         continue;
       }
-      const uint32_t w = cm->w, rw = cm->rw, left = (rw - C) / 2, col0 = cm->col0;
-      const uint32_t xmin = cm->xmin;
+      const uint32_t w = cm->w, rw = cm->rw, col0 = cm->col0, xmin = cm->xmin;
+      const Axis ax = make_axis(w, rw, (rw - C) / 2, C);
       ln.valid = 0;
 #pragma unroll
       for (int m = 0; m < static_cast<int>(kLaneCols); ++m) {
         const uint32_t j = col0 + lane_col(lane, m);
         if (j < C) ln.valid |= 1u << m;
-        const Tap t = axis_tap(w, rw, left, j < C ? j : C - 1);
+        const Tap t = axis_tap(ax, j < C ? j : C - 1);
         ln.off[m] = 3 * (t.i0 - xmin);
         ln.lam[m] = t.lam;
       }
-      ln.pairs = (C & 1u) == 0;
-      img_out = static_cast<OutT*>(p.out) + static_cast<size_t>(cm->img) * 3 * plane;
-      out_idx = cm->k0 * C + col0 + 2 * lane;
+      full = (C & 1u) == 0 && __all_sync(0xffffffffu, ln.valid == 0x7fu);
+      q_out = static_cast<OutT*>(p.out) + static_cast<size_t>(cm->img) * 3 * plane +
+              (cm->k0 * C + col0 + 2 * lane);
       c_nlist = cm->n_list;
       c_rpg = cm->rows_per_group;
       c_stride = cm->stride;
       c_row = 0;
       t_out = 0;
       need_task = false;
-      if (c_kind == kGather) {
+      if (kind == kGather) {
         // direct path: taps straight from global memory (footprint too wide for the ring)
-        const uint8_t* __restrict__ src = p.pixels + cm->src;
+        const uint8_t* __restrict__ src = p.pixels + cm->src + 3 * xmin;
         const size_t pitch = 3 * static_cast<size_t>(w);
-        const uint32_t h = cm->h, rh = cm->rh, top = (rh - C) / 2;
-        for (uint32_t t = 0; t < cm->rows_out; ++t, out_idx += C) {
-          const Tap ty = axis_tap(h, rh, top, cm->k0 + t);
-          const uint8_t* r0 = src + ty.i0 * pitch + 3 * xmin;
-          const uint8_t* r1 = src + ty.i1 * pitch + 3 * xmin;
+        const uint32_t h = cm->h, rh = cm->rh;
+        const Axis ay = make_axis(h, rh, (rh - C) / 2, C);
+        for (uint32_t t = 0; t < cm->rows_out; ++t, q_out += C) {
+          const Tap ty = axis_tap(ay, cm->k0 + t);
+          const uint8_t* r0 = src + ty.i0 * pitch;
+          const uint8_t* r1 = src + ty.i1 * pitch;
 #pragma unroll
           for (int m = 0; m < static_cast<int>(kLaneCols); ++m) {
+            // the right neighbour is read only where it carries weight (it exists then)
+            const uint32_t nbr = ln.lam[m] > 0.f ? 3u : 0u;
 #pragma unroll
             for (int ch = 0; ch < 3; ++ch) {
-              // the right neighbour is read only where it carries weight (it exists then)
-              const uint32_t nb = ln.lam[m] > 0.f ? 3u : 0u;
-              float a = __ldg(r0 + ln.off[m] + ch), b = __ldg(r0 + ln.off[m] + nb + ch);
+              float a = __ldg(r0 + ln.off[m] + ch), b = __ldg(r0 + ln.off[m] + nbr + ch);
               hA[m][ch] = fmaf(ln.lam[m], b - a, a);
-              a = __ldg(r1 + ln.off[m] + ch), b = __ldg(r1 + ln.off[m] + nb + ch);
+              a = __ldg(r1 + ln.off[m] + ch), b = __ldg(r1 + ln.off[m] + nbr + ch);
               hB[m][ch] = fmaf(ln.lam[m], b - a, a);
             }
           }
-          emit_row<OutT>(img_out, out_idx, plane, lane, ty.lam, hA, hB, p, ln);
+          emit_row<OutT, false>(q_out, plane, lane, ty.lam, hA, hB, na, nb, ln.valid);
         }
         ++finished;
         need_task = true;
@@ -551,29 +595,43 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
       uint32_t row_addr = smem_addr(&ws.ring[slot][0]);
       for (uint32_t r = 0; r < cnt; ++r, row_addr += c_stride) {
         const uint32_t info = cm->info[c_row + r];
-        const uint32_t skew = info & 0xffu;
+        const uint32_t base = row_addr + (info & 0xffu);  // the row's first tapped byte
         uint32_t e = info >> 8;
         if (par == 0) {
 #pragma unroll
           for (int m = 0; m < static_cast<int>(kLaneCols); ++m)
-            hlerp_row(row_addr, ln.off[m] + skew, ln.lam[m], hA[m]);
-          for (; e > 0; --e, ++t_out, out_idx += C) {
+            hlerp_row(base + ln.off[m], ln.lam[m], hA[m]);
+          for (; e > 0; --e, ++t_out, q_out += C) {
             const uint32_t lbits = cm->lam[t_out];
-            if (lbits >> 31)  // both taps are this row
-              emit_row<OutT>(img_out, out_idx, plane, lane, 0.f, hA, hA, p, ln);
+            if (lbits >> 31) {  // both taps are this row
+#pragma unroll
+              for (int m = 0; m < static_cast<int>(kLaneCols); ++m)
+#pragma unroll
+                for (int ch = 0; ch < 3; ++ch) hB[m][ch] = hA[m][ch];
+            }
+            const float ly = __uint_as_float(lbits & 0x7fffffffu);
+            if (full)
+              emit_row<OutT, true>(q_out, plane, lane, ly, hB, hA, na, nb, ln.valid);
             else
-              emit_row<OutT>(img_out, out_idx, plane, lane, __uint_as_float(lbits), hB, hA, p, ln);
+              emit_row<OutT, false>(q_out, plane, lane, ly, hB, hA, na, nb, ln.valid);
           }
         } else {
 #pragma unroll
           for (int m = 0; m < static_cast<int>(kLaneCols); ++m)
-            hlerp_row(row_addr, ln.off[m] + skew, ln.lam[m], hB[m]);
-          for (; e > 0; --e, ++t_out, out_idx += C) {
+            hlerp_row(base + ln.off[m], ln.lam[m], hB[m]);
+          for (; e > 0; --e, ++t_out, q_out += C) {
             const uint32_t lbits = cm->lam[t_out];
-            if (lbits >> 31)
-              emit_row<OutT>(img_out, out_idx, plane, lane, 0.f, hB, hB, p, ln);
+            if (lbits >> 31) {
+#pragma unroll
+              for (int m = 0; m < static_cast<int>(kLaneCols); ++m)
+#pragma unroll
+                for (int ch = 0; ch < 3; ++ch) hA[m][ch] = hB[m][ch];
+            }
+            const float ly = __uint_as_float(lbits & 0x7fffffffu);
+            if (full)
+              emit_row<OutT, true>(q_out, plane, lane, ly, hA, hB, na, nb, ln.valid);
             else
-              emit_row<OutT>(img_out, out_idx, plane, lane, __uint_as_float(lbits), hA, hB, p, ln);
+              emit_row<OutT, false>(q_out, plane, lane, ly, hA, hB, na, nb, ln.valid);
           }
         }
         par ^= 1u;
