@@ -218,10 +218,12 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
     outs = [torch.empty((n, 3, C, C), dtype=tdt, device=dev) for _ in range(sets)]
     tab = torch.from_numpy(table.view(np.uint8)).to(dev)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
+    scratch = torch.zeros(pb.SCRATCH_BYTES // 4, dtype=torch.int32, device=dev)
     stream = torch.cuda.current_stream()
 
     calls = [pb.PreparedPreprocess(pix[i], tab, n, outs[i], C, S, wl.MEAN, wl.STD, out_dtype,
-                                   stream=stream, status=status) for i in range(sets)]
+                                   stream=stream, status=status, scratch=scratch)
+             for i in range(sets)]
 
     def barrier():
         if dist is not None:
@@ -260,7 +262,8 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
         done[b].synchronize()                       # the set's previous copies have finished
         pb.preba_pack(images, ph[b].numpy(), th[b])
         pb.preba_preprocess_host(ph[b], th[b], n, oh[b], pix[b], dtab[b], outs[b], C, S, wl.MEAN,
-                                 wl.STD, out_dtype, stream=stream, dev_status=status)
+                                 wl.STD, out_dtype, stream=stream, dev_status=status,
+                                 dev_scratch=scratch)
         done[b].record(stream)
 
     for i in range(2):

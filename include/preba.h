@@ -32,6 +32,7 @@ extern "C" {
 #define PREBA_PACK_ALIGN 128u     /* every image offset, and the packed size, is a multiple */
 #define PREBA_MAX_DIM 32768u      /* largest accepted image height or width */
 #define PREBA_MAX_RESIZE 16384u   /* largest accepted resize_short (and so out_size) */
+#define PREBA_SCRATCH_BYTES 256u  /* size of the scheduling scratch a batch may carry */
 
 #define PREBA_OK 0
 #define PREBA_ERR_INVALID_ARG (-1)      /* NULL, zero or out-of-range argument, misaligned buffer */
@@ -71,6 +72,13 @@ typedef struct {
   uint64_t out_bytes;            /* bytes writable at `out` (>= sizes.out_bytes) */
   int32_t* status;               /* DEVICE word or NULL: the kernel stores the first PREBA_ERR_*
                                     it meets (bad table entry, wait that ran out); caller zeroes it */
+  uint32_t* scratch;             /* DEVICE, PREBA_SCRATCH_BYTES, 16-byte aligned, or NULL.  Task
+                                    counters: with it, warps claim slabs as they finish, which
+                                    evens out a ragged batch; without it every warp takes a fixed
+                                    share.  The caller zeroes it once; each launch leaves it
+                                    zeroed again.  Launches that may overlap on the device (other
+                                    streams) need scratch of their own; zero it again after a
+                                    launch that reported an error status. */
 } preba_batch_t;
 
 /* A batch resident in host memory, with the device buffers the call stages it through. */
@@ -86,6 +94,7 @@ typedef struct {
   preba_img_t* dev_table;        /* DEVICE staging, n entries */
   void* dev_out;                 /* DEVICE staging, >= out_bytes, 16-byte aligned */
   int32_t* dev_status;           /* DEVICE word or NULL, as preba_batch_t.status */
+  uint32_t* dev_scratch;         /* DEVICE or NULL, as preba_batch_t.scratch */
 } preba_host_batch_t;
 
 /*

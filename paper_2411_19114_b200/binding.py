@@ -14,6 +14,7 @@ import numpy as np
 _LIB_PATH = Path(__file__).resolve().parent / "libpreba.so"
 
 PACK_ALIGN = 128
+SCRATCH_BYTES = 256
 F32, F16 = 0, 1
 
 OK = 0
@@ -42,7 +43,7 @@ class PrebaBatch(ctypes.Structure):
                 ("table", ctypes.c_void_p), ("table_host", ctypes.c_void_p),
                 ("n", ctypes.c_uint32), ("reserved", ctypes.c_uint32),
                 ("out", ctypes.c_void_p), ("out_bytes", ctypes.c_uint64),
-                ("status", ctypes.c_void_p)]
+                ("status", ctypes.c_void_p), ("scratch", ctypes.c_void_p)]
 
 
 class PrebaHostBatch(ctypes.Structure):
@@ -51,7 +52,7 @@ class PrebaHostBatch(ctypes.Structure):
                 ("reserved", ctypes.c_uint32), ("out_host", ctypes.c_void_p),
                 ("out_bytes", ctypes.c_uint64), ("dev_pixels", ctypes.c_void_p),
                 ("dev_table", ctypes.c_void_p), ("dev_out", ctypes.c_void_p),
-                ("dev_status", ctypes.c_void_p)]
+                ("dev_status", ctypes.c_void_p), ("dev_scratch", ctypes.c_void_p)]
 
 
 TABLE_DTYPE = np.dtype([("offset", "<u8"), ("h", "<u4"), ("w", "<u4")])
@@ -157,7 +158,7 @@ def preba_pack(images, packed: np.ndarray | None = None, table: np.ndarray | Non
 def preba_preprocess(pixels, table, n: int, out, out_size: int, resize_short: int, mean, std,
                      out_dtype: int, stream=None, table_host: np.ndarray | None = None,
                      status=None, pixels_bytes: int | None = None,
-                     out_bytes: int | None = None) -> None:
+                     out_bytes: int | None = None, scratch=None) -> None:
     """``pixels``, ``table``, ``out`` and ``status`` are CUDA tensors (or raw device
     addresses); ``stream`` is a torch stream, a raw cudaStream_t or None for torch's
     current stream."""
@@ -184,6 +185,7 @@ def preba_preprocess(pixels, table, n: int, out, out_size: int, resize_short: in
     batch.out = addr(out)
     batch.out_bytes = nbytes(out, out_bytes)
     batch.status = addr(status) if status is not None else None
+    batch.scratch = addr(scratch) if scratch is not None else None
     m, s = _f3(mean), _f3(std)
     rc = lib().preba_preprocess(ctypes.byref(batch), out_size, resize_short,
                                 _p(m, ctypes.c_float), _p(s, ctypes.c_float), out_dtype,
@@ -197,14 +199,15 @@ class PreparedPreprocess:
     makes the foreign call and nothing else (for loops that launch back to back)."""
 
     def __init__(self, pixels, table, n: int, out, out_size: int, resize_short: int, mean, std,
-                 out_dtype: int, stream=None, table_host: np.ndarray | None = None, status=None):
+                 out_dtype: int, stream=None, table_host: np.ndarray | None = None, status=None,
+                 scratch=None):
         import torch
 
         if stream is None:
             stream = torch.cuda.current_stream().cuda_stream
         elif hasattr(stream, "cuda_stream"):
             stream = stream.cuda_stream
-        self._keep = (pixels, table, out, status, table_host)
+        self._keep = (pixels, table, out, status, table_host, scratch)
         b = PrebaBatch()
         b.pixels = pixels.data_ptr()
         b.pixels_bytes = pixels.numel() * pixels.element_size()
@@ -214,6 +217,7 @@ class PreparedPreprocess:
         b.out = out.data_ptr()
         b.out_bytes = out.numel() * out.element_size()
         b.status = status.data_ptr() if status is not None else None
+        b.scratch = scratch.data_ptr() if scratch is not None else None
         self._batch = b
         self._mean, self._std = _f3(mean), _f3(std)
         self._args = (ctypes.byref(b), out_size, resize_short, _p(self._mean, ctypes.c_float),
@@ -228,7 +232,7 @@ class PreparedPreprocess:
 
 def preba_preprocess_host(packed_host, table_host: np.ndarray, n: int, out_host, dev_pixels,
                           dev_table, dev_out, out_size: int, resize_short: int, mean, std,
-                          out_dtype: int, stream=None, dev_status=None) -> None:
+                          out_dtype: int, stream=None, dev_status=None, dev_scratch=None) -> None:
     """``packed_host``/``out_host`` are (pinned) CPU tensors or numpy arrays; ``dev_*`` are
     CUDA tensors used as staging."""
     import torch
@@ -258,6 +262,7 @@ def preba_preprocess_host(packed_host, table_host: np.ndarray, n: int, out_host,
     b.dev_table = dev_table.data_ptr()
     b.dev_out = dev_out.data_ptr()
     b.dev_status = dev_status.data_ptr() if dev_status is not None else None
+    b.dev_scratch = dev_scratch.data_ptr() if dev_scratch is not None else None
     m, s = _f3(mean), _f3(std)
     rc = lib().preba_preprocess_host(ctypes.byref(b), out_size, resize_short,
                                      _p(m, ctypes.c_float), _p(s, ctypes.c_float), out_dtype,

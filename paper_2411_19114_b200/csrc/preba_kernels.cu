@@ -225,10 +225,14 @@ __device__ __forceinline__ void fence_async_shared() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 
-__device__ __forceinline__ uint32_t lds32(uint32_t addr) {
-  uint32_t v;
-  asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
-  return v;
+// Three consecutive aligned words of shared memory.
+__device__ __forceinline__ void lds32x3(uint32_t addr, uint32_t& w0, uint32_t& w1, uint32_t& w2) {
+  asm volatile(
+      "ld.shared.u32 %0, [%3];\n\t"
+      "ld.shared.u32 %1, [%3+4];\n\t"
+      "ld.shared.u32 %2, [%3+8];"
+      : "=r"(w0), "=r"(w1), "=r"(w2)
+      : "r"(addr));
 }
 
 // ---- arithmetic ---------------------------------------------------------------------------------
@@ -244,7 +248,8 @@ __device__ __forceinline__ float byte_biased(uint32_t x) {
 __device__ __forceinline__ void hlerp_row(uint32_t x, float lam, float h[3]) {
   const uint32_t addr = x & ~3u;
   const uint32_t sh = x << 3;  // the funnel shift takes it modulo 32
-  const uint32_t w0 = lds32(addr), w1 = lds32(addr + 4), w2 = lds32(addr + 8);
+  uint32_t w0, w1, w2;
+  lds32x3(addr, w0, w1, w2);
   const uint32_t lo = __funnelshift_r(w0, w1, sh);  // R0 G0 B0 R1
   const uint32_t hi = __funnelshift_r(w1, w2, sh);  // G1 B1 .. ..
   const float a0 = byte_biased<0>(lo), a1 = byte_biased<1>(lo), a2 = byte_biased<2>(lo);
@@ -358,7 +363,8 @@ __device__ __forceinline__ uint32_t prepare(const Params& p, uint32_t task, Task
     // a lane reads 12 bytes from the word holding its first tap, which may be the last
     // staged pixel: leave room for one more pixel and the word overshoot
     const uint32_t stride = (15 + 3 * copy_px + 3 + 12 + 15) & ~15u;
-    const uint32_t rpg = min(kGroupRows, kGroupBytes / stride);
+    uint32_t rpg = min(kGroupRows, kGroupBytes / stride);
+    if (rpg > 1) rpg &= ~1u;  // groups of an even number of rows keep the row parity fixed
     const uint64_t end16 = (e.offset + 3ull * e.h * e.w + 15) & ~15ull;
     kind = (rpg >= 1 && end16 <= p.pixels_bytes) ? kStream : kGather;
 
@@ -457,7 +463,6 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
   bool failed = false;
   Lane ln;
   float hA[kLaneCols][3], hB[kLaneCols][3];
-  uint32_t par = 0;          // which of hA/hB receives the next row
   uint32_t c_row = 0, c_nlist = 0, c_rpg = 1, c_stride = 0, t_out = 0;
   bool full = false;
   const TaskMeta* cm = &ws.meta[0];
@@ -593,49 +598,44 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
       }
       const uint32_t cnt = min(c_rpg, c_nlist - c_row);
       uint32_t row_addr = smem_addr(&ws.ring[slot][0]);
-      for (uint32_t r = 0; r < cnt; ++r, row_addr += c_stride) {
-        const uint32_t info = cm->info[c_row + r];
-        const uint32_t base = row_addr + (info & 0xffu);  // the row's first tapped byte
-        uint32_t e = info >> 8;
-        if (par == 0) {
-#pragma unroll
-          for (int m = 0; m < static_cast<int>(kLaneCols); ++m)
-            hlerp_row(base + ln.off[m], ln.lam[m], hA[m]);
-          for (; e > 0; --e, ++t_out, q_out += C) {
-            const uint32_t lbits = cm->lam[t_out];
-            if (lbits >> 31) {  // both taps are this row
-#pragma unroll
-              for (int m = 0; m < static_cast<int>(kLaneCols); ++m)
-#pragma unroll
-                for (int ch = 0; ch < 3; ++ch) hB[m][ch] = hA[m][ch];
-            }
-            const float ly = __uint_as_float(lbits & 0x7fffffffu);
-            if (full)
-              emit_row<OutT, true>(q_out, plane, lane, ly, hB, hA, na, nb, ln.valid);
-            else
-              emit_row<OutT, false>(q_out, plane, lane, ly, hB, hA, na, nb, ln.valid);
-          }
-        } else {
-#pragma unroll
-          for (int m = 0; m < static_cast<int>(kLaneCols); ++m)
-            hlerp_row(base + ln.off[m], ln.lam[m], hB[m]);
-          for (; e > 0; --e, ++t_out, q_out += C) {
-            const uint32_t lbits = cm->lam[t_out];
-            if (lbits >> 31) {
-#pragma unroll
-              for (int m = 0; m < static_cast<int>(kLaneCols); ++m)
-#pragma unroll
-                for (int ch = 0; ch < 3; ++ch) hA[m][ch] = hB[m][ch];
-            }
-            const float ly = __uint_as_float(lbits & 0x7fffffffu);
-            if (full)
-              emit_row<OutT, true>(q_out, plane, lane, ly, hA, hB, na, nb, ln.valid);
-            else
-              emit_row<OutT, false>(q_out, plane, lane, ly, hA, hB, na, nb, ln.valid);
-          }
+      // One staged row: horizontal pass into `cur`, then every output row it completes.
+#define PREBA_STEP(cur, prev, index)                                                        \
+  {                                                                                         \
+    const uint32_t info = cm->info[index];                                                  \
+    const uint32_t base = row_addr + (info & 0xffu); /* the row's first tapped byte */      \
+    _Pragma("unroll") for (int m = 0; m < static_cast<int>(kLaneCols); ++m)                 \
+        hlerp_row(base + ln.off[m], ln.lam[m], cur[m]);                                     \
+    for (uint32_t e = info >> 8; e > 0; --e, ++t_out, q_out += C) {                         \
+      const uint32_t lbits = cm->lam[t_out];                                                \
+      if (lbits >> 31) { /* both taps are this row */                                       \
+        _Pragma("unroll") for (int m = 0; m < static_cast<int>(kLaneCols); ++m)             \
+            _Pragma("unroll") for (int ch = 0; ch < 3; ++ch) prev[m][ch] = cur[m][ch];      \
+      }                                                                                     \
+      const float ly = __uint_as_float(lbits & 0x7fffffffu);                                \
+      if (full)                                                                             \
+        emit_row<OutT, true>(q_out, plane, lane, ly, prev, cur, na, nb, ln.valid);          \
+      else                                                                                  \
+        emit_row<OutT, false>(q_out, plane, lane, ly, prev, cur, na, nb, ln.valid);         \
+    }                                                                                       \
+    row_addr += c_stride;                                                                   \
+  }
+      if (c_rpg > 1) {
+        // rows alternate between hA and hB; every group but a task's last is even
+        uint32_t r = 0;
+        for (; r + 2 <= cnt; r += 2) {
+          PREBA_STEP(hA, hB, c_row + r)
+          PREBA_STEP(hB, hA, c_row + r + 1)
         }
-        par ^= 1u;
+        if (r < cnt) PREBA_STEP(hA, hB, c_row + r)
+      } else {
+        // one row per group (very wide footprints): keep the latest row in hA
+#pragma unroll
+        for (int m = 0; m < static_cast<int>(kLaneCols); ++m)
+#pragma unroll
+          for (int ch = 0; ch < 3; ++ch) hB[m][ch] = hA[m][ch];
+        PREBA_STEP(hA, hB, c_row)
       }
+#undef PREBA_STEP
       c_row += cnt;
       ++consumed;
       __syncwarp();  // every lane is done with the slot before the stream refills it
@@ -760,7 +760,7 @@ int launch(const Params& p, int out_dtype, cudaStream_t stream) {
 }
 
 Params make_params(const uint8_t* pixels, uint64_t pixels_bytes, const preba_img_t* table,
-                   uint32_t n, void* out, int32_t* status, uint32_t out_size,
+                   uint32_t n, void* out, int32_t* status, uint32_t* scratch, uint32_t out_size,
                    uint32_t resize_short, const float mean[3], const float std[3]) {
   Params p;
   p.pixels = pixels;
@@ -771,7 +771,7 @@ Params make_params(const uint8_t* pixels, uint64_t pixels_bytes, const preba_img
   p.n = n;
   p.C = out_size;
   p.S = resize_short;
-  p.sched = nullptr;
+  p.sched = scratch;
   p.slabs = (out_size + kSlabRows - 1) / kSlabRows;
   p.col_blocks = (out_size + kTaskCols - 1) / kTaskCols;
   p.tasks = static_cast<uint32_t>(static_cast<uint64_t>(n) * p.slabs * p.col_blocks);
@@ -793,12 +793,14 @@ extern "C" int preba_preprocess(const preba_batch_t* batch, uint32_t out_size,
   int rc = check_args(batch->pixels, batch->pixels_bytes, batch->table, batch->n, batch->out,
                       batch->out_bytes, out_size, resize_short, mean, std, out_dtype);
   if (rc != PREBA_OK) return rc;
+  if (reinterpret_cast<uintptr_t>(batch->scratch) % 16) return PREBA_ERR_INVALID_ARG;
   if (batch->table_host) {
     rc = check_table(batch->table_host, batch->n, batch->pixels_bytes);
     if (rc != PREBA_OK) return rc;
   }
   const Params p = make_params(batch->pixels, batch->pixels_bytes, batch->table, batch->n,
-                               batch->out, batch->status, out_size, resize_short, mean, std);
+                               batch->out, batch->status, batch->scratch, out_size, resize_short,
+                               mean, std);
   return launch(p, out_dtype, static_cast<cudaStream_t>(stream));
 }
 
@@ -811,6 +813,7 @@ extern "C" int preba_preprocess_host(const preba_host_batch_t* b, uint32_t out_s
   int rc = check_args(b->dev_pixels, b->packed_bytes, b->dev_table, b->n, b->dev_out,
                       b->out_bytes, out_size, resize_short, mean, std, out_dtype);
   if (rc != PREBA_OK) return rc;
+  if (reinterpret_cast<uintptr_t>(b->dev_scratch) % 16) return PREBA_ERR_INVALID_ARG;
   rc = check_table(b->table_host, b->n, b->packed_bytes);
   if (rc != PREBA_OK) return rc;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -826,7 +829,7 @@ extern "C" int preba_preprocess_host(const preba_host_batch_t* b, uint32_t out_s
     return PREBA_ERR_CUDA;
   }
   const Params p = make_params(b->dev_pixels, b->packed_bytes, b->dev_table, b->n, b->dev_out,
-                               b->dev_status, out_size, resize_short, mean, std);
+                               b->dev_status, b->dev_scratch, out_size, resize_short, mean, std);
   rc = launch(p, out_dtype, s);
   if (rc != PREBA_OK) return rc;
   err = cudaMemcpyAsync(b->out_host, b->dev_out, need, cudaMemcpyDeviceToHost, s);

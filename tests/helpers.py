@@ -21,7 +21,7 @@ def host_threads() -> int:
 
 
 def run_gpu(images, c, s, mean=MEAN, std=STD, out_dtype=pb.F32, stream=None, prefix_pad=0,
-            check_host_table=True):
+            check_host_table=True, dynamic=True):
     """Pack on the host, copy to the device between guard bands, run, return the result
     as a numpy array [n,3,c,c].  Checks the status word and the guard bands."""
     import torch
@@ -37,13 +37,18 @@ def run_gpu(images, c, s, mean=MEAN, std=STD, out_dtype=pb.F32, stream=None, pre
     out_buf = torch.full((GUARD + ob + GUARD,), CANARY, dtype=torch.uint8, device=dev)
     tab = torch.from_numpy(table.view(np.uint8)).to(dev)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
+    # dynamic: warps claim slabs through the scratch counters; else fixed shares
+    scratch = torch.zeros(pb.SCRATCH_BYTES // 4, dtype=torch.int32, device=dev) if dynamic else None
     pix = pix_buf[GUARD:GUARD + nb]
     out = out_buf[GUARD:GUARD + ob]
     torch.cuda.synchronize()
     pb.preba_preprocess(pix, tab, n, out, c, s, mean, std, out_dtype, stream=stream,
-                        table_host=table if check_host_table else None, status=status)
+                        table_host=table if check_host_table else None, status=status,
+                        scratch=scratch)
     torch.cuda.synchronize()
     assert int(status.item()) == 0, pb.preba_strerror(int(status.item()))
+    if scratch is not None:
+        assert int(scratch.abs().sum().item()) == 0, "the launch did not leave its scratch zeroed"
     ob_host = out_buf.cpu().numpy()
     assert np.all(ob_host[:GUARD] == CANARY) and np.all(ob_host[GUARD + ob:] == CANARY), \
         "kernel wrote outside the output tensor"

@@ -42,8 +42,8 @@ def test_library_exports_every_declared_function():
 def test_struct_layouts_match_header():
     assert ctypes.sizeof(pb.PrebaImg) == 16 and pb.TABLE_DTYPE.itemsize == 16
     assert ctypes.sizeof(pb.PrebaSizes) == 32
-    assert ctypes.sizeof(pb.PrebaBatch) == 64
-    assert ctypes.sizeof(pb.PrebaHostBatch) == 80
+    assert ctypes.sizeof(pb.PrebaBatch) == 72
+    assert ctypes.sizeof(pb.PrebaHostBatch) == 88
 
 
 def test_query_sizes():
@@ -144,6 +144,7 @@ def test_preprocess_rejects_bad_arguments_before_any_launch():
     assert _call(_batch(n=0)) == pb.ERR_INVALID_ARG
     assert _call(_batch(pixels=0x10001)) == pb.ERR_INVALID_ARG      # misaligned pixels
     assert _call(_batch(out=0x30008)) == pb.ERR_INVALID_ARG         # misaligned out
+    assert _call(_batch(scratch=0x40004)) == pb.ERR_INVALID_ARG     # misaligned scratch
     assert _call(_batch(), c=0) == pb.ERR_INVALID_ARG
     assert _call(_batch(), c=17, s=16) == pb.ERR_INVALID_ARG        # crop larger than resize
     assert _call(_batch(), s=16385) == pb.ERR_INVALID_ARG

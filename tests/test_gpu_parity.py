@@ -46,13 +46,14 @@ def test_other_crop_and_resize_sizes(dt, c, s):
     assert_parity(got, oracle_f64(imgs, c, s), dt)
 
 
+@pytest.mark.parametrize("dynamic", [True, False])
 @pytest.mark.parametrize("dt", DTYPES)
-def test_ragged_batch_with_odd_strides(dt):
+def test_ragged_batch_with_odd_strides(dt, dynamic):
     # widths whose row pitch 3*w is not a multiple of 16, images that end at the buffer end
     sizes = [(241, 243), (250, 499), (499, 250), (300, 301), (263, 487), (1, 1), (240, 240),
              (311, 313), (500, 500), (247, 331)]
     imgs = [uniform(500 + i, h, w) for i, (h, w) in enumerate(sizes)]
-    got = run_gpu(imgs, 224, 256, out_dtype=dt)
+    got = run_gpu(imgs, 224, 256, out_dtype=dt, dynamic=dynamic)
     assert_parity(got, oracle_f64(imgs, 224, 256), dt)
 
 
@@ -89,6 +90,30 @@ def test_workload_mixed_smooth_fp16_full():
     got = run_gpu(imgs, wl.OUT_SIZE, wl.RESIZE_SHORT, out_dtype=pb.F16)
     rep = assert_parity(got, oracle_f64(imgs, wl.OUT_SIZE, wl.RESIZE_SHORT), pb.F16)
     print("mixed fp16:", rep)
+    # the fixed-share schedule gives the same bits as the claiming one
+    fixed = run_gpu(imgs, wl.OUT_SIZE, wl.RESIZE_SHORT, out_dtype=pb.F16, dynamic=False)
+    assert np.array_equal(fixed.view(np.uint16), got.view(np.uint16))
+
+
+def test_scratch_is_reusable_across_launches():
+    import torch
+
+    imgs = wl.mixed_smooth(40, seed=21)
+    packed, table = pb.preba_pack(imgs)
+    dev = torch.device("cuda:0")
+    pix = torch.from_numpy(packed).to(dev)
+    tab = torch.from_numpy(table.view(np.uint8)).to(dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    scratch = torch.zeros(pb.SCRATCH_BYTES // 4, dtype=torch.int32, device=dev)
+    outs = [torch.zeros((40, 3, 224, 224), dtype=torch.float16, device=dev) for _ in range(5)]
+    for o in outs:  # back to back on one stream, one scratch
+        pb.preba_preprocess(pix, tab, 40, o, 224, 256, MEAN, STD, pb.F16, status=status,
+                            scratch=scratch)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0 and int(scratch.abs().sum().item()) == 0
+    want = oracle_f64(imgs, 224, 256)
+    for o in outs:
+        assert_parity(o.cpu().numpy(), want, pb.F16)
 
 
 def test_workload_hires_1080p_fp32_full():
