@@ -27,13 +27,16 @@ namespace preba {
 #define PREBA_WARPS_PER_CTA 4
 #endif
 #ifndef PREBA_CTAS_PER_SM
-#define PREBA_CTAS_PER_SM 4
+#define PREBA_CTAS_PER_SM 6
 #endif
 #ifndef PREBA_SLAB_ROWS
 #define PREBA_SLAB_ROWS 16
 #endif
 #ifndef PREBA_GROUP_BYTES
-#define PREBA_GROUP_BYTES 4608
+#define PREBA_GROUP_BYTES 2816
+#endif
+#ifndef PREBA_GROUP_ROWS
+#define PREBA_GROUP_ROWS 2
 #endif
 
 constexpr int kWarpsPerCta = PREBA_WARPS_PER_CTA;
@@ -45,8 +48,7 @@ constexpr uint32_t kSlabRows = PREBA_SLAB_ROWS;    // output rows per task (one 
 constexpr uint32_t kMaxList = 2 * 32;              // distinct source rows of a slab
 constexpr uint32_t kGroups = 2;                    // ring: one group computed, one in flight
 constexpr uint32_t kGroupBytes = PREBA_GROUP_BYTES;
-constexpr uint32_t kGroupRows = 4;                 // rows per group at most
-constexpr uint32_t kMetaBufs = 3;                  // the copy stream is at most two tasks ahead
+constexpr uint32_t kGroupRows = PREBA_GROUP_ROWS;  // rows per group at most
 constexpr uint32_t kSpinLimit = 1u << 20;          // bounded waits: give up, report, leave
 static_assert(kSlabRows >= 1 && kSlabRows <= 32, "one lane per output row of a slab");
 static_assert(kGroupBytes % 16 == 0, "bulk copies need 16-byte aligned destinations");
@@ -79,10 +81,10 @@ struct TaskMeta {
   uint32_t stride;        // bytes between staged rows of a group
   uint32_t rows_per_group;
   uint32_t n_list;        // distinct source rows of the slab, ascending
-  uint32_t pad;
+  uint32_t copy_bytes;    // tapped bytes of a staged row
   uint64_t src;           // byte offset of the image in the pixel buffer
   uint32_t info[kMaxList];  // per listed row: low byte = byte skew of the staged row,
-                            // next byte = output rows completed by this row
+                            // next byte = output rows completed by this row (<= 32)
   uint32_t lam[32];         // per output row: weight of the lower source row (float bits);
                             // sign bit set when both taps are the same row
   uint32_t row[kMaxList];   // per listed row: source row index
@@ -90,7 +92,7 @@ struct TaskMeta {
 
 struct __align__(16) WarpShared {
   uint8_t ring[kGroups][kGroupBytes];
-  TaskMeta meta[kMetaBufs];
+  TaskMeta meta;
   uint64_t full[kGroups];
 };
 
@@ -286,53 +288,81 @@ struct Lane {
   uint32_t valid;           // bit m: column m exists
 };
 
-// Vertical interpolation, normalisation and store of one output row (seven columns).
-// q points at this row's column 2 * lane in plane 0.  FULL: every column of every lane
-// exists and rows start on even element indices, so pairs go out as one vector each.
-template <typename OutT, bool FULL>
-__device__ __forceinline__ void emit_row(OutT* __restrict__ q, uint32_t plane, uint32_t lane,
-                                         float ly, const float (&hp)[kLaneCols][3],
-                                         const float (&hc)[kLaneCols][3], const float (&na)[3],
-                                         const float (&nb)[3], uint32_t valid) {
+// Normalised output value from the two horizontal results around it.
+__device__ __forceinline__ float blend(float prev, float cur, float ly, float a, float b) {
+  return fmaf(fmaf(ly, cur - prev, prev), a, b);
+}
+
+// Column group g of a lane: g < 3 is the pair (2g, 2g + 1), g == 3 the single column 6.
+// Stores the group's outputs of one row; q points at column 2 * lane of plane 0.
+template <typename OutT, bool FULL, int G>
+__device__ __forceinline__ void store_group(OutT* __restrict__ q, uint32_t plane, uint32_t lane,
+                                            const float (&prev)[kLaneCols][3],
+                                            const float (&c0)[3], const float (&c1)[3], float ly,
+                                            const float (&na)[3], const float (&nb)[3],
+                                            uint32_t valid) {
 #pragma unroll
   for (int ch = 0; ch < 3; ++ch, q += plane) {
-    float o[kLaneCols];
-#pragma unroll
-    for (int m = 0; m < static_cast<int>(kLaneCols); ++m) {
-      const float v = fmaf(ly, hc[m][ch] - hp[m][ch], hp[m][ch]);
-      o[m] = fmaf(v, na[ch], nb[ch]);
-    }
-    OutT* single = q + 192 - lane;  // column 192 + lane
-    if (FULL) {
-#pragma unroll
-      for (int pr = 0; pr < 3; ++pr)
-        *reinterpret_cast<typename Pack<OutT>::Vec*>(q + 64 * pr) =
-            Pack<OutT>::pair(o[2 * pr], o[2 * pr + 1]);
-      *single = Pack<OutT>::one(o[6]);
+    if (G < 3) {
+      const float o0 = blend(prev[2 * G][ch], c0[ch], ly, na[ch], nb[ch]);
+      const float o1 = blend(prev[2 * G + 1][ch], c1[ch], ly, na[ch], nb[ch]);
+      if (FULL) {
+        *reinterpret_cast<typename Pack<OutT>::Vec*>(q + 64 * G) = Pack<OutT>::pair(o0, o1);
+      } else {
+        if ((valid >> (2 * G)) & 1u) q[64 * G] = Pack<OutT>::one(o0);
+        if ((valid >> (2 * G + 1)) & 1u) q[64 * G + 1] = Pack<OutT>::one(o1);
+      }
     } else {
+      const float o0 = blend(prev[6][ch], c0[ch], ly, na[ch], nb[ch]);
+      if (FULL || ((valid >> 6) & 1u)) q[192 - lane] = Pack<OutT>::one(o0);
+    }
+  }
+}
+
+// One staged row: per column group the horizontal pass, then the `e` output rows the row
+// completes (weights from lam[], sign bit = both taps are this row), then the row's result
+// becomes `prev` of the next step.
+template <typename OutT, bool FULL>
+__device__ __forceinline__ void step_row(uint32_t base, uint32_t e, const uint32_t* lam,
+                                         OutT* __restrict__ q, uint32_t C, uint32_t plane,
+                                         uint32_t lane, const Lane& ln,
+                                         float (&prev)[kLaneCols][3], const float (&na)[3],
+                                         const float (&nb)[3]) {
 #pragma unroll
-      for (int m = 0; m < 6; ++m)
-        if ((valid >> m) & 1u) q[64 * (m >> 1) + (m & 1)] = Pack<OutT>::one(o[m]);
-      if ((valid >> 6) & 1u) *single = Pack<OutT>::one(o[6]);
+  for (int g = 0; g < 4; ++g) {
+    const int m0 = g < 3 ? 2 * g : 6, m1 = g < 3 ? 2 * g + 1 : 6;
+    float a0[3], a1[3] = {0.f, 0.f, 0.f};
+    hlerp_row(base + ln.off[m0], ln.lam[m0], a0);
+    if (g < 3) hlerp_row(base + ln.off[m1], ln.lam[m1], a1);
+    OutT* qq = q;
+    for (uint32_t j = 0; j < e; ++j, qq += C) {
+      const uint32_t lbits = lam[j];
+      const float ly = __uint_as_float(lbits & 0x7fffffffu);
+      if (lbits >> 31) {  // both taps are this row: the result is the row itself
+#pragma unroll
+        for (int ch = 0; ch < 3; ++ch) {
+          prev[m0][ch] = a0[ch];
+          if (g < 3) prev[m1][ch] = a1[ch];
+        }
+      }
+      if (g == 0) store_group<OutT, FULL, 0>(qq, plane, lane, prev, a0, a1, ly, na, nb, ln.valid);
+      if (g == 1) store_group<OutT, FULL, 1>(qq, plane, lane, prev, a0, a1, ly, na, nb, ln.valid);
+      if (g == 2) store_group<OutT, FULL, 2>(qq, plane, lane, prev, a0, a1, ly, na, nb, ln.valid);
+      if (g == 3) store_group<OutT, FULL, 3>(qq, plane, lane, prev, a0, a1, ly, na, nb, ln.valid);
+    }
+#pragma unroll
+    for (int ch = 0; ch < 3; ++ch) {
+      prev[m0][ch] = a0[ch];
+      if (g < 3) prev[m1][ch] = a1[ch];
     }
   }
 }
 
 // ---- task preparation: geometry of a slab into the warp's meta buffer --------------------------
 
-struct Issue {          // the copy stream's view of the task it is issuing
-  const uint8_t* base;  // image base + 3 * xmin
-  uint32_t pitch;       // 3 * w
-  uint32_t copy_bytes;  // tapped bytes of a row
-  uint32_t stride;
-  uint32_t rpg;         // rows per group
-  uint32_t n_list;
-  uint32_t buf;         // meta buffer of the task
-};
-
 // Fills `m` for task `task`; returns its kind.  All lanes take part.
 __device__ __forceinline__ uint32_t prepare(const Params& p, uint32_t task, TaskMeta& m,
-                                            uint32_t lane, Issue& is) {
+                                            uint32_t lane) {
   const uint32_t C = p.C;
   const uint32_t per_img = p.slabs * p.col_blocks;
   const uint32_t img = task / per_img;
@@ -363,8 +393,7 @@ __device__ __forceinline__ uint32_t prepare(const Params& p, uint32_t task, Task
     // a lane reads 12 bytes from the word holding its first tap, which may be the last
     // staged pixel: leave room for one more pixel and the word overshoot
     const uint32_t stride = (15 + 3 * copy_px + 3 + 12 + 15) & ~15u;
-    uint32_t rpg = min(kGroupRows, kGroupBytes / stride);
-    if (rpg > 1) rpg &= ~1u;  // groups of an even number of rows keep the row parity fixed
+    const uint32_t rpg = min(kGroupRows, kGroupBytes / stride);
     const uint64_t end16 = (e.offset + 3ull * e.h * e.w + 15) & ~15ull;
     kind = (rpg >= 1 && end16 <= p.pixels_bytes) ? kStream : kGather;
 
@@ -412,17 +441,11 @@ __device__ __forceinline__ uint32_t prepare(const Params& p, uint32_t task, Task
       m.stride = stride;
       m.rows_per_group = rpg;
       m.n_list = n_list;
+      m.copy_bytes = 3 * copy_px;
       m.src = e.offset;
     }
-    is.base = p.pixels + e.offset + 3 * xmin;
-    is.pitch = 3 * e.w;
-    is.copy_bytes = 3 * copy_px;
-    is.stride = stride;
-    is.rpg = rpg;
-    is.n_list = kind == kStream ? n_list : 0;
   } else {
     if (lane == 0) report(p.status, PREBA_ERR_BAD_TABLE);
-    is.n_list = 0;
   }
   if (lane == 0) m.kind = kind;
   __syncwarp();
@@ -431,6 +454,28 @@ __device__ __forceinline__ uint32_t prepare(const Params& p, uint32_t task, Task
 
 // ---- the warp program ---------------------------------------------------------------------------------
 
+// Issues the copies of one group of listed rows [first, first + cnt) into ring slot `slot`.
+__device__ __forceinline__ void issue_group(WarpShared& ws, uint32_t slot, uint32_t first,
+                                            uint32_t cnt, const uint8_t* base, uint32_t pitch,
+                                            uint32_t copy_bytes, uint32_t stride, uint32_t lane) {
+  const uint32_t bar = smem_addr(&ws.full[slot]);
+  if (lane < kGroupRows) {
+    if (lane < cnt) {
+      const uint8_t* src = base + static_cast<size_t>(ws.meta.row[first + lane]) * pitch;
+      const uintptr_t s = reinterpret_cast<uintptr_t>(src);
+      const uintptr_t s0 = s & ~static_cast<uintptr_t>(15);
+      const uint32_t bytes =
+          static_cast<uint32_t>(((s + copy_bytes + 15) & ~static_cast<uintptr_t>(15)) - s0);
+      fence_async_shared();
+      mbar_arrive_expect_tx(bar, bytes);
+      bulk_copy_g2s(smem_addr(&ws.ring[slot][lane * stride]), reinterpret_cast<const void*>(s0),
+                    bytes, bar);
+    } else {
+      mbar_arrive(bar);
+    }
+  }
+}
+
 template <typename OutT>
 __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint32_t lane,
                                           uint32_t gwarp, uint32_t nwarps) {
@@ -438,221 +483,125 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
   const uint32_t plane = C * C;
   const float na[3] = {p.a[0], p.a[1], p.a[2]};
   const float nb[3] = {p.b[0], p.b[1], p.b[2]};
-
-  // task claims: a warp's first task is its own index; later ones come from the shared
-  // counter (dynamic) or every nwarps-th task (static)
-  uint32_t next_task = gwarp;
-  uint32_t turn = 0;
-
-  // copy stream
-  Issue is;
-  is.base = p.pixels;
-  is.pitch = is.copy_bytes = is.stride = 0;
-  is.n_list = 0;
-  is.rpg = 1;
-  is.buf = 0;
-  uint32_t is_row = 0;       // next listed row of the issuing task to copy
-  uint32_t prepared = 0;     // tasks prepared (meta buffers written)
-  uint32_t issued = 0;       // groups issued
-  bool ended = false;        // no task left to prepare
-
-  // compute stream
-  uint32_t finished = 0;     // tasks computed
-  uint32_t consumed = 0;     // groups computed
-  bool need_task = true;
+  const TaskMeta& m = ws.meta;
+  uint32_t groups_done = 0;  // groups waited for so far: ring slot and barrier phase
   bool failed = false;
   Lane ln;
-  float hA[kLaneCols][3], hB[kLaneCols][3];
-  uint32_t c_row = 0, c_nlist = 0, c_rpg = 1, c_stride = 0, t_out = 0;
-  bool full = false;
-  const TaskMeta* cm = &ws.meta[0];
-  OutT* q_out = static_cast<OutT*>(p.out);  // column 2 * lane of the next output row, plane 0
+  float prev[kLaneCols][3];
 #pragma unroll
-  for (int m = 0; m < static_cast<int>(kLaneCols); ++m) {
-    ln.off[m] = 0;
-    ln.lam[m] = 0.f;
+  for (int c = 0; c < static_cast<int>(kLaneCols); ++c)
 #pragma unroll
-    for (int ch = 0; ch < 3; ++ch) hA[m][ch] = hB[m][ch] = 0.f;
-  }
-  ln.valid = 0;
+    for (int ch = 0; ch < 3; ++ch) prev[c][ch] = 0.f;
 
-  for (;;) {
-    // -- advance the copy stream: at most kGroups groups and kMetaBufs - 1 tasks ahead -------
-    for (;;) {
-      if (is_row < is.n_list) {
-        if (issued >= consumed + kGroups) break;
-        const uint32_t slot = issued % kGroups;
-        const uint32_t cnt = min(is.rpg, is.n_list - is_row);
-        const uint32_t bar = smem_addr(&ws.full[slot]);
-        if (lane < kGroupRows) {
-          if (lane < cnt) {
-            const uint8_t* src = is.base +
-                static_cast<size_t>(ws.meta[is.buf].row[is_row + lane]) * is.pitch;
-            const uintptr_t s = reinterpret_cast<uintptr_t>(src);
-            const uintptr_t s0 = s & ~static_cast<uintptr_t>(15);
-            const uint32_t bytes = static_cast<uint32_t>(
-                ((s + is.copy_bytes + 15) & ~static_cast<uintptr_t>(15)) - s0);
-            fence_async_shared();
-            mbar_arrive_expect_tx(bar, bytes);
-            bulk_copy_g2s(smem_addr(&ws.ring[slot][lane * is.stride]),
-                          reinterpret_cast<const void*>(s0), bytes, bar);
-          } else {
-            mbar_arrive(bar);
-          }
-        }
-        is_row += cnt;
-        ++issued;
-      } else {
-        if (ended || prepared - finished >= kMetaBufs) break;
-        const uint32_t task = next_task;
-        if (p.sched) {
-          uint32_t got = 0;
-          if (lane == 0) got = atomicAdd(&p.sched[0], 1u);
-          next_task = nwarps + __shfl_sync(0xffffffffu, got, 0);
-        } else {
-          ++turn;
-          const uint64_t t = static_cast<uint64_t>(gwarp) + static_cast<uint64_t>(turn) * nwarps;
-          next_task = t < p.tasks ? static_cast<uint32_t>(t) : p.tasks;
-        }
-        const uint32_t buf = prepared % kMetaBufs;
-        if (task >= p.tasks) {
-          if (lane == 0) ws.meta[buf].kind = kEnd;
-          __syncwarp();
-          ended = true;
-          is.n_list = 0;
-        } else {
-          (void)prepare(p, task, ws.meta[buf], lane, is);
-        }
-        is.buf = buf;
-        is_row = 0;
-        ++prepared;
-      }
-    }
-
-    // -- compute stream: start the next task, or one group of the current one ------------------
-    if (need_task) {
-      if (finished == prepared) break;
-      cm = &ws.meta[finished % kMetaBufs];
-      const uint32_t kind = cm->kind;
-      if (kind == kEnd) break;
-      if (kind == kSkip) {
-        ++finished;
-        continue;
-      }
-      const uint32_t w = cm->w, rw = cm->rw, col0 = cm->col0, xmin = cm->xmin;
+  // a warp's first task is its own index; later ones come from the shared counter (claimed
+  // when a task ends) or, without scratch, every nwarps-th task
+  for (uint32_t task = gwarp; task < p.tasks && !failed;) {
+    const uint32_t kind = prepare(p, task, ws.meta, lane);
+    if (kind != kSkip) {
+      const uint32_t w = m.w, rw = m.rw, col0 = m.col0, xmin = m.xmin;
       const Axis ax = make_axis(w, rw, (rw - C) / 2, C);
       ln.valid = 0;
 #pragma unroll
-      for (int m = 0; m < static_cast<int>(kLaneCols); ++m) {
-        const uint32_t j = col0 + lane_col(lane, m);
-        if (j < C) ln.valid |= 1u << m;
+      for (int c = 0; c < static_cast<int>(kLaneCols); ++c) {
+        const uint32_t j = col0 + lane_col(lane, c);
+        if (j < C) ln.valid |= 1u << c;
         const Tap t = axis_tap(ax, j < C ? j : C - 1);
-        ln.off[m] = 3 * (t.i0 - xmin);
-        ln.lam[m] = t.lam;
+        ln.off[c] = 3 * (t.i0 - xmin);
+        ln.lam[c] = t.lam;
       }
-      full = (C & 1u) == 0 && __all_sync(0xffffffffu, ln.valid == 0x7fu);
-      q_out = static_cast<OutT*>(p.out) + static_cast<size_t>(cm->img) * 3 * plane +
-              (cm->k0 * C + col0 + 2 * lane);
-      c_nlist = cm->n_list;
-      c_rpg = cm->rows_per_group;
-      c_stride = cm->stride;
-      c_row = 0;
-      t_out = 0;
-      need_task = false;
-      if (kind == kGather) {
+      const bool full = (C & 1u) == 0 && __all_sync(0xffffffffu, ln.valid == 0x7fu);
+      // column 2 * lane of the task's first output row, plane 0
+      OutT* q_out = static_cast<OutT*>(p.out) + static_cast<size_t>(m.img) * 3 * plane +
+                    (m.k0 * C + col0 + 2 * lane);
+      if (kind == kStream) {
+        const uint32_t n_list = m.n_list, rpg = m.rows_per_group, stride = m.stride;
+        const uint8_t* base = p.pixels + m.src + 3 * xmin;
+        const uint32_t pitch = 3 * w, copy_bytes = m.copy_bytes;
+        // two groups in flight, then one more each time a group has been computed
+        issue_group(ws, groups_done % kGroups, 0, min(rpg, n_list), base, pitch, copy_bytes, stride,
+                    lane);
+        if (rpg < n_list)
+          issue_group(ws, (groups_done + 1) % kGroups, rpg, min(rpg, n_list - rpg), base, pitch,
+                      copy_bytes, stride, lane);
+        uint32_t t_out = 0;
+        for (uint32_t row = 0; row < n_list; row += rpg) {
+          const uint32_t slot = groups_done % kGroups;
+          if (!mbar_wait(smem_addr(&ws.full[slot]), (groups_done / kGroups) & 1)) {
+            failed = true;
+            break;
+          }
+          ++groups_done;
+          const uint32_t cnt = min(rpg, n_list - row);
+          uint32_t row_addr = smem_addr(&ws.ring[slot][0]);
+          for (uint32_t r = 0; r < cnt; ++r, row_addr += stride) {
+            const uint32_t info = m.info[row + r];
+            const uint32_t e = (info >> 8) & 0xffu;
+            if (full)
+              step_row<OutT, true>(row_addr + (info & 0xffu), e, &m.lam[t_out], q_out, C, plane,
+                                   lane, ln, prev, na, nb);
+            else
+              step_row<OutT, false>(row_addr + (info & 0xffu), e, &m.lam[t_out], q_out, C, plane,
+                                    lane, ln, prev, na, nb);
+            t_out += e;
+            q_out += e * C;
+          }
+          __syncwarp();  // every lane is done with the slot before it is refilled
+          const uint32_t next = row + kGroups * rpg;
+          if (next < n_list)
+            issue_group(ws, slot, next, min(rpg, n_list - next), base, pitch, copy_bytes, stride,
+                        lane);
+        }
+        if (failed) {
+          // copies already issued may still be landing in the ring: wait for them (bounded)
+          // before the CTA can retire
+          for (uint32_t g = 0; g < kGroups; ++g)
+            (void)mbar_wait(smem_addr(&ws.full[(groups_done + g) % kGroups]),
+                            ((groups_done + g) / kGroups) & 1);
+        }
+      } else {
         // direct path: taps straight from global memory (footprint too wide for the ring)
-        const uint8_t* __restrict__ src = p.pixels + cm->src + 3 * xmin;
+        const uint8_t* __restrict__ src = p.pixels + m.src + 3 * xmin;
         const size_t pitch = 3 * static_cast<size_t>(w);
-        const uint32_t h = cm->h, rh = cm->rh;
+        const uint32_t h = m.h, rh = m.rh, k0 = m.k0, rows_out = m.rows_out;
         const Axis ay = make_axis(h, rh, (rh - C) / 2, C);
-        for (uint32_t t = 0; t < cm->rows_out; ++t, q_out += C) {
-          const Tap ty = axis_tap(ay, cm->k0 + t);
+        for (uint32_t t = 0; t < rows_out; ++t, q_out += C) {
+          const Tap ty = axis_tap(ay, k0 + t);
           const uint8_t* r0 = src + ty.i0 * pitch;
           const uint8_t* r1 = src + ty.i1 * pitch;
 #pragma unroll
-          for (int m = 0; m < static_cast<int>(kLaneCols); ++m) {
+          for (int c = 0; c < static_cast<int>(kLaneCols); ++c) {
             // the right neighbour is read only where it carries weight (it exists then)
-            const uint32_t nbr = ln.lam[m] > 0.f ? 3u : 0u;
+            const uint32_t nbr = ln.lam[c] > 0.f ? 3u : 0u;
+            float h1[3];
 #pragma unroll
             for (int ch = 0; ch < 3; ++ch) {
-              float a = __ldg(r0 + ln.off[m] + ch), b = __ldg(r0 + ln.off[m] + nbr + ch);
-              hA[m][ch] = fmaf(ln.lam[m], b - a, a);
-              a = __ldg(r1 + ln.off[m] + ch), b = __ldg(r1 + ln.off[m] + nbr + ch);
-              hB[m][ch] = fmaf(ln.lam[m], b - a, a);
+              float a = __ldg(r0 + ln.off[c] + ch), b = __ldg(r0 + ln.off[c] + nbr + ch);
+              prev[c][ch] = fmaf(ln.lam[c], b - a, a);
+              a = __ldg(r1 + ln.off[c] + ch), b = __ldg(r1 + ln.off[c] + nbr + ch);
+              h1[ch] = fmaf(ln.lam[c], b - a, a);
+            }
+            OutT* qc = q_out + (c < 6 ? 64 * (c >> 1) + (c & 1) : 192 - static_cast<int>(lane));
+            if ((ln.valid >> c) & 1u) {
+#pragma unroll
+              for (int ch = 0; ch < 3; ++ch)
+                qc[static_cast<size_t>(ch) * plane] =
+                    Pack<OutT>::one(blend(prev[c][ch], h1[ch], ty.lam, na[ch], nb[ch]));
             }
           }
-          emit_row<OutT, false>(q_out, plane, lane, ty.lam, hA, hB, na, nb, ln.valid);
         }
-        ++finished;
-        need_task = true;
       }
-      continue;
     }
-
-    // one group of staged rows
-    {
-      const uint32_t slot = consumed % kGroups;
-      if (!mbar_wait(smem_addr(&ws.full[slot]), (consumed / kGroups) & 1)) {
-        failed = true;
-        break;
-      }
-      const uint32_t cnt = min(c_rpg, c_nlist - c_row);
-      uint32_t row_addr = smem_addr(&ws.ring[slot][0]);
-      // One staged row: horizontal pass into `cur`, then every output row it completes.
-#define PREBA_STEP(cur, prev, index)                                                        \
-  {                                                                                         \
-    const uint32_t info = cm->info[index];                                                  \
-    const uint32_t base = row_addr + (info & 0xffu); /* the row's first tapped byte */      \
-    _Pragma("unroll") for (int m = 0; m < static_cast<int>(kLaneCols); ++m)                 \
-        hlerp_row(base + ln.off[m], ln.lam[m], cur[m]);                                     \
-    for (uint32_t e = info >> 8; e > 0; --e, ++t_out, q_out += C) {                         \
-      const uint32_t lbits = cm->lam[t_out];                                                \
-      if (lbits >> 31) { /* both taps are this row */                                       \
-        _Pragma("unroll") for (int m = 0; m < static_cast<int>(kLaneCols); ++m)             \
-            _Pragma("unroll") for (int ch = 0; ch < 3; ++ch) prev[m][ch] = cur[m][ch];      \
-      }                                                                                     \
-      const float ly = __uint_as_float(lbits & 0x7fffffffu);                                \
-      if (full)                                                                             \
-        emit_row<OutT, true>(q_out, plane, lane, ly, prev, cur, na, nb, ln.valid);          \
-      else                                                                                  \
-        emit_row<OutT, false>(q_out, plane, lane, ly, prev, cur, na, nb, ln.valid);         \
-    }                                                                                       \
-    row_addr += c_stride;                                                                   \
-  }
-      if (c_rpg > 1) {
-        // rows alternate between hA and hB; every group but a task's last is even
-        uint32_t r = 0;
-        for (; r + 2 <= cnt; r += 2) {
-          PREBA_STEP(hA, hB, c_row + r)
-          PREBA_STEP(hB, hA, c_row + r + 1)
-        }
-        if (r < cnt) PREBA_STEP(hA, hB, c_row + r)
-      } else {
-        // one row per group (very wide footprints): keep the latest row in hA
-#pragma unroll
-        for (int m = 0; m < static_cast<int>(kLaneCols); ++m)
-#pragma unroll
-          for (int ch = 0; ch < 3; ++ch) hB[m][ch] = hA[m][ch];
-        PREBA_STEP(hA, hB, c_row)
-      }
-#undef PREBA_STEP
-      c_row += cnt;
-      ++consumed;
-      __syncwarp();  // every lane is done with the slot before the stream refills it
-      if (c_row >= c_nlist) {
-        ++finished;
-        need_task = true;
-      }
+    __syncwarp();  // the meta buffer is free again
+    if (p.sched) {
+      uint32_t got = 0;
+      if (lane == 0) got = atomicAdd(&p.sched[0], 1u);
+      task = nwarps + __shfl_sync(0xffffffffu, got, 0);
+    } else {
+      task = task + nwarps >= task ? task + nwarps : p.tasks;
     }
   }
 
-  if (failed) {
-    if (lane == 0) report(p.status, PREBA_ERR_TIMEOUT);
-    // copies already issued may still be landing in this warp's ring: wait for them
-    // (bounded) before the CTA can retire
-    for (uint32_t q = consumed; q < issued; ++q)
-      (void)mbar_wait(smem_addr(&ws.full[q % kGroups]), (q / kGroups) & 1);
-  }
+  if (failed && lane == 0) report(p.status, PREBA_ERR_TIMEOUT);
   // the last warp out leaves the claim counters at zero for the next launch
   if (p.sched && lane == 0) {
     __threadfence();
