@@ -625,6 +625,236 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) preba_fused_kernel(const
   warp_main<OutT>(p, ws, lane, blockIdx.x * kWarpsPerCta + warp, gridDim.x * kWarpsPerCta);
 }
 
+// ---- tile kernel: a CTA stages the rows of a slab once, threads evaluate pixels --------------------
+
+#ifndef PREBA_TILE_ROWS
+#define PREBA_TILE_ROWS 16
+#endif
+#ifndef PREBA_TILE_BYTES
+#define PREBA_TILE_BYTES 32768
+#endif
+#ifndef PREBA_TILE_CTAS
+#define PREBA_TILE_CTAS 5
+#endif
+
+constexpr uint32_t kTileRows = PREBA_TILE_ROWS;    // output rows per tile
+constexpr uint32_t kTileCols = 224;                // output columns per tile
+constexpr uint32_t kTilePairs = kTileCols / 2;     // a thread owns two adjacent columns
+constexpr uint32_t kTileThreads = 2 * kTilePairs;  // even and odd rows of a pass
+constexpr uint32_t kTileBytes = PREBA_TILE_BYTES;  // staged rows
+static_assert(kTileRows <= 32 && (kTileRows & (kTileRows - 1)) == 0, "power of two, <= 32");
+static_assert(kTileThreads % 32 == 0, "whole warps");
+
+struct __align__(16) TileShared {
+  uint8_t rows[kTileBytes];
+  uint64_t full;             // completion of a pass's copies
+  uint32_t kind;             // kStream, kGather or kSkip
+  uint32_t pass_rows;        // output rows of the current pass
+  uint32_t img, k0, rows_out, col0, w, h, rw, rh, xmin;
+  uint64_t src;              // byte offset of the image in the pixel buffer
+  uint32_t a0[kTileRows];    // per output row of the pass: shared address of the first
+  uint32_t a1[kTileRows];    //   tapped byte of its upper / lower source row
+  uint32_t ly[kTileRows];    // weight of the lower row (float bits)
+  uint32_t list[32];         // source rows of the pass (producer's scratch)
+  uint32_t xoff[kTileCols];  // per output column: byte offset of its first tap in a staged row
+  float xlam[kTileCols];     //   and the weight of the second tap
+};
+
+// Builds the pass [r0, r0 + rows) of the tile: tables and copies.  Warp 0, all lanes.
+// Returns false if the pass does not fit the staging buffer.
+__device__ __forceinline__ bool tile_pass(const Params& p, TileShared& ts, const Axis& ay,
+                                          uint32_t r0, uint32_t rows, uint32_t stride,
+                                          uint32_t copy_bytes, const uint8_t* base, uint32_t pitch,
+                                          uint32_t lane, uint32_t* n_list_out) {
+  const bool active = lane < rows;
+  Tap ty = {0, 0, 0.f};
+  if (active) ty = axis_tap(ay, ts.k0 + r0 + lane);
+  const uint32_t y1_prev = __shfl_up_sync(0xffffffffu, ty.i1, 1);
+  const bool new0 = active && (lane == 0 || ty.i0 > y1_prev);
+  const bool new1 = active && ty.i1 != ty.i0 && (lane == 0 || ty.i1 > y1_prev);
+  const uint32_t cnt = (new0 ? 1u : 0u) + (new1 ? 1u : 0u);
+  uint32_t incl = cnt;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const uint32_t v = __shfl_up_sync(0xffffffffu, incl, d);
+    if (lane >= static_cast<uint32_t>(d)) incl += v;
+  }
+  const uint32_t n_list = __shfl_sync(0xffffffffu, incl, 31);
+  *n_list_out = n_list;
+  if (n_list > 32 || n_list * stride > kTileBytes) return false;
+  const uint32_t excl = incl - cnt;
+  if (new0) ts.list[excl] = ty.i0;
+  if (new1) ts.list[excl + (new0 ? 1u : 0u)] = ty.i1;
+  // slot of the lower row = last listed so far; the upper row is the one before it
+  // unless both taps coincide
+  const uint32_t s1 = incl - 1;
+  const uint32_t s0 = ty.i1 == ty.i0 ? s1 : s1 - 1;
+  const uint32_t ring = smem_addr(&ts.rows[0]);
+  if (active) {
+    const uint32_t skew0 = (3u * (ty.i0 * ts.w + ts.xmin)) & 15u;
+    const uint32_t skew1 = (3u * (ty.i1 * ts.w + ts.xmin)) & 15u;
+    ts.a0[lane] = ring + s0 * stride + skew0;
+    ts.a1[lane] = ring + s1 * stride + skew1;
+    ts.ly[lane] = __float_as_uint(ty.lam);
+  }
+  __syncwarp();
+  const uint32_t bar = smem_addr(&ts.full);
+  // one arrival per lane: a copy (with its byte count) or a plain arrival
+  if (lane < n_list) {
+    const uint8_t* src = base + static_cast<size_t>(ts.list[lane]) * pitch;
+    const uintptr_t s = reinterpret_cast<uintptr_t>(src);
+    const uintptr_t sa = s & ~static_cast<uintptr_t>(15);
+    const uint32_t bytes =
+        static_cast<uint32_t>(((s + copy_bytes + 15) & ~static_cast<uintptr_t>(15)) - sa);
+    fence_async_shared();
+    mbar_arrive_expect_tx(bar, bytes);
+    bulk_copy_g2s(ring + lane * stride, reinterpret_cast<const void*>(sa), bytes, bar);
+  } else {
+    mbar_arrive(bar);
+  }
+  return true;
+}
+
+template <typename OutT>
+__global__ void __launch_bounds__(kTileThreads, PREBA_TILE_CTAS) preba_tile_kernel(const Params p) {
+  __shared__ TileShared ts;
+  const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint32_t C = p.C;
+  const uint32_t plane = C * C;
+
+  // which tile
+  const uint32_t per_img = p.slabs * p.col_blocks;
+  const uint32_t img = blockIdx.x / per_img;
+  const uint32_t rest = blockIdx.x - img * per_img;
+  const uint32_t slab = rest / p.col_blocks;
+  const uint32_t cb = rest - slab * p.col_blocks;
+  const preba_img_t e = p.table[img];
+  if (!entry_ok(e, p.pixels_bytes)) {
+    if (tid == 0) report(p.status, PREBA_ERR_BAD_TABLE);
+    return;
+  }
+  uint32_t rh, rw;
+  if (e.h <= e.w) {
+    rh = p.S;
+    rw = static_cast<uint32_t>(static_cast<uint64_t>(p.S) * e.w / e.h);
+  } else {
+    rw = p.S;
+    rh = static_cast<uint32_t>(static_cast<uint64_t>(p.S) * e.h / e.w);
+  }
+  const uint32_t k0 = slab * kTileRows;
+  const uint32_t rows_out = min(kTileRows, C - k0);
+  const uint32_t col0 = cb * kTileCols;
+  const uint32_t cols = min(kTileCols, C - col0);
+  const Axis ax = make_axis(e.w, rw, (rw - C) / 2, C);
+  const Tap tf = axis_tap(ax, col0);
+  const Tap tl = axis_tap(ax, col0 + cols - 1);
+  const uint32_t xmin = tf.i0;
+  const uint32_t copy_px = tl.i1 - xmin + 1;
+  // a thread reads 12 bytes from the word holding its first tap, which may be the last
+  // staged pixel: leave room for one more pixel and the word overshoot
+  const uint32_t stride = (15 + 3 * copy_px + 3 + 12 + 15) & ~15u;
+  const uint64_t end16 = (e.offset + 3ull * e.h * e.w + 15) & ~15ull;
+  const bool stream = 2 * stride <= kTileBytes && end16 <= p.pixels_bytes;
+
+  if (tid == 0) {
+    mbar_init(smem_addr(&ts.full), 32);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    ts.k0 = k0;
+    ts.w = e.w;
+    ts.xmin = xmin;
+  }
+  // column taps of the tile, one per thread
+  if (tid < cols) {
+    const Tap t = axis_tap(ax, col0 + tid);
+    ts.xoff[tid] = 3 * (t.i0 - xmin);
+    ts.xlam[tid] = t.lam;
+  }
+  __syncthreads();
+
+  const uint32_t cp = tid % kTilePairs, rg = tid / kTilePairs;  // column pair, row parity
+  const uint32_t jA = 2 * cp;
+  const bool validA = jA < cols, validB = jA + 1 < cols;
+  const uint32_t offA = ts.xoff[validA ? jA : 0], offB = ts.xoff[validB ? jA + 1 : 0];
+  const float lamA = ts.xlam[validA ? jA : 0], lamB = ts.xlam[validB ? jA + 1 : 0];
+  const bool pair_ok = (C & 1u) == 0 && validB;
+  const float na[3] = {p.a[0], p.a[1], p.a[2]};
+  const float nb[3] = {p.b[0], p.b[1], p.b[2]};
+  OutT* out_img = static_cast<OutT*>(p.out) + static_cast<size_t>(img) * 3 * plane + col0 + jA;
+  const Axis ay = make_axis(e.h, rh, (rh - C) / 2, C);
+
+  if (stream) {
+    const uint8_t* base = p.pixels + e.offset + 3 * xmin;
+    const uint32_t pitch = 3 * e.w;
+    uint32_t pass_rows = kTileRows;  // shrinks (by halves) until a pass fits the buffer
+    uint32_t pass = 0;
+    for (uint32_t r0 = 0; r0 < rows_out; ++pass) {
+      if (warp == 0) {
+        uint32_t n_list = 0;
+        uint32_t rows = min(pass_rows, rows_out - r0);
+        while (!tile_pass(p, ts, ay, r0, rows, stride, 3 * copy_px, base, pitch, lane, &n_list)) {
+          pass_rows >>= 1;  // two rows always fit (checked above), so this ends at >= 1
+          rows = min(pass_rows, rows_out - r0);
+        }
+        if (lane == 0) ts.pass_rows = rows;
+      }
+      __syncthreads();
+      const uint32_t rows = ts.pass_rows;
+      if (!mbar_wait(smem_addr(&ts.full), pass & 1)) {
+        if (lane == 0) report(p.status, PREBA_ERR_TIMEOUT);
+        return;  // (the copies land in this CTA's memory or not at all: nothing to undo)
+      }
+      for (uint32_t r = rg; r < rows; r += 2) {
+        const uint32_t a0 = ts.a0[r], a1 = ts.a1[r];
+        const float ly = __uint_as_float(ts.ly[r]);
+        float tA[3], bA[3], tB[3], bB[3];
+        hlerp_row(a0 + offA, lamA, tA);
+        hlerp_row(a1 + offA, lamA, bA);
+        hlerp_row(a0 + offB, lamB, tB);
+        hlerp_row(a1 + offB, lamB, bB);
+        OutT* q = out_img + static_cast<size_t>(k0 + r0 + r) * C;
+#pragma unroll
+        for (int ch = 0; ch < 3; ++ch, q += plane) {
+          const float oA = blend(tA[ch], bA[ch], ly, na[ch], nb[ch]);
+          const float oB = blend(tB[ch], bB[ch], ly, na[ch], nb[ch]);
+          if (pair_ok) {
+            *reinterpret_cast<typename Pack<OutT>::Vec*>(q) = Pack<OutT>::pair(oA, oB);
+          } else {
+            if (validA) q[0] = Pack<OutT>::one(oA);
+            if (validB) q[1] = Pack<OutT>::one(oB);
+          }
+        }
+      }
+      r0 += rows;
+      if (r0 < rows_out) __syncthreads();  // everyone is done with the buffer
+    }
+  } else {
+    // direct path: taps straight from global memory (a row pair exceeds the buffer)
+    const uint8_t* __restrict__ src = p.pixels + e.offset + 3 * xmin;
+    const size_t pitch = 3 * static_cast<size_t>(e.w);
+    const uint32_t nA = lamA > 0.f ? 3u : 0u, nB = lamB > 0.f ? 3u : 0u;
+    for (uint32_t r = rg; r < rows_out; r += 2) {
+      const Tap ty = axis_tap(ay, k0 + r);
+      const uint8_t* r0p = src + ty.i0 * pitch;
+      const uint8_t* r1p = src + ty.i1 * pitch;
+      OutT* q = out_img + static_cast<size_t>(k0 + r) * C;
+#pragma unroll
+      for (int ch = 0; ch < 3; ++ch, q += plane) {
+        // the right neighbour is read only where it carries weight (it exists then)
+        float a = __ldg(r0p + offA + ch), b = __ldg(r0p + offA + nA + ch);
+        const float tA = fmaf(lamA, b - a, a);
+        a = __ldg(r1p + offA + ch), b = __ldg(r1p + offA + nA + ch);
+        const float bA = fmaf(lamA, b - a, a);
+        a = __ldg(r0p + offB + ch), b = __ldg(r0p + offB + nB + ch);
+        const float tB = fmaf(lamB, b - a, a);
+        a = __ldg(r1p + offB + ch), b = __ldg(r1p + offB + nB + ch);
+        const float bB = fmaf(lamB, b - a, a);
+        if (validA) q[0] = Pack<OutT>::one(blend(tA, bA, ty.lam, na[ch], nb[ch]));
+        if (validB) q[1] = Pack<OutT>::one(blend(tB, bB, ty.lam, na[ch], nb[ch]));
+      }
+    }
+  }
+}
+
 thread_local int g_last_cuda_error = 0;
 
 int check_args(const uint8_t* pixels, uint64_t pixels_bytes, const void* table, uint32_t n,
@@ -689,8 +919,31 @@ int resident_ctas(int out_dtype, cudaError_t* err) {
   return resident;
 }
 
+#ifndef PREBA_KERNEL
+#define PREBA_KERNEL 1
+#endif
+
 int launch(const Params& p, int out_dtype, cudaStream_t stream) {
   cudaError_t err = cudaSuccess;
+#if PREBA_KERNEL == 1
+  {
+    Params q = p;
+    q.slabs = (p.C + kTileRows - 1) / kTileRows;
+    q.col_blocks = (p.C + kTileCols - 1) / kTileCols;
+    const uint64_t blocks = static_cast<uint64_t>(p.n) * q.slabs * q.col_blocks;
+    if (blocks > 0x7fffffffull) return PREBA_ERR_INVALID_ARG;
+    if (out_dtype == PREBA_F16)
+      preba_tile_kernel<__half><<<static_cast<unsigned>(blocks), kTileThreads, 0, stream>>>(q);
+    else
+      preba_tile_kernel<float><<<static_cast<unsigned>(blocks), kTileThreads, 0, stream>>>(q);
+    err = cudaGetLastError();
+    if (err != cudaSuccess) {
+      g_last_cuda_error = static_cast<int>(err);
+      return PREBA_ERR_CUDA;
+    }
+    return PREBA_OK;
+  }
+#endif
   const int resident = resident_ctas(out_dtype, &err);
   if (err == cudaSuccess) {
     const uint32_t want = (p.tasks + kWarpsPerCta - 1) / kWarpsPerCta;
