@@ -34,6 +34,15 @@ extern "C" {
 #define PREBA_MAX_RESIZE 16384u   /* largest accepted resize_short (and so out_size) */
 #define PREBA_SCRATCH_BYTES 256u  /* size of the scheduling scratch a batch may carry */
 
+/* preba_batch_t.flags */
+#define PREBA_OVERLAP_PREVIOUS 1u /* the launch need not wait for the kernel before it on the
+                                     stream to finish (programmatic dependent launch): as that
+                                     kernel's warps retire, this one's take their place.  Set it
+                                     only if that kernel neither writes this batch's pixels, table
+                                     or scratch nor touches its out buffer, e.g. back-to-back
+                                     batches with buffers of their own.  Copies, and kernels
+                                     launched without the flag, order as usual. */
+
 #define PREBA_OK 0
 #define PREBA_ERR_INVALID_ARG (-1)      /* NULL, zero or out-of-range argument, misaligned buffer */
 #define PREBA_ERR_BUFFER_TOO_SMALL (-2) /* a capacity is below what preba_query reports */
@@ -67,7 +76,7 @@ typedef struct {
   const preba_img_t* table;      /* DEVICE, n entries */
   const preba_img_t* table_host; /* HOST copy of the table for checking before launch, or NULL */
   uint32_t n;                    /* images in the batch, >= 1 */
-  uint32_t reserved;
+  uint32_t flags;                /* 0 or PREBA_OVERLAP_PREVIOUS */
   void* out;                     /* DEVICE, [n,3,out_size,out_size] contiguous, 16-byte aligned */
   uint64_t out_bytes;            /* bytes writable at `out` (>= sizes.out_bytes) */
   int32_t* status;               /* DEVICE word or NULL: the kernel stores the first PREBA_ERR_*

@@ -15,6 +15,7 @@ _LIB_PATH = Path(__file__).resolve().parent / "libpreba.so"
 
 PACK_ALIGN = 128
 SCRATCH_BYTES = 256
+OVERLAP_PREVIOUS = 1
 F32, F16 = 0, 1
 
 OK = 0
@@ -41,7 +42,7 @@ class PrebaSizes(ctypes.Structure):
 class PrebaBatch(ctypes.Structure):
     _fields_ = [("pixels", ctypes.c_void_p), ("pixels_bytes", ctypes.c_uint64),
                 ("table", ctypes.c_void_p), ("table_host", ctypes.c_void_p),
-                ("n", ctypes.c_uint32), ("reserved", ctypes.c_uint32),
+                ("n", ctypes.c_uint32), ("flags", ctypes.c_uint32),
                 ("out", ctypes.c_void_p), ("out_bytes", ctypes.c_uint64),
                 ("status", ctypes.c_void_p), ("scratch", ctypes.c_void_p)]
 
@@ -158,7 +159,7 @@ def preba_pack(images, packed: np.ndarray | None = None, table: np.ndarray | Non
 def preba_preprocess(pixels, table, n: int, out, out_size: int, resize_short: int, mean, std,
                      out_dtype: int, stream=None, table_host: np.ndarray | None = None,
                      status=None, pixels_bytes: int | None = None,
-                     out_bytes: int | None = None, scratch=None) -> None:
+                     out_bytes: int | None = None, scratch=None, flags: int = 0) -> None:
     """``pixels``, ``table``, ``out`` and ``status`` are CUDA tensors (or raw device
     addresses); ``stream`` is a torch stream, a raw cudaStream_t or None for torch's
     current stream."""
@@ -186,6 +187,7 @@ def preba_preprocess(pixels, table, n: int, out, out_size: int, resize_short: in
     batch.out_bytes = nbytes(out, out_bytes)
     batch.status = addr(status) if status is not None else None
     batch.scratch = addr(scratch) if scratch is not None else None
+    batch.flags = flags
     m, s = _f3(mean), _f3(std)
     rc = lib().preba_preprocess(ctypes.byref(batch), out_size, resize_short,
                                 _p(m, ctypes.c_float), _p(s, ctypes.c_float), out_dtype,
@@ -200,7 +202,7 @@ class PreparedPreprocess:
 
     def __init__(self, pixels, table, n: int, out, out_size: int, resize_short: int, mean, std,
                  out_dtype: int, stream=None, table_host: np.ndarray | None = None, status=None,
-                 scratch=None):
+                 scratch=None, flags: int = 0):
         import torch
 
         if stream is None:
@@ -218,6 +220,7 @@ class PreparedPreprocess:
         b.out_bytes = out.numel() * out.element_size()
         b.status = status.data_ptr() if status is not None else None
         b.scratch = scratch.data_ptr() if scratch is not None else None
+        b.flags = flags
         self._batch = b
         self._mean, self._std = _f3(mean), _f3(std)
         self._args = (ctypes.byref(b), out_size, resize_short, _p(self._mean, ctypes.c_float),

@@ -145,6 +145,7 @@ def test_preprocess_rejects_bad_arguments_before_any_launch():
     assert _call(_batch(pixels=0x10001)) == pb.ERR_INVALID_ARG      # misaligned pixels
     assert _call(_batch(out=0x30008)) == pb.ERR_INVALID_ARG         # misaligned out
     assert _call(_batch(scratch=0x40004)) == pb.ERR_INVALID_ARG     # misaligned scratch
+    assert _call(_batch(flags=2)) == pb.ERR_INVALID_ARG             # unknown flag
     assert _call(_batch(), c=0) == pb.ERR_INVALID_ARG
     assert _call(_batch(), c=17, s=16) == pb.ERR_INVALID_ARG        # crop larger than resize
     assert _call(_batch(), s=16385) == pb.ERR_INVALID_ARG
