@@ -30,7 +30,7 @@ namespace preba {
 #define PREBA_CTAS_PER_SM 4
 #endif
 #ifndef PREBA_SLAB_ROWS
-#define PREBA_SLAB_ROWS 16
+#define PREBA_SLAB_ROWS 32
 #endif
 #ifndef PREBA_GROUP_BYTES
 #define PREBA_GROUP_BYTES 4608
@@ -499,11 +499,10 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
         ++issued;
       } else {
         if (ended || prepared - finished >= kMetaBufs) break;
-        const uint32_t task = next_task;
+        // the claim made while the previous task was prepared has arrived by now
+        const uint32_t task = p.sched ? __shfl_sync(0xffffffffu, next_task, 0) : next_task;
         if (p.sched) {
-          uint32_t got = 0;
-          if (lane == 0) got = atomicAdd(&p.sched[0], 1u);
-          next_task = nwarps + __shfl_sync(0xffffffffu, got, 0);
+          if (lane == 0) next_task = nwarps + atomicAdd(&p.sched[0], 1u);
         } else {
           ++turn;
           const uint64_t t = static_cast<uint64_t>(gwarp) + static_cast<uint64_t>(turn) * nwarps;

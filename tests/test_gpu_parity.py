@@ -158,6 +158,36 @@ def test_streams_give_the_same_bits_as_a_serial_run():
         assert np.array_equal(got.view(np.uint16), want.view(np.uint16))
 
 
+@pytest.mark.parametrize("dynamic", [False, True])
+def test_overlapping_launches_into_buffers_of_their_own(dynamic):
+    """Back-to-back launches marked independent of their predecessor: each batch has its own
+    pixels, output and (when claiming) scratch, so the results must be those of isolated runs."""
+    import torch
+
+    dev = torch.device("cuda:0")
+    batches = [wl.mixed_smooth(48, seed=40 + i) for i in range(3)]
+    wants = [oracle_f64(b, 224, 256) for b in batches]
+    packs = [pb.preba_pack(b) for b in batches]
+    pix = [torch.from_numpy(pk).to(dev) for pk, _ in packs]
+    tabs = [torch.from_numpy(tb.view(np.uint8)).to(dev) for _, tb in packs]
+    outs = [torch.full((48, 3, 224, 224), float("nan"), dtype=torch.float16, device=dev)
+            for _ in batches]
+    scr = [torch.zeros(pb.SCRATCH_BYTES // 4, dtype=torch.int32, device=dev) if dynamic else None
+           for _ in batches]
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    torch.cuda.synchronize()
+    for rnd in range(4):
+        for i in range(3):
+            pb.preba_preprocess(pix[i], tabs[i], 48, outs[i], 224, 256, MEAN, STD, pb.F16,
+                                status=status, scratch=scr[i], flags=pb.OVERLAP_PREVIOUS)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    for o, want, sc in zip(outs, wants, scr):
+        assert_parity(o.cpu().numpy(), want, pb.F16)
+        if sc is not None:
+            assert int(sc.abs().sum().item()) == 0
+
+
 def test_device_side_table_check_skips_bad_entries():
     import torch
 
