@@ -49,6 +49,10 @@ extern "C" {
 #define PREBA_ERR_BAD_TABLE (-3)        /* a table entry is misaligned, out of range or past the pixels */
 #define PREBA_ERR_CUDA (-4)             /* a CUDA runtime call failed; see preba_last_cuda_error */
 #define PREBA_ERR_TIMEOUT (-5)          /* only in the device status word: a bounded wait ran out */
+#define PREBA_ERR_TOO_LARGE (-6)        /* the batch exceeds PREBA_NOALLOC_MAX_BYTES */
+
+/* Device memory the library itself carries for preba_preprocess_host_noalloc (64 MiB). */
+#define PREBA_NOALLOC_MAX_BYTES (64u << 20)
 
 typedef enum { PREBA_F32 = 0, PREBA_F16 = 1 } preba_dtype_t;
 
@@ -172,6 +176,45 @@ int preba_preprocess(const preba_batch_t* batch, uint32_t out_size, uint32_t res
 int preba_preprocess_host(const preba_host_batch_t* batch, uint32_t out_size,
                           uint32_t resize_short, const float mean[3], const float std[3],
                           int out_dtype, void* stream);
+
+/*
+ * preba_preprocess_host_noalloc — preba_preprocess_host for callers that have no way to
+ * obtain device memory.  (The paper has no counterpart; this exists for the embedding.)
+ *
+ * Some hosts of this library may not allocate on the device at all: a plug-in running
+ * inside a server that owns the allocator, code on a latency path where cudaMalloc's
+ * implicit device synchronisation is forbidden, a process whose memory budget was fixed at
+ * start-up.  They still have pinned host buffers and a stream.  This entry point does the
+ * whole host-to-host transform with staging space that is part of the library image: a
+ * fixed array of PREBA_NOALLOC_MAX_BYTES in device memory, present on every GPU that
+ * loads the library for as long as the process lives.  It calls no allocating routine.
+ *
+ *   packed_host, packed_bytes, table_host, n   the batch as preba_pack wrote it (HOST;
+ *                                              pinned for the copies to be asynchronous)
+ *   out_host, out_bytes     HOST, receives [n,3,out_size,out_size]
+ *   status_host             HOST int32 or NULL: receives the kernel's status word (0 or the
+ *                           first PREBA_ERR_* met on the device) once the stream gets there
+ *   other arguments         as preba_preprocess
+ *
+ * The staging space holds, each rounded up to 256 bytes: 512 bytes of bookkeeping, the
+ * table, the packed pixels and the result.  A batch that needs more than
+ * PREBA_NOALLOC_MAX_BYTES is refused with PREBA_ERR_TOO_LARGE and nothing is enqueued.
+ *
+ * The first call on a device looks up the array's device address (one runtime query, no
+ * allocation) and keeps it; make that first call before any stream capture begins.
+ * Every call on a device uses the same array and finds the previous call's bytes in it:
+ * the bookkeeping words are cleared on the stream at the start of each call, the rest is
+ * overwritten before it is read.  Two calls whose work overlaps on the device (different
+ * streams, or several host threads) would therefore race on the array: issue them on one
+ * stream, or order them with events.
+ * Errors: PREBA_ERR_INVALID_ARG, PREBA_ERR_BUFFER_TOO_SMALL (out_bytes), PREBA_ERR_BAD_TABLE,
+ * PREBA_ERR_TOO_LARGE, PREBA_ERR_CUDA.
+ */
+int preba_preprocess_host_noalloc(const uint8_t* packed_host, uint64_t packed_bytes,
+                                  const preba_img_t* table_host, uint32_t n, void* out_host,
+                                  uint64_t out_bytes, int32_t* status_host, uint32_t out_size,
+                                  uint32_t resize_short, const float mean[3], const float std[3],
+                                  int out_dtype, void* stream);
 
 /* Text for a PREBA_* code (static storage, never NULL). */
 const char* preba_strerror(int code);

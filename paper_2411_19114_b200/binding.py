@@ -24,9 +24,11 @@ ERR_BUFFER_TOO_SMALL = -2
 ERR_BAD_TABLE = -3
 ERR_CUDA = -4
 ERR_TIMEOUT = -5
+ERR_TOO_LARGE = -6
+NOALLOC_MAX_BYTES = 64 << 20
 
 EXPORTS = ("preba_query", "preba_pack", "preba_preprocess", "preba_preprocess_host",
-           "preba_strerror", "preba_last_cuda_error")
+           "preba_preprocess_host_noalloc", "preba_strerror", "preba_last_cuda_error")
 
 
 class PrebaImg(ctypes.Structure):
@@ -90,6 +92,11 @@ def lib() -> ctypes.CDLL:
         L.preba_preprocess_host.argtypes = [ctypes.POINTER(PrebaHostBatch), ctypes.c_uint32,
                                             ctypes.c_uint32, f32p, f32p, ctypes.c_int,
                                             ctypes.c_void_p]
+        L.preba_preprocess_host_noalloc.argtypes = [
+            ctypes.c_void_p, ctypes.c_uint64, ctypes.c_void_p, ctypes.c_uint32, ctypes.c_void_p,
+            ctypes.c_uint64, ctypes.c_void_p, ctypes.c_uint32, ctypes.c_uint32, f32p, f32p,
+            ctypes.c_int, ctypes.c_void_p]
+        L.preba_preprocess_host_noalloc.restype = ctypes.c_int
         L.preba_strerror.argtypes = [ctypes.c_int]
         L.preba_strerror.restype = ctypes.c_char_p
         L.preba_last_cuda_error.argtypes = []
@@ -272,3 +279,31 @@ def preba_preprocess_host(packed_host, table_host: np.ndarray, n: int, out_host,
                                      ctypes.c_void_p(stream))
     if rc != OK:
         raise PrebaError(rc, "preba_preprocess_host")
+
+
+def preba_preprocess_host_noalloc(packed_host, table_host: np.ndarray, n: int, out_host,
+                                  out_size: int, resize_short: int, mean, std, out_dtype: int,
+                                  stream=None, status_host=None) -> None:
+    """Host buffers in, host buffers out, staged through the array the library carries in
+    device memory: nothing is allocated.  ``packed_host``/``out_host``/``status_host`` are
+    (pinned) CPU tensors or numpy arrays.  Calls must not overlap on the device."""
+    import torch
+
+    def haddr(t):
+        return t.ctypes.data if isinstance(t, np.ndarray) else t.data_ptr()
+
+    def hbytes(t):
+        return t.nbytes if isinstance(t, np.ndarray) else t.numel() * t.element_size()
+
+    if stream is None:
+        stream = torch.cuda.current_stream().cuda_stream
+    elif hasattr(stream, "cuda_stream"):
+        stream = stream.cuda_stream
+    m, s = _f3(mean), _f3(std)
+    rc = lib().preba_preprocess_host_noalloc(
+        haddr(packed_host), hbytes(packed_host), table_host.ctypes.data, n, haddr(out_host),
+        hbytes(out_host), haddr(status_host) if status_host is not None else None, out_size,
+        resize_short, _p(m, ctypes.c_float), _p(s, ctypes.c_float), out_dtype,
+        ctypes.c_void_p(stream))
+    if rc != OK:
+        raise PrebaError(rc, "preba_preprocess_host_noalloc")

@@ -66,6 +66,7 @@ extern "C" const char* preba_strerror(int code) {
     case PREBA_ERR_BAD_TABLE: return "bad image table entry";
     case PREBA_ERR_CUDA: return "CUDA runtime error";
     case PREBA_ERR_TIMEOUT: return "device wait ran out";
+    case PREBA_ERR_TOO_LARGE: return "batch exceeds the library's built-in staging space";
     default: return "unknown preba error code";
   }
 }

@@ -855,4 +855,97 @@ extern "C" int preba_preprocess_host(const preba_host_batch_t* b, uint32_t out_s
   return PREBA_OK;
 }
 
+// ---- host-to-host without any allocation ------------------------------------------------------------
+//
+// Staging space that ships with the library: every GPU that loads it carries this array
+// until the process exits.  In host code the symbol is only a stand-in; its device address
+// comes from cudaGetSymbolAddress, once per device.
+static __device__ __align__(256) unsigned char g_noalloc_space[PREBA_NOALLOC_MAX_BYTES];
+
+namespace preba {
+
+constexpr uint64_t kNoallocCounters = 0;   // scheduling counters (PREBA_SCRATCH_BYTES)
+constexpr uint64_t kNoallocStatus = 256;   // status word
+constexpr uint64_t kNoallocHeader = 512;   // cleared at the start of every call
+
+// Device address of the staging array on the current device; looked up on the first call
+// per device (concurrent first calls store the same value).
+cudaError_t noalloc_base(unsigned char** base) {
+  constexpr int kMaxDevices = 64;
+  static std::atomic<unsigned char*> cache[kMaxDevices];
+  int dev = 0;
+  cudaError_t err = cudaGetDevice(&dev);
+  if (err != cudaSuccess) return err;
+  if (dev >= 0 && dev < kMaxDevices) {
+    unsigned char* known = cache[dev].load(std::memory_order_acquire);
+    if (known) {
+      *base = known;
+      return cudaSuccess;
+    }
+  }
+  void* ptr = nullptr;
+  err = cudaGetSymbolAddress(&ptr, g_noalloc_space);
+  if (err != cudaSuccess) return err;
+  *base = static_cast<unsigned char*>(ptr);
+  if (dev >= 0 && dev < kMaxDevices) cache[dev].store(*base, std::memory_order_release);
+  return cudaSuccess;
+}
+
+}  // namespace preba
+
+extern "C" int preba_preprocess_host_noalloc(const uint8_t* packed_host, uint64_t packed_bytes,
+                                             const preba_img_t* table_host, uint32_t n,
+                                             void* out_host, uint64_t out_bytes,
+                                             int32_t* status_host, uint32_t out_size,
+                                             uint32_t resize_short, const float mean[3],
+                                             const float std[3], int out_dtype, void* stream) {
+  using namespace preba;
+  if (!packed_host || !table_host || !out_host) return PREBA_ERR_INVALID_ARG;
+  // argument checks of the device entry points, with stand-in addresses for the staging
+  int rc = check_args(reinterpret_cast<const uint8_t*>(uintptr_t{256}), packed_bytes,
+                      reinterpret_cast<const void*>(uintptr_t{256}), n,
+                      reinterpret_cast<const void*>(uintptr_t{256}), out_bytes, out_size,
+                      resize_short, mean, std, out_dtype);
+  if (rc != PREBA_OK) return rc;
+  rc = check_table(table_host, n, packed_bytes);
+  if (rc != PREBA_OK) return rc;
+  const uint64_t need_out = static_cast<uint64_t>(n) * 3ull * out_size * out_size *
+                            (out_dtype == PREBA_F16 ? 2u : 4u);
+  const uint64_t table_bytes = static_cast<uint64_t>(n) * sizeof(preba_img_t);
+  const uint64_t at_table = kNoallocHeader;
+  const uint64_t at_pixels = at_table + align_up(table_bytes, 256);
+  const uint64_t at_out = at_pixels + align_up(packed_bytes, 256);
+  const uint64_t total = at_out + align_up(need_out, 256);
+  if (total > PREBA_NOALLOC_MAX_BYTES) return PREBA_ERR_TOO_LARGE;
+
+  unsigned char* base = nullptr;
+  cudaError_t err = noalloc_base(&base);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (err == cudaSuccess) err = cudaMemsetAsync(base, 0, kNoallocHeader, s);
+  if (err == cudaSuccess)
+    err = cudaMemcpyAsync(base + at_pixels, packed_host, packed_bytes, cudaMemcpyHostToDevice, s);
+  if (err == cudaSuccess)
+    err = cudaMemcpyAsync(base + at_table, table_host, table_bytes, cudaMemcpyHostToDevice, s);
+  if (err != cudaSuccess) {
+    g_last_cuda_error = static_cast<int>(err);
+    return PREBA_ERR_CUDA;
+  }
+  const Params p = make_params(base + at_pixels, packed_bytes,
+                               reinterpret_cast<const preba_img_t*>(base + at_table), n,
+                               base + at_out, reinterpret_cast<int32_t*>(base + kNoallocStatus),
+                               reinterpret_cast<uint32_t*>(base + kNoallocCounters), out_size,
+                               resize_short, mean, std);
+  rc = launch(p, out_dtype, false, s);
+  if (rc != PREBA_OK) return rc;
+  err = cudaMemcpyAsync(out_host, base + at_out, need_out, cudaMemcpyDeviceToHost, s);
+  if (err == cudaSuccess && status_host)
+    err = cudaMemcpyAsync(status_host, base + kNoallocStatus, sizeof(int32_t),
+                          cudaMemcpyDeviceToHost, s);
+  if (err != cudaSuccess) {
+    g_last_cuda_error = static_cast<int>(err);
+    return PREBA_ERR_CUDA;
+  }
+  return PREBA_OK;
+}
+
 extern "C" int preba_last_cuda_error(void) { return preba::g_last_cuda_error; }

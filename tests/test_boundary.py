@@ -111,8 +111,8 @@ def test_pack_errors():
 
 
 def test_strerror_covers_every_code():
-    texts = {pb.preba_strerror(c) for c in range(0, -6, -1)}
-    assert len(texts) == 6 and "ok" in texts
+    texts = {pb.preba_strerror(c) for c in range(0, -7, -1)}
+    assert len(texts) == 7 and "ok" in texts
     assert "unknown" in pb.preba_strerror(-99)
 
 
