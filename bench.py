@@ -8,7 +8,7 @@ step); `e2e` is images/s from separate decoded host images: pack into pinned mem
 in, kernel, copy the result out.  Prints one JSON line (rank 0).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                    [--workload mixed|320x240|1080p|sweep] [--batch N]
+                    [--workload mixed|320x240|1080p|sweep|streams] [--batch N]
 """
 from __future__ import annotations
 
@@ -63,11 +63,33 @@ def make_workload(name: str, batch: int | None, rank: int):
         n = batch or 64
         return wl.hires_1080p(n, seed=4 + shift), "f32", \
             f"{n} images 1920x1080, smooth noise, fp32 out"
+    if name == "streams":
+        n = batch or 32
+        return wl.server_batch_500x375(0, n), "f16", \
+            f"{n} images 500x375, smooth noise, fp16 out (one of 7 servers)"
     if name == "sweep":
         n = batch or 2048
         return wl.sweep_500x375(n, seed=5 + shift), "f16", \
             f"{n} images 500x375, uniform bytes, fp16 out"
     raise SystemExit(f"unknown workload {name}")
+
+
+def config_of(desc: str, dtype: str, n: int, world: int) -> dict:
+    """The workload description both arms report."""
+    return {"workload": desc, "resize_short": wl.RESIZE_SHORT, "out_size": wl.OUT_SIZE,
+            "out_dtype": dtype, "images_per_step_per_gpu": n,
+            "parallelism": f"dp{world} (independent batches, no collective)"}
+
+
+def max_over_ranks(values, dist, device):
+    """Element-wise maximum of a list of floats over all ranks (identity without a group)."""
+    if dist is None:
+        return [float(v) for v in values]
+    import torch
+
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t.tolist()]
 
 
 def measured_peak() -> tuple[float, str]:
@@ -177,12 +199,101 @@ def run_reference(args, rank: int, world: int) -> None:
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": len(times), "warmup": len(warm), "ms_per_step": 1e3 * total / len(times),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-        "data": "synthetic", "config": {"workload": desc, "resize_short": wl.RESIZE_SHORT,
-                                        "out_size": wl.OUT_SIZE},
+        "data": "synthetic", "config": config_of(desc, dtype, n, max(1, args.gpus)),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
                          "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def run_streams(args, local_rank: int) -> None:
+    """Seven small inference servers sharing one GPU (the paper's 1g.5gb x 7 set-up, Sec. 3):
+    seven host threads, each with its own stream and a batch of 32 images of 500x375, launch
+    batch after batch; reports aggregate images/s and per-batch latency percentiles."""
+    import torch
+
+    from paper_2411_19114_b200 import binding as pb
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device (the CUDA path has no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    pb.lib()
+    n_streams, n, C, S = 7, args.batch or 32, wl.OUT_SIZE, wl.RESIZE_SHORT
+    steps, warm = args.steps, max(args.warmup, 3)
+    ctx = []
+    acct_total = 0
+    for sidx in range(n_streams):
+        images = wl.server_batch_500x375(sidx, n)
+        packed, table = pb.preba_pack(images)
+        acct_total += accounting.batch_bytes(table, C, S, 2)["total"]
+        st = torch.cuda.Stream(device=dev)
+        pix = torch.from_numpy(packed).to(dev)
+        tab = torch.from_numpy(table.view(np.uint8)).to(dev)
+        out = torch.empty((n, 3, C, C), dtype=torch.float16, device=dev)
+        status = torch.zeros(1, dtype=torch.int32, device=dev)
+        call = pb.PreparedPreprocess(pix, tab, n, out, C, S, wl.MEAN, wl.STD, pb.F16, stream=st,
+                                     status=status)
+        # the same batch alone on the default stream: the concurrent run must give these bits
+        alone = torch.empty_like(out)
+        pb.preba_preprocess(pix, tab, n, alone, C, S, wl.MEAN, wl.STD, pb.F16, status=status)
+        ctx.append(dict(stream=st, call=call, out=out, alone=alone, status=status, keep=(pix, tab)))
+    torch.cuda.synchronize()
+    gate = threading.Barrier(n_streams)
+    lat = [None] * n_streams
+    span = [None] * n_streams
+
+    def server(sidx):
+        c = ctx[sidx]
+        st, call = c["stream"], c["call"]
+        for _ in range(warm):
+            call()
+        st.synchronize()
+        begins = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+        ends = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+        gate.wait()
+        for i in range(steps):
+            begins[i].record(st)
+            call()
+            ends[i].record(st)
+        st.synchronize()
+        lat[sidx] = np.array([b.elapsed_time(e) * 1e3 for b, e in zip(begins, ends)])
+        span[sidx] = begins[0].elapsed_time(ends[-1])
+
+    with ClockSampler(local_rank) as clocks:
+        threads = [threading.Thread(target=server, args=(i,)) for i in range(n_streams)]
+        for t in threads:
+            t.start()
+        for t in threads:
+            t.join()
+    torch.cuda.synchronize()
+    same = all(int(c["status"].item()) == 0 and bool(torch.equal(c["out"], c["alone"])) for c in ctx)
+    assert same, "concurrent streams changed the result"
+    elapsed_ms = max(span)
+    peak, peak_src = measured_peak()
+    achieved = acct_total * steps / (elapsed_ms * 1e-3) / 1e9
+    all_lat = np.concatenate(lat)
+    line = {
+        "metric": METRIC, "value": n_streams * n * steps / (elapsed_ms * 1e-3), "unit": UNIT,
+        "n_gpus": 1, "steps": steps, "warmup": warm, "ms_per_step": elapsed_ms / steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic",
+        "config": dict(config_of(f"{n_streams} concurrent streams x {n} images 500x375, smooth "
+                                 "noise, fp16 out", "f16", n, 1),
+                       launch="7 host threads, one stream each, no flags",
+                       l2="inputs and outputs of all streams stay resident (warm L2)"),
+        "streams": {"count": n_streams,
+                    "batch_latency_us": {"p50": float(np.percentile(all_lat, 50)),
+                                         "p95": float(np.percentile(all_lat, 95)),
+                                         "p99": float(np.percentile(all_lat, 99))},
+                    "per_stream_p99_us": [float(np.percentile(v, 99)) for v in lat],
+                    "bits_identical_to_serial": same},
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "traffic": None, "peak_source": peak_src,
+                     "algorithmic_bytes_per_launch": acct_total // n_streams},
+        "gpu_launches": n_streams * steps, "clocks": clocks.summary(),
     }
     print(json.dumps(line), flush=True)
 
@@ -264,15 +375,17 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
     th = [np.zeros(n, dtype=pb.TABLE_DTYPE) for _ in range(nbuf)]
     dtab = [torch.empty(n * 16, dtype=torch.uint8, device=dev) for _ in range(nbuf)]
     done = [torch.cuda.Event() for _ in range(nbuf)]
+    side = [torch.cuda.Stream(device=dev) for _ in range(nbuf)]  # one stream per buffer set:
+    scr = [torch.zeros(pb.SCRATCH_BYTES // 4, dtype=torch.int32, device=dev) for _ in range(nbuf)]
 
     def e2e_step(i):
         b = i % nbuf
         done[b].synchronize()                       # the set's previous copies have finished
         pb.preba_pack(images, ph[b].numpy(), th[b])
         pb.preba_preprocess_host(ph[b], th[b], n, oh[b], pix[b], dtab[b], outs[b], C, S, wl.MEAN,
-                                 wl.STD, out_dtype, stream=stream, dev_status=status,
-                                 dev_scratch=scratch)
-        done[b].record(stream)
+                                 wl.STD, out_dtype, stream=side[b], dev_status=status,
+                                 dev_scratch=scr[b])
+        done[b].record(side[b])
 
     for i in range(2):
         e2e_step(i)
@@ -280,19 +393,20 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
     e_start, e_stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t_pack = 0.0
     e_start.record(stream)
+    for st in side:
+        st.wait_stream(stream)                      # the timed region starts on both streams
     for i in range(e2e_steps):
         t0 = time.perf_counter()
         e2e_step(i)
         t_pack += time.perf_counter() - t0
+    for st in side:
+        stream.wait_stream(st)                      # ... and ends when both are done
     e_stop.record(stream)
     barrier()
     e2e_ms = e_start.elapsed_time(e_stop)
     assert int(status.item()) == 0
 
-    if dist is not None:
-        t = torch.tensor([elapsed_ms, e2e_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms, e2e_ms = (float(v) for v in t.tolist())
+    elapsed_ms, e2e_ms = max_over_ranks([elapsed_ms, e2e_ms], dist, dev)
 
     if rank == 0:
         peak, peak_src = measured_peak()
@@ -308,12 +422,11 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
             "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
             "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": desc, "resize_short": S, "out_size": C, "out_dtype": dtype,
-                       "images_per_step_per_gpu": n, "parallelism": f"dp{world} (independent batches)",
-                       "launch": "one stream, back-to-back launches marked independent of "
-                                 "their predecessor (programmatic dependent launch)",
-                       "l2": f"rotating {sets} input/output buffer sets "
-                             f"({sets * step_bytes / 1e6:.0f} MB) > L2 ({l2 / 1e6:.0f} MB)"},
+            "config": dict(config_of(desc, dtype, n, world),
+                           launch="one stream, back-to-back launches marked independent of "
+                                  "their predecessor (programmatic dependent launch)",
+                           l2=f"rotating {sets} input/output buffer sets "
+                              f"({sets * step_bytes / 1e6:.0f} MB) > L2 ({l2 / 1e6:.0f} MB)"),
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                          "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src,
                          "algorithmic_bytes_per_launch": acct["total"],
@@ -328,7 +441,8 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
                     "d2h_bytes_per_step": int(sizes.out_bytes), "steps": e2e_steps,
                     "ms_per_step": e2e_ms / e2e_steps,
                     "host_ms_per_step": 1e3 * t_pack / e2e_steps,
-                    "includes": "preba_pack into pinned memory + H2D + kernel + D2H"},
+                    "includes": "preba_pack into pinned memory + H2D + kernel + D2H, two "
+                                "buffer sets on two streams"},
             "gpu_launches": args.steps,
             "clocks": clocks.summary(),
         }
@@ -344,7 +458,8 @@ def main() -> None:
     ap.add_argument("--steps", type=int, default=20000)
     ap.add_argument("--warmup", type=int, default=200)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="mixed", choices=["mixed", "320x240", "1080p", "sweep"])
+    ap.add_argument("--workload", default="mixed",
+                    choices=["mixed", "320x240", "1080p", "sweep", "streams"])
     ap.add_argument("--batch", type=int, default=None)
     ap.add_argument("--e2e-steps", type=int, default=20)
     ap.add_argument("--cpu-budget", type=float, default=12.0,
@@ -355,6 +470,9 @@ def main() -> None:
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     if args.impl == "reference":
         run_reference(args, rank, world)
+    elif args.workload == "streams":
+        if rank == 0:
+            run_streams(args, local_rank)
     else:
         run_ours(args, rank, world, local_rank)
 

@@ -129,7 +129,8 @@ int preba_query(const uint32_t* h, const uint32_t* w, uint32_t n, uint32_t out_s
  * preba_pack — step 0 of the path: builds the packed pixel buffer and the
  * {offset, h, w} table from n separate decoded images (each HWC uint8, row
  * pitch 3*w).  Padding bytes between images and at the tail are written as 0,
- * so the result is a pure function of the inputs.
+ * so the result is a pure function of the inputs.  Batches above a few megabytes
+ * are copied by up to 8 short-lived worker threads.
  *   images    HOST array of n HOST pointers
  *   packed    HOST, `capacity` bytes; must hold sizes.packed_bytes
  *   table     HOST, n entries, written

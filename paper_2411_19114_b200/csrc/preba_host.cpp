@@ -1,5 +1,8 @@
 // Host-side entry points that need no device: sizes, packing, error text.
+#include <algorithm>
 #include <cstring>
+#include <thread>
+#include <vector>
 
 #include "preba.h"
 #include "preba_internal.h"
@@ -46,14 +49,41 @@ extern "C" int preba_pack(const uint8_t* const* images, const uint32_t* h, const
   if (capacity < need) return PREBA_ERR_BUFFER_TOO_SMALL;
   uint64_t at = 0;
   for (uint32_t i = 0; i < n; ++i) {
-    const uint64_t bytes = 3ull * h[i] * w[i];
     table[i].offset = at;
     table[i].h = h[i];
     table[i].w = w[i];
-    std::memcpy(packed + at, images[i], bytes);
-    const uint64_t next = preba::align_up(at + bytes, PREBA_PACK_ALIGN);
-    std::memset(packed + at + bytes, 0, next - (at + bytes));
-    at = next;
+    at = preba::align_up(at + 3ull * h[i] * w[i], PREBA_PACK_ALIGN);
+  }
+  // the copies: images are independent, so large batches are split over a few threads
+  // (contiguous runs of images of about equal bytes)
+  auto copy_run = [&](uint32_t first, uint32_t last) {
+    for (uint32_t i = first; i < last; ++i) {
+      const uint64_t bytes = 3ull * h[i] * w[i];
+      const uint64_t off = table[i].offset;
+      std::memcpy(packed + off, images[i], bytes);
+      const uint64_t next = preba::align_up(off + bytes, PREBA_PACK_ALIGN);
+      std::memset(packed + off + bytes, 0, next - (off + bytes));
+    }
+  };
+  constexpr uint64_t kBytesPerThread = 4ull << 20;
+  const unsigned hw = std::max(1u, std::thread::hardware_concurrency());
+  const unsigned workers = static_cast<unsigned>(
+      std::min<uint64_t>({8, hw, need / kBytesPerThread, static_cast<uint64_t>(n)}));
+  if (workers <= 1) {
+    copy_run(0, n);
+  } else {
+    std::vector<std::thread> pool;
+    uint32_t first = 0;
+    for (unsigned t = 0; t < workers; ++t) {
+      // run t ends where the byte count passes its share
+      uint32_t last = first;
+      const uint64_t goal = need * (t + 1) / workers;
+      while (last < n && (t + 1 == workers || table[last].offset < goal)) ++last;
+      if (t + 1 == workers) last = n;
+      pool.emplace_back(copy_run, first, last);
+      first = last;
+    }
+    for (auto& th : pool) th.join();
   }
   return PREBA_OK;
 }
