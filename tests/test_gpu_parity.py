@@ -76,6 +76,40 @@ def test_extreme_downscale_and_upscale():
         assert_parity(got, oracle_f64(imgs, 224, 256), dt)
 
 
+def test_largest_accepted_dimensions():
+    imgs = [uniform(610, 8, 32768), uniform(611, 32768, 8), uniform(612, 1, 32768)]
+    for dt in DTYPES:
+        got = run_gpu(imgs, 224, 256, out_dtype=dt)
+        assert_parity(got, oracle_f64(imgs, 224, 256), dt)
+
+
+def test_large_crop_with_several_column_blocks_and_strong_upscale():
+    imgs = [uniform(620, 300, 400), uniform(621, 90, 61)]
+    got = run_gpu(imgs, 1000, 1024, out_dtype=pb.F32)
+    assert_parity(got, oracle_f64(imgs, 1000, 1024), pb.F32)
+
+
+def test_pixel_buffer_without_tail_padding_is_not_read_past_its_end():
+    """The caller may state the exact byte count (no 16-byte slack after the last image):
+    the kernel then may not round the last rows' copies up, and must still be right."""
+    import torch
+
+    img = uniform(630, 37, 53)                      # 5883 bytes, not a multiple of 16
+    packed, table = pb.preba_pack([img])
+    exact = 3 * 37 * 53
+    dev = torch.device("cuda:0")
+    buf = torch.full((4096 + len(packed) + 4096,), 0xA5, dtype=torch.uint8, device=dev)
+    buf[4096:4096 + exact] = torch.from_numpy(packed[:exact]).to(dev)   # canary right behind it
+    tab = torch.from_numpy(table.view(np.uint8)).to(dev)
+    out = torch.zeros((1, 3, 24, 24), dtype=torch.float32, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    pb.preba_preprocess(buf[4096:], tab, 1, out, 24, 32, MEAN, STD, pb.F32, status=status,
+                        pixels_bytes=exact, table_host=table)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert_parity(out.cpu().numpy(), oracle_f64([img], 24, 32), pb.F32)
+
+
 # ---- the workloads at full size -------------------------------------------------------------------
 
 def test_workload_uniform_320x240_fp32_full():
