@@ -217,6 +217,39 @@ int preba_preprocess_host_noalloc(const uint8_t* packed_host, uint64_t packed_by
                                   uint32_t resize_short, const float mean[3], const float std[3],
                                   int out_dtype, void* stream);
 
+/*
+ * Batching front-end (host only) — the stage between preprocessing and model execution
+ * (paper Sec. 2.3 item 2): single-input requests wait in arrival order and leave as a batch
+ * when Batch_max of them are queued or when the oldest has waited Time_queue.  The paper's
+ * batching system (Sec. 4.3) sets the two hyper-parameters from a one-time profile:
+ * Batch_max = Batch_knee, the batch size at the knee of the latency curve, and
+ * Time_queue = Time_knee / number of servers sharing the GPU (Time_knee itself for one big
+ * GPU).  For this library's kernel the profile is bench.py's batch-size sweep.
+ *
+ * preba_batching_params   the two hyper-parameters from the profile (Sec. 4.3).
+ * preba_batcher_create    a queue with those parameters (batch_max >= 1); NULL on failure.
+ * preba_batcher_push      enqueue request `id` that arrived at `arrival_ns`; arrival times
+ *                         must not decrease.  PREBA_ERR_INVALID_ARG otherwise.
+ * preba_batcher_poll      at time `now_ns`: if a batch is due, writes its request ids (oldest
+ *                         first) to `ids` and returns their count; else returns 0.  A batch is
+ *                         due when batch_max requests are queued (it takes the oldest
+ *                         batch_max) or when now_ns >= oldest arrival + time_queue_ns (it
+ *                         takes everything queued).  `next_deadline_ns`, if not NULL, receives
+ *                         the time at which the then-oldest request runs out of waiting time
+ *                         (UINT64_MAX when the queue is empty).  `capacity` must be >=
+ *                         batch_max (PREBA_ERR_BUFFER_TOO_SMALL).
+ * preba_batcher_destroy   frees the queue.
+ * Calls on one queue may come from several threads (one lock per queue).
+ */
+typedef struct preba_batcher preba_batcher_t;
+int preba_batching_params(uint32_t batch_knee, uint64_t time_knee_ns, uint32_t n_servers,
+                          uint32_t* batch_max, uint64_t* time_queue_ns);
+preba_batcher_t* preba_batcher_create(uint32_t batch_max, uint64_t time_queue_ns);
+void preba_batcher_destroy(preba_batcher_t* b);
+int preba_batcher_push(preba_batcher_t* b, uint64_t id, uint64_t arrival_ns);
+int preba_batcher_poll(preba_batcher_t* b, uint64_t now_ns, uint64_t* ids, uint32_t capacity,
+                       uint64_t* next_deadline_ns);
+
 /* Text for a PREBA_* code (static storage, never NULL). */
 const char* preba_strerror(int code);
 

@@ -28,7 +28,9 @@ ERR_TOO_LARGE = -6
 NOALLOC_MAX_BYTES = 64 << 20
 
 EXPORTS = ("preba_query", "preba_pack", "preba_preprocess", "preba_preprocess_host",
-           "preba_preprocess_host_noalloc", "preba_strerror", "preba_last_cuda_error")
+           "preba_preprocess_host_noalloc", "preba_strerror", "preba_last_cuda_error",
+           "preba_batching_params", "preba_batcher_create", "preba_batcher_destroy",
+           "preba_batcher_push", "preba_batcher_poll")
 
 
 class PrebaImg(ctypes.Structure):
@@ -97,6 +99,19 @@ def lib() -> ctypes.CDLL:
             ctypes.c_uint64, ctypes.c_void_p, ctypes.c_uint32, ctypes.c_uint32, f32p, f32p,
             ctypes.c_int, ctypes.c_void_p]
         L.preba_preprocess_host_noalloc.restype = ctypes.c_int
+        u64p = ctypes.POINTER(ctypes.c_uint64)
+        L.preba_batching_params.argtypes = [ctypes.c_uint32, ctypes.c_uint64, ctypes.c_uint32,
+                                            u32p, u64p]
+        L.preba_batching_params.restype = ctypes.c_int
+        L.preba_batcher_create.argtypes = [ctypes.c_uint32, ctypes.c_uint64]
+        L.preba_batcher_create.restype = ctypes.c_void_p
+        L.preba_batcher_destroy.argtypes = [ctypes.c_void_p]
+        L.preba_batcher_destroy.restype = None
+        L.preba_batcher_push.argtypes = [ctypes.c_void_p, ctypes.c_uint64, ctypes.c_uint64]
+        L.preba_batcher_push.restype = ctypes.c_int
+        L.preba_batcher_poll.argtypes = [ctypes.c_void_p, ctypes.c_uint64, u64p, ctypes.c_uint32,
+                                         u64p]
+        L.preba_batcher_poll.restype = ctypes.c_int
         L.preba_strerror.argtypes = [ctypes.c_int]
         L.preba_strerror.restype = ctypes.c_char_p
         L.preba_last_cuda_error.argtypes = []
@@ -307,3 +322,47 @@ def preba_preprocess_host_noalloc(packed_host, table_host: np.ndarray, n: int, o
         ctypes.c_void_p(stream))
     if rc != OK:
         raise PrebaError(rc, "preba_preprocess_host_noalloc")
+
+
+NEVER = (1 << 64) - 1
+
+
+def preba_batching_params(batch_knee: int, time_knee_ns: int, n_servers: int) -> tuple[int, int]:
+    bm, tq = ctypes.c_uint32(), ctypes.c_uint64()
+    rc = lib().preba_batching_params(batch_knee, time_knee_ns, n_servers, ctypes.byref(bm),
+                                     ctypes.byref(tq))
+    if rc != OK:
+        raise PrebaError(rc, "preba_batching_params")
+    return bm.value, tq.value
+
+
+class PrebaBatcher:
+    """A queue of the batching front-end (``preba_batcher_*``)."""
+
+    def __init__(self, batch_max: int, time_queue_ns: int):
+        self._h = lib().preba_batcher_create(batch_max, time_queue_ns)
+        if not self._h:
+            raise PrebaError(ERR_INVALID_ARG, "preba_batcher_create")
+        self._ids = (ctypes.c_uint64 * batch_max)()
+        self._cap = batch_max
+
+    def push(self, request_id: int, arrival_ns: int) -> None:
+        rc = lib().preba_batcher_push(self._h, request_id, arrival_ns)
+        if rc != OK:
+            raise PrebaError(rc, "preba_batcher_push")
+
+    def poll(self, now_ns: int) -> tuple[list[int], int]:
+        """(ids of the batch that is due, or []; next deadline or NEVER)."""
+        nxt = ctypes.c_uint64()
+        rc = lib().preba_batcher_poll(self._h, now_ns, self._ids, self._cap, ctypes.byref(nxt))
+        if rc < 0:
+            raise PrebaError(rc, "preba_batcher_poll")
+        return [int(self._ids[i]) for i in range(rc)], nxt.value
+
+    def close(self) -> None:
+        if self._h:
+            lib().preba_batcher_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        self.close()
