@@ -43,9 +43,15 @@ constexpr uint32_t kLaneCols = 7;                  // output columns per lane
 constexpr uint32_t kTaskCols = 32 * kLaneCols;     // 224 output columns per task
 constexpr uint32_t kSlabRows = PREBA_SLAB_ROWS;    // output rows per task (one lane per row)
 constexpr uint32_t kMaxList = 2 * 32;              // distinct source rows of a slab
-constexpr uint32_t kGroups = 2;                    // ring: one group computed, one in flight
+#ifndef PREBA_GROUPS
+#define PREBA_GROUPS 2
+#endif
+#ifndef PREBA_GROUP_ROWS
+#define PREBA_GROUP_ROWS 6
+#endif
+constexpr uint32_t kGroups = PREBA_GROUPS;         // ring: one group computed, the rest in flight
 constexpr uint32_t kGroupBytes = PREBA_GROUP_BYTES;
-constexpr uint32_t kGroupRows = 4;                 // rows per group at most
+constexpr uint32_t kGroupRows = PREBA_GROUP_ROWS;  // rows per group at most
 constexpr uint32_t kMetaBufs = 3;                  // the copy stream is at most two tasks ahead
 constexpr uint32_t kSpinLimit = 1u << 20;          // bounded waits: give up, report, leave
 static_assert(kSlabRows >= 1 && kSlabRows <= 32, "one lane per output row of a slab");
@@ -301,9 +307,9 @@ __device__ __forceinline__ void emit_row(OutT* __restrict__ q, uint32_t plane, u
     if (FULL) {
 #pragma unroll
       for (int pr = 0; pr < 3; ++pr)
-        *reinterpret_cast<typename Pack<OutT>::Vec*>(q + 64 * pr) =
-            Pack<OutT>::pair(o[2 * pr], o[2 * pr + 1]);
-      *single = Pack<OutT>::one(o[6]);
+        __stcs(reinterpret_cast<typename Pack<OutT>::Vec*>(q + 64 * pr),
+               Pack<OutT>::pair(o[2 * pr], o[2 * pr + 1]));
+      __stcs(single, Pack<OutT>::one(o[6]));
     } else {
 #pragma unroll
       for (int m = 0; m < 6; ++m)
