@@ -13,7 +13,6 @@ in, kernel, copy the result out.  Prints one JSON line (rank 0).
 from __future__ import annotations
 
 import argparse
-import ctypes
 import hashlib
 import json
 import os

@@ -20,7 +20,7 @@ def host_threads() -> int:
     return max(1, len(os.sched_getaffinity(0)))
 
 
-def run_gpu(images, c, s, mean=MEAN, std=STD, out_dtype=pb.F32, stream=None, prefix_pad=0,
+def run_gpu(images, c, s, mean=MEAN, std=STD, out_dtype=pb.F32, stream=None,
             check_host_table=True, dynamic=True):
     """Pack on the host, copy to the device between guard bands, run, return the result
     as a numpy array [n,3,c,c].  Checks the status word and the guard bands."""

@@ -129,6 +129,33 @@ def test_workload_mixed_smooth_fp16_full():
     assert np.array_equal(fixed.view(np.uint16), got.view(np.uint16))
 
 
+def test_workload_mixed_smooth_fp16_full_in_the_benchmark_launch_configuration():
+    """The 256-image ragged batch as bench.py launches it: back to back on one stream, every
+    launch marked independent of its predecessor, rotating over several buffer sets."""
+    import torch
+
+    imgs = wl.mixed_smooth()
+    n = len(imgs)
+    want = oracle_f64(imgs, wl.OUT_SIZE, wl.RESIZE_SHORT)
+    packed, table = pb.preba_pack(imgs)
+    dev = torch.device("cuda:0")
+    sets = 4
+    pix = [torch.from_numpy(packed).to(dev) for _ in range(sets)]
+    tab = torch.from_numpy(table.view(np.uint8)).to(dev)
+    outs = [torch.full((n, 3, 224, 224), float("nan"), dtype=torch.float16, device=dev)
+            for _ in range(sets)]
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    calls = [pb.PreparedPreprocess(pix[i], tab, n, outs[i], 224, 256, MEAN, STD, pb.F16,
+                                   status=status, flags=pb.OVERLAP_PREVIOUS) for i in range(sets)]
+    torch.cuda.synchronize()
+    for i in range(10 * sets):
+        calls[i % sets]()
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    for o in outs:
+        assert_parity(o.cpu().numpy(), want, pb.F16)
+
+
 def test_scratch_is_reusable_across_launches():
     import torch
 
