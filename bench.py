@@ -241,26 +241,32 @@ def run_streams(args, local_rank: int) -> None:
         pb.preba_preprocess(pix, tab, n, alone, C, S, wl.MEAN, wl.STD, pb.F16, status=status)
         ctx.append(dict(stream=st, call=call, out=out, alone=alone, status=status, keep=(pix, tab)))
     torch.cuda.synchronize()
-    # One host thread feeds the seven streams in turn (in Python, seven threads would spend
-    # their time handing the interpreter lock around); the streams run concurrently on the
-    # device.  Every batch is bracketed by events on its own stream.
-    for _ in range(warm):
-        for c in ctx:
-            c["call"]()
-    torch.cuda.synchronize()
-    begins = [[torch.cuda.Event(enable_timing=True) for _ in range(steps)] for _ in ctx]
-    ends = [[torch.cuda.Event(enable_timing=True) for _ in range(steps)] for _ in ctx]
+    # Seven host threads, one per stream; each runs its launch loop inside the library
+    # (preba_preprocess_repeated: every launch bracketed by events), so the threads do not
+    # queue for the interpreter lock.
+    gate = threading.Barrier(n_streams)
+    lat = [None] * n_streams
+    span = [None] * n_streams
+    errors = []
+
+    def server(sidx):
+        try:
+            call = ctx[sidx]["call"]
+            call.repeated(warm)
+            gate.wait()
+            lat[sidx], span[sidx] = call.repeated(steps)
+        except Exception as exc:  # surfaced after the join
+            errors.append(exc)
+            gate.abort()
+
     with ClockSampler(local_rank) as clocks:
-        for i in range(steps):
-            for sidx, c in enumerate(ctx):
-                begins[sidx][i].record(c["stream"])
-                c["call"]()
-                ends[sidx][i].record(c["stream"])
-        torch.cuda.synchronize()
-    lat = [np.array([b.elapsed_time(e) * 1e3 for b, e in zip(bs, es)])
-           for bs, es in zip(begins, ends)]
-    # the job runs from the first stream's first batch to the last batch to finish
-    span = [begins[0][0].elapsed_time(es[-1]) for es in ends]
+        threads = [threading.Thread(target=server, args=(i,)) for i in range(n_streams)]
+        for t in threads:
+            t.start()
+        for t in threads:
+            t.join()
+    if errors:
+        raise errors[0]
     torch.cuda.synchronize()
     same = all(int(c["status"].item()) == 0 and bool(torch.equal(c["out"], c["alone"])) for c in ctx)
     assert same, "concurrent streams changed the result"
@@ -275,7 +281,7 @@ def run_streams(args, local_rank: int) -> None:
         "data": "synthetic",
         "config": dict(config_of(f"{n_streams} concurrent streams x {n} images 500x375, smooth "
                                  "noise, fp16 out", "f16", n, 1),
-                       launch="one host thread feeding 7 streams in turn, no flags",
+                       launch="7 host threads, one stream each, launch loops inside the library",
                        l2="inputs and outputs of all streams stay resident (warm L2)"),
         "streams": {"count": n_streams,
                     "batch_latency_us": {"p50": float(np.percentile(all_lat, 50)),

@@ -218,6 +218,23 @@ int preba_preprocess_host_noalloc(const uint8_t* packed_host, uint64_t packed_by
                                   int out_dtype, void* stream);
 
 /*
+ * preba_preprocess_repeated — a measuring aid for serving-style loops (the paper's several
+ * small inference servers sharing one GPU, Sec. 3): launches the same device-resident batch
+ * `iterations` times on `stream`, one kernel each, every launch bracketed by a pair of
+ * events, then waits for the stream and writes each launch's device time.  Unlike the other
+ * entry points it creates (and destroys) CUDA events and synchronises the stream; several
+ * host threads may run it at once on streams of their own.
+ *   latency_us   HOST, `iterations` floats (microseconds per launch), or NULL
+ *   span_ms      HOST float or NULL: device time from the first launch's start to the last
+ *                launch's end
+ * Errors: as preba_preprocess.
+ */
+int preba_preprocess_repeated(const preba_batch_t* batch, uint32_t out_size,
+                              uint32_t resize_short, const float mean[3], const float std[3],
+                              int out_dtype, void* stream, uint32_t iterations,
+                              float* latency_us, float* span_ms);
+
+/*
  * Batching front-end (host only) — the stage between preprocessing and model execution
  * (paper Sec. 2.3 item 2): single-input requests wait in arrival order and leave as a batch
  * when Batch_max of them are queued or when the oldest has waited Time_queue.  The paper's

@@ -28,7 +28,8 @@ ERR_TOO_LARGE = -6
 NOALLOC_MAX_BYTES = 64 << 20
 
 EXPORTS = ("preba_query", "preba_pack", "preba_preprocess", "preba_preprocess_host",
-           "preba_preprocess_host_noalloc", "preba_strerror", "preba_last_cuda_error",
+           "preba_preprocess_host_noalloc", "preba_preprocess_repeated", "preba_strerror",
+           "preba_last_cuda_error",
            "preba_batching_params", "preba_batcher_create", "preba_batcher_destroy",
            "preba_batcher_push", "preba_batcher_poll")
 
@@ -94,6 +95,10 @@ def lib() -> ctypes.CDLL:
         L.preba_preprocess_host.argtypes = [ctypes.POINTER(PrebaHostBatch), ctypes.c_uint32,
                                             ctypes.c_uint32, f32p, f32p, ctypes.c_int,
                                             ctypes.c_void_p]
+        L.preba_preprocess_repeated.argtypes = [ctypes.POINTER(PrebaBatch), ctypes.c_uint32,
+                                                ctypes.c_uint32, f32p, f32p, ctypes.c_int,
+                                                ctypes.c_void_p, ctypes.c_uint32, f32p, f32p]
+        L.preba_preprocess_repeated.restype = ctypes.c_int
         L.preba_preprocess_host_noalloc.argtypes = [
             ctypes.c_void_p, ctypes.c_uint64, ctypes.c_void_p, ctypes.c_uint32, ctypes.c_void_p,
             ctypes.c_uint64, ctypes.c_void_p, ctypes.c_uint32, ctypes.c_uint32, f32p, f32p,
@@ -253,6 +258,17 @@ class PreparedPreprocess:
         rc = self._fn(*self._args)
         if rc != OK:
             raise PrebaError(rc, "preba_preprocess")
+
+    def repeated(self, iterations: int) -> tuple[np.ndarray, float]:
+        """``preba_preprocess_repeated``: (device time of every launch in us, span in ms).
+        Blocks until the stream is done; the interpreter lock is released meanwhile."""
+        lat = np.zeros(iterations, dtype=np.float32)
+        span = ctypes.c_float()
+        rc = lib().preba_preprocess_repeated(*self._args, iterations, _p(lat, ctypes.c_float),
+                                             ctypes.byref(span))
+        if rc != OK:
+            raise PrebaError(rc, "preba_preprocess_repeated")
+        return lat, span.value
 
 
 def preba_preprocess_host(packed_host, table_host: np.ndarray, n: int, out_host, dev_pixels,

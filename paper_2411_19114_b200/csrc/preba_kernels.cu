@@ -17,6 +17,7 @@
 
 #include <atomic>
 #include <cmath>
+#include <vector>
 
 #include "preba.h"
 #include "preba_internal.h"
@@ -854,6 +855,59 @@ extern "C" int preba_preprocess_host(const preba_host_batch_t* b, uint32_t out_s
   rc = launch(p, out_dtype, false, s);
   if (rc != PREBA_OK) return rc;
   err = cudaMemcpyAsync(b->out_host, b->dev_out, need, cudaMemcpyDeviceToHost, s);
+  if (err != cudaSuccess) {
+    g_last_cuda_error = static_cast<int>(err);
+    return PREBA_ERR_CUDA;
+  }
+  return PREBA_OK;
+}
+
+extern "C" int preba_preprocess_repeated(const preba_batch_t* batch, uint32_t out_size,
+                                         uint32_t resize_short, const float mean[3],
+                                         const float std[3], int out_dtype, void* stream,
+                                         uint32_t iterations, float* latency_us,
+                                         float* span_ms) {
+  using namespace preba;
+  if (!batch || iterations == 0) return PREBA_ERR_INVALID_ARG;
+  int rc = check_args(batch->pixels, batch->pixels_bytes, batch->table, batch->n, batch->out,
+                      batch->out_bytes, out_size, resize_short, mean, std, out_dtype);
+  if (rc != PREBA_OK) return rc;
+  if (reinterpret_cast<uintptr_t>(batch->scratch) % 16) return PREBA_ERR_INVALID_ARG;
+  if (batch->flags & ~PREBA_OVERLAP_PREVIOUS) return PREBA_ERR_INVALID_ARG;
+  if (batch->table_host) {
+    rc = check_table(batch->table_host, batch->n, batch->pixels_bytes);
+    if (rc != PREBA_OK) return rc;
+  }
+  const Params p = make_params(batch->pixels, batch->pixels_bytes, batch->table, batch->n,
+                               batch->out, batch->status, batch->scratch, out_size, resize_short,
+                               mean, std);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const bool overlap = (batch->flags & PREBA_OVERLAP_PREVIOUS) != 0;
+  std::vector<cudaEvent_t> ev(2 * static_cast<size_t>(iterations), nullptr);
+  cudaError_t err = cudaSuccess;
+  for (auto& e : ev) {
+    err = cudaEventCreate(&e);
+    if (err != cudaSuccess) break;
+  }
+  rc = PREBA_OK;
+  for (uint32_t i = 0; i < iterations && err == cudaSuccess && rc == PREBA_OK; ++i) {
+    err = cudaEventRecord(ev[2 * i], s);
+    if (err == cudaSuccess) rc = launch(p, out_dtype, overlap, s);
+    if (err == cudaSuccess && rc == PREBA_OK) err = cudaEventRecord(ev[2 * i + 1], s);
+  }
+  if (err == cudaSuccess) err = cudaStreamSynchronize(s);
+  if (err == cudaSuccess && rc == PREBA_OK) {
+    for (uint32_t i = 0; i < iterations && latency_us && err == cudaSuccess; ++i) {
+      float ms = 0.f;
+      err = cudaEventElapsedTime(&ms, ev[2 * i], ev[2 * i + 1]);
+      latency_us[i] = ms * 1000.0f;
+    }
+    if (span_ms && err == cudaSuccess)
+      err = cudaEventElapsedTime(span_ms, ev[0], ev[2 * static_cast<size_t>(iterations) - 1]);
+  }
+  for (auto& e : ev)
+    if (e) cudaEventDestroy(e);
+  if (rc != PREBA_OK) return rc;
   if (err != cudaSuccess) {
     g_last_cuda_error = static_cast<int>(err);
     return PREBA_ERR_CUDA;

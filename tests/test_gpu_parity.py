@@ -249,6 +249,27 @@ def test_overlapping_launches_into_buffers_of_their_own(dynamic):
             assert int(sc.abs().sum().item()) == 0
 
 
+def test_repeated_launch_aid_gives_the_same_result_and_times_every_launch():
+    import torch
+
+    imgs = wl.server_batch_500x375(0, 8)
+    packed, table = pb.preba_pack(imgs)
+    dev = torch.device("cuda:0")
+    pix = torch.from_numpy(packed).to(dev)
+    tab = torch.from_numpy(table.view(np.uint8)).to(dev)
+    out = torch.zeros((8, 3, 224, 224), dtype=torch.float16, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    st = torch.cuda.Stream()
+    call = pb.PreparedPreprocess(pix, tab, 8, out, 224, 256, MEAN, STD, pb.F16, stream=st,
+                                 status=status)
+    lat, span_ms = call.repeated(25)
+    assert int(status.item()) == 0
+    assert lat.shape == (25,) and np.all(lat > 0) and np.all(lat < 1e5)
+    assert span_ms * 1e3 >= lat.max()
+    want = run_gpu(imgs, 224, 256, out_dtype=pb.F16)
+    assert np.array_equal(out.cpu().numpy().view(np.uint16), want.view(np.uint16))
+
+
 def test_device_side_table_check_skips_bad_entries():
     import torch
 
