@@ -54,7 +54,7 @@ extern "C" {
 /* Device memory the library itself carries for preba_preprocess_host_noalloc (64 MiB). */
 #define PREBA_NOALLOC_MAX_BYTES (64u << 20)
 
-typedef enum { PREBA_F32 = 0, PREBA_F16 = 1 } preba_dtype_t;
+typedef enum { PREBA_F32 = 0, PREBA_F16 = 1, PREBA_BF16 = 2 } preba_dtype_t;
 
 /* One image of the packed batch: `offset` is in bytes from the start of the
  * pixel buffer and a multiple of PREBA_PACK_ALIGN; the image is h rows of w
@@ -118,7 +118,7 @@ typedef struct {
  * up to PREBA_PACK_ALIGN, and the total is rounded up as well.
  *   h, w      HOST, n entries each, every value in [1, PREBA_MAX_DIM]
  *   out_size  side of the square crop, >= 1
- *   out_dtype PREBA_F32 or PREBA_F16
+ *   out_dtype PREBA_F32, PREBA_F16 or PREBA_BF16
  *   sizes     HOST, written on success
  * Errors: PREBA_ERR_INVALID_ARG.
  */
@@ -147,7 +147,7 @@ int preba_pack(const uint8_t* const* images, const uint32_t* h, const uint32_t* 
  *   resize_short  target length S of the shorter side, <= PREBA_MAX_RESIZE;
  *                 the longer side becomes floor(S*long/short)
  *   mean, std     HOST, 3 floats each, copied at call time; std finite, non-zero
- *   out_dtype     PREBA_F32 or PREBA_F16 (round to nearest even)
+ *   out_dtype     PREBA_F32, PREBA_F16 or PREBA_BF16 (one rounding to nearest even)
  *   stream        a cudaStream_t (NULL = the default stream)
  * Per image: crop origin floor((R - C)/2) on each axis; output index j samples
  * source coordinate ((j + origin) + 1/2) * in/R - 1/2, clamped to [0, in-1];

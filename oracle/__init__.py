@@ -21,7 +21,7 @@ _SRC = _HERE / "preba_oracle.c"
 _LIB = _HERE / "liboracle.so"
 
 PACK_ALIGN = 128
-OUT_F64, OUT_F32, OUT_F16 = 0, 1, 2
+OUT_F64, OUT_F32, OUT_F16, OUT_BF16 = 0, 1, 2, 3
 
 _lib = None
 
@@ -57,6 +57,8 @@ def _load():
                                        ctypes.c_uint32, ctypes.c_uint32, f64p]
         lib.oracle_round_f16.argtypes = [ctypes.c_double]
         lib.oracle_round_f16.restype = ctypes.c_uint16
+        lib.oracle_round_bf16.argtypes = [ctypes.c_double]
+        lib.oracle_round_bf16.restype = ctypes.c_uint16
         lib.oracle_pack_size.argtypes = [u32p, u32p, ctypes.c_uint32, u64p]
         lib.oracle_pack.argtypes = [ctypes.POINTER(u8p), u32p, u32p, ctypes.c_uint32, u8p,
                                     ctypes.c_uint64, u64p]
@@ -116,6 +118,11 @@ def round_f16_bits(x: float) -> int:
     return int(_load().oracle_round_f16(float(x)))
 
 
+def round_bf16_bits(x: float) -> int:
+    """bfloat16 bit pattern of x rounded once, ties to even."""
+    return int(_load().oracle_round_bf16(float(x)))
+
+
 def pack(images: list[np.ndarray]) -> tuple[np.ndarray, np.ndarray, np.ndarray, np.ndarray]:
     """Packed byte buffer, offsets (uint64), h, w (uint32) of a list of HWC uint8 images."""
     imgs = [np.ascontiguousarray(im, dtype=np.uint8) for im in images]
@@ -139,13 +146,14 @@ def pack(images: list[np.ndarray]) -> tuple[np.ndarray, np.ndarray, np.ndarray, 
 def preprocess_packed(packed: np.ndarray, offsets: np.ndarray, h: np.ndarray, w: np.ndarray,
                       c: int, s: int, mean, std, out_kind: int = OUT_F64,
                       nthreads: int = 1) -> np.ndarray:
-    """[n,3,c,c] result for a packed batch; float64, float32 or float16 (one rounding)."""
+    """[n,3,c,c] result for a packed batch; float64, float32, float16, or bfloat16 as uint16
+    bit patterns (one rounding each)."""
     packed = np.ascontiguousarray(packed, dtype=np.uint8)
     offsets = np.ascontiguousarray(offsets, dtype=np.uint64)
     h = np.ascontiguousarray(h, dtype=np.uint32)
     w = np.ascontiguousarray(w, dtype=np.uint32)
     n = len(h)
-    dt = {OUT_F64: np.float64, OUT_F32: np.float32, OUT_F16: np.uint16}[out_kind]
+    dt = {OUT_F64: np.float64, OUT_F32: np.float32, OUT_F16: np.uint16, OUT_BF16: np.uint16}[out_kind]
     out = np.empty((n, 3, c, c), dtype=dt)
     m, sd = _f3(mean), _f3(std)
     _check(_load().oracle_preprocess(_ptr(packed, ctypes.c_uint8), _ptr(offsets, ctypes.c_uint64),

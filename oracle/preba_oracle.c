@@ -136,6 +136,35 @@ uint16_t oracle_round_f16(double x) {
   return (uint16_t)(sign | bits);
 }
 
+/* Round a double once to bfloat16 (1 sign, 8 exponent bits with bias 127, 7 fraction bits),
+ * ties to even; returns the bit pattern.  Subnormals are multiples of 2^-133; values that
+ * round to 2^128 or more overflow to infinity. */
+uint16_t oracle_round_bf16(double x) {
+  const uint16_t sign = signbit(x) ? 0x8000u : 0u;
+  if (isnan(x)) return (uint16_t)(sign | 0x7fc0u);
+  double a = fabs(x);
+  if (isinf(a)) return (uint16_t)(sign | 0x7f80u);
+  if (a == 0.0) return sign;
+  int e;
+  (void)frexp(a, &e);
+  int exp2 = e - 1;
+  if (exp2 < -126) exp2 = -126;
+  const double q = ldexp(a, 7 - exp2); /* a in units of the spacing 2^(exp2-7); exact */
+  uint64_t units = (uint64_t)nearbyint(q);
+  uint32_t bits;
+  if (exp2 == -126 && units < 128) {
+    bits = (uint32_t)units;
+  } else {
+    if (units == 256) {
+      units = 128;
+      exp2 += 1;
+    }
+    if (exp2 > 127) return (uint16_t)(sign | 0x7f80u);
+    bits = ((uint32_t)(exp2 + 127) << 7) | (uint32_t)(units - 128);
+  }
+  return (uint16_t)(sign | bits);
+}
+
 /* Packing (step 0 of the path; defined by the problem statement, not by the
  * paper): images are concatenated, each starting at the running byte count
  * rounded up to ORACLE_PACK_ALIGN; the total is rounded up too. */
@@ -172,7 +201,8 @@ int oracle_pack(const uint8_t* const* images, const uint32_t* h, const uint32_t*
 }
 
 /* The whole batch: out is [n][3][c][c].  out_kind 0: double, 1: float (one
- * rounding from double), 2: binary16 bit patterns (one rounding from double). */
+ * rounding from double), 2: binary16 bit patterns, 3: bfloat16 bit patterns (one
+ * rounding from double each). */
 typedef struct {
   const uint8_t* packed;
   const uint64_t* offsets;
@@ -190,7 +220,8 @@ typedef struct {
 static void oracle_store(void* out, int kind, size_t idx, double v) {
   if (kind == 0) ((double*)out)[idx] = v;
   else if (kind == 1) ((float*)out)[idx] = (float)v;
-  else ((uint16_t*)out)[idx] = oracle_round_f16(v);
+  else if (kind == 2) ((uint16_t*)out)[idx] = oracle_round_f16(v);
+  else ((uint16_t*)out)[idx] = oracle_round_bf16(v);
 }
 
 static void* oracle_worker(void* arg) {
@@ -220,7 +251,7 @@ int oracle_preprocess(const uint8_t* packed, const uint64_t* offsets, const uint
                       uint32_t nthreads) {
   if (!packed || !offsets || !h || !w || !mean || !std || !out || n == 0 || c == 0 || s < c)
     return ORACLE_ERR_ARG;
-  if (out_kind < 0 || out_kind > 2) return ORACLE_ERR_ARG;
+  if (out_kind < 0 || out_kind > 3) return ORACLE_ERR_ARG;
   for (int ch = 0; ch < 3; ++ch)
     if (!(std[ch] != 0.0f) || !isfinite(std[ch]) || !isfinite(mean[ch])) return ORACLE_ERR_ARG;
   for (uint32_t i = 0; i < n; ++i) {

@@ -16,7 +16,7 @@ _LIB_PATH = Path(__file__).resolve().parent / "libpreba.so"
 PACK_ALIGN = 128
 SCRATCH_BYTES = 256
 OVERLAP_PREVIOUS = 1
-F32, F16 = 0, 1
+F32, F16, BF16 = 0, 1, 2
 
 OK = 0
 ERR_INVALID_ARG = -1

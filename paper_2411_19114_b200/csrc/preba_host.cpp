@@ -9,7 +9,11 @@
 
 namespace preba {
 
-bool dtype_ok(int out_dtype) { return out_dtype == PREBA_F32 || out_dtype == PREBA_F16; }
+bool dtype_ok(int out_dtype) {
+  return out_dtype == PREBA_F32 || out_dtype == PREBA_F16 || out_dtype == PREBA_BF16;
+}
+
+uint32_t dtype_bytes(int out_dtype) { return out_dtype == PREBA_F32 ? 4u : 2u; }
 
 uint64_t align_up(uint64_t v, uint64_t a) { return (v + a - 1) / a * a; }
 
@@ -32,7 +36,7 @@ extern "C" int preba_query(const uint32_t* h, const uint32_t* w, uint32_t n, uin
   sizes->packed_bytes = at;
   sizes->table_bytes = static_cast<uint64_t>(n) * sizeof(preba_img_t);
   sizes->out_bytes = static_cast<uint64_t>(n) * 3ull * out_size * out_size *
-                     (out_dtype == PREBA_F16 ? 2u : 4u);
+                     preba::dtype_bytes(out_dtype);
   sizes->align = PREBA_PACK_ALIGN;
   sizes->reserved = 0;
   return PREBA_OK;

@@ -9,6 +9,7 @@
 namespace preba {
 
 bool dtype_ok(int out_dtype);
+uint32_t dtype_bytes(int out_dtype);  // size of one output element
 bool dims_ok(uint32_t h, uint32_t w);
 uint64_t align_up(uint64_t v, uint64_t a);
 

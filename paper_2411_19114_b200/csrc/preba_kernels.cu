@@ -12,6 +12,7 @@
 // planar output.  The copy stream runs ahead across task boundaries, so a warp's next task
 // is already arriving while it finishes the current one.  Nothing but the input bytes and
 // the output tensor touches device memory; warps never wait for one another.
+#include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
@@ -268,6 +269,14 @@ struct Pack<float> {
   using Vec = float2;
   static __device__ __forceinline__ Vec pair(float x, float y) { return make_float2(x, y); }
   static __device__ __forceinline__ float one(float x) { return x; }
+};
+template <>
+struct Pack<__nv_bfloat16> {
+  using Vec = __nv_bfloat162;
+  static __device__ __forceinline__ Vec pair(float x, float y) {
+    return __floats2bfloat162_rn(x, y);
+  }
+  static __device__ __forceinline__ __nv_bfloat16 one(float x) { return __float2bfloat16_rn(x); }
 };
 template <>
 struct Pack<__half> {
@@ -703,7 +712,7 @@ int check_args(const uint8_t* pixels, uint64_t pixels_bytes, const void* table, 
       reinterpret_cast<uintptr_t>(table) % 8)
     return PREBA_ERR_INVALID_ARG;
   const uint64_t need = static_cast<uint64_t>(n) * 3ull * out_size * out_size *
-                        (out_dtype == PREBA_F16 ? 2u : 4u);
+                        dtype_bytes(out_dtype);
   if (out_bytes < need) return PREBA_ERR_BUFFER_TOO_SMALL;
   if (pixels_bytes == 0) return PREBA_ERR_BUFFER_TOO_SMALL;
   const uint64_t tasks = static_cast<uint64_t>(n) * ((out_size + kSlabRows - 1) / kSlabRows) *
@@ -727,11 +736,11 @@ int check_table(const preba_img_t* t, uint32_t n, uint64_t pixels_bytes) {
 // output type and kept (a benign race: concurrent first calls store the same value).
 int resident_ctas(int out_dtype, cudaError_t* err) {
   constexpr int kMaxDevices = 64;
-  static std::atomic<int> cache[2][kMaxDevices];
+  static std::atomic<int> cache[3][kMaxDevices];
   int dev = 0;
   *err = cudaGetDevice(&dev);
   if (*err != cudaSuccess) return 0;
-  const int kind = out_dtype == PREBA_F16 ? 1 : 0;
+  const int kind = out_dtype == PREBA_F16 ? 1 : out_dtype == PREBA_BF16 ? 2 : 0;
   if (dev >= 0 && dev < kMaxDevices) {
     const int known = cache[kind][dev].load(std::memory_order_relaxed);
     if (known > 0) return known;
@@ -742,6 +751,9 @@ int resident_ctas(int out_dtype, cudaError_t* err) {
   if (kind == 1)
     *err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, preba_fused_kernel<__half>,
                                                          kThreads, 0);
+  else if (kind == 2)
+    *err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(
+        &per_sm, preba_fused_kernel<__nv_bfloat16>, kThreads, 0);
   else
     *err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, preba_fused_kernel<float>,
                                                          kThreads, 0);
@@ -769,6 +781,8 @@ int launch(const Params& p, int out_dtype, bool overlap, cudaStream_t stream) {
     cfg.numAttrs = overlap ? 1 : 0;
     if (out_dtype == PREBA_F16)
       err = cudaLaunchKernelEx(&cfg, preba_fused_kernel<__half>, p);
+    else if (out_dtype == PREBA_BF16)
+      err = cudaLaunchKernelEx(&cfg, preba_fused_kernel<__nv_bfloat16>, p);
     else
       err = cudaLaunchKernelEx(&cfg, preba_fused_kernel<float>, p);
   }
@@ -840,7 +854,7 @@ extern "C" int preba_preprocess_host(const preba_host_batch_t* b, uint32_t out_s
   if (rc != PREBA_OK) return rc;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const uint64_t need = static_cast<uint64_t>(b->n) * 3ull * out_size * out_size *
-                        (out_dtype == PREBA_F16 ? 2u : 4u);
+                        dtype_bytes(out_dtype);
   cudaError_t err = cudaMemcpyAsync(b->dev_pixels, b->packed_host, b->packed_bytes,
                                     cudaMemcpyHostToDevice, s);
   if (err == cudaSuccess)
@@ -970,7 +984,7 @@ extern "C" int preba_preprocess_host_noalloc(const uint8_t* packed_host, uint64_
   rc = check_table(table_host, n, packed_bytes);
   if (rc != PREBA_OK) return rc;
   const uint64_t need_out = static_cast<uint64_t>(n) * 3ull * out_size * out_size *
-                            (out_dtype == PREBA_F16 ? 2u : 4u);
+                            dtype_bytes(out_dtype);
   const uint64_t table_bytes = static_cast<uint64_t>(n) * sizeof(preba_img_t);
   const uint64_t at_table = kNoallocHeader;
   const uint64_t at_pixels = at_table + align_up(table_bytes, 256);

@@ -29,7 +29,7 @@ def run_gpu(images, c, s, mean=MEAN, std=STD, out_dtype=pb.F32, stream=None,
     n = len(images)
     packed, table = pb.preba_pack(images)
     nb = packed.nbytes
-    itemsize = 2 if out_dtype == pb.F16 else 4
+    itemsize = 4 if out_dtype == pb.F32 else 2
     ob = n * 3 * c * c * itemsize
     dev = torch.device("cuda:0")
     pix_buf = torch.full((GUARD + nb + GUARD,), CANARY, dtype=torch.uint8, device=dev)
@@ -56,8 +56,8 @@ def run_gpu(images, c, s, mean=MEAN, std=STD, out_dtype=pb.F32, stream=None,
     assert np.all(pb_host[:GUARD] == CANARY) and np.all(pb_host[GUARD + nb:] == CANARY)
     assert np.array_equal(pb_host[GUARD:GUARD + nb], packed), "kernel modified its input"
     res = ob_host[GUARD:GUARD + ob].copy()
-    res = res.view(np.float16 if out_dtype == pb.F16 else np.float32).reshape(n, 3, c, c)
-    return res
+    view = {pb.F32: np.float32, pb.F16: np.float16, pb.BF16: np.uint16}[out_dtype]
+    return res.view(view).reshape(n, 3, c, c)  # bfloat16 comes back as bit patterns
 
 
 def oracle_f64(images, c, s, mean=MEAN, std=STD):
@@ -86,8 +86,30 @@ def fp16_report(gpu_h: np.ndarray, want64: np.ndarray) -> dict:
                 max_abs_err=float(abs_err.max()))
 
 
+def bf16_bits_to_float(bits: np.ndarray) -> np.ndarray:
+    return (bits.astype(np.uint32) << 16).view(np.float32)
+
+
+def bf16_report(gpu_bits: np.ndarray, want64: np.ndarray) -> dict:
+    """The fp16 criterion carried over to bfloat16: within one bfloat16 ulp of the double
+    result rounded once (by the oracle's own rounding routine), or within FP16_ABS of it."""
+    flat = want64.reshape(-1)
+    want_bits = np.fromiter((oracle.round_bf16_bits(v) for v in flat), dtype=np.uint16,
+                            count=flat.size).reshape(want64.shape)
+    ulps = np.abs(_ordered(gpu_bits) - _ordered(want_bits))
+    abs_err = np.abs(bf16_bits_to_float(gpu_bits).astype(np.float64) - want64)
+    strict = ulps <= 1
+    ok = strict | (abs_err <= FP16_ABS)
+    return dict(failures=int((~ok).sum()), needed_abs_clause=int((~strict & ok).sum()),
+                max_ulps=int(ulps.max()), exact=int((ulps == 0).sum()), total=int(ulps.size))
+
+
 def assert_parity(gpu: np.ndarray, want64: np.ndarray, out_dtype: int) -> dict:
     assert gpu.shape == want64.shape
+    if out_dtype == pb.BF16:
+        rep = bf16_report(gpu, want64)
+        assert rep["failures"] == 0, rep
+        return rep
     if out_dtype == pb.F32:
         err = float(np.max(np.abs(gpu.astype(np.float64) - want64)))
         assert err <= FP32_TOL, f"fp32 max abs error {err:.3e} > {FP32_TOL}"

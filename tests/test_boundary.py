@@ -56,13 +56,14 @@ def test_query_sizes():
     assert s.table_bytes == 16 * 4
     assert s.out_bytes == 4 * 3 * 224 * 224 * 2
     assert pb.preba_query(h, w, 224, pb.F32).out_bytes == 4 * 3 * 224 * 224 * 4
+    assert pb.preba_query(h, w, 224, pb.BF16).out_bytes == 4 * 3 * 224 * 224 * 2
     # largest accepted image: no overflow
     s = pb.preba_query([32768, 32768], [32768, 32768], 1, pb.F32)
     assert s.packed_bytes == 2 * 3 * 32768 * 32768
 
 
 @pytest.mark.parametrize("h,w,c,dt", [([0], [5], 8, 0), ([5], [0], 8, 0), ([32769], [5], 8, 0),
-                                      ([5], [5], 0, 0), ([5], [5], 8, 2), ([5], [5], 8, -1),
+                                      ([5], [5], 0, 0), ([5], [5], 8, 3), ([5], [5], 8, -1),
                                       ([], [], 8, 0)])
 def test_query_rejects(h, w, c, dt):
     with pytest.raises(pb.PrebaError) as e:
@@ -149,7 +150,7 @@ def test_preprocess_rejects_bad_arguments_before_any_launch():
     assert _call(_batch(), c=0) == pb.ERR_INVALID_ARG
     assert _call(_batch(), c=17, s=16) == pb.ERR_INVALID_ARG        # crop larger than resize
     assert _call(_batch(), s=16385) == pb.ERR_INVALID_ARG
-    assert _call(_batch(), dt=2) == pb.ERR_INVALID_ARG
+    assert _call(_batch(), dt=3) == pb.ERR_INVALID_ARG
     assert _call(_batch(), std=(0.2, 0.0, 0.2)) == pb.ERR_INVALID_ARG
     assert _call(_batch(), std=(0.2, float("inf"), 0.2)) == pb.ERR_INVALID_ARG
     assert _call(_batch(), mean=(float("nan"), 0.1, 0.2)) == pb.ERR_INVALID_ARG

@@ -57,6 +57,14 @@ def test_ragged_batch_with_odd_strides(dt, dynamic):
     assert_parity(got, oracle_f64(imgs, 224, 256), dt)
 
 
+def test_bfloat16_output():
+    sizes = [(240, 320), (375, 500), (333, 471), (1080, 1920), (17, 29)]
+    imgs = [uniform(450 + i, h, w) for i, (h, w) in enumerate(sizes)]
+    got = run_gpu(imgs, 224, 256, out_dtype=pb.BF16)
+    rep = assert_parity(got, oracle_f64(imgs, 224, 256), pb.BF16)
+    assert rep["exact"] > 0.99 * rep["total"]
+
+
 def test_other_normalisation_constants_and_constant_images():
     imgs = [np.full((260, 300, 3), v, dtype=np.uint8) for v in (0, 1, 128, 255)]
     mean, std = (0.1, 0.5, 0.9), (1.0, 0.05, 2.5)

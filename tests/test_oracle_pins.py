@@ -316,6 +316,27 @@ def test_round_to_binary16_matches_two_other_implementations():
         assert got == _half_bits_struct(v), v
 
 
+def test_round_to_bfloat16():
+    torch = pytest.importorskip("torch")
+    # hand cases: 1 + 2^-8 is halfway between 1 and 1 + 2^-7 -> even (1.0); 1 + 3*2^-8 -> 1 + 2^-6
+    assert oracle.round_bf16_bits(1.0) == 0x3F80
+    assert oracle.round_bf16_bits(1.0 + 2.0 ** -8) == 0x3F80
+    assert oracle.round_bf16_bits(np.nextafter(1.0 + 2.0 ** -8, 2.0)) == 0x3F81
+    assert oracle.round_bf16_bits(1.0 + 3 * 2.0 ** -8) == 0x3F82
+    assert oracle.round_bf16_bits(-2.5) == 0xC020
+    assert oracle.round_bf16_bits(0.0) == 0 and oracle.round_bf16_bits(-0.0) == 0x8000
+    assert oracle.round_bf16_bits(3.5e38) == 0x7F80           # beyond the largest finite value
+    assert oracle.round_bf16_bits(2.0 ** -133) == 0x0001       # smallest subnormal
+    assert oracle.round_bf16_bits(2.0 ** -134) == 0x0000       # half of it: tie to even (zero)
+    # a library's conversion on values that are exact in float32 (so no second rounding)
+    rng = np.random.default_rng(20)
+    vals = np.concatenate([rng.uniform(-3, 3, 3000), rng.normal(size=1000) * 1e-3,
+                           rng.uniform(-1e30, 1e30, 200)]).astype(np.float32)
+    want = torch.from_numpy(vals).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    got = np.array([oracle.round_bf16_bits(float(v)) for v in vals], dtype=np.uint16)
+    assert np.array_equal(got, want)
+
+
 def test_output_kinds_are_single_roundings():
     rng = np.random.default_rng(19)
     imgs = [rng.integers(0, 256, size=(20, 27, 3), dtype=np.uint8) for _ in range(3)]
@@ -324,6 +345,9 @@ def test_output_kinds_are_single_roundings():
     f16 = oracle.preprocess(imgs, 12, 14, MEAN, STD, oracle.OUT_F16, nthreads=3)
     assert f32.dtype == np.float32 and np.array_equal(f32, f64.astype(np.float32))
     assert f16.dtype == np.float16 and np.array_equal(f16, f64.astype(np.float16))
+    bf = oracle.preprocess(imgs, 12, 14, MEAN, STD, oracle.OUT_BF16)
+    assert bf.dtype == np.uint16
+    assert all(int(b) == oracle.round_bf16_bits(float(v)) for b, v in zip(bf.ravel(), f64.ravel()))
 
 
 def test_rejects_bad_arguments():
