@@ -235,6 +235,17 @@ int preba_preprocess_repeated(const preba_batch_t* batch, uint32_t out_size,
                               float* latency_us, float* span_ms);
 
 /*
+ * preba_selftest_wait_limit — exercises the kernel's bounded wait on the device: one warp
+ * waits on a shared-memory barrier that nothing ever completes, gives up after the same poll
+ * limit the transform uses, stores PREBA_ERR_TIMEOUT in `status` and returns normally; the
+ * context stays usable.  (Every wait in the transform's kernel is of this kind, so a copy
+ * that never lands ends in an error status instead of a hang.)
+ *   status   DEVICE word, zeroed by the caller
+ * Enqueues one small kernel on `stream`.  Errors: PREBA_ERR_INVALID_ARG, PREBA_ERR_CUDA.
+ */
+int preba_selftest_wait_limit(int32_t* status, void* stream);
+
+/*
  * Batching front-end (host only) — the stage between preprocessing and model execution
  * (paper Sec. 2.3 item 2): single-input requests wait in arrival order and leave as a batch
  * when Batch_max of them are queued or when the oldest has waited Time_queue.  The paper's

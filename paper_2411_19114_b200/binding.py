@@ -28,7 +28,8 @@ ERR_TOO_LARGE = -6
 NOALLOC_MAX_BYTES = 64 << 20
 
 EXPORTS = ("preba_query", "preba_pack", "preba_preprocess", "preba_preprocess_host",
-           "preba_preprocess_host_noalloc", "preba_preprocess_repeated", "preba_strerror",
+           "preba_preprocess_host_noalloc", "preba_preprocess_repeated", "preba_selftest_wait_limit",
+           "preba_strerror",
            "preba_last_cuda_error",
            "preba_batching_params", "preba_batcher_create", "preba_batcher_destroy",
            "preba_batcher_push", "preba_batcher_poll")
@@ -99,6 +100,8 @@ def lib() -> ctypes.CDLL:
                                                 ctypes.c_uint32, f32p, f32p, ctypes.c_int,
                                                 ctypes.c_void_p, ctypes.c_uint32, f32p, f32p]
         L.preba_preprocess_repeated.restype = ctypes.c_int
+        L.preba_selftest_wait_limit.argtypes = [ctypes.c_void_p, ctypes.c_void_p]
+        L.preba_selftest_wait_limit.restype = ctypes.c_int
         L.preba_preprocess_host_noalloc.argtypes = [
             ctypes.c_void_p, ctypes.c_uint64, ctypes.c_void_p, ctypes.c_uint32, ctypes.c_void_p,
             ctypes.c_uint64, ctypes.c_void_p, ctypes.c_uint32, ctypes.c_uint32, f32p, f32p,
@@ -338,6 +341,19 @@ def preba_preprocess_host_noalloc(packed_host, table_host: np.ndarray, n: int, o
         ctypes.c_void_p(stream))
     if rc != OK:
         raise PrebaError(rc, "preba_preprocess_host_noalloc")
+
+
+def preba_selftest_wait_limit(status, stream=None) -> None:
+    """``status`` is a zeroed CUDA int32 tensor; after the stream has run it holds ERR_TIMEOUT."""
+    import torch
+
+    if stream is None:
+        stream = torch.cuda.current_stream().cuda_stream
+    elif hasattr(stream, "cuda_stream"):
+        stream = stream.cuda_stream
+    rc = lib().preba_selftest_wait_limit(status.data_ptr(), ctypes.c_void_p(stream))
+    if rc != OK:
+        raise PrebaError(rc, "preba_selftest_wait_limit")
 
 
 NEVER = (1 << 64) - 1

@@ -929,6 +929,32 @@ extern "C" int preba_preprocess_repeated(const preba_batch_t* batch, uint32_t ou
   return PREBA_OK;
 }
 
+namespace preba {
+
+// One warp waits on a barrier nobody arrives at: the wait runs out and reports.
+__global__ void __launch_bounds__(32) preba_wait_limit_kernel(int32_t* status) {
+  __shared__ uint64_t never;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_addr(&never), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncwarp();
+  if (!mbar_wait(smem_addr(&never), 0) && threadIdx.x == 0) report(status, PREBA_ERR_TIMEOUT);
+}
+
+}  // namespace preba
+
+extern "C" int preba_selftest_wait_limit(int32_t* status, void* stream) {
+  if (!status) return PREBA_ERR_INVALID_ARG;
+  preba::preba_wait_limit_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(status);
+  const cudaError_t err = cudaGetLastError();
+  if (err != cudaSuccess) {
+    preba::g_last_cuda_error = static_cast<int>(err);
+    return PREBA_ERR_CUDA;
+  }
+  return PREBA_OK;
+}
+
 // ---- host-to-host without any allocation ------------------------------------------------------------
 //
 // Staging space that ships with the library: every GPU that loads it carries this array

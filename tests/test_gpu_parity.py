@@ -278,6 +278,20 @@ def test_repeated_launch_aid_gives_the_same_result_and_times_every_launch():
     assert np.array_equal(out.cpu().numpy().view(np.uint16), want.view(np.uint16))
 
 
+def test_a_wait_that_nothing_completes_runs_out_and_reports():
+    """The bounded wait used throughout the kernel: it gives up, stores the time-out code and
+    returns; the context is still good for real work afterwards."""
+    import torch
+
+    dev = torch.device("cuda:0")
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    pb.preba_selftest_wait_limit(status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == pb.ERR_TIMEOUT
+    img = uniform(900, 64, 80)
+    assert_parity(run_gpu([img], 32, 40, out_dtype=pb.F32), oracle_f64([img], 32, 40), pb.F32)
+
+
 def test_device_side_table_check_skips_bad_entries():
     import torch
 
