@@ -36,8 +36,8 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM bytes (read + write) per launch of the kernel on the default workload, from one
 # ncu capture, valid only for the kernel sources with this digest (else reported as null).
-NCU_TRAFFIC = {"csrc_sha1": "4f53a5be6c2586cfa64784f39ca0018f8ff4e3a2",
-               "bytes_per_launch": 75664640 + 25935872}  # dram read + write, one launch
+NCU_TRAFFIC = {"csrc_sha1": "dbcf26e173d92cec57c0c8caf2c17abdfecc8d74",
+               "bytes_per_launch": 75649536 + 26482688}  # dram read + write, one launch
 
 
 def csrc_digest() -> str:
