@@ -118,6 +118,30 @@ def test_pixel_buffer_without_tail_padding_is_not_read_past_its_end():
     assert_parity(out.cpu().numpy(), oracle_f64([img], 24, 32), pb.F32)
 
 
+@pytest.mark.parametrize("seed", range(4))
+def test_random_shapes_crops_and_constants(seed):
+    """Seeded random batches: image sizes from 1 to 700 on each side, random crop and resize
+    sizes, random normalisation constants, all three output types."""
+    rng = np.random.default_rng(7000 + seed)
+    s_short = int(rng.integers(1, 400))
+    c = int(rng.integers(1, s_short + 1))
+    n = int(rng.integers(1, 12))
+    imgs = [wl.uniform_image(rng, int(rng.integers(1, 701)), int(rng.integers(1, 701)))
+            for _ in range(n)]
+    mean = rng.uniform(0.0, 1.0, size=3).astype(np.float32)
+    std = rng.uniform(0.05, 2.0, size=3).astype(np.float32)
+    want = oracle_f64(imgs, c, s_short, mean, std)
+    for dt in (pb.F32, pb.F16, pb.BF16):
+        got = run_gpu(imgs, c, s_short, mean, std, dt, dynamic=bool(seed & 1))
+        if dt == pb.F32:
+            # the bound scales with the normalising gain 1/(255*std): 1e-5 is stated for the
+            # ImageNet constants (std ~ 0.225); smaller std amplifies the same pixel error
+            tol = 1e-5 * max(1.0, 0.224 / float(std.min()))
+            assert float(np.max(np.abs(got.astype(np.float64) - want))) <= tol
+        else:
+            assert_parity(got, want, dt)
+
+
 # ---- the workloads at full size -------------------------------------------------------------------
 
 def test_workload_uniform_320x240_fp32_full():

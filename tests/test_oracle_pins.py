@@ -158,6 +158,28 @@ def test_matches_exact_fraction_brute_force(seed):
                 assert abs(Fraction(got[ch, k, j]) - want[ch][k][j]) < Fraction(1, 10**12)
 
 
+def test_matches_exact_fraction_on_hypothesis_cases():
+    hyp = pytest.importorskip("hypothesis")
+    st = hyp.strategies
+
+    @hyp.settings(max_examples=60, deadline=None, derandomize=True)
+    @hyp.given(h=st.integers(1, 9), w=st.integers(1, 9), s=st.integers(1, 12), seed=st.integers(0, 10**6),
+               frac=st.floats(0.0, 1.0))
+    def check(h, w, s, seed, frac):
+        rh, rw = xf.resized_size(h, w, s)
+        c = max(1, min(rh, rw, s, int(round(frac * s)) or 1))
+        img = np.random.default_rng(seed).integers(0, 256, size=(h, w, 3), dtype=np.uint8)
+        got = run1(img, c, s)
+        # the constants as the float32 values the interface carries
+        want = xf.preprocess(img.tolist(), c, s, np.float32(MEAN), np.float32(STD))
+        for ch in range(3):
+            for k in range(c):
+                for j in range(c):
+                    assert abs(Fraction(got[ch, k, j]) - want[ch][k][j]) < Fraction(1, 10**12)
+
+    check()
+
+
 def _read_hand_cases():
     planes = {"R": {}, "G": {}, "B": {}}
     cases, expects = {}, []
