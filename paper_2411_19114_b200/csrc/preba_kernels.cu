@@ -137,37 +137,43 @@ __device__ __forceinline__ Axis make_axis(uint32_t in, uint32_t r, uint32_t orig
   return a;
 }
 
-__device__ __forceinline__ Tap axis_tap(const Axis& a, uint32_t j) {
+// The tap when a.small holds: straight-line 32-bit code, so that several taps interleave.
+// The quotient comes from an fp32 estimate (relative error < 2^-21, so off by at most one)
+// and is made exact by the integer remainder.
+__device__ __forceinline__ Tap axis_tap_small(const Axis& a, uint32_t j) {
   Tap t;
-  if (a.small) {
-    // quotient from an fp32 estimate (relative error < 2^-21, so off by at most one),
-    // made exact by the integer remainder
-    const uint32_t pos = (2 * (a.origin + j) + 1) * a.in;
-    uint32_t num = pos > a.r ? pos - a.r : 0;
-    num = min(num, a.hi);
-    uint32_t q = __float2uint_rz(__uint2float_rz(num) * a.rden);
-    int32_t rem = static_cast<int32_t>(num - q * a.den);
-    if (rem < 0) {
-      --q;
-      rem += static_cast<int32_t>(a.den);
-    } else if (rem >= static_cast<int32_t>(a.den)) {
-      ++q;
-      rem -= static_cast<int32_t>(a.den);
-    }
-    t.i0 = q;
-    t.lam = static_cast<float>(rem) * a.rden;
-  } else {
-    const uint64_t den = 2ull * a.r;
-    const uint64_t pos = (2 * (static_cast<uint64_t>(a.origin) + j) + 1) * a.in;  // < 2^46
-    uint64_t num = pos > a.r ? pos - a.r : 0;
-    const uint64_t hi = static_cast<uint64_t>(a.in - 1) * den;
-    num = num < hi ? num : hi;
-    const uint64_t q = num / den;
-    t.i0 = static_cast<uint32_t>(q);
-    t.lam = static_cast<float>(num - q * den) / static_cast<float>(den);
-  }
+  const uint32_t pos = (2 * (a.origin + j) + 1) * a.in;
+  uint32_t num = max(pos, a.r) - a.r;
+  num = min(num, a.hi);
+  uint32_t q = __float2uint_rz(__uint2float_rz(num) * a.rden);
+  int32_t rem = static_cast<int32_t>(num - q * a.den);
+  const int32_t den = static_cast<int32_t>(a.den);
+  const int32_t fix = rem < 0 ? -1 : (rem >= den ? 1 : 0);
+  q += static_cast<uint32_t>(fix);
+  rem -= fix * den;
+  t.i0 = q;
+  t.lam = static_cast<float>(rem) * a.rden;
+  t.i1 = min(q + 1, a.in - 1);
+  return t;
+}
+
+// The tap for any size the interface admits (64-bit numerators).
+__device__ __forceinline__ Tap axis_tap_wide(const Axis& a, uint32_t j) {
+  Tap t;
+  const uint64_t den = 2ull * a.r;
+  const uint64_t pos = (2 * (static_cast<uint64_t>(a.origin) + j) + 1) * a.in;  // < 2^46
+  uint64_t num = pos > a.r ? pos - a.r : 0;
+  const uint64_t hi = static_cast<uint64_t>(a.in - 1) * den;
+  num = num < hi ? num : hi;
+  const uint64_t q = num / den;
+  t.i0 = static_cast<uint32_t>(q);
+  t.lam = static_cast<float>(num - q * den) / static_cast<float>(den);
   t.i1 = t.i0 + 1 < a.in ? t.i0 + 1 : a.in - 1;
   return t;
+}
+
+__device__ __forceinline__ Tap axis_tap(const Axis& a, uint32_t j) {
+  return a.small ? axis_tap_small(a, j) : axis_tap_wide(a, j);
 }
 
 __device__ __forceinline__ void report(int32_t* status, int code) {
@@ -353,22 +359,29 @@ __device__ __forceinline__ uint32_t prepare(const Params& p, uint32_t task, Task
   const preba_img_t e = p.table[img];
   uint32_t kind = kSkip;
   if (entry_ok(e, p.pixels_bytes)) {
-    uint32_t rh, rw;
-    if (e.h <= e.w) {
-      rh = p.S;
-      rw = static_cast<uint32_t>(static_cast<uint64_t>(p.S) * e.w / e.h);
-    } else {
-      rw = p.S;
-      rh = static_cast<uint32_t>(static_cast<uint64_t>(p.S) * e.h / e.w);
-    }
+    // S <= 2^14 and sides <= 2^15: the product fits 32 bits
+    const uint32_t lng = max(e.h, e.w), sht = min(e.h, e.w);
+    const uint32_t rl = p.S * lng / sht;
+    const uint32_t rh = e.h <= e.w ? p.S : rl;
+    const uint32_t rw = e.h <= e.w ? rl : p.S;
     const uint32_t top = (rh - C) / 2, left = (rw - C) / 2;
     const uint32_t k0 = slab * kSlabRows;
     const uint32_t rows_out = min(kSlabRows, C - k0);
     const uint32_t col0 = cb * kTaskCols;
     const uint32_t cols = min(kTaskCols, C - col0);
     const Axis ax = make_axis(e.w, rw, left, C);
-    const Tap tf = axis_tap(ax, col0);
-    const Tap tl = axis_tap(ax, col0 + cols - 1);
+    const Axis ay = make_axis(e.h, rh, top, C);
+    const bool active = lane < rows_out;
+    Tap tf, tl, ty;
+    if (ax.small && ay.small) {
+      tf = axis_tap_small(ax, col0);
+      tl = axis_tap_small(ax, col0 + cols - 1);
+      ty = axis_tap_small(ay, k0 + (active ? lane : 0u));
+    } else {
+      tf = axis_tap(ax, col0);
+      tl = axis_tap(ax, col0 + cols - 1);
+      ty = axis_tap(ay, k0 + (active ? lane : 0u));
+    }
     const uint32_t xmin = tf.i0;
     const uint32_t copy_px = tl.i1 - xmin + 1;
     // a lane reads 12 bytes from the word holding its first tap, which may be the last
@@ -378,37 +391,31 @@ __device__ __forceinline__ uint32_t prepare(const Params& p, uint32_t task, Task
     const uint64_t end16 = (e.offset + 3ull * e.h * e.w + 15) & ~15ull;
     kind = (rpg >= 1 && end16 <= p.pixels_bytes) ? kStream : kGather;
 
-    // rows of the slab: taps, then the ascending list of distinct source rows
-    const bool active = lane < rows_out;
-    const Axis ay = make_axis(e.h, rh, top, C);
-    Tap ty = {0, 0, 0.f};
-    if (active) ty = axis_tap(ay, k0 + lane);
+    // rows of the slab: the ascending list of distinct source rows.  Output row `lane`
+    // lists its lower tap if that lies beyond the previous row's upper tap, and its upper
+    // tap if that is a new row too.
     const uint32_t y1_prev = __shfl_up_sync(0xffffffffu, ty.i1, 1);
     const bool new0 = active && (lane == 0 || ty.i0 > y1_prev);
     const bool new1 = active && ty.i1 != ty.i0 && (lane == 0 || ty.i1 > y1_prev);
-    const uint32_t cnt = (new0 ? 1u : 0u) + (new1 ? 1u : 0u);
-    uint32_t incl = cnt;
-#pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-      const uint32_t v = __shfl_up_sync(0xffffffffu, incl, d);
-      if (lane >= static_cast<uint32_t>(d)) incl += v;
+    const uint32_t b0 = __ballot_sync(0xffffffffu, new0);
+    const uint32_t b1 = __ballot_sync(0xffffffffu, new1);
+    const uint32_t below = (1u << lane) - 1u;
+    const uint32_t excl = static_cast<uint32_t>(__popc(b0 & below) + __popc(b1 & below));
+    const uint32_t n_list = static_cast<uint32_t>(__popc(b0) + __popc(b1));
+    // The last row a lane lists completes this output row and those after it up to the
+    // next lane that lists a row.
+    const uint32_t above = (b0 | b1) & ~((2u << lane) - 1u);
+    const uint32_t done = (above ? static_cast<uint32_t>(__ffs(above) - 1) : rows_out) - lane;
+    if (new0) {
+      m.row[excl] = ty.i0;
+      m.info[excl] = ((new1 ? 0u : done) << 8) | ((3u * (ty.i0 * e.w + xmin)) & 15u);
     }
-    const uint32_t n_list = __shfl_sync(0xffffffffu, incl, 31);
-    const uint32_t excl = incl - cnt;
-    if (new0) m.row[excl] = ty.i0;
-    if (new1) m.row[excl + (new0 ? 1u : 0u)] = ty.i1;
-    m.info[lane] = 0;
-    m.info[lane + 32] = 0;
-    __syncwarp();
-    // the row that completes output row `lane` is the last one listed so far
-    const uint32_t key = active ? incl - 1 : 0x80000000u + lane;
-    const uint32_t peers = __match_any_sync(0xffffffffu, key);
-    if (active && lane == static_cast<uint32_t>(__ffs(peers) - 1))
-      m.info[key] = static_cast<uint32_t>(__popc(peers)) << 8;
+    if (new1) {
+      const uint32_t at = excl + (new0 ? 1u : 0u);
+      m.row[at] = ty.i1;
+      m.info[at] = (done << 8) | ((3u * (ty.i1 * e.w + xmin)) & 15u);
+    }
     if (active) m.lam[lane] = __float_as_uint(ty.lam) | (ty.i1 == ty.i0 ? 0x80000000u : 0u);
-    __syncwarp();
-    for (uint32_t i = lane; i < n_list; i += 32)
-      m.info[i] |= (3u * (m.row[i] * e.w + xmin)) & 15u;
     if (lane == 0) {
       m.img = img;
       m.k0 = k0;
@@ -552,13 +559,24 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
       const uint32_t w = cm->w, rw = cm->rw, col0 = cm->col0, xmin = cm->xmin;
       const Axis ax = make_axis(w, rw, (rw - C) / 2, C);
       ln.valid = 0;
+      if (ax.small) {
 #pragma unroll
-      for (int m = 0; m < static_cast<int>(kLaneCols); ++m) {
-        const uint32_t j = col0 + lane_col(lane, m);
-        if (j < C) ln.valid |= 1u << m;
-        const Tap t = axis_tap(ax, j < C ? j : C - 1);
-        ln.off[m] = 3 * (t.i0 - xmin);
-        ln.lam[m] = t.lam;
+        for (int m = 0; m < static_cast<int>(kLaneCols); ++m) {
+          const uint32_t j = col0 + lane_col(lane, m);
+          if (j < C) ln.valid |= 1u << m;
+          const Tap t = axis_tap_small(ax, min(j, C - 1));
+          ln.off[m] = 3 * (t.i0 - xmin);
+          ln.lam[m] = t.lam;
+        }
+      } else {
+#pragma unroll
+        for (int m = 0; m < static_cast<int>(kLaneCols); ++m) {
+          const uint32_t j = col0 + lane_col(lane, m);
+          if (j < C) ln.valid |= 1u << m;
+          const Tap t = axis_tap_wide(ax, min(j, C - 1));
+          ln.off[m] = 3 * (t.i0 - xmin);
+          ln.lam[m] = t.lam;
+        }
       }
       full = (C & 1u) == 0 && __all_sync(0xffffffffu, ln.valid == 0x7fu);
       q_out = static_cast<OutT*>(p.out) + static_cast<size_t>(cm->img) * 3 * plane +
