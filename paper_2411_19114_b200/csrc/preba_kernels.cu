@@ -109,6 +109,7 @@ struct __align__(16) WarpShared {
 struct Tap {
   uint32_t i0;
   uint32_t i1;
+  uint32_t rem;  // num mod den (filled by the 32-bit path only)
   float lam;
 };
 
@@ -152,6 +153,7 @@ __device__ __forceinline__ Tap axis_tap_small(const Axis& a, uint32_t j) {
   q += static_cast<uint32_t>(fix);
   rem -= fix * den;
   t.i0 = q;
+  t.rem = static_cast<uint32_t>(rem);
   t.lam = static_cast<float>(rem) * a.rden;
   t.i1 = min(q + 1, a.in - 1);
   return t;
@@ -167,6 +169,7 @@ __device__ __forceinline__ Tap axis_tap_wide(const Axis& a, uint32_t j) {
   num = num < hi ? num : hi;
   const uint64_t q = num / den;
   t.i0 = static_cast<uint32_t>(q);
+  t.rem = 0;
   t.lam = static_cast<float>(num - q * den) / static_cast<float>(den);
   t.i1 = t.i0 + 1 < a.in ? t.i0 + 1 : a.in - 1;
   return t;
@@ -247,25 +250,27 @@ __device__ __forceinline__ uint32_t lds32(uint32_t addr) {
 
 // ---- arithmetic ---------------------------------------------------------------------------------
 
-// Byte `idx` of x as 2^23 + byte: the byte dropped into the mantissa of 8388608.0f.
-template <int idx>
-__device__ __forceinline__ float byte_biased(uint32_t x) {
-  return __uint_as_float(__byte_perm(x, 0x4B000000u, 0x7440 + idx));
-}
+// Largest 2 * (resized width) the staged path takes: both weights of a column fit 16 bits
+// and 255 * den stays below 2^23, so a weighted sum fits the mantissa of 8388608.0f.
+constexpr uint32_t kMaxPackedDen = 32768;
 
-// Horizontal interpolation at shared-memory byte address x (pixel x0, then x0 + 1); x is
-// unaligned: three aligned words are read and shifted.
-__device__ __forceinline__ void hlerp_row(uint32_t x, float lam, float h[3]) {
+// Horizontal interpolation at shared-memory byte address x (pixel x0, then x0 + 1) as exact
+// integers: per channel a * (den - rem) + b * rem, i.e. den times the interpolated value.
+// wgt holds (den - rem) in its low half and rem in its high half.  x is unaligned: three
+// aligned words are read and shifted; one permute lines up the two taps of two channels for
+// a 16-bit-by-8-bit two-way dot product, whose accumulator input 0x4B000000 makes the sum
+// the bit pattern of 2^23 + sum; the subtraction that removes 2^23 is exact.
+__device__ __forceinline__ void hlerp_row(uint32_t x, uint32_t wgt, float n[3]) {
   const uint32_t addr = x & ~3u;
   const uint32_t sh = x << 3;  // the funnel shift takes it modulo 32
   const uint32_t w0 = lds32(addr), w1 = lds32(addr + 4), w2 = lds32(addr + 8);
   const uint32_t lo = __funnelshift_r(w0, w1, sh);  // R0 G0 B0 R1
   const uint32_t hi = __funnelshift_r(w1, w2, sh);  // G1 B1 .. ..
-  const float a0 = byte_biased<0>(lo), a1 = byte_biased<1>(lo), a2 = byte_biased<2>(lo);
-  const float b0 = byte_biased<3>(lo), b1 = byte_biased<0>(hi), b2 = byte_biased<1>(hi);
-  h[0] = fmaf(lam, b0 - a0, a0 - 8388608.0f);
-  h[1] = fmaf(lam, b1 - a1, a1 - 8388608.0f);
-  h[2] = fmaf(lam, b2 - a2, a2 - 8388608.0f);
+  const uint32_t rg = __byte_perm(lo, hi, 0x4130);  // R0 R1 G0 G1
+  const uint32_t bb = __byte_perm(lo, hi, 0x5252);  // B0 B1 B0 B1
+  n[0] = __uint_as_float(__dp2a_lo(wgt, rg, 0x4B000000u)) - 8388608.0f;
+  n[1] = __uint_as_float(__dp2a_hi(wgt, rg, 0x4B000000u)) - 8388608.0f;
+  n[2] = __uint_as_float(__dp2a_lo(wgt, bb, 0x4B000000u)) - 8388608.0f;
 }
 
 template <typename OutT>
@@ -299,7 +304,8 @@ __device__ __forceinline__ uint32_t lane_col(uint32_t lane, uint32_t m) {
 // What a lane keeps for the task it computes on.
 struct Lane {
   uint32_t off[kLaneCols];  // byte offset of the first tap in a staged row (before its skew)
-  float lam[kLaneCols];     // weight of the second tap
+  uint32_t wgt[kLaneCols];  // staged path: (den - rem) | rem << 16, the integer weights of the
+                            // two taps; direct path: the second tap's weight as float bits
   uint32_t valid;           // bit m: column m exists
 };
 
@@ -389,7 +395,8 @@ __device__ __forceinline__ uint32_t prepare(const Params& p, uint32_t task, Task
     const uint32_t stride = (15 + 3 * copy_px + 3 + 12 + 15) & ~15u;
     const uint32_t rpg = min(kGroupRows, kGroupBytes / stride);
     const uint64_t end16 = (e.offset + 3ull * e.h * e.w + 15) & ~15ull;
-    kind = (rpg >= 1 && end16 <= p.pixels_bytes) ? kStream : kGather;
+    kind = (rpg >= 1 && end16 <= p.pixels_bytes && ax.small && ax.den <= kMaxPackedDen)
+               ? kStream : kGather;
 
     // rows of the slab: the ascending list of distinct source rows.  Output row `lane`
     // lists its lower tap if that lies beyond the previous row's upper tap, and its upper
@@ -453,8 +460,8 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
                                           uint32_t gwarp, uint32_t nwarps) {
   const uint32_t C = p.C;
   const uint32_t plane = C * C;
-  const float na[3] = {p.a[0], p.a[1], p.a[2]};
   const float nb[3] = {p.b[0], p.b[1], p.b[2]};
+  float sa[3] = {0.f, 0.f, 0.f};  // staged path: 1 / (255 * std * den) of the task's image
 
   // task claims: a warp's first task is its own index; later ones come from the shared
   // counter (dynamic) or every nwarps-th task (static)
@@ -488,7 +495,7 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
 #pragma unroll
   for (int m = 0; m < static_cast<int>(kLaneCols); ++m) {
     ln.off[m] = 0;
-    ln.lam[m] = 0.f;
+    ln.wgt[m] = 0;
 #pragma unroll
     for (int ch = 0; ch < 3; ++ch) hA[m][ch] = hB[m][ch] = 0.f;
   }
@@ -559,23 +566,26 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
       const uint32_t w = cm->w, rw = cm->rw, col0 = cm->col0, xmin = cm->xmin;
       const Axis ax = make_axis(w, rw, (rw - C) / 2, C);
       ln.valid = 0;
-      if (ax.small) {
+      if (kind == kStream) {  // implies ax.small and den <= kMaxPackedDen
 #pragma unroll
         for (int m = 0; m < static_cast<int>(kLaneCols); ++m) {
           const uint32_t j = col0 + lane_col(lane, m);
           if (j < C) ln.valid |= 1u << m;
           const Tap t = axis_tap_small(ax, min(j, C - 1));
           ln.off[m] = 3 * (t.i0 - xmin);
-          ln.lam[m] = t.lam;
+          ln.wgt[m] = (ax.den - t.rem) | (t.rem << 16);
         }
+        // staged rows carry den times the pixel value: fold 1 / den into the scale
+#pragma unroll
+        for (int ch = 0; ch < 3; ++ch) sa[ch] = p.a[ch] * ax.rden;
       } else {
 #pragma unroll
         for (int m = 0; m < static_cast<int>(kLaneCols); ++m) {
           const uint32_t j = col0 + lane_col(lane, m);
           if (j < C) ln.valid |= 1u << m;
-          const Tap t = axis_tap_wide(ax, min(j, C - 1));
+          const Tap t = axis_tap(ax, min(j, C - 1));
           ln.off[m] = 3 * (t.i0 - xmin);
-          ln.lam[m] = t.lam;
+          ln.wgt[m] = __float_as_uint(t.lam);
         }
       }
       full = (C & 1u) == 0 && __all_sync(0xffffffffu, ln.valid == 0x7fu);
@@ -593,6 +603,7 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
         const size_t pitch = 3 * static_cast<size_t>(w);
         const uint32_t h = cm->h, rh = cm->rh;
         const Axis ay = make_axis(h, rh, (rh - C) / 2, C);
+        const float na[3] = {p.a[0], p.a[1], p.a[2]};
         for (uint32_t t = 0; t < cm->rows_out; ++t, q_out += C) {
           const Tap ty = axis_tap(ay, cm->k0 + t);
           const uint8_t* r0 = src + ty.i0 * pitch;
@@ -600,13 +611,14 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
 #pragma unroll
           for (int m = 0; m < static_cast<int>(kLaneCols); ++m) {
             // the right neighbour is read only where it carries weight (it exists then)
-            const uint32_t nbr = ln.lam[m] > 0.f ? 3u : 0u;
+            const float lam = __uint_as_float(ln.wgt[m]);
+            const uint32_t nbr = lam > 0.f ? 3u : 0u;
 #pragma unroll
             for (int ch = 0; ch < 3; ++ch) {
               float a = __ldg(r0 + ln.off[m] + ch), b = __ldg(r0 + ln.off[m] + nbr + ch);
-              hA[m][ch] = fmaf(ln.lam[m], b - a, a);
+              hA[m][ch] = fmaf(lam, b - a, a);
               a = __ldg(r1 + ln.off[m] + ch), b = __ldg(r1 + ln.off[m] + nbr + ch);
-              hB[m][ch] = fmaf(ln.lam[m], b - a, a);
+              hB[m][ch] = fmaf(lam, b - a, a);
             }
           }
           emit_row<OutT, false>(q_out, plane, lane, ty.lam, hA, hB, na, nb, ln.valid);
@@ -633,7 +645,7 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
         if (par == 0) {
 #pragma unroll
           for (int m = 0; m < static_cast<int>(kLaneCols); ++m)
-            hlerp_row(base + ln.off[m], ln.lam[m], hA[m]);
+            hlerp_row(base + ln.off[m], ln.wgt[m], hA[m]);
 #pragma unroll 1
           for (; e > 0; --e, ++t_out, q_out += C) {
             const uint32_t lbits = cm->lam[t_out];
@@ -645,14 +657,14 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
             }
             const float ly = __uint_as_float(lbits & 0x7fffffffu);
             if (full)
-              emit_row<OutT, true>(q_out, plane, lane, ly, hB, hA, na, nb, ln.valid);
+              emit_row<OutT, true>(q_out, plane, lane, ly, hB, hA, sa, nb, ln.valid);
             else
-              emit_row<OutT, false>(q_out, plane, lane, ly, hB, hA, na, nb, ln.valid);
+              emit_row<OutT, false>(q_out, plane, lane, ly, hB, hA, sa, nb, ln.valid);
           }
         } else {
 #pragma unroll
           for (int m = 0; m < static_cast<int>(kLaneCols); ++m)
-            hlerp_row(base + ln.off[m], ln.lam[m], hB[m]);
+            hlerp_row(base + ln.off[m], ln.wgt[m], hB[m]);
 #pragma unroll 1
           for (; e > 0; --e, ++t_out, q_out += C) {
             const uint32_t lbits = cm->lam[t_out];
@@ -664,9 +676,9 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
             }
             const float ly = __uint_as_float(lbits & 0x7fffffffu);
             if (full)
-              emit_row<OutT, true>(q_out, plane, lane, ly, hA, hB, na, nb, ln.valid);
+              emit_row<OutT, true>(q_out, plane, lane, ly, hA, hB, sa, nb, ln.valid);
             else
-              emit_row<OutT, false>(q_out, plane, lane, ly, hA, hB, na, nb, ln.valid);
+              emit_row<OutT, false>(q_out, plane, lane, ly, hA, hB, sa, nb, ln.valid);
           }
         }
         par ^= 1u;
