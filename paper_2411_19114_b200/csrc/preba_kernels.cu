@@ -6,10 +6,11 @@
 // streams the tapped source rows into its private shared-memory ring with bulk asynchronous
 // copies (one per row, 16-byte aligned, completion counted on an mbarrier).  While a group
 // of rows is in flight the warp computes on the previous one: per staged row each lane
-// interpolates horizontally for its seven output columns and keeps the previous row's
-// result in registers; whenever both source rows of an output row have passed, it
-// interpolates vertically, applies the normalising multiply-add, converts and stores
-// planar output.  The copy stream runs ahead across task boundaries, so a warp's next task
+// interpolates horizontally for its seven output columns in exact integers (two taps times
+// their integer weights, a 16-bit-by-8-bit two-way dot product per channel) and keeps the
+// previous row's result in registers; whenever both source rows of an output row have
+// passed, it interpolates vertically in fp32, applies the normalising multiply-add (which
+// also divides by the weights' common denominator), converts and stores planar output.  The copy stream runs ahead across task boundaries, so a warp's next task
 // is already arriving while it finishes the current one.  Nothing but the input bytes and
 // the output tensor touches device memory; warps never wait for one another.
 #include <cuda_bf16.h>
@@ -92,7 +93,9 @@ struct TaskMeta {
   uint32_t info[kMaxList];  // per listed row: low byte = byte skew of the staged row,
                             // next byte = output rows completed by this row
   uint32_t lam[32];         // per output row: weight of the lower source row (float bits);
-                            // sign bit set when both taps are the same row
+                            // 1.0f when both taps are the same row (the row just staged):
+                            // staged values are whole numbers below 2^24, so
+                            // prev + 1 * (cur - prev) is cur exactly, whatever prev holds
   uint32_t row[kMaxList];   // per listed row: source row index
 };
 
@@ -242,9 +245,10 @@ __device__ __forceinline__ void fence_async_shared() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 
+template <int OFF>
 __device__ __forceinline__ uint32_t lds32(uint32_t addr) {
   uint32_t v;
-  asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+  asm volatile("ld.shared.u32 %0, [%1+%2];" : "=r"(v) : "r"(addr), "n"(OFF));
   return v;
 }
 
@@ -263,7 +267,7 @@ constexpr uint32_t kMaxPackedDen = 32768;
 __device__ __forceinline__ void hlerp_row(uint32_t x, uint32_t wgt, float n[3]) {
   const uint32_t addr = x & ~3u;
   const uint32_t sh = x << 3;  // the funnel shift takes it modulo 32
-  const uint32_t w0 = lds32(addr), w1 = lds32(addr + 4), w2 = lds32(addr + 8);
+  const uint32_t w0 = lds32<0>(addr), w1 = lds32<4>(addr), w2 = lds32<8>(addr);
   const uint32_t lo = __funnelshift_r(w0, w1, sh);  // R0 G0 B0 R1
   const uint32_t hi = __funnelshift_r(w1, w2, sh);  // G1 B1 .. ..
   const uint32_t rg = __byte_perm(lo, hi, 0x4130);  // R0 R1 G0 G1
@@ -422,7 +426,7 @@ __device__ __forceinline__ uint32_t prepare(const Params& p, uint32_t task, Task
       m.row[at] = ty.i1;
       m.info[at] = (done << 8) | ((3u * (ty.i1 * e.w + xmin)) & 15u);
     }
-    if (active) m.lam[lane] = __float_as_uint(ty.lam) | (ty.i1 == ty.i0 ? 0x80000000u : 0u);
+    if (active) m.lam[lane] = __float_as_uint(ty.i1 == ty.i0 ? 1.0f : ty.lam);
     if (lane == 0) {
       m.img = img;
       m.k0 = k0;
@@ -623,6 +627,11 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
           }
           emit_row<OutT, false>(q_out, plane, lane, ty.lam, hA, hB, na, nb, ln.valid);
         }
+        // the staged path relies on whole numbers in the row buffers
+#pragma unroll
+        for (int m = 0; m < static_cast<int>(kLaneCols); ++m)
+#pragma unroll
+          for (int ch = 0; ch < 3; ++ch) hA[m][ch] = hB[m][ch] = 0.f;
         ++finished;
         need_task = true;
       }
@@ -648,14 +657,7 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
             hlerp_row(base + ln.off[m], ln.wgt[m], hA[m]);
 #pragma unroll 1
           for (; e > 0; --e, ++t_out, q_out += C) {
-            const uint32_t lbits = cm->lam[t_out];
-            if (lbits >> 31) {  // both taps are this row
-#pragma unroll
-              for (int m = 0; m < static_cast<int>(kLaneCols); ++m)
-#pragma unroll
-                for (int ch = 0; ch < 3; ++ch) hB[m][ch] = hA[m][ch];
-            }
-            const float ly = __uint_as_float(lbits & 0x7fffffffu);
+            const float ly = __uint_as_float(cm->lam[t_out]);
             if (full)
               emit_row<OutT, true>(q_out, plane, lane, ly, hB, hA, sa, nb, ln.valid);
             else
@@ -667,14 +669,7 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
             hlerp_row(base + ln.off[m], ln.wgt[m], hB[m]);
 #pragma unroll 1
           for (; e > 0; --e, ++t_out, q_out += C) {
-            const uint32_t lbits = cm->lam[t_out];
-            if (lbits >> 31) {
-#pragma unroll
-              for (int m = 0; m < static_cast<int>(kLaneCols); ++m)
-#pragma unroll
-                for (int ch = 0; ch < 3; ++ch) hA[m][ch] = hB[m][ch];
-            }
-            const float ly = __uint_as_float(lbits & 0x7fffffffu);
+            const float ly = __uint_as_float(cm->lam[t_out]);
             if (full)
               emit_row<OutT, true>(q_out, plane, lane, ly, hA, hB, sa, nb, ln.valid);
             else
@@ -716,7 +711,10 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) preba_fused_kernel(const
   // a following launch that was marked independent of this one may start as soon as
   // resources free up
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const uint32_t lane = threadIdx.x & 31;
+  // read through a shuffle so that the compiler treats the warp's index, and the shared-memory
+  // addresses derived from it, as the same in every lane
+  const uint32_t warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0);
   WarpShared& ws = sm[warp];
   if (lane == 0) {
     for (uint32_t g = 0; g < kGroups; ++g) mbar_init(smem_addr(&ws.full[g]), kGroupRows);
