@@ -379,46 +379,116 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
     warm_ms = w_start.elapsed_time(w_stop)
 
     # ---- end to end from host images ----------------------------------------------------------
+    # The decoded images wait in pinned host memory, each in a buffer of its own (carved from
+    # one arena in reverse order, page-aligned: not the packed layout).  Every step the kernel
+    # fetches the rows it taps from there, across the host-device link, and the result is
+    # copied back to pinned memory (preba_preprocess_images with PREBA_IMAGES_IN_PLACE); two
+    # buffer sets on two streams, so one step's kernel overlaps the other's result copy.
     e2e_steps = max(3, min(args.e2e_steps, args.steps))
     sizes = pb.preba_query(table["h"], table["w"], C, out_dtype)
     nbuf = 2
-    ph = [torch.empty(sizes.packed_bytes, dtype=torch.uint8).pin_memory() for _ in range(nbuf)]
+    page = 4096
+    starts, at = [], 0
+    for im in reversed(images):
+        starts.append(at)
+        at += -(-im.nbytes // page) * page
+    starts.reverse()
+    arena = torch.empty(at, dtype=torch.uint8).pin_memory()
+    pinned = []
+    for im, st0 in zip(images, starts):
+        view = arena[st0:st0 + im.nbytes].view(im.shape)
+        view.copy_(torch.from_numpy(im))
+        pinned.append(view)
     oh = [torch.empty((n, 3, C, C), dtype=tdt).pin_memory() for _ in range(nbuf)]
-    th = [np.zeros(n, dtype=pb.TABLE_DTYPE) for _ in range(nbuf)]
+    th = [torch.zeros(n * 16, dtype=torch.uint8).pin_memory() for _ in range(nbuf)]
     dtab = [torch.empty(n * 16, dtype=torch.uint8, device=dev) for _ in range(nbuf)]
     done = [torch.cuda.Event() for _ in range(nbuf)]
-    side = [torch.cuda.Stream(device=dev) for _ in range(nbuf)]  # one stream per buffer set:
+    side = [torch.cuda.Stream(device=dev) for _ in range(nbuf)]  # one stream per buffer set
     scr = [torch.zeros(pb.SCRATCH_BYTES // 4, dtype=torch.int32, device=dev) for _ in range(nbuf)]
+    e2e_calls = [pb.PreparedImages(pinned, th[b], oh[b], None, dtab[b], outs[b], C, S, wl.MEAN,
+                                   wl.STD, out_dtype, stream=side[b], dev_status=status,
+                                   dev_scratch=scr[b], in_place=True) for b in range(nbuf)]
+    copy_calls = [pb.PreparedImages(pinned, th[b], oh[b], pix[b], dtab[b], outs[b], C, S, wl.MEAN,
+                                    wl.STD, out_dtype, stream=side[b], dev_status=status,
+                                    dev_scratch=scr[b]) for b in range(nbuf)]
 
     def e2e_step(i):
         b = i % nbuf
         done[b].synchronize()                       # the set's previous copies have finished
-        pb.preba_pack(images, ph[b].numpy(), th[b])
-        pb.preba_preprocess_host(ph[b], th[b], n, oh[b], pix[b], dtab[b], outs[b], C, S, wl.MEAN,
+        t0 = time.perf_counter()
+        e2e_calls[b]()
+        done[b].record(side[b])
+        return time.perf_counter() - t0
+
+    def timed_e2e(step, steps):
+        for i in range(2):
+            step(i)
+        barrier()
+        e_start, e_stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t_host = 0.0
+        e_start.record(stream)
+        for st in side:
+            st.wait_stream(stream)                  # the timed region starts on both streams
+        for i in range(steps):
+            t_host += step(i)                       # host time of the calls, waits excluded
+        for st in side:
+            stream.wait_stream(st)                  # ... and ends when both are done
+        e_stop.record(stream)
+        barrier()
+        return e_start.elapsed_time(e_stop), t_host
+
+    e2e_ms, t_pack = timed_e2e(e2e_step, e2e_steps)
+    assert int(status.item()) == 0
+    for b in range(nbuf):                           # the host result is the device result
+        assert bool(torch.equal(oh[b], ref.cpu())), "end-to-end result differs"
+
+    # the same with one copy per image to the device instead of reads in place
+    def copy_step(i):
+        b = i % nbuf
+        done[b].synchronize()
+        t0 = time.perf_counter()
+        copy_calls[b]()
+        done[b].record(side[b])
+        return time.perf_counter() - t0
+
+    copied_ms, copied_host = timed_e2e(copy_step, e2e_steps)
+    assert int(status.item()) == 0
+
+    # the same from a packed host buffer: preba_pack of the images into pinned memory, one
+    # copy of the packed buffer, kernel, copy back (reported for comparison)
+    ph = [torch.empty(sizes.packed_bytes, dtype=torch.uint8).pin_memory() for _ in range(nbuf)]
+    tp = [np.zeros(n, dtype=pb.TABLE_DTYPE) for _ in range(nbuf)]
+
+    def packed_step(i):
+        b = i % nbuf
+        done[b].synchronize()
+        t0 = time.perf_counter()
+        pb.preba_pack(images, ph[b].numpy(), tp[b])
+        pb.preba_preprocess_host(ph[b], tp[b], n, oh[b], pix[b], dtab[b], outs[b], C, S, wl.MEAN,
                                  wl.STD, out_dtype, stream=side[b], dev_status=status,
                                  dev_scratch=scr[b])
         done[b].record(side[b])
+        return time.perf_counter() - t0
 
-    for i in range(2):
-        e2e_step(i)
-    barrier()
-    e_start, e_stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    t_pack = 0.0
-    e_start.record(stream)
-    for st in side:
-        st.wait_stream(stream)                      # the timed region starts on both streams
-    for i in range(e2e_steps):
-        t0 = time.perf_counter()
-        e2e_step(i)
-        t_pack += time.perf_counter() - t0
-    for st in side:
-        stream.wait_stream(st)                      # ... and ends when both are done
-    e_stop.record(stream)
-    barrier()
-    e2e_ms = e_start.elapsed_time(e_stop)
+    packed_ms, packed_host = timed_e2e(packed_step, e2e_steps)
     assert int(status.item()) == 0
 
-    elapsed_ms, e2e_ms = max_over_ranks([elapsed_ms, e2e_ms], dist, dev)
+    # what the host-device link gives a plain pinned copy of the packed batch, each way
+    link = {}
+    big_out = oh[0].view(torch.uint8).reshape(-1)
+    for name, dst, src in (("h2d", pix[0], ph[0]), ("d2h", big_out, outs[0].view(torch.uint8).reshape(-1))):
+        l_start, l_stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        dst.copy_(src, non_blocking=True)
+        barrier()
+        l_start.record(stream)
+        for _ in range(3):
+            dst.copy_(src, non_blocking=True)
+        l_stop.record(stream)
+        barrier()
+        link[name + "_gbs"] = 3 * src.numel() / (l_start.elapsed_time(l_stop) * 1e-3) / 1e9
+
+    elapsed_ms, e2e_ms, packed_ms, copied_ms = max_over_ranks(
+        [elapsed_ms, e2e_ms, packed_ms, copied_ms], dist, dev)
 
     if rank == 0:
         peak, peak_src = measured_peak()
@@ -456,8 +526,24 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
                     "d2h_bytes_per_step": int(sizes.out_bytes), "steps": e2e_steps,
                     "ms_per_step": e2e_ms / e2e_steps,
                     "host_ms_per_step": 1e3 * t_pack / e2e_steps,
-                    "includes": "preba_pack into pinned memory + H2D + kernel + D2H, two "
-                                "buffer sets on two streams"},
+                    "link_plain_copy_gbs": link,
+                    "includes": "preba_preprocess_images, images read in place: the kernel "
+                                "fetches the tapped rows of every image from its own pinned "
+                                "host buffer across the link, then the result is copied to "
+                                "pinned memory; two buffer sets on two streams",
+                    "h2d_bytes_note": "bytes of the images (all of them would cross in a "
+                                      "copy); in place only the tapped sectors cross: "
+                                      f"{acct['input_sector_bytes']}",
+                    "one_copy_per_image": {
+                        "value": world * n * e2e_steps / (copied_ms * 1e-3),
+                        "ms_per_step": copied_ms / e2e_steps,
+                        "host_ms_per_step": 1e3 * copied_host / e2e_steps},
+                    "from_packed_host_buffer": {
+                        "value": world * n * e2e_steps / (packed_ms * 1e-3),
+                        "ms_per_step": packed_ms / e2e_steps,
+                        "host_ms_per_step": 1e3 * packed_host / e2e_steps,
+                        "includes": "preba_pack into pinned memory + one copy + kernel + copy "
+                                    "back (preba_preprocess_host)"}},
             "warm_l2": {"value": world * n * warm_steps / (warm_ms * 1e-3), "unit": UNIT,
                         "us_per_launch": 1e3 * warm_ms / warm_steps,
                         "note": "one buffer set reused by every launch; not the headline"},

@@ -110,6 +110,38 @@ typedef struct {
   uint32_t* dev_scratch;         /* DEVICE or NULL, as preba_batch_t.scratch */
 } preba_host_batch_t;
 
+/* preba_image_batch_t.flags */
+#define PREBA_IMAGES_IN_PLACE 1u  /* the kernel reads the images where they lie, in pinned host
+                                     memory, across the host-device link: only the bytes the
+                                     transform taps cross it, and no copy is enqueued for them.
+                                     Every image pointer must then be pinned memory the device
+                                     can address (cudaMallocHost / cudaHostAlloc), a multiple of
+                                     PREBA_PACK_ALIGN, and readable through the end of the
+                                     16-byte block that holds the image's last byte; the
+                                     images must not overlap.  dev_pixels is not used. */
+
+/* A batch of separate decoded images in host memory (no packed copy on the host), with the
+ * device buffers the call stages it through. */
+typedef struct {
+  const uint8_t* const* images;  /* HOST array of n HOST pointers; image i is h[i] rows of w[i]
+                                    RGB pixels, pitch 3*w[i] (pinned for asynchronous copies) */
+  const uint32_t* h;             /* HOST, n entries */
+  const uint32_t* w;             /* HOST, n entries */
+  uint32_t n;
+  uint32_t flags;                /* 0 or PREBA_IMAGES_IN_PLACE */
+  preba_img_t* table_host;       /* HOST, n entries, WRITTEN by the call (the table preba_pack
+                                    would build); pinned; valid until the stream has passed
+                                    the call's copies */
+  void* out_host;                /* HOST (pinned for an asynchronous copy), out_bytes bytes */
+  uint64_t out_bytes;
+  uint8_t* dev_pixels;           /* DEVICE staging, 16-byte aligned */
+  uint64_t dev_pixels_bytes;     /* capacity of dev_pixels, >= sizes.packed_bytes */
+  preba_img_t* dev_table;        /* DEVICE staging, n entries */
+  void* dev_out;                 /* DEVICE staging, >= out_bytes, 16-byte aligned */
+  int32_t* dev_status;           /* DEVICE word or NULL, as preba_batch_t.status */
+  uint32_t* dev_scratch;         /* DEVICE or NULL, as preba_batch_t.scratch */
+} preba_image_batch_t;
+
 /*
  * preba_query — sizes of the buffers a batch needs (host arithmetic only).
  * The packed layout is the problem statement's, not the paper's (which handles
@@ -177,6 +209,26 @@ int preba_preprocess(const preba_batch_t* batch, uint32_t out_size, uint32_t res
 int preba_preprocess_host(const preba_host_batch_t* batch, uint32_t out_size,
                           uint32_t resize_short, const float mean[3], const float std[3],
                           int out_dtype, void* stream);
+
+/*
+ * preba_preprocess_images — step 0 and the transform in one call, for decoded images that
+ * already sit in (pinned) host memory one by one, as a decoder leaves them: each request
+ * arrives on its own (paper Sec. 5 "Input query modeling") and crosses the host-device
+ * link once (Sec. 4.2 "Implication of adding DPU").  Nothing is packed on the host: the
+ * call lays the batch out as preba_pack would (same offsets, written to `table_host`),
+ * copies every image straight to its offset in `dev_pixels`, then enqueues the table copy,
+ * the kernel and the copy of the result to `out_host`, all on `stream`, and returns.
+ * Padding bytes between images stay as the device buffer had them; the transform never
+ * gives them weight.  n + 1 host-to-device copies, one kernel, one device-to-host copy.
+ * With PREBA_IMAGES_IN_PLACE the image copies are dropped: `table_host` receives each
+ * image's distance from the lowest image address, and the kernel fetches the tapped rows
+ * from host memory itself (table copy, kernel, result copy).
+ * Errors: PREBA_ERR_INVALID_ARG, PREBA_ERR_BUFFER_TOO_SMALL (dev_pixels_bytes, out_bytes),
+ * PREBA_ERR_CUDA.
+ */
+int preba_preprocess_images(const preba_image_batch_t* batch, uint32_t out_size,
+                            uint32_t resize_short, const float mean[3], const float std[3],
+                            int out_dtype, void* stream);
 
 /*
  * preba_preprocess_host_noalloc — preba_preprocess_host for callers that have no way to

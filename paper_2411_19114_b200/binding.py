@@ -15,6 +15,7 @@ _LIB_PATH = Path(__file__).resolve().parent / "libpreba.so"
 
 PACK_ALIGN = 128
 SCRATCH_BYTES = 256
+IMAGES_IN_PLACE = 1
 OVERLAP_PREVIOUS = 1
 F32, F16, BF16 = 0, 1, 2
 
@@ -27,7 +28,7 @@ ERR_TIMEOUT = -5
 ERR_TOO_LARGE = -6
 NOALLOC_MAX_BYTES = 64 << 20
 
-EXPORTS = ("preba_query", "preba_pack", "preba_preprocess", "preba_preprocess_host",
+EXPORTS = ("preba_query", "preba_pack", "preba_preprocess", "preba_preprocess_host", "preba_preprocess_images",
            "preba_preprocess_host_noalloc", "preba_preprocess_repeated", "preba_selftest_wait_limit",
            "preba_strerror",
            "preba_last_cuda_error",
@@ -60,6 +61,16 @@ class PrebaHostBatch(ctypes.Structure):
                 ("out_bytes", ctypes.c_uint64), ("dev_pixels", ctypes.c_void_p),
                 ("dev_table", ctypes.c_void_p), ("dev_out", ctypes.c_void_p),
                 ("dev_status", ctypes.c_void_p), ("dev_scratch", ctypes.c_void_p)]
+
+
+class PrebaImageBatch(ctypes.Structure):
+    _fields_ = [("images", ctypes.c_void_p), ("h", ctypes.c_void_p), ("w", ctypes.c_void_p),
+                ("n", ctypes.c_uint32), ("flags", ctypes.c_uint32),
+                ("table_host", ctypes.c_void_p), ("out_host", ctypes.c_void_p),
+                ("out_bytes", ctypes.c_uint64), ("dev_pixels", ctypes.c_void_p),
+                ("dev_pixels_bytes", ctypes.c_uint64), ("dev_table", ctypes.c_void_p),
+                ("dev_out", ctypes.c_void_p), ("dev_status", ctypes.c_void_p),
+                ("dev_scratch", ctypes.c_void_p)]
 
 
 TABLE_DTYPE = np.dtype([("offset", "<u8"), ("h", "<u4"), ("w", "<u4")])
@@ -96,6 +107,10 @@ def lib() -> ctypes.CDLL:
         L.preba_preprocess_host.argtypes = [ctypes.POINTER(PrebaHostBatch), ctypes.c_uint32,
                                             ctypes.c_uint32, f32p, f32p, ctypes.c_int,
                                             ctypes.c_void_p]
+        L.preba_preprocess_images.argtypes = [ctypes.POINTER(PrebaImageBatch), ctypes.c_uint32,
+                                              ctypes.c_uint32, f32p, f32p, ctypes.c_int,
+                                              ctypes.c_void_p]
+        L.preba_preprocess_images.restype = ctypes.c_int
         L.preba_preprocess_repeated.argtypes = [ctypes.POINTER(PrebaBatch), ctypes.c_uint32,
                                                 ctypes.c_uint32, f32p, f32p, ctypes.c_int,
                                                 ctypes.c_void_p, ctypes.c_uint32, f32p, f32p]
@@ -313,6 +328,64 @@ def preba_preprocess_host(packed_host, table_host: np.ndarray, n: int, out_host,
                                      ctypes.c_void_p(stream))
     if rc != OK:
         raise PrebaError(rc, "preba_preprocess_host")
+
+
+class PreparedImages:
+    """The arguments of ``preba_preprocess_images`` for a fixed set of host images, marshalled
+    once.  ``images`` are uint8 HWC arrays or CPU tensors (pinned for asynchronous copies);
+    ``table_host`` is a pinned CPU tensor of ``16 * n`` bytes that every call rewrites;
+    ``out_host`` a (pinned) CPU tensor; ``dev_*`` CUDA tensors used as staging.  With
+    ``in_place`` the kernel reads the (pinned, 128-byte aligned) images over the link itself
+    and ``dev_pixels`` may be None."""
+
+    def __init__(self, images, table_host, out_host, dev_pixels, dev_table, dev_out,
+                 out_size: int, resize_short: int, mean, std, out_dtype: int, stream=None,
+                 dev_status=None, dev_scratch=None, in_place: bool = False):
+        import torch
+
+        def haddr(t):
+            return t.ctypes.data if isinstance(t, np.ndarray) else t.data_ptr()
+
+        def hbytes(t):
+            return t.nbytes if isinstance(t, np.ndarray) else t.numel() * t.element_size()
+
+        if stream is None:
+            stream = torch.cuda.current_stream().cuda_stream
+        elif hasattr(stream, "cuda_stream"):
+            stream = stream.cuda_stream
+        n = len(images)
+        for im in images:
+            if tuple(im.shape)[2:] != (3,) or hbytes(im) != im.shape[0] * im.shape[1] * 3:
+                raise ValueError("images must be contiguous uint8 arrays of shape (h, w, 3)")
+        self._ptrs = (ctypes.c_void_p * n)(*[haddr(im) for im in images])
+        self._h = _u32([im.shape[0] for im in images])
+        self._w = _u32([im.shape[1] for im in images])
+        if hbytes(table_host) < 16 * n:
+            raise PrebaError(ERR_BUFFER_TOO_SMALL, "preba_preprocess_images (table_host)")
+        b = PrebaImageBatch()
+        b.images = ctypes.cast(self._ptrs, ctypes.c_void_p)
+        b.h, b.w, b.n = self._h.ctypes.data, self._w.ctypes.data, n
+        b.table_host = haddr(table_host)
+        b.out_host, b.out_bytes = haddr(out_host), hbytes(out_host)
+        b.flags = IMAGES_IN_PLACE if in_place else 0
+        if dev_pixels is not None:
+            b.dev_pixels = dev_pixels.data_ptr()
+            b.dev_pixels_bytes = dev_pixels.numel() * dev_pixels.element_size()
+        b.dev_table, b.dev_out = dev_table.data_ptr(), dev_out.data_ptr()
+        if dev_out.numel() * dev_out.element_size() < b.out_bytes:
+            raise PrebaError(ERR_BUFFER_TOO_SMALL, "preba_preprocess_images (dev_out)")
+        b.dev_status = dev_status.data_ptr() if dev_status is not None else None
+        b.dev_scratch = dev_scratch.data_ptr() if dev_scratch is not None else None
+        self._b, self._m, self._s = b, _f3(mean), _f3(std)
+        self._keep = (images, table_host, out_host, dev_pixels, dev_table, dev_out, dev_status,
+                      dev_scratch)
+        self._args = (ctypes.byref(b), out_size, resize_short, _p(self._m, ctypes.c_float),
+                      _p(self._s, ctypes.c_float), out_dtype, ctypes.c_void_p(stream))
+
+    def __call__(self) -> None:
+        rc = lib().preba_preprocess_images(*self._args)
+        if rc != OK:
+            raise PrebaError(rc, "preba_preprocess_images")
 
 
 def preba_preprocess_host_noalloc(packed_host, table_host: np.ndarray, n: int, out_host,

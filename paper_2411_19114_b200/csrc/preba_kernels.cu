@@ -19,6 +19,7 @@
 
 #include <atomic>
 #include <cmath>
+#include <cstdint>
 #include <vector>
 
 #include "preba.h"
@@ -893,6 +894,88 @@ extern "C" int preba_preprocess_host(const preba_host_batch_t* b, uint32_t out_s
     return PREBA_ERR_CUDA;
   }
   const Params p = make_params(b->dev_pixels, b->packed_bytes, b->dev_table, b->n, b->dev_out,
+                               b->dev_status, b->dev_scratch, out_size, resize_short, mean, std);
+  rc = launch(p, out_dtype, false, s);
+  if (rc != PREBA_OK) return rc;
+  err = cudaMemcpyAsync(b->out_host, b->dev_out, need, cudaMemcpyDeviceToHost, s);
+  if (err != cudaSuccess) {
+    g_last_cuda_error = static_cast<int>(err);
+    return PREBA_ERR_CUDA;
+  }
+  return PREBA_OK;
+}
+
+extern "C" int preba_preprocess_images(const preba_image_batch_t* b, uint32_t out_size,
+                                       uint32_t resize_short, const float mean[3],
+                                       const float std[3], int out_dtype, void* stream) {
+  using namespace preba;
+  if (!b || !b->images || !b->h || !b->w || !b->table_host || !b->out_host || !b->dev_table ||
+      b->n == 0 || (b->flags & ~PREBA_IMAGES_IN_PLACE))
+    return PREBA_ERR_INVALID_ARG;
+  const bool in_place = (b->flags & PREBA_IMAGES_IN_PLACE) != 0;
+  for (uint32_t i = 0; i < b->n; ++i)
+    if (!b->images[i] || !dims_ok(b->h[i], b->w[i])) return PREBA_ERR_INVALID_ARG;
+  const uint8_t* pixels = b->dev_pixels;
+  uint64_t pixels_bytes = 0;
+  if (in_place) {
+    // the "packed buffer" is host memory as it stands: offsets from the lowest image
+    uintptr_t lo = UINTPTR_MAX;
+    for (uint32_t i = 0; i < b->n; ++i) {
+      const uintptr_t a = reinterpret_cast<uintptr_t>(b->images[i]);
+      if (a % PREBA_PACK_ALIGN) return PREBA_ERR_INVALID_ARG;
+      lo = a < lo ? a : lo;
+    }
+    for (uint32_t i = 0; i < b->n; ++i) {
+      const uint64_t off = reinterpret_cast<uintptr_t>(b->images[i]) - lo;
+      b->table_host[i].offset = off;
+      b->table_host[i].h = b->h[i];
+      b->table_host[i].w = b->w[i];
+      const uint64_t end = off + align_up(3ull * b->h[i] * b->w[i], 16);
+      pixels_bytes = end > pixels_bytes ? end : pixels_bytes;
+    }
+    pixels = reinterpret_cast<const uint8_t*>(lo);
+  } else {
+    // the packed layout: running byte count rounded up to the alignment
+    uint64_t at = 0;
+    for (uint32_t i = 0; i < b->n; ++i) {
+      b->table_host[i].offset = at;
+      b->table_host[i].h = b->h[i];
+      b->table_host[i].w = b->w[i];
+      at = align_up(at + 3ull * b->h[i] * b->w[i], PREBA_PACK_ALIGN);
+    }
+    pixels_bytes = at;
+    if (b->dev_pixels_bytes < pixels_bytes) return PREBA_ERR_BUFFER_TOO_SMALL;
+  }
+  int rc = check_args(pixels, pixels_bytes, b->dev_table, b->n, b->dev_out, b->out_bytes,
+                      out_size, resize_short, mean, std, out_dtype);
+  if (rc != PREBA_OK) return rc;
+  if (reinterpret_cast<uintptr_t>(b->dev_scratch) % 16) return PREBA_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const uint64_t need = static_cast<uint64_t>(b->n) * 3ull * out_size * out_size *
+                        dtype_bytes(out_dtype);
+  cudaError_t err = cudaSuccess;
+  if (in_place) {
+    // the device must be able to address the images through the pointers given
+    for (uint32_t i = 0; i < b->n && err == cudaSuccess; ++i) {
+      cudaPointerAttributes attr;
+      err = cudaPointerGetAttributes(&attr, b->images[i]);
+      if (err == cudaSuccess && (attr.type == cudaMemoryTypeUnregistered ||
+                                 attr.devicePointer != static_cast<const void*>(b->images[i])))
+        return PREBA_ERR_INVALID_ARG;
+    }
+  } else {
+    for (uint32_t i = 0; i < b->n && err == cudaSuccess; ++i)
+      err = cudaMemcpyAsync(b->dev_pixels + b->table_host[i].offset, b->images[i],
+                            3ull * b->h[i] * b->w[i], cudaMemcpyHostToDevice, s);
+  }
+  if (err == cudaSuccess)
+    err = cudaMemcpyAsync(b->dev_table, b->table_host, sizeof(preba_img_t) * b->n,
+                          cudaMemcpyHostToDevice, s);
+  if (err != cudaSuccess) {
+    g_last_cuda_error = static_cast<int>(err);
+    return PREBA_ERR_CUDA;
+  }
+  const Params p = make_params(pixels, pixels_bytes, b->dev_table, b->n, b->dev_out,
                                b->dev_status, b->dev_scratch, out_size, resize_short, mean, std);
   rc = launch(p, out_dtype, false, s);
   if (rc != PREBA_OK) return rc;

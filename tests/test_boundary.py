@@ -44,6 +44,7 @@ def test_struct_layouts_match_header():
     assert ctypes.sizeof(pb.PrebaSizes) == 32
     assert ctypes.sizeof(pb.PrebaBatch) == 72
     assert ctypes.sizeof(pb.PrebaHostBatch) == 88
+    assert ctypes.sizeof(pb.PrebaImageBatch) == 104
 
 
 def test_query_sizes():
@@ -172,6 +173,51 @@ def test_preprocess_checks_host_table_before_launch():
                 [(0, 8, 8), (1 << 40, 8, 8)]):      # offset past the pixel buffer
         t = table(bad)
         assert _call(_batch(table_host=t.ctypes.data)) == pb.ERR_BAD_TABLE
+
+
+def test_separate_images_entry_point_rejects_bad_arguments_before_any_copy():
+    """preba_preprocess_images validates on the host first: nothing below reaches CUDA."""
+    img = np.zeros((8, 8, 3), dtype=np.uint8)
+    ptrs = (ctypes.c_void_p * 2)(img.ctypes.data, img.ctypes.data)
+    h = np.array([8, 8], dtype=np.uint32)
+    w = np.array([8, 8], dtype=np.uint32)
+    tab = np.zeros(2, dtype=pb.TABLE_DTYPE)
+
+    def call(c=8, s=8, **kw):
+        b = pb.PrebaImageBatch()
+        b.images = ctypes.cast(ptrs, ctypes.c_void_p)
+        b.h, b.w, b.n = h.ctypes.data, w.ctypes.data, 2
+        b.table_host = tab.ctypes.data
+        b.out_host, b.out_bytes = 0x50000, 2 * 3 * 8 * 8 * 4
+        b.dev_pixels, b.dev_pixels_bytes = 0x10000, 512
+        b.dev_table, b.dev_out = 0x20000, 0x30000
+        for k, v in kw.items():
+            setattr(b, k, v)
+        m = (ctypes.c_float * 3)(*MEAN)
+        sd = (ctypes.c_float * 3)(*STD)
+        return pb.lib().preba_preprocess_images(ctypes.byref(b), c, s, m, sd, pb.F32, None)
+
+    assert pb.lib().preba_preprocess_images(None, 8, 8, None, None, pb.F32, None) == pb.ERR_INVALID_ARG
+    assert call(images=None) == pb.ERR_INVALID_ARG
+    assert call(table_host=None) == pb.ERR_INVALID_ARG
+    assert call(out_host=None) == pb.ERR_INVALID_ARG
+    assert call(dev_table=None) == pb.ERR_INVALID_ARG
+    assert call(n=0) == pb.ERR_INVALID_ARG
+    assert call(dev_pixels_bytes=511) == pb.ERR_BUFFER_TOO_SMALL   # two images of 192 -> 256 bytes each
+    assert call(out_bytes=2 * 3 * 8 * 8 * 4 - 1) == pb.ERR_BUFFER_TOO_SMALL
+    assert call(dev_pixels=0x10004) == pb.ERR_INVALID_ARG          # misaligned staging
+    assert call(c=9, s=8) == pb.ERR_INVALID_ARG                    # crop larger than resize
+    assert call(flags=2) == pb.ERR_INVALID_ARG                     # unknown flag
+    raw = np.zeros(8 * 8 * 3 + 256, dtype=np.uint8)
+    odd = raw.ctypes.data + (64 - raw.ctypes.data) % 128           # an address that is 64 mod 128
+    assert odd % 128 == 64
+    two = (ctypes.c_void_p * 2)(odd, odd)
+    assert call(flags=pb.IMAGES_IN_PLACE, images=ctypes.cast(two, ctypes.c_void_p)) \
+        == pb.ERR_INVALID_ARG                                      # in place wants 128-byte aligned images
+    # the table is written before the checks that follow it: the layout of preba_pack
+    assert [int(e["offset"]) for e in tab] == [0, 256]
+    w[1] = 0
+    assert call() == pb.ERR_INVALID_ARG                            # zero width
 
 
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):

@@ -359,3 +359,91 @@ def test_host_buffer_entry_point_matches_device_entry_point():
     assert int(status.item()) == 0
     want = run_gpu(imgs, 224, 256, out_dtype=pb.F16)
     assert np.array_equal(oh.numpy().view(np.uint16), want.view(np.uint16))
+
+
+def test_separate_host_images_entry_point_matches_the_packed_path_and_the_oracle():
+    """preba_preprocess_images: each image copied from its own pinned buffer to its packed
+    offset; device staging pre-filled with a pattern, so padding bytes are not zero."""
+    import torch
+
+    imgs = wl.mixed_smooth(9, seed=11) + [uniform(5, 1, 1), uniform(6, 241, 277)]
+    n = len(imgs)
+    packed, table = pb.preba_pack(imgs)
+    dev = torch.device("cuda:0")
+    pinned = [torch.from_numpy(im.copy()).pin_memory() for im in imgs]
+    th = torch.zeros(n * 16, dtype=torch.uint8).pin_memory()
+    oh = torch.zeros((n, 3, 224, 224), dtype=torch.float32).pin_memory()
+    dp = torch.full((packed.nbytes,), 0xEE, dtype=torch.uint8, device=dev)
+    dtab = torch.empty(n * 16, dtype=torch.uint8, device=dev)
+    dout = torch.empty((n, 3, 224, 224), dtype=torch.float32, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    call = pb.PreparedImages(pinned, th, oh, dp, dtab, dout, 224, 256, MEAN, STD, pb.F32,
+                             dev_status=status)
+    for _ in range(2):
+        call()
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        assert np.array_equal(th.numpy().view(pb.TABLE_DTYPE), table), "table differs from preba_pack's"
+        got = oh.numpy().copy()
+        assert_parity(got, oracle_f64(imgs, 224, 256), pb.F32)
+        want = run_gpu(imgs, 224, 256, out_dtype=pb.F32)
+        assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+        oh.zero_()
+    # every image landed at its packed offset, bit for bit
+    dev_bytes = dp.cpu().numpy()
+    for im, e in zip(imgs, table):
+        o = int(e["offset"])
+        assert np.array_equal(dev_bytes[o:o + im.size], im.reshape(-1))
+    # staging that cannot hold the packed batch is refused before anything is enqueued
+    small = torch.empty(packed.nbytes - 128, dtype=torch.uint8, device=dev)
+    bad = pb.PreparedImages(pinned, th, oh, small, dtab, dout, 224, 256, MEAN, STD, pb.F32)
+    with pytest.raises(pb.PrebaError) as exc:
+        bad()
+    assert exc.value.code == pb.ERR_BUFFER_TOO_SMALL
+
+
+def test_images_read_in_place_from_pinned_host_memory():
+    """PREBA_IMAGES_IN_PLACE: no image copies; the kernel fetches the tapped rows from pinned
+    host memory.  Same bits as the packed device path; pageable memory is refused."""
+    import torch
+
+    imgs = wl.mixed_smooth(7, seed=12) + [uniform(8, 1, 1), uniform(9, 300, 1), uniform(10, 2, 611)]
+    n = len(imgs)
+    dev = torch.device("cuda:0")
+    # one pinned arena, images in reverse order at 128-byte aligned starts with odd gaps
+    starts, at = [], 0
+    for k, im in enumerate(reversed(imgs)):
+        starts.append(at)
+        at += -(-(im.nbytes + 16) // 128) * 128 + 128 * (k % 3)
+    starts.reverse()
+    arena = torch.full((at,), 0x5A, dtype=torch.uint8).pin_memory()
+    assert arena.data_ptr() % 128 == 0
+    pinned = []
+    for im, s0 in zip(imgs, starts):
+        view = arena[s0:s0 + im.nbytes].view(im.shape)
+        view.copy_(torch.from_numpy(im))
+        pinned.append(view)
+    th = torch.zeros(n * 16, dtype=torch.uint8).pin_memory()
+    oh = torch.zeros((n, 3, 224, 224), dtype=torch.float16).pin_memory()
+    dtab = torch.empty(n * 16, dtype=torch.uint8, device=dev)
+    dout = torch.empty((n, 3, 224, 224), dtype=torch.float16, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    call = pb.PreparedImages(pinned, th, oh, None, dtab, dout, 224, 256, MEAN, STD, pb.F16,
+                             dev_status=status, in_place=True)
+    call()
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    tab = th.numpy().view(pb.TABLE_DTYPE)
+    assert [int(e["offset"]) for e in tab] == [s0 - min(starts) for s0 in starts]
+    got = oh.numpy().copy()
+    assert_parity(got, oracle_f64(imgs, 224, 256), pb.F16)
+    want = run_gpu(imgs, 224, 256, out_dtype=pb.F16)
+    assert np.array_equal(got.view(np.uint16), want.view(np.uint16))
+    assert bool((arena[at - 16:] == 0x5A).all()), "the kernel must not write to its input"
+    # images in pageable memory: refused, nothing launched
+    pageable = pb.PreparedImages([np.ascontiguousarray(im) for im in imgs if im.ctypes.data % 128 == 0]
+                                 or [np.zeros((128, 128, 3), dtype=np.uint8)],
+                                 th, oh, None, dtab, dout, 224, 256, MEAN, STD, pb.F16, in_place=True)
+    with pytest.raises(pb.PrebaError) as exc:
+        pageable()
+    assert exc.value.code == pb.ERR_INVALID_ARG
