@@ -18,21 +18,23 @@ import numpy as np
 
 _HERE = Path(__file__).resolve().parent
 _SRC = _HERE / "preba_oracle.c"
+_SRC_VARIANTS = _HERE / "preba_oracle_variants.c"
 _LIB = _HERE / "liboracle.so"
 
 PACK_ALIGN = 128
-OUT_F64, OUT_F32, OUT_F16, OUT_BF16 = 0, 1, 2, 3
+OUT_F64, OUT_F32, OUT_F16, OUT_BF16, OUT_U8_HWC = 0, 1, 2, 3, 4
 
 _lib = None
 
 
 def build(force: bool = False) -> Path:
     """Compile the oracle (gcc -O2, no fast-math) if the library is missing or stale."""
-    if force or not _LIB.exists() or _LIB.stat().st_mtime < _SRC.stat().st_mtime:
+    newest = max(_SRC.stat().st_mtime, _SRC_VARIANTS.stat().st_mtime)
+    if force or not _LIB.exists() or _LIB.stat().st_mtime < newest:
         tmp = _LIB.with_suffix(f".tmp{os.getpid()}.so")
         subprocess.run(
             ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-Wall", "-Wextra",
-             "-o", str(tmp), str(_SRC), "-lm", "-lpthread"],
+             "-o", str(tmp), str(_SRC), str(_SRC_VARIANTS), "-lm", "-lpthread"],
             check=True,
         )
         os.replace(tmp, _LIB)
@@ -65,6 +67,18 @@ def _load():
         lib.oracle_preprocess.argtypes = [u8p, u64p, u32p, u32p, ctypes.c_uint32,
                                           ctypes.c_uint32, ctypes.c_uint32, f32p, f32p,
                                           ctypes.c_int, ctypes.c_void_p, ctypes.c_uint32]
+        lib.oracle_var_axis.argtypes = [ctypes.c_uint32, ctypes.c_uint64, ctypes.c_uint64,
+                                        ctypes.c_uint32, u32p, u32p, u64p, u64p]
+        lib.oracle_var_value.argtypes = [u8p, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32,
+                                         ctypes.c_uint32, ctypes.c_uint64, ctypes.c_uint64,
+                                         ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32, f64p]
+        lib.oracle_var_pixel_u8.argtypes = [u8p, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32,
+                                            ctypes.c_uint32, ctypes.c_uint64, ctypes.c_uint64,
+                                            ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32, u8p]
+        lib.oracle_var_preprocess.argtypes = [u8p, u64p, u32p, u32p, ctypes.c_uint32,
+                                              ctypes.c_uint32, ctypes.c_uint32, f32p, f32p, u32p,
+                                              ctypes.c_int, ctypes.c_int, ctypes.c_void_p,
+                                              ctypes.c_uint32]
         _lib = lib
     return _lib
 
@@ -169,3 +183,50 @@ def preprocess(images: list[np.ndarray], c: int, s: int, mean, std, out_kind: in
     """Pack a list of HWC uint8 images and run the oracle over the batch."""
     packed, offsets, h, w = pack(images)
     return preprocess_packed(packed, offsets, h, w, c, s, mean, std, out_kind, nthreads)
+
+
+# ---- variants: explicit crop origins, rounding to uint8 (preba_oracle_variants.c) ---------------
+
+def var_axis(n_in: int, r: int, origin: int, j: int) -> tuple[int, int, int, int]:
+    """Taps (i0, i1), remainder and denominator for resized index origin + j along one axis."""
+    i0, i1 = ctypes.c_uint32(), ctypes.c_uint32()
+    rem, den = ctypes.c_uint64(), ctypes.c_uint64()
+    _check(_load().oracle_var_axis(n_in, r, origin, j, ctypes.byref(i0), ctypes.byref(i1),
+                                   ctypes.byref(rem), ctypes.byref(den)), "var_axis")
+    return i0.value, i1.value, rem.value, den.value
+
+
+def var_pixel_u8(img: np.ndarray, c: int, s: int, top: int, left: int, ch: int, k: int,
+                 j: int) -> int:
+    """Rounded (ties up) bilinear pixel of one HWC uint8 image for a window at (top, left)."""
+    img = np.ascontiguousarray(img, dtype=np.uint8)
+    h, w, _ = img.shape
+    q = ctypes.c_uint8()
+    _check(_load().oracle_var_pixel_u8(_ptr(img, ctypes.c_uint8), h, w, c, s, top, left, ch, k, j,
+                                       ctypes.byref(q)), "var_pixel_u8")
+    return q.value
+
+
+def preprocess_ex(images: list[np.ndarray], c: int, s: int, mean, std, out_kind: int = OUT_F64,
+                  crop_origin=None, round_u8: bool = False, nthreads: int = 1) -> np.ndarray:
+    """The batch with an explicit crop origin per image (``crop_origin``: n pairs (top, left)
+    on the resized grid, None = centre) and/or rounding of the resized pixel to uint8.
+    Float kinds give [n,3,c,c]; OUT_U8_HWC gives the rounded pixels as [n,c,c,3] uint8."""
+    packed, offsets, h, w = pack(images)
+    n = len(images)
+    if out_kind == OUT_U8_HWC:
+        out = np.empty((n, c, c, 3), dtype=np.uint8)
+    else:
+        dt = {OUT_F64: np.float64, OUT_F32: np.float32, OUT_F16: np.uint16,
+              OUT_BF16: np.uint16}[out_kind]
+        out = np.empty((n, 3, c, c), dtype=dt)
+    m, sd = _f3(mean), _f3(std)
+    co = None
+    if crop_origin is not None:
+        co = np.ascontiguousarray(np.asarray(crop_origin, dtype=np.uint32).reshape(n, 2))
+    _check(_load().oracle_var_preprocess(
+        _ptr(packed, ctypes.c_uint8), _ptr(offsets, ctypes.c_uint64), _ptr(h, ctypes.c_uint32),
+        _ptr(w, ctypes.c_uint32), n, c, s, _ptr(m, ctypes.c_float), _ptr(sd, ctypes.c_float),
+        _ptr(co, ctypes.c_uint32) if co is not None else None, int(round_u8), out_kind,
+        out.ctypes.data_as(ctypes.c_void_p), nthreads), "preprocess_ex")
+    return out.view(np.float16) if out_kind == OUT_F16 else out

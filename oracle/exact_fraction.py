@@ -49,3 +49,27 @@ def preprocess(img, c: int, s: int, mean, std) -> list:
     xs = [sample_coord(w, rw, c, j) for j in range(c)]
     return [[[(bilinear(img, h, w, ys[k], xs[j], ch) / 255 - mean[ch]) / std[ch]
               for j in range(c)] for k in range(c)] for ch in range(3)]
+
+
+def sample_coord_at(n_in: int, r: int, X: int) -> Fraction:
+    """Source coordinate of resized index X along one axis (centre of resized pixel X)."""
+    sx = Fraction(2 * X + 1, 2) * Fraction(n_in, r) - Fraction(1, 2)
+    return min(max(sx, Fraction(0)), Fraction(n_in - 1))
+
+
+def resized_pixels(img, c: int, s: int, top: int | None = None, left: int | None = None) -> list:
+    """v[k][j][ch] as Fractions: the bilinear value at the c x c window whose first resized
+    row/column is (top, left) (centre crop when None), before any rounding or normalisation."""
+    h, w = len(img), len(img[0])
+    rh, rw = resized_size(h, w, s)
+    top = (rh - c) // 2 if top is None else top
+    left = (rw - c) // 2 if left is None else left
+    assert top + c <= rh and left + c <= rw
+    ys = [sample_coord_at(h, rh, top + k) for k in range(c)]
+    xs = [sample_coord_at(w, rw, left + j) for j in range(c)]
+    return [[[bilinear(img, h, w, ys[k], xs[j], ch) for ch in range(3)]
+             for j in range(c)] for k in range(c)]
+
+
+def round_half_up(v: Fraction) -> int:
+    return floor(v + Fraction(1, 2))
