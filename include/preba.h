@@ -50,11 +50,17 @@ extern "C" {
 #define PREBA_ERR_CUDA (-4)             /* a CUDA runtime call failed; see preba_last_cuda_error */
 #define PREBA_ERR_TIMEOUT (-5)          /* only in the device status word: a bounded wait ran out */
 #define PREBA_ERR_TOO_LARGE (-6)        /* the batch exceeds PREBA_NOALLOC_MAX_BYTES */
+#define PREBA_ERR_BAD_CROP (-7)         /* a crop window does not lie on its image's resized grid */
 
 /* Device memory the library itself carries for preba_preprocess_host_noalloc (64 MiB). */
 #define PREBA_NOALLOC_MAX_BYTES (64u << 20)
 
-typedef enum { PREBA_F32 = 0, PREBA_F16 = 1, PREBA_BF16 = 2 } preba_dtype_t;
+typedef enum {
+  PREBA_F32 = 0,
+  PREBA_F16 = 1,
+  PREBA_BF16 = 2,
+  PREBA_U8 = 3 /* preba_preprocess_ex only: the rounded pixel itself, uint8, HWC */
+} preba_dtype_t;
 
 /* One image of the packed batch: `offset` is in bytes from the start of the
  * pixel buffer and a multiple of PREBA_PACK_ALIGN; the image is h rows of w
@@ -194,6 +200,44 @@ int preba_pack(const uint8_t* const* images, const uint32_t* h, const uint32_t* 
  */
 int preba_preprocess(const preba_batch_t* batch, uint32_t out_size, uint32_t resize_short,
                      const float mean[3], const float std[3], int out_dtype, void* stream);
+
+/* preba_options_t.flags */
+#define PREBA_EX_ROUND_U8 1u /* round the interpolated value to the nearest integer (ties up,
+                                decided in exact integer arithmetic) before normalising, as a
+                                pipeline that resizes into a uint8 image does */
+
+typedef struct {
+  uint32_t out_size;      /* crop side C */
+  uint32_t resize_short;  /* resized length S of the shorter side */
+  float mean[3];          /* as preba_preprocess (ignored for PREBA_U8) */
+  float std[3];
+  int32_t out_dtype;      /* PREBA_F32, PREBA_F16, PREBA_BF16: [n,3,C,C] planar;
+                             PREBA_U8 (needs PREBA_EX_ROUND_U8): [n,C,C,3] uint8, no normalisation */
+  uint32_t flags;         /* 0 or PREBA_EX_ROUND_U8 */
+  const uint32_t* crop_origin;      /* DEVICE, 2n values: (top, left) of image i's window on its
+                                       resized grid, top + C <= R_h, left + C <= R_w; NULL: the
+                                       centre crop floor((R - C)/2) */
+  const uint32_t* crop_origin_host; /* HOST copy for checking before launch (with
+                                       batch->table_host), or NULL */
+} preba_options_t;
+
+/*
+ * preba_preprocess_ex — the transform with the adjustments other models ask of the same
+ * Resize / Crop / Normalize units (paper Sec. 4.2, "Flexible design based on reconfigurable
+ * hardware": preprocessing differs between models only by incremental changes): a crop
+ * window per image instead of the centre crop, rounding of the resized pixel to uint8
+ * before normalisation, and the rounded uint8 crop itself as output.  Sampling geometry,
+ * resized size, batch layout, status word, scratch and flags are those of preba_preprocess;
+ * one kernel is enqueued on `stream`.
+ * With PREBA_EX_ROUND_U8 the pixel is floor(v + 1/2) of the exact bilinear value v (a ratio
+ * of integers), so the uint8 output is reproducible bit for bit; images whose resized size
+ * makes 511 * 4 * R_h * R_w reach 2^32 take a slower exact path.
+ * A window that does not fit is refused before launch when the host copies are given
+ * (PREBA_ERR_BAD_CROP); the kernel checks again, skips such an image and stores
+ * PREBA_ERR_BAD_CROP in the status word.
+ * Errors: as preba_preprocess, and PREBA_ERR_BAD_CROP.
+ */
+int preba_preprocess_ex(const preba_batch_t* batch, const preba_options_t* opt, void* stream);
 
 /*
  * preba_preprocess_host — the same transform for a batch held in host memory

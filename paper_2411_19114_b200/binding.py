@@ -16,8 +16,9 @@ _LIB_PATH = Path(__file__).resolve().parent / "libpreba.so"
 PACK_ALIGN = 128
 SCRATCH_BYTES = 256
 IMAGES_IN_PLACE = 1
+EX_ROUND_U8 = 1
 OVERLAP_PREVIOUS = 1
-F32, F16, BF16 = 0, 1, 2
+F32, F16, BF16, U8 = 0, 1, 2, 3
 
 OK = 0
 ERR_INVALID_ARG = -1
@@ -26,9 +27,11 @@ ERR_BAD_TABLE = -3
 ERR_CUDA = -4
 ERR_TIMEOUT = -5
 ERR_TOO_LARGE = -6
+ERR_BAD_CROP = -7
 NOALLOC_MAX_BYTES = 64 << 20
 
-EXPORTS = ("preba_query", "preba_pack", "preba_preprocess", "preba_preprocess_host", "preba_preprocess_images",
+EXPORTS = ("preba_query", "preba_pack", "preba_preprocess", "preba_preprocess_ex", "preba_preprocess_host",
+           "preba_preprocess_images",
            "preba_preprocess_host_noalloc", "preba_preprocess_repeated", "preba_selftest_wait_limit",
            "preba_strerror",
            "preba_last_cuda_error",
@@ -61,6 +64,13 @@ class PrebaHostBatch(ctypes.Structure):
                 ("out_bytes", ctypes.c_uint64), ("dev_pixels", ctypes.c_void_p),
                 ("dev_table", ctypes.c_void_p), ("dev_out", ctypes.c_void_p),
                 ("dev_status", ctypes.c_void_p), ("dev_scratch", ctypes.c_void_p)]
+
+
+class PrebaOptions(ctypes.Structure):
+    _fields_ = [("out_size", ctypes.c_uint32), ("resize_short", ctypes.c_uint32),
+                ("mean", ctypes.c_float * 3), ("std", ctypes.c_float * 3),
+                ("out_dtype", ctypes.c_int32), ("flags", ctypes.c_uint32),
+                ("crop_origin", ctypes.c_void_p), ("crop_origin_host", ctypes.c_void_p)]
 
 
 class PrebaImageBatch(ctypes.Structure):
@@ -107,6 +117,9 @@ def lib() -> ctypes.CDLL:
         L.preba_preprocess_host.argtypes = [ctypes.POINTER(PrebaHostBatch), ctypes.c_uint32,
                                             ctypes.c_uint32, f32p, f32p, ctypes.c_int,
                                             ctypes.c_void_p]
+        L.preba_preprocess_ex.argtypes = [ctypes.POINTER(PrebaBatch), ctypes.POINTER(PrebaOptions),
+                                          ctypes.c_void_p]
+        L.preba_preprocess_ex.restype = ctypes.c_int
         L.preba_preprocess_images.argtypes = [ctypes.POINTER(PrebaImageBatch), ctypes.c_uint32,
                                               ctypes.c_uint32, f32p, f32p, ctypes.c_int,
                                               ctypes.c_void_p]
@@ -239,6 +252,46 @@ def preba_preprocess(pixels, table, n: int, out, out_size: int, resize_short: in
                                 ctypes.c_void_p(stream))
     if rc != OK:
         raise PrebaError(rc, "preba_preprocess")
+
+
+def preba_preprocess_ex(pixels, table, n: int, out, out_size: int, resize_short: int, mean, std,
+                        out_dtype: int, round_u8: bool = False, crop_origin=None,
+                        crop_origin_host: np.ndarray | None = None, stream=None,
+                        table_host: np.ndarray | None = None, status=None, scratch=None,
+                        flags: int = 0) -> None:
+    """``preba_preprocess`` with a crop window per image (``crop_origin``: CUDA int32/uint32
+    tensor of 2n values (top, left); ``crop_origin_host``: uint32 array for the host check) and
+    optional rounding of the resized pixel to uint8 (``out_dtype`` U8 writes it as [n,C,C,3])."""
+    import torch
+
+    if stream is None:
+        stream = torch.cuda.current_stream().cuda_stream
+    elif hasattr(stream, "cuda_stream"):
+        stream = stream.cuda_stream
+    batch = PrebaBatch()
+    batch.pixels = pixels.data_ptr()
+    batch.pixels_bytes = pixels.numel() * pixels.element_size()
+    batch.table = table.data_ptr()
+    batch.table_host = table_host.ctypes.data if table_host is not None else None
+    batch.n = n
+    batch.out = out.data_ptr()
+    batch.out_bytes = out.numel() * out.element_size()
+    batch.status = status.data_ptr() if status is not None else None
+    batch.scratch = scratch.data_ptr() if scratch is not None else None
+    batch.flags = flags
+    opt = PrebaOptions()
+    opt.out_size, opt.resize_short = out_size, resize_short
+    opt.mean = (ctypes.c_float * 3)(*[float(v) for v in _f3(mean)])
+    opt.std = (ctypes.c_float * 3)(*[float(v) for v in _f3(std)])
+    opt.out_dtype = out_dtype
+    opt.flags = EX_ROUND_U8 if round_u8 else 0
+    opt.crop_origin = crop_origin.data_ptr() if crop_origin is not None else None
+    if crop_origin_host is not None:
+        crop_origin_host = np.ascontiguousarray(crop_origin_host, dtype=np.uint32)
+        opt.crop_origin_host = crop_origin_host.ctypes.data
+    rc = lib().preba_preprocess_ex(ctypes.byref(batch), ctypes.byref(opt), ctypes.c_void_p(stream))
+    if rc != OK:
+        raise PrebaError(rc, "preba_preprocess_ex")
 
 
 class PreparedPreprocess:

@@ -13,7 +13,9 @@ bool dtype_ok(int out_dtype) {
   return out_dtype == PREBA_F32 || out_dtype == PREBA_F16 || out_dtype == PREBA_BF16;
 }
 
-uint32_t dtype_bytes(int out_dtype) { return out_dtype == PREBA_F32 ? 4u : 2u; }
+uint32_t dtype_bytes(int out_dtype) {
+  return out_dtype == PREBA_F32 ? 4u : out_dtype == PREBA_U8 ? 1u : 2u;
+}
 
 uint64_t align_up(uint64_t v, uint64_t a) { return (v + a - 1) / a * a; }
 
@@ -101,6 +103,7 @@ extern "C" const char* preba_strerror(int code) {
     case PREBA_ERR_CUDA: return "CUDA runtime error";
     case PREBA_ERR_TIMEOUT: return "device wait ran out";
     case PREBA_ERR_TOO_LARGE: return "batch exceeds the library's built-in staging space";
+    case PREBA_ERR_BAD_CROP: return "crop window outside the resized image";
     default: return "unknown preba error code";
   }
 }

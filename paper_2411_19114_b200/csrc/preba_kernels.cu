@@ -63,6 +63,11 @@ static_assert(kGroupBytes % 16 == 0, "bulk copies need 16-byte aligned destinati
 
 enum TaskKind : uint32_t { kEnd = 0, kStream = 1, kGather = 2, kSkip = 3 };
 
+// What leaves the vertical stage.  kFloat: the interpolated value, normalised (fp32
+// arithmetic).  kRoundFloat: the value rounded to the nearest integer, ties up, decided in
+// exact integer arithmetic, then normalised.  kU8: that integer itself as uint8, HWC.
+enum Mode : int { kFloat = 0, kRoundFloat = 1, kU8 = 2 };
+
 struct Params {
   const uint8_t* pixels;
   uint64_t pixels_bytes;
@@ -70,6 +75,7 @@ struct Params {
   void* out;
   int32_t* status;
   uint32_t* sched;      // two zeroed words for dynamic task claims, or NULL for static turns
+  const uint32_t* crop; // per image (top, left) of the window on the resized grid, or NULL: centre
   uint32_t n;
   uint32_t C;           // crop side
   uint32_t S;           // resized shorter side
@@ -89,6 +95,12 @@ struct TaskMeta {
   uint32_t stride;        // bytes between staged rows of a group
   uint32_t rows_per_group;
   uint32_t n_list;        // distinct source rows of the slab, ascending
+  uint32_t top, left;     // first row and column of the window on the resized grid
+  // rounded modes: the value of an output pixel is num / dd with dd = den_x * den_y
+  uint32_t deny2;         // 2 * den_y
+  uint32_t dd;            // den_x * den_y
+  uint32_t magic;         // floor(2^(31 + k) / (2 * dd)) with 2^k <= 2 * dd < 2^(k + 1)
+  uint32_t shift;         // k - 1
   uint32_t pad;
   uint64_t src;           // byte offset of the image in the pixel buffer
   uint32_t info[kMaxList];  // per listed row: low byte = byte skew of the staged row,
@@ -265,6 +277,7 @@ constexpr uint32_t kMaxPackedDen = 32768;
 // aligned words are read and shifted; one permute lines up the two taps of two channels for
 // a 16-bit-by-8-bit two-way dot product, whose accumulator input 0x4B000000 makes the sum
 // the bit pattern of 2^23 + sum; the subtraction that removes 2^23 is exact.
+template <int MODE>
 __device__ __forceinline__ void hlerp_row(uint32_t x, uint32_t wgt, float n[3]) {
   const uint32_t addr = x & ~3u;
   const uint32_t sh = x << 3;  // the funnel shift takes it modulo 32
@@ -273,9 +286,15 @@ __device__ __forceinline__ void hlerp_row(uint32_t x, uint32_t wgt, float n[3]) 
   const uint32_t hi = __funnelshift_r(w1, w2, sh);  // G1 B1 .. ..
   const uint32_t rg = __byte_perm(lo, hi, 0x4130);  // R0 R1 G0 G1
   const uint32_t bb = __byte_perm(lo, hi, 0x5252);  // B0 B1 B0 B1
-  n[0] = __uint_as_float(__dp2a_lo(wgt, rg, 0x4B000000u)) - 8388608.0f;
-  n[1] = __uint_as_float(__dp2a_hi(wgt, rg, 0x4B000000u)) - 8388608.0f;
-  n[2] = __uint_as_float(__dp2a_lo(wgt, bb, 0x4B000000u)) - 8388608.0f;
+  if (MODE == kFloat) {
+    n[0] = __uint_as_float(__dp2a_lo(wgt, rg, 0x4B000000u)) - 8388608.0f;
+    n[1] = __uint_as_float(__dp2a_hi(wgt, rg, 0x4B000000u)) - 8388608.0f;
+    n[2] = __uint_as_float(__dp2a_lo(wgt, bb, 0x4B000000u)) - 8388608.0f;
+  } else {  // the rounded modes keep the sums as integers (bit patterns)
+    n[0] = __uint_as_float(__dp2a_lo(wgt, rg, 0u));
+    n[1] = __uint_as_float(__dp2a_hi(wgt, rg, 0u));
+    n[2] = __uint_as_float(__dp2a_lo(wgt, bb, 0u));
+  }
 }
 
 template <typename OutT>
@@ -346,6 +365,133 @@ __device__ __forceinline__ void emit_row(OutT* __restrict__ q, uint32_t plane, u
   }
 }
 
+// The rounded modes keep den_x times the horizontally interpolated value as a whole number
+// (bit pattern of an unsigned integer in the row buffers).  An output pixel is
+// floor(num / dd + 1/2) = floor(t / (2 dd)) with t = 2 num + dd, num = prev * (den_y - rem)
+// + cur * rem.  The quotient (at most 255) comes from a multiply-high by a reciprocal that
+// never overshoots and is one short at most, then one correction by the remainder.
+struct Quant {
+  uint32_t deny2, dd, d2, magic, shift;
+};
+
+__device__ __forceinline__ uint32_t rounded_pixel(uint32_t prev, uint32_t cur, uint32_t w0,
+                                                  uint32_t w1, const Quant& qz) {
+  const uint32_t t = prev * w0 + cur * w1 + qz.dd;  // < 2^32 by the fast path's precondition
+  uint32_t q = __umulhi(t, qz.magic) >> qz.shift;
+  if (t - q * qz.d2 >= qz.d2) ++q;
+  return q;
+}
+
+// Vertical stage of the rounded modes for one output row.  rem is the lower row's integer
+// weight (den_y when both taps are the row just staged).  kRoundFloat: q points at column
+// 2 * lane of plane 0, as in emit_row.  kU8: q points at the first byte of pixel 2 * lane of
+// the output row (HWC); a lane writes its pairs as three 16-bit words each and its single
+// column byte by byte.
+template <typename OutT, bool FULL, int MODE>
+__device__ __forceinline__ void emit_row_rounded(OutT* __restrict__ q, uint32_t plane,
+                                                 uint32_t lane, uint32_t rem,
+                                                 const float (&hp)[kLaneCols][3],
+                                                 const float (&hc)[kLaneCols][3],
+                                                 const Quant& qz, const float (&na)[3],
+                                                 const float (&nb)[3], uint32_t valid) {
+  const uint32_t w1 = 2 * rem, w0 = qz.deny2 - w1;
+  uint32_t px[kLaneCols][3];
+#pragma unroll
+  for (int m = 0; m < static_cast<int>(kLaneCols); ++m)
+#pragma unroll
+    for (int ch = 0; ch < 3; ++ch)
+      px[m][ch] = rounded_pixel(__float_as_uint(hp[m][ch]), __float_as_uint(hc[m][ch]), w0, w1, qz);
+  if constexpr (MODE == kU8) {
+    uint8_t* b = reinterpret_cast<uint8_t*>(q);
+#pragma unroll
+    for (int pr = 0; pr < 3; ++pr) {
+      const uint32_t (&l)[3] = px[2 * pr];
+      const uint32_t (&r)[3] = px[2 * pr + 1];
+      uint8_t* at = b + 192 * pr;  // 64 pixels further
+      if (FULL) {
+        uint16_t* h16 = reinterpret_cast<uint16_t*>(at);  // even byte offset: 6 * lane + 192 * pr
+        __stcs(h16, static_cast<uint16_t>(l[0] | (l[1] << 8)));
+        __stcs(h16 + 1, static_cast<uint16_t>(l[2] | (r[0] << 8)));
+        __stcs(h16 + 2, static_cast<uint16_t>(r[1] | (r[2] << 8)));
+      } else {
+#pragma unroll
+        for (int ch = 0; ch < 3; ++ch) {
+          if ((valid >> (2 * pr)) & 1u) at[ch] = static_cast<uint8_t>(l[ch]);
+          if ((valid >> (2 * pr + 1)) & 1u) at[3 + ch] = static_cast<uint8_t>(r[ch]);
+        }
+      }
+    }
+    uint8_t* single = b + 3 * (192 - lane);  // pixel 192 + lane
+    if (FULL || ((valid >> 6) & 1u)) {
+#pragma unroll
+      for (int ch = 0; ch < 3; ++ch) single[ch] = static_cast<uint8_t>(px[6][ch]);
+    }
+  } else {
+#pragma unroll
+    for (int ch = 0; ch < 3; ++ch, q += plane) {
+      float o[kLaneCols];
+#pragma unroll
+      for (int m = 0; m < static_cast<int>(kLaneCols); ++m)
+        o[m] = fmaf(__uint_as_float(0x4B000000u | px[m][ch]) - 8388608.0f, na[ch], nb[ch]);
+      OutT* single = q + 192 - lane;
+      if (FULL) {
+#pragma unroll
+        for (int pr = 0; pr < 3; ++pr)
+          __stcs(reinterpret_cast<typename Pack<OutT>::Vec*>(q + 64 * pr),
+                 Pack<OutT>::pair(o[2 * pr], o[2 * pr + 1]));
+        __stcs(single, Pack<OutT>::one(o[6]));
+      } else {
+#pragma unroll
+        for (int m = 0; m < 6; ++m)
+          if ((valid >> m) & 1u) q[64 * (m >> 1) + (m & 1)] = Pack<OutT>::one(o[m]);
+        if ((valid >> 6) & 1u) *single = Pack<OutT>::one(o[6]);
+      }
+    }
+  }
+}
+
+// One axis in 64-bit integers: tap, clamped neighbour, remainder and denominator (the direct
+// path of the rounded modes, any size the interface admits).
+struct TapInt {
+  uint32_t i0, i1;
+  uint64_t rem, den;
+};
+
+__device__ __forceinline__ TapInt axis_tap_int(uint32_t in, uint32_t r, uint32_t origin,
+                                               uint32_t j) {
+  TapInt t;
+  t.den = 2ull * r;
+  const uint64_t pos = (2 * (static_cast<uint64_t>(origin) + j) + 1) * in;
+  uint64_t num = pos > r ? pos - r : 0;
+  const uint64_t hi = static_cast<uint64_t>(in - 1) * t.den;
+  num = num < hi ? num : hi;
+  const uint64_t q = num / t.den;
+  t.i0 = static_cast<uint32_t>(q);
+  t.i1 = t.i0 + 1 < in ? t.i0 + 1 : in - 1;
+  t.rem = num - q * t.den;
+  return t;
+}
+
+// The rounded pixel from its four taps, exact at any size (products pass 2^64).
+__device__ __forceinline__ uint32_t rounded_pixel_wide(uint32_t p00, uint32_t p01, uint32_t p10,
+                                                       uint32_t p11, const TapInt& tx,
+                                                       const TapInt& ty) {
+  typedef unsigned __int128 u128;
+  const u128 upper = static_cast<u128>(p00) * (tx.den - tx.rem) + static_cast<u128>(p01) * tx.rem;
+  const u128 lower = static_cast<u128>(p10) * (tx.den - tx.rem) + static_cast<u128>(p11) * tx.rem;
+  const u128 num = upper * (ty.den - ty.rem) + lower * ty.rem;
+  const u128 den = static_cast<u128>(tx.den) * ty.den;
+  // the quotient is at most 255: find it by comparison instead of a 128-bit division
+  const u128 t = 2 * num + den, d2 = 2 * den;
+  uint32_t q = 0;
+#pragma unroll 1
+  for (int bit = 7; bit >= 0; --bit) {
+    const uint32_t trial = q | (1u << bit);
+    if (static_cast<u128>(trial) * d2 <= t) q = trial;
+  }
+  return q;
+}
+
 // ---- task preparation: geometry of a slab into the warp's meta buffer --------------------------
 
 struct Issue {          // the copy stream's view of the task it is issuing
@@ -359,6 +505,7 @@ struct Issue {          // the copy stream's view of the task it is issuing
 };
 
 // Fills `m` for task `task`; returns its kind.  All lanes take part.
+template <int MODE>
 __device__ __forceinline__ uint32_t prepare(const Params& p, uint32_t task, TaskMeta& m,
                                             uint32_t lane, Issue& is) {
   const uint32_t C = p.C;
@@ -375,7 +522,14 @@ __device__ __forceinline__ uint32_t prepare(const Params& p, uint32_t task, Task
     const uint32_t rl = p.S * lng / sht;
     const uint32_t rh = e.h <= e.w ? p.S : rl;
     const uint32_t rw = e.h <= e.w ? rl : p.S;
-    const uint32_t top = (rh - C) / 2, left = (rw - C) / 2;
+    uint32_t top = (rh - C) / 2, left = (rw - C) / 2;  // rh, rw >= S >= C
+    bool window_ok = true;
+    if (p.crop) {
+      const uint32_t t = p.crop[2 * img], l = p.crop[2 * img + 1];
+      window_ok = t <= rh - C && l <= rw - C;
+      top = min(t, rh - C);  // a window that does not fit is reported and skipped below
+      left = min(l, rw - C);
+    }
     const uint32_t k0 = slab * kSlabRows;
     const uint32_t rows_out = min(kSlabRows, C - k0);
     const uint32_t col0 = cb * kTaskCols;
@@ -402,6 +556,10 @@ __device__ __forceinline__ uint32_t prepare(const Params& p, uint32_t task, Task
     const uint64_t end16 = (e.offset + 3ull * e.h * e.w + 15) & ~15ull;
     kind = (rpg >= 1 && end16 <= p.pixels_bytes && ax.small && ax.den <= kMaxPackedDen)
                ? kStream : kGather;
+    // rounded modes: 32-bit arithmetic needs 2 * num + dd <= 511 * dd below 2^32
+    const uint64_t dd = static_cast<uint64_t>(ax.den) * ay.den;
+    if (MODE != kFloat && !(ay.small && 511ull * dd < (1ull << 32))) kind = kGather;
+    if (!window_ok) kind = kSkip;
 
     // rows of the slab: the ascending list of distinct source rows.  Output row `lane`
     // lists its lower tap if that lies beyond the previous row's upper tap, and its upper
@@ -427,8 +585,23 @@ __device__ __forceinline__ uint32_t prepare(const Params& p, uint32_t task, Task
       m.row[at] = ty.i1;
       m.info[at] = (done << 8) | ((3u * (ty.i1 * e.w + xmin)) & 15u);
     }
-    if (active) m.lam[lane] = __float_as_uint(ty.i1 == ty.i0 ? 1.0f : ty.lam);
+    if (MODE == kFloat) {
+      if (active) m.lam[lane] = __float_as_uint(ty.i1 == ty.i0 ? 1.0f : ty.lam);
+    } else {
+      // integer weight of the lower row; all of it when both taps are the row just staged
+      if (active) m.lam[lane] = ty.i1 == ty.i0 ? ay.den : ty.rem;
+      if (lane == 0 && kind == kStream) {
+        const uint32_t d2 = 2 * static_cast<uint32_t>(dd);
+        const uint32_t k = 31 - static_cast<uint32_t>(__clz(d2));
+        m.deny2 = 2 * ay.den;
+        m.dd = static_cast<uint32_t>(dd);
+        m.magic = static_cast<uint32_t>((1ull << (31 + k)) / d2);
+        m.shift = k - 1;
+      }
+    }
     if (lane == 0) {
+      m.top = top;
+      m.left = left;
       m.img = img;
       m.k0 = k0;
       m.rows_out = rows_out;
@@ -449,6 +622,7 @@ __device__ __forceinline__ uint32_t prepare(const Params& p, uint32_t task, Task
     is.stride = stride;
     is.rpg = rpg;
     is.n_list = kind == kStream ? n_list : 0;
+    if (!window_ok && lane == 0) report(p.status, PREBA_ERR_BAD_CROP);
   } else {
     if (lane == 0) report(p.status, PREBA_ERR_BAD_TABLE);
     is.n_list = 0;
@@ -458,15 +632,29 @@ __device__ __forceinline__ uint32_t prepare(const Params& p, uint32_t task, Task
   return kind;
 }
 
+template <typename OutT, bool FULL, int MODE>
+__device__ __forceinline__ void emit_any(OutT* __restrict__ q, uint32_t plane, uint32_t lane,
+                                         uint32_t weight_bits,
+                                         const float (&prev)[kLaneCols][3],
+                                         const float (&cur)[kLaneCols][3], const float (&sa)[3],
+                                         const float (&nb)[3], const Quant& qz, uint32_t valid) {
+  if constexpr (MODE == kFloat)
+    emit_row<OutT, FULL>(q, plane, lane, __uint_as_float(weight_bits), prev, cur, sa, nb, valid);
+  else
+    emit_row_rounded<OutT, FULL, MODE>(q, plane, lane, weight_bits, prev, cur, qz, sa, nb, valid);
+}
+
 // ---- the warp program ---------------------------------------------------------------------------------
 
-template <typename OutT>
+template <typename OutT, int MODE>
 __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint32_t lane,
                                           uint32_t gwarp, uint32_t nwarps) {
   const uint32_t C = p.C;
   const uint32_t plane = C * C;
+  const uint32_t row_step = MODE == kU8 ? 3 * C : C;  // elements of OutT between output rows
   const float nb[3] = {p.b[0], p.b[1], p.b[2]};
   float sa[3] = {0.f, 0.f, 0.f};  // staged path: 1 / (255 * std * den) of the task's image
+  Quant qz = {0, 0, 0, 0, 0};     // rounded modes: the task's division constants
 
   // task claims: a warp's first task is its own index; later ones come from the shared
   // counter (dynamic) or every nwarps-th task (static)
@@ -550,7 +738,7 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
           ended = true;
           is.n_list = 0;
         } else {
-          (void)prepare(p, task, ws.meta[buf], lane, is);
+          (void)prepare<MODE>(p, task, ws.meta[buf], lane, is);
         }
         is.buf = buf;
         is_row = 0;
@@ -569,7 +757,7 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
         continue;
       }
       const uint32_t w = cm->w, rw = cm->rw, col0 = cm->col0, xmin = cm->xmin;
-      const Axis ax = make_axis(w, rw, (rw - C) / 2, C);
+      const Axis ax = make_axis(w, rw, cm->left, C);
       ln.valid = 0;
       if (kind == kStream) {  // implies ax.small and den <= kMaxPackedDen
 #pragma unroll
@@ -580,9 +768,19 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
           ln.off[m] = 3 * (t.i0 - xmin);
           ln.wgt[m] = (ax.den - t.rem) | (t.rem << 16);
         }
-        // staged rows carry den times the pixel value: fold 1 / den into the scale
+        if (MODE == kFloat) {
+          // staged rows carry den times the pixel value: fold 1 / den into the scale
 #pragma unroll
-        for (int ch = 0; ch < 3; ++ch) sa[ch] = p.a[ch] * ax.rden;
+          for (int ch = 0; ch < 3; ++ch) sa[ch] = p.a[ch] * ax.rden;
+        } else {
+          qz.deny2 = cm->deny2;
+          qz.dd = cm->dd;
+          qz.d2 = 2 * qz.dd;
+          qz.magic = cm->magic;
+          qz.shift = cm->shift;
+#pragma unroll
+          for (int ch = 0; ch < 3; ++ch) sa[ch] = p.a[ch];
+        }
       } else {
 #pragma unroll
         for (int m = 0; m < static_cast<int>(kLaneCols); ++m) {
@@ -594,22 +792,63 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
         }
       }
       full = (C & 1u) == 0 && __all_sync(0xffffffffu, ln.valid == 0x7fu);
-      q_out = static_cast<OutT*>(p.out) + static_cast<size_t>(cm->img) * 3 * plane +
-              (cm->k0 * C + col0 + 2 * lane);
+      if (MODE == kU8)  // HWC: first byte of pixel col0 + 2 * lane in row k0
+        q_out = static_cast<OutT*>(p.out) +
+                3 * (static_cast<size_t>(cm->img) * plane + (cm->k0 * C + col0 + 2 * lane));
+      else
+        q_out = static_cast<OutT*>(p.out) + static_cast<size_t>(cm->img) * 3 * plane +
+                (cm->k0 * C + col0 + 2 * lane);
       c_nlist = cm->n_list;
       c_rpg = cm->rows_per_group;
       c_stride = cm->stride;
       c_row = 0;
       t_out = 0;
       need_task = false;
-      if (kind == kGather) {
+      if (kind != kGather) {
+        // staged: the groups follow
+      } else if constexpr (MODE != kFloat) {
+        // direct path of the rounded modes: exact integers of any size, taps from global memory
+        const uint8_t* __restrict__ src = p.pixels + cm->src;
+        const size_t pitch = 3 * static_cast<size_t>(w);
+        const uint32_t h = cm->h, rh = cm->rh;
+        for (uint32_t t = 0; t < cm->rows_out; ++t) {
+          const TapInt ty = axis_tap_int(h, rh, cm->top, cm->k0 + t);
+          const uint8_t* r0 = src + ty.i0 * pitch;
+          const uint8_t* r1 = src + ty.i1 * pitch;
+#pragma unroll 1
+          for (int m = 0; m < static_cast<int>(kLaneCols); ++m) {
+            const uint32_t j = col0 + lane_col(lane, m);
+            if (j >= C) continue;
+            const TapInt tx = axis_tap_int(w, rw, cm->left, j);
+#pragma unroll 1
+            for (uint32_t ch = 0; ch < 3; ++ch) {
+              const uint32_t v = rounded_pixel_wide(
+                  __ldg(r0 + 3 * static_cast<size_t>(tx.i0) + ch),
+                  __ldg(r0 + 3 * static_cast<size_t>(tx.i1) + ch),
+                  __ldg(r1 + 3 * static_cast<size_t>(tx.i0) + ch),
+                  __ldg(r1 + 3 * static_cast<size_t>(tx.i1) + ch), tx, ty);
+              const size_t row = static_cast<size_t>(cm->k0 + t) * C + j;
+              if constexpr (MODE == kU8) {
+                reinterpret_cast<uint8_t*>(p.out)[3 * (static_cast<size_t>(cm->img) * plane + row) +
+                                                  ch] = static_cast<uint8_t>(v);
+              } else {
+                const float o = fmaf(static_cast<float>(v), p.a[ch], p.b[ch]);
+                static_cast<OutT*>(p.out)[(static_cast<size_t>(cm->img) * 3 + ch) * plane + row] =
+                    Pack<OutT>::one(o);
+              }
+            }
+          }
+        }
+        ++finished;
+        need_task = true;
+      } else {
         // direct path: taps straight from global memory (footprint too wide for the ring)
         const uint8_t* __restrict__ src = p.pixels + cm->src + 3 * xmin;
         const size_t pitch = 3 * static_cast<size_t>(w);
         const uint32_t h = cm->h, rh = cm->rh;
-        const Axis ay = make_axis(h, rh, (rh - C) / 2, C);
+        const Axis ay = make_axis(h, rh, cm->top, C);
         const float na[3] = {p.a[0], p.a[1], p.a[2]};
-        for (uint32_t t = 0; t < cm->rows_out; ++t, q_out += C) {
+        for (uint32_t t = 0; t < cm->rows_out; ++t, q_out += row_step) {
           const Tap ty = axis_tap(ay, cm->k0 + t);
           const uint8_t* r0 = src + ty.i0 * pitch;
           const uint8_t* r1 = src + ty.i1 * pitch;
@@ -655,26 +894,26 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
         if (par == 0) {
 #pragma unroll
           for (int m = 0; m < static_cast<int>(kLaneCols); ++m)
-            hlerp_row(base + ln.off[m], ln.wgt[m], hA[m]);
+            hlerp_row<MODE>(base + ln.off[m], ln.wgt[m], hA[m]);
 #pragma unroll 1
-          for (; e > 0; --e, ++t_out, q_out += C) {
-            const float ly = __uint_as_float(cm->lam[t_out]);
+          for (; e > 0; --e, ++t_out, q_out += row_step) {
+            const uint32_t wy = cm->lam[t_out];
             if (full)
-              emit_row<OutT, true>(q_out, plane, lane, ly, hB, hA, sa, nb, ln.valid);
+              emit_any<OutT, true, MODE>(q_out, plane, lane, wy, hB, hA, sa, nb, qz, ln.valid);
             else
-              emit_row<OutT, false>(q_out, plane, lane, ly, hB, hA, sa, nb, ln.valid);
+              emit_any<OutT, false, MODE>(q_out, plane, lane, wy, hB, hA, sa, nb, qz, ln.valid);
           }
         } else {
 #pragma unroll
           for (int m = 0; m < static_cast<int>(kLaneCols); ++m)
-            hlerp_row(base + ln.off[m], ln.wgt[m], hB[m]);
+            hlerp_row<MODE>(base + ln.off[m], ln.wgt[m], hB[m]);
 #pragma unroll 1
-          for (; e > 0; --e, ++t_out, q_out += C) {
-            const float ly = __uint_as_float(cm->lam[t_out]);
+          for (; e > 0; --e, ++t_out, q_out += row_step) {
+            const uint32_t wy = cm->lam[t_out];
             if (full)
-              emit_row<OutT, true>(q_out, plane, lane, ly, hA, hB, sa, nb, ln.valid);
+              emit_any<OutT, true, MODE>(q_out, plane, lane, wy, hA, hB, sa, nb, qz, ln.valid);
             else
-              emit_row<OutT, false>(q_out, plane, lane, ly, hA, hB, sa, nb, ln.valid);
+              emit_any<OutT, false, MODE>(q_out, plane, lane, wy, hA, hB, sa, nb, qz, ln.valid);
           }
         }
         par ^= 1u;
@@ -706,7 +945,7 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
   }
 }
 
-template <typename OutT>
+template <typename OutT, int MODE>
 __global__ void __launch_bounds__(kThreads, kCtasPerSm) preba_fused_kernel(const Params p) {
   __shared__ WarpShared sm[kWarpsPerCta];
   // a following launch that was marked independent of this one may start as soon as
@@ -722,16 +961,16 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) preba_fused_kernel(const
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncwarp();
-  warp_main<OutT>(p, ws, lane, blockIdx.x * kWarpsPerCta + warp, gridDim.x * kWarpsPerCta);
+  warp_main<OutT, MODE>(p, ws, lane, blockIdx.x * kWarpsPerCta + warp, gridDim.x * kWarpsPerCta);
 }
 
 thread_local int g_last_cuda_error = 0;
 
 int check_args(const uint8_t* pixels, uint64_t pixels_bytes, const void* table, uint32_t n,
                const void* out, uint64_t out_bytes, uint32_t out_size, uint32_t resize_short,
-               const float mean[3], const float std[3], int out_dtype) {
+               const float mean[3], const float std[3], int out_dtype, bool allow_u8 = false) {
   if (!pixels || !table || !out || !mean || !std || n == 0) return PREBA_ERR_INVALID_ARG;
-  if (!dtype_ok(out_dtype) || out_size == 0 || resize_short < out_size ||
+  if (!(dtype_ok(out_dtype) || (allow_u8 && out_dtype == PREBA_U8)) || out_size == 0 || resize_short < out_size ||
       resize_short > PREBA_MAX_RESIZE)
     return PREBA_ERR_INVALID_ARG;
   for (int c = 0; c < 3; ++c)
@@ -760,41 +999,56 @@ int check_table(const preba_img_t* t, uint32_t n, uint64_t pixels_bytes) {
   return PREBA_OK;
 }
 
+// The kernel for an output type and mode.
+using KernelFn = void (*)(const Params);
+constexpr int kVariants = 7;
+
+int variant_of(int out_dtype, int mode) {
+  if (mode == kU8) return 6;
+  const int t = out_dtype == PREBA_F16 ? 1 : out_dtype == PREBA_BF16 ? 2 : 0;
+  return (mode == kRoundFloat ? 3 : 0) + t;
+}
+
+KernelFn kernel_of(int variant) {
+  switch (variant) {
+    case 1: return preba_fused_kernel<__half, kFloat>;
+    case 2: return preba_fused_kernel<__nv_bfloat16, kFloat>;
+    case 3: return preba_fused_kernel<float, kRoundFloat>;
+    case 4: return preba_fused_kernel<__half, kRoundFloat>;
+    case 5: return preba_fused_kernel<__nv_bfloat16, kRoundFloat>;
+    case 6: return preba_fused_kernel<uint8_t, kU8>;
+    default: return preba_fused_kernel<float, kFloat>;
+  }
+}
+
 // Resident CTAs of the fused kernel on the current device (grid of a persistent launch).
 // The answer depends on the device and the kernel only; it is computed once per device and
-// output type and kept (a benign race: concurrent first calls store the same value).
-int resident_ctas(int out_dtype, cudaError_t* err) {
+// kernel variant and kept (a benign race: concurrent first calls store the same value).
+int resident_ctas(int variant, cudaError_t* err) {
   constexpr int kMaxDevices = 64;
-  static std::atomic<int> cache[3][kMaxDevices];
+  static std::atomic<int> cache[kVariants][kMaxDevices];
   int dev = 0;
   *err = cudaGetDevice(&dev);
   if (*err != cudaSuccess) return 0;
-  const int kind = out_dtype == PREBA_F16 ? 1 : out_dtype == PREBA_BF16 ? 2 : 0;
   if (dev >= 0 && dev < kMaxDevices) {
-    const int known = cache[kind][dev].load(std::memory_order_relaxed);
+    const int known = cache[variant][dev].load(std::memory_order_relaxed);
     if (known > 0) return known;
   }
   int sms = 0, per_sm = 0;
   *err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   if (*err != cudaSuccess) return 0;
-  if (kind == 1)
-    *err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, preba_fused_kernel<__half>,
-                                                         kThreads, 0);
-  else if (kind == 2)
-    *err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(
-        &per_sm, preba_fused_kernel<__nv_bfloat16>, kThreads, 0);
-  else
-    *err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, preba_fused_kernel<float>,
-                                                         kThreads, 0);
+  *err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel_of(variant), kThreads, 0);
   if (*err != cudaSuccess) return 0;
   const int resident = sms * (per_sm > 0 ? per_sm : 1);
-  if (dev >= 0 && dev < kMaxDevices) cache[kind][dev].store(resident, std::memory_order_relaxed);
+  if (dev >= 0 && dev < kMaxDevices)
+    cache[variant][dev].store(resident, std::memory_order_relaxed);
   return resident;
 }
 
-int launch(const Params& p, int out_dtype, bool overlap, cudaStream_t stream) {
+int launch(const Params& p, int out_dtype, bool overlap, cudaStream_t stream, int mode = kFloat) {
   cudaError_t err = cudaSuccess;
-  const int resident = resident_ctas(out_dtype, &err);
+  const int variant = variant_of(out_dtype, mode);
+  const int resident = resident_ctas(variant, &err);
   if (err == cudaSuccess) {
     const uint32_t want = (p.tasks + kWarpsPerCta - 1) / kWarpsPerCta;
     const uint32_t blocks = want < static_cast<uint32_t>(resident) ? want : resident;
@@ -808,12 +1062,7 @@ int launch(const Params& p, int out_dtype, bool overlap, cudaStream_t stream) {
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = overlap ? 1 : 0;
-    if (out_dtype == PREBA_F16)
-      err = cudaLaunchKernelEx(&cfg, preba_fused_kernel<__half>, p);
-    else if (out_dtype == PREBA_BF16)
-      err = cudaLaunchKernelEx(&cfg, preba_fused_kernel<__nv_bfloat16>, p);
-    else
-      err = cudaLaunchKernelEx(&cfg, preba_fused_kernel<float>, p);
+    err = cudaLaunchKernelEx(&cfg, kernel_of(variant), p);
   }
   if (err != cudaSuccess) {
     g_last_cuda_error = static_cast<int>(err);
@@ -835,6 +1084,7 @@ Params make_params(const uint8_t* pixels, uint64_t pixels_bytes, const preba_img
   p.C = out_size;
   p.S = resize_short;
   p.sched = scratch;
+  p.crop = nullptr;
   p.slabs = (out_size + kSlabRows - 1) / kSlabRows;
   p.col_blocks = (out_size + kTaskCols - 1) / kTaskCols;
   p.tasks = static_cast<uint32_t>(static_cast<uint64_t>(n) * p.slabs * p.col_blocks);
@@ -867,6 +1117,44 @@ extern "C" int preba_preprocess(const preba_batch_t* batch, uint32_t out_size,
                                mean, std);
   return launch(p, out_dtype, (batch->flags & PREBA_OVERLAP_PREVIOUS) != 0,
                 static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int preba_preprocess_ex(const preba_batch_t* batch, const preba_options_t* opt,
+                                   void* stream) {
+  using namespace preba;
+  if (!batch || !opt) return PREBA_ERR_INVALID_ARG;
+  if (opt->flags & ~PREBA_EX_ROUND_U8) return PREBA_ERR_INVALID_ARG;
+  const bool round_u8 = (opt->flags & PREBA_EX_ROUND_U8) != 0;
+  if (opt->out_dtype == PREBA_U8 && !round_u8) return PREBA_ERR_INVALID_ARG;
+  int rc = check_args(batch->pixels, batch->pixels_bytes, batch->table, batch->n, batch->out,
+                      batch->out_bytes, opt->out_size, opt->resize_short, opt->mean, opt->std,
+                      opt->out_dtype, true);
+  if (rc != PREBA_OK) return rc;
+  if (reinterpret_cast<uintptr_t>(batch->scratch) % 16) return PREBA_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(opt->crop_origin) % 4) return PREBA_ERR_INVALID_ARG;
+  if (batch->flags & ~PREBA_OVERLAP_PREVIOUS) return PREBA_ERR_INVALID_ARG;
+  if (batch->table_host) {
+    rc = check_table(batch->table_host, batch->n, batch->pixels_bytes);
+    if (rc != PREBA_OK) return rc;
+    if (opt->crop_origin_host) {
+      // every window must lie on its image's resized grid
+      for (uint32_t i = 0; i < batch->n; ++i) {
+        const uint64_t h = batch->table_host[i].h, w = batch->table_host[i].w;
+        const uint64_t rl = opt->resize_short * (h > w ? h : w) / (h > w ? w : h);
+        const uint64_t rh = h <= w ? opt->resize_short : rl, rw = h <= w ? rl : opt->resize_short;
+        if (opt->crop_origin_host[2 * i] + static_cast<uint64_t>(opt->out_size) > rh ||
+            opt->crop_origin_host[2 * i + 1] + static_cast<uint64_t>(opt->out_size) > rw)
+          return PREBA_ERR_BAD_CROP;
+      }
+    }
+  }
+  Params p = make_params(batch->pixels, batch->pixels_bytes, batch->table, batch->n, batch->out,
+                         batch->status, batch->scratch, opt->out_size, opt->resize_short,
+                         opt->mean, opt->std);
+  p.crop = opt->crop_origin;
+  const int mode = opt->out_dtype == PREBA_U8 ? kU8 : (round_u8 ? kRoundFloat : kFloat);
+  return launch(p, opt->out_dtype, (batch->flags & PREBA_OVERLAP_PREVIOUS) != 0,
+                static_cast<cudaStream_t>(stream), mode);
 }
 
 extern "C" int preba_preprocess_host(const preba_host_batch_t* b, uint32_t out_size,
