@@ -113,8 +113,8 @@ def test_pack_errors():
 
 
 def test_strerror_covers_every_code():
-    texts = {pb.preba_strerror(c) for c in range(0, -7, -1)}
-    assert len(texts) == 7 and "ok" in texts
+    texts = {pb.preba_strerror(c) for c in range(0, -8, -1)}
+    assert len(texts) == 8 and "ok" in texts
     assert "unknown" in pb.preba_strerror(-99)
 
 
@@ -173,6 +173,36 @@ def test_preprocess_checks_host_table_before_launch():
                 [(0, 8, 8), (1 << 40, 8, 8)]):      # offset past the pixel buffer
         t = table(bad)
         assert _call(_batch(table_host=t.ctypes.data)) == pb.ERR_BAD_TABLE
+
+
+def test_extended_entry_point_rejects_bad_arguments_before_any_launch():
+    def call(batch=None, **kw):
+        b = batch if batch is not None else _batch(out_bytes=2 * 3 * 16 * 16 * 4)
+        o = pb.PrebaOptions()
+        o.out_size, o.resize_short = 16, 16
+        o.mean = (ctypes.c_float * 3)(*MEAN)
+        o.std = (ctypes.c_float * 3)(*STD)
+        o.out_dtype, o.flags = pb.F32, 0
+        for k, v in kw.items():
+            setattr(o, k, v)
+        return pb.lib().preba_preprocess_ex(ctypes.byref(b), ctypes.byref(o), None)
+
+    assert pb.lib().preba_preprocess_ex(None, None, None) == pb.ERR_INVALID_ARG
+    assert call(flags=2) == pb.ERR_INVALID_ARG                       # unknown flag
+    assert call(out_dtype=pb.U8) == pb.ERR_INVALID_ARG               # uint8 output needs rounding
+    assert call(out_dtype=4, flags=pb.EX_ROUND_U8) == pb.ERR_INVALID_ARG
+    assert call(out_size=17) == pb.ERR_INVALID_ARG
+    assert call(crop_origin=0x50002) == pb.ERR_INVALID_ARG           # misaligned table of windows
+    assert call(std=(ctypes.c_float * 3)(0.2, 0.0, 0.2)) == pb.ERR_INVALID_ARG
+    assert call(_batch(out_bytes=2 * 16 * 16 * 3 - 1), out_dtype=pb.U8,
+                flags=pb.EX_ROUND_U8) == pb.ERR_BUFFER_TOO_SMALL     # one byte per element
+    # windows checked on the host when both host copies are there: S = 16, C = 16
+    t = np.zeros(2, dtype=pb.TABLE_DTYPE)
+    t[0], t[1] = (0, 8, 8), (256, 8, 16)                             # resized 16 x 16 and 16 x 32
+    bad = np.asarray([0, 0, 0, 17], dtype=np.uint32)                 # 17 + 16 > 32
+    b = _batch(out_bytes=2 * 3 * 16 * 16 * 4, table_host=t.ctypes.data)
+    assert call(b, crop_origin=0x50000, crop_origin_host=bad.ctypes.data) == pb.ERR_BAD_CROP
+    assert pb.preba_strerror(pb.ERR_BAD_CROP) != pb.preba_strerror(-99)
 
 
 def test_separate_images_entry_point_rejects_bad_arguments_before_any_copy():
