@@ -505,7 +505,7 @@ struct Issue {          // the copy stream's view of the task it is issuing
 };
 
 // Fills `m` for task `task`; returns its kind.  All lanes take part.
-template <int MODE>
+template <int MODE, bool CROP>
 __device__ __forceinline__ uint32_t prepare(const Params& p, uint32_t task, TaskMeta& m,
                                             uint32_t lane, Issue& is) {
   const uint32_t C = p.C;
@@ -524,7 +524,7 @@ __device__ __forceinline__ uint32_t prepare(const Params& p, uint32_t task, Task
     const uint32_t rw = e.h <= e.w ? rl : p.S;
     uint32_t top = (rh - C) / 2, left = (rw - C) / 2;  // rh, rw >= S >= C
     bool window_ok = true;
-    if (p.crop) {
+    if (CROP) {
       const uint32_t t = p.crop[2 * img], l = p.crop[2 * img + 1];
       window_ok = t <= rh - C && l <= rw - C;
       top = min(t, rh - C);  // a window that does not fit is reported and skipped below
@@ -646,7 +646,7 @@ __device__ __forceinline__ void emit_any(OutT* __restrict__ q, uint32_t plane, u
 
 // ---- the warp program ---------------------------------------------------------------------------------
 
-template <typename OutT, int MODE>
+template <typename OutT, int MODE, bool CROP>
 __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint32_t lane,
                                           uint32_t gwarp, uint32_t nwarps) {
   const uint32_t C = p.C;
@@ -738,7 +738,7 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
           ended = true;
           is.n_list = 0;
         } else {
-          (void)prepare<MODE>(p, task, ws.meta[buf], lane, is);
+          (void)prepare<MODE, CROP>(p, task, ws.meta[buf], lane, is);
         }
         is.buf = buf;
         is_row = 0;
@@ -757,7 +757,7 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
         continue;
       }
       const uint32_t w = cm->w, rw = cm->rw, col0 = cm->col0, xmin = cm->xmin;
-      const Axis ax = make_axis(w, rw, cm->left, C);
+      const Axis ax = make_axis(w, rw, CROP ? cm->left : (rw - C) / 2, C);
       ln.valid = 0;
       if (kind == kStream) {  // implies ax.small and den <= kMaxPackedDen
 #pragma unroll
@@ -846,7 +846,7 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
         const uint8_t* __restrict__ src = p.pixels + cm->src + 3 * xmin;
         const size_t pitch = 3 * static_cast<size_t>(w);
         const uint32_t h = cm->h, rh = cm->rh;
-        const Axis ay = make_axis(h, rh, cm->top, C);
+        const Axis ay = make_axis(h, rh, CROP ? cm->top : (rh - C) / 2, C);
         const float na[3] = {p.a[0], p.a[1], p.a[2]};
         for (uint32_t t = 0; t < cm->rows_out; ++t, q_out += row_step) {
           const Tap ty = axis_tap(ay, cm->k0 + t);
@@ -945,7 +945,7 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
   }
 }
 
-template <typename OutT, int MODE>
+template <typename OutT, int MODE, bool CROP>
 __global__ void __launch_bounds__(kThreads, kCtasPerSm) preba_fused_kernel(const Params p) {
   __shared__ WarpShared sm[kWarpsPerCta];
   // a following launch that was marked independent of this one may start as soon as
@@ -961,7 +961,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) preba_fused_kernel(const
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncwarp();
-  warp_main<OutT, MODE>(p, ws, lane, blockIdx.x * kWarpsPerCta + warp, gridDim.x * kWarpsPerCta);
+  warp_main<OutT, MODE, CROP>(p, ws, lane, blockIdx.x * kWarpsPerCta + warp, gridDim.x * kWarpsPerCta);
 }
 
 thread_local int g_last_cuda_error = 0;
@@ -1001,24 +1001,31 @@ int check_table(const preba_img_t* t, uint32_t n, uint64_t pixels_bytes) {
 
 // The kernel for an output type and mode.
 using KernelFn = void (*)(const Params);
-constexpr int kVariants = 7;
+constexpr int kVariants = 14;
 
-int variant_of(int out_dtype, int mode) {
-  if (mode == kU8) return 6;
+// 0..2: fp32/fp16/bf16 out; 3..5: the same after rounding; 6: uint8 out; +7: with a crop
+// window per image (Params::crop).
+int variant_of(int out_dtype, int mode, bool crop) {
   const int t = out_dtype == PREBA_F16 ? 1 : out_dtype == PREBA_BF16 ? 2 : 0;
-  return (mode == kRoundFloat ? 3 : 0) + t;
+  const int base = mode == kU8 ? 6 : (mode == kRoundFloat ? 3 : 0) + t;
+  return base + (crop ? 7 : 0);
+}
+
+template <bool CROP>
+KernelFn kernel_with(int base) {
+  switch (base) {
+    case 1: return preba_fused_kernel<__half, kFloat, CROP>;
+    case 2: return preba_fused_kernel<__nv_bfloat16, kFloat, CROP>;
+    case 3: return preba_fused_kernel<float, kRoundFloat, CROP>;
+    case 4: return preba_fused_kernel<__half, kRoundFloat, CROP>;
+    case 5: return preba_fused_kernel<__nv_bfloat16, kRoundFloat, CROP>;
+    case 6: return preba_fused_kernel<uint8_t, kU8, CROP>;
+    default: return preba_fused_kernel<float, kFloat, CROP>;
+  }
 }
 
 KernelFn kernel_of(int variant) {
-  switch (variant) {
-    case 1: return preba_fused_kernel<__half, kFloat>;
-    case 2: return preba_fused_kernel<__nv_bfloat16, kFloat>;
-    case 3: return preba_fused_kernel<float, kRoundFloat>;
-    case 4: return preba_fused_kernel<__half, kRoundFloat>;
-    case 5: return preba_fused_kernel<__nv_bfloat16, kRoundFloat>;
-    case 6: return preba_fused_kernel<uint8_t, kU8>;
-    default: return preba_fused_kernel<float, kFloat>;
-  }
+  return variant >= 7 ? kernel_with<true>(variant - 7) : kernel_with<false>(variant);
 }
 
 // Resident CTAs of the fused kernel on the current device (grid of a persistent launch).
@@ -1047,7 +1054,7 @@ int resident_ctas(int variant, cudaError_t* err) {
 
 int launch(const Params& p, int out_dtype, bool overlap, cudaStream_t stream, int mode = kFloat) {
   cudaError_t err = cudaSuccess;
-  const int variant = variant_of(out_dtype, mode);
+  const int variant = variant_of(out_dtype, mode, p.crop != nullptr);
   const int resident = resident_ctas(variant, &err);
   if (err == cudaSuccess) {
     const uint32_t want = (p.tasks + kWarpsPerCta - 1) / kWarpsPerCta;
