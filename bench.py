@@ -297,6 +297,40 @@ def run_streams(args, local_rank: int) -> None:
     print(json.dumps(line), flush=True)
 
 
+def report_variant(args, rank, world, n, elapsed_ms, acct, desc, dtype, sets, step_bytes, l2,
+                   clocks, dist, dev, t_host) -> None:
+    """The JSON line of a --variant run: the device-resident leg only."""
+    (elapsed_ms,) = max_over_ranks([elapsed_ms], dist, dev)
+    if rank == 0:
+        peak, peak_src = measured_peak()
+        per_launch_s = elapsed_ms * 1e-3 / args.steps
+        achieved = acct["total"] / per_launch_s / 1e9
+        line = {
+            "metric": METRIC, "value": world * n * args.steps / (elapsed_ms * 1e-3), "unit": UNIT,
+            "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+            "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "int32" if dtype == "u8" else "int32+f32",
+            "data": "synthetic",
+            "config": dict(config_of(desc, dtype, n, world),
+                           launch="one stream, back-to-back launches marked independent of "
+                                  "their predecessor (programmatic dependent launch)",
+                           l2=f"rotating {sets} input/output buffer sets "
+                              f"({sets * step_bytes / 1e6:.0f} MB) > L2 ({l2 / 1e6:.0f} MB)"),
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                         "frac": achieved / peak, "traffic": None, "peak_source": peak_src,
+                         "algorithmic_bytes_per_launch": acct["total"],
+                         "input_sector_bytes": acct["input_sector_bytes"],
+                         "output_bytes": acct["output_bytes"],
+                         "kernel_us": per_launch_s * 1e6,
+                         "host_launch_us": 1e6 * t_host / args.steps},
+            "gpu_launches": args.steps, "clocks": clocks.summary(),
+        }
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
 def run_ours(args, rank: int, world: int, local_rank: int) -> None:
     import torch
 
@@ -320,12 +354,18 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
     C, S = wl.OUT_SIZE, wl.RESIZE_SHORT
 
     packed, table = pb.preba_pack(images)
-    acct = accounting.batch_bytes(table, C, S, 2 if dtype == "f16" else 4)
+    if args.variant == "u8":
+        out_dtype, tdt, dtype = pb.U8, torch.uint8, "u8"
+        desc += ", rounded uint8 HWC output (preba_preprocess_ex)"
+    elif args.variant == "round":
+        desc += ", resized pixel rounded to uint8 before normalising (preba_preprocess_ex)"
+    acct = accounting.batch_bytes(table, C, S, {"f16": 2, "f32": 4, "u8": 1}[dtype])
     l2 = torch.cuda.get_device_properties(dev).L2_cache_size
     step_bytes = packed.nbytes + acct["output_bytes"]
     sets = max(2, min(64, -(-4 * l2 // step_bytes)))
     pix = [torch.from_numpy(packed).to(dev) for _ in range(sets)]
-    outs = [torch.empty((n, 3, C, C), dtype=tdt, device=dev) for _ in range(sets)]
+    out_shape = (n, C, C, 3) if args.variant == "u8" else (n, 3, C, C)
+    outs = [torch.empty(out_shape, dtype=tdt, device=dev) for _ in range(sets)]
     tab = torch.from_numpy(table.view(np.uint8)).to(dev)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     scratch = torch.zeros(pb.SCRATCH_BYTES // 4, dtype=torch.int32, device=dev)
@@ -333,9 +373,14 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
 
     # Timed launches go to one stream, each into the next buffer set and marked independent
     # of its predecessor, so a launch starts as the previous one's warps retire.
-    calls = [pb.PreparedPreprocess(pix[i], tab, n, outs[i], C, S, wl.MEAN, wl.STD, out_dtype,
-                                   stream=stream, status=status, flags=pb.OVERLAP_PREVIOUS)
-             for i in range(sets)]
+    if args.variant == "plain":
+        calls = [pb.PreparedPreprocess(pix[i], tab, n, outs[i], C, S, wl.MEAN, wl.STD, out_dtype,
+                                       stream=stream, status=status, flags=pb.OVERLAP_PREVIOUS)
+                 for i in range(sets)]
+    else:
+        calls = [pb.PreparedPreprocessEx(pix[i], tab, n, outs[i], C, S, wl.MEAN, wl.STD,
+                                         out_dtype, round_u8=True, stream=stream, status=status,
+                                         flags=pb.OVERLAP_PREVIOUS) for i in range(sets)]
 
     def barrier():
         if dist is not None:
@@ -360,10 +405,18 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
     assert int(status.item()) == 0, "kernel reported an error status"
     # every buffer set must hold the result of an isolated launch
     ref = torch.empty_like(outs[0])
-    pb.preba_preprocess(pix[0], tab, n, ref, C, S, wl.MEAN, wl.STD, out_dtype, stream=stream,
-                        status=status, scratch=scratch)
+    if args.variant == "plain":
+        pb.preba_preprocess(pix[0], tab, n, ref, C, S, wl.MEAN, wl.STD, out_dtype, stream=stream,
+                            status=status, scratch=scratch)
+    else:
+        pb.preba_preprocess_ex(pix[0], tab, n, ref, C, S, wl.MEAN, wl.STD, out_dtype,
+                               round_u8=True, stream=stream, status=status, scratch=scratch)
     torch.cuda.synchronize()
     assert all(bool(torch.equal(o, ref)) for o in outs), "overlapped launches changed the result"
+    if args.variant != "plain":
+        report_variant(args, rank, world, n, elapsed_ms, acct, desc, dtype, sets, step_bytes, l2,
+                       clocks, dist, dev, t_host)
+        return
 
     # ---- the same launch over and over on one buffer set (whatever fits stays in L2) -----------
     warm_steps = max(3, min(args.steps, 2000))
@@ -565,6 +618,9 @@ def main() -> None:
     ap.add_argument("--workload", default="mixed",
                     choices=["mixed", "320x240", "1080p", "sweep", "streams"])
     ap.add_argument("--batch", type=int, default=None)
+    ap.add_argument("--variant", default="plain", choices=["plain", "u8", "round"],
+                    help="device-resident leg through preba_preprocess_ex: u8 = rounded uint8 "
+                         "HWC output, round = rounded to uint8 then normalised (workload's dtype)")
     ap.add_argument("--e2e-steps", type=int, default=20)
     ap.add_argument("--cpu-budget", type=float, default=12.0,
                     help="seconds of wall time given to the CPU-baseline leg")

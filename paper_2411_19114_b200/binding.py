@@ -254,6 +254,52 @@ def preba_preprocess(pixels, table, n: int, out, out_size: int, resize_short: in
         raise PrebaError(rc, "preba_preprocess")
 
 
+class PreparedPreprocessEx:
+    """The arguments of one ``preba_preprocess_ex`` call, marshalled once (see
+    ``preba_preprocess_ex``); calling the object makes the foreign call and nothing else."""
+
+    def __init__(self, pixels, table, n: int, out, out_size: int, resize_short: int, mean, std,
+                 out_dtype: int, round_u8: bool = False, crop_origin=None,
+                 crop_origin_host: np.ndarray | None = None, stream=None,
+                 table_host: np.ndarray | None = None, status=None, scratch=None,
+                 flags: int = 0):
+        import torch
+
+        if stream is None:
+            stream = torch.cuda.current_stream().cuda_stream
+        elif hasattr(stream, "cuda_stream"):
+            stream = stream.cuda_stream
+        batch = PrebaBatch()
+        batch.pixels = pixels.data_ptr()
+        batch.pixels_bytes = pixels.numel() * pixels.element_size()
+        batch.table = table.data_ptr()
+        batch.table_host = table_host.ctypes.data if table_host is not None else None
+        batch.n = n
+        batch.out = out.data_ptr()
+        batch.out_bytes = out.numel() * out.element_size()
+        batch.status = status.data_ptr() if status is not None else None
+        batch.scratch = scratch.data_ptr() if scratch is not None else None
+        batch.flags = flags
+        opt = PrebaOptions()
+        opt.out_size, opt.resize_short = out_size, resize_short
+        opt.mean = (ctypes.c_float * 3)(*[float(v) for v in _f3(mean)])
+        opt.std = (ctypes.c_float * 3)(*[float(v) for v in _f3(std)])
+        opt.out_dtype = out_dtype
+        opt.flags = EX_ROUND_U8 if round_u8 else 0
+        opt.crop_origin = crop_origin.data_ptr() if crop_origin is not None else None
+        if crop_origin_host is not None:
+            crop_origin_host = np.ascontiguousarray(crop_origin_host, dtype=np.uint32)
+            opt.crop_origin_host = crop_origin_host.ctypes.data
+        self._keep = (pixels, table, out, status, scratch, table_host, crop_origin,
+                      crop_origin_host, batch, opt)
+        self._args = (ctypes.byref(batch), ctypes.byref(opt), ctypes.c_void_p(stream))
+
+    def __call__(self) -> None:
+        rc = lib().preba_preprocess_ex(*self._args)
+        if rc != OK:
+            raise PrebaError(rc, "preba_preprocess_ex")
+
+
 def preba_preprocess_ex(pixels, table, n: int, out, out_size: int, resize_short: int, mean, std,
                         out_dtype: int, round_u8: bool = False, crop_origin=None,
                         crop_origin_host: np.ndarray | None = None, stream=None,
@@ -262,36 +308,9 @@ def preba_preprocess_ex(pixels, table, n: int, out, out_size: int, resize_short:
     """``preba_preprocess`` with a crop window per image (``crop_origin``: CUDA int32/uint32
     tensor of 2n values (top, left); ``crop_origin_host``: uint32 array for the host check) and
     optional rounding of the resized pixel to uint8 (``out_dtype`` U8 writes it as [n,C,C,3])."""
-    import torch
-
-    if stream is None:
-        stream = torch.cuda.current_stream().cuda_stream
-    elif hasattr(stream, "cuda_stream"):
-        stream = stream.cuda_stream
-    batch = PrebaBatch()
-    batch.pixels = pixels.data_ptr()
-    batch.pixels_bytes = pixels.numel() * pixels.element_size()
-    batch.table = table.data_ptr()
-    batch.table_host = table_host.ctypes.data if table_host is not None else None
-    batch.n = n
-    batch.out = out.data_ptr()
-    batch.out_bytes = out.numel() * out.element_size()
-    batch.status = status.data_ptr() if status is not None else None
-    batch.scratch = scratch.data_ptr() if scratch is not None else None
-    batch.flags = flags
-    opt = PrebaOptions()
-    opt.out_size, opt.resize_short = out_size, resize_short
-    opt.mean = (ctypes.c_float * 3)(*[float(v) for v in _f3(mean)])
-    opt.std = (ctypes.c_float * 3)(*[float(v) for v in _f3(std)])
-    opt.out_dtype = out_dtype
-    opt.flags = EX_ROUND_U8 if round_u8 else 0
-    opt.crop_origin = crop_origin.data_ptr() if crop_origin is not None else None
-    if crop_origin_host is not None:
-        crop_origin_host = np.ascontiguousarray(crop_origin_host, dtype=np.uint32)
-        opt.crop_origin_host = crop_origin_host.ctypes.data
-    rc = lib().preba_preprocess_ex(ctypes.byref(batch), ctypes.byref(opt), ctypes.c_void_p(stream))
-    if rc != OK:
-        raise PrebaError(rc, "preba_preprocess_ex")
+    PreparedPreprocessEx(pixels, table, n, out, out_size, resize_short, mean, std, out_dtype,
+                         round_u8, crop_origin, crop_origin_host, stream, table_host, status,
+                         scratch, flags)()
 
 
 class PreparedPreprocess:

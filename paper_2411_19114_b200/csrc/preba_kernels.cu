@@ -99,9 +99,8 @@ struct TaskMeta {
   // rounded modes: the value of an output pixel is num / dd with dd = den_x * den_y
   uint32_t deny2;         // 2 * den_y
   uint32_t dd;            // den_x * den_y
-  uint32_t magic;         // floor(2^(31 + k) / (2 * dd)) with 2^k <= 2 * dd < 2^(k + 1)
-  uint32_t shift;         // k - 1
-  uint32_t pad;
+  uint32_t magic;         // floor(2^32 / (2 * dd))
+  uint32_t pad[2];
   uint64_t src;           // byte offset of the image in the pixel buffer
   uint32_t info[kMaxList];  // per listed row: low byte = byte skew of the staged row,
                             // next byte = output rows completed by this row
@@ -368,16 +367,17 @@ __device__ __forceinline__ void emit_row(OutT* __restrict__ q, uint32_t plane, u
 // The rounded modes keep den_x times the horizontally interpolated value as a whole number
 // (bit pattern of an unsigned integer in the row buffers).  An output pixel is
 // floor(num / dd + 1/2) = floor(t / (2 dd)) with t = 2 num + dd, num = prev * (den_y - rem)
-// + cur * rem.  The quotient (at most 255) comes from a multiply-high by a reciprocal that
-// never overshoots and is one short at most, then one correction by the remainder.
+// + cur * rem.  The quotient (at most 255) comes from a multiply-high by floor(2^32 / (2 dd)):
+// t < 2^32 makes that estimate exact or one short, and the remainder corrects it.
 struct Quant {
-  uint32_t deny2, dd, d2, magic, shift;
+  uint32_t deny2, dd, d2, magic;
 };
 
-__device__ __forceinline__ uint32_t rounded_pixel(uint32_t prev, uint32_t cur, uint32_t w0,
-                                                  uint32_t w1, const Quant& qz) {
-  const uint32_t t = prev * w0 + cur * w1 + qz.dd;  // < 2^32 by the fast path's precondition
-  uint32_t q = __umulhi(t, qz.magic) >> qz.shift;
+__device__ __forceinline__ uint32_t rounded_pixel(float prev, float cur, uint32_t w0, uint32_t w1,
+                                                  const Quant& qz) {
+  // < 2^32 by the fast path's precondition
+  const uint32_t t = __float_as_uint(prev) * w0 + (__float_as_uint(cur) * w1 + qz.dd);
+  uint32_t q = __umulhi(t, qz.magic);
   if (t - q * qz.d2 >= qz.d2) ++q;
   return q;
 }
@@ -395,18 +395,16 @@ __device__ __forceinline__ void emit_row_rounded(OutT* __restrict__ q, uint32_t 
                                                  const Quant& qz, const float (&na)[3],
                                                  const float (&nb)[3], uint32_t valid) {
   const uint32_t w1 = 2 * rem, w0 = qz.deny2 - w1;
-  uint32_t px[kLaneCols][3];
-#pragma unroll
-  for (int m = 0; m < static_cast<int>(kLaneCols); ++m)
-#pragma unroll
-    for (int ch = 0; ch < 3; ++ch)
-      px[m][ch] = rounded_pixel(__float_as_uint(hp[m][ch]), __float_as_uint(hc[m][ch]), w0, w1, qz);
   if constexpr (MODE == kU8) {
     uint8_t* b = reinterpret_cast<uint8_t*>(q);
 #pragma unroll
     for (int pr = 0; pr < 3; ++pr) {
-      const uint32_t (&l)[3] = px[2 * pr];
-      const uint32_t (&r)[3] = px[2 * pr + 1];
+      uint32_t l[3], r[3];
+#pragma unroll
+      for (int ch = 0; ch < 3; ++ch) {
+        l[ch] = rounded_pixel(hp[2 * pr][ch], hc[2 * pr][ch], w0, w1, qz);
+        r[ch] = rounded_pixel(hp[2 * pr + 1][ch], hc[2 * pr + 1][ch], w0, w1, qz);
+      }
       uint8_t* at = b + 192 * pr;  // 64 pixels further
       if (FULL) {
         uint16_t* h16 = reinterpret_cast<uint16_t*>(at);  // even byte offset: 6 * lane + 192 * pr
@@ -424,15 +422,18 @@ __device__ __forceinline__ void emit_row_rounded(OutT* __restrict__ q, uint32_t 
     uint8_t* single = b + 3 * (192 - lane);  // pixel 192 + lane
     if (FULL || ((valid >> 6) & 1u)) {
 #pragma unroll
-      for (int ch = 0; ch < 3; ++ch) single[ch] = static_cast<uint8_t>(px[6][ch]);
+      for (int ch = 0; ch < 3; ++ch)
+        single[ch] = static_cast<uint8_t>(rounded_pixel(hp[6][ch], hc[6][ch], w0, w1, qz));
     }
   } else {
 #pragma unroll
     for (int ch = 0; ch < 3; ++ch, q += plane) {
       float o[kLaneCols];
 #pragma unroll
-      for (int m = 0; m < static_cast<int>(kLaneCols); ++m)
-        o[m] = fmaf(__uint_as_float(0x4B000000u | px[m][ch]) - 8388608.0f, na[ch], nb[ch]);
+      for (int m = 0; m < static_cast<int>(kLaneCols); ++m) {
+        const uint32_t px = rounded_pixel(hp[m][ch], hc[m][ch], w0, w1, qz);
+        o[m] = fmaf(__uint_as_float(0x4B000000u | px) - 8388608.0f, na[ch], nb[ch]);
+      }
       OutT* single = q + 192 - lane;
       if (FULL) {
 #pragma unroll
@@ -591,12 +592,9 @@ __device__ __forceinline__ uint32_t prepare(const Params& p, uint32_t task, Task
       // integer weight of the lower row; all of it when both taps are the row just staged
       if (active) m.lam[lane] = ty.i1 == ty.i0 ? ay.den : ty.rem;
       if (lane == 0 && kind == kStream) {
-        const uint32_t d2 = 2 * static_cast<uint32_t>(dd);
-        const uint32_t k = 31 - static_cast<uint32_t>(__clz(d2));
         m.deny2 = 2 * ay.den;
         m.dd = static_cast<uint32_t>(dd);
-        m.magic = static_cast<uint32_t>((1ull << (31 + k)) / d2);
-        m.shift = k - 1;
+        m.magic = static_cast<uint32_t>((1ull << 32) / (2 * dd));  // 2 dd >= 8
       }
     }
     if (lane == 0) {
@@ -632,6 +630,44 @@ __device__ __forceinline__ uint32_t prepare(const Params& p, uint32_t task, Task
   return kind;
 }
 
+// Direct path of the rounded modes for one task: exact integers of any size, taps from
+// global memory.
+template <typename OutT, int MODE>
+__device__ __forceinline__ void gather_rounded(const Params& p, const TaskMeta& cm, uint32_t lane) {
+  const uint32_t C = p.C;
+  const size_t plane = static_cast<size_t>(C) * C;
+  const uint32_t w = cm.w, h = cm.h, rw = cm.rw, rh = cm.rh, col0 = cm.col0;
+  const uint8_t* __restrict__ src = p.pixels + cm.src;
+  const size_t pitch = 3 * static_cast<size_t>(w);
+  for (uint32_t t = 0; t < cm.rows_out; ++t) {
+    const TapInt ty = axis_tap_int(h, rh, cm.top, cm.k0 + t);
+    const uint8_t* r0 = src + ty.i0 * pitch;
+    const uint8_t* r1 = src + ty.i1 * pitch;
+#pragma unroll 1
+    for (int m = 0; m < static_cast<int>(kLaneCols); ++m) {
+      const uint32_t j = col0 + lane_col(lane, m);
+      if (j >= C) continue;
+      const TapInt tx = axis_tap_int(w, rw, cm.left, j);
+#pragma unroll 1
+      for (uint32_t ch = 0; ch < 3; ++ch) {
+        const uint32_t v = rounded_pixel_wide(__ldg(r0 + 3 * static_cast<size_t>(tx.i0) + ch),
+                                              __ldg(r0 + 3 * static_cast<size_t>(tx.i1) + ch),
+                                              __ldg(r1 + 3 * static_cast<size_t>(tx.i0) + ch),
+                                              __ldg(r1 + 3 * static_cast<size_t>(tx.i1) + ch), tx, ty);
+        const size_t row = static_cast<size_t>(cm.k0 + t) * C + j;
+        if constexpr (MODE == kU8) {
+          reinterpret_cast<uint8_t*>(p.out)[3 * (static_cast<size_t>(cm.img) * plane + row) + ch] =
+              static_cast<uint8_t>(v);
+        } else {
+          const float o = fmaf(static_cast<float>(v), p.a[ch], p.b[ch]);
+          static_cast<OutT*>(p.out)[(static_cast<size_t>(cm.img) * 3 + ch) * plane + row] =
+              Pack<OutT>::one(o);
+        }
+      }
+    }
+  }
+}
+
 template <typename OutT, bool FULL, int MODE>
 __device__ __forceinline__ void emit_any(OutT* __restrict__ q, uint32_t plane, uint32_t lane,
                                          uint32_t weight_bits,
@@ -654,7 +690,7 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
   const uint32_t row_step = MODE == kU8 ? 3 * C : C;  // elements of OutT between output rows
   const float nb[3] = {p.b[0], p.b[1], p.b[2]};
   float sa[3] = {0.f, 0.f, 0.f};  // staged path: 1 / (255 * std * den) of the task's image
-  Quant qz = {0, 0, 0, 0, 0};     // rounded modes: the task's division constants
+  Quant qz = {0, 0, 0, 0};     // rounded modes: the task's division constants
 
   // task claims: a warp's first task is its own index; later ones come from the shared
   // counter (dynamic) or every nwarps-th task (static)
@@ -777,7 +813,6 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
           qz.dd = cm->dd;
           qz.d2 = 2 * qz.dd;
           qz.magic = cm->magic;
-          qz.shift = cm->shift;
 #pragma unroll
           for (int ch = 0; ch < 3; ++ch) sa[ch] = p.a[ch];
         }
@@ -807,38 +842,7 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
       if (kind != kGather) {
         // staged: the groups follow
       } else if constexpr (MODE != kFloat) {
-        // direct path of the rounded modes: exact integers of any size, taps from global memory
-        const uint8_t* __restrict__ src = p.pixels + cm->src;
-        const size_t pitch = 3 * static_cast<size_t>(w);
-        const uint32_t h = cm->h, rh = cm->rh;
-        for (uint32_t t = 0; t < cm->rows_out; ++t) {
-          const TapInt ty = axis_tap_int(h, rh, cm->top, cm->k0 + t);
-          const uint8_t* r0 = src + ty.i0 * pitch;
-          const uint8_t* r1 = src + ty.i1 * pitch;
-#pragma unroll 1
-          for (int m = 0; m < static_cast<int>(kLaneCols); ++m) {
-            const uint32_t j = col0 + lane_col(lane, m);
-            if (j >= C) continue;
-            const TapInt tx = axis_tap_int(w, rw, cm->left, j);
-#pragma unroll 1
-            for (uint32_t ch = 0; ch < 3; ++ch) {
-              const uint32_t v = rounded_pixel_wide(
-                  __ldg(r0 + 3 * static_cast<size_t>(tx.i0) + ch),
-                  __ldg(r0 + 3 * static_cast<size_t>(tx.i1) + ch),
-                  __ldg(r1 + 3 * static_cast<size_t>(tx.i0) + ch),
-                  __ldg(r1 + 3 * static_cast<size_t>(tx.i1) + ch), tx, ty);
-              const size_t row = static_cast<size_t>(cm->k0 + t) * C + j;
-              if constexpr (MODE == kU8) {
-                reinterpret_cast<uint8_t*>(p.out)[3 * (static_cast<size_t>(cm->img) * plane + row) +
-                                                  ch] = static_cast<uint8_t>(v);
-              } else {
-                const float o = fmaf(static_cast<float>(v), p.a[ch], p.b[ch]);
-                static_cast<OutT*>(p.out)[(static_cast<size_t>(cm->img) * 3 + ch) * plane + row] =
-                    Pack<OutT>::one(o);
-              }
-            }
-          }
-        }
+        gather_rounded<OutT, MODE>(p, *cm, lane);
         ++finished;
         need_task = true;
       } else {
