@@ -171,3 +171,25 @@ def test_window_outside_the_resized_image_is_refused_or_skipped():
     host = out.cpu().numpy()
     assert np.all(host[1] == 7)
     assert np.array_equal(host[0], want_u8(imgs[:1], 224, 256, bad[:1])[0])
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_random_shapes_windows_and_modes(seed):
+    """Seeded random batches: sides from 1 to 700, random crop and resize sizes, a random
+    window per image, all modes.  uint8 bit for bit; float kinds by the base criteria."""
+    rng = np.random.default_rng(9000 + seed)
+    s_short = int(rng.integers(1, 400))
+    c = int(rng.integers(1, s_short + 1))
+    n = int(rng.integers(1, 10))
+    imgs = [wl.uniform_image(rng, int(rng.integers(1, 701)), int(rng.integers(1, 701)))
+            for _ in range(n)]
+    origins = origins_for(imgs, c, s_short, 100 + seed) if seed % 3 else None
+    dynamic = bool(seed & 1)
+    got = run_ex(imgs, c, s_short, pb.U8, True, origins, dynamic=dynamic)
+    assert np.array_equal(got, want_u8(imgs, c, s_short, origins))
+    for dt in (pb.F32, pb.F16, pb.BF16):
+        got = run_ex(imgs, c, s_short, dt, True, origins, dynamic=dynamic)
+        assert_parity(got, want_f64(imgs, c, s_short, origins, True), dt)
+    if origins is not None:
+        got = run_ex(imgs, c, s_short, pb.F32, False, origins, dynamic=dynamic)
+        assert_parity(got, want_f64(imgs, c, s_short, origins, False), pb.F32)
