@@ -46,6 +46,10 @@ constexpr int kCtasPerSm = PREBA_CTAS_PER_SM;
 constexpr uint32_t kLaneCols = 7;                  // output columns per lane
 constexpr uint32_t kTaskCols = 32 * kLaneCols;     // 224 output columns per task
 constexpr uint32_t kSlabRows = PREBA_SLAB_ROWS;    // output rows per task (one lane per row)
+#ifndef PREBA_MIN_SLAB_ROWS
+#define PREBA_MIN_SLAB_ROWS 4
+#endif
+constexpr uint32_t kMinSlabRows = PREBA_MIN_SLAB_ROWS;  // smallest slab a small batch is cut into
 constexpr uint32_t kMaxList = 2 * 32;              // distinct source rows of a slab
 #ifndef PREBA_GROUPS
 #define PREBA_GROUPS 2
@@ -79,6 +83,8 @@ struct Params {
   uint32_t n;
   uint32_t C;           // crop side
   uint32_t S;           // resized shorter side
+  uint32_t slab_rows;   // output rows per task: 32, or 16 / 8 / 4 when a launch that runs alone
+                        // would leave warps without a task
   uint32_t slabs;       // slabs per image
   uint32_t col_blocks;  // column blocks per image
   uint32_t tasks;       // n * slabs * col_blocks
@@ -531,8 +537,8 @@ __device__ __forceinline__ uint32_t prepare(const Params& p, uint32_t task, Task
       top = min(t, rh - C);  // a window that does not fit is reported and skipped below
       left = min(l, rw - C);
     }
-    const uint32_t k0 = slab * kSlabRows;
-    const uint32_t rows_out = min(kSlabRows, C - k0);
+    const uint32_t k0 = slab * p.slab_rows;
+    const uint32_t rows_out = min(p.slab_rows, C - k0);
     const uint32_t col0 = cb * kTaskCols;
     const uint32_t cols = min(kTaskCols, C - col0);
     const Axis ax = make_axis(e.w, rw, left, C);
@@ -987,7 +993,7 @@ int check_args(const uint8_t* pixels, uint64_t pixels_bytes, const void* table, 
                         dtype_bytes(out_dtype);
   if (out_bytes < need) return PREBA_ERR_BUFFER_TOO_SMALL;
   if (pixels_bytes == 0) return PREBA_ERR_BUFFER_TOO_SMALL;
-  const uint64_t tasks = static_cast<uint64_t>(n) * ((out_size + kSlabRows - 1) / kSlabRows) *
+  const uint64_t tasks = static_cast<uint64_t>(n) * ((out_size + kMinSlabRows - 1) / kMinSlabRows) *
                          ((out_size + kTaskCols - 1) / kTaskCols);
   if (tasks > 0x7fffffffull) return PREBA_ERR_INVALID_ARG;
   return PREBA_OK;
@@ -1056,10 +1062,27 @@ int resident_ctas(int variant, cudaError_t* err) {
   return resident;
 }
 
-int launch(const Params& p, int out_dtype, bool overlap, cudaStream_t stream, int mode = kFloat) {
+int launch(const Params& given, int out_dtype, bool overlap, cudaStream_t stream,
+           int mode = kFloat) {
   cudaError_t err = cudaSuccess;
-  const int variant = variant_of(out_dtype, mode, p.crop != nullptr);
+  const int variant = variant_of(out_dtype, mode, given.crop != nullptr);
   const int resident = resident_ctas(variant, &err);
+  Params p = given;
+  if (err == cudaSuccess && !overlap) {
+    // A launch that runs alone is as long as its longest task.  While the batch has fewer
+    // tasks than the GPU has resident warps, halve the slabs (32 -> 16 -> 8 -> 4 output
+    // rows): more warps share the batch and the launch gets shorter, at the price of more
+    // staged halo rows.  The arithmetic per output element, and so the result, does not
+    // depend on the split.  Launches marked as overlapping their predecessor keep 32-row
+    // slabs: there the GPU is kept busy by the neighbouring launches and throughput counts.
+    const uint64_t warps = static_cast<uint64_t>(resident) * kWarpsPerCta;
+    while (p.slab_rows > kMinSlabRows &&
+           static_cast<uint64_t>(p.n) * ((p.C + p.slab_rows - 1) / p.slab_rows) * p.col_blocks <
+               warps)
+      p.slab_rows /= 2;
+    p.slabs = (p.C + p.slab_rows - 1) / p.slab_rows;
+    p.tasks = static_cast<uint32_t>(static_cast<uint64_t>(p.n) * p.slabs * p.col_blocks);
+  }
   if (err == cudaSuccess) {
     const uint32_t want = (p.tasks + kWarpsPerCta - 1) / kWarpsPerCta;
     const uint32_t blocks = want < static_cast<uint32_t>(resident) ? want : resident;
@@ -1096,8 +1119,9 @@ Params make_params(const uint8_t* pixels, uint64_t pixels_bytes, const preba_img
   p.S = resize_short;
   p.sched = scratch;
   p.crop = nullptr;
-  p.slabs = (out_size + kSlabRows - 1) / kSlabRows;
   p.col_blocks = (out_size + kTaskCols - 1) / kTaskCols;
+  p.slab_rows = kSlabRows;
+  p.slabs = (out_size + p.slab_rows - 1) / p.slab_rows;
   p.tasks = static_cast<uint32_t>(static_cast<uint64_t>(n) * p.slabs * p.col_blocks);
   for (int c = 0; c < 3; ++c) {
     const double sd = static_cast<double>(std[c]);
