@@ -36,8 +36,8 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM bytes (read + write) per launch of the kernel on the default workload, from one
 # ncu capture, valid only for the kernel sources with this digest (else reported as null).
-NCU_TRAFFIC = {"csrc_sha1": "98cdbe57aa922b75f5ee9a02211c5f2270e4f809",
-               "bytes_per_launch": 75619840 + 25727232}  # dram read + write, one launch
+NCU_TRAFFIC = {"csrc_sha1": "1b6a4a6fd8d22fa0a26cd0d99fc6c253c1095b2a",
+               "bytes_per_launch": 75636224 + 25414912}  # dram read + write, one launch
 
 
 def csrc_digest() -> str:
