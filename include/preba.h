@@ -374,6 +374,76 @@ int preba_batcher_push(preba_batcher_t* b, uint64_t id, uint64_t arrival_ns);
 int preba_batcher_poll(preba_batcher_t* b, uint64_t now_ns, uint64_t* ids, uint32_t capacity,
                        uint64_t* next_deadline_ns);
 
+/*
+ * Audio path — the paper's second preprocessing pipeline (Table 1 units "Mel spectrogram" and
+ * "Normalize"; Sec. 2.3 item 1: "Fast Fourier Transform (FFT), and applying Mel filters";
+ * Sec. 4.2: Normalize as three passes, the mean over all samples, the variance from that mean,
+ * then the normalisation).  "Resample" is not built: samples arrive at 16 kHz.  The paper
+ * fixes no numerics; the readings are: frames of 400 samples every 160 (no padding, so
+ * T = 1 + (L - 400)/160 frames for L >= 400, else 0), periodic Hann window, zero-padding to a
+ * 512-point DFT, power spectrum, 80 unit-height triangular filters equally spaced on the HTK
+ * mel scale between 0 and 8000 Hz, natural log of (energy + 2^-24), and per utterance and
+ * filter (x - mean)/(sqrt(var) + 1e-5) over the utterance's frames, var = mean squared
+ * deviation.  fp32 arithmetic on the device.
+ *
+ * A ragged batch is one float buffer with every utterance starting at a multiple of
+ * PREBA_AUDIO_ALIGN samples (padding samples are 0) and a table {offset, length, frames}.
+ * The result is [n, 80, t_max] float32, t_max the largest frame count of the batch; frames
+ * beyond an utterance's own count are written as 0.
+ */
+#define PREBA_AUDIO_ALIGN 4u     /* samples: every utterance starts on a 16-byte boundary */
+#define PREBA_AUDIO_RATE 16000u
+#define PREBA_AUDIO_WIN 400u
+#define PREBA_AUDIO_HOP 160u
+#define PREBA_AUDIO_NFFT 512u
+#define PREBA_AUDIO_MELS 80u
+#define PREBA_AUDIO_MAX_SAMPLES (1u << 28) /* per utterance */
+
+typedef struct {
+  uint64_t offset; /* in samples from the start of the sample buffer, multiple of PREBA_AUDIO_ALIGN */
+  uint32_t length; /* samples */
+  uint32_t frames; /* 1 + (length - 400)/160, or 0 when length < 400 */
+} preba_utt_t;
+
+typedef struct {
+  uint64_t packed_samples; /* floats in the packed sample buffer */
+  uint64_t table_bytes;    /* n * sizeof(preba_utt_t) */
+  uint64_t out_bytes;      /* n * 80 * t_max * 4 */
+  uint32_t t_max;          /* largest frame count of the batch */
+  uint32_t reserved;
+} preba_audio_sizes_t;
+
+typedef struct {
+  const float* samples;          /* DEVICE, 16-byte aligned, packed as preba_audio_pack lays out */
+  uint64_t samples_count;        /* floats readable at `samples` */
+  const preba_utt_t* table;      /* DEVICE, n entries */
+  const preba_utt_t* table_host; /* HOST copy for checking before launch, or NULL */
+  uint32_t n;
+  uint32_t t_max;                /* frames per utterance in `out` (>= every entry's frames) */
+  float* out;                    /* DEVICE, [n, 80, t_max] contiguous */
+  uint64_t out_bytes;
+  int32_t* status;               /* DEVICE word or NULL: first PREBA_ERR_* the kernels meet */
+} preba_audio_batch_t;
+
+/* Sizes for a batch of utterances of the given lengths (host arithmetic).
+ * Errors: PREBA_ERR_INVALID_ARG (NULL, n == 0, a length above PREBA_AUDIO_MAX_SAMPLES). */
+int preba_audio_query(const uint32_t* lengths, uint32_t n, preba_audio_sizes_t* sizes);
+
+/* Builds the packed sample buffer (padding written as 0) and the table from n separate
+ * utterances.  Errors: PREBA_ERR_INVALID_ARG, PREBA_ERR_BUFFER_TOO_SMALL. */
+int preba_audio_pack(const float* const* utterances, const uint32_t* lengths, uint32_t n,
+                     float* packed, uint64_t capacity_samples, preba_utt_t* table);
+
+/* Mel spectrogram (+ Normalize when `normalize` is non-zero) of a device-resident batch:
+ * enqueues one kernel for the log Mel energies (a warp transforms two frames with one complex
+ * 512-point FFT in shared memory) and, when normalising, one more for the three passes over
+ * every (utterance, filter) row; then returns.  No allocation, no synchronisation.  A table
+ * entry that is misaligned, runs past the samples or whose frame count does not follow from
+ * its length is refused on the host when `table_host` is given (PREBA_ERR_BAD_TABLE) and
+ * skipped and reported by the kernel otherwise.
+ * Errors: PREBA_ERR_INVALID_ARG, PREBA_ERR_BUFFER_TOO_SMALL, PREBA_ERR_BAD_TABLE, PREBA_ERR_CUDA. */
+int preba_audio_logmel(const preba_audio_batch_t* batch, int normalize, void* stream);
+
 /* Text for a PREBA_* code (static storage, never NULL). */
 const char* preba_strerror(int code);
 

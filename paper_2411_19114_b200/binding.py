@@ -36,7 +36,8 @@ EXPORTS = ("preba_query", "preba_pack", "preba_preprocess", "preba_preprocess_ex
            "preba_strerror",
            "preba_last_cuda_error",
            "preba_batching_params", "preba_batcher_create", "preba_batcher_destroy",
-           "preba_batcher_push", "preba_batcher_poll")
+           "preba_batcher_push", "preba_batcher_poll",
+           "preba_audio_query", "preba_audio_pack", "preba_audio_logmel")
 
 
 class PrebaImg(ctypes.Structure):
@@ -83,6 +84,22 @@ class PrebaImageBatch(ctypes.Structure):
                 ("dev_scratch", ctypes.c_void_p)]
 
 
+class PrebaAudioSizes(ctypes.Structure):
+    _fields_ = [("packed_samples", ctypes.c_uint64), ("table_bytes", ctypes.c_uint64),
+                ("out_bytes", ctypes.c_uint64), ("t_max", ctypes.c_uint32),
+                ("reserved", ctypes.c_uint32)]
+
+
+class PrebaAudioBatch(ctypes.Structure):
+    _fields_ = [("samples", ctypes.c_void_p), ("samples_count", ctypes.c_uint64),
+                ("table", ctypes.c_void_p), ("table_host", ctypes.c_void_p),
+                ("n", ctypes.c_uint32), ("t_max", ctypes.c_uint32),
+                ("out", ctypes.c_void_p), ("out_bytes", ctypes.c_uint64),
+                ("status", ctypes.c_void_p)]
+
+
+UTT_DTYPE = np.dtype([("offset", "<u8"), ("length", "<u4"), ("frames", "<u4")])
+AUDIO_MELS = 80
 TABLE_DTYPE = np.dtype([("offset", "<u8"), ("h", "<u4"), ("w", "<u4")])
 
 
@@ -148,6 +165,14 @@ def lib() -> ctypes.CDLL:
         L.preba_batcher_poll.argtypes = [ctypes.c_void_p, ctypes.c_uint64, u64p, ctypes.c_uint32,
                                          u64p]
         L.preba_batcher_poll.restype = ctypes.c_int
+        L.preba_audio_query.argtypes = [u32p, ctypes.c_uint32, ctypes.POINTER(PrebaAudioSizes)]
+        L.preba_audio_query.restype = ctypes.c_int
+        L.preba_audio_pack.argtypes = [ctypes.POINTER(ctypes.c_void_p), u32p, ctypes.c_uint32,
+                                       ctypes.c_void_p, ctypes.c_uint64, ctypes.c_void_p]
+        L.preba_audio_pack.restype = ctypes.c_int
+        L.preba_audio_logmel.argtypes = [ctypes.POINTER(PrebaAudioBatch), ctypes.c_int,
+                                         ctypes.c_void_p]
+        L.preba_audio_logmel.restype = ctypes.c_int
         L.preba_strerror.argtypes = [ctypes.c_int]
         L.preba_strerror.restype = ctypes.c_char_p
         L.preba_last_cuda_error.argtypes = []
@@ -543,3 +568,67 @@ class PrebaBatcher:
 
     def __del__(self):
         self.close()
+
+
+# ---- audio path ------------------------------------------------------------------------------------
+
+def preba_audio_query(lengths) -> PrebaAudioSizes:
+    ln = _u32(lengths)
+    sizes = PrebaAudioSizes()
+    rc = lib().preba_audio_query(_p(ln, ctypes.c_uint32), len(ln), ctypes.byref(sizes))
+    if rc != OK:
+        raise PrebaError(rc, "preba_audio_query")
+    return sizes
+
+
+def preba_audio_pack(utterances, packed: np.ndarray | None = None,
+                     table: np.ndarray | None = None):
+    """Packed float32 sample buffer and {offset, length, frames} table of a list of 1-D
+    float32 utterances."""
+    utts = [np.ascontiguousarray(u, dtype=np.float32).reshape(-1) for u in utterances]
+    n = len(utts)
+    ln = _u32([u.size for u in utts])
+    sizes = preba_audio_query(ln)
+    if packed is None:
+        packed = np.full(sizes.packed_samples, np.nan, dtype=np.float32)  # pack writes every sample
+    if table is None:
+        table = np.zeros(n, dtype=UTT_DTYPE)
+    ptrs = (ctypes.c_void_p * n)(*[u.ctypes.data for u in utts])
+    rc = lib().preba_audio_pack(ptrs, _p(ln, ctypes.c_uint32), n, packed.ctypes.data,
+                                packed.size, table.ctypes.data)
+    if rc != OK:
+        raise PrebaError(rc, "preba_audio_pack")
+    return packed, table
+
+
+class PreparedAudio:
+    """The arguments of one ``preba_audio_logmel`` call, marshalled once.  ``samples``, ``table``,
+    ``out`` (float32 [n, 80, t_max]) and ``status`` are CUDA tensors."""
+
+    def __init__(self, samples, table, n: int, t_max: int, out, normalize: bool = True,
+                 stream=None, table_host: np.ndarray | None = None, status=None):
+        import torch
+
+        if stream is None:
+            stream = torch.cuda.current_stream().cuda_stream
+        elif hasattr(stream, "cuda_stream"):
+            stream = stream.cuda_stream
+        b = PrebaAudioBatch()
+        b.samples, b.samples_count = samples.data_ptr(), samples.numel()
+        b.table = table.data_ptr()
+        b.table_host = table_host.ctypes.data if table_host is not None else None
+        b.n, b.t_max = n, t_max
+        b.out, b.out_bytes = out.data_ptr(), out.numel() * out.element_size()
+        b.status = status.data_ptr() if status is not None else None
+        self._keep = (samples, table, out, status, table_host, b)
+        self._args = (ctypes.byref(b), int(bool(normalize)), ctypes.c_void_p(stream))
+
+    def __call__(self) -> None:
+        rc = lib().preba_audio_logmel(*self._args)
+        if rc != OK:
+            raise PrebaError(rc, "preba_audio_logmel")
+
+
+def preba_audio_logmel(samples, table, n: int, t_max: int, out, normalize: bool = True,
+                       stream=None, table_host: np.ndarray | None = None, status=None) -> None:
+    PreparedAudio(samples, table, n, t_max, out, normalize, stream, table_host, status)()

@@ -1,0 +1,301 @@
+// Audio path: log Mel spectrogram and per-utterance normalisation of a ragged batch (sm_100a).
+//
+// Kernel 1: a warp takes two consecutive frames of one utterance, multiplies them by the Hann
+// window, packs them as the real and imaginary part of one complex sequence, runs a 512-point
+// radix-2 FFT in its own shared memory, separates the two spectra, forms the power spectra,
+// applies the triangular Mel filters (a lane per filter, the filter's few bins read from
+// shared memory) and writes log(energy + 2^-24).  Frames past an utterance's own count are
+// written as 0, so the result tensor needs no clearing.
+// Kernel 2 (Normalize): a warp per (utterance, filter) row makes the paper's three passes:
+// mean, variance from that mean, normalisation.
+// fp32 throughout; the path is bound by arithmetic and shared memory, not by HBM.
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+
+#include "preba.h"
+#include "preba_internal.h"
+
+namespace preba {
+namespace audio {
+
+constexpr uint32_t kWin = PREBA_AUDIO_WIN;
+constexpr uint32_t kHop = PREBA_AUDIO_HOP;
+constexpr uint32_t kFft = PREBA_AUDIO_NFFT;
+constexpr uint32_t kBins = kFft / 2 + 1;
+constexpr uint32_t kMels = PREBA_AUDIO_MELS;
+constexpr int kWarps = 4;            // warps per CTA of the spectrogram kernel
+constexpr int kFramesPerCta = 2 * kWarps;
+constexpr float kLogGuard = 5.9604644775390625e-08f;  // 2^-24
+constexpr float kStdGuard = 1e-5f;
+
+// The Mel filters in the form the kernel uses.  Bin k lies between corner frequencies
+// c[m] <= f < c[m+1]; it adds `up[k]` of its power to filter m (rising edge) and 1 - up[k] to
+// filter m - 1 (falling edge).  Filter j therefore gathers the bins whose m is j or j + 1:
+// the contiguous range [first[j], last[j]).
+struct MelTable {
+  float up[kBins];
+  uint8_t m[kBins + 3];   // 255: the bin lies outside every filter
+  uint16_t first[kMels];
+  uint16_t last[kMels];
+};
+
+uint32_t frames_of(uint32_t length) { return length < kWin ? 0u : 1u + (length - kWin) / kHop; }
+
+// Corner frequencies equally spaced on the HTK mel scale between 0 and rate / 2 (double).
+MelTable make_mel_table() {
+  MelTable t;
+  std::memset(&t, 0, sizeof(t));
+  const double top = 2595.0 * std::log10(1.0 + (PREBA_AUDIO_RATE / 2.0) / 700.0);
+  double corner[kMels + 2];
+  for (uint32_t i = 0; i < kMels + 2; ++i)
+    corner[i] = 700.0 * (std::pow(10.0, (top * i / (kMels + 1)) / 2595.0) - 1.0);
+  corner[0] = 0.0;
+  corner[kMels + 1] = PREBA_AUDIO_RATE / 2.0;
+  for (uint32_t j = 0; j < kMels; ++j) {
+    t.first[j] = 0xffff;
+    t.last[j] = 0;
+  }
+  for (uint32_t k = 0; k < kBins; ++k) {
+    const double f = static_cast<double>(k) * PREBA_AUDIO_RATE / kFft;
+    t.m[k] = 255;
+    if (f >= corner[kMels + 1]) continue;  // the top corner carries no weight
+    uint32_t m = 0;
+    while (m + 1 < kMels + 1 && f >= corner[m + 1]) ++m;
+    t.m[k] = static_cast<uint8_t>(m);
+    t.up[k] = static_cast<float>((f - corner[m]) / (corner[m + 1] - corner[m]));
+    for (int d = 0; d < 2; ++d) {          // filters m (rising) and m - 1 (falling)
+      const int j = static_cast<int>(m) - d;
+      if (j < 0 || j >= static_cast<int>(kMels)) continue;
+      if (t.first[j] == 0xffff) t.first[j] = static_cast<uint16_t>(k);
+      t.last[j] = static_cast<uint16_t>(k + 1);
+    }
+  }
+  for (uint32_t j = 0; j < kMels; ++j)
+    if (t.first[j] == 0xffff) t.first[j] = t.last[j] = 0;  // a filter without a bin
+  return t;
+}
+
+struct AudioParams {
+  const float* samples;
+  uint64_t samples_count;
+  const preba_utt_t* table;
+  float* out;
+  int32_t* status;
+  uint32_t n;
+  uint32_t t_max;
+};
+
+__device__ __forceinline__ bool utt_ok(const preba_utt_t& u, uint64_t samples_count) {
+  if (u.offset % PREBA_AUDIO_ALIGN || u.length > PREBA_AUDIO_MAX_SAMPLES) return false;
+  if (u.offset > samples_count || u.length > samples_count - u.offset) return false;
+  const uint32_t frames = u.length < kWin ? 0u : 1u + (u.length - kWin) / kHop;
+  return u.frames == frames;
+}
+
+struct __align__(16) WarpFft {
+  float2 z[kFft];       // the complex sequence, then its spectrum
+  float power[2][kBins + 3];
+};
+
+__global__ void __launch_bounds__(32 * kWarps)
+logmel_kernel(const AudioParams p, const MelTable mel) {
+  __shared__ WarpFft sm[kWarps];
+  __shared__ float2 twiddle[kFft / 2];  // exp(-2 pi i k / 512)
+  __shared__ float window[kWin];
+  const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (uint32_t k = threadIdx.x; k < kFft / 2; k += blockDim.x) {
+    float s, c;
+    sincospif(-2.0f * static_cast<float>(k) / kFft, &s, &c);
+    twiddle[k] = make_float2(c, s);
+  }
+  for (uint32_t i = threadIdx.x; i < kWin; i += blockDim.x)
+    window[i] = 0.5f - 0.5f * cospif(2.0f * static_cast<float>(i) / kWin);
+  __syncthreads();
+
+  const uint32_t utt = blockIdx.y;
+  const preba_utt_t u = p.table[utt];
+  const bool ok = utt_ok(u, p.samples_count);
+  if (!ok && threadIdx.x == 0 && p.status) atomicCAS(p.status, 0, PREBA_ERR_BAD_TABLE);
+  const uint32_t frames = ok ? min(u.frames, p.t_max) : 0u;
+  const uint32_t t0 = blockIdx.x * kFramesPerCta + 2 * warp;  // this warp's two frames
+  if (t0 >= p.t_max) return;
+  float* __restrict__ out = p.out + static_cast<size_t>(utt) * kMels * p.t_max;
+  const bool have0 = t0 < frames, have1 = t0 + 1 < frames;
+  if (!have0) {
+    // padding (or a refused entry): zeros for both frames of this warp
+    for (uint32_t j = lane; j < kMels; j += 32) {
+      out[static_cast<size_t>(j) * p.t_max + t0] = 0.f;
+      if (t0 + 1 < p.t_max) out[static_cast<size_t>(j) * p.t_max + t0 + 1] = 0.f;
+    }
+    return;
+  }
+  WarpFft& ws = sm[warp];
+  const float* __restrict__ x = p.samples + u.offset + static_cast<size_t>(t0) * kHop;
+  // windowed frames as real and imaginary part, stored in bit-reversed order
+  for (uint32_t i = lane; i < kFft; i += 32) {
+    float re = 0.f, im = 0.f;
+    if (i < kWin) {
+      re = x[i] * window[i];
+      if (have1) im = x[i + kHop] * window[i];
+    }
+    ws.z[__brev(i) >> 23] = make_float2(re, im);
+  }
+  __syncwarp();
+  // nine radix-2 stages, eight butterflies per lane and stage
+#pragma unroll 1
+  for (uint32_t s = 0; s < 9; ++s) {
+    const uint32_t half = 1u << s;
+#pragma unroll
+    for (uint32_t q = 0; q < 8; ++q) {
+      const uint32_t b = lane + 32 * q;
+      const uint32_t pos = b & (half - 1);
+      const uint32_t i = ((b >> s) << (s + 1)) + pos;
+      const float2 w = twiddle[pos << (8 - s)];
+      const float2 a = ws.z[i], c = ws.z[i + half];
+      const float2 v = make_float2(c.x * w.x - c.y * w.y, c.x * w.y + c.y * w.x);
+      ws.z[i] = make_float2(a.x + v.x, a.y + v.y);
+      ws.z[i + half] = make_float2(a.x - v.x, a.y - v.y);
+    }
+    __syncwarp();
+  }
+  // Z = A + iB with A, B the spectra of the two real frames:
+  // A[k] = (Z[k] + conj(Z[N-k]))/2, B[k] = (Z[k] - conj(Z[N-k]))/(2i)
+  for (uint32_t k = lane; k < kBins; k += 32) {
+    const float2 zk = ws.z[k], zn = ws.z[(kFft - k) & (kFft - 1)];
+    const float ar = 0.5f * (zk.x + zn.x), ai = 0.5f * (zk.y - zn.y);
+    const float br = 0.5f * (zk.y + zn.y), bi = 0.5f * (zn.x - zk.x);
+    ws.power[0][k] = ar * ar + ai * ai;
+    ws.power[1][k] = br * br + bi * bi;
+  }
+  __syncwarp();
+  for (uint32_t j = lane; j < kMels; j += 32) {
+    float e0 = 0.f, e1 = 0.f;
+    for (uint32_t k = mel.first[j]; k < mel.last[j]; ++k) {
+      const float wgt = mel.m[k] == j ? mel.up[k] : 1.0f - mel.up[k];
+      e0 = fmaf(wgt, ws.power[0][k], e0);
+      e1 = fmaf(wgt, ws.power[1][k], e1);
+    }
+    out[static_cast<size_t>(j) * p.t_max + t0] = logf(e0 + kLogGuard);
+    if (t0 + 1 < p.t_max)
+      out[static_cast<size_t>(j) * p.t_max + t0 + 1] = have1 ? logf(e1 + kLogGuard) : 0.f;
+  }
+}
+
+// Normalize: a warp per (utterance, filter) row.
+__global__ void __launch_bounds__(128) normalize_kernel(const AudioParams p) {
+  const uint32_t lane = threadIdx.x & 31;
+  const uint32_t row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (row >= p.n * kMels) return;
+  const uint32_t utt = row / kMels;
+  const preba_utt_t u = p.table[utt];
+  if (!utt_ok(u, p.samples_count)) return;
+  const uint32_t frames = min(u.frames, p.t_max);
+  if (frames == 0) return;
+  float* __restrict__ r = p.out + static_cast<size_t>(row) * p.t_max;
+  float sum = 0.f;
+  for (uint32_t t = lane; t < frames; t += 32) sum += r[t];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+  const float mean = sum / static_cast<float>(frames);
+  float sq = 0.f;
+  for (uint32_t t = lane; t < frames; t += 32) {
+    const float d = r[t] - mean;
+    sq = fmaf(d, d, sq);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+  const float inv = 1.0f / (sqrtf(sq / static_cast<float>(frames)) + kStdGuard);
+  for (uint32_t t = lane; t < frames; t += 32) r[t] = (r[t] - mean) * inv;
+}
+
+}  // namespace audio
+}  // namespace preba
+
+extern "C" int preba_audio_query(const uint32_t* lengths, uint32_t n, preba_audio_sizes_t* sizes) {
+  if (!lengths || !sizes || n == 0) return PREBA_ERR_INVALID_ARG;
+  uint64_t at = 0;
+  uint32_t t_max = 0;
+  for (uint32_t i = 0; i < n; ++i) {
+    if (lengths[i] > PREBA_AUDIO_MAX_SAMPLES) return PREBA_ERR_INVALID_ARG;
+    at = preba::align_up(at + lengths[i], PREBA_AUDIO_ALIGN);
+    const uint32_t f = preba::audio::frames_of(lengths[i]);
+    t_max = f > t_max ? f : t_max;
+  }
+  sizes->packed_samples = at;
+  sizes->table_bytes = static_cast<uint64_t>(n) * sizeof(preba_utt_t);
+  sizes->out_bytes = static_cast<uint64_t>(n) * PREBA_AUDIO_MELS * t_max * sizeof(float);
+  sizes->t_max = t_max;
+  sizes->reserved = 0;
+  return PREBA_OK;
+}
+
+extern "C" int preba_audio_pack(const float* const* utterances, const uint32_t* lengths,
+                                uint32_t n, float* packed, uint64_t capacity_samples,
+                                preba_utt_t* table) {
+  if (!utterances || !lengths || !packed || !table || n == 0) return PREBA_ERR_INVALID_ARG;
+  uint64_t need = 0;
+  for (uint32_t i = 0; i < n; ++i) {
+    if ((!utterances[i] && lengths[i]) || lengths[i] > PREBA_AUDIO_MAX_SAMPLES)
+      return PREBA_ERR_INVALID_ARG;
+    need = preba::align_up(need + lengths[i], PREBA_AUDIO_ALIGN);
+  }
+  if (capacity_samples < need) return PREBA_ERR_BUFFER_TOO_SMALL;
+  uint64_t at = 0;
+  for (uint32_t i = 0; i < n; ++i) {
+    table[i].offset = at;
+    table[i].length = lengths[i];
+    table[i].frames = preba::audio::frames_of(lengths[i]);
+    if (lengths[i]) std::memcpy(packed + at, utterances[i], sizeof(float) * lengths[i]);
+    const uint64_t next = preba::align_up(at + lengths[i], PREBA_AUDIO_ALIGN);
+    for (uint64_t k = at + lengths[i]; k < next; ++k) packed[k] = 0.0f;
+    at = next;
+  }
+  return PREBA_OK;
+}
+
+extern "C" int preba_audio_logmel(const preba_audio_batch_t* b, int normalize, void* stream) {
+  using namespace preba::audio;
+  if (!b || !b->samples || !b->table || !b->out || b->n == 0 || b->n > 65535 || b->t_max == 0)
+    return PREBA_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(b->samples) % 16 || reinterpret_cast<uintptr_t>(b->out) % 4 ||
+      reinterpret_cast<uintptr_t>(b->table) % 8)
+    return PREBA_ERR_INVALID_ARG;
+  const uint64_t need = static_cast<uint64_t>(b->n) * kMels * b->t_max * sizeof(float);
+  if (b->out_bytes < need) return PREBA_ERR_BUFFER_TOO_SMALL;
+  if (static_cast<uint64_t>(b->n) * kMels * b->t_max > 0xffffffffull) return PREBA_ERR_INVALID_ARG;
+  if (b->table_host) {
+    for (uint32_t i = 0; i < b->n; ++i) {
+      const preba_utt_t& u = b->table_host[i];
+      if (u.offset % PREBA_AUDIO_ALIGN || u.length > PREBA_AUDIO_MAX_SAMPLES ||
+          u.offset > b->samples_count || u.length > b->samples_count - u.offset ||
+          u.frames != frames_of(u.length) || u.frames > b->t_max)
+        return PREBA_ERR_BAD_TABLE;
+    }
+  }
+  static const MelTable mel = make_mel_table();
+  AudioParams p;
+  p.samples = b->samples;
+  p.samples_count = b->samples_count;
+  p.table = b->table;
+  p.out = b->out;
+  p.status = b->status;
+  p.n = b->n;
+  p.t_max = b->t_max;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const dim3 grid((b->t_max + kFramesPerCta - 1) / kFramesPerCta, b->n);
+  logmel_kernel<<<grid, 32 * kWarps, 0, s>>>(p, mel);
+  cudaError_t err = cudaGetLastError();
+  if (err == cudaSuccess && normalize) {
+    const uint32_t rows = b->n * kMels;
+    normalize_kernel<<<(rows + 3) / 4, 128, 0, s>>>(p);
+    err = cudaGetLastError();
+  }
+  if (err != cudaSuccess) {
+    preba::g_last_cuda_error = static_cast<int>(err);
+    return PREBA_ERR_CUDA;
+  }
+  return PREBA_OK;
+}

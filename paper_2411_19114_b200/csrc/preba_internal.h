@@ -13,6 +13,9 @@ uint32_t dtype_bytes(int out_dtype);  // size of one output element
 bool dims_ok(uint32_t h, uint32_t w);
 uint64_t align_up(uint64_t v, uint64_t a);
 
+// The cudaError_t behind the calling thread's last PREBA_ERR_CUDA (preba_last_cuda_error).
+extern thread_local int g_last_cuda_error;
+
 }  // namespace preba
 
 #endif  // PREBA_INTERNAL_H_

@@ -104,3 +104,35 @@ def hires_1080p(n: int = 64, seed: int = 4) -> list[np.ndarray]:
 def sweep_500x375(n: int = 2048, seed: int = 5) -> list[np.ndarray]:
     """n images of 500x375 with uniform random bytes; prefixes serve the batch sweep."""
     return fixed_size_batch(seed, n, 375, 500, "uniform")
+
+
+# ---- audio: seeded synthetic utterances (inputs only) -------------------------------------------
+
+AUDIO_RATE = 16000
+
+
+def utterance(rng: np.random.Generator, seconds: float) -> np.ndarray:
+    """A speech-like test signal: a handful of harmonics of a slowly gliding pitch under a
+    syllable-rate envelope, plus white noise 40 dB below; float32 in [-1, 1] at 16 kHz.
+    It stands in for the read speech of the paper's audio corpus (Sec. 5): broadband, with
+    pauses; no corpus item is reproduced."""
+    n = int(round(seconds * AUDIO_RATE))
+    t = np.arange(n, dtype=np.float64) / AUDIO_RATE
+    f0 = rng.uniform(90.0, 220.0)
+    glide = 1.0 + 0.15 * np.sin(2 * np.pi * rng.uniform(0.2, 0.7) * t + rng.uniform(0, 6.28))
+    phase = 2 * np.pi * np.cumsum(f0 * glide) / AUDIO_RATE
+    x = np.zeros(n)
+    for h in range(1, 24):
+        x += rng.uniform(0.2, 1.0) / h * np.sin(h * phase + rng.uniform(0, 6.28))
+    env = np.clip(np.sin(2 * np.pi * rng.uniform(2.0, 4.0) * t + rng.uniform(0, 6.28)), 0.0, 1.0)
+    x = x * env ** 2
+    x = 0.5 * x / max(1e-9, np.max(np.abs(x)))
+    x += 0.005 * rng.standard_normal(n)
+    return np.clip(x, -1.0, 1.0).astype(np.float32)
+
+
+def utterances(n: int, seed: int, min_s: float = 1.5, max_s: float = 15.0) -> list[np.ndarray]:
+    """n utterances with lengths uniform in [min_s, max_s] seconds (a ragged batch)."""
+    seqs = np.random.SeedSequence(seed).spawn(n + 1)
+    lens = np.random.default_rng(seqs[0]).uniform(min_s, max_s, size=n)
+    return [utterance(np.random.default_rng(seqs[i + 1]), float(lens[i])) for i in range(n)]

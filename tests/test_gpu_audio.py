@@ -1,0 +1,153 @@
+"""GPU parity of the audio path (log Mel spectrogram, three-pass normalisation) against the
+float64 oracle, through the C ABI; host-side checks of sizes, packing and arguments."""
+from __future__ import annotations
+
+import ctypes
+
+import numpy as np
+import pytest
+
+from oracle import audio as oa
+from paper_2411_19114_b200 import binding as pb
+from paper_2411_19114_b200 import workloads as wl
+
+# fp32 FFT of 512 points, fp32 Mel sums and logf against float64: see the design doc
+LOGMEL_TOL = 2e-3
+NORM_TOL = 2e-3
+
+
+def test_sizes_and_pack_layout():
+    rng = np.random.default_rng(1)
+    utts = [rng.uniform(-1, 1, size=n).astype(np.float32) for n in (401, 0, 399, 1601, 16000)]
+    s = pb.preba_audio_query([u.size for u in utts])
+    offs, at = [], 0
+    for u in utts:
+        offs.append(at)
+        at = -(-(at + u.size) // 4) * 4
+    assert s.packed_samples == at and s.table_bytes == 16 * 5
+    assert s.t_max == oa.num_frames(16000) == 98 and s.out_bytes == 5 * 80 * 98 * 4
+    packed, table = pb.preba_audio_pack(utts)
+    assert [int(e["offset"]) for e in table] == offs
+    assert [int(e["frames"]) for e in table] == [oa.num_frames(u.size) for u in utts]
+    covered = np.zeros(at, dtype=bool)
+    for u, o in zip(utts, offs):
+        assert np.array_equal(packed[o:o + u.size], u)
+        covered[o:o + u.size] = True
+    assert np.all(packed[~covered] == 0.0)
+
+
+def test_audio_entry_point_rejects_bad_arguments_before_any_launch():
+    L = pb.lib()
+    assert L.preba_audio_logmel(None, 1, None) == pb.ERR_INVALID_ARG
+    t = np.zeros(1, dtype=pb.UTT_DTYPE)
+    t[0] = (0, 800, 3)
+
+    def call(**kw):
+        b = pb.PrebaAudioBatch()
+        b.samples, b.samples_count = 0x10000, 800
+        b.table, b.table_host = 0x20000, t.ctypes.data
+        b.n, b.t_max = 1, 3
+        b.out, b.out_bytes = 0x30000, 80 * 3 * 4
+        for k, v in kw.items():
+            setattr(b, k, v)
+        return L.preba_audio_logmel(ctypes.byref(b), 1, None)
+
+    assert call(samples=None) == pb.ERR_INVALID_ARG
+    assert call(samples=0x10004) == pb.ERR_INVALID_ARG          # misaligned samples
+    assert call(n=0) == pb.ERR_INVALID_ARG
+    assert call(t_max=0) == pb.ERR_INVALID_ARG
+    assert call(out_bytes=80 * 3 * 4 - 1) == pb.ERR_BUFFER_TOO_SMALL
+    assert call(samples_count=799) == pb.ERR_BAD_TABLE          # runs past the samples
+    assert call(t_max=2, out_bytes=80 * 3 * 4) == pb.ERR_BAD_TABLE  # more frames than the result holds
+    t[0] = (0, 800, 4)
+    assert call() == pb.ERR_BAD_TABLE                           # frame count does not follow from length
+    t[0] = (2, 700, 2)
+    assert call() == pb.ERR_BAD_TABLE                           # misaligned offset
+
+
+def run_audio(utts, normalize):
+    import torch
+
+    n = len(utts)
+    packed, table = pb.preba_audio_pack(utts)
+    t_max = max(1, pb.preba_audio_query([u.size for u in utts]).t_max)
+    dev = torch.device("cuda:0")
+    smp = torch.from_numpy(packed).to(dev)
+    tab = torch.from_numpy(table.view(np.uint8)).to(dev)
+    guard = 1024
+    buf = torch.full((guard + n * 80 * t_max + guard,), 777.0, dtype=torch.float32, device=dev)
+    out = buf[guard:guard + n * 80 * t_max]
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    pb.preba_audio_logmel(smp, tab, n, t_max, out, normalize, table_host=table, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    host = buf.cpu().numpy()
+    assert np.all(host[:guard] == 777.0) and np.all(host[guard + n * 80 * t_max:] == 777.0)
+    return host[guard:guard + n * 80 * t_max].reshape(n, 80, t_max).copy()
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("normalize", [False, True])
+def test_ragged_batch_matches_the_oracle(normalize):
+    rng = np.random.default_rng(2)
+    utts = wl.utterances(6, seed=3, min_s=0.2, max_s=2.5)
+    utts += [rng.uniform(-1, 1, size=n).astype(np.float32) for n in (400, 399, 0, 559, 560, 561, 720)]
+    utts.append(np.zeros(1000, dtype=np.float32))               # silence: every energy is the guard
+    got = run_audio(utts, normalize)
+    want = oa.preprocess(utts, normalized=normalize)
+    assert got.shape == want.shape
+    err = np.abs(got.astype(np.float64) - want)
+    assert float(err.max()) <= (NORM_TOL if normalize else LOGMEL_TOL), float(err.max())
+    for i, u in enumerate(utts):                                 # padding is exactly zero
+        assert np.all(got[i, :, oa.num_frames(u.size):] == 0.0)
+
+
+@pytest.mark.gpu
+def test_pure_tones_and_impulses_on_the_gpu():
+    """Closed forms on the device itself: a constant gives (200 c)^2 at bin 0 only through the
+    first filter's rising edge (weight 0 at 0 Hz): all-guard energies except leakage; an impulse
+    gives a flat spectrum w^2, so every filter's energy is w^2 times the sum of its weights."""
+    x = np.zeros(400 + 160, dtype=np.float32)
+    x[290] = 1.0                                                # frame 0 position 290, frame 1 position 130
+    got = run_audio([x], False)[0]
+    w = 0.5 - 0.5 * np.cos(2 * np.pi * np.arange(400) / 400)
+    fb_sum = oa.mel_filterbank().sum(axis=1)
+    for t, pos in ((0, 290), (1, 130)):
+        want = np.log(w[pos] ** 2 * fb_sum + 2.0 ** -24)
+        assert np.max(np.abs(got[:, t] - want)) <= 1e-3
+
+
+@pytest.mark.gpu
+def test_full_size_utterances_sampled_rows():
+    utts = wl.utterances(8, seed=5)
+    got = run_audio(utts, True)
+    rng = np.random.default_rng(6)
+    for i in rng.choice(len(utts), size=3, replace=False):
+        want = oa.preprocess([utts[i]])[0]
+        t = want.shape[1]
+        assert float(np.max(np.abs(got[i, :, :t] - want))) <= NORM_TOL
+        assert np.all(got[i, :, t:] == 0.0)
+
+
+@pytest.mark.gpu
+def test_device_side_table_check_skips_bad_entries():
+    import torch
+
+    utts = wl.utterances(3, seed=7, min_s=0.2, max_s=0.6)
+    packed, table = pb.preba_audio_pack(utts)
+    t_max = int(table["frames"].max())
+    bad = table.copy()
+    bad[1]["frames"] += 1                                        # does not follow from its length
+    dev = torch.device("cuda:0")
+    smp = torch.from_numpy(packed).to(dev)
+    tab = torch.from_numpy(bad.view(np.uint8)).to(dev)
+    out = torch.full((3, 80, t_max), 5.0, dtype=torch.float32, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    pb.preba_audio_logmel(smp, tab, 3, t_max, out, True, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == pb.ERR_BAD_TABLE
+    host = out.cpu().numpy()
+    assert np.all(host[1] == 0.0)                                # refused entry: zeros
+    want = oa.preprocess(utts)
+    for i in (0, 2):
+        assert float(np.max(np.abs(host[i] - want[i, :, :t_max]))) <= NORM_TOL
