@@ -297,6 +297,136 @@ def run_streams(args, local_rank: int) -> None:
     print(json.dumps(line), flush=True)
 
 
+# Algorithmic fp32 operations of the audio path per frame: window 400, real 512-point FFT
+# 2.5 N log2 N = 11520, power spectrum 3 x 257, Mel filters 2 per non-zero weight (510),
+# log 80, three-pass normalisation 6 x 80.
+AUDIO_FLOPS_PER_FRAME = 400 + 11520 + 3 * 257 + 2 * 510 + 80 + 6 * 80
+# fp32 multiply-add peak from unit counts and the clock: SMs x 128 lanes x 2 x max SM clock
+AUDIO_ALU_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
+
+
+def run_audio(args, local_rank: int) -> None:
+    """The paper's second path (Table 1 "Mel spectrogram" + "Normalize") on a ragged batch of
+    synthetic utterances: device-resident throughput, end to end from pinned host samples, and
+    the numpy oracle timed on the host."""
+    import torch
+
+    from oracle import audio as oa
+    from paper_2411_19114_b200 import binding as pb
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device (the CUDA path has no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    pb.lib()
+    n = args.batch or 64
+    utts = wl.utterances(n, seed=11)
+    packed, table = pb.preba_audio_pack(utts)
+    t_max = int(table["frames"].max())
+    frames = int(table["frames"].sum())
+    seconds = sum(u.size for u in utts) / wl.AUDIO_RATE
+    steps, warm = min(args.steps, 2000), max(args.warmup, 3)
+    l2 = torch.cuda.get_device_properties(dev).L2_cache_size
+    step_bytes = packed.nbytes + n * 80 * t_max * 4
+    sets = max(2, min(32, -(-4 * l2 // step_bytes)))
+    smp = [torch.from_numpy(packed).to(dev) for _ in range(sets)]
+    outs = [torch.empty((n, 80, t_max), dtype=torch.float32, device=dev) for _ in range(sets)]
+    tab = torch.from_numpy(table.view(np.uint8)).to(dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    stream = torch.cuda.current_stream()
+    calls = [pb.PreparedAudio(smp[i], tab, n, t_max, outs[i], True, stream=stream, status=status)
+             for i in range(sets)]
+    for i in range(warm):
+        calls[i % sets]()
+    torch.cuda.synchronize()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local_rank) as clocks:
+        torch.cuda.synchronize()
+        start.record(stream)
+        for i in range(steps):
+            calls[i % sets]()
+        stop.record(stream)
+        torch.cuda.synchronize()
+    ms = start.elapsed_time(stop)
+    assert int(status.item()) == 0
+    # parity of what was timed, on a sample of utterances
+    got = outs[0].cpu().numpy()
+    for i in (0, n // 2, n - 1):
+        want = oa.preprocess([utts[i]])[0]
+        err = float(np.max(np.abs(got[i, :, :want.shape[1]] - want)))
+        assert err <= 2e-3, f"audio result differs from the oracle: {err:.3e}"
+    # end to end: pinned samples -> device, two kernels, result -> pinned memory
+    e2e_steps = max(3, min(args.e2e_steps, steps))
+    ph = torch.from_numpy(packed).pin_memory()
+    oh = [torch.empty((n, 80, t_max), dtype=torch.float32).pin_memory() for _ in range(2)]
+    side = [torch.cuda.Stream(device=dev) for _ in range(2)]
+    done = [torch.cuda.Event() for _ in range(2)]
+    e_calls = [pb.PreparedAudio(smp[b], tab, n, t_max, outs[b], True, stream=side[b],
+                                status=status) for b in range(2)]
+
+    def e2e_step(i):
+        b = i % 2
+        done[b].synchronize()
+        with torch.cuda.stream(side[b]):
+            smp[b].copy_(ph, non_blocking=True)
+            e_calls[b]()
+            oh[b].copy_(outs[b], non_blocking=True)
+        done[b].record(side[b])
+
+    for i in range(2):
+        e2e_step(i)
+    torch.cuda.synchronize()
+    e_start, e_stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e_start.record(stream)
+    for st in side:
+        st.wait_stream(stream)
+    for i in range(e2e_steps):
+        e2e_step(i)
+    for st in side:
+        stream.wait_stream(st)
+    e_stop.record(stream)
+    torch.cuda.synchronize()
+    e2e_ms = e_start.elapsed_time(e_stop)
+    # the oracle as it stands (numpy, one thread), on a sample of the batch
+    t_end, done_frames, spent, k = time.perf_counter() + args.cpu_budget, 0, 0.0, 0
+    while k < n and (k == 0 or time.perf_counter() < t_end):
+        t0 = time.perf_counter()
+        oa.preprocess([utts[k]])
+        spent += time.perf_counter() - t0
+        done_frames += int(table["frames"][k])
+        k += 1
+    per_launch_s = ms * 1e-3 / steps
+    achieved = frames * AUDIO_FLOPS_PER_FRAME / per_launch_s / 1e12
+    line = {
+        "metric": "log-Mel frames/sec (audio path)", "value": frames / per_launch_s,
+        "unit": "frames/s", "n_gpus": 1, "steps": steps, "warmup": warm,
+        "ms_per_step": ms / steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"{n} synthetic utterances, 1.5-15 s at 16 kHz ({seconds:.0f} s of "
+                               f"audio, {frames} frames of 400 samples every 160), 80 log-Mel "
+                               "features, per-utterance normalisation, fp32 out",
+                   "utterances_per_step": n, "audio_seconds_per_step": seconds,
+                   "launch": "two kernels per step (spectrogram, normalise), one stream",
+                   "l2": f"rotating {sets} buffer sets ({sets * step_bytes / 1e6:.0f} MB) > L2 "
+                         f"({l2 / 1e6:.0f} MB)"},
+        "roofline": {"bound": "alu", "achieved": achieved, "peak": AUDIO_ALU_PEAK_TFLOPS,
+                     "unit": "TFLOP/s", "frac": achieved / AUDIO_ALU_PEAK_TFLOPS, "traffic": None,
+                     "peak_source": "148 SMs x 128 fp32 lanes x 2 x 1.965 GHz",
+                     "algorithmic_flops_per_frame": AUDIO_FLOPS_PER_FRAME,
+                     "kernel_us": per_launch_s * 1e6},
+        "cpu_baseline": {"value": done_frames / spent, "unit": "frames/s", "cores": 1,
+                         "kind": "oracle", "sample": f"{k} of the {n} utterances, one pass"},
+        "e2e": {"value": frames * e2e_steps / (e2e_ms * 1e-3), "unit": "frames/s",
+                "h2d_bytes_per_step": int(packed.nbytes), "d2h_bytes_per_step": n * 80 * t_max * 4,
+                "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps,
+                "includes": "packed samples pinned -> device, both kernels, result -> pinned "
+                            "memory; two buffer sets on two streams"},
+        "audio_seconds_per_second": seconds / per_launch_s,
+        "gpu_launches": 2 * steps, "clocks": clocks.summary(),
+    }
+    print(json.dumps(line), flush=True)
+
+
 def report_variant(args, rank, world, n, elapsed_ms, acct, desc, dtype, sets, step_bytes, l2,
                    clocks, dist, dev, t_host) -> None:
     """The JSON line of a --variant run: the device-resident leg only."""
@@ -634,7 +764,7 @@ def main() -> None:
     ap.add_argument("--warmup", type=int, default=200)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="mixed",
-                    choices=["mixed", "320x240", "1080p", "sweep", "streams"])
+                    choices=["mixed", "320x240", "1080p", "sweep", "streams", "audio"])
     ap.add_argument("--batch", type=int, default=None)
     ap.add_argument("--variant", default="plain", choices=["plain", "u8", "round"],
                     help="device-resident leg through preba_preprocess_ex: u8 = rounded uint8 "
@@ -651,6 +781,9 @@ def main() -> None:
     elif args.workload == "streams":
         if rank == 0:
             run_streams(args, local_rank)
+    elif args.workload == "audio":
+        if rank == 0:
+            run_audio(args, local_rank)
     else:
         run_ours(args, rank, world, local_rank)
 

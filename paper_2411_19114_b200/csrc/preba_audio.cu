@@ -27,7 +27,8 @@ constexpr uint32_t kFft = PREBA_AUDIO_NFFT;
 constexpr uint32_t kBins = kFft / 2 + 1;
 constexpr uint32_t kMels = PREBA_AUDIO_MELS;
 constexpr int kWarps = 4;            // warps per CTA of the spectrogram kernel
-constexpr int kFramesPerCta = 2 * kWarps;
+constexpr int kPairsPerWarp = 4;      // frame pairs a warp transforms one after the other
+constexpr int kFramesPerCta = 2 * kWarps * kPairsPerWarp;
 constexpr float kLogGuard = 5.9604644775390625e-08f;  // 2^-24
 constexpr float kStdGuard = 1e-5f;
 
@@ -95,92 +96,118 @@ __device__ __forceinline__ bool utt_ok(const preba_utt_t& u, uint64_t samples_co
   return u.frames == frames;
 }
 
+// Element i of the complex sequence lives at i + i / 16: one element of padding after every
+// sixteen keeps the bit-reversed stores and the strided butterflies free of bank conflicts.
+__device__ __forceinline__ uint32_t zi(uint32_t i) { return i + (i >> 4); }
+
 struct __align__(16) WarpFft {
-  float2 z[kFft];       // the complex sequence, then its spectrum
+  float2 z[kFft + kFft / 16];  // the complex sequence, then its spectrum (padded, see zi)
   float power[2][kBins + 3];
 };
 
 __global__ void __launch_bounds__(32 * kWarps)
-logmel_kernel(const AudioParams p, const MelTable mel) {
+logmel_kernel(const AudioParams p, const MelTable mel_param) {
   __shared__ WarpFft sm[kWarps];
-  __shared__ float2 twiddle[kFft / 2];  // exp(-2 pi i k / 512)
+  // stage s (butterflies of span 2^s) uses exp(-2 pi i pos / 2^(s+1)), pos < 2^s, stored
+  // one stage after the other from index 2^s - 1, so that a stage reads consecutive entries
+  __shared__ float2 twiddle[kFft - 1];
   __shared__ float window[kWin];
+  __shared__ MelTable mel;  // lanes read different entries: shared memory, not the constant bank
   const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  for (uint32_t k = threadIdx.x; k < kFft / 2; k += blockDim.x) {
+  const uint32_t utt = blockIdx.y;
+  const preba_utt_t u = p.table[utt];
+  const bool ok = utt_ok(u, p.samples_count);
+  if (!ok && threadIdx.x == 0 && blockIdx.x == 0 && p.status)
+    atomicCAS(p.status, 0, PREBA_ERR_BAD_TABLE);
+  const uint32_t frames = ok ? min(u.frames, p.t_max) : 0u;
+  float* __restrict__ out = p.out + static_cast<size_t>(utt) * kMels * p.t_max;
+  const uint32_t cta_t0 = blockIdx.x * kFramesPerCta;
+  if (cta_t0 >= frames) {
+    // padding (or a refused entry): zeros for all of this CTA's frames
+    const uint32_t t_end = min(cta_t0 + kFramesPerCta, p.t_max);
+    for (uint32_t j = warp; j < kMels; j += kWarps)
+      for (uint32_t t = cta_t0 + lane; t < t_end; t += 32) out[static_cast<size_t>(j) * p.t_max + t] = 0.f;
+    return;
+  }
+  for (uint32_t k = threadIdx.x; k < kFft - 1; k += blockDim.x) {
+    const uint32_t stage = 31 - __clz(k + 1), pos = k + 1 - (1u << stage);
     float s, c;
-    sincospif(-2.0f * static_cast<float>(k) / kFft, &s, &c);
+    sincospif(-static_cast<float>(pos) / static_cast<float>(1u << stage), &s, &c);
     twiddle[k] = make_float2(c, s);
   }
   for (uint32_t i = threadIdx.x; i < kWin; i += blockDim.x)
     window[i] = 0.5f - 0.5f * cospif(2.0f * static_cast<float>(i) / kWin);
+  {
+    const uint32_t* src = reinterpret_cast<const uint32_t*>(&mel_param);
+    uint32_t* dst = reinterpret_cast<uint32_t*>(&mel);
+    for (uint32_t i = threadIdx.x; i < sizeof(MelTable) / 4; i += blockDim.x) dst[i] = src[i];
+  }
   __syncthreads();
 
-  const uint32_t utt = blockIdx.y;
-  const preba_utt_t u = p.table[utt];
-  const bool ok = utt_ok(u, p.samples_count);
-  if (!ok && threadIdx.x == 0 && p.status) atomicCAS(p.status, 0, PREBA_ERR_BAD_TABLE);
-  const uint32_t frames = ok ? min(u.frames, p.t_max) : 0u;
-  const uint32_t t0 = blockIdx.x * kFramesPerCta + 2 * warp;  // this warp's two frames
-  if (t0 >= p.t_max) return;
-  float* __restrict__ out = p.out + static_cast<size_t>(utt) * kMels * p.t_max;
-  const bool have0 = t0 < frames, have1 = t0 + 1 < frames;
-  if (!have0) {
-    // padding (or a refused entry): zeros for both frames of this warp
-    for (uint32_t j = lane; j < kMels; j += 32) {
-      out[static_cast<size_t>(j) * p.t_max + t0] = 0.f;
-      if (t0 + 1 < p.t_max) out[static_cast<size_t>(j) * p.t_max + t0 + 1] = 0.f;
-    }
-    return;
-  }
   WarpFft& ws = sm[warp];
-  const float* __restrict__ x = p.samples + u.offset + static_cast<size_t>(t0) * kHop;
-  // windowed frames as real and imaginary part, stored in bit-reversed order
-  for (uint32_t i = lane; i < kFft; i += 32) {
-    float re = 0.f, im = 0.f;
-    if (i < kWin) {
-      re = x[i] * window[i];
-      if (have1) im = x[i + kHop] * window[i];
-    }
-    ws.z[__brev(i) >> 23] = make_float2(re, im);
-  }
-  __syncwarp();
-  // nine radix-2 stages, eight butterflies per lane and stage
 #pragma unroll 1
-  for (uint32_t s = 0; s < 9; ++s) {
-    const uint32_t half = 1u << s;
-#pragma unroll
-    for (uint32_t q = 0; q < 8; ++q) {
-      const uint32_t b = lane + 32 * q;
-      const uint32_t pos = b & (half - 1);
-      const uint32_t i = ((b >> s) << (s + 1)) + pos;
-      const float2 w = twiddle[pos << (8 - s)];
-      const float2 a = ws.z[i], c = ws.z[i + half];
-      const float2 v = make_float2(c.x * w.x - c.y * w.y, c.x * w.y + c.y * w.x);
-      ws.z[i] = make_float2(a.x + v.x, a.y + v.y);
-      ws.z[i + half] = make_float2(a.x - v.x, a.y - v.y);
+  for (uint32_t pair = 0; pair < kPairsPerWarp; ++pair) {
+    const uint32_t t0 = cta_t0 + 2 * (warp + kWarps * pair);  // this warp's two frames
+    if (t0 >= p.t_max) break;
+    const bool have0 = t0 < frames, have1 = t0 + 1 < frames;
+    if (!have0) {
+      for (uint32_t j = lane; j < kMels; j += 32) {
+        out[static_cast<size_t>(j) * p.t_max + t0] = 0.f;
+        if (t0 + 1 < p.t_max) out[static_cast<size_t>(j) * p.t_max + t0 + 1] = 0.f;
+      }
+      continue;
+    }
+    const float* __restrict__ x = p.samples + u.offset + static_cast<size_t>(t0) * kHop;
+    // windowed frames as real and imaginary part, stored in bit-reversed order
+    for (uint32_t i = lane; i < kFft; i += 32) {
+      float re = 0.f, im = 0.f;
+      if (i < kWin) {
+        re = x[i] * window[i];
+        if (have1) im = x[i + kHop] * window[i];
+      }
+      ws.z[zi(__brev(i) >> 23)] = make_float2(re, im);
     }
     __syncwarp();
-  }
-  // Z = A + iB with A, B the spectra of the two real frames:
-  // A[k] = (Z[k] + conj(Z[N-k]))/2, B[k] = (Z[k] - conj(Z[N-k]))/(2i)
-  for (uint32_t k = lane; k < kBins; k += 32) {
-    const float2 zk = ws.z[k], zn = ws.z[(kFft - k) & (kFft - 1)];
-    const float ar = 0.5f * (zk.x + zn.x), ai = 0.5f * (zk.y - zn.y);
-    const float br = 0.5f * (zk.y + zn.y), bi = 0.5f * (zn.x - zk.x);
-    ws.power[0][k] = ar * ar + ai * ai;
-    ws.power[1][k] = br * br + bi * bi;
-  }
-  __syncwarp();
-  for (uint32_t j = lane; j < kMels; j += 32) {
-    float e0 = 0.f, e1 = 0.f;
-    for (uint32_t k = mel.first[j]; k < mel.last[j]; ++k) {
-      const float wgt = mel.m[k] == j ? mel.up[k] : 1.0f - mel.up[k];
-      e0 = fmaf(wgt, ws.power[0][k], e0);
-      e1 = fmaf(wgt, ws.power[1][k], e1);
+    // nine radix-2 stages, eight butterflies per lane and stage
+#pragma unroll 1
+    for (uint32_t s = 0; s < 9; ++s) {
+      const uint32_t half = 1u << s;
+#pragma unroll
+      for (uint32_t q = 0; q < 8; ++q) {
+        const uint32_t b = lane + 32 * q;
+        const uint32_t pos = b & (half - 1);
+        const uint32_t i = ((b >> s) << (s + 1)) + pos;
+        const float2 w = twiddle[half - 1 + pos];
+        const uint32_t ia = zi(i), ic = zi(i + half);
+        const float2 a = ws.z[ia], c = ws.z[ic];
+        const float2 v = make_float2(c.x * w.x - c.y * w.y, c.x * w.y + c.y * w.x);
+        ws.z[ia] = make_float2(a.x + v.x, a.y + v.y);
+        ws.z[ic] = make_float2(a.x - v.x, a.y - v.y);
+      }
+      __syncwarp();
     }
-    out[static_cast<size_t>(j) * p.t_max + t0] = logf(e0 + kLogGuard);
-    if (t0 + 1 < p.t_max)
-      out[static_cast<size_t>(j) * p.t_max + t0 + 1] = have1 ? logf(e1 + kLogGuard) : 0.f;
+    // Z = A + iB with A, B the spectra of the two real frames:
+    // A[k] = (Z[k] + conj(Z[N-k]))/2, B[k] = (Z[k] - conj(Z[N-k]))/(2i)
+    for (uint32_t k = lane; k < kBins; k += 32) {
+      const float2 zk = ws.z[zi(k)], zn = ws.z[zi((kFft - k) & (kFft - 1))];
+      const float ar = 0.5f * (zk.x + zn.x), ai = 0.5f * (zk.y - zn.y);
+      const float br = 0.5f * (zk.y + zn.y), bi = 0.5f * (zn.x - zk.x);
+      ws.power[0][k] = ar * ar + ai * ai;
+      ws.power[1][k] = br * br + bi * bi;
+    }
+    __syncwarp();
+    for (uint32_t j = lane; j < kMels; j += 32) {
+      float e0 = 0.f, e1 = 0.f;
+      for (uint32_t k = mel.first[j]; k < mel.last[j]; ++k) {
+        const float wgt = mel.m[k] == j ? mel.up[k] : 1.0f - mel.up[k];
+        e0 = fmaf(wgt, ws.power[0][k], e0);
+        e1 = fmaf(wgt, ws.power[1][k], e1);
+      }
+      out[static_cast<size_t>(j) * p.t_max + t0] = logf(e0 + kLogGuard);
+      if (t0 + 1 < p.t_max)
+        out[static_cast<size_t>(j) * p.t_max + t0 + 1] = have1 ? logf(e1 + kLogGuard) : 0.f;
+    }
+    __syncwarp();  // the next pair reuses this warp's buffers
   }
 }
 
