@@ -2,7 +2,8 @@
 //
 // Kernel 1: a warp takes two consecutive frames of one utterance, multiplies them by the Hann
 // window, packs them as the real and imaginary part of one complex sequence, runs a 512-point
-// radix-2 FFT in its own shared memory, separates the two spectra, forms the power spectra,
+// FFT as three passes of radix-8 butterflies in registers (exchanging through its own shared
+// memory between passes), separates the two spectra, forms the power spectra,
 // applies the triangular Mel filters (a lane per filter, the filter's few bins read from
 // shared memory) and writes log(energy + 2^-24).  Frames past an utterance's own count are
 // written as 0, so the result tensor needs no clearing.
@@ -96,21 +97,53 @@ __device__ __forceinline__ bool utt_ok(const preba_utt_t& u, uint64_t samples_co
   return u.frames == frames;
 }
 
-// Element i of the complex sequence lives at i + i / 16: one element of padding after every
-// sixteen keeps the bit-reversed stores and the strided butterflies free of bank conflicts.
-__device__ __forceinline__ uint32_t zi(uint32_t i) { return i + (i >> 4); }
+// The 512-point FFT runs as three passes of radix-8 butterflies held in registers
+// (512 = 8 * 8 * 8); between passes the warp exchanges its values through an 8 x 64 array in
+// shared memory whose rows are 68 elements apart, which keeps every exchange at the two
+// wavefronts a 64-bit access of 32 lanes needs.
+constexpr uint32_t kPitch = 68;
 
 struct __align__(16) WarpFft {
-  float2 z[kFft + kFft / 16];  // the complex sequence, then its spectrum (padded, see zi)
+  float2 z[8 * kPitch];  // exchange array, then the spectrum in natural order (first 512)
   float power[2][kBins + 3];
 };
+
+__device__ __forceinline__ float2 cadd(float2 a, float2 b) { return make_float2(a.x + b.x, a.y + b.y); }
+__device__ __forceinline__ float2 csub(float2 a, float2 b) { return make_float2(a.x - b.x, a.y - b.y); }
+__device__ __forceinline__ float2 cmul(float2 a, float2 b) {
+  return make_float2(a.x * b.x - a.y * b.y, a.x * b.y + a.y * b.x);
+}
+__device__ __forceinline__ float2 mul_neg_i(float2 a) { return make_float2(a.y, -a.x); }
+
+// 8-point DFT in place, X[k] = sum_n v[n] exp(-2 pi i n k / 8), natural order in and out.
+__device__ __forceinline__ void fft8(float2 (&v)[8]) {
+  const float h = 0.70710678118654752440f;
+  const float2 s0 = cadd(v[0], v[4]), s1 = cadd(v[1], v[5]), s2 = cadd(v[2], v[6]),
+               s3 = cadd(v[3], v[7]);
+  const float2 t0 = csub(v[0], v[4]), t1 = csub(v[1], v[5]), t2 = csub(v[2], v[6]),
+               t3 = csub(v[3], v[7]);
+  const float2 d0 = t0;
+  const float2 d1 = make_float2(h * (t1.x + t1.y), h * (t1.y - t1.x));   // * exp(-i pi/4)
+  const float2 d2 = mul_neg_i(t2);                                      // * exp(-i pi/2)
+  const float2 d3 = make_float2(h * (t3.y - t3.x), -h * (t3.x + t3.y));  // * exp(-3i pi/4)
+  const float2 e0 = cadd(s0, s2), e1 = csub(s0, s2), e2 = cadd(s1, s3),
+               e3 = mul_neg_i(csub(s1, s3));
+  const float2 o0 = cadd(d0, d2), o1 = csub(d0, d2), o2 = cadd(d1, d3),
+               o3 = mul_neg_i(csub(d1, d3));
+  v[0] = cadd(e0, e2);
+  v[4] = csub(e0, e2);
+  v[2] = cadd(e1, e3);
+  v[6] = csub(e1, e3);
+  v[1] = cadd(o0, o2);
+  v[5] = csub(o0, o2);
+  v[3] = cadd(o1, o3);
+  v[7] = csub(o1, o3);
+}
 
 __global__ void __launch_bounds__(32 * kWarps)
 logmel_kernel(const AudioParams p, const MelTable mel_param) {
   __shared__ WarpFft sm[kWarps];
-  // stage s (butterflies of span 2^s) uses exp(-2 pi i pos / 2^(s+1)), pos < 2^s, stored
-  // one stage after the other from index 2^s - 1, so that a stage reads consecutive entries
-  __shared__ float2 twiddle[kFft - 1];
+  __shared__ float2 twiddle[kFft];  // exp(-2 pi i j / 512)
   __shared__ float window[kWin];
   __shared__ MelTable mel;  // lanes read different entries: shared memory, not the constant bank
   const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -129,10 +162,9 @@ logmel_kernel(const AudioParams p, const MelTable mel_param) {
       for (uint32_t t = cta_t0 + lane; t < t_end; t += 32) out[static_cast<size_t>(j) * p.t_max + t] = 0.f;
     return;
   }
-  for (uint32_t k = threadIdx.x; k < kFft - 1; k += blockDim.x) {
-    const uint32_t stage = 31 - __clz(k + 1), pos = k + 1 - (1u << stage);
+  for (uint32_t k = threadIdx.x; k < kFft; k += blockDim.x) {
     float s, c;
-    sincospif(-static_cast<float>(pos) / static_cast<float>(1u << stage), &s, &c);
+    sincospif(-2.0f * static_cast<float>(k) / kFft, &s, &c);
     twiddle[k] = make_float2(c, s);
   }
   for (uint32_t i = threadIdx.x; i < kWin; i += blockDim.x)
@@ -158,38 +190,69 @@ logmel_kernel(const AudioParams p, const MelTable mel_param) {
       continue;
     }
     const float* __restrict__ x = p.samples + u.offset + static_cast<size_t>(t0) * kHop;
-    // windowed frames as real and imaginary part, stored in bit-reversed order
-    for (uint32_t i = lane; i < kFft; i += 32) {
-      float re = 0.f, im = 0.f;
-      if (i < kWin) {
-        re = x[i] * window[i];
-        if (have1) im = x[i + kHop] * window[i];
+    // With n = 64 n2 + 8 n1 + n0 and k = k0 + 8 k1 + 64 k2:
+    //   X[k] = sum_n0 W8^(n0 k2) W512^(n0 (k0 + 8 k1))
+    //          sum_n1 W8^(n1 k1) W64^(n1 k0) sum_n2 W8^(n2 k0) x[n].
+    // Pass 1 (over n2): a lane takes the columns p = 8 n1 + n0 = lane and lane + 32 of the two
+    // windowed frames (real and imaginary part).
+    float2 v[2][8];
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+      const uint32_t pcol = lane + 32 * c;
+#pragma unroll
+      for (uint32_t n2 = 0; n2 < 8; ++n2) {
+        const uint32_t i = 64 * n2 + pcol;
+        float re = 0.f, im = 0.f;
+        if (i < kWin) {
+          re = x[i] * window[i];
+          if (have1) im = x[i + kHop] * window[i];
+        }
+        v[c][n2] = make_float2(re, im);
       }
-      ws.z[zi(__brev(i) >> 23)] = make_float2(re, im);
+      fft8(v[c]);
+      const uint32_t n1 = pcol >> 3;
+#pragma unroll
+      for (uint32_t k0 = 0; k0 < 8; ++k0)
+        ws.z[k0 * kPitch + pcol] = k0 ? cmul(v[c][k0], twiddle[8 * n1 * k0]) : v[c][0];
     }
     __syncwarp();
-    // nine radix-2 stages, eight butterflies per lane and stage
-#pragma unroll 1
-    for (uint32_t s = 0; s < 9; ++s) {
-      const uint32_t half = 1u << s;
+    // Pass 2 (over n1): a lane takes q = 8 k0 + n0.
 #pragma unroll
-      for (uint32_t q = 0; q < 8; ++q) {
-        const uint32_t b = lane + 32 * q;
-        const uint32_t pos = b & (half - 1);
-        const uint32_t i = ((b >> s) << (s + 1)) + pos;
-        const float2 w = twiddle[half - 1 + pos];
-        const uint32_t ia = zi(i), ic = zi(i + half);
-        const float2 a = ws.z[ia], c = ws.z[ic];
-        const float2 v = make_float2(c.x * w.x - c.y * w.y, c.x * w.y + c.y * w.x);
-        ws.z[ia] = make_float2(a.x + v.x, a.y + v.y);
-        ws.z[ic] = make_float2(a.x - v.x, a.y - v.y);
-      }
-      __syncwarp();
+    for (int c = 0; c < 2; ++c) {
+      const uint32_t q = lane + 32 * c, k0 = q >> 3, n0 = q & 7;
+#pragma unroll
+      for (uint32_t n1 = 0; n1 < 8; ++n1) v[c][n1] = ws.z[k0 * kPitch + 8 * n1 + n0];
     }
+    __syncwarp();
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+      const uint32_t q = lane + 32 * c, k0 = q >> 3, n0 = q & 7;
+      fft8(v[c]);
+#pragma unroll
+      for (uint32_t k1 = 0; k1 < 8; ++k1)
+        ws.z[n0 * kPitch + k0 + 8 * k1] = cmul(v[c][k1], twiddle[n0 * (k0 + 8 * k1)]);
+    }
+    __syncwarp();
+    // Pass 3 (over n0): a lane takes r = k0 + 8 k1 and produces X[r + 64 k2].
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+      const uint32_t r = lane + 32 * c;
+#pragma unroll
+      for (uint32_t n0 = 0; n0 < 8; ++n0) v[c][n0] = ws.z[n0 * kPitch + r];
+    }
+    __syncwarp();
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+      const uint32_t r = lane + 32 * c;
+      fft8(v[c]);
+#pragma unroll
+      for (uint32_t k2 = 0; k2 < 8; ++k2) ws.z[r + 64 * k2] = v[c][k2];
+    }
+    __syncwarp();
     // Z = A + iB with A, B the spectra of the two real frames:
     // A[k] = (Z[k] + conj(Z[N-k]))/2, B[k] = (Z[k] - conj(Z[N-k]))/(2i)
     for (uint32_t k = lane; k < kBins; k += 32) {
-      const float2 zk = ws.z[zi(k)], zn = ws.z[zi((kFft - k) & (kFft - 1))];
+      const float2 zk = ws.z[k], zn = ws.z[(kFft - k) & (kFft - 1)];
       const float ar = 0.5f * (zk.x + zn.x), ai = 0.5f * (zk.y - zn.y);
       const float br = 0.5f * (zk.y + zn.y), bi = 0.5f * (zn.x - zk.x);
       ws.power[0][k] = ar * ar + ai * ai;
