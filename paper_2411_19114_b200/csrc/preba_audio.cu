@@ -33,20 +33,22 @@ constexpr int kFramesPerCta = 2 * kWarps * kPairsPerWarp;
 constexpr float kLogGuard = 5.9604644775390625e-08f;  // 2^-24
 constexpr float kStdGuard = 1e-5f;
 
-// The Mel filters in the form the kernel uses.  Bin k lies between corner frequencies
-// c[m] <= f < c[m+1]; it adds `up[k]` of its power to filter m (rising edge) and 1 - up[k] to
-// filter m - 1 (falling edge).  Filter j therefore gathers the bins whose m is j or j + 1:
-// the contiguous range [first[j], last[j]).
+// The Mel filters in the form the kernel uses: filter j covers the consecutive bins
+// first[j] .. first[j] + count[j] - 1 and their weights lie one after the other in w from
+// start[j] (rising edge, then falling edge; every bin belongs to at most two filters).
+constexpr uint32_t kMelWeights = 2 * kBins + 2;
 struct MelTable {
-  float up[kBins];
-  uint8_t m[kBins + 3];   // 255: the bin lies outside every filter
+  float w[kMelWeights];
   uint16_t first[kMels];
-  uint16_t last[kMels];
+  uint16_t count[kMels];
+  uint16_t start[kMels];
 };
+static_assert(sizeof(MelTable) % 4 == 0 && sizeof(MelTable) < 3800, "passed as a kernel parameter");
 
 uint32_t frames_of(uint32_t length) { return length < kWin ? 0u : 1u + (length - kWin) / kHop; }
 
-// Corner frequencies equally spaced on the HTK mel scale between 0 and rate / 2 (double).
+// Corner frequencies equally spaced on the HTK mel scale between 0 and rate / 2 (double);
+// filter j rises from corner j to corner j + 1 and falls to corner j + 2.
 MelTable make_mel_table() {
   MelTable t;
   std::memset(&t, 0, sizeof(t));
@@ -56,27 +58,21 @@ MelTable make_mel_table() {
     corner[i] = 700.0 * (std::pow(10.0, (top * i / (kMels + 1)) / 2595.0) - 1.0);
   corner[0] = 0.0;
   corner[kMels + 1] = PREBA_AUDIO_RATE / 2.0;
+  uint32_t at = 0;
   for (uint32_t j = 0; j < kMels; ++j) {
-    t.first[j] = 0xffff;
-    t.last[j] = 0;
-  }
-  for (uint32_t k = 0; k < kBins; ++k) {
-    const double f = static_cast<double>(k) * PREBA_AUDIO_RATE / kFft;
-    t.m[k] = 255;
-    if (f >= corner[kMels + 1]) continue;  // the top corner carries no weight
-    uint32_t m = 0;
-    while (m + 1 < kMels + 1 && f >= corner[m + 1]) ++m;
-    t.m[k] = static_cast<uint8_t>(m);
-    t.up[k] = static_cast<float>((f - corner[m]) / (corner[m + 1] - corner[m]));
-    for (int d = 0; d < 2; ++d) {          // filters m (rising) and m - 1 (falling)
-      const int j = static_cast<int>(m) - d;
-      if (j < 0 || j >= static_cast<int>(kMels)) continue;
-      if (t.first[j] == 0xffff) t.first[j] = static_cast<uint16_t>(k);
-      t.last[j] = static_cast<uint16_t>(k + 1);
+    const double lo = corner[j], mid = corner[j + 1], hi = corner[j + 2];
+    t.start[j] = static_cast<uint16_t>(at);
+    bool any = false;
+    for (uint32_t k = 0; k < kBins; ++k) {
+      const double f = static_cast<double>(k) * PREBA_AUDIO_RATE / kFft;
+      if (f <= lo || f >= hi) continue;  // weight 0 at and beyond the feet
+      const double wgt = f < mid ? (f - lo) / (mid - lo) : (hi - f) / (hi - mid);
+      if (!any) t.first[j] = static_cast<uint16_t>(k);
+      any = true;
+      if (at < kMelWeights) t.w[at++] = static_cast<float>(wgt);
+      t.count[j] = static_cast<uint16_t>(k + 1 - t.first[j]);
     }
   }
-  for (uint32_t j = 0; j < kMels; ++j)
-    if (t.first[j] == 0xffff) t.first[j] = t.last[j] = 0;  // a filter without a bin
   return t;
 }
 
@@ -105,7 +101,7 @@ constexpr uint32_t kPitch = 68;
 
 struct __align__(16) WarpFft {
   float2 z[8 * kPitch];  // exchange array, then the spectrum in natural order (first 512)
-  float power[2][kBins + 3];
+  float2 power[kBins + 1];  // the two frames' power spectra side by side
 };
 
 __device__ __forceinline__ float2 cadd(float2 a, float2 b) { return make_float2(a.x + b.x, a.y + b.y); }
@@ -255,16 +251,17 @@ logmel_kernel(const AudioParams p, const MelTable mel_param) {
       const float2 zk = ws.z[k], zn = ws.z[(kFft - k) & (kFft - 1)];
       const float ar = 0.5f * (zk.x + zn.x), ai = 0.5f * (zk.y - zn.y);
       const float br = 0.5f * (zk.y + zn.y), bi = 0.5f * (zn.x - zk.x);
-      ws.power[0][k] = ar * ar + ai * ai;
-      ws.power[1][k] = br * br + bi * bi;
+      ws.power[k] = make_float2(ar * ar + ai * ai, br * br + bi * bi);
     }
     __syncwarp();
     for (uint32_t j = lane; j < kMels; j += 32) {
       float e0 = 0.f, e1 = 0.f;
-      for (uint32_t k = mel.first[j]; k < mel.last[j]; ++k) {
-        const float wgt = mel.m[k] == j ? mel.up[k] : 1.0f - mel.up[k];
-        e0 = fmaf(wgt, ws.power[0][k], e0);
-        e1 = fmaf(wgt, ws.power[1][k], e1);
+      const uint32_t first = mel.first[j], count = mel.count[j], start = mel.start[j];
+      for (uint32_t i = 0; i < count; ++i) {
+        const float wgt = mel.w[start + i];
+        const float2 pw = ws.power[first + i];
+        e0 = fmaf(wgt, pw.x, e0);
+        e1 = fmaf(wgt, pw.y, e1);
       }
       out[static_cast<size_t>(j) * p.t_max + t0] = logf(e0 + kLogGuard);
       if (t0 + 1 < p.t_max)
