@@ -39,6 +39,30 @@ def test_library_exports_every_declared_function():
         assert getattr(handle, name) is not None
 
 
+def test_header_is_plain_c(tmp_path):
+    """include/preba.h promises plain C: it must compile as C11 on its own, and the struct
+    sizes the binding assumes must be the compiler's."""
+    import subprocess
+
+    src = tmp_path / "use_header.c"
+    src.write_text(
+        '#include "preba.h"\n#include <stdio.h>\n'
+        "int main(void) { printf(\"%zu %zu %zu %zu %zu %zu %zu %zu %zu\\n\", sizeof(preba_img_t), "
+        "sizeof(preba_sizes_t), sizeof(preba_batch_t), sizeof(preba_host_batch_t), "
+        "sizeof(preba_image_batch_t), sizeof(preba_options_t), sizeof(preba_utt_t), "
+        "sizeof(preba_audio_sizes_t), sizeof(preba_audio_batch_t)); return 0; }\n")
+    exe = tmp_path / "use_header"
+    subprocess.run(["gcc", "-std=c11", "-Wall", "-Wextra", "-Werror", "-pedantic",
+                    "-I", str(ROOT / "include"), "-o", str(exe), str(src)], check=True)
+    sizes = [int(v) for v in subprocess.run([str(exe)], check=True, capture_output=True,
+                                            text=True).stdout.split()]
+    assert sizes == [ctypes.sizeof(pb.PrebaImg), ctypes.sizeof(pb.PrebaSizes),
+                     ctypes.sizeof(pb.PrebaBatch), ctypes.sizeof(pb.PrebaHostBatch),
+                     ctypes.sizeof(pb.PrebaImageBatch), ctypes.sizeof(pb.PrebaOptions),
+                     pb.UTT_DTYPE.itemsize, ctypes.sizeof(pb.PrebaAudioSizes),
+                     ctypes.sizeof(pb.PrebaAudioBatch)]
+
+
 def test_struct_layouts_match_header():
     assert ctypes.sizeof(pb.PrebaImg) == 16 and pb.TABLE_DTYPE.itemsize == 16
     assert ctypes.sizeof(pb.PrebaSizes) == 32
