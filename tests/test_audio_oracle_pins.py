@@ -5,7 +5,6 @@ function under test."""
 from __future__ import annotations
 
 import numpy as np
-import pytest
 
 from oracle import audio as oa
 

@@ -4,7 +4,6 @@ from exact-rational brute force written from the continuous statement, and from 
 of the base oracle's output (a different source file)."""
 from __future__ import annotations
 
-from fractions import Fraction
 
 import numpy as np
 import pytest
