@@ -375,6 +375,43 @@ int preba_batcher_poll(preba_batcher_t* b, uint64_t now_ns, uint64_t* ids, uint3
                        uint64_t* next_deadline_ns);
 
 /*
+ * Batching front-end for variable-length inputs (paper Sec. 4.3, Fig. "dynamic batching system
+ * for audio processing workloads"): input lengths are bucketised into non-overlapping windows
+ * (2.5 s in the paper), every bucket has a batching queue of its own with its own Batch_max
+ * (the Batch_knee profiled for that length), and no request may wait longer than Time_queue.
+ * A bucket's batch is due when Batch_max of its requests are queued (it takes the oldest
+ * Batch_max) or when its oldest request has waited Time_queue.  In the second case the batch
+ * is short, and the paper fills it from adjacent buckets without exceeding the Batch_max of
+ * the longest input in the batch.  Readings taken here: "adjacent" means the two neighbouring
+ * buckets; the lower one (shorter inputs, which leave the limit unchanged) is drained first,
+ * oldest request first, then the upper one, whose own Batch_max caps the batch once one of
+ * its requests is in; when several buckets are due, full ones go first (lowest bucket first),
+ * then the one whose deadline passed earliest.
+ *
+ * preba_bucket_batcher_create   n_buckets >= 1 queues; bucket i takes lengths in
+ *                               [i*window, (i+1)*window), the last one everything longer;
+ *                               batch_max[i] >= 1; NULL on failure.  `window` and the lengths
+ *                               passed to push share one unit (samples, milliseconds, ...).
+ * preba_bucket_batcher_push     enqueue request `id` of the given length that arrived at
+ *                               `arrival_ns`; arrival times must not decrease.
+ * preba_bucket_batcher_poll     at time `now_ns`: writes the ids of one due batch (the due
+ *                               bucket's requests oldest first, then those merged from the
+ *                               lower and the upper neighbour) and returns their count, or 0;
+ *                               call again until it returns 0.  `capacity` must be >= the
+ *                               largest batch_max.  `next_deadline_ns` as preba_batcher_poll.
+ * Calls on one batcher may come from several threads (one lock per batcher).
+ */
+typedef struct preba_bucket_batcher preba_bucket_batcher_t;
+preba_bucket_batcher_t* preba_bucket_batcher_create(uint32_t n_buckets, uint64_t window,
+                                                    const uint32_t* batch_max,
+                                                    uint64_t time_queue_ns);
+void preba_bucket_batcher_destroy(preba_bucket_batcher_t* b);
+int preba_bucket_batcher_push(preba_bucket_batcher_t* b, uint64_t id, uint64_t arrival_ns,
+                              uint64_t length);
+int preba_bucket_batcher_poll(preba_bucket_batcher_t* b, uint64_t now_ns, uint64_t* ids,
+                              uint32_t capacity, uint64_t* next_deadline_ns);
+
+/*
  * Audio path — the paper's second preprocessing pipeline (Table 1 units "Mel spectrogram" and
  * "Normalize"; Sec. 2.3 item 1: "Fast Fourier Transform (FFT), and applying Mel filters";
  * Sec. 4.2: Normalize as three passes, the mean over all samples, the variance from that mean,

@@ -38,3 +38,62 @@ def batches(arrivals_ns: list[int], batch_max: int, time_queue_ns: int) -> list[
             out.append((limit, waiting))
             waiting = []
     return out
+
+
+def bucket_of(length: int, window: int, n_buckets: int) -> int:
+    """Sec. 4.3: lengths are bucketised into non-overlapping windows; the last bucket is open."""
+    return min(n_buckets - 1, length // window)
+
+
+def bucketed_batches(arrivals_ns: list[int], lengths: list[int], window: int,
+                     batch_max: list[int], time_queue_ns: int) -> list[tuple[int, list[int]]]:
+    """(release time, request indices) of every batch of the bucketised system of Sec. 4.3,
+    when the queues are looked at exactly at every arrival and every waiting-time limit, one
+    batch after the other until none is due.
+
+    A bucket is due when it holds its Batch_max (full buckets first, lowest first; it releases
+    its oldest Batch_max), or when its oldest request has waited Time_queue (earliest limit
+    first).  A bucket released by the time limit is short: it is filled from the lower
+    neighbour, then from the upper neighbour, oldest first, and the batch never exceeds the
+    Batch_max of the longest input's bucket."""
+    n_b = len(batch_max)
+    waiting: list[list[int]] = [[] for _ in range(n_b)]
+    out: list[tuple[int, list[int]]] = []
+
+    def release(now: int) -> bool:
+        for b in range(n_b):
+            if len(waiting[b]) >= batch_max[b]:
+                out.append((now, waiting[b][:batch_max[b]]))
+                del waiting[b][:batch_max[b]]
+                return True
+        due = [(arrivals_ns[waiting[b][0]] + time_queue_ns, b) for b in range(n_b) if waiting[b]]
+        due = [d for d in due if d[0] <= now]
+        if not due:
+            return False
+        _, b = min(due)
+        batch = waiting[b][:]
+        waiting[b].clear()
+        limit = batch_max[b]
+        if b > 0:
+            while len(batch) < limit and waiting[b - 1]:
+                batch.append(waiting[b - 1].pop(0))
+        if b + 1 < n_b:
+            limit = min(limit, batch_max[b + 1])
+            while len(batch) < limit and waiting[b + 1]:
+                batch.append(waiting[b + 1].pop(0))
+        out.append((now, batch))
+        return True
+
+    i, n = 0, len(arrivals_ns)
+    while i < n or any(waiting):
+        limits = [arrivals_ns[w[0]] + time_queue_ns for w in waiting if w]
+        limit = min(limits) if limits else None
+        if i < n and (limit is None or arrivals_ns[i] <= limit):
+            now = arrivals_ns[i]
+            waiting[bucket_of(lengths[i], window, n_b)].append(i)
+            i += 1
+        else:
+            now = limit
+        while release(now):
+            pass
+    return out

@@ -37,6 +37,8 @@ EXPORTS = ("preba_query", "preba_pack", "preba_preprocess", "preba_preprocess_ex
            "preba_last_cuda_error",
            "preba_batching_params", "preba_batcher_create", "preba_batcher_destroy",
            "preba_batcher_push", "preba_batcher_poll",
+           "preba_bucket_batcher_create", "preba_bucket_batcher_destroy",
+           "preba_bucket_batcher_push", "preba_bucket_batcher_poll",
            "preba_audio_query", "preba_audio_pack", "preba_audio_logmel")
 
 
@@ -173,6 +175,17 @@ def lib() -> ctypes.CDLL:
         L.preba_audio_logmel.argtypes = [ctypes.POINTER(PrebaAudioBatch), ctypes.c_int,
                                          ctypes.c_void_p]
         L.preba_audio_logmel.restype = ctypes.c_int
+        L.preba_bucket_batcher_create.argtypes = [ctypes.c_uint32, ctypes.c_uint64, u32p,
+                                                  ctypes.c_uint64]
+        L.preba_bucket_batcher_create.restype = ctypes.c_void_p
+        L.preba_bucket_batcher_destroy.argtypes = [ctypes.c_void_p]
+        L.preba_bucket_batcher_destroy.restype = None
+        L.preba_bucket_batcher_push.argtypes = [ctypes.c_void_p, ctypes.c_uint64, ctypes.c_uint64,
+                                                ctypes.c_uint64]
+        L.preba_bucket_batcher_push.restype = ctypes.c_int
+        L.preba_bucket_batcher_poll.argtypes = [ctypes.c_void_p, ctypes.c_uint64, u64p,
+                                                ctypes.c_uint32, u64p]
+        L.preba_bucket_batcher_poll.restype = ctypes.c_int
         L.preba_strerror.argtypes = [ctypes.c_int]
         L.preba_strerror.restype = ctypes.c_char_p
         L.preba_last_cuda_error.argtypes = []
@@ -632,3 +645,35 @@ class PreparedAudio:
 def preba_audio_logmel(samples, table, n: int, t_max: int, out, normalize: bool = True,
                        stream=None, table_host: np.ndarray | None = None, status=None) -> None:
     PreparedAudio(samples, table, n, t_max, out, normalize, stream, table_host, status)()
+
+
+class BucketBatcher:
+    """The batching front-end for variable-length inputs (``preba_bucket_batcher_*``)."""
+
+    def __init__(self, window: int, batch_max, time_queue_ns: int):
+        bm = _u32(batch_max)
+        self._h = lib().preba_bucket_batcher_create(len(bm), window, _p(bm, ctypes.c_uint32),
+                                                    time_queue_ns)
+        if not self._h:
+            raise PrebaError(ERR_INVALID_ARG, "preba_bucket_batcher_create")
+        self._cap = int(bm.max())
+        self._ids = (ctypes.c_uint64 * self._cap)()
+
+    def push(self, request_id: int, arrival_ns: int, length: int) -> None:
+        rc = lib().preba_bucket_batcher_push(self._h, request_id, arrival_ns, length)
+        if rc != OK:
+            raise PrebaError(rc, "preba_bucket_batcher_push")
+
+    def poll(self, now_ns: int) -> tuple[list[int], int]:
+        """(ids of one due batch or [], time at which the oldest waiting request runs out)."""
+        nxt = ctypes.c_uint64()
+        rc = lib().preba_bucket_batcher_poll(self._h, now_ns, self._ids, self._cap,
+                                             ctypes.byref(nxt))
+        if rc < 0:
+            raise PrebaError(rc, "preba_bucket_batcher_poll")
+        return [int(self._ids[i]) for i in range(rc)], int(nxt.value)
+
+    def __del__(self):
+        if getattr(self, "_h", None):
+            lib().preba_bucket_batcher_destroy(self._h)
+            self._h = None
