@@ -105,8 +105,9 @@ struct TaskMeta {
   // rounded modes: the value of an output pixel is num / dd with dd = den_x * den_y
   uint32_t deny2;         // 2 * den_y
   uint32_t dd;            // den_x * den_y
-  uint32_t magic;         // floor(2^32 / (2 * dd))
-  uint32_t pad[2];
+  uint32_t magic;         // reciprocal of 2 * dd (see Quant)
+  uint32_t shift;         // k - 1 when the reciprocal is exact, else kNoShift
+  uint32_t pad;
   uint64_t src;           // byte offset of the image in the pixel buffer
   uint32_t info[kMaxList];  // per listed row: low byte = byte skew of the staged row,
                             // next byte = output rows completed by this row
@@ -373,16 +374,22 @@ __device__ __forceinline__ void emit_row(OutT* __restrict__ q, uint32_t plane, u
 // The rounded modes keep den_x times the horizontally interpolated value as a whole number
 // (bit pattern of an unsigned integer in the row buffers).  An output pixel is
 // floor(num / dd + 1/2) = floor(t / (2 dd)) with t = 2 num + dd, num = prev * (den_y - rem)
-// + cur * rem.  The quotient (at most 255) comes from a multiply-high by floor(2^32 / (2 dd)):
+// + cur * rem.  The quotient (at most 255) comes from a multiply-high by a reciprocal.
+// EXACT (2 dd < 2^22): with 2^k <= 2 dd < 2^(k+1) and magic = ceil(2^(31+k) / (2 dd)),
+// floor(t * magic / 2^(31+k)) is the quotient for every t <= 511 dd, because the excess
+// t * (magic * 2 dd - 2^(31+k)) stays below 2^(31+k).  Otherwise magic = floor(2^32 / (2 dd)):
 // t < 2^32 makes that estimate exact or one short, and the remainder corrects it.
+constexpr uint32_t kNoShift = 0xffffffffu;  // Quant::shift when the division needs its correction
 struct Quant {
-  uint32_t deny2, dd, d2, magic;
+  uint32_t deny2, dd, d2, magic, shift;
 };
 
+template <bool EXACT>
 __device__ __forceinline__ uint32_t rounded_pixel(float prev, float cur, uint32_t w0, uint32_t w1,
                                                   const Quant& qz) {
   // < 2^32 by the fast path's precondition
   const uint32_t t = __float_as_uint(prev) * w0 + (__float_as_uint(cur) * w1 + qz.dd);
+  if (EXACT) return __umulhi(t, qz.magic) >> qz.shift;
   uint32_t q = __umulhi(t, qz.magic);
   if (t - q * qz.d2 >= qz.d2) ++q;
   return q;
@@ -393,7 +400,7 @@ __device__ __forceinline__ uint32_t rounded_pixel(float prev, float cur, uint32_
 // 2 * lane of plane 0, as in emit_row.  kU8: q points at the first byte of pixel 2 * lane of
 // the output row (HWC); a lane writes its pairs as three 16-bit words each and its single
 // column byte by byte.
-template <typename OutT, bool FULL, int MODE>
+template <typename OutT, bool FULL, int MODE, bool EXACT>
 __device__ __forceinline__ void emit_row_rounded(OutT* __restrict__ q, uint32_t plane,
                                                  uint32_t lane, uint32_t rem,
                                                  const float (&hp)[kLaneCols][3],
@@ -408,8 +415,8 @@ __device__ __forceinline__ void emit_row_rounded(OutT* __restrict__ q, uint32_t 
       uint32_t l[3], r[3];
 #pragma unroll
       for (int ch = 0; ch < 3; ++ch) {
-        l[ch] = rounded_pixel(hp[2 * pr][ch], hc[2 * pr][ch], w0, w1, qz);
-        r[ch] = rounded_pixel(hp[2 * pr + 1][ch], hc[2 * pr + 1][ch], w0, w1, qz);
+        l[ch] = rounded_pixel<EXACT>(hp[2 * pr][ch], hc[2 * pr][ch], w0, w1, qz);
+        r[ch] = rounded_pixel<EXACT>(hp[2 * pr + 1][ch], hc[2 * pr + 1][ch], w0, w1, qz);
       }
       uint8_t* at = b + 192 * pr;  // 64 pixels further
       if (FULL) {
@@ -429,7 +436,7 @@ __device__ __forceinline__ void emit_row_rounded(OutT* __restrict__ q, uint32_t 
     if (FULL || ((valid >> 6) & 1u)) {
 #pragma unroll
       for (int ch = 0; ch < 3; ++ch)
-        single[ch] = static_cast<uint8_t>(rounded_pixel(hp[6][ch], hc[6][ch], w0, w1, qz));
+        single[ch] = static_cast<uint8_t>(rounded_pixel<EXACT>(hp[6][ch], hc[6][ch], w0, w1, qz));
     }
   } else {
 #pragma unroll
@@ -437,7 +444,7 @@ __device__ __forceinline__ void emit_row_rounded(OutT* __restrict__ q, uint32_t 
       float o[kLaneCols];
 #pragma unroll
       for (int m = 0; m < static_cast<int>(kLaneCols); ++m) {
-        const uint32_t px = rounded_pixel(hp[m][ch], hc[m][ch], w0, w1, qz);
+        const uint32_t px = rounded_pixel<EXACT>(hp[m][ch], hc[m][ch], w0, w1, qz);
         o[m] = fmaf(__uint_as_float(0x4B000000u | px) - 8388608.0f, na[ch], nb[ch]);
       }
       OutT* single = q + 192 - lane;
@@ -600,7 +607,15 @@ __device__ __forceinline__ uint32_t prepare(const Params& p, uint32_t task, Task
       if (lane == 0 && kind == kStream) {
         m.deny2 = 2 * ay.den;
         m.dd = static_cast<uint32_t>(dd);
-        m.magic = static_cast<uint32_t>((1ull << 32) / (2 * dd));  // 2 dd >= 8
+        const uint64_t d2 = 2 * dd;  // >= 8
+        if (d2 < (1ull << 22)) {
+          const uint32_t k = 31 - static_cast<uint32_t>(__clz(static_cast<uint32_t>(d2)));
+          m.magic = static_cast<uint32_t>(((1ull << (31 + k)) + d2 - 1) / d2);
+          m.shift = k - 1;
+        } else {
+          m.magic = static_cast<uint32_t>((1ull << 32) / d2);
+          m.shift = kNoShift;
+        }
       }
     }
     if (lane == 0) {
@@ -682,8 +697,12 @@ __device__ __forceinline__ void emit_any(OutT* __restrict__ q, uint32_t plane, u
                                          const float (&nb)[3], const Quant& qz, uint32_t valid) {
   if constexpr (MODE == kFloat)
     emit_row<OutT, FULL>(q, plane, lane, __uint_as_float(weight_bits), prev, cur, sa, nb, valid);
+  else if (qz.shift != kNoShift)
+    emit_row_rounded<OutT, FULL, MODE, true>(q, plane, lane, weight_bits, prev, cur, qz, sa, nb,
+                                             valid);
   else
-    emit_row_rounded<OutT, FULL, MODE>(q, plane, lane, weight_bits, prev, cur, qz, sa, nb, valid);
+    emit_row_rounded<OutT, FULL, MODE, false>(q, plane, lane, weight_bits, prev, cur, qz, sa, nb,
+                                              valid);
 }
 
 // ---- the warp program ---------------------------------------------------------------------------------
@@ -696,7 +715,7 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
   const uint32_t row_step = MODE == kU8 ? 3 * C : C;  // elements of OutT between output rows
   const float nb[3] = {p.b[0], p.b[1], p.b[2]};
   float sa[3] = {0.f, 0.f, 0.f};  // staged path: 1 / (255 * std * den) of the task's image
-  Quant qz = {0, 0, 0, 0};     // rounded modes: the task's division constants
+  Quant qz = {0, 0, 0, 0, 0};     // rounded modes: the task's division constants
 
   // task claims: a warp's first task is its own index; later ones come from the shared
   // counter (dynamic) or every nwarps-th task (static)
@@ -819,6 +838,7 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
           qz.dd = cm->dd;
           qz.d2 = 2 * qz.dd;
           qz.magic = cm->magic;
+          qz.shift = cm->shift;
 #pragma unroll
           for (int ch = 0; ch < 3; ++ch) sa[ch] = p.a[ch];
         }

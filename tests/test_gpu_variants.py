@@ -84,7 +84,8 @@ def test_uint8_output_is_bit_exact_on_a_ragged_batch(dynamic):
         assert np.array_equal(got, want_u8(imgs, 224, 256, origins))
 
 
-@pytest.mark.parametrize("c,s", [(1, 1), (7, 7), (9, 17), (33, 40), (224, 224), (225, 300), (449, 460)])
+@pytest.mark.parametrize("c,s", [(1, 1), (7, 7), (9, 17), (33, 40), (224, 224), (225, 300), (449, 460),
+                                 (40, 800), (230, 1000)])  # the last two: division with correction
 def test_uint8_output_other_sizes_and_partial_column_blocks(c, s):
     imgs = [uniform(50, 37, 53), uniform(51, 64, 48), uniform(52, 5, 9), uniform(53, 300, 200)]
     origins = origins_for(imgs, c, s, 2)
