@@ -36,8 +36,8 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM bytes (read + write) per launch of the kernel on the default workload, from one
 # ncu capture, valid only for the kernel sources with this digest (else reported as null).
-NCU_TRAFFIC = {"csrc_sha1": "37c7b2e9c510aed115ba4ab74b79e31ad72bb040",
-               "bytes_per_launch": 75636224 + 25414912}  # dram read + write, one launch
+NCU_TRAFFIC = {"csrc_sha1": "92be46a6cb22008f113ffa424f83203f814aa897",
+               "bytes_per_launch": 75637248 + 25767936}  # dram read + write, one launch
 
 
 def csrc_digest() -> str:
