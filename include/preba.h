@@ -415,7 +415,8 @@ int preba_bucket_batcher_poll(preba_bucket_batcher_t* b, uint64_t now_ns, uint64
  * Audio path — the paper's second preprocessing pipeline (Table 1 units "Mel spectrogram" and
  * "Normalize"; Sec. 2.3 item 1: "Fast Fourier Transform (FFT), and applying Mel filters";
  * Sec. 4.2: Normalize as three passes, the mean over all samples, the variance from that mean,
- * then the normalisation).  "Resample" is not built: samples arrive at 16 kHz.  The paper
+ * then the normalisation).  Samples are taken at 16 kHz; preba_audio_resample (below) brings
+ * other rates there.  The paper
  * fixes no numerics; the readings are: frames of 400 samples every 160 (no padding, so
  * T = 1 + (L - 400)/160 frames for L >= 400, else 0), periodic Hann window, zero-padding to a
  * 512-point DFT, power spectrum, 80 unit-height triangular filters equally spaced on the HTK
@@ -480,6 +481,41 @@ int preba_audio_pack(const float* const* utterances, const uint32_t* lengths, ui
  * skipped and reported by the kernel otherwise.
  * Errors: PREBA_ERR_INVALID_ARG, PREBA_ERR_BUFFER_TOO_SMALL, PREBA_ERR_BAD_TABLE, PREBA_ERR_CUDA. */
 int preba_audio_logmel(const preba_audio_batch_t* batch, int normalize, void* stream);
+
+/*
+ * Resample — the first audio unit of Table 1 ("resampling", Sec. 2.3 item 1), for utterances
+ * that do not arrive at the model's rate.  The paper only names it; the reading is the
+ * classical bandlimited interpolation with a Hann-windowed sinc, six zero crossings each
+ * side, cutoff at 0.99 of the lower Nyquist frequency:
+ *   y[m] = sum_n x[n] * h(n - m*rate_in/rate_out),  h(t) = fc*sinc(fc*t)*cos^2(pi*fc*t/12)
+ *   for |fc*t| < 6 (else 0),  fc = 0.99*min(1, rate_out/rate_in),
+ * M = ceil(L*rate_out/rate_in) outputs per utterance, samples outside the utterance taken
+ * as 0; fp32 on the device.
+ *
+ * preba_audio_layout          the table {offset, length, frames} of a packed buffer for the
+ *                             given lengths (offsets as preba_audio_pack lays them out), without
+ *                             copying samples.
+ * preba_audio_resample_query  the output length of every utterance (HOST arithmetic).
+ * preba_audio_resample        enqueues one kernel on `stream`: every utterance of the packed
+ *                             input (DEVICE `samples_in`, `table_in`) is resampled into its
+ *                             place in the packed output (DEVICE `samples_out`, `table_out`,
+ *                             whose lengths must be those of the query; alignment padding is
+ *                             written as 0).  `longest_out` is the largest output length.
+ *                             Rate pairs whose phase table (rate_out/gcd phases of about
+ *                             12*rate_in/rate_out + 4 taps) exceeds 12000 entries are refused.
+ *                             A table entry that is misaligned, runs past its buffer or whose
+ *                             output length does not follow from its input length is skipped
+ *                             and PREBA_ERR_BAD_TABLE stored in `status`.
+ * Errors: PREBA_ERR_INVALID_ARG, PREBA_ERR_CUDA.
+ */
+int preba_audio_layout(const uint32_t* lengths, uint32_t n, preba_utt_t* table);
+int preba_audio_resample_query(const uint32_t* lengths_in, uint32_t n, uint32_t rate_in,
+                               uint32_t rate_out, uint32_t* lengths_out);
+int preba_audio_resample(const float* samples_in, uint64_t samples_in_count,
+                         const preba_utt_t* table_in, float* samples_out,
+                         uint64_t samples_out_count, const preba_utt_t* table_out, uint32_t n,
+                         uint32_t longest_out, uint32_t rate_in, uint32_t rate_out,
+                         int32_t* status, void* stream);
 
 /* Text for a PREBA_* code (static storage, never NULL). */
 const char* preba_strerror(int code);

@@ -39,7 +39,8 @@ EXPORTS = ("preba_query", "preba_pack", "preba_preprocess", "preba_preprocess_ex
            "preba_batcher_push", "preba_batcher_poll",
            "preba_bucket_batcher_create", "preba_bucket_batcher_destroy",
            "preba_bucket_batcher_push", "preba_bucket_batcher_poll",
-           "preba_audio_query", "preba_audio_pack", "preba_audio_logmel")
+           "preba_audio_query", "preba_audio_pack", "preba_audio_logmel",
+           "preba_audio_layout", "preba_audio_resample_query", "preba_audio_resample")
 
 
 class PrebaImg(ctypes.Structure):
@@ -186,6 +187,16 @@ def lib() -> ctypes.CDLL:
         L.preba_bucket_batcher_poll.argtypes = [ctypes.c_void_p, ctypes.c_uint64, u64p,
                                                 ctypes.c_uint32, u64p]
         L.preba_bucket_batcher_poll.restype = ctypes.c_int
+        L.preba_audio_layout.argtypes = [u32p, ctypes.c_uint32, ctypes.c_void_p]
+        L.preba_audio_layout.restype = ctypes.c_int
+        L.preba_audio_resample_query.argtypes = [u32p, ctypes.c_uint32, ctypes.c_uint32,
+                                                 ctypes.c_uint32, u32p]
+        L.preba_audio_resample_query.restype = ctypes.c_int
+        L.preba_audio_resample.argtypes = [ctypes.c_void_p, ctypes.c_uint64, ctypes.c_void_p,
+                                           ctypes.c_void_p, ctypes.c_uint64, ctypes.c_void_p,
+                                           ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32,
+                                           ctypes.c_uint32, ctypes.c_void_p, ctypes.c_void_p]
+        L.preba_audio_resample.restype = ctypes.c_int
         L.preba_strerror.argtypes = [ctypes.c_int]
         L.preba_strerror.restype = ctypes.c_char_p
         L.preba_last_cuda_error.argtypes = []
@@ -677,3 +688,41 @@ class BucketBatcher:
         if getattr(self, "_h", None):
             lib().preba_bucket_batcher_destroy(self._h)
             self._h = None
+
+
+def preba_audio_layout(lengths) -> np.ndarray:
+    """The {offset, length, frames} table of a packed sample buffer for the given lengths."""
+    ln = _u32(lengths)
+    table = np.zeros(len(ln), dtype=UTT_DTYPE)
+    rc = lib().preba_audio_layout(_p(ln, ctypes.c_uint32), len(ln), table.ctypes.data)
+    if rc != OK:
+        raise PrebaError(rc, "preba_audio_layout")
+    return table
+
+
+def preba_audio_resample_query(lengths_in, rate_in: int, rate_out: int) -> np.ndarray:
+    ln = _u32(lengths_in)
+    out = np.zeros(len(ln), dtype=np.uint32)
+    rc = lib().preba_audio_resample_query(_p(ln, ctypes.c_uint32), len(ln), rate_in, rate_out,
+                                          _p(out, ctypes.c_uint32))
+    if rc != OK:
+        raise PrebaError(rc, "preba_audio_resample_query")
+    return out
+
+
+def preba_audio_resample(samples_in, table_in, samples_out, table_out, n: int, longest_out: int,
+                         rate_in: int, rate_out: int, status=None, stream=None) -> None:
+    """``samples_*`` and ``table_*`` are CUDA tensors (packed float32 samples, tables as bytes)."""
+    import torch
+
+    if stream is None:
+        stream = torch.cuda.current_stream().cuda_stream
+    elif hasattr(stream, "cuda_stream"):
+        stream = stream.cuda_stream
+    rc = lib().preba_audio_resample(samples_in.data_ptr(), samples_in.numel(), table_in.data_ptr(),
+                                    samples_out.data_ptr(), samples_out.numel(),
+                                    table_out.data_ptr(), n, longest_out, rate_in, rate_out,
+                                    status.data_ptr() if status is not None else None,
+                                    ctypes.c_void_p(stream))
+    if rc != OK:
+        raise PrebaError(rc, "preba_audio_resample")

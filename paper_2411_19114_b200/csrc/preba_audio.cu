@@ -343,6 +343,162 @@ extern "C" int preba_audio_pack(const float* const* utterances, const uint32_t* 
   return PREBA_OK;
 }
 
+namespace preba {
+namespace audio {
+
+// ---- Resample: bandlimited interpolation with a Hann-windowed sinc ---------------------------------
+constexpr uint32_t kResampleZeros = 6;
+constexpr float kResampleRolloff = 0.99f;
+constexpr uint32_t kResampleChunk = 4096;        // output samples per CTA
+constexpr uint32_t kResampleTableMax = 12000;    // floats of shared memory for the phase table
+
+struct ResampleParams {
+  const float* in;
+  uint64_t in_count;
+  const preba_utt_t* table_in;
+  float* out;
+  uint64_t out_count;
+  const preba_utt_t* table_out;
+  int32_t* status;
+  uint32_t n;
+  uint32_t orig, fresh;  // the two rates divided by their greatest common divisor
+  uint32_t reach;        // taps reach from centre - reach to centre + reach + 1
+  float fc;              // cutoff relative to the input rate
+};
+
+// Output sample m of an utterance sits at position m * orig / fresh of the input; with
+// centre = floor of that and phase p = (m * orig) mod fresh, its value is
+// sum_j x[centre - reach + j] * h((j - reach) - p / fresh).  A CTA tabulates h for every
+// phase once and then produces a run of outputs.
+__global__ void __launch_bounds__(256) resample_kernel(const ResampleParams p) {
+  __shared__ float table[kResampleTableMax];
+  const uint32_t taps = 2 * p.reach + 2;
+  const preba_utt_t ui = p.table_in[blockIdx.y], uo = p.table_out[blockIdx.y];
+  const uint64_t want = (static_cast<uint64_t>(ui.length) * p.fresh + p.orig - 1) / p.orig;
+  const bool ok = ui.offset % PREBA_AUDIO_ALIGN == 0 && uo.offset % PREBA_AUDIO_ALIGN == 0 &&
+                  ui.offset <= p.in_count && ui.length <= p.in_count - ui.offset &&
+                  uo.length == want && uo.offset <= p.out_count &&
+                  (static_cast<uint64_t>(uo.length) + 3) / 4 * 4 <= p.out_count - uo.offset;
+  if (!ok) {
+    if (threadIdx.x == 0 && blockIdx.x == 0 && p.status)
+      atomicCAS(p.status, 0, PREBA_ERR_BAD_TABLE);
+    return;
+  }
+  const uint32_t m0 = blockIdx.x * kResampleChunk;
+  const uint32_t padded = (uo.length + 3) / 4 * 4;  // alignment padding is written as 0
+  if (m0 >= padded) return;
+  for (uint32_t i = threadIdx.x; i < p.fresh * taps; i += blockDim.x) {
+    const uint32_t phase = i / taps, j = i - phase * taps;
+    const float t = (static_cast<float>(j) - static_cast<float>(p.reach)) -
+                    static_cast<float>(phase) / static_cast<float>(p.fresh);
+    const float u = p.fc * t;
+    float h = 0.f;
+    if (fabsf(u) < static_cast<float>(kResampleZeros)) {
+      const float sinc = u == 0.f ? 1.0f : sinpif(u) / (3.14159265358979323846f * u);
+      const float c = cospif(u / (2.0f * kResampleZeros));
+      h = p.fc * sinc * c * c;
+    }
+    table[i] = h;
+  }
+  __syncthreads();
+  const float* __restrict__ x = p.in + ui.offset;
+  float* __restrict__ y = p.out + uo.offset;
+  const uint32_t m_end = min(m0 + kResampleChunk, padded);
+  for (uint32_t m = m0 + threadIdx.x; m < m_end; m += blockDim.x) {
+    float acc = 0.f;
+    if (m < uo.length) {
+      const uint64_t pos = static_cast<uint64_t>(m) * p.orig;
+      const int64_t first = static_cast<int64_t>(pos / p.fresh) - p.reach;
+      const float* __restrict__ h = table + (pos % p.fresh) * taps;
+      for (uint32_t j = 0; j < taps; ++j) {
+        const int64_t idx = first + j;
+        if (idx >= 0 && idx < static_cast<int64_t>(ui.length)) acc = fmaf(x[idx], h[j], acc);
+      }
+    }
+    y[m] = acc;
+  }
+}
+
+uint32_t gcd32(uint32_t a, uint32_t b) {
+  while (b) {
+    const uint32_t r = a % b;
+    a = b;
+    b = r;
+  }
+  return a;
+}
+
+}  // namespace audio
+}  // namespace preba
+
+extern "C" int preba_audio_layout(const uint32_t* lengths, uint32_t n, preba_utt_t* table) {
+  if (!lengths || !table || n == 0) return PREBA_ERR_INVALID_ARG;
+  uint64_t at = 0;
+  for (uint32_t i = 0; i < n; ++i) {
+    if (lengths[i] > PREBA_AUDIO_MAX_SAMPLES) return PREBA_ERR_INVALID_ARG;
+    table[i].offset = at;
+    table[i].length = lengths[i];
+    table[i].frames = preba::audio::frames_of(lengths[i]);
+    at = preba::align_up(at + lengths[i], PREBA_AUDIO_ALIGN);
+  }
+  return PREBA_OK;
+}
+
+extern "C" int preba_audio_resample_query(const uint32_t* lengths_in, uint32_t n, uint32_t rate_in,
+                                          uint32_t rate_out, uint32_t* lengths_out) {
+  if (!lengths_in || !lengths_out || n == 0 || rate_in == 0 || rate_out == 0)
+    return PREBA_ERR_INVALID_ARG;
+  const uint32_t g = preba::audio::gcd32(rate_in, rate_out);
+  const uint64_t orig = rate_in / g, fresh = rate_out / g;
+  for (uint32_t i = 0; i < n; ++i) {
+    const uint64_t m = (lengths_in[i] * fresh + orig - 1) / orig;
+    if (lengths_in[i] > PREBA_AUDIO_MAX_SAMPLES || m > PREBA_AUDIO_MAX_SAMPLES)
+      return PREBA_ERR_INVALID_ARG;
+    lengths_out[i] = static_cast<uint32_t>(m);
+  }
+  return PREBA_OK;
+}
+
+extern "C" int preba_audio_resample(const float* samples_in, uint64_t samples_in_count,
+                                    const preba_utt_t* table_in, float* samples_out,
+                                    uint64_t samples_out_count, const preba_utt_t* table_out,
+                                    uint32_t n, uint32_t longest_out, uint32_t rate_in,
+                                    uint32_t rate_out, int32_t* status, void* stream) {
+  using namespace preba::audio;
+  if (!samples_in || !table_in || !samples_out || !table_out || n == 0 || n > 65535 ||
+      rate_in == 0 || rate_out == 0 || longest_out > PREBA_AUDIO_MAX_SAMPLES)
+    return PREBA_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(samples_in) % 16 || reinterpret_cast<uintptr_t>(samples_out) % 16)
+    return PREBA_ERR_INVALID_ARG;
+  ResampleParams p;
+  const uint32_t g = gcd32(rate_in, rate_out);
+  p.orig = rate_in / g;
+  p.fresh = rate_out / g;
+  const double fc = static_cast<double>(kResampleRolloff) *
+                    (p.fresh < p.orig ? static_cast<double>(p.fresh) / p.orig : 1.0);
+  p.fc = static_cast<float>(fc);
+  p.reach = static_cast<uint32_t>(std::ceil(kResampleZeros / fc)) + 1;
+  if (static_cast<uint64_t>(p.fresh) * (2 * p.reach + 2) > kResampleTableMax)
+    return PREBA_ERR_INVALID_ARG;  // the phase table of this rate pair does not fit
+  p.in = samples_in;
+  p.in_count = samples_in_count;
+  p.table_in = table_in;
+  p.out = samples_out;
+  p.out_count = samples_out_count;
+  p.table_out = table_out;
+  p.status = status;
+  p.n = n;
+  if (longest_out == 0) return PREBA_OK;
+  const dim3 grid((longest_out + 3 + kResampleChunk - 1) / kResampleChunk, n);
+  resample_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(p);
+  const cudaError_t err = cudaGetLastError();
+  if (err != cudaSuccess) {
+    preba::g_last_cuda_error = static_cast<int>(err);
+    return PREBA_ERR_CUDA;
+  }
+  return PREBA_OK;
+}
+
 extern "C" int preba_audio_logmel(const preba_audio_batch_t* b, int normalize, void* stream) {
   using namespace preba::audio;
   if (!b || !b->samples || !b->table || !b->out || b->n == 0 || b->n > 65535 || b->t_max == 0)

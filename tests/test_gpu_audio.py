@@ -151,3 +151,98 @@ def test_device_side_table_check_skips_bad_entries():
     want = oa.preprocess(utts)
     for i in (0, 2):
         assert float(np.max(np.abs(host[i] - want[i, :, :t_max]))) <= NORM_TOL
+
+
+# ---- Resample ------------------------------------------------------------------------------------------
+
+RESAMPLE_TOL = 2e-5   # fp32 taps and sums of <= 80 products of magnitude <= 1 against float64
+
+
+def test_resample_sizes_and_layout():
+    out = pb.preba_audio_resample_query([48000, 44101, 0, 7], 44100, 16000)
+    assert out.tolist() == [oa.resampled_length(v, 44100, 16000) for v in (48000, 44101, 0, 7)]
+    t = pb.preba_audio_layout([401, 0, 399, 1601])
+    assert [int(e["offset"]) for e in t] == [0, 404, 404, 804]
+    assert [int(e["frames"]) for e in t] == [1, 0, 0, 8]
+    L = pb.lib()
+    one = np.zeros(1, dtype=np.uint32)
+    assert L.preba_audio_resample_query(one.ctypes.data_as(ctypes.POINTER(ctypes.c_uint32)), 1, 0, 16000,
+                                        one.ctypes.data_as(ctypes.POINTER(ctypes.c_uint32))) \
+        == pb.ERR_INVALID_ARG
+    # rate pairs whose phase table is too large are refused before any launch
+    assert L.preba_audio_resample(0x1000, 16, 0x2000, 0x3000, 16, 0x4000, 1, 8, 15999, 16000, None,
+                                  None) == pb.ERR_INVALID_ARG
+    assert L.preba_audio_resample(None, 16, 0x2000, 0x3000, 16, 0x4000, 1, 8, 48000, 16000, None,
+                                  None) == pb.ERR_INVALID_ARG
+
+
+def run_resample(utts, rate_in, rate_out=16000):
+    import torch
+
+    n = len(utts)
+    packed, table_in = pb.preba_audio_pack(utts)
+    lens_out = pb.preba_audio_resample_query([u.size for u in utts], rate_in, rate_out)
+    table_out = pb.preba_audio_layout(lens_out)
+    total_out = int(pb.preba_audio_query(lens_out).packed_samples)
+    dev = torch.device("cuda:0")
+    guard = 256
+    buf = torch.full((guard + max(4, total_out) + guard,), 777.0, dtype=torch.float32, device=dev)
+    out = buf[guard:guard + max(4, total_out)]
+    smp = torch.from_numpy(packed).to(dev) if packed.size else torch.zeros(4, device=dev)
+    tin = torch.from_numpy(table_in.view(np.uint8)).to(dev)
+    tout = torch.from_numpy(table_out.view(np.uint8)).to(dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    pb.preba_audio_resample(smp, tin, out, tout, n, int(lens_out.max()), rate_in, rate_out,
+                            status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    host = buf.cpu().numpy()
+    assert np.all(host[:guard] == 777.0) and np.all(host[guard + max(4, total_out):] == 777.0)
+    res = host[guard:guard + total_out]
+    got = []
+    for e in table_out:
+        o, ln = int(e["offset"]), int(e["length"])
+        got.append(res[o:o + ln].copy())
+        assert np.all(res[o + ln:-(-(o + ln) // 4) * 4] == 0.0)       # alignment padding is zero
+    return got, table_out
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("rate_in", [48000, 44100, 22050, 8000, 16000, 11025])
+def test_resample_matches_the_oracle(rate_in):
+    rng = np.random.default_rng(rate_in)
+    # the samples' meaning does not matter to the interpolator: speech-like signals generated
+    # at 16 kHz are simply taken as rate_in material; one empty utterance
+    utts = [wl.utterance(rng, s) for s in (0.31, 0.05, 0.2)] + [np.zeros(0, dtype=np.float32)]
+    utts.append(rng.uniform(-1, 1, size=977).astype(np.float32))   # white noise: all frequencies
+    utts.append(np.ones(5, dtype=np.float32))                       # shorter than the filter
+    got, _ = run_resample(utts, rate_in)
+    for u, g in zip(utts, got):
+        want = oa.resample(u, rate_in, 16000)
+        assert g.shape == want.shape
+        if want.size:
+            assert float(np.max(np.abs(g - want))) <= RESAMPLE_TOL
+
+
+@pytest.mark.gpu
+def test_resample_then_log_mel_end_to_end():
+    """48 kHz utterances through Resample, Mel spectrogram and Normalize on the device against
+    the same chain of the oracle."""
+    import torch
+
+    rng = np.random.default_rng(9)
+    utts = [rng.normal(0, 0.2, size=n).clip(-1, 1).astype(np.float32) for n in (48000 // 2, 30011, 1500)]
+    got16, table16 = run_resample(utts, 48000)
+    dev = torch.device("cuda:0")
+    # feed the resampled batch straight into the spectrogram path (packed as the kernel wrote it)
+    packed16, _ = pb.preba_audio_pack(got16)
+    t_max = max(1, int(table16["frames"].max()))
+    feat = torch.empty((3, 80, t_max), dtype=torch.float32, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    pb.preba_audio_logmel(torch.from_numpy(packed16).to(dev),
+                          torch.from_numpy(table16.view(np.uint8)).to(dev), 3, t_max, feat, True,
+                          table_host=table16, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    want = oa.preprocess([oa.resample(u, 48000, 16000) for u in utts])
+    assert float(np.max(np.abs(feat.cpu().numpy().astype(np.float64) - want[:, :, :t_max]))) <= NORM_TOL
