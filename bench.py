@@ -353,6 +353,32 @@ def run_audio(args, local_rank: int) -> None:
         want = oa.preprocess([utts[i]])[0]
         err = float(np.max(np.abs(got[i, :, :want.shape[1]] - want)))
         assert err <= 2e-3, f"audio result differs from the oracle: {err:.3e}"
+    # the Resample unit on the same samples taken as 48 kHz material (48 kHz -> 16 kHz)
+    lens48 = pb.preba_audio_resample_query(table["length"], 48000, 16000)
+    table48 = pb.preba_audio_layout(lens48)
+    out48 = torch.empty(int(pb.preba_audio_query(lens48).packed_samples), dtype=torch.float32,
+                        device=dev)
+    tab48 = torch.from_numpy(table48.view(np.uint8)).to(dev)
+    for _ in range(3):
+        pb.preba_audio_resample(smp[0], tab, out48, tab48, n, int(lens48.max()), 48000, 16000,
+                                status=status)
+    torch.cuda.synchronize()
+    r_start, r_stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    r_steps = 200
+    r_start.record(stream)
+    for i in range(r_steps):
+        pb.preba_audio_resample(smp[i % sets], tab, out48, tab48, n, int(lens48.max()), 48000,
+                                16000, status=status)
+    r_stop.record(stream)
+    torch.cuda.synchronize()
+    resample_us = r_start.elapsed_time(r_stop) / r_steps * 1e3
+    assert int(status.item()) == 0
+    got48 = out48.cpu().numpy()
+    k48 = int(np.argmin(table["length"]))
+    want48 = oa.resample(utts[k48], 48000, 16000)
+    o48 = int(table48["offset"][k48])
+    err48 = float(np.max(np.abs(got48[o48:o48 + want48.size] - want48)))
+    assert err48 <= 2e-5, f"resampled audio differs from the oracle: {err48:.3e}"
     # end to end: pinned samples -> device, two kernels, result -> pinned memory
     e2e_steps = max(3, min(args.e2e_steps, steps))
     ph = torch.from_numpy(packed).pin_memory()
@@ -420,6 +446,12 @@ def run_audio(args, local_rank: int) -> None:
                 "includes": "packed samples pinned -> device, both kernels, result -> pinned "
                             "memory; two buffer sets on two streams"},
         "audio_seconds_per_second": seconds / per_launch_s,
+        "resample_48k_to_16k": {"us_per_launch": resample_us,
+                                "input_samples_per_s": float(table["length"].sum()) /
+                                                       (resample_us * 1e-6),
+                                "note": "the same packed samples taken as 48 kHz material, one "
+                                        "kernel per batch; checked against the oracle on the "
+                                        "shortest utterance"},
         "gpu_launches": 2 * steps, "clocks": clocks.summary(),
     }
     print(json.dumps(line), flush=True)

@@ -349,7 +349,7 @@ namespace audio {
 // ---- Resample: bandlimited interpolation with a Hann-windowed sinc ---------------------------------
 constexpr uint32_t kResampleZeros = 6;
 constexpr float kResampleRolloff = 0.99f;
-constexpr uint32_t kResampleChunk = 4096;        // output samples per CTA
+constexpr uint32_t kResampleChunk = 2048;        // output samples per CTA
 constexpr uint32_t kResampleTableMax = 12000;    // floats of shared memory for the phase table
 
 struct ResampleParams {
@@ -408,11 +408,19 @@ __global__ void __launch_bounds__(256) resample_kernel(const ResampleParams p) {
     float acc = 0.f;
     if (m < uo.length) {
       const uint64_t pos = static_cast<uint64_t>(m) * p.orig;
-      const int64_t first = static_cast<int64_t>(pos / p.fresh) - p.reach;
-      const float* __restrict__ h = table + (pos % p.fresh) * taps;
-      for (uint32_t j = 0; j < taps; ++j) {
-        const int64_t idx = first + j;
-        if (idx >= 0 && idx < static_cast<int64_t>(ui.length)) acc = fmaf(x[idx], h[j], acc);
+      const uint32_t centre = static_cast<uint32_t>(pos / p.fresh);
+      const float* __restrict__ h = table + (pos - static_cast<uint64_t>(centre) * p.fresh) * taps;
+      if (centre >= p.reach && centre - p.reach + taps <= ui.length) {
+        // every tap lies inside the utterance
+        const float* __restrict__ xs = x + (centre - p.reach);
+#pragma unroll 4
+        for (uint32_t j = 0; j < taps; ++j) acc = fmaf(xs[j], h[j], acc);
+      } else {
+        const int64_t first = static_cast<int64_t>(centre) - p.reach;
+        for (uint32_t j = 0; j < taps; ++j) {
+          const int64_t idx = first + j;
+          if (idx >= 0 && idx < static_cast<int64_t>(ui.length)) acc = fmaf(x[idx], h[j], acc);
+        }
       }
     }
     y[m] = acc;
