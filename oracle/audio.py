@@ -6,7 +6,7 @@ item 1); Sec. 4.2 spells out Normalize as three passes: the mean over all sample
 variance using that mean, then the normalisation of each sample by both.  It fixes no numerics.
 The readings taken here (every one of them a choice, listed in the design doc):
 
-  - input: mono float32 PCM at the model's rate already (16 kHz); resampling is not built;
+  - input: mono float32 PCM at the model's rate (16 kHz); other rates go through `resample` below;
   - framing: frame t holds samples [t*hop, t*hop + win), win = 400, hop = 160, no padding, so an
     utterance of L >= win samples gives T = 1 + (L - win) // hop frames (none when L < win);
   - window: periodic Hann, w[n] = 0.5 - 0.5*cos(2*pi*n/win); the windowed frame is zero-padded to
