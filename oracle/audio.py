@@ -4,7 +4,7 @@ The paper lists the audio units as Resample, Mel spectrogram and Normalize (Tabl
 operations as "resampling, Fast Fourier Transform (FFT), and applying Mel filters" (Sec. 2.3
 item 1); Sec. 4.2 spells out Normalize as three passes: the mean over all samples, the
 variance using that mean, then the normalisation of each sample by both.  It fixes no numerics.
-The readings taken here (every one of them a choice, listed in the design doc):
+The readings taken here (every one of them a choice of this library, not of the paper):
 
   - input: mono float32 PCM at the model's rate (16 kHz); other rates go through `resample` below;
   - framing: frame t holds samples [t*hop, t*hop + win), win = 400, hop = 160, no padding, so an
