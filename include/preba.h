@@ -49,7 +49,8 @@ extern "C" {
 #define PREBA_ERR_BAD_TABLE (-3)        /* a table entry is misaligned, out of range or past the pixels */
 #define PREBA_ERR_CUDA (-4)             /* a CUDA runtime call failed; see preba_last_cuda_error */
 #define PREBA_ERR_TIMEOUT (-5)          /* only in the device status word: a bounded wait ran out */
-#define PREBA_ERR_TOO_LARGE (-6)        /* the batch exceeds PREBA_NOALLOC_MAX_BYTES */
+#define PREBA_ERR_TOO_LARGE (-6)        /* the batch exceeds PREBA_NOALLOC_MAX_BYTES, or an image is
+                                           reduced by more than the antialiased kernel can hold */
 #define PREBA_ERR_BAD_CROP (-7)         /* a crop window does not lie on its image's resized grid */
 
 /* Device memory the library itself carries for preba_preprocess_host_noalloc (64 MiB). */
@@ -238,6 +239,31 @@ typedef struct {
  * Errors: as preba_preprocess, and PREBA_ERR_BAD_CROP.
  */
 int preba_preprocess_ex(const preba_batch_t* batch, const preba_options_t* opt, void* stream);
+
+/*
+ * preba_preprocess_antialias — the transform with an antialiased Resize unit, for inputs much
+ * larger than the model's resolution (paper Table 1's Resize reconfigured, Sec. 4.2 "Flexible
+ * design based on reconfigurable hardware"; the paper fixes no filter): a separable triangle
+ * filter whose half-width is the reduction factor.  On each axis, with n_in input pixels, R
+ * resized pixels (the sizes of preba_preprocess) and M = max(n_in, R), input pixel j weighs
+ *     W = max(0, 2M - |(2j+1) R - (2X+1) n_in|)
+ * in resized pixel X, normalised by the sum over the pixels 0 <= j < n_in; the value is
+ * sum_i sum_j wy_i wx_j p[i][j], then (v/255 - mean)/std.  An axis that is not reduced gets
+ * the two-tap interpolation of preba_preprocess.  Integer taps and weights, fp32 sums.
+ * `opt` is read as by preba_preprocess_ex (crop windows included) with flags == 0 and a float
+ * out_dtype; batch layout, table checks and status word are those of preba_preprocess;
+ * batch->scratch is not used and PREBA_OVERLAP_PREVIOUS has no effect.  One kernel is
+ * enqueued on `stream`.
+ * A CTA keeps one channel-planar row of the window's footprint and the weight tables in
+ * shared memory; with `table_host` the launch carries what the largest image needs and an
+ * image that needs more than the device allows is refused (PREBA_ERR_TOO_LARGE: reductions
+ * beyond about 40 at out_size 224); without it the launch carries all the device allows and
+ * the kernel skips and reports such an image in the status word.
+ * Errors: PREBA_ERR_INVALID_ARG, PREBA_ERR_BUFFER_TOO_SMALL, PREBA_ERR_BAD_TABLE,
+ * PREBA_ERR_BAD_CROP, PREBA_ERR_TOO_LARGE, PREBA_ERR_CUDA.
+ */
+int preba_preprocess_antialias(const preba_batch_t* batch, const preba_options_t* opt,
+                               void* stream);
 
 /*
  * preba_preprocess_host — the same transform for a batch held in host memory

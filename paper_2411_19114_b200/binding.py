@@ -30,7 +30,8 @@ ERR_TOO_LARGE = -6
 ERR_BAD_CROP = -7
 NOALLOC_MAX_BYTES = 64 << 20
 
-EXPORTS = ("preba_query", "preba_pack", "preba_preprocess", "preba_preprocess_ex", "preba_preprocess_host",
+EXPORTS = ("preba_query", "preba_pack", "preba_preprocess", "preba_preprocess_ex",
+           "preba_preprocess_antialias", "preba_preprocess_host",
            "preba_preprocess_images",
            "preba_preprocess_host_noalloc", "preba_preprocess_repeated", "preba_selftest_wait_limit",
            "preba_strerror",
@@ -140,6 +141,8 @@ def lib() -> ctypes.CDLL:
         L.preba_preprocess_ex.argtypes = [ctypes.POINTER(PrebaBatch), ctypes.POINTER(PrebaOptions),
                                           ctypes.c_void_p]
         L.preba_preprocess_ex.restype = ctypes.c_int
+        L.preba_preprocess_antialias.argtypes = L.preba_preprocess_ex.argtypes
+        L.preba_preprocess_antialias.restype = ctypes.c_int
         L.preba_preprocess_images.argtypes = [ctypes.POINTER(PrebaImageBatch), ctypes.c_uint32,
                                               ctypes.c_uint32, f32p, f32p, ctypes.c_int,
                                               ctypes.c_void_p]
@@ -311,13 +314,15 @@ class PreparedPreprocessEx:
                  out_dtype: int, round_u8: bool = False, crop_origin=None,
                  crop_origin_host: np.ndarray | None = None, stream=None,
                  table_host: np.ndarray | None = None, status=None, scratch=None,
-                 flags: int = 0):
+                 flags: int = 0, entry: str = "preba_preprocess_ex"):
         import torch
 
         if stream is None:
             stream = torch.cuda.current_stream().cuda_stream
         elif hasattr(stream, "cuda_stream"):
             stream = stream.cuda_stream
+        self._entry = entry
+        self._fn = getattr(lib(), entry)
         batch = PrebaBatch()
         batch.pixels = pixels.data_ptr()
         batch.pixels_bytes = pixels.numel() * pixels.element_size()
@@ -344,9 +349,9 @@ class PreparedPreprocessEx:
         self._args = (ctypes.byref(batch), ctypes.byref(opt), ctypes.c_void_p(stream))
 
     def __call__(self) -> None:
-        rc = lib().preba_preprocess_ex(*self._args)
+        rc = self._fn(*self._args)
         if rc != OK:
-            raise PrebaError(rc, "preba_preprocess_ex")
+            raise PrebaError(rc, self._entry)
 
 
 def preba_preprocess_ex(pixels, table, n: int, out, out_size: int, resize_short: int, mean, std,
@@ -360,6 +365,17 @@ def preba_preprocess_ex(pixels, table, n: int, out, out_size: int, resize_short:
     PreparedPreprocessEx(pixels, table, n, out, out_size, resize_short, mean, std, out_dtype,
                          round_u8, crop_origin, crop_origin_host, stream, table_host, status,
                          scratch, flags)()
+
+
+def preba_preprocess_antialias(pixels, table, n: int, out, out_size: int, resize_short: int, mean,
+                               std, out_dtype: int, crop_origin=None,
+                               crop_origin_host: np.ndarray | None = None, stream=None,
+                               table_host: np.ndarray | None = None, status=None) -> None:
+    """``preba_preprocess_antialias``: the transform with the triangle filter widened by the
+    reduction factor; arguments as ``preba_preprocess_ex`` without rounding."""
+    PreparedPreprocessEx(pixels, table, n, out, out_size, resize_short, mean, std, out_dtype,
+                         False, crop_origin, crop_origin_host, stream, table_host, status,
+                         None, 0, entry="preba_preprocess_antialias")()
 
 
 class PreparedPreprocess:

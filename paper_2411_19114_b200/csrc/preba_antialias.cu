@@ -1,0 +1,404 @@
+// Antialiased Resize -> Crop -> Normalize (the Resize unit of the paper's Table 1 reconfigured,
+// Sec. 4.2 "Flexible design based on reconfigurable hardware", for inputs much larger than the
+// model's resolution): a separable triangle filter whose half-width is the reduction factor.
+//
+// On each axis, with n_in input pixels and R resized pixels, M = max(n_in, R):
+//   weight of input pixel j for resized pixel X  =  W / sum W,
+//   W = max(0, 2M - |(2j+1) R - (2X+1) n_in|)        (an integer; the triangle times 2M)
+// so taps and un-normalised weights come from exact integer arithmetic; the sums run in fp32.
+//
+// One CTA produces `rows` consecutive output rows of one image.  Per output row:
+//   vertical pass   every thread owns 4-byte words of the input rows' needed byte range and
+//                   accumulates the weighted rows (each input byte is converted once per output
+//                   row that uses it); the result goes to shared memory, one plane per channel,
+//                   one element of padding every 32 so that the strided reads below spread over
+//                   the banks;
+//   horizontal pass a thread per output column sums its taps for the three channels, applies the
+//                   normalising multiply-add and stores the three planes' elements.
+// The horizontal weights are the same for every row of the image, so they are tabulated once
+// per CTA in shared memory.  HBM traffic is every input byte under the crop's footprint once
+// (rows shared by neighbouring CTAs come from L2) plus the output.
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <atomic>
+
+#include "preba.h"
+#include "preba_internal.h"
+
+namespace preba {
+namespace aa {
+
+constexpr int kThreads = 256;
+constexpr uint32_t kMaxRows = 16;  // output rows per CTA, at most
+
+struct Params {
+  const uint8_t* pixels;
+  uint64_t pixels_bytes;
+  const preba_img_t* table;
+  const uint32_t* crop;  // 2n (top, left) or nullptr
+  void* out;
+  int32_t* status;
+  uint32_t n, C, S;
+  uint32_t rows;         // output rows per CTA
+  uint32_t smem_floats;  // shared memory the launch carries, in 4-byte units
+  float mul[3], add[3];  // y = v * mul + add
+};
+
+// One axis of one image.
+struct Axis {
+  uint32_t n_in, R, M;  // M = max(n_in, R)
+  uint32_t taps;        // upper bound of the taps of one resized pixel
+};
+
+__host__ __device__ inline Axis make_axis(uint32_t n_in, uint32_t R) {
+  Axis a;
+  a.n_in = n_in;
+  a.R = R;
+  a.M = n_in > R ? n_in : R;
+  // (2j+1) R lies strictly inside an interval of length 4M: fewer than 2M/R + 1 values of j
+  a.taps = 2u * a.M / R + 2u;
+  return a;
+}
+
+__host__ __device__ inline int64_t floor_div(int64_t a, int64_t b) {  // b > 0
+  const int64_t q = a / b;
+  return (a % b != 0 && a < 0) ? q - 1 : q;
+}
+
+// First tap and one past the last tap of resized pixel X (those with W > 0, inside the image).
+__host__ __device__ inline void tap_range(const Axis& a, uint32_t X, uint32_t* lo, uint32_t* hi) {
+  const int64_t centre = static_cast<int64_t>(2ull * X + 1) * a.n_in;
+  const int64_t R = a.R, M2 = 2ll * a.M;
+  // (2j+1) R > centre - 2M  <=>  j > (centre - 2M - R) / 2R
+  int64_t first = floor_div(centre - M2 - R, 2 * R) + 1;
+  // (2j+1) R < centre + 2M  <=>  j < (centre + 2M - R) / 2R
+  int64_t last = floor_div(centre + M2 - R + 2 * R - 1, 2 * R);  // ceiling: one past the last
+  if (first < 0) first = 0;
+  if (last > static_cast<int64_t>(a.n_in)) last = a.n_in;
+  *lo = static_cast<uint32_t>(first);
+  *hi = static_cast<uint32_t>(last);
+}
+
+// Un-normalised integer weight of input pixel j for resized pixel X (positive inside tap_range).
+__host__ __device__ inline int32_t tap_weight(const Axis& a, uint32_t X, uint32_t j) {
+  const int64_t d = static_cast<int64_t>(2ull * j + 1) * a.R -
+                    static_cast<int64_t>(2ull * X + 1) * a.n_in;
+  const int64_t w = 2ll * a.M - (d < 0 ? -d : d);
+  return w > 0 ? static_cast<int32_t>(w) : 0;
+}
+
+__host__ __device__ inline void resized_size(uint32_t h, uint32_t w, uint32_t S, uint32_t* rh,
+                                             uint32_t* rw) {
+  if (h <= w) {
+    *rh = S;
+    *rw = static_cast<uint32_t>(static_cast<uint64_t>(S) * w / h);
+  } else {
+    *rh = static_cast<uint32_t>(static_cast<uint64_t>(S) * h / w);
+    *rw = S;
+  }
+}
+
+// Shared-memory plan of one CTA (in 4-byte units), from bounds that hold for any crop origin.
+struct Plan {
+  uint32_t tx, ty;     // pitch of the weight tables (odd, so that table reads spread over banks)
+  uint32_t plane;      // elements of one channel plane of the vertical pass's result
+  uint32_t off_wx, off_xlo, off_xcnt, off_wy, off_ylo, off_ycnt, off_v, total;
+};
+
+__host__ __device__ inline Plan make_plan(const Axis& ax, const Axis& ay, uint32_t C,
+                                          uint32_t rows) {
+  Plan p;
+  p.tx = ax.taps | 1u;
+  p.ty = ay.taps | 1u;
+  // pixels under C resized pixels: ((C-1) n_in + 2M)/R + 2 <= (C+1) M/R + 2; one pixel before
+  // and two after for the word-aligned ends
+  const uint64_t span = (static_cast<uint64_t>(C + 1) * ax.M + ax.R - 1) / ax.R + 2 + 4;
+  const uint32_t px = static_cast<uint32_t>(span < ax.n_in + 4ull ? span : ax.n_in + 4ull);
+  p.plane = px + px / 32 + 1;
+  uint32_t at = 0;
+  p.off_wx = at, at += C * p.tx;
+  p.off_xlo = at, at += C;
+  p.off_xcnt = at, at += C;
+  p.off_wy = at, at += rows * p.ty;
+  p.off_ylo = at, at += rows;
+  p.off_ycnt = at, at += rows;
+  p.off_v = at, at += 3 * p.plane;
+  p.total = at;
+  return p;
+}
+
+__device__ __forceinline__ void report(int32_t* status, int code) {
+  if (status) atomicCAS(status, 0, code);
+}
+
+template <typename OutT>
+__device__ __forceinline__ OutT to_out(float v);
+template <>
+__device__ __forceinline__ float to_out<float>(float v) { return v; }
+template <>
+__device__ __forceinline__ __half to_out<__half>(float v) { return __float2half_rn(v); }
+template <>
+__device__ __forceinline__ __nv_bfloat16 to_out<__nv_bfloat16>(float v) {
+  return __float2bfloat16_rn(v);
+}
+
+// Tabulates taps and normalised weights of resized pixels first .. first + count - 1 of one
+// axis: row q of `w` (pitch `pitch`) holds the weights of pixel first + q from tap lo[q] on.
+__device__ void tabulate(const Axis& a, uint32_t first, uint32_t count, uint32_t pitch, float* w,
+                         uint32_t* lo, uint32_t* cnt) {
+  for (uint32_t q = threadIdx.x; q < count; q += kThreads) {
+    uint32_t j0, j1;
+    tap_range(a, first + q, &j0, &j1);
+    uint64_t sum = 0;
+    for (uint32_t j = j0; j < j1; ++j) sum += static_cast<uint32_t>(tap_weight(a, first + q, j));
+    const float inv = 1.0f / static_cast<float>(sum);
+    for (uint32_t j = j0; j < j1; ++j)
+      w[q * pitch + (j - j0)] = static_cast<float>(tap_weight(a, first + q, j)) * inv;
+    lo[q] = j0;
+    cnt[q] = j1 - j0;
+  }
+}
+
+template <typename OutT>
+__global__ void __launch_bounds__(kThreads) preba_antialias_kernel(const Params p) {
+  extern __shared__ float smem[];
+  const uint32_t tid = threadIdx.x, C = p.C;
+  const uint32_t groups = (C + p.rows - 1) / p.rows;
+  const uint32_t img = blockIdx.x / groups;
+  const uint32_t k0 = (blockIdx.x % groups) * p.rows;
+  const preba_img_t e = p.table[img];
+  // the entry is checked again here: a bad one is skipped and reported (uniform over the CTA)
+  if (e.h < 1 || e.w < 1 || e.h > PREBA_MAX_DIM || e.w > PREBA_MAX_DIM ||
+      e.offset % PREBA_PACK_ALIGN != 0 || e.offset > p.pixels_bytes ||
+      3ull * e.h * e.w > p.pixels_bytes - e.offset) {
+    if (tid == 0) report(p.status, PREBA_ERR_BAD_TABLE);
+    return;
+  }
+  uint32_t rh, rw, top, left;
+  resized_size(e.h, e.w, p.S, &rh, &rw);
+  if (p.crop) {
+    top = p.crop[2 * img];
+    left = p.crop[2 * img + 1];
+    if (static_cast<uint64_t>(top) + C > rh || static_cast<uint64_t>(left) + C > rw) {
+      if (tid == 0) report(p.status, PREBA_ERR_BAD_CROP);
+      return;
+    }
+  } else {
+    top = (rh - C) / 2;
+    left = (rw - C) / 2;
+  }
+  const Axis ax = make_axis(e.w, rw), ay = make_axis(e.h, rh);
+  const Plan pl = make_plan(ax, ay, C, p.rows);
+  if (pl.total > p.smem_floats) {
+    if (tid == 0) report(p.status, PREBA_ERR_TOO_LARGE);
+    return;
+  }
+  const uint32_t rows_here = C - k0 < p.rows ? C - k0 : p.rows;
+  float* wx = smem + pl.off_wx;
+  uint32_t* xlo = reinterpret_cast<uint32_t*>(smem + pl.off_xlo);
+  uint32_t* xcnt = reinterpret_cast<uint32_t*>(smem + pl.off_xcnt);
+  float* wy = smem + pl.off_wy;
+  uint32_t* ylo = reinterpret_cast<uint32_t*>(smem + pl.off_ylo);
+  uint32_t* ycnt = reinterpret_cast<uint32_t*>(smem + pl.off_ycnt);
+  float* v = smem + pl.off_v;
+  tabulate(ax, left, C, pl.tx, wx, xlo, xcnt);
+  tabulate(ay, top + k0, rows_here, pl.ty, wy, ylo, ycnt);
+  __syncthreads();
+
+  // the byte range of a row that the window's taps cover, from a 4-byte boundary of the row
+  const uint32_t b0 = (3u * xlo[0]) & ~3u;
+  const uint32_t b1 = 3u * (xlo[C - 1] + xcnt[C - 1]);
+  const uint32_t nwords = (b1 - b0 + 3u) / 4u;
+  const uint32_t p0 = b0 / 3u;  // the pixel plane element 0 stands for
+  {
+    const uint32_t last = (b0 + 4u * nwords - 1u) / 3u - p0;
+    if (last + (last >> 5) >= pl.plane) {  // cannot happen within the plan's bounds
+      if (tid == 0) report(p.status, PREBA_ERR_TOO_LARGE);
+      return;
+    }
+  }
+  const uint64_t pitch = 3ull * e.w;
+  const uint32_t* words = reinterpret_cast<const uint32_t*>(p.pixels);
+  OutT* out = static_cast<OutT*>(p.out) + static_cast<uint64_t>(img) * 3u * C * C;
+
+  for (uint32_t q = 0; q < rows_here; ++q) {
+    // ---- vertical pass ----
+    const uint32_t y0 = ylo[q], ny = ycnt[q];
+    const float* wq = wy + q * pl.ty;
+    for (uint32_t wv = tid; wv < nwords; wv += kThreads) {
+      float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+      uint64_t at = e.offset + y0 * pitch + b0 + 4ull * wv;  // the word's first byte
+#pragma unroll 4
+      for (uint32_t i = 0; i < ny; ++i, at += pitch) {
+        const uint32_t m = static_cast<uint32_t>(at) & 3u;  // the same for every thread
+        const uint64_t aligned = at - m;
+        uint32_t px = aligned + 4 <= p.pixels_bytes ? __ldg(words + aligned / 4) : 0u;
+        if (m) {
+          const uint32_t hi = aligned + 8 <= p.pixels_bytes ? __ldg(words + aligned / 4 + 1) : 0u;
+          px = __funnelshift_r(px, hi, 8u * m);
+        }
+        const float w = wq[i];
+        a0 = fmaf(w, static_cast<float>(px & 0xffu), a0);
+        a1 = fmaf(w, static_cast<float>((px >> 8) & 0xffu), a1);
+        a2 = fmaf(w, static_cast<float>((px >> 16) & 0xffu), a2);
+        a3 = fmaf(w, static_cast<float>(px >> 24), a3);
+      }
+      const float acc[4] = {a0, a1, a2, a3};
+#pragma unroll
+      for (uint32_t t = 0; t < 4; ++t) {
+        const uint32_t byte = b0 + 4u * wv + t;
+        const uint32_t pix = byte / 3u, ch = byte - 3u * pix, rel = pix - p0;
+        v[ch * pl.plane + rel + (rel >> 5)] = acc[t];
+      }
+    }
+    __syncthreads();
+    // ---- horizontal pass, normalisation, store ----
+    for (uint32_t X = tid; X < C; X += kThreads) {
+      const uint32_t rel0 = xlo[X] - p0, nx = xcnt[X];
+      const float* w = wx + X * pl.tx;
+      float s0 = 0.f, s1 = 0.f, s2 = 0.f;
+      for (uint32_t t = 0; t < nx; ++t) {
+        uint32_t idx = rel0 + t;
+        idx += idx >> 5;
+        const float wt = w[t];
+        s0 = fmaf(wt, v[idx], s0);
+        s1 = fmaf(wt, v[pl.plane + idx], s1);
+        s2 = fmaf(wt, v[2 * pl.plane + idx], s2);
+      }
+      const uint64_t o = static_cast<uint64_t>(k0 + q) * C + X;
+      out[o] = to_out<OutT>(fmaf(s0, p.mul[0], p.add[0]));
+      out[o + static_cast<uint64_t>(C) * C] = to_out<OutT>(fmaf(s1, p.mul[1], p.add[1]));
+      out[o + 2ull * C * C] = to_out<OutT>(fmaf(s2, p.mul[2], p.add[2]));
+    }
+    __syncthreads();
+  }
+}
+
+}  // namespace aa
+}  // namespace preba
+
+namespace {
+
+using preba::aa::Params;
+
+typedef void (*Kernel)(const Params);
+
+Kernel kernel_for(int out_dtype) {
+  return out_dtype == PREBA_F32   ? preba::aa::preba_antialias_kernel<float>
+         : out_dtype == PREBA_F16 ? preba::aa::preba_antialias_kernel<__half>
+                                  : preba::aa::preba_antialias_kernel<__nv_bfloat16>;
+}
+
+// Largest dynamic shared memory a CTA may ask for on the current device; the three kernels
+// are opted in to it once per device.
+int shared_memory_limit(cudaError_t* err) {
+  constexpr int kMaxDevices = 64;
+  static std::atomic<int> cache[kMaxDevices];
+  int dev = -1;
+  *err = cudaGetDevice(&dev);
+  if (*err != cudaSuccess) return 0;
+  if (dev >= 0 && dev < kMaxDevices) {
+    const int known = cache[dev].load(std::memory_order_relaxed);
+    if (known > 0) return known;
+  }
+  int optin = 0;
+  *err = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+  for (int dt : {PREBA_F32, PREBA_F16, PREBA_BF16})
+    if (*err == cudaSuccess)
+      *err = cudaFuncSetAttribute(kernel_for(dt), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  optin);
+  if (*err != cudaSuccess) return 0;
+  if (dev >= 0 && dev < kMaxDevices) cache[dev].store(optin, std::memory_order_relaxed);
+  return optin;
+}
+
+}  // namespace
+
+extern "C" int preba_preprocess_antialias(const preba_batch_t* batch, const preba_options_t* opt,
+                                          void* stream) {
+  using namespace preba;
+  using namespace preba::aa;
+  if (!batch || !opt || !batch->pixels || !batch->table || !batch->out || batch->n == 0)
+    return PREBA_ERR_INVALID_ARG;
+  if (opt->flags != 0 || !dtype_ok(opt->out_dtype)) return PREBA_ERR_INVALID_ARG;
+  if (batch->flags & ~PREBA_OVERLAP_PREVIOUS) return PREBA_ERR_INVALID_ARG;
+  const uint32_t C = opt->out_size, S = opt->resize_short;
+  if (C == 0 || S == 0 || S > PREBA_MAX_RESIZE || C > S) return PREBA_ERR_INVALID_ARG;
+  for (int c = 0; c < 3; ++c)
+    if (!(opt->mean[c] == opt->mean[c]) || !(opt->std[c] == opt->std[c]) || opt->std[c] == 0.f ||
+        opt->std[c] - opt->std[c] != 0.f || opt->mean[c] - opt->mean[c] != 0.f)
+      return PREBA_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(batch->pixels) % 16 || reinterpret_cast<uintptr_t>(batch->out) % 16 ||
+      reinterpret_cast<uintptr_t>(batch->table) % 8 || reinterpret_cast<uintptr_t>(opt->crop_origin) % 4)
+    return PREBA_ERR_INVALID_ARG;
+  const uint64_t need = static_cast<uint64_t>(batch->n) * 3ull * C * C * dtype_bytes(opt->out_dtype);
+  if (batch->out_bytes < need) return PREBA_ERR_BUFFER_TOO_SMALL;
+  const uint32_t groups_at_one = C;  // CTAs of one image when every CTA makes one row
+  if (static_cast<uint64_t>(batch->n) * groups_at_one > 0x7fffffffull) return PREBA_ERR_INVALID_ARG;
+
+  cudaError_t err = cudaSuccess;
+  const int limit = shared_memory_limit(&err);
+  int sms = 0, dev = 0;
+  if (err == cudaSuccess) err = cudaGetDevice(&dev);
+  if (err == cudaSuccess) err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (err != cudaSuccess) {
+    g_last_cuda_error = static_cast<int>(err);
+    return PREBA_ERR_CUDA;
+  }
+  // rows per CTA: as many as kMaxRows while the batch still gives every SM a few CTAs
+  uint32_t rows = kMaxRows;
+  while (rows > 1 && static_cast<uint64_t>(batch->n) * ((C + rows - 1) / rows) < 4ull * sms)
+    rows /= 2;
+
+  // Shared memory: with the host's copy of the table, what the largest image needs; without
+  // it, all a CTA may have (images that need more are reported by the kernel).
+  uint32_t floats = static_cast<uint32_t>(limit) / 4u;
+  if (batch->table_host) {
+    uint32_t most = 0;
+    for (uint32_t i = 0; i < batch->n; ++i) {
+      const preba_img_t& e = batch->table_host[i];
+      if (!dims_ok(e.h, e.w) || e.offset % PREBA_PACK_ALIGN || e.offset > batch->pixels_bytes ||
+          3ull * e.h * e.w > batch->pixels_bytes - e.offset)
+        return PREBA_ERR_BAD_TABLE;
+      uint32_t rh, rw;
+      resized_size(e.h, e.w, S, &rh, &rw);
+      if (opt->crop_origin_host &&
+          (opt->crop_origin_host[2 * i] + static_cast<uint64_t>(C) > rh ||
+           opt->crop_origin_host[2 * i + 1] + static_cast<uint64_t>(C) > rw))
+        return PREBA_ERR_BAD_CROP;
+      const Plan pl = make_plan(make_axis(e.w, rw), make_axis(e.h, rh), C, rows);
+      if (pl.total > most) most = pl.total;
+    }
+    if (most > floats) return PREBA_ERR_TOO_LARGE;
+    floats = most;
+  }
+
+  Params p = {};
+  p.pixels = batch->pixels;
+  p.pixels_bytes = batch->pixels_bytes;
+  p.table = batch->table;
+  p.crop = opt->crop_origin;
+  p.out = batch->out;
+  p.status = batch->status;
+  p.n = batch->n;
+  p.C = C;
+  p.S = S;
+  p.rows = rows;
+  p.smem_floats = floats;
+  for (int c = 0; c < 3; ++c) {
+    p.mul[c] = static_cast<float>(1.0 / (255.0 * static_cast<double>(opt->std[c])));
+    p.add[c] = static_cast<float>(-static_cast<double>(opt->mean[c]) /
+                                  static_cast<double>(opt->std[c]));
+  }
+  const uint32_t grid = batch->n * ((C + rows - 1) / rows);
+  kernel_for(opt->out_dtype)<<<grid, kThreads, floats * 4u, static_cast<cudaStream_t>(stream)>>>(p);
+  err = cudaGetLastError();
+  if (err != cudaSuccess) {
+    g_last_cuda_error = static_cast<int>(err);
+    return PREBA_ERR_CUDA;
+  }
+  return PREBA_OK;
+}
