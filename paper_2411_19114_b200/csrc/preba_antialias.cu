@@ -7,14 +7,15 @@
 //   W = max(0, 2M - |(2j+1) R - (2X+1) n_in|)        (an integer; the triangle times 2M)
 // so taps and un-normalised weights come from exact integer arithmetic; the sums run in fp32.
 //
-// One CTA produces `rows` consecutive output rows of one image.  Per output row:
-//   vertical pass   every thread owns 4-byte words of the input rows' needed byte range and
-//                   accumulates the weighted rows (each input byte is converted once per output
-//                   row that uses it); the result goes to shared memory, one plane per channel,
-//                   one element of padding every 32 so that the strided reads below spread over
-//                   the banks;
-//   horizontal pass a thread per output column sums its taps for the three channels, applies the
-//                   normalising multiply-add and stores the three planes' elements.
+// One CTA produces `rows` consecutive output rows of one image, two at a time (neighbouring
+// rows share about half of their input rows).  Per pair of output rows:
+//   vertical pass   every thread owns up to kWords 4-byte words of the needed byte range of
+//                   the input rows and accumulates them into both rows' sums, all loads of a
+//                   row in flight together; the results go to shared memory, one plane per
+//                   channel and row, one element of padding every 32 so that the strided reads
+//                   below spread over the banks;
+//   horizontal pass a thread per output column sums its taps for the three channels of both
+//                   rows, applies the normalising multiply-add and stores the elements.
 // The horizontal weights are the same for every row of the image, so they are tabulated once
 // per CTA in shared memory.  HBM traffic is every input byte under the crop's footprint once
 // (rows shared by neighbouring CTAs come from L2) plus the output.
@@ -32,7 +33,8 @@ namespace preba {
 namespace aa {
 
 constexpr int kThreads = 256;
-constexpr uint32_t kMaxRows = 16;  // output rows per CTA, at most
+constexpr uint32_t kMaxRows = 32;  // output rows per CTA, at most
+constexpr uint32_t kWords = 3;     // 4-byte words of a row a thread holds at a time
 
 struct Params {
   const uint8_t* pixels;
@@ -102,30 +104,35 @@ __host__ __device__ inline void resized_size(uint32_t h, uint32_t w, uint32_t S,
 }
 
 // Shared-memory plan of one CTA (in 4-byte units), from bounds that hold for any crop origin.
+// Output rows are made two at a time: neighbouring rows share about half of their input rows.
 struct Plan {
-  uint32_t tx, ty;     // pitch of the weight tables (odd, so that table reads spread over banks)
-  uint32_t plane;      // elements of one channel plane of the vertical pass's result
-  uint32_t off_wx, off_xlo, off_xcnt, off_wy, off_ylo, off_ycnt, off_v, total;
+  uint32_t tx;     // pitch of the horizontal weight table (odd: table reads spread over banks)
+  uint32_t tp;     // pitch, in (weight of row a, weight of row b) pairs, of the row-pair tables
+  uint32_t plane;  // elements of one channel plane of the vertical pass's result
+  uint32_t off_wx, off_xlo, off_xcnt, off_wp, off_plo, off_pcnt, off_v, total;
 };
 
 __host__ __device__ inline Plan make_plan(const Axis& ax, const Axis& ay, uint32_t C,
                                           uint32_t rows) {
   Plan p;
   p.tx = ax.taps | 1u;
-  p.ty = ay.taps | 1u;
+  // taps of one row plus the distance between the first taps of neighbouring rows
+  p.tp = ay.taps + ay.M / ay.R + 2u;
   // pixels under C resized pixels: ((C-1) n_in + 2M)/R + 2 <= (C+1) M/R + 2; one pixel before
   // and two after for the word-aligned ends
   const uint64_t span = (static_cast<uint64_t>(C + 1) * ax.M + ax.R - 1) / ax.R + 2 + 4;
   const uint32_t px = static_cast<uint32_t>(span < ax.n_in + 4ull ? span : ax.n_in + 4ull);
   p.plane = px + px / 32 + 1;
+  const uint32_t pairs = (rows + 1) / 2;
   uint32_t at = 0;
   p.off_wx = at, at += C * p.tx;
   p.off_xlo = at, at += C;
   p.off_xcnt = at, at += C;
-  p.off_wy = at, at += rows * p.ty;
-  p.off_ylo = at, at += rows;
-  p.off_ycnt = at, at += rows;
-  p.off_v = at, at += 3 * p.plane;
+  at += at & 1u;  // the pair table is read 8 bytes at a time
+  p.off_wp = at, at += pairs * p.tp * 2;
+  p.off_plo = at, at += pairs;
+  p.off_pcnt = at, at += pairs;
+  p.off_v = at, at += 6 * p.plane;
   p.total = at;
   return p;
 }
@@ -145,8 +152,8 @@ __device__ __forceinline__ __nv_bfloat16 to_out<__nv_bfloat16>(float v) {
   return __float2bfloat16_rn(v);
 }
 
-// Tabulates taps and normalised weights of resized pixels first .. first + count - 1 of one
-// axis: row q of `w` (pitch `pitch`) holds the weights of pixel first + q from tap lo[q] on.
+// Horizontal table: row q of `w` (pitch `pitch`) holds the normalised weights of resized
+// pixel first + q from tap lo[q] on.
 __device__ void tabulate(const Axis& a, uint32_t first, uint32_t count, uint32_t pitch, float* w,
                          uint32_t* lo, uint32_t* cnt) {
   for (uint32_t q = threadIdx.x; q < count; q += kThreads) {
@@ -159,6 +166,35 @@ __device__ void tabulate(const Axis& a, uint32_t first, uint32_t count, uint32_t
       w[q * pitch + (j - j0)] = static_cast<float>(tap_weight(a, first + q, j)) * inv;
     lo[q] = j0;
     cnt[q] = j1 - j0;
+  }
+}
+
+// Vertical tables: pair r covers resized rows first + 2r (a) and first + 2r + 1 (b, if below
+// `count`); entry i of its table holds both rows' normalised weights of input row lo[r] + i
+// (zero where a row does not reach), over the union of the two rows' taps.
+__device__ void tabulate_pairs(const Axis& a, uint32_t first, uint32_t count, uint32_t pitch,
+                               float2* w, uint32_t* lo, uint32_t* cnt) {
+  for (uint32_t r = threadIdx.x; 2 * r < count; r += kThreads) {
+    const uint32_t ya = first + 2 * r;
+    const bool has_b = 2 * r + 1 < count;
+    uint32_t a0, a1, b0, b1;
+    tap_range(a, ya, &a0, &a1);
+    b0 = a0, b1 = a1;
+    if (has_b) tap_range(a, ya + 1, &b0, &b1);
+    const uint32_t j0 = a0, j1 = a1 > b1 ? a1 : b1;  // first taps do not decrease with the row
+    uint64_t sum_a = 0, sum_b = 0;
+    for (uint32_t j = j0; j < j1; ++j) {
+      sum_a += static_cast<uint32_t>(tap_weight(a, ya, j));
+      if (has_b) sum_b += static_cast<uint32_t>(tap_weight(a, ya + 1, j));
+    }
+    const float inv_a = 1.0f / static_cast<float>(sum_a);
+    const float inv_b = has_b ? 1.0f / static_cast<float>(sum_b) : 0.f;
+    for (uint32_t j = j0; j < j1; ++j)
+      w[r * pitch + (j - j0)] =
+          make_float2(static_cast<float>(tap_weight(a, ya, j)) * inv_a,
+                      has_b ? static_cast<float>(tap_weight(a, ya + 1, j)) * inv_b : 0.f);
+    lo[r] = j0;
+    cnt[r] = j1 - j0;
   }
 }
 
@@ -200,19 +236,20 @@ __global__ void __launch_bounds__(kThreads) preba_antialias_kernel(const Params 
   float* wx = smem + pl.off_wx;
   uint32_t* xlo = reinterpret_cast<uint32_t*>(smem + pl.off_xlo);
   uint32_t* xcnt = reinterpret_cast<uint32_t*>(smem + pl.off_xcnt);
-  float* wy = smem + pl.off_wy;
-  uint32_t* ylo = reinterpret_cast<uint32_t*>(smem + pl.off_ylo);
-  uint32_t* ycnt = reinterpret_cast<uint32_t*>(smem + pl.off_ycnt);
-  float* v = smem + pl.off_v;
+  float2* wp = reinterpret_cast<float2*>(smem + pl.off_wp);
+  uint32_t* plo = reinterpret_cast<uint32_t*>(smem + pl.off_plo);
+  uint32_t* pcnt = reinterpret_cast<uint32_t*>(smem + pl.off_pcnt);
+  float* va = smem + pl.off_v;       // three planes of row a, then three of row b
+  float* vb = va + 3 * pl.plane;
   tabulate(ax, left, C, pl.tx, wx, xlo, xcnt);
-  tabulate(ay, top + k0, rows_here, pl.ty, wy, ylo, ycnt);
+  tabulate_pairs(ay, top + k0, rows_here, pl.tp, wp, plo, pcnt);
   __syncthreads();
 
   // the byte range of a row that the window's taps cover, from a 4-byte boundary of the row
   const uint32_t b0 = (3u * xlo[0]) & ~3u;
   const uint32_t b1 = 3u * (xlo[C - 1] + xcnt[C - 1]);
   const uint32_t nwords = (b1 - b0 + 3u) / 4u;
-  const uint32_t p0 = b0 / 3u;  // the pixel plane element 0 stands for
+  const uint32_t p0 = b0 / 3u;  // the pixel that element 0 of a plane stands for
   {
     const uint32_t last = (b0 + 4u * nwords - 1u) / 3u - p0;
     if (last + (last >> 5) >= pl.plane) {  // cannot happen within the plan's bounds
@@ -224,54 +261,89 @@ __global__ void __launch_bounds__(kThreads) preba_antialias_kernel(const Params 
   const uint32_t* words = reinterpret_cast<const uint32_t*>(p.pixels);
   OutT* out = static_cast<OutT*>(p.out) + static_cast<uint64_t>(img) * 3u * C * C;
 
-  for (uint32_t q = 0; q < rows_here; ++q) {
-    // ---- vertical pass ----
-    const uint32_t y0 = ylo[q], ny = ycnt[q];
-    const float* wq = wy + q * pl.ty;
-    for (uint32_t wv = tid; wv < nwords; wv += kThreads) {
-      float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-      uint64_t at = e.offset + y0 * pitch + b0 + 4ull * wv;  // the word's first byte
-#pragma unroll 4
-      for (uint32_t i = 0; i < ny; ++i, at += pitch) {
-        const uint32_t m = static_cast<uint32_t>(at) & 3u;  // the same for every thread
-        const uint64_t aligned = at - m;
-        uint32_t px = aligned + 4 <= p.pixels_bytes ? __ldg(words + aligned / 4) : 0u;
-        if (m) {
-          const uint32_t hi = aligned + 8 <= p.pixels_bytes ? __ldg(words + aligned / 4 + 1) : 0u;
-          px = __funnelshift_r(px, hi, 8u * m);
-        }
-        const float w = wq[i];
-        a0 = fmaf(w, static_cast<float>(px & 0xffu), a0);
-        a1 = fmaf(w, static_cast<float>((px >> 8) & 0xffu), a1);
-        a2 = fmaf(w, static_cast<float>((px >> 16) & 0xffu), a2);
-        a3 = fmaf(w, static_cast<float>(px >> 24), a3);
-      }
-      const float acc[4] = {a0, a1, a2, a3};
+  for (uint32_t r = 0; 2 * r < rows_here; ++r) {
+    // ---- vertical pass: both rows of the pair from one sweep over the input rows ----
+    const uint32_t y0 = plo[r], ny = pcnt[r];
+    const float2* wq = wp + r * pl.tp;
+    for (uint32_t w0 = tid; w0 < nwords; w0 += kThreads * kWords) {
+      float acc[kWords][8];
 #pragma unroll
-      for (uint32_t t = 0; t < 4; ++t) {
-        const uint32_t byte = b0 + 4u * wv + t;
-        const uint32_t pix = byte / 3u, ch = byte - 3u * pix, rel = pix - p0;
-        v[ch * pl.plane + rel + (rel >> 5)] = acc[t];
+      for (uint32_t k = 0; k < kWords; ++k)
+#pragma unroll
+        for (uint32_t t = 0; t < 8; ++t) acc[k][t] = 0.f;
+      uint64_t at0 = e.offset + y0 * pitch + b0 + 4ull * w0;  // first byte of the first word
+#pragma unroll 2
+      for (uint32_t i = 0; i < ny; ++i, at0 += pitch) {
+        const float2 w = wq[i];
+        const uint32_t m = static_cast<uint32_t>(at0) & 3u;  // the same for every thread
+        uint32_t px[kWords];
+#pragma unroll
+        for (uint32_t k = 0; k < kWords; ++k) {
+          px[k] = 0u;
+          if (w0 + k * kThreads < nwords) {
+            const uint64_t aligned = at0 + 4ull * k * kThreads - m;
+            if (aligned + 4 <= p.pixels_bytes) px[k] = __ldg(words + aligned / 4);
+            if (m) {
+              const uint32_t hi =
+                  aligned + 8 <= p.pixels_bytes ? __ldg(words + aligned / 4 + 1) : 0u;
+              px[k] = __funnelshift_r(px[k], hi, 8u * m);
+            }
+          }
+        }
+#pragma unroll
+        for (uint32_t k = 0; k < kWords; ++k) {
+          const float f0 = static_cast<float>(px[k] & 0xffu);
+          const float f1 = static_cast<float>((px[k] >> 8) & 0xffu);
+          const float f2 = static_cast<float>((px[k] >> 16) & 0xffu);
+          const float f3 = static_cast<float>(px[k] >> 24);
+          acc[k][0] = fmaf(w.x, f0, acc[k][0]);
+          acc[k][1] = fmaf(w.x, f1, acc[k][1]);
+          acc[k][2] = fmaf(w.x, f2, acc[k][2]);
+          acc[k][3] = fmaf(w.x, f3, acc[k][3]);
+          acc[k][4] = fmaf(w.y, f0, acc[k][4]);
+          acc[k][5] = fmaf(w.y, f1, acc[k][5]);
+          acc[k][6] = fmaf(w.y, f2, acc[k][6]);
+          acc[k][7] = fmaf(w.y, f3, acc[k][7]);
+        }
+      }
+#pragma unroll
+      for (uint32_t k = 0; k < kWords; ++k) {
+        if (w0 + k * kThreads < nwords) {
+#pragma unroll
+          for (uint32_t t = 0; t < 4; ++t) {
+            const uint32_t byte = b0 + 4u * (w0 + k * kThreads) + t;
+            const uint32_t pix = byte / 3u, ch = byte - 3u * pix, rel = pix - p0;
+            const uint32_t at = ch * pl.plane + rel + (rel >> 5);
+            va[at] = acc[k][t];
+            vb[at] = acc[k][4 + t];
+          }
+        }
       }
     }
     __syncthreads();
     // ---- horizontal pass, normalisation, store ----
+    const bool has_b = 2 * r + 1 < rows_here;
     for (uint32_t X = tid; X < C; X += kThreads) {
       const uint32_t rel0 = xlo[X] - p0, nx = xcnt[X];
       const float* w = wx + X * pl.tx;
-      float s0 = 0.f, s1 = 0.f, s2 = 0.f;
+      float s[6] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
       for (uint32_t t = 0; t < nx; ++t) {
         uint32_t idx = rel0 + t;
         idx += idx >> 5;
         const float wt = w[t];
-        s0 = fmaf(wt, v[idx], s0);
-        s1 = fmaf(wt, v[pl.plane + idx], s1);
-        s2 = fmaf(wt, v[2 * pl.plane + idx], s2);
+#pragma unroll
+        for (uint32_t c = 0; c < 3; ++c) {
+          s[c] = fmaf(wt, va[c * pl.plane + idx], s[c]);
+          s[3 + c] = fmaf(wt, vb[c * pl.plane + idx], s[3 + c]);
+        }
       }
-      const uint64_t o = static_cast<uint64_t>(k0 + q) * C + X;
-      out[o] = to_out<OutT>(fmaf(s0, p.mul[0], p.add[0]));
-      out[o + static_cast<uint64_t>(C) * C] = to_out<OutT>(fmaf(s1, p.mul[1], p.add[1]));
-      out[o + 2ull * C * C] = to_out<OutT>(fmaf(s2, p.mul[2], p.add[2]));
+      const uint64_t o = static_cast<uint64_t>(k0 + 2 * r) * C + X;
+#pragma unroll
+      for (uint32_t c = 0; c < 3; ++c) {
+        const uint64_t oc = o + static_cast<uint64_t>(c) * C * C;
+        out[oc] = to_out<OutT>(fmaf(s[c], p.mul[c], p.add[c]));
+        if (has_b) out[oc + C] = to_out<OutT>(fmaf(s[3 + c], p.mul[c], p.add[c]));
+      }
     }
     __syncthreads();
   }
@@ -348,14 +420,10 @@ extern "C" int preba_preprocess_antialias(const preba_batch_t* batch, const preb
     g_last_cuda_error = static_cast<int>(err);
     return PREBA_ERR_CUDA;
   }
-  // rows per CTA: as many as kMaxRows while the batch still gives every SM a few CTAs
-  uint32_t rows = kMaxRows;
-  while (rows > 1 && static_cast<uint64_t>(batch->n) * ((C + rows - 1) / rows) < 4ull * sms)
-    rows /= 2;
-
   // Shared memory: with the host's copy of the table, what the largest image needs; without
   // it, all a CTA may have (images that need more are reported by the kernel).
   uint32_t floats = static_cast<uint32_t>(limit) / 4u;
+  const uint32_t most_rows = C + 1 < kMaxRows ? (C + 1u) & ~1u : kMaxRows;  // no CTA makes more
   if (batch->table_host) {
     uint32_t most = 0;
     for (uint32_t i = 0; i < batch->n; ++i) {
@@ -369,11 +437,30 @@ extern "C" int preba_preprocess_antialias(const preba_batch_t* batch, const preb
           (opt->crop_origin_host[2 * i] + static_cast<uint64_t>(C) > rh ||
            opt->crop_origin_host[2 * i + 1] + static_cast<uint64_t>(C) > rw))
         return PREBA_ERR_BAD_CROP;
-      const Plan pl = make_plan(make_axis(e.w, rw), make_axis(e.h, rh), C, rows);
+      const Plan pl = make_plan(make_axis(e.w, rw), make_axis(e.h, rh), C, most_rows);
       if (pl.total > most) most = pl.total;
     }
     if (most > floats) return PREBA_ERR_TOO_LARGE;
     floats = most;
+  }
+  // Rows per CTA: the CTAs of one image are cut so that the batch fills a whole number of
+  // rounds of the CTAs the GPU holds at once (a round more than needed would run nearly
+  // empty), with an even number of rows (rows are made in pairs), at most kMaxRows, per CTA.
+  int per_sm = 0;
+  err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel_for(opt->out_dtype),
+                                                      kThreads, floats * 4ull);
+  if (err != cudaSuccess || per_sm < 1) {
+    g_last_cuda_error = static_cast<int>(err);
+    return PREBA_ERR_CUDA;
+  }
+  const uint64_t slots = static_cast<uint64_t>(per_sm) * sms;
+  uint32_t rows = kMaxRows;
+  for (uint64_t rounds = 1;; ++rounds) {
+    const uint64_t per_image = rounds * slots / batch->n;
+    if (per_image == 0) continue;
+    rows = per_image >= C ? 1u : static_cast<uint32_t>((C + per_image - 1) / per_image);
+    rows = (rows + 1u) & ~1u;
+    if (rows <= most_rows) break;
   }
 
   Params p = {};

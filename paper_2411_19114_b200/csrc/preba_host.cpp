@@ -102,7 +102,7 @@ extern "C" const char* preba_strerror(int code) {
     case PREBA_ERR_BAD_TABLE: return "bad image table entry";
     case PREBA_ERR_CUDA: return "CUDA runtime error";
     case PREBA_ERR_TIMEOUT: return "device wait ran out";
-    case PREBA_ERR_TOO_LARGE: return "batch exceeds the library's built-in staging space";
+    case PREBA_ERR_TOO_LARGE: return "batch exceeds the library's built-in staging space, or an image is reduced by more than the kernel can hold";
     case PREBA_ERR_BAD_CROP: return "crop window outside the resized image";
     default: return "unknown preba error code";
   }
