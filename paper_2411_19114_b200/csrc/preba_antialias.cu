@@ -109,7 +109,8 @@ struct Plan {
   uint32_t tx;     // pitch of the horizontal weight table (odd: table reads spread over banks)
   uint32_t tp;     // pitch, in (weight of row a, weight of row b) pairs, of the row-pair tables
   uint32_t plane;  // elements of one channel plane of the vertical pass's result
-  uint32_t off_wx, off_xlo, off_xcnt, off_wp, off_plo, off_pcnt, off_v, total;
+  uint32_t off_wx, off_xlo, off_xcnt, off_wp, off_plo, off_pcnt, off_v, off_ring;
+  uint32_t seg;    // bytes of one slot of the ring of staged input rows
 };
 
 __host__ __device__ inline Plan make_plan(const Axis& ax, const Axis& ay, uint32_t C,
@@ -133,8 +134,22 @@ __host__ __device__ inline Plan make_plan(const Axis& ax, const Axis& ay, uint32
   p.off_plo = at, at += pairs;
   p.off_pcnt = at, at += pairs;
   p.off_v = at, at += 6 * p.plane;
-  p.total = at;
+  at = (at + 3u) & ~3u;  // the ring of staged input rows starts on a 16-byte boundary
+  p.off_ring = at;
+  // a staged row: the needed bytes from a 16-byte boundary of global memory, a multiple of 16
+  p.seg = (3u * px + 32u + 15u) & ~15u;
   return p;
+}
+
+// Slots of the ring that `floats` 4-byte units of shared memory leave room for (each slot: a
+// staged row and its 8-byte barrier).
+__host__ __device__ inline uint32_t ring_slots(const Plan& p, uint32_t floats) {
+  return floats <= p.off_ring ? 0u : (floats - p.off_ring) * 4u / (p.seg + 8u);
+}
+
+// Shared memory (4-byte units) for a ring of `slots` rows.
+__host__ __device__ inline uint64_t plan_floats(const Plan& p, uint64_t slots) {
+  return p.off_ring + (slots * (p.seg + 8ull) + 3ull) / 4ull;
 }
 
 __device__ __forceinline__ void report(int32_t* status, int code) {
@@ -198,18 +213,121 @@ __device__ void tabulate_pairs(const Axis& a, uint32_t first, uint32_t count, ui
   }
 }
 
+// ---- shared-memory barriers and bulk copies (PTX) -------------------------------------------
+
+constexpr uint32_t kSpinLimit = 1u << 20;  // bounded waits: give up, report, leave
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+               : "memory");
+}
+
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+
+// Waits for the phase with the given parity to complete; false if the limit ran out.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  for (uint32_t it = 0; it < kSpinLimit; ++it)
+    if (mbar_try_wait(bar, parity)) return true;
+  return false;
+}
+
+// Global -> shared bulk copy; both addresses and the size are multiples of 16 bytes.
+__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uint32_t bytes,
+                                              uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+      ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+      : "memory");
+}
+
+// Orders earlier shared-memory reads before later asynchronous-copy writes.
+__device__ __forceinline__ void fence_async_shared() {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+// The ring of staged input rows of one CTA.  Row y of the image lives in slot (y - first) % slots
+// from the time thread 0 issues its copy until every row below the next pair's first row is
+// dead; the slot's barrier completes once per use, so use u of a slot is awaited with parity u & 1.
+struct Ring {
+  uint32_t data, bars;  // shared-memory addresses
+  uint32_t slots, seg;
+  uint32_t first;       // image row in use 0 of slot 0
+  uint32_t issued;      // rows below this have been asked for (meaningful in thread 0)
+  uint32_t end;         // one past the last row the CTA needs
+  const uint8_t* image; // first byte of the image
+  const uint8_t* stop;  // end of the last whole 16-byte unit of the pixel buffer
+  uint64_t pitch;       // bytes per image row
+  uint32_t b0, bytes;   // first needed byte of a row and the count of needed bytes
+};
+
+// Thread 0: asks for every row below `limit` that has not been asked for.
+__device__ __forceinline__ void ring_issue(Ring& rg, uint32_t limit) {
+  if (limit > rg.end) limit = rg.end;
+  for (; rg.issued < limit; ++rg.issued) {
+    const uint32_t slot = (rg.issued - rg.first) % rg.slots;
+    const uint8_t* src = rg.image + rg.issued * rg.pitch + rg.b0;
+    const uint32_t skew = static_cast<uint32_t>(reinterpret_cast<uintptr_t>(src)) & 15u;
+    uint32_t bytes = (skew + rg.bytes + 15u) & ~15u;
+    if (bytes > static_cast<uint64_t>(rg.stop - (src - skew)))  // only padding is lost
+      bytes = static_cast<uint32_t>(rg.stop - (src - skew));
+    const uint32_t bar = rg.bars + 8u * slot;
+    mbar_arrive_expect_tx(bar, bytes);
+    bulk_copy_g2s(rg.data + slot * rg.seg, src - skew, bytes, bar);
+  }
+}
+
+// Adds one input row's four bytes per word, weighted for both output rows of the pair.
+__device__ __forceinline__ void accumulate(float (&acc)[kWords][8], const uint32_t (&px)[kWords],
+                                           const float2 w) {
+#pragma unroll
+  for (uint32_t k = 0; k < kWords; ++k) {
+    const float f0 = static_cast<float>(px[k] & 0xffu);
+    const float f1 = static_cast<float>((px[k] >> 8) & 0xffu);
+    const float f2 = static_cast<float>((px[k] >> 16) & 0xffu);
+    const float f3 = static_cast<float>(px[k] >> 24);
+    acc[k][0] = fmaf(w.x, f0, acc[k][0]);
+    acc[k][1] = fmaf(w.x, f1, acc[k][1]);
+    acc[k][2] = fmaf(w.x, f2, acc[k][2]);
+    acc[k][3] = fmaf(w.x, f3, acc[k][3]);
+    acc[k][4] = fmaf(w.y, f0, acc[k][4]);
+    acc[k][5] = fmaf(w.y, f1, acc[k][5]);
+    acc[k][6] = fmaf(w.y, f2, acc[k][6]);
+    acc[k][7] = fmaf(w.y, f3, acc[k][7]);
+  }
+}
+
 template <typename OutT>
 __global__ void __launch_bounds__(kThreads) preba_antialias_kernel(const Params p) {
-  extern __shared__ float smem[];
+  extern __shared__ __align__(16) float smem[];
   const uint32_t tid = threadIdx.x, C = p.C;
   const uint32_t groups = (C + p.rows - 1) / p.rows;
   const uint32_t img = blockIdx.x / groups;
   const uint32_t k0 = (blockIdx.x % groups) * p.rows;
   const preba_img_t e = p.table[img];
-  // the entry is checked again here: a bad one is skipped and reported (uniform over the CTA)
+  // The entry is checked again here: a bad one is skipped and reported (uniform over the CTA).
+  // Rows are fetched in 16-byte units, so the buffer counts up to its last whole unit.
+  const uint64_t usable = p.pixels_bytes & ~15ull;
   if (e.h < 1 || e.w < 1 || e.h > PREBA_MAX_DIM || e.w > PREBA_MAX_DIM ||
-      e.offset % PREBA_PACK_ALIGN != 0 || e.offset > p.pixels_bytes ||
-      3ull * e.h * e.w > p.pixels_bytes - e.offset) {
+      e.offset % PREBA_PACK_ALIGN != 0 || e.offset > usable ||
+      3ull * e.h * e.w > usable - e.offset) {
     if (tid == 0) report(p.status, PREBA_ERR_BAD_TABLE);
     return;
   }
@@ -228,21 +346,36 @@ __global__ void __launch_bounds__(kThreads) preba_antialias_kernel(const Params 
   }
   const Axis ax = make_axis(e.w, rw), ay = make_axis(e.h, rh);
   const Plan pl = make_plan(ax, ay, C, p.rows);
-  if (pl.total > p.smem_floats) {
+  if (pl.off_ring > p.smem_floats) {
     if (tid == 0) report(p.status, PREBA_ERR_TOO_LARGE);
     return;
   }
+  // Input rows are staged in shared memory by bulk copies when a ring that holds the rows of
+  // one pair of output rows fits; images reduced by more are read from global memory directly.
+  const uint32_t slots = ring_slots(pl, p.smem_floats);
+  const bool staged = slots >= pl.tp;
   const uint32_t rows_here = C - k0 < p.rows ? C - k0 : p.rows;
+  const uint32_t pairs_here = (rows_here + 1) / 2;
   float* wx = smem + pl.off_wx;
   uint32_t* xlo = reinterpret_cast<uint32_t*>(smem + pl.off_xlo);
   uint32_t* xcnt = reinterpret_cast<uint32_t*>(smem + pl.off_xcnt);
   float2* wp = reinterpret_cast<float2*>(smem + pl.off_wp);
   uint32_t* plo = reinterpret_cast<uint32_t*>(smem + pl.off_plo);
   uint32_t* pcnt = reinterpret_cast<uint32_t*>(smem + pl.off_pcnt);
-  float* va = smem + pl.off_v;       // three planes of row a, then three of row b
+  float* va = smem + pl.off_v;  // three planes of row a, then three of row b
   float* vb = va + 3 * pl.plane;
+  const uint8_t* ring = reinterpret_cast<const uint8_t*>(smem + pl.off_ring);
+  Ring rg;
+  rg.data = smem_addr(ring);
+  rg.bars = rg.data + slots * pl.seg;
+  rg.slots = slots;
+  rg.seg = pl.seg;
   tabulate(ax, left, C, pl.tx, wx, xlo, xcnt);
   tabulate_pairs(ay, top + k0, rows_here, pl.tp, wp, plo, pcnt);
+  if (tid == 0 && staged) {
+    for (uint32_t s = 0; s < slots; ++s) mbar_init(rg.bars + 8u * s, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
   __syncthreads();
 
   // the byte range of a row that the window's taps cover, from a 4-byte boundary of the row
@@ -252,58 +385,83 @@ __global__ void __launch_bounds__(kThreads) preba_antialias_kernel(const Params 
   const uint32_t p0 = b0 / 3u;  // the pixel that element 0 of a plane stands for
   {
     const uint32_t last = (b0 + 4u * nwords - 1u) / 3u - p0;
-    if (last + (last >> 5) >= pl.plane) {  // cannot happen within the plan's bounds
+    // cannot happen within the plan's bounds
+    if (last + (last >> 5) >= pl.plane ||
+        (staged && ((15u + 4u * nwords + 15u) & ~15u) > pl.seg)) {
       if (tid == 0) report(p.status, PREBA_ERR_TOO_LARGE);
       return;
     }
   }
-  const uint64_t pitch = 3ull * e.w;
-  const uint32_t* words = reinterpret_cast<const uint32_t*>(p.pixels);
+  rg.image = p.pixels + e.offset;
+  rg.stop = p.pixels + usable;
+  rg.pitch = 3ull * e.w;
+  rg.b0 = b0;
+  rg.bytes = 4u * nwords;
+  rg.first = plo[0];
+  rg.issued = rg.first;
+  rg.end = plo[pairs_here - 1] + pcnt[pairs_here - 1];
+  if (tid == 0 && staged) ring_issue(rg, rg.first + slots);
   OutT* out = static_cast<OutT*>(p.out) + static_cast<uint64_t>(img) * 3u * C * C;
+  bool failed = false;
 
-  for (uint32_t r = 0; 2 * r < rows_here; ++r) {
-    // ---- vertical pass: both rows of the pair from one sweep over the input rows ----
+  for (uint32_t r = 0; r < pairs_here; ++r) {
+    // ---- vertical pass: both rows of the pair from one sweep over the staged input rows ----
     const uint32_t y0 = plo[r], ny = pcnt[r];
     const float2* wq = wp + r * pl.tp;
+    const uint32_t slot0 = staged ? (y0 - rg.first) % slots : 0u;
+    const uint32_t use0 = staged ? (y0 - rg.first) / slots : 0u;
     for (uint32_t w0 = tid; w0 < nwords; w0 += kThreads * kWords) {
       float acc[kWords][8];
 #pragma unroll
       for (uint32_t k = 0; k < kWords; ++k)
 #pragma unroll
         for (uint32_t t = 0; t < 8; ++t) acc[k][t] = 0.f;
-      uint64_t at0 = e.offset + y0 * pitch + b0 + 4ull * w0;  // first byte of the first word
+      if (staged) {
+        uint32_t slot = slot0, use = use0;
+        uint32_t skew = static_cast<uint32_t>(
+            reinterpret_cast<uintptr_t>(rg.image + y0 * rg.pitch + b0));  // low bits are used
+        const uint32_t step = static_cast<uint32_t>(rg.pitch);
 #pragma unroll 2
-      for (uint32_t i = 0; i < ny; ++i, at0 += pitch) {
-        const float2 w = wq[i];
-        const uint32_t m = static_cast<uint32_t>(at0) & 3u;  // the same for every thread
-        uint32_t px[kWords];
+        for (uint32_t i = 0; i < ny; ++i, skew += step) {
+          if (!failed) failed = !mbar_wait(rg.bars + 8u * slot, use & 1u);
+          const float2 w = wq[i];
+          const uint32_t m = skew & 3u;  // the same for every thread
+          const uint32_t* src =
+              reinterpret_cast<const uint32_t*>(ring + slot * pl.seg + (skew & 12u)) + w0;
+          uint32_t px[kWords];
 #pragma unroll
-        for (uint32_t k = 0; k < kWords; ++k) {
-          px[k] = 0u;
-          if (w0 + k * kThreads < nwords) {
-            const uint64_t aligned = at0 + 4ull * k * kThreads - m;
-            if (aligned + 4 <= p.pixels_bytes) px[k] = __ldg(words + aligned / 4);
-            if (m) {
-              const uint32_t hi =
-                  aligned + 8 <= p.pixels_bytes ? __ldg(words + aligned / 4 + 1) : 0u;
-              px[k] = __funnelshift_r(px[k], hi, 8u * m);
+          for (uint32_t k = 0; k < kWords; ++k) {
+            px[k] = 0u;
+            if (!failed && w0 + k * kThreads < nwords) {
+              px[k] = src[k * kThreads];
+              if (m) px[k] = __funnelshift_r(px[k], src[k * kThreads + 1], 8u * m);
             }
           }
+          accumulate(acc, px, w);
+          if (++slot == slots) slot = 0, ++use;
         }
+      } else {
+        const uint32_t* words = reinterpret_cast<const uint32_t*>(p.pixels);
+        uint64_t at0 = e.offset + y0 * rg.pitch + b0 + 4ull * w0;  // first byte of the first word
+#pragma unroll 2
+        for (uint32_t i = 0; i < ny; ++i, at0 += rg.pitch) {
+          const float2 w = wq[i];
+          const uint32_t m = static_cast<uint32_t>(at0) & 3u;  // the same for every thread
+          uint32_t px[kWords];
 #pragma unroll
-        for (uint32_t k = 0; k < kWords; ++k) {
-          const float f0 = static_cast<float>(px[k] & 0xffu);
-          const float f1 = static_cast<float>((px[k] >> 8) & 0xffu);
-          const float f2 = static_cast<float>((px[k] >> 16) & 0xffu);
-          const float f3 = static_cast<float>(px[k] >> 24);
-          acc[k][0] = fmaf(w.x, f0, acc[k][0]);
-          acc[k][1] = fmaf(w.x, f1, acc[k][1]);
-          acc[k][2] = fmaf(w.x, f2, acc[k][2]);
-          acc[k][3] = fmaf(w.x, f3, acc[k][3]);
-          acc[k][4] = fmaf(w.y, f0, acc[k][4]);
-          acc[k][5] = fmaf(w.y, f1, acc[k][5]);
-          acc[k][6] = fmaf(w.y, f2, acc[k][6]);
-          acc[k][7] = fmaf(w.y, f3, acc[k][7]);
+          for (uint32_t k = 0; k < kWords; ++k) {
+            px[k] = 0u;
+            if (w0 + k * kThreads < nwords) {
+              const uint64_t aligned = at0 + 4ull * k * kThreads - m;
+              if (aligned + 4 <= p.pixels_bytes) px[k] = __ldg(words + aligned / 4);
+              if (m) {
+                const uint32_t hi =
+                    aligned + 8 <= p.pixels_bytes ? __ldg(words + aligned / 4 + 1) : 0u;
+                px[k] = __funnelshift_r(px[k], hi, 8u * m);
+              }
+            }
+          }
+          accumulate(acc, px, w);
         }
       }
 #pragma unroll
@@ -320,7 +478,14 @@ __global__ void __launch_bounds__(kThreads) preba_antialias_kernel(const Params 
         }
       }
     }
-    __syncthreads();
+    failed = __syncthreads_or(failed) != 0;  // from here on the same in every thread
+    if (failed) break;
+    // every row below the next pair's first row is dead: its slot takes a new row, which
+    // arrives while the horizontal pass runs
+    if (tid == 0 && staged && r + 1 < pairs_here) {
+      fence_async_shared();
+      ring_issue(rg, plo[r + 1] + slots);
+    }
     // ---- horizontal pass, normalisation, store ----
     const bool has_b = 2 * r + 1 < rows_here;
     for (uint32_t X = tid; X < C; X += kThreads) {
@@ -346,6 +511,15 @@ __global__ void __launch_bounds__(kThreads) preba_antialias_kernel(const Params 
       }
     }
     __syncthreads();
+  }
+
+  if (failed && tid == 0) {
+    report(p.status, PREBA_ERR_TIMEOUT);
+    // copies already asked for may still be landing in the ring: wait for them (bounded)
+    // before the CTA retires
+    const uint32_t from = rg.issued - rg.first > slots ? rg.issued - slots : rg.first;
+    for (uint32_t y = from; y < rg.issued; ++y)
+      (void)mbar_wait(rg.bars + 8u * ((y - rg.first) % slots), ((y - rg.first) / slots) & 1u);
   }
 }
 
@@ -422,10 +596,11 @@ extern "C" int preba_preprocess_antialias(const preba_batch_t* batch, const preb
   }
   // Shared memory: with the host's copy of the table, what the largest image needs; without
   // it, all a CTA may have (images that need more are reported by the kernel).
-  uint32_t floats = static_cast<uint32_t>(limit) / 4u;
+  const uint32_t limit_floats = static_cast<uint32_t>(limit) / 4u;
+  uint32_t floats = limit_floats;
   const uint32_t most_rows = C + 1 < kMaxRows ? (C + 1u) & ~1u : kMaxRows;  // no CTA makes more
   if (batch->table_host) {
-    uint32_t most = 0;
+    uint64_t most = 0;
     for (uint32_t i = 0; i < batch->n; ++i) {
       const preba_img_t& e = batch->table_host[i];
       if (!dims_ok(e.h, e.w) || e.offset % PREBA_PACK_ALIGN || e.offset > batch->pixels_bytes ||
@@ -438,10 +613,14 @@ extern "C" int preba_preprocess_antialias(const preba_batch_t* batch, const preb
            opt->crop_origin_host[2 * i + 1] + static_cast<uint64_t>(C) > rw))
         return PREBA_ERR_BAD_CROP;
       const Plan pl = make_plan(make_axis(e.w, rw), make_axis(e.h, rh), C, most_rows);
-      if (pl.total > most) most = pl.total;
+      if (pl.off_ring > limit_floats) return PREBA_ERR_TOO_LARGE;
+      // with a ring of staged rows (one pair's rows and half as many again in flight) when
+      // at least the pair's rows fit, else without
+      uint64_t want = pl.off_ring;
+      if (plan_floats(pl, pl.tp) <= limit_floats) want = plan_floats(pl, pl.tp + pl.tp / 2 + 2);
+      if (want > most) most = want;
     }
-    if (most > floats) return PREBA_ERR_TOO_LARGE;
-    floats = most;
+    if (most < floats) floats = static_cast<uint32_t>(most);
   }
   // Rows per CTA: the CTAs of one image are cut so that the batch fills a whole number of
   // rounds of the CTAs the GPU holds at once (a round more than needed would run nearly
