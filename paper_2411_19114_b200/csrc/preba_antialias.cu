@@ -65,6 +65,12 @@ __host__ __device__ inline Axis make_axis(uint32_t n_in, uint32_t R) {
   return a;
 }
 
+// Whether the un-normalised weights fit 16 bits and a row's weighted byte sum 32 bits, so that
+// the vertical pass can run on integer dot products.
+__host__ __device__ inline bool integer_weights_fit(const Axis& a) {
+  return 2ull * a.M <= 65535ull && 255ull * a.taps * 2ull * a.M < (1ull << 32);
+}
+
 __host__ __device__ inline int64_t floor_div(int64_t a, int64_t b) {  // b > 0
   const int64_t q = a / b;
   return (a % b != 0 && a < 0) ? q - 1 : q;
@@ -109,7 +115,8 @@ struct Plan {
   uint32_t tx;     // pitch of the horizontal weight table (odd: table reads spread over banks)
   uint32_t tp;     // pitch, in (weight of row a, weight of row b) pairs, of the row-pair tables
   uint32_t plane;  // elements of one channel plane of the vertical pass's result
-  uint32_t off_wx, off_xlo, off_xcnt, off_wp, off_plo, off_pcnt, off_v, off_ring;
+  uint32_t ti;     // pitch of the integer row-pair tables: an entry per two input rows
+  uint32_t off_wx, off_xlo, off_xcnt, off_wp, off_wi, off_inv, off_plo, off_pcnt, off_v, off_ring;
   uint32_t seg;    // bytes of one slot of the ring of staged input rows
 };
 
@@ -131,6 +138,9 @@ __host__ __device__ inline Plan make_plan(const Axis& ax, const Axis& ay, uint32
   p.off_xcnt = at, at += C;
   at += at & 1u;  // the pair table is read 8 bytes at a time
   p.off_wp = at, at += pairs * p.tp * 2;
+  p.ti = (p.tp + 1u) / 2u;
+  p.off_wi = at, at += pairs * p.ti * 2;
+  p.off_inv = at, at += pairs * 2;
   p.off_plo = at, at += pairs;
   p.off_pcnt = at, at += pairs;
   p.off_v = at, at += 6 * p.plane;
@@ -187,8 +197,12 @@ __device__ void tabulate(const Axis& a, uint32_t first, uint32_t count, uint32_t
 // Vertical tables: pair r covers resized rows first + 2r (a) and first + 2r + 1 (b, if below
 // `count`); entry i of its table holds both rows' normalised weights of input row lo[r] + i
 // (zero where a row does not reach), over the union of the two rows' taps.
+// With `wi`: entry i / 2 of the pair's integer table packs the un-normalised 16-bit weights of
+// input rows lo[r] + i (low half) and lo[r] + i + 1 (high half), .x for row a and .y for row b,
+// and inv[r] holds the reciprocals of the two rows' weight sums.
 __device__ void tabulate_pairs(const Axis& a, uint32_t first, uint32_t count, uint32_t pitch,
-                               float2* w, uint32_t* lo, uint32_t* cnt) {
+                               float2* w, uint32_t* lo, uint32_t* cnt, uint32_t ipitch, uint2* wi,
+                               float2* inv) {
   for (uint32_t r = threadIdx.x; 2 * r < count; r += kThreads) {
     const uint32_t ya = first + 2 * r;
     const bool has_b = 2 * r + 1 < count;
@@ -208,6 +222,18 @@ __device__ void tabulate_pairs(const Axis& a, uint32_t first, uint32_t count, ui
       w[r * pitch + (j - j0)] =
           make_float2(static_cast<float>(tap_weight(a, ya, j)) * inv_a,
                       has_b ? static_cast<float>(tap_weight(a, ya + 1, j)) * inv_b : 0.f);
+    if (wi) {
+      for (uint32_t j = j0; j < j1; j += 2) {
+        const bool two = j + 1 < j1;
+        const uint32_t a_lo = static_cast<uint32_t>(tap_weight(a, ya, j));
+        const uint32_t a_hi = two ? static_cast<uint32_t>(tap_weight(a, ya, j + 1)) : 0u;
+        const uint32_t b_lo = has_b ? static_cast<uint32_t>(tap_weight(a, ya + 1, j)) : 0u;
+        const uint32_t b_hi =
+            has_b && two ? static_cast<uint32_t>(tap_weight(a, ya + 1, j + 1)) : 0u;
+        wi[r * ipitch + (j - j0) / 2] = make_uint2(a_lo | (a_hi << 16), b_lo | (b_hi << 16));
+      }
+      inv[r] = make_float2(inv_a, inv_b);
+    }
     lo[r] = j0;
     cnt[r] = j1 - j0;
   }
@@ -350,10 +376,11 @@ __global__ void __launch_bounds__(kThreads) preba_antialias_kernel(const Params 
     if (tid == 0) report(p.status, PREBA_ERR_TOO_LARGE);
     return;
   }
-  // Input rows are staged in shared memory by bulk copies when a ring that holds the rows of
-  // one pair of output rows fits; images reduced by more are read from global memory directly.
+  // Input rows are staged in shared memory by bulk copies, and summed by integer dot products,
+  // when a ring that holds the rows of one pair of output rows fits and the integer weights are
+  // narrow enough; other images are read from global memory directly and summed in fp32.
   const uint32_t slots = ring_slots(pl, p.smem_floats);
-  const bool staged = slots >= pl.tp;
+  const bool staged = slots >= pl.tp && integer_weights_fit(ay);
   const uint32_t rows_here = C - k0 < p.rows ? C - k0 : p.rows;
   const uint32_t pairs_here = (rows_here + 1) / 2;
   float* wx = smem + pl.off_wx;
@@ -371,7 +398,9 @@ __global__ void __launch_bounds__(kThreads) preba_antialias_kernel(const Params 
   rg.slots = slots;
   rg.seg = pl.seg;
   tabulate(ax, left, C, pl.tx, wx, xlo, xcnt);
-  tabulate_pairs(ay, top + k0, rows_here, pl.tp, wp, plo, pcnt);
+  uint2* wi = reinterpret_cast<uint2*>(smem + pl.off_wi);
+  float2* inv = reinterpret_cast<float2*>(smem + pl.off_inv);
+  tabulate_pairs(ay, top + k0, rows_here, pl.tp, wp, plo, pcnt, pl.ti, staged ? wi : nullptr, inv);
   if (tid == 0 && staged) {
     for (uint32_t s = 0; s < slots; ++s) mbar_init(rg.bars + 8u * s, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -417,29 +446,62 @@ __global__ void __launch_bounds__(kThreads) preba_antialias_kernel(const Params 
 #pragma unroll
         for (uint32_t t = 0; t < 8; ++t) acc[k][t] = 0.f;
       if (staged) {
+        // two input rows per step: their bytes are interleaved so that one two-way dot product
+        // adds both rows' contributions to a byte position (16-bit weights, 32-bit sums, exact)
+        uint32_t sum[kWords][8];
+#pragma unroll
+        for (uint32_t k = 0; k < kWords; ++k)
+#pragma unroll
+          for (uint32_t t = 0; t < 8; ++t) sum[k][t] = 0u;
+        const uint2* wq2 = wi + r * pl.ti;
         uint32_t slot = slot0, use = use0;
         uint32_t skew = static_cast<uint32_t>(
             reinterpret_cast<uintptr_t>(rg.image + y0 * rg.pitch + b0));  // low bits are used
         const uint32_t step = static_cast<uint32_t>(rg.pitch);
-#pragma unroll 2
-        for (uint32_t i = 0; i < ny; ++i, skew += step) {
+        for (uint32_t i = 0; i < ny; i += 2) {
+          // the second row of the last step of an odd count has weight zero: its slot is read
+          // (whatever it holds) but not waited for
+          uint32_t slot1 = slot + 1, use1 = use;
+          if (slot1 == slots) slot1 = 0, ++use1;
           if (!failed) failed = !mbar_wait(rg.bars + 8u * slot, use & 1u);
-          const float2 w = wq[i];
-          const uint32_t m = skew & 3u;  // the same for every thread
-          const uint32_t* src =
+          if (!failed && i + 1 < ny) failed = !mbar_wait(rg.bars + 8u * slot1, use1 & 1u);
+          const uint2 w = wq2[i / 2];
+          const uint32_t skew1 = skew + step;
+          const uint32_t m0 = skew & 3u, m1 = skew1 & 3u;  // the same for every thread
+          const uint32_t* src0 =
               reinterpret_cast<const uint32_t*>(ring + slot * pl.seg + (skew & 12u)) + w0;
-          uint32_t px[kWords];
+          const uint32_t* src1 =
+              reinterpret_cast<const uint32_t*>(ring + slot1 * pl.seg + (skew1 & 12u)) + w0;
 #pragma unroll
           for (uint32_t k = 0; k < kWords; ++k) {
-            px[k] = 0u;
             if (!failed && w0 + k * kThreads < nwords) {
-              px[k] = src[k * kThreads];
-              if (m) px[k] = __funnelshift_r(px[k], src[k * kThreads + 1], 8u * m);
+              uint32_t q0 = src0[k * kThreads], q1 = src1[k * kThreads];
+              if (m0) q0 = __funnelshift_r(q0, src0[k * kThreads + 1], 8u * m0);
+              if (m1) q1 = __funnelshift_r(q1, src1[k * kThreads + 1], 8u * m1);
+              const uint32_t lo = __byte_perm(q0, q1, 0x5140);  // bytes 0 and 1 of both rows
+              const uint32_t hi = __byte_perm(q0, q1, 0x7362);  // bytes 2 and 3 of both rows
+              sum[k][0] = __dp2a_lo(w.x, lo, sum[k][0]);
+              sum[k][1] = __dp2a_hi(w.x, lo, sum[k][1]);
+              sum[k][2] = __dp2a_lo(w.x, hi, sum[k][2]);
+              sum[k][3] = __dp2a_hi(w.x, hi, sum[k][3]);
+              sum[k][4] = __dp2a_lo(w.y, lo, sum[k][4]);
+              sum[k][5] = __dp2a_hi(w.y, lo, sum[k][5]);
+              sum[k][6] = __dp2a_lo(w.y, hi, sum[k][6]);
+              sum[k][7] = __dp2a_hi(w.y, hi, sum[k][7]);
             }
           }
-          accumulate(acc, px, w);
-          if (++slot == slots) slot = 0, ++use;
+          slot = slot1 + 1, use = use1;
+          if (slot == slots) slot = 0, ++use;
+          skew = skew1 + step;
         }
+        const float2 scale = inv[r];
+#pragma unroll
+        for (uint32_t k = 0; k < kWords; ++k)
+#pragma unroll
+          for (uint32_t t = 0; t < 4; ++t) {
+            acc[k][t] = static_cast<float>(sum[k][t]) * scale.x;
+            acc[k][4 + t] = static_cast<float>(sum[k][4 + t]) * scale.y;
+          }
       } else {
         const uint32_t* words = reinterpret_cast<const uint32_t*>(p.pixels);
         uint64_t at0 = e.offset + y0 * rg.pitch + b0 + 4ull * w0;  // first byte of the first word
