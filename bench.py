@@ -457,6 +457,127 @@ def run_audio(args, local_rank: int) -> None:
     print(json.dumps(line), flush=True)
 
 
+def run_antialias(args, local_rank: int) -> None:
+    """The antialiased Resize variant on the heavy-reduction batch (64 frames of 1080 x 1920 ->
+    224 x 224, fp32): device-resident throughput against the HBM roofline of its footprint,
+    end to end from a pinned packed buffer, and its numpy oracle timed on the host."""
+    import torch
+
+    from oracle import antialias as oaa
+    from paper_2411_19114_b200 import accounting
+    from paper_2411_19114_b200 import binding as pb
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device (the CUDA path has no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    pb.lib()
+    n = args.batch or 64
+    images = wl.hires_1080p(n)
+    packed, table = pb.preba_pack(images)
+    acct = accounting.antialias_batch_bytes(table, wl.OUT_SIZE, wl.RESIZE_SHORT, 4)
+    steps, warm = min(args.steps, 500), max(args.warmup, 3)
+    l2 = torch.cuda.get_device_properties(dev).L2_cache_size
+    sets = 2 if acct["total"] > 2 * l2 else max(2, min(16, -(-4 * l2 // acct["total"])))
+    pix = [torch.from_numpy(packed).to(dev) for _ in range(sets)]
+    outs = [torch.empty((n, 3, wl.OUT_SIZE, wl.OUT_SIZE), dtype=torch.float32, device=dev)
+            for _ in range(sets)]
+    tab = torch.from_numpy(table.view(np.uint8)).to(dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    stream = torch.cuda.current_stream()
+    calls = [pb.PreparedPreprocessEx(pix[i], tab, n, outs[i], wl.OUT_SIZE, wl.RESIZE_SHORT, wl.MEAN, wl.STD,
+                                     pb.F32, stream=stream, table_host=table, status=status,
+                                     entry="preba_preprocess_antialias") for i in range(sets)]
+    for i in range(warm):
+        calls[i % sets]()
+    torch.cuda.synchronize()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local_rank) as clocks:
+        torch.cuda.synchronize()
+        start.record(stream)
+        for i in range(steps):
+            calls[i % sets]()
+        stop.record(stream)
+        torch.cuda.synchronize()
+    ms = start.elapsed_time(stop)
+    if int(status.item()) != 0:
+        raise SystemExit(f"bench.py: kernel status {int(status.item())}")
+    per_launch_s = ms * 1e-3 / steps
+    # the plain transform on the same batch, for scale
+    plain = pb.PreparedPreprocess(pix[0], tab, n, outs[0], wl.OUT_SIZE, wl.RESIZE_SHORT, wl.MEAN, wl.STD,
+                                  pb.F32, stream=stream, table_host=table, status=status)
+    for _ in range(3):
+        plain()
+    torch.cuda.synchronize()
+    start.record(stream)
+    for _ in range(200):
+        plain()
+    stop.record(stream)
+    torch.cuda.synchronize()
+    plain_us = start.elapsed_time(stop) * 1000.0 / 200
+    # end to end: pinned packed pixels -> device, kernel, result -> pinned memory
+    e2e_steps = max(3, min(args.e2e_steps, 10))
+    ph = torch.from_numpy(packed).pin_memory()
+    oh = torch.empty((n, 3, wl.OUT_SIZE, wl.OUT_SIZE), dtype=torch.float32).pin_memory()
+
+    def e2e_step():
+        pix[0].copy_(ph, non_blocking=True)
+        calls[0]()
+        oh.copy_(outs[0], non_blocking=True)
+
+    e2e_step()
+    torch.cuda.synchronize()
+    start.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    stop.record(stream)
+    torch.cuda.synchronize()
+    e2e_ms = start.elapsed_time(stop)
+    # parity on the spot: the first image of the last set against the oracle
+    want = oaa.preprocess(images[:1], wl.OUT_SIZE, wl.RESIZE_SHORT, wl.MEAN, wl.STD)[0]
+    err = float(np.max(np.abs(outs[0][0].cpu().numpy() - want)))
+    if err > 1e-5:
+        raise SystemExit(f"bench.py: antialiased output differs from the oracle by {err:.3g}")
+    # the oracle as it stands (numpy), on a sample of the batch
+    t_end, done, spent = time.perf_counter() + args.cpu_budget, 0, 0.0
+    while done < n and (done == 0 or time.perf_counter() < t_end):
+        t0 = time.perf_counter()
+        oaa.preprocess(images[done:done + 1], wl.OUT_SIZE, wl.RESIZE_SHORT, wl.MEAN, wl.STD)
+        spent += time.perf_counter() - t0
+        done += 1
+    peak, peak_source = measured_peak()
+    achieved = acct["total"] / per_launch_s / 1e9
+    line = {
+        "metric": "preprocessed images/sec (antialiased Resize)", "value": n / per_launch_s,
+        "unit": "images/s", "n_gpus": 1, "steps": steps, "warmup": warm,
+        "ms_per_step": ms / steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"{n} frames of 1080 x 1920, smooth noise, antialiased resize to "
+                               "256 on the shorter side (triangle filter, reduction 4.2), centre "
+                               "crop 224, fp32 out",
+                   "resize_short": wl.RESIZE_SHORT, "out_size": wl.OUT_SIZE, "images_per_step_per_gpu": n,
+                   "launch": "one kernel per step, one stream",
+                   "l2": f"{sets} buffer sets of {acct['total'] / 1e6:.0f} MB touched each > L2 "
+                         f"({l2 / 1e6:.0f} MB)"},
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "traffic": None, "peak_source": peak_source,
+                     "algorithmic_bytes_per_launch": acct["total"],
+                     "input_bytes": acct["input_bytes"], "output_bytes": acct["output_bytes"],
+                     "kernel_us": per_launch_s * 1e6},
+        "cpu_baseline": {"value": done / spent, "unit": "images/s", "cores": cpu_threads(),
+                         "kind": "oracle",
+                         "sample": f"{done} of the {n} images, one pass (numpy, its BLAS threads)"},
+        "e2e": {"value": n * e2e_steps / (e2e_ms * 1e-3), "unit": "images/s",
+                "h2d_bytes_per_step": int(packed.nbytes), "d2h_bytes_per_step": int(oh.numel() * 4),
+                "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps,
+                "includes": "packed pixels pinned -> device (whole frames), kernel, result -> "
+                            "pinned memory; one stream"},
+        "plain_transform_us": plain_us, "max_abs_err_vs_oracle": err,
+        "gpu_launches": steps, "clocks": clocks.summary(),
+    }
+    print(json.dumps(line), flush=True)
+
+
 def report_variant(args, rank, world, n, elapsed_ms, acct, desc, dtype, sets, step_bytes, l2,
                    clocks, dist, dev, t_host) -> None:
     """The JSON line of a --variant run: the device-resident leg only."""
@@ -794,7 +915,7 @@ def main() -> None:
     ap.add_argument("--warmup", type=int, default=200)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="mixed",
-                    choices=["mixed", "320x240", "1080p", "sweep", "streams", "audio"])
+                    choices=["mixed", "320x240", "1080p", "sweep", "streams", "audio", "antialias"])
     ap.add_argument("--batch", type=int, default=None)
     ap.add_argument("--variant", default="plain", choices=["plain", "u8", "round"],
                     help="device-resident leg through preba_preprocess_ex: u8 = rounded uint8 "
@@ -814,6 +935,9 @@ def main() -> None:
     elif args.workload == "audio":
         if rank == 0:
             run_audio(args, local_rank)
+    elif args.workload == "antialias":
+        if rank == 0:
+            run_antialias(args, local_rank)
     else:
         run_ours(args, rank, world, local_rank)
 

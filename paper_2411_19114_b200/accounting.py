@@ -49,3 +49,28 @@ def batch_bytes(table, c: int, s: int, out_itemsize: int) -> dict:
     a_out = len(table) * 3 * c * c * out_itemsize
     return dict(input_sector_bytes=a_in, input_pixel_bytes=a_px, output_bytes=a_out,
                 total=a_in + a_out)
+
+
+def _support(n_in: int, r: int, first: int, count: int) -> tuple[int, int]:
+    """[lo, hi): input pixels that carry weight in some resized pixel first .. first+count-1 of
+    the antialiased Resize: |(2j+1) r - (2X+1) n_in| < 2 max(n_in, r), inside the image."""
+    m2 = 2 * max(n_in, r)
+    lo_c = (2 * first + 1) * n_in
+    hi_c = (2 * (first + count - 1) + 1) * n_in
+    lo = max(0, (lo_c - m2 - r) // (2 * r) + 1)
+    hi = min(n_in, -(-(hi_c + m2 - r) // (2 * r)))
+    return lo, hi
+
+
+def antialias_batch_bytes(table, c: int, s: int, out_itemsize: int) -> dict:
+    """Bytes one antialiased batch must move through HBM: every byte of the rectangle of
+    input pixels under the centre crop's support, once, plus the dense output."""
+    inp = 0
+    for t in table:
+        h, w = int(t["h"]), int(t["w"])
+        rh, rw = resized(h, w, s)
+        y0, y1 = _support(h, rh, (rh - c) // 2, c)
+        x0, x1 = _support(w, rw, (rw - c) // 2, c)
+        inp += 3 * (y1 - y0) * (x1 - x0)
+    out = len(table) * 3 * c * c * out_itemsize
+    return {"input_bytes": inp, "output_bytes": out, "total": inp + out}

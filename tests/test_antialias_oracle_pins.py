@@ -216,3 +216,23 @@ def test_batch_position_and_origin():
         assert np.array_equal(whole[i], want)
     with pytest.raises(ValueError):
         aa.preprocess(imgs[:1], c, s, MEAN, STD, crop_origin=[(5, 0)])   # 5 + 12 > 16
+
+
+# ---- the benchmark's byte accounting (host logic of the package, checked against the oracle) ------
+
+def test_accounting_counts_the_rectangle_of_weighted_pixels():
+    from paper_2411_19114_b200 import accounting as ac
+
+    table = np.zeros(3, dtype=[("offset", "<u8"), ("h", "<u4"), ("w", "<u4")])
+    sizes = [(1080, 1920), (375, 500), (100, 150)]
+    c, s = 224, 256
+    want_in = 0
+    for t, (h, w) in zip(table, sizes):
+        t["h"], t["w"] = h, w
+        rh, rw = aa.resized_size(h, w, s)
+        rows = np.nonzero(aa.axis_weights(h, rh, (rh - c) // 2, c).sum(axis=0) > 1e-15)[0]
+        cols = np.nonzero(aa.axis_weights(w, rw, (rw - c) // 2, c).sum(axis=0) > 1e-15)[0]
+        want_in += 3 * (rows[-1] - rows[0] + 1) * (cols[-1] - cols[0] + 1)
+    got = ac.antialias_batch_bytes(table, c, s, 4)
+    assert got["input_bytes"] == want_in
+    assert got["output_bytes"] == 3 * 3 * c * c * 4 and got["total"] == want_in + got["output_bytes"]
