@@ -177,6 +177,16 @@ __device__ __forceinline__ __nv_bfloat16 to_out<__nv_bfloat16>(float v) {
   return __float2bfloat16_rn(v);
 }
 
+// Sum of the integer weights of taps j0 .. j1 - 1 of resized pixel X: the distance term moves
+// by 2R from one tap to the next, so one 64-bit product starts the run.
+__device__ __forceinline__ uint64_t weight_sum(const Axis& a, uint32_t X, uint32_t j0, uint32_t j1) {
+  int64_t d = static_cast<int64_t>(2ull * j0 + 1) * a.R - static_cast<int64_t>(2ull * X + 1) * a.n_in;
+  const int64_t two_m = 2ll * a.M, step = 2ll * a.R;
+  uint64_t sum = 0;
+  for (uint32_t j = j0; j < j1; ++j, d += step) sum += static_cast<uint64_t>(two_m - (d < 0 ? -d : d));
+  return sum;
+}
+
 // Horizontal table: row q of `w` (pitch `pitch`) holds the normalised weights of resized
 // pixel first + q from tap lo[q] on.
 __device__ void tabulate(const Axis& a, uint32_t first, uint32_t count, uint32_t pitch, float* w,
@@ -184,11 +194,12 @@ __device__ void tabulate(const Axis& a, uint32_t first, uint32_t count, uint32_t
   for (uint32_t q = threadIdx.x; q < count; q += kThreads) {
     uint32_t j0, j1;
     tap_range(a, first + q, &j0, &j1);
-    uint64_t sum = 0;
-    for (uint32_t j = j0; j < j1; ++j) sum += static_cast<uint32_t>(tap_weight(a, first + q, j));
-    const float inv = 1.0f / static_cast<float>(sum);
-    for (uint32_t j = j0; j < j1; ++j)
-      w[q * pitch + (j - j0)] = static_cast<float>(tap_weight(a, first + q, j)) * inv;
+    const float inv = 1.0f / static_cast<float>(weight_sum(a, first + q, j0, j1));
+    int64_t d = static_cast<int64_t>(2ull * j0 + 1) * a.R -
+                static_cast<int64_t>(2ull * (first + q) + 1) * a.n_in;
+    const int64_t two_m = 2ll * a.M, step = 2ll * a.R;
+    for (uint32_t j = j0; j < j1; ++j, d += step)
+      w[q * pitch + (j - j0)] = static_cast<float>(two_m - (d < 0 ? -d : d)) * inv;
     lo[q] = j0;
     cnt[q] = j1 - j0;
   }
@@ -198,44 +209,46 @@ __device__ void tabulate(const Axis& a, uint32_t first, uint32_t count, uint32_t
 // `count`); entry i of its table holds both rows' normalised weights of input row lo[r] + i
 // (zero where a row does not reach), over the union of the two rows' taps.
 // With `wi`: entry i / 2 of the pair's integer table packs the un-normalised 16-bit weights of
-// input rows lo[r] + i (low half) and lo[r] + i + 1 (high half), .x for row a and .y for row b,
-// and inv[r] holds the reciprocals of the two rows' weight sums.
+// input rows lo[r] + i (low half) and lo[r] + i + 1 (high half), .x for row a and .y for row b.
+// inv[r] holds the reciprocals of the two rows' weight sums.  A thread per pair finds the
+// ranges and the sums; after a barrier a thread per table entry writes the weights.
 __device__ void tabulate_pairs(const Axis& a, uint32_t first, uint32_t count, uint32_t pitch,
                                float2* w, uint32_t* lo, uint32_t* cnt, uint32_t ipitch, uint2* wi,
                                float2* inv) {
-  for (uint32_t r = threadIdx.x; 2 * r < count; r += kThreads) {
+  const uint32_t pairs = (count + 1) / 2;
+  for (uint32_t r = threadIdx.x; r < pairs; r += kThreads) {
     const uint32_t ya = first + 2 * r;
     const bool has_b = 2 * r + 1 < count;
     uint32_t a0, a1, b0, b1;
     tap_range(a, ya, &a0, &a1);
     b0 = a0, b1 = a1;
     if (has_b) tap_range(a, ya + 1, &b0, &b1);
-    const uint32_t j0 = a0, j1 = a1 > b1 ? a1 : b1;  // first taps do not decrease with the row
-    uint64_t sum_a = 0, sum_b = 0;
-    for (uint32_t j = j0; j < j1; ++j) {
-      sum_a += static_cast<uint32_t>(tap_weight(a, ya, j));
-      if (has_b) sum_b += static_cast<uint32_t>(tap_weight(a, ya + 1, j));
-    }
-    const float inv_a = 1.0f / static_cast<float>(sum_a);
-    const float inv_b = has_b ? 1.0f / static_cast<float>(sum_b) : 0.f;
-    for (uint32_t j = j0; j < j1; ++j)
-      w[r * pitch + (j - j0)] =
-          make_float2(static_cast<float>(tap_weight(a, ya, j)) * inv_a,
-                      has_b ? static_cast<float>(tap_weight(a, ya + 1, j)) * inv_b : 0.f);
-    if (wi) {
-      for (uint32_t j = j0; j < j1; j += 2) {
-        const bool two = j + 1 < j1;
-        const uint32_t a_lo = static_cast<uint32_t>(tap_weight(a, ya, j));
-        const uint32_t a_hi = two ? static_cast<uint32_t>(tap_weight(a, ya, j + 1)) : 0u;
-        const uint32_t b_lo = has_b ? static_cast<uint32_t>(tap_weight(a, ya + 1, j)) : 0u;
-        const uint32_t b_hi =
-            has_b && two ? static_cast<uint32_t>(tap_weight(a, ya + 1, j + 1)) : 0u;
-        wi[r * ipitch + (j - j0) / 2] = make_uint2(a_lo | (a_hi << 16), b_lo | (b_hi << 16));
-      }
-      inv[r] = make_float2(inv_a, inv_b);
-    }
-    lo[r] = j0;
-    cnt[r] = j1 - j0;
+    lo[r] = a0;  // first taps do not decrease with the row
+    cnt[r] = (a1 > b1 ? a1 : b1) - a0;
+    inv[r] = make_float2(1.0f / static_cast<float>(weight_sum(a, ya, a0, a1)),
+                         has_b ? 1.0f / static_cast<float>(weight_sum(a, ya + 1, b0, b1)) : 0.f);
+  }
+  __syncthreads();
+  for (uint32_t at = threadIdx.x; at < pairs * pitch; at += kThreads) {
+    const uint32_t r = at / pitch, i = at - r * pitch;
+    if (i >= cnt[r]) continue;
+    const uint32_t ya = first + 2 * r, j = lo[r] + i;
+    const bool has_b = 2 * r + 1 < count;
+    const float2 scale = inv[r];
+    w[at] = make_float2(static_cast<float>(tap_weight(a, ya, j)) * scale.x,
+                        has_b ? static_cast<float>(tap_weight(a, ya + 1, j)) * scale.y : 0.f);
+  }
+  if (!wi) return;
+  for (uint32_t at = threadIdx.x; at < pairs * ipitch; at += kThreads) {
+    const uint32_t r = at / ipitch, i = 2 * (at - r * ipitch);
+    if (i >= cnt[r]) continue;
+    const uint32_t ya = first + 2 * r, j = lo[r] + i;
+    const bool has_b = 2 * r + 1 < count, two = i + 1 < cnt[r];
+    const uint32_t a_lo = static_cast<uint32_t>(tap_weight(a, ya, j));
+    const uint32_t a_hi = two ? static_cast<uint32_t>(tap_weight(a, ya, j + 1)) : 0u;
+    const uint32_t b_lo = has_b ? static_cast<uint32_t>(tap_weight(a, ya + 1, j)) : 0u;
+    const uint32_t b_hi = has_b && two ? static_cast<uint32_t>(tap_weight(a, ya + 1, j + 1)) : 0u;
+    wi[at] = make_uint2(a_lo | (a_hi << 16), b_lo | (b_hi << 16));
   }
 }
 
