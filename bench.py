@@ -40,9 +40,15 @@ NCU_TRAFFIC = {"csrc_sha1": "92be46a6cb22008f113ffa424f83203f814aa897",
                "bytes_per_launch": 75637248 + 25767936}  # dram read + write, one launch
 
 
-def csrc_digest() -> str:
-    """SHA-1 of the source file that holds the fused kernel and its launch code."""
-    path = ROOT / "paper_2411_19114_b200" / "csrc" / "preba_kernels.cu"
+# The same for the antialiased kernel: captured on 32 frames of 1080 x 1920 (traffic grows in
+# proportion to the frames, so a launch over n frames is taken as n / 32 of it).
+AA_NCU_TRAFFIC = {"csrc_sha1": "ec70208c7fbcd001aabcdd3ef84bcaec23248a4f", "frames": 32,
+                  "bytes": 91977216 + 4739840}
+
+
+def csrc_digest(name: str = "preba_kernels.cu") -> str:
+    """SHA-1 of the source file that holds a kernel and its launch code."""
+    path = ROOT / "paper_2411_19114_b200" / "csrc" / name
     return hashlib.sha1(path.read_bytes()).hexdigest()
 
 
@@ -547,6 +553,8 @@ def run_antialias(args, local_rank: int) -> None:
         done += 1
     peak, peak_source = measured_peak()
     achieved = acct["total"] / per_launch_s / 1e9
+    traffic = AA_NCU_TRAFFIC["bytes"] * n // AA_NCU_TRAFFIC["frames"] \
+        if AA_NCU_TRAFFIC["csrc_sha1"] == csrc_digest("preba_antialias.cu") else None
     line = {
         "metric": "preprocessed images/sec (antialiased Resize)", "value": n / per_launch_s,
         "unit": "images/s", "n_gpus": 1, "steps": steps, "warmup": warm,
@@ -560,7 +568,7 @@ def run_antialias(args, local_rank: int) -> None:
                    "l2": f"{sets} buffer sets of {acct['total'] / 1e6:.0f} MB touched each > L2 "
                          f"({l2 / 1e6:.0f} MB)"},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                     "frac": achieved / peak, "traffic": None, "peak_source": peak_source,
+                     "frac": achieved / peak, "traffic": traffic, "peak_source": peak_source,
                      "algorithmic_bytes_per_launch": acct["total"],
                      "input_bytes": acct["input_bytes"], "output_bytes": acct["output_bytes"],
                      "kernel_us": per_launch_s * 1e6},
