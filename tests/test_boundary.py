@@ -229,6 +229,30 @@ def test_extended_entry_point_rejects_bad_arguments_before_any_launch():
     assert pb.preba_strerror(pb.ERR_BAD_CROP) != pb.preba_strerror(-99)
 
 
+def test_antialiased_entry_point_rejects_bad_arguments_before_any_launch():
+    def call(batch=None, **kw):
+        b = batch if batch is not None else _batch(out_bytes=2 * 3 * 16 * 16 * 4)
+        o = pb.PrebaOptions()
+        o.out_size, o.resize_short = 16, 16
+        o.mean = (ctypes.c_float * 3)(*MEAN)
+        o.std = (ctypes.c_float * 3)(*STD)
+        o.out_dtype, o.flags = pb.F32, 0
+        for k, v in kw.items():
+            setattr(o, k, v)
+        return pb.lib().preba_preprocess_antialias(ctypes.byref(b), ctypes.byref(o), None)
+
+    assert pb.lib().preba_preprocess_antialias(None, None, None) == pb.ERR_INVALID_ARG
+    assert call(flags=pb.EX_ROUND_U8) == pb.ERR_INVALID_ARG          # no rounding in this variant
+    assert call(out_dtype=pb.U8) == pb.ERR_INVALID_ARG
+    assert call(out_size=17) == pb.ERR_INVALID_ARG                   # crop larger than the resize
+    assert call(out_size=0) == pb.ERR_INVALID_ARG
+    assert call(resize_short=16384 + 1, out_size=16) == pb.ERR_INVALID_ARG   # PREBA_MAX_RESIZE
+    assert call(crop_origin=0x50002) == pb.ERR_INVALID_ARG           # misaligned table of windows
+    assert call(std=(ctypes.c_float * 3)(0.2, 0.0, 0.2)) == pb.ERR_INVALID_ARG
+    assert call(mean=(ctypes.c_float * 3)(0.2, float("nan"), 0.2)) == pb.ERR_INVALID_ARG
+    assert call(_batch(out_bytes=2 * 3 * 16 * 16 * 4 - 1)) == pb.ERR_BUFFER_TOO_SMALL
+
+
 def test_separate_images_entry_point_rejects_bad_arguments_before_any_copy():
     """preba_preprocess_images validates on the host first: nothing below reaches CUDA."""
     img = np.zeros((8, 8, 3), dtype=np.uint8)
