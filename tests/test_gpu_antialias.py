@@ -112,6 +112,17 @@ def test_degenerate_images():
     assert np.max(np.abs(got - want(images, 4, 4))) <= 1e-5
 
 
+def test_enlargements_whose_integer_weights_pass_16_bits_take_the_fp32_path():
+    """300 x 4 and 4 x 300 at resize_short = 16384: one axis is enlarged to 1,228,800 pixels, so
+    its un-normalised weights need 22 bits; the vertical pass then sums in fp32."""
+    images = [uniform(550, 300, 4), uniform(551, 4, 300), uniform(552, 7, 5)]
+    got = run(images, 8, 16384)
+    assert np.max(np.abs(got - want(images, 8, 16384))) <= 1e-5
+    origins = np.asarray([[1228800 - 8, 16384 - 8], [0, 1228800 - 8], [11, 3]], dtype=np.uint32)
+    got = run(images, 8, 16384, origins=origins)
+    assert np.max(np.abs(got - want(images, 8, 16384, origins))) <= 1e-5
+
+
 def test_small_batches_take_fewer_rows_per_block():
     """One image: the launch splits it into single rows; the result does not depend on it."""
     img = uniform(600, 1080, 1920)
