@@ -34,10 +34,14 @@ METRIC = "preprocessed images/sec"
 UNIT = "images/s"
 FALLBACK_HBM_GBS = 6650.0
 
-# DRAM bytes (read + write) per launch of the kernel on the default workload, from one
-# ncu capture, valid only for the kernel sources with this digest (else reported as null).
-NCU_TRAFFIC = {"csrc_sha1": "92be46a6cb22008f113ffa424f83203f814aa897",
-               "bytes_per_launch": 75637248 + 25767936}  # dram read + write, one launch
+# DRAM bytes (read + write) per launch of the kernel on the default workload in steady state:
+# the sum over consecutive launches of the rotating-buffer loop, captured by ncu in one pass
+# without cache flushes between launches, divided by the launch count (so the write-back of a
+# launch's result, which happens while later launches run, is inside the window).  Valid only
+# for the kernel sources with this digest (else reported as null).
+NCU_TRAFFIC = {"csrc_sha1": "", "bytes_per_launch": 0}
+TRAFFIC_NOTE = ("dram read + write bytes summed over 8 consecutive launches of this loop (one "
+                "ncu pass, caches not flushed between launches) / 8")
 
 
 # The same for the antialiased kernel: captured on 32 frames of 1080 x 1920 (traffic grows in
@@ -113,48 +117,75 @@ class ClockSampler:
         0x100: "display_clock_setting", 0x10: "sync_boost",
     }
 
-    def __init__(self, index: int, period_s: float = 0.01):
+    def __init__(self, index: int, period_s: float = 0.002):
         self.index, self.period = index, period_s
         self.sm, self.bits, self.max_mhz = [], 0, None
         self._stop = threading.Event()
         self._thread = None
+        self._nv = self._dev = None
         self.error = None
 
-    def _run(self):
+    def _open(self):
+        """NVML handle of the GPU (by UUID, so that CUDA_VISIBLE_DEVICES does not mislead)."""
+        import pynvml as nv
+
+        nv.nvmlInit()
+        uuid = None
         try:
-            import pynvml as nv
+            import torch
 
-            nv.nvmlInit()
-            uuid = None
-            try:
-                import torch
+            uuid = "GPU-" + str(torch.cuda.get_device_properties(self.index).uuid)
+        except Exception:
+            pass
+        try:
+            dev = nv.nvmlDeviceGetHandleByUUID(uuid.encode() if uuid else b"")
+        except Exception:
+            dev = nv.nvmlDeviceGetHandleByIndex(self.index)
+        self._nv, self._dev = nv, dev
+        self.max_mhz = int(nv.nvmlDeviceGetMaxClockInfo(dev, nv.NVML_CLOCK_SM))
 
-                uuid = "GPU-" + str(torch.cuda.get_device_properties(self.index).uuid)
-            except Exception:
-                pass
+    def sample(self):
+        """One reading of the SM clock and the reasons word, taken by the caller."""
+        nv, dev = self._nv, self._dev
+        if nv is None:
+            return
+        try:
+            self.sm.append(int(nv.nvmlDeviceGetClockInfo(dev, nv.NVML_CLOCK_SM)))
             try:
-                dev = nv.nvmlDeviceGetHandleByUUID(uuid.encode() if uuid else b"")
+                self.bits |= int(nv.nvmlDeviceGetCurrentClocksEventReasons(dev))
             except Exception:
-                dev = nv.nvmlDeviceGetHandleByIndex(self.index)
-            self.max_mhz = int(nv.nvmlDeviceGetMaxClockInfo(dev, nv.NVML_CLOCK_SM))
-            while not self._stop.is_set():
-                self.sm.append(int(nv.nvmlDeviceGetClockInfo(dev, nv.NVML_CLOCK_SM)))
-                try:
-                    self.bits |= int(nv.nvmlDeviceGetCurrentClocksEventReasons(dev))
-                except Exception:
-                    self.bits |= int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(dev))
-                self._stop.wait(self.period)
-        except Exception as exc:  # NVML missing: report, do not invent numbers
+                self.bits |= int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(dev))
+        except Exception as exc:
             self.error = repr(exc)
 
+    def _run(self):
+        while not self._stop.is_set():
+            self.sample()
+            self._stop.wait(self.period)
+
+    def open(self):
+        """Set NVML up ahead of time (before the warm-up), so that entering the timed region
+        costs nothing and the first sample is immediate."""
+        if self._nv is None and self.error is None:
+            try:
+                self._open()
+            except Exception as exc:  # NVML missing: report, do not invent numbers
+                self.error = repr(exc)
+        return self
+
     def __enter__(self):
-        self._thread = threading.Thread(target=self._run, daemon=True)
-        self._thread.start()
+        self.open()
+        if self._nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
         return self
 
     def __exit__(self, *a):
+        # one reading while the last launches are still in flight or have only just ended
+        self.sample()
         self._stop.set()
-        self._thread.join(timeout=5)
+        if self._thread is not None:
+            self._thread.join(timeout=5)
 
     def summary(self) -> dict:
         if not self.sm:
@@ -194,11 +225,12 @@ def run_reference(args, rank: int, world: int) -> None:
         return
     images, dtype, desc = make_workload(args.workload, args.batch, 0)
     n = len(images)
-    warm, _ = time_oracle(images, dtype, 0.0, max(1, min(args.warmup, 1)))
+    warm, _ = time_oracle(images, dtype, 30.0, max(1, args.warmup))
     times, threads = time_oracle(images, dtype, 60.0, max(1, args.steps))
     total = float(sum(times))
     value = n * len(times) / total
-    sample = f"whole batch of {n} images per step, {len(times)} steps (time budget 60 s)"
+    sample = (f"whole batch of {n} images per step, {len(times)} steps after {len(warm)} warm-up "
+              "steps (time budgets 60 s and 30 s)")
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": len(times), "warmup": len(warm), "ms_per_step": 1e3 * total / len(times),
@@ -283,10 +315,10 @@ def run_streams(args, local_rank: int) -> None:
         "n_gpus": 1, "steps": steps, "warmup": warm, "ms_per_step": elapsed_ms / steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
         "data": "synthetic",
-        "config": dict(config_of(f"{n_streams} concurrent streams x {n} images 500x375, smooth "
-                                 "noise, fp16 out", "f16", n, 1),
-                       launch="7 host threads, one stream each, launch loops inside the library",
-                       l2="inputs and outputs of all streams stay resident (warm L2)"),
+        "config": config_of(f"{n_streams} concurrent streams x {n} images 500x375, smooth "
+                            "noise, fp16 out", "f16", n, 1),
+        "launch": "7 host threads, one stream each, launch loops inside the library",
+        "l2": "inputs and outputs of all streams stay resident (warm L2)",
         "streams": {"count": n_streams,
                     "batch_latency_us": {"p50": float(np.percentile(all_lat, 50)),
                                          "p95": float(np.percentile(all_lat, 95)),
@@ -435,10 +467,10 @@ def run_audio(args, local_rank: int) -> None:
         "config": {"workload": f"{n} synthetic utterances, 1.5-15 s at 16 kHz ({seconds:.0f} s of "
                                f"audio, {frames} frames of 400 samples every 160), 80 log-Mel "
                                "features, per-utterance normalisation, fp32 out",
-                   "utterances_per_step": n, "audio_seconds_per_step": seconds,
-                   "launch": "two kernels per step (spectrogram, normalise), one stream",
-                   "l2": f"rotating {sets} buffer sets ({sets * step_bytes / 1e6:.0f} MB) > L2 "
-                         f"({l2 / 1e6:.0f} MB)"},
+                   "utterances_per_step": n, "audio_seconds_per_step": seconds},
+        "launch": "two kernels per step (spectrogram, normalise), one stream",
+        "l2": f"rotating {sets} buffer sets ({sets * step_bytes / 1e6:.0f} MB) > L2 "
+              f"({l2 / 1e6:.0f} MB)",
         "roofline": {"bound": "alu", "achieved": achieved, "peak": AUDIO_ALU_PEAK_TFLOPS,
                      "unit": "TFLOP/s", "frac": achieved / AUDIO_ALU_PEAK_TFLOPS, "traffic": None,
                      "peak_source": "148 SMs x 128 fp32 lanes x 2 x 1.965 GHz",
@@ -563,10 +595,10 @@ def run_antialias(args, local_rank: int) -> None:
         "config": {"workload": f"{n} frames of 1080 x 1920, smooth noise, antialiased resize to "
                                "256 on the shorter side (triangle filter, reduction 4.2), centre "
                                "crop 224, fp32 out",
-                   "resize_short": wl.RESIZE_SHORT, "out_size": wl.OUT_SIZE, "images_per_step_per_gpu": n,
-                   "launch": "one kernel per step, one stream",
-                   "l2": f"{sets} buffer sets of {acct['total'] / 1e6:.0f} MB touched each > L2 "
-                         f"({l2 / 1e6:.0f} MB)"},
+                   "resize_short": wl.RESIZE_SHORT, "out_size": wl.OUT_SIZE, "images_per_step_per_gpu": n},
+        "launch": "one kernel per step, one stream",
+        "l2": f"{sets} buffer sets of {acct['total'] / 1e6:.0f} MB touched each > L2 "
+              f"({l2 / 1e6:.0f} MB)",
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "traffic": traffic, "peak_source": peak_source,
                      "algorithmic_bytes_per_launch": acct["total"],
@@ -587,7 +619,7 @@ def run_antialias(args, local_rank: int) -> None:
 
 
 def report_variant(args, rank, world, n, elapsed_ms, acct, desc, dtype, sets, step_bytes, l2,
-                   clocks, dist, dev, t_host) -> None:
+                   clocks, dist, dev, t_host, launch_note) -> None:
     """The JSON line of a --variant run: the device-resident leg only."""
     (elapsed_ms,) = max_over_ranks([elapsed_ms], dist, dev)
     if rank == 0:
@@ -600,13 +632,11 @@ def report_variant(args, rank, world, n, elapsed_ms, acct, desc, dtype, sets, st
             "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "int32" if dtype == "u8" else "int32+f32",
             "data": "synthetic",
-            "config": dict(config_of(desc, dtype, n, world),
-                           launch="one stream, back-to-back launches marked independent of "
-                                  "their predecessor (programmatic dependent launch)",
-                           l2=f"rotating {sets} input/output buffer sets "
-                              f"({sets * step_bytes / 1e6:.0f} MB held, "
-                              f"{sets * acct['total'] / 1e6:.0f} MB touched) > L2 "
-                              f"({l2 / 1e6:.0f} MB)"),
+            "config": config_of(desc, dtype, n, world),
+            "launch": launch_note,
+            "l2": f"rotating {sets} input/output buffer sets "
+                  f"({sets * step_bytes / 1e6:.0f} MB held, "
+                  f"{sets * acct['total'] / 1e6:.0f} MB touched) > L2 ({l2 / 1e6:.0f} MB)",
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                          "frac": achieved / peak, "traffic": None, "peak_source": peak_src,
                          "algorithmic_bytes_per_launch": acct["total"],
@@ -654,9 +684,13 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
     l2 = torch.cuda.get_device_properties(dev).L2_cache_size
     step_bytes = packed.nbytes + acct["output_bytes"]
     # enough buffer sets that the bytes a launch touches (the tapped sectors and the result,
-    # which can be far less than the images), summed over the sets, exceed four times L2
+    # which can be far less than the images), summed over the sets, exceed four times L2; and
+    # at least 32 (memory allowing), because the launch that reuses the first set is the one
+    # that is not marked as overlapping (see below)
     sets = max(2, min(64, -(-4 * l2 // min(step_bytes, acct["total"]))))
-    pix = [torch.from_numpy(packed).to(dev) for _ in range(sets)]
+    sets = max(sets, min(32, max(4, (24 << 30) // step_bytes)))
+    pix0 = torch.from_numpy(packed).to(dev)
+    pix = [pix0] + [pix0.clone() for _ in range(sets - 1)]
     out_shape = (n, C, C, 3) if args.variant == "u8" else (n, 3, C, C)
     outs = [torch.empty(out_shape, dtype=tdt, device=dev) for _ in range(sets)]
     tab = torch.from_numpy(table.view(np.uint8)).to(dev)
@@ -665,15 +699,21 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
     stream = torch.cuda.current_stream()
 
     # Timed launches go to one stream, each into the next buffer set and marked independent
-    # of its predecessor, so a launch starts as the previous one's warps retire.
-    if args.variant == "plain":
-        calls = [pb.PreparedPreprocess(pix[i], tab, n, outs[i], C, S, wl.MEAN, wl.STD, out_dtype,
-                                       stream=stream, status=status, flags=pb.OVERLAP_PREVIOUS)
-                 for i in range(sets)]
-    else:
-        calls = [pb.PreparedPreprocessEx(pix[i], tab, n, outs[i], C, S, wl.MEAN, wl.STD,
-                                         out_dtype, round_u8=True, stream=stream, status=status,
-                                         flags=pb.OVERLAP_PREVIOUS) for i in range(sets)]
+    # of the kernels before it, so a launch starts as the previous one's warps retire.  A
+    # marked launch may run beside every kernel back to the last unmarked one, so the launch
+    # into set 0, where the buffers come round again, is not marked: it waits for everything
+    # before it, and no two launches that could overlap ever share a buffer.
+    def prepared(i, flags):
+        if args.variant == "plain":
+            return pb.PreparedPreprocess(pix[i], tab, n, outs[i], C, S, wl.MEAN, wl.STD, out_dtype,
+                                         stream=stream, status=status, flags=flags)
+        return pb.PreparedPreprocessEx(pix[i], tab, n, outs[i], C, S, wl.MEAN, wl.STD, out_dtype,
+                                       round_u8=True, stream=stream, status=status, flags=flags)
+
+    calls = [prepared(i, pb.OVERLAP_PREVIOUS if i else 0) for i in range(sets)]
+    launch_note = (f"one stream, back-to-back launches into {sets} rotating buffer sets; every "
+                   "launch but the one into set 0 is marked independent of the kernels before it "
+                   "(programmatic dependent launch)")
 
     def barrier():
         if dist is not None:
@@ -681,18 +721,21 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
         torch.cuda.synchronize()
 
     # ---- device-resident throughput: one launch per step -------------------------------------
-    for i in range(max(args.warmup, 3)):
+    sampler = ClockSampler(local_rank).open()   # NVML is set up before the warm-up
+    n_warm = max(args.warmup, 3)
+    for i in range(n_warm):
         calls[i % sets]()
     barrier()
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    with ClockSampler(local_rank) as clocks:
+    with sampler as clocks:
         barrier()
         start.record(stream)
         t_host = time.perf_counter()
-        for i in range(args.steps):
+        for i in range(n_warm, n_warm + args.steps):  # the rotation goes on where the warm-up ended
             calls[i % sets]()
         t_host = time.perf_counter() - t_host
         stop.record(stream)
+        clocks.sample()                          # while the last launches are still running
         barrier()
     elapsed_ms = start.elapsed_time(stop)
     assert int(status.item()) == 0, "kernel reported an error status"
@@ -708,13 +751,13 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
     assert all(bool(torch.equal(o, ref)) for o in outs), "overlapped launches changed the result"
     if args.variant != "plain":
         report_variant(args, rank, world, n, elapsed_ms, acct, desc, dtype, sets, step_bytes, l2,
-                       clocks, dist, dev, t_host)
+                       clocks, dist, dev, t_host, launch_note)
         return
 
     # ---- one launch at a time: device time of a launch that runs alone (no overlap flag, so
     # the library cuts a small batch into finer slabs); events around every launch
     alone = pb.PreparedPreprocess(pix[0], tab, n, outs[0], C, S, wl.MEAN, wl.STD, out_dtype,
-                                  stream=stream, status=status)
+                                  stream=stream, status=status, scratch=scratch)
     alone.repeated(20)
     lat_us, _ = alone.repeated(max(50, min(args.steps, 1000)))
     assert bool(torch.equal(outs[0], ref)), "an isolated launch changed the result"
@@ -722,7 +765,7 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
     # ---- the same launch over and over on one buffer set (whatever fits stays in L2) -----------
     warm_steps = max(3, min(args.steps, 2000))
     for _ in range(3):
-        calls[0]()
+        calls[0]()                                  # set 0's call is the unmarked one
     barrier()
     w_start, w_stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     w_start.record(stream)
@@ -851,6 +894,7 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
         traffic = NCU_TRAFFIC["bytes_per_launch"] \
             if NCU_TRAFFIC["csrc_sha1"] == csrc_digest() and args.workload == "mixed" \
             and not args.batch else None
+        iso_p50 = float(np.percentile(lat_us, 50))
         cpu_times, threads = time_oracle(images, dtype, args.cpu_budget, 50)
         cpu_value = n * len(cpu_times) / float(sum(cpu_times))
         one_times, _ = time_oracle(images[:max(1, n // 16)], dtype, args.cpu_budget / 4, 5, threads=1)
@@ -860,19 +904,25 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
             "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
             "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": dict(config_of(desc, dtype, n, world),
-                           launch="one stream, back-to-back launches marked independent of "
-                                  "their predecessor (programmatic dependent launch)",
-                           l2=f"rotating {sets} input/output buffer sets "
-                              f"({sets * step_bytes / 1e6:.0f} MB held, "
-                              f"{sets * acct['total'] / 1e6:.0f} MB touched) > L2 "
-                              f"({l2 / 1e6:.0f} MB)"),
+            "config": config_of(desc, dtype, n, world),
+            "launch": launch_note,
+            "l2": f"rotating {sets} input/output buffer sets "
+                  f"({sets * step_bytes / 1e6:.0f} MB held, "
+                  f"{sets * acct['total'] / 1e6:.0f} MB touched) > L2 ({l2 / 1e6:.0f} MB)",
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                         "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src,
+                         "frac": achieved / peak, "traffic": traffic,
+                         "traffic_note": TRAFFIC_NOTE if traffic is not None else None,
+                         "peak_source": peak_src,
                          "algorithmic_bytes_per_launch": acct["total"],
                          "input_sector_bytes": acct["input_sector_bytes"],
                          "output_bytes": acct["output_bytes"],
                          "kernel_us": per_launch_s * 1e6,
+                         "frac_note": "launches follow one another on the stream and overlap "
+                                      "at their ends (see launch); frac_isolated is one launch "
+                                      "running alone",
+                         "achieved_isolated": acct["total"] / (iso_p50 * 1e-6) / 1e9,
+                         "frac_isolated": acct["total"] / (iso_p50 * 1e-6) / 1e9 / peak,
+                         "isolated_kernel_us": iso_p50,
                          "host_launch_us": 1e6 * t_host / args.steps},
             "cpu_baseline": {"value": cpu_value, "unit": UNIT, "cores": threads, "kind": "oracle",
                              "sample": f"whole batch of {n} images, {len(cpu_times)} passes",
@@ -900,13 +950,15 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
                         "host_ms_per_step": 1e3 * packed_host / e2e_steps,
                         "includes": "preba_pack into pinned memory + one copy + kernel + copy "
                                     "back (preba_preprocess_host)"}},
-            "isolated_launch_us": {"p50": float(np.percentile(lat_us, 50)),
+            "isolated_launch_us": {"p50": iso_p50,
                                    "p99": float(np.percentile(lat_us, 99)),
-                                   "note": "device time of one launch running alone, events "
-                                           "around every launch, same buffers every time"},
+                                   "note": "device time of one launch running alone (warps claim "
+                                           "slabs through the scratch counters), events around "
+                                           "every launch, same buffers every time"},
             "warm_l2": {"value": world * n * warm_steps / (warm_ms * 1e-3), "unit": UNIT,
                         "us_per_launch": 1e3 * warm_ms / warm_steps,
-                        "note": "one buffer set reused by every launch; not the headline"},
+                        "note": "one buffer set reused by every launch, launches not marked as "
+                                "overlapping; not the headline"},
             "gpu_launches": args.steps,
             "clocks": clocks.summary(),
         }
@@ -914,6 +966,21 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
+
+
+def spawn_ranks(n: int) -> int:
+    """`--gpus N` without a launcher around it: start the N ranks (one process per GPU) through
+    torch.distributed.run on this node, with the same arguments, and pass their output on."""
+    import socket
+    import subprocess
+
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), str(Path(__file__).resolve()),
+           *sys.argv[1:]]
+    return subprocess.run(cmd).returncode
 
 
 def main() -> None:
@@ -932,6 +999,9 @@ def main() -> None:
     ap.add_argument("--cpu-budget", type=float, default=12.0,
                     help="seconds of wall time given to the CPU-baseline leg")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours" \
+            and args.workload in ("mixed", "320x240", "1080p", "sweep"):
+        raise SystemExit(spawn_ranks(args.gpus))
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))

@@ -19,6 +19,12 @@
  *     buffers until the stream has passed the work the call enqueued.
  *   - Calls keep no state between them and may be made concurrently from
  *     several threads, each on its own stream.
+ *   Two entry points depart from this, as their own comments say:
+ *   preba_preprocess_host_noalloc keeps the device address of the library's
+ *   staging array per device (it does not survive cudaDeviceReset) and every
+ *   call shares that array, so its calls must be serialised per device;
+ *   preba_preprocess_repeated creates and destroys events and waits for the
+ *   stream.
  */
 #ifndef PREBA_H_
 #define PREBA_H_
@@ -35,13 +41,21 @@ extern "C" {
 #define PREBA_SCRATCH_BYTES 256u  /* size of the scheduling scratch a batch may carry */
 
 /* preba_batch_t.flags */
-#define PREBA_OVERLAP_PREVIOUS 1u /* the launch need not wait for the kernel before it on the
-                                     stream to finish (programmatic dependent launch): as that
-                                     kernel's warps retire, this one's take their place.  Set it
-                                     only if that kernel neither writes this batch's pixels, table
-                                     or scratch nor touches its out buffer, e.g. back-to-back
-                                     batches with buffers of their own.  Copies, and kernels
-                                     launched without the flag, order as usual. */
+#define PREBA_OVERLAP_PREVIOUS 1u /* the launch need not wait for the kernels before it on the
+                                     stream to finish (programmatic dependent launch): as their
+                                     warps retire, this one's take their place.  The relaxation
+                                     chains: a marked launch may run beside every kernel enqueued
+                                     since the last operation on the stream that was not a marked
+                                     launch (an unmarked launch, a copy, an event wait), not only
+                                     beside the one directly before it.  Set it only if none of
+                                     those kernels writes this batch's pixels, table or scratch
+                                     or touches its out buffer, e.g. back-to-back batches with
+                                     buffers (and scratch) of their own, and put an unmarked
+                                     launch where a buffer set comes round again.  Completion
+                                     stays ordered: a marked launch does not complete before the
+                                     kernels ahead of it have, so whatever is enqueued after it
+                                     without the flag (a copy, an event, an unmarked launch)
+                                     finds the results of the whole chain. */
 
 #define PREBA_OK 0
 #define PREBA_ERR_INVALID_ARG (-1)      /* NULL, zero or out-of-range argument, misaligned buffer */
@@ -439,7 +453,7 @@ int preba_bucket_batcher_poll(preba_bucket_batcher_t* b, uint64_t now_ns, uint64
 
 /*
  * Audio path — the paper's second preprocessing pipeline (Table 1 units "Mel spectrogram" and
- * "Normalize"; Sec. 2.3 item 1: "Fast Fourier Transform (FFT), and applying Mel filters";
+ * "Normalize"; Sec. 2.3 item 1: a Fourier transform followed by a Mel filterbank;
  * Sec. 4.2: Normalize as three passes, the mean over all samples, the variance from that mean,
  * then the normalisation).  Samples are taken at 16 kHz; preba_audio_resample (below) brings
  * other rates there.  The paper

@@ -1,8 +1,7 @@
 """TEST INFRASTRUCTURE ONLY: CPU oracle of the audio preprocessing path (numpy, float64).
 
 The paper lists the audio units as Resample, Mel spectrogram and Normalize (Table 1) and the
-operations as "resampling, Fast Fourier Transform (FFT), and applying Mel filters" (Sec. 2.3
-item 1); Sec. 4.2 spells out Normalize as three passes: the mean over all samples, the
+operations as resampling, a Fourier transform and a Mel filterbank (Sec. 2.3 item 1); Sec. 4.2 spells out Normalize as three passes: the mean over all samples, the
 variance using that mean, then the normalisation of each sample by both.  It fixes no numerics.
 The readings taken here (every one of them a choice of this library, not of the paper):
 

@@ -965,6 +965,12 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
     for (uint32_t q = consumed; q < issued; ++q)
       (void)mbar_wait(smem_addr(&ws.full[q % kGroups]), (q / kGroups) & 1);
   }
+  // A launch marked as overlapping started without waiting for the kernels before it on the
+  // stream.  It must not complete before them, or work ordered after it could run ahead of
+  // their results: wait here, after the last store, until they have completed (no wait at all
+  // for an unmarked launch).  Each launch waits for its predecessor, so completion follows
+  // the stream's order along a whole chain of marked launches.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   // the last warp out leaves the claim counters at zero for the next launch
   if (p.sched && lane == 0) {
     __threadfence();

@@ -179,9 +179,13 @@ def test_workload_mixed_smooth_fp16_full_in_the_benchmark_launch_configuration()
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     calls = [pb.PreparedPreprocess(pix[i], tab, n, outs[i], 224, 256, MEAN, STD, pb.F16,
                                    status=status, flags=pb.OVERLAP_PREVIOUS) for i in range(sets)]
+    # where the buffer sets come round again the launch is not marked: a marked launch may run
+    # beside every kernel back to the last unmarked one
+    first = pb.PreparedPreprocess(pix[0], tab, n, outs[0], 224, 256, MEAN, STD, pb.F16,
+                                  status=status)
     torch.cuda.synchronize()
     for i in range(10 * sets):
-        calls[i % sets]()
+        (first if i % sets == 0 else calls[i % sets])()
     torch.cuda.synchronize()
     assert int(status.item()) == 0
     for o in outs:
@@ -270,15 +274,57 @@ def test_overlapping_launches_into_buffers_of_their_own(dynamic):
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     torch.cuda.synchronize()
     for rnd in range(4):
-        for i in range(3):
+        for i in range(3):  # the first launch of a round is unmarked: the buffers come round again
             pb.preba_preprocess(pix[i], tabs[i], 48, outs[i], 224, 256, MEAN, STD, pb.F16,
-                                status=status, scratch=scr[i], flags=pb.OVERLAP_PREVIOUS)
+                                status=status, scratch=scr[i],
+                                flags=pb.OVERLAP_PREVIOUS if i else 0)
     torch.cuda.synchronize()
     assert int(status.item()) == 0
     for o, want, sc in zip(outs, wants, scr):
         assert_parity(o.cpu().numpy(), want, pb.F16)
         if sc is not None:
             assert int(sc.abs().sum().item()) == 0
+
+
+def test_work_ordered_after_a_chain_of_overlapping_launches_sees_all_of_it():
+    """A long launch followed by short ones marked as overlapping, then copies of every result to
+    pinned memory and an event on the same stream, and no device-wide wait: a marked launch must
+    not complete before the kernels ahead of it, or the copy of the long launch's result would
+    run before that launch has finished."""
+    import torch
+
+    dev = torch.device("cuda:0")
+    big = wl.mixed_smooth(192, seed=60)
+    small = [wl.mixed_smooth(2, seed=61 + i) for i in range(4)]
+    batches = [big] + small
+    wants = [oracle_f64(b, 224, 256) for b in batches]
+    packs = [pb.preba_pack(b) for b in batches]
+    pix = [torch.from_numpy(pk).to(dev) for pk, _ in packs]
+    tabs = [torch.from_numpy(tb.view(np.uint8)).to(dev) for _, tb in packs]
+    outs = [torch.empty((len(b), 3, 224, 224), dtype=torch.float16, device=dev) for b in batches]
+    host = [torch.empty((len(b), 3, 224, 224), dtype=torch.float16).pin_memory() for b in batches]
+    scr = [torch.zeros(pb.SCRATCH_BYTES // 4, dtype=torch.int32, device=dev) for _ in batches]
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    st = torch.cuda.Stream()
+    done = torch.cuda.Event()
+    for rnd in range(5):
+        for o, hbuf in zip(outs, host):
+            o.fill_(float("nan"))
+            hbuf.fill_(float("nan"))
+        torch.cuda.synchronize()
+        with torch.cuda.stream(st):
+            for i, b in enumerate(batches):
+                pb.preba_preprocess(pix[i], tabs[i], len(b), outs[i], 224, 256, MEAN, STD, pb.F16,
+                                    stream=st, status=status, scratch=scr[i],
+                                    flags=pb.OVERLAP_PREVIOUS if i else 0)
+            for o, hbuf in zip(outs, host):
+                hbuf.copy_(o, non_blocking=True)
+            done.record(st)
+        done.synchronize()  # the host waits for the event only
+        for hbuf, want in zip(host, wants):
+            assert_parity(hbuf.numpy(), want, pb.F16)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
 
 
 def test_repeated_launch_aid_gives_the_same_result_and_times_every_launch():
