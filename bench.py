@@ -390,7 +390,7 @@ def run_audio(args, local_rank: int) -> None:
     for i in (0, n // 2, n - 1):
         want = oa.preprocess([utts[i]])[0]
         err = float(np.max(np.abs(got[i, :, :want.shape[1]] - want)))
-        assert err <= 2e-3, f"audio result differs from the oracle: {err:.3e}"
+        assert err <= 3e-4, f"audio result differs from the oracle: {err:.3e}"
     # the Resample unit on the same samples taken as 48 kHz material (48 kHz -> 16 kHz)
     lens48 = pb.preba_audio_resample_query(table["length"], 48000, 16000)
     table48 = pb.preba_audio_layout(lens48)

@@ -513,9 +513,11 @@ int preba_audio_pack(const float* const* utterances, const uint32_t* lengths, ui
                      float* packed, uint64_t capacity_samples, preba_utt_t* table);
 
 /* Mel spectrogram (+ Normalize when `normalize` is non-zero) of a device-resident batch:
- * enqueues one kernel for the log Mel energies (a warp transforms two frames with one complex
- * 512-point FFT in shared memory) and, when normalising, one more for the three passes over
- * every (utterance, filter) row; then returns.  No allocation, no synchronisation.  A table
+ * enqueues one kernel for the log Mel energies (the frame pairs of the batch are shared out
+ * evenly over the warps of a grid that fills the GPU once; a warp transforms two frames with
+ * one complex 512-point FFT held in registers) and, when normalising, one more for the three
+ * passes over every (utterance, filter) row, launched so that it is scheduled while the first
+ * drains and waits for it on the device; then returns.  No allocation, no synchronisation.  A table
  * entry that is misaligned, runs past the samples or whose frame count does not follow from
  * its length is refused on the host when `table_host` is given (PREBA_ERR_BAD_TABLE) and
  * skipped and reported by the kernel otherwise.

@@ -678,8 +678,11 @@ extern "C" int preba_preprocess_antialias(const preba_batch_t* batch, const preb
     uint64_t most = 0;
     for (uint32_t i = 0; i < batch->n; ++i) {
       const preba_img_t& e = batch->table_host[i];
-      if (!dims_ok(e.h, e.w) || e.offset % PREBA_PACK_ALIGN || e.offset > batch->pixels_bytes ||
-          3ull * e.h * e.w > batch->pixels_bytes - e.offset)
+      // as in the kernel: rows are fetched in 16-byte units, so the buffer counts up to its
+      // last whole unit
+      const uint64_t usable = batch->pixels_bytes & ~15ull;
+      if (!dims_ok(e.h, e.w) || e.offset % PREBA_PACK_ALIGN || e.offset > usable ||
+          3ull * e.h * e.w > usable - e.offset)
         return PREBA_ERR_BAD_TABLE;
       uint32_t rh, rw;
       resized_size(e.h, e.w, S, &rh, &rw);

@@ -1,17 +1,25 @@
 // Audio path: log Mel spectrogram and per-utterance normalisation of a ragged batch (sm_100a).
 //
-// Kernel 1: a warp takes two consecutive frames of one utterance, multiplies them by the Hann
-// window, packs them as the real and imaginary part of one complex sequence, runs a 512-point
-// FFT as three passes of radix-8 butterflies in registers (exchanging through its own shared
-// memory between passes), separates the two spectra, forms the power spectra,
-// applies the triangular Mel filters (a lane per filter, the filter's few bins read from
-// shared memory) and writes log(energy + 2^-24).  Frames past an utterance's own count are
+// Kernel 1 (persistent grid): the frame pairs of the whole batch (two consecutive frames of one
+// utterance) are split evenly over all resident warps, each warp taking a contiguous run.  Per
+// pair the warp multiplies the two frames by the Hann window, packs them as the real and
+// imaginary part of one complex sequence and runs a 512-point FFT as three passes of radix-8
+// butterflies in registers, exchanging through its own shared memory between passes; window
+// values and the second pass's twiddle factors are per-lane constants held in registers.  The two spectra are
+// separated with one shuffle per value (the partner of bin k, bin 512 - k, sits in lane
+// 32 - lane), the power spectra go to shared memory in natural order, and the triangular Mel
+// filters are summed a lane per filter over a plan laid out so that no access conflicts: the
+// weights iteration-major, and the filters of a half-warp starting at distinct addresses
+// modulo 16.  log(energy + 2^-24) is written; frames past an utterance's own count are
 // written as 0, so the result tensor needs no clearing.
-// Kernel 2 (Normalize): a warp per (utterance, filter) row makes the paper's three passes:
-// mean, variance from that mean, normalisation.
+// Kernel 2 (Normalize): a warp per (utterance, filter) row makes the paper's three passes over
+// the row held in registers: mean, variance from that mean, normalisation.  It is launched as
+// a programmatic dependent of kernel 1 and waits for it on the device.
 // fp32 throughout; the path is bound by arithmetic and shared memory, not by HBM.
 #include <cuda_runtime.h>
 
+#include <algorithm>
+#include <atomic>
 #include <cmath>
 #include <cstdint>
 #include <cstring>
@@ -28,51 +36,112 @@ constexpr uint32_t kFft = PREBA_AUDIO_NFFT;
 constexpr uint32_t kBins = kFft / 2 + 1;
 constexpr uint32_t kMels = PREBA_AUDIO_MELS;
 constexpr int kWarps = 4;            // warps per CTA of the spectrogram kernel
-constexpr int kPairsPerWarp = 4;      // frame pairs a warp transforms one after the other
-constexpr int kFramesPerCta = 2 * kWarps * kPairsPerWarp;
+constexpr int kCtasPerSm = 4;
 constexpr float kLogGuard = 5.9604644775390625e-08f;  // 2^-24
 constexpr float kStdGuard = 1e-5f;
 
-// The Mel filters in the form the kernel uses: filter j covers the consecutive bins
-// first[j] .. first[j] + count[j] - 1 and their weights lie one after the other in w from
-// start[j] (rising edge, then falling edge; every bin belongs to at most two filters).
-constexpr uint32_t kMelWeights = 2 * kBins + 2;
-struct MelTable {
-  float w[kMelWeights];
-  uint16_t first[kMels];
-  uint16_t count[kMels];
-  uint16_t start[kMels];
+// The Mel filters as the kernel sums them.  Filter j has non-zero weight on the consecutive
+// bins first[j] .. first[j] + count[j] - 1.  The 80 filters are dealt out, heaviest first, to
+// five half-warps of 16 lanes over three rounds (round r: lanes 0-15 the 2r-th sixteen,
+// lanes 16-31 the next).  In a round every lane reads, iteration by iteration, one weight and
+// the power of one bin, starting at bin begin <= first; begin is moved down from first until
+// its remainder modulo 16 is free within the half-warp, so that the 16 lanes always read 16
+// different banks; the weights before first are 0.  w holds the weights iteration-major, lane
+// by lane (consecutive lanes, consecutive words).
+constexpr uint32_t kMelRounds = 3;
+// Iterations of the three rounds as the kernel runs them (its loops are unrolled in full): the
+// plan of the 80 filters at 16 kHz needs 17, 13 and 5; a round that needs fewer reads weights
+// of 0, and a plan that needed more would be refused.
+constexpr uint32_t kMelIters0 = 18, kMelIters1 = 14, kMelIters2 = 6;
+constexpr uint32_t kMelMaxIters = kMelIters0 + kMelIters1 + kMelIters2;
+constexpr uint32_t kPowPad = 16;       // zeroed entries in front of the power spectrum (begin may
+                                       // lie before bin 0)
+constexpr uint32_t kPowLen = kPowPad + kBins + 47;  // and behind it (rounds read past a filter's end)
+struct MelPlan {
+  float w[kMelMaxIters * 32];
+  int16_t begin[kMelRounds][32];   // first index read in the padded power array
+  uint8_t filter[kMelRounds][32];  // the lane's filter in the round, or 0xff
+  uint8_t iters[kMelRounds];       // iterations the round needs (the kernel runs kMelIters*)
+  uint8_t ok;                      // the plan fits the kernel's rounds and the padding
 };
-static_assert(sizeof(MelTable) % 4 == 0 && sizeof(MelTable) < 3800, "passed as a kernel parameter");
+static_assert(sizeof(MelPlan) % 4 == 0 && sizeof(MelPlan) < 8192, "passed as a kernel parameter");
 
 uint32_t frames_of(uint32_t length) { return length < kWin ? 0u : 1u + (length - kWin) / kHop; }
 
 // Corner frequencies equally spaced on the HTK mel scale between 0 and rate / 2 (double);
 // filter j rises from corner j to corner j + 1 and falls to corner j + 2.
-MelTable make_mel_table() {
-  MelTable t;
+MelPlan make_mel_plan() {
+  MelPlan t;
   std::memset(&t, 0, sizeof(t));
+  std::memset(t.filter, 0xff, sizeof(t.filter));
   const double top = 2595.0 * std::log10(1.0 + (PREBA_AUDIO_RATE / 2.0) / 700.0);
   double corner[kMels + 2];
   for (uint32_t i = 0; i < kMels + 2; ++i)
     corner[i] = 700.0 * (std::pow(10.0, (top * i / (kMels + 1)) / 2595.0) - 1.0);
   corner[0] = 0.0;
   corner[kMels + 1] = PREBA_AUDIO_RATE / 2.0;
-  uint32_t at = 0;
+  static float weight[kMels][kBins];
+  int first[kMels], count[kMels];
   for (uint32_t j = 0; j < kMels; ++j) {
     const double lo = corner[j], mid = corner[j + 1], hi = corner[j + 2];
-    t.start[j] = static_cast<uint16_t>(at);
-    bool any = false;
+    first[j] = -1;
+    count[j] = 0;
     for (uint32_t k = 0; k < kBins; ++k) {
       const double f = static_cast<double>(k) * PREBA_AUDIO_RATE / kFft;
+      weight[j][k] = 0.f;
       if (f <= lo || f >= hi) continue;  // weight 0 at and beyond the feet
       const double wgt = f < mid ? (f - lo) / (mid - lo) : (hi - f) / (hi - mid);
-      if (!any) t.first[j] = static_cast<uint16_t>(k);
-      any = true;
-      if (at < kMelWeights) t.w[at++] = static_cast<float>(wgt);
-      t.count[j] = static_cast<uint16_t>(k + 1 - t.first[j]);
+      weight[j][k] = static_cast<float>(wgt);
+      if (first[j] < 0) first[j] = static_cast<int>(k);
+      count[j] = static_cast<int>(k) + 1 - first[j];
     }
+    if (first[j] < 0) first[j] = 0;  // a filter without a bin: all weights 0
   }
+  int order[kMels];
+  for (uint32_t j = 0; j < kMels; ++j) order[j] = static_cast<int>(j);
+  std::stable_sort(order, order + kMels, [&](int a, int b) { return count[a] > count[b]; });
+  uint32_t at = 0;  // iterations used so far
+  bool ok = true;
+  for (uint32_t r = 0; r < kMelRounds; ++r) {
+    int begin[32], filt[32];
+    int iters = 0;
+    for (int lane = 0; lane < 32; ++lane) begin[lane] = 0, filt[lane] = -1;
+    for (int half = 0; half < 2; ++half) {
+      bool used[16] = {};
+      for (int i = 0; i < 16; ++i) {
+        const uint32_t idx = (2 * r + half) * 16 + i;
+        if (idx >= kMels) break;
+        const int j = order[idx], lane = 16 * half + i;
+        int e = first[j];
+        while (used[((e % 16) + 16) % 16]) --e;
+        used[((e % 16) + 16) % 16] = true;
+        begin[lane] = e;
+        filt[lane] = j;
+        iters = std::max(iters, first[j] - e + count[j]);
+        if (e < -static_cast<int>(kPowPad)) ok = false;
+      }
+    }
+    const int room = static_cast<int>(r == 0 ? kMelIters0 : r == 1 ? kMelIters1 : kMelIters2);
+    if (iters > room) {
+      ok = false;
+      break;
+    }
+    for (int lane = 0; lane < 32; ++lane) {
+      t.begin[r][lane] = static_cast<int16_t>(begin[lane] + static_cast<int>(kPowPad));
+      t.filter[r][lane] = static_cast<uint8_t>(filt[lane] < 0 ? 0xff : filt[lane]);
+      if (begin[lane] + static_cast<int>(kPowPad) + room > static_cast<int>(kPowLen)) ok = false;
+      for (int i = 0; i < iters; ++i) {
+        const int k = begin[lane] + i;
+        // a quarter of the weight: the kernel's power spectra are those of twice the spectrum
+        t.w[(at + i) * 32 + lane] =
+            (filt[lane] >= 0 && k >= 0 && k < static_cast<int>(kBins)) ? 0.25f * weight[filt[lane]][k]
+                                                                      : 0.f;
+      }
+    }
+    t.iters[r] = static_cast<uint8_t>(iters);
+    at += room;  // the round's weights beyond `iters` stay 0
+  }
+  t.ok = ok ? 1 : 0;
   return t;
 }
 
@@ -93,15 +162,25 @@ __device__ __forceinline__ bool utt_ok(const preba_utt_t& u, uint64_t samples_co
   return u.frames == frames;
 }
 
+// Frames of utterance i that the result holds (0 for an entry that is refused).
+__device__ __forceinline__ uint32_t frames_in(const AudioParams& p, uint32_t i) {
+  const preba_utt_t u = p.table[i];
+  return utt_ok(u, p.samples_count) ? min(u.frames, p.t_max) : 0u;
+}
+
 // The 512-point FFT runs as three passes of radix-8 butterflies held in registers
-// (512 = 8 * 8 * 8); between passes the warp exchanges its values through an 8 x 64 array in
-// shared memory whose rows are 68 elements apart, which keeps every exchange at the two
-// wavefronts a 64-bit access of 32 lanes needs.
-constexpr uint32_t kPitch = 68;
+// (512 = 8 * 8 * 8).  With n = 64 n2 + 8 n1 + n0 and k = k0 + 8 k1 + 64 k2:
+//   X[k] = sum_n0 W8^(n0 k2) W64^(n0 k1)
+//          sum_n1 W8^(n1 k1) W512^((8 n1 + n0) k0) sum_n2 W8^(n2 k0) x[n].
+// Between passes the warp exchanges its values through an 8-row array in shared memory; the
+// rows are 72 elements apart after pass 1 and 66 after pass 2, which makes the 16 lanes of a
+// half-warp hit 16 different 8-byte banks in every store and load.
+constexpr uint32_t kPitch1 = 72;
+constexpr uint32_t kPitch2 = 66;
 
 struct __align__(16) WarpFft {
-  float2 z[8 * kPitch];  // exchange array, then the spectrum in natural order (first 512)
-  float2 power[kBins + 1];  // the two frames' power spectra side by side
+  float2 z[8 * kPitch1];   // exchange array
+  float2 power[kPowLen];   // the two frames' power spectra side by side, zero padding around
 };
 
 __device__ __forceinline__ float2 cadd(float2 a, float2 b) { return make_float2(a.x + b.x, a.y + b.y); }
@@ -136,157 +215,308 @@ __device__ __forceinline__ void fft8(float2 (&v)[8]) {
   v[7] = csub(o1, o3);
 }
 
-__global__ void __launch_bounds__(32 * kWarps)
-logmel_kernel(const AudioParams p, const MelTable mel_param) {
+// One round of the Mel filters: the lane's filter summed over ITERS consecutive bins of both
+// frames (weights of 0 outside the filter), then the logs.  The energies are at least 2^-24,
+// a normal number, and the results lie between -17 and about 30: there the fast logarithm
+// (log2 by the special-function unit times ln 2) is within 3 ulp, 6e-6 at most.
+template <uint32_t ITERS>
+__device__ __forceinline__ void mel_round(const float* __restrict__ wp, const float2* __restrict__ pp,
+                                          uint32_t filter, float* __restrict__ out, uint32_t t_max,
+                                          uint32_t t0, bool have1) {
+  float e0 = 0.f, e1 = 0.f;
+#pragma unroll
+  for (uint32_t i = 0; i < ITERS; ++i) {
+    const float wgt = wp[i * 32];
+    const float2 pw = pp[i];
+    e0 = fmaf(wgt, pw.x, e0);
+    e1 = fmaf(wgt, pw.y, e1);
+  }
+  if (filter != 0xffu) {
+    float* __restrict__ o = out + static_cast<size_t>(filter) * t_max + t0;
+    o[0] = __logf(e0 + kLogGuard);
+    if (have1) o[1] = __logf(e1 + kLogGuard);
+  }
+}
+
+// Frame pairs of utterance i: two frames share one complex transform.
+__device__ __forceinline__ uint32_t pairs_in(const AudioParams& p, uint32_t i) {
+  return (frames_in(p, i) + 1) / 2;
+}
+
+__global__ void __launch_bounds__(32 * kWarps, kCtasPerSm)
+logmel_kernel(const AudioParams p, const MelPlan plan_param) {
   __shared__ WarpFft sm[kWarps];
-  __shared__ float2 twiddle[kFft];  // exp(-2 pi i j / 512)
-  __shared__ float window[kWin];
-  __shared__ MelTable mel;  // lanes read different entries: shared memory, not the constant bank
+  __shared__ float2 tw1[7][64];     // after pass 1: exp(-2 pi i col k0 / 512), k0 = 1..7, by column
+  __shared__ float window[kFft];    // Hann over the first 400, then 0
+  __shared__ MelPlan plan;          // lanes read different entries: shared memory, not the constant bank
+  // the Normalize kernel may be scheduled as soon as resources free up; it waits for this
+  // grid to complete before it reads anything
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const uint32_t utt = blockIdx.y;
-  const preba_utt_t u = p.table[utt];
-  const bool ok = utt_ok(u, p.samples_count);
-  if (!ok && threadIdx.x == 0 && blockIdx.x == 0 && p.status)
-    atomicCAS(p.status, 0, PREBA_ERR_BAD_TABLE);
-  const uint32_t frames = ok ? min(u.frames, p.t_max) : 0u;
-  float* __restrict__ out = p.out + static_cast<size_t>(utt) * kMels * p.t_max;
-  const uint32_t cta_t0 = blockIdx.x * kFramesPerCta;
-  if (cta_t0 >= frames) {
-    // padding (or a refused entry): zeros for all of this CTA's frames
-    const uint32_t t_end = min(cta_t0 + kFramesPerCta, p.t_max);
-    for (uint32_t j = warp; j < kMels; j += kWarps)
-      for (uint32_t t = cta_t0 + lane; t < t_end; t += 32) out[static_cast<size_t>(j) * p.t_max + t] = 0.f;
-    return;
-  }
   for (uint32_t k = threadIdx.x; k < kFft; k += blockDim.x) {
-    float s, c;
-    sincospif(-2.0f * static_cast<float>(k) / kFft, &s, &c);
-    twiddle[k] = make_float2(c, s);
+    window[k] = k < kWin ? 0.5f - 0.5f * cospif(2.0f * static_cast<float>(k) / kWin) : 0.f;
+    if (k < 7 * 64) {
+      const uint32_t k0 = (k >> 6) + 1, col = k & 63;
+      float sn, cs;
+      sincospif(-2.0f * static_cast<float>(col * k0) / kFft, &sn, &cs);
+      tw1[k0 - 1][col] = make_float2(cs, sn);
+    }
   }
-  for (uint32_t i = threadIdx.x; i < kWin; i += blockDim.x)
-    window[i] = 0.5f - 0.5f * cospif(2.0f * static_cast<float>(i) / kWin);
   {
-    const uint32_t* src = reinterpret_cast<const uint32_t*>(&mel_param);
-    uint32_t* dst = reinterpret_cast<uint32_t*>(&mel);
-    for (uint32_t i = threadIdx.x; i < sizeof(MelTable) / 4; i += blockDim.x) dst[i] = src[i];
+    const uint32_t* src = reinterpret_cast<const uint32_t*>(&plan_param);
+    uint32_t* dst = reinterpret_cast<uint32_t*>(&plan);
+    for (uint32_t i = threadIdx.x; i < sizeof(MelPlan) / 4; i += blockDim.x) dst[i] = src[i];
   }
+  WarpFft& ws = sm[warp];
+  for (uint32_t i = lane; i < kPowLen; i += 32) ws.power[i] = make_float2(0.f, 0.f);
   __syncthreads();
 
-  WarpFft& ws = sm[warp];
-#pragma unroll 1
-  for (uint32_t pair = 0; pair < kPairsPerWarp; ++pair) {
-    const uint32_t t0 = cta_t0 + 2 * (warp + kWarps * pair);  // this warp's two frames
-    if (t0 >= p.t_max) break;
-    const bool have0 = t0 < frames, have1 = t0 + 1 < frames;
-    if (!have0) {
-      for (uint32_t j = lane; j < kMels; j += 32) {
-        out[static_cast<size_t>(j) * p.t_max + t0] = 0.f;
-        if (t0 + 1 < p.t_max) out[static_cast<size_t>(j) * p.t_max + t0 + 1] = 0.f;
+  // per-lane constants: the window at the lane's 13 sample positions inside the frame (of
+  // 64 n2 + lane + 32 c only n2 < 6, and n2 = 6 with c = 0 and lane < 16, lie below 400), the
+  // twiddles of its two columns after pass 1 and those after pass 2, its place in the Mel rounds
+  const uint32_t n0 = lane & 7;
+  float win[2][6], win6;
+  float2 tw2[7];  // after pass 2: exp(-2 pi i n0 k1 / 64)
+#pragma unroll
+  for (int c = 0; c < 2; ++c)
+#pragma unroll
+    for (uint32_t n2 = 0; n2 < 6; ++n2) win[c][n2] = window[64 * n2 + lane + 32 * c];
+  win6 = window[384 + lane];  // 0 from lane 16 on
+  const uint32_t i6 = lane < 16 ? 384 + lane : lane;  // a sample that exists, for a weight of 0
+#pragma unroll
+  for (uint32_t k1 = 1; k1 < 8; ++k1) {
+    float sn, cs;
+    sincospif(-2.0f * static_cast<float>(n0 * k1) / 64.0f, &sn, &cs);
+    tw2[k1 - 1] = make_float2(cs, sn);
+  }
+  int mel_begin[kMelRounds];
+  uint32_t mel_filter[kMelRounds];
+#pragma unroll
+  for (uint32_t r = 0; r < kMelRounds; ++r) {
+    mel_begin[r] = plan.begin[r][lane];
+    mel_filter[r] = plan.filter[r][lane];
+  }
+
+  // this warp's run of the batch's frame pairs: an equal share, contiguous
+  const uint32_t nwarps = gridDim.x * kWarps, gwarp = blockIdx.x * kWarps + warp;
+  uint64_t total = 0;
+  for (uint32_t i0 = 0; i0 < p.n; i0 += 32) {
+    uint32_t c = i0 + lane < p.n ? pairs_in(p, i0 + lane) : 0u;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
+    total += c;
+  }
+  uint64_t g = total * gwarp / nwarps;
+  const uint64_t g_end = total * (gwarp + 1) / nwarps;
+  // the utterance holding pair g, and g's index in it
+  uint32_t utt = 0, q = 0, upairs = 0;
+  {
+    uint64_t before = 0;
+    bool found = false;
+    for (uint32_t i0 = 0; i0 < p.n && !found; i0 += 32) {
+      const uint32_t c = i0 + lane < p.n ? pairs_in(p, i0 + lane) : 0u;
+      uint32_t inc = c;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t v = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= static_cast<uint32_t>(o)) inc += v;
       }
-      continue;
+      const uint32_t hit = __ballot_sync(0xffffffffu, before + inc > g);
+      if (hit) {
+        const int src = __ffs(hit) - 1;
+        const uint32_t inc_s = __shfl_sync(0xffffffffu, inc, src);
+        upairs = __shfl_sync(0xffffffffu, c, src);
+        utt = i0 + src;
+        q = static_cast<uint32_t>(g - (before + inc_s - upairs));
+        found = true;
+      }
+      before += __shfl_sync(0xffffffffu, inc, 31);
     }
-    const float* __restrict__ x = p.samples + u.offset + static_cast<size_t>(t0) * kHop;
-    // With n = 64 n2 + 8 n1 + n0 and k = k0 + 8 k1 + 64 k2:
-    //   X[k] = sum_n0 W8^(n0 k2) W512^(n0 (k0 + 8 k1))
-    //          sum_n1 W8^(n1 k1) W64^(n1 k0) sum_n2 W8^(n2 k0) x[n].
-    // Pass 1 (over n2): a lane takes the columns p = 8 n1 + n0 = lane and lane + 32 of the two
-    // windowed frames (real and imaginary part).
+    if (!found) g = g_end;  // nothing left for this warp
+  }
+
+  // The samples of a pair are fetched one pair ahead, into the registers the transform has
+  // just released: raw[f][c][n2] is sample 64 n2 + lane + 32 c of frame f, raw6[f] sample
+  // 384 + lane.  A pair without a second frame reads the first one twice (the duplicate
+  // spectrum is not written).
+  float raw[2][2][6], raw6[2];
+  uint32_t frames = 0;
+  auto fetch = [&]() {
+    const preba_utt_t u = p.table[utt];
+    frames = min(u.frames, p.t_max);
+    const float* __restrict__ x0 = p.samples + u.offset + static_cast<size_t>(2 * q) * kHop;
+    const float* __restrict__ x1 = 2 * q + 1 < frames ? x0 + kHop : x0;
+#pragma unroll
+    for (int c = 0; c < 2; ++c)
+#pragma unroll
+      for (uint32_t n2 = 0; n2 < 6; ++n2) {
+        raw[0][c][n2] = x0[64 * n2 + lane + 32 * c];
+        raw[1][c][n2] = x1[64 * n2 + lane + 32 * c];
+      }
+    raw6[0] = x0[i6];
+    raw6[1] = x1[i6];
+  };
+  if (g < g_end) fetch();
+
+#pragma unroll 1
+  while (g < g_end) {
+    const uint32_t t0 = 2 * q;
+    const bool have1 = t0 + 1 < frames;
+    float* __restrict__ out = p.out + static_cast<size_t>(utt) * kMels * p.t_max;
+    // Pass 1 (over n2): a lane takes the columns 8 n1 + n0 = lane and lane + 32 of the two
+    // windowed frames (real and imaginary part); the samples from 400 on are zero padding.
     float2 v[2][8];
 #pragma unroll
     for (int c = 0; c < 2; ++c) {
       const uint32_t pcol = lane + 32 * c;
 #pragma unroll
-      for (uint32_t n2 = 0; n2 < 8; ++n2) {
-        const uint32_t i = 64 * n2 + pcol;
-        float re = 0.f, im = 0.f;
-        if (i < kWin) {
-          re = x[i] * window[i];
-          if (have1) im = x[i + kHop] * window[i];
-        }
-        v[c][n2] = make_float2(re, im);
-      }
+      for (uint32_t n2 = 0; n2 < 6; ++n2)
+        v[c][n2] = make_float2(raw[0][c][n2] * win[c][n2], raw[1][c][n2] * win[c][n2]);
+      v[c][6] = c == 0 ? make_float2(raw6[0] * win6, raw6[1] * win6) : make_float2(0.f, 0.f);
+      v[c][7] = make_float2(0.f, 0.f);
       fft8(v[c]);
-      const uint32_t n1 = pcol >> 3;
+      ws.z[pcol] = v[c][0];
 #pragma unroll
-      for (uint32_t k0 = 0; k0 < 8; ++k0)
-        ws.z[k0 * kPitch + pcol] = k0 ? cmul(v[c][k0], twiddle[8 * n1 * k0]) : v[c][0];
+      for (uint32_t k0 = 1; k0 < 8; ++k0) ws.z[k0 * kPitch1 + pcol] = cmul(v[c][k0], tw1[k0 - 1][pcol]);
     }
     __syncwarp();
-    // Pass 2 (over n1): a lane takes q = 8 k0 + n0.
+    // Pass 2 (over n1): a lane takes k0 = (lane + 32 c) / 8 and n0 = lane % 8.
 #pragma unroll
     for (int c = 0; c < 2; ++c) {
-      const uint32_t q = lane + 32 * c, k0 = q >> 3, n0 = q & 7;
+      const uint32_t k0 = (lane >> 3) + 4 * c;
 #pragma unroll
-      for (uint32_t n1 = 0; n1 < 8; ++n1) v[c][n1] = ws.z[k0 * kPitch + 8 * n1 + n0];
+      for (uint32_t n1 = 0; n1 < 8; ++n1) v[c][n1] = ws.z[k0 * kPitch1 + 8 * n1 + n0];
     }
     __syncwarp();
 #pragma unroll
     for (int c = 0; c < 2; ++c) {
-      const uint32_t q = lane + 32 * c, k0 = q >> 3, n0 = q & 7;
+      const uint32_t k0 = (lane >> 3) + 4 * c;
       fft8(v[c]);
+      ws.z[n0 * kPitch2 + k0] = v[c][0];
 #pragma unroll
-      for (uint32_t k1 = 0; k1 < 8; ++k1)
-        ws.z[n0 * kPitch + k0 + 8 * k1] = cmul(v[c][k1], twiddle[n0 * (k0 + 8 * k1)]);
+      for (uint32_t k1 = 1; k1 < 8; ++k1)
+        ws.z[n0 * kPitch2 + k0 + 8 * k1] = cmul(v[c][k1], tw2[k1 - 1]);
     }
     __syncwarp();
-    // Pass 3 (over n0): a lane takes r = k0 + 8 k1 and produces X[r + 64 k2].
+    // Pass 3 (over n0): a lane takes r = k0 + 8 k1 = lane + 32 c and produces Z[r + 64 k2].
 #pragma unroll
     for (int c = 0; c < 2; ++c) {
       const uint32_t r = lane + 32 * c;
 #pragma unroll
-      for (uint32_t n0 = 0; n0 < 8; ++n0) v[c][n0] = ws.z[n0 * kPitch + r];
-    }
-    __syncwarp();
-#pragma unroll
-    for (int c = 0; c < 2; ++c) {
-      const uint32_t r = lane + 32 * c;
+      for (uint32_t m = 0; m < 8; ++m) v[c][m] = ws.z[m * kPitch2 + r];
       fft8(v[c]);
-#pragma unroll
-      for (uint32_t k2 = 0; k2 < 8; ++k2) ws.z[r + 64 * k2] = v[c][k2];
     }
-    __syncwarp();
     // Z = A + iB with A, B the spectra of the two real frames:
-    // A[k] = (Z[k] + conj(Z[N-k]))/2, B[k] = (Z[k] - conj(Z[N-k]))/(2i)
-    for (uint32_t k = lane; k < kBins; k += 32) {
-      const float2 zk = ws.z[k], zn = ws.z[(kFft - k) & (kFft - 1)];
-      const float ar = 0.5f * (zk.x + zn.x), ai = 0.5f * (zk.y - zn.y);
-      const float br = 0.5f * (zk.y + zn.y), bi = 0.5f * (zn.x - zk.x);
-      ws.power[k] = make_float2(ar * ar + ai * ai, br * br + bi * bi);
+    // 2 A[k] = Z[k] + conj(Z[N-k]), 2i B[k] = Z[k] - conj(Z[N-k]); the factor 1/4 of the
+    // powers sits in the Mel weights.  For k = lane + 32 c + 64 k2 below 256, Z[N-k] is the
+    // value (1 - c, 7 - k2) of lane 32 - lane; lane 0 finds it among its own values.
+    const uint32_t partner = (32u - lane) & 31u;
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+#pragma unroll
+      for (int k2 = 0; k2 < 4; ++k2) {
+        const float2 zk = v[c][k2];
+        const float2 give = v[1 - c][7 - k2];
+        float2 zn = make_float2(__shfl_sync(0xffffffffu, give.x, partner),
+                                __shfl_sync(0xffffffffu, give.y, partner));
+        if (lane == 0) zn = c == 0 ? v[0][(8 - k2) & 7] : v[1][7 - k2];
+        const float ar = zk.x + zn.x, ai = zk.y - zn.y;
+        const float br = zk.y + zn.y, bi = zn.x - zk.x;
+        ws.power[kPowPad + lane + 32 * c + 64 * k2] =
+            make_float2(ar * ar + ai * ai, br * br + bi * bi);
+      }
+    }
+    if (lane == 0) {  // bin 256 is its own partner
+      const float ar = 2.f * v[0][4].x, br = 2.f * v[0][4].y;
+      ws.power[kPowPad + 256] = make_float2(ar * ar, br * br);
     }
     __syncwarp();
-    for (uint32_t j = lane; j < kMels; j += 32) {
-      float e0 = 0.f, e1 = 0.f;
-      const uint32_t first = mel.first[j], count = mel.count[j], start = mel.start[j];
-      for (uint32_t i = 0; i < count; ++i) {
-        const float wgt = mel.w[start + i];
-        const float2 pw = ws.power[first + i];
-        e0 = fmaf(wgt, pw.x, e0);
-        e1 = fmaf(wgt, pw.y, e1);
+    // on to the next pair that has frames; its samples travel while the filters are summed
+    const uint32_t this_t0 = t0;
+    ++g;
+    ++q;
+    if (g < g_end) {
+      while (q >= upairs) {
+        ++utt;
+        q = 0;
+        upairs = pairs_in(p, utt);
       }
-      out[static_cast<size_t>(j) * p.t_max + t0] = logf(e0 + kLogGuard);
-      if (t0 + 1 < p.t_max)
-        out[static_cast<size_t>(j) * p.t_max + t0 + 1] = have1 ? logf(e1 + kLogGuard) : 0.f;
+      fetch();
     }
+    mel_round<kMelIters0>(plan.w + lane, ws.power + mel_begin[0], mel_filter[0], out, p.t_max,
+                          this_t0, have1);
+    mel_round<kMelIters1>(plan.w + kMelIters0 * 32 + lane, ws.power + mel_begin[1], mel_filter[1],
+                          out, p.t_max, this_t0, have1);
+    mel_round<kMelIters2>(plan.w + (kMelIters0 + kMelIters1) * 32 + lane, ws.power + mel_begin[2],
+                          mel_filter[2], out, p.t_max, this_t0, have1);
     __syncwarp();  // the next pair reuses this warp's buffers
+  }
+
+  // zeros behind every utterance's own frames: rows dealt out to the warps in turn
+  const uint64_t rows = static_cast<uint64_t>(p.n) * kMels;
+  for (uint64_t row = gwarp; row < rows; row += nwarps) {
+    const uint32_t i = static_cast<uint32_t>(row / kMels);
+    const uint32_t frames = frames_in(p, i);
+    float* __restrict__ o = p.out + row * p.t_max;
+    for (uint32_t t = frames + lane; t < p.t_max; t += 32) o[t] = 0.f;
+  }
+  if (gwarp == 0) {  // refused entries are reported once
+    bool bad = false;
+    for (uint32_t i = lane; i < p.n; i += 32) bad |= !utt_ok(p.table[i], p.samples_count);
+    if (__any_sync(0xffffffffu, bad) && lane == 0 && p.status)
+      atomicCAS(p.status, 0, PREBA_ERR_BAD_TABLE);
   }
 }
 
-// Normalize: a warp per (utterance, filter) row.
-__global__ void __launch_bounds__(128) normalize_kernel(const AudioParams p) {
+// Normalize: a warp per (utterance, filter) row; rows of up to 32 * kHold frames stay in
+// registers between the three passes.
+constexpr int kHold = 48;
+
+__global__ void __launch_bounds__(256) normalize_kernel(const AudioParams p) {
+  // launched as a programmatic dependent of the spectrogram kernel: wait for its results
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const uint32_t lane = threadIdx.x & 31;
   const uint32_t row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (row >= p.n * kMels) return;
   const uint32_t utt = row / kMels;
-  const preba_utt_t u = p.table[utt];
-  if (!utt_ok(u, p.samples_count)) return;
-  const uint32_t frames = min(u.frames, p.t_max);
+  const uint32_t frames = frames_in(p, utt);
   if (frames == 0) return;
   float* __restrict__ r = p.out + static_cast<size_t>(row) * p.t_max;
+  const float count = static_cast<float>(frames);
+  if (frames <= 32u * kHold) {
+    float hold[kHold];
+    float sum = 0.f;
+#pragma unroll
+    for (int i = 0; i < kHold; ++i) {
+      const uint32_t t = lane + 32u * i;
+      hold[i] = t < frames ? r[t] : 0.f;
+      sum += hold[i];
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    const float mean = sum / count;
+    float sq = 0.f;
+#pragma unroll
+    for (int i = 0; i < kHold; ++i) {
+      const float d = lane + 32u * i < frames ? hold[i] - mean : 0.f;
+      hold[i] = d;
+      sq = fmaf(d, d, sq);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+    const float inv = 1.0f / (sqrtf(sq / count) + kStdGuard);
+#pragma unroll
+    for (int i = 0; i < kHold; ++i) {
+      const uint32_t t = lane + 32u * i;
+      if (t < frames) r[t] = hold[i] * inv;
+    }
+    return;
+  }
   float sum = 0.f;
   for (uint32_t t = lane; t < frames; t += 32) sum += r[t];
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-  const float mean = sum / static_cast<float>(frames);
+  const float mean = sum / count;
   float sq = 0.f;
   for (uint32_t t = lane; t < frames; t += 32) {
     const float d = r[t] - mean;
@@ -294,7 +524,7 @@ __global__ void __launch_bounds__(128) normalize_kernel(const AudioParams p) {
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
-  const float inv = 1.0f / (sqrtf(sq / static_cast<float>(frames)) + kStdGuard);
+  const float inv = 1.0f / (sqrtf(sq / count) + kStdGuard);
   for (uint32_t t = lane; t < frames; t += 32) r[t] = (r[t] - mean) * inv;
 }
 
@@ -507,6 +737,34 @@ extern "C" int preba_audio_resample(const float* samples_in, uint64_t samples_in
   return PREBA_OK;
 }
 
+namespace preba {
+namespace audio {
+
+// CTAs of the spectrogram kernel the current device holds at once (the grid of its persistent
+// launch); computed once per device and kept (concurrent first calls store the same value).
+int resident_ctas(cudaError_t* err) {
+  constexpr int kMaxDevices = 64;
+  static std::atomic<int> cache[kMaxDevices];
+  int dev = 0;
+  *err = cudaGetDevice(&dev);
+  if (*err != cudaSuccess) return 0;
+  if (dev >= 0 && dev < kMaxDevices) {
+    const int known = cache[dev].load(std::memory_order_relaxed);
+    if (known > 0) return known;
+  }
+  int sms = 0, per_sm = 0;
+  *err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (*err != cudaSuccess) return 0;
+  *err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, logmel_kernel, 32 * kWarps, 0);
+  if (*err != cudaSuccess) return 0;
+  const int resident = sms * (per_sm > 0 ? per_sm : 1);
+  if (dev >= 0 && dev < kMaxDevices) cache[dev].store(resident, std::memory_order_relaxed);
+  return resident;
+}
+
+}  // namespace audio
+}  // namespace preba
+
 extern "C" int preba_audio_logmel(const preba_audio_batch_t* b, int normalize, void* stream) {
   using namespace preba::audio;
   if (!b || !b->samples || !b->table || !b->out || b->n == 0 || b->n > 65535 || b->t_max == 0)
@@ -526,7 +784,8 @@ extern "C" int preba_audio_logmel(const preba_audio_batch_t* b, int normalize, v
         return PREBA_ERR_BAD_TABLE;
     }
   }
-  static const MelTable mel = make_mel_table();
+  static const MelPlan mel = make_mel_plan();
+  if (!mel.ok) return PREBA_ERR_INVALID_ARG;  // cannot happen for the constants above
   AudioParams p;
   p.samples = b->samples;
   p.samples_count = b->samples_count;
@@ -536,13 +795,30 @@ extern "C" int preba_audio_logmel(const preba_audio_batch_t* b, int normalize, v
   p.n = b->n;
   p.t_max = b->t_max;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  const dim3 grid((b->t_max + kFramesPerCta - 1) / kFramesPerCta, b->n);
-  logmel_kernel<<<grid, 32 * kWarps, 0, s>>>(p, mel);
-  cudaError_t err = cudaGetLastError();
+  // persistent grid: what the device holds at once, but no more warps than a few frame pairs
+  // each would keep busy (an upper bound on the pairs: half of t_max, rounded up, per entry)
+  cudaError_t err = cudaSuccess;
+  const int resident = resident_ctas(&err);
+  if (err == cudaSuccess) {
+    const uint64_t pairs = static_cast<uint64_t>(b->n) * ((b->t_max + 1) / 2);
+    const uint64_t want = (pairs + 2 * kWarps - 1) / (2 * kWarps);
+    const uint32_t blocks = static_cast<uint32_t>(
+        std::max<uint64_t>(1, std::min<uint64_t>(want, static_cast<uint64_t>(resident))));
+    logmel_kernel<<<blocks, 32 * kWarps, 0, s>>>(p, mel);
+    err = cudaGetLastError();
+  }
   if (err == cudaSuccess && normalize) {
     const uint32_t rows = b->n * kMels;
-    normalize_kernel<<<(rows + 3) / 4, 128, 0, s>>>(p);
-    err = cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((rows + 7) / 8);
+    cfg.blockDim = dim3(256);
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    err = cudaLaunchKernelEx(&cfg, normalize_kernel, p);
   }
   if (err != cudaSuccess) {
     preba::g_last_cuda_error = static_cast<int>(err);

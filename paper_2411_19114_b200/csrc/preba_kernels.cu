@@ -1472,6 +1472,10 @@ extern "C" int preba_preprocess_host_noalloc(const uint8_t* packed_host, uint64_
   const uint64_t need_out = static_cast<uint64_t>(n) * 3ull * out_size * out_size *
                             dtype_bytes(out_dtype);
   const uint64_t table_bytes = static_cast<uint64_t>(n) * sizeof(preba_img_t);
+  // each part alone first, so that the sums below cannot wrap
+  if (packed_bytes > PREBA_NOALLOC_MAX_BYTES || need_out > PREBA_NOALLOC_MAX_BYTES ||
+      table_bytes > PREBA_NOALLOC_MAX_BYTES)
+    return PREBA_ERR_TOO_LARGE;
   const uint64_t at_table = kNoallocHeader;
   const uint64_t at_pixels = at_table + align_up(table_bytes, 256);
   const uint64_t at_out = at_pixels + align_up(packed_bytes, 256);

@@ -11,11 +11,15 @@ from oracle import audio as oa
 from paper_2411_19114_b200 import binding as pb
 from paper_2411_19114_b200 import workloads as wl
 
-# fp32 FFT of 512 points, fp32 Mel sums and logf against float64: the weakest Mel band of the
-# test signals lies about 45 dB below the strongest, so its energy carries a relative error up
-# to about 1e-4, which the log turns into the same absolute error (measured 1.2e-4)
-LOGMEL_TOL = 2e-3
-NORM_TOL = 2e-3
+# fp32 FFT of 512 points, fp32 Mel sums and logf against float64.  The transform's error is
+# about 9 roundings (3 radix-8 passes) relative to the norm of the frame's spectrum, 9 * 2^-24 =
+# 5e-7; the weakest Mel band of the test signals lies about 45 dB (3e4 in power, 180 in
+# amplitude) below the strongest, so its energy carries a relative error up to about
+# 2 * 180 * 5e-7 = 2e-4 in the worst case and about 1e-4 typically, which the log turns into
+# the same absolute error (measured 1.2e-4 and 8.6e-5).  The tests allow three times the
+# typical figure.
+LOGMEL_TOL = 3e-4
+NORM_TOL = 3e-4
 
 
 def test_sizes_and_pack_layout():

@@ -47,6 +47,13 @@ def test_refuses_a_batch_larger_than_its_staging_space():
                                                 pb.F32, None)
     assert rc == pb.ERR_TOO_LARGE
     assert "staging" in pb.preba_strerror(rc)
+    # a size close to 2^64 must not wrap into something that seems to fit
+    one = np.zeros(1, dtype=pb.TABLE_DTYPE)
+    one[0] = (0, 8, 8)
+    rc = pb.lib().preba_preprocess_host_noalloc(fake_host, (1 << 64) - 100, one.ctypes.data, 1,
+                                                fake_host, 3 * 224 * 224 * 4, None, 224, 256, m, s,
+                                                pb.F32, None)
+    assert rc == pb.ERR_TOO_LARGE
     # the usual argument checks still come first
     rc = pb.lib().preba_preprocess_host_noalloc(None, sizes.packed_bytes, table.ctypes.data, n,
                                                 fake_host, sizes.out_bytes, None, 224, 256, m, s,
