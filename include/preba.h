@@ -452,6 +452,69 @@ int preba_bucket_batcher_poll(preba_bucket_batcher_t* b, uint64_t now_ns, uint64
                               uint32_t capacity, uint64_t* next_deadline_ns);
 
 /*
+ * preba_serve_run — a measuring aid for the whole front-end under load (paper Sec. 5 "Input
+ * query modeling": single-input requests whose arrival times follow a Poisson process;
+ * Sec. 2.3 item 2 and Sec. 4.3: the batching queue with Batch_max and Time_queue; Sec. 3:
+ * several servers sharing one GPU).  Runs in real time: one thread puts request i into a
+ * preba_batcher queue when the clock reaches arrival_ns[i]; one thread per server polls the
+ * queue, takes the batch that is due, runs it through preba_preprocess_images with
+ * PREBA_IMAGES_IN_PLACE on the server's stream, waits for the stream and stamps the batch's
+ * requests with the completion time.  Requests leave in arrival order, so every batch is a run
+ * of consecutive requests.  Returns when every request has been served.  Unlike the transform's
+ * entry points this one creates threads, a queue and blocks; it allocates nothing on the device.
+ *   arrival_ns        HOST, n_requests times in ns from the start of the run, non-decreasing
+ *   image_index       HOST, n_requests: the pool image request i carries
+ *   pool_images/h/w   HOST arrays of pool_size entries: decoded images in pinned memory as
+ *                     PREBA_IMAGES_IN_PLACE wants them (128-byte aligned, device-addressable)
+ *   batch_max, time_queue_ns   the queue's two hyper-parameters (preba_batching_params)
+ *   n_servers         1..64; table_host, out_host, dev_table, dev_out, dev_status, dev_scratch
+ *                     and streams are arrays of n_servers pointers, one staging set per server
+ *                     as preba_image_batch_t describes them, each sized for batch_max images
+ *                     (dev_status and dev_scratch, or single entries of them, may be NULL)
+ *   out_arena         HOST pinned, n_requests results, or NULL: with it request i's result is
+ *                     kept at i * 3 * out_size^2 * sizeof(element); without it every server
+ *                     writes its batches' results to its own out_host again and again
+ *   done_ns           HOST, n_requests, written: completion time of each request (ns from start)
+ *   batch_size, batch_first, batch_release_ns, batch_server
+ *                     HOST, n_requests entries each, written for batches 0 .. *n_batches - 1 (in
+ *                     no particular order): images in the batch, its first request, the time
+ *                     the queue released it, the server that ran it
+ * Errors: PREBA_ERR_INVALID_ARG, and whatever preba_preprocess_images returns.
+ */
+typedef struct {
+  const uint64_t* arrival_ns;
+  const uint32_t* image_index;
+  uint32_t n_requests;
+  uint32_t pool_size;
+  const uint8_t* const* pool_images;
+  const uint32_t* pool_h;
+  const uint32_t* pool_w;
+  uint32_t batch_max;
+  uint32_t n_servers;
+  uint64_t time_queue_ns;
+  uint32_t out_size;
+  uint32_t resize_short;
+  float mean[3];
+  float std[3];
+  int32_t out_dtype;
+  int32_t device;                /* CUDA device the servers' streams and staging belong to */
+  preba_img_t* const* table_host;
+  void* const* out_host;
+  preba_img_t* const* dev_table;
+  void* const* dev_out;
+  int32_t* const* dev_status;
+  uint32_t* const* dev_scratch;
+  void* const* streams;
+  void* out_arena;
+  uint64_t* done_ns;
+  uint32_t* batch_size;
+  uint32_t* batch_first;
+  uint64_t* batch_release_ns;
+  uint32_t* batch_server;
+} preba_serve_t;
+int preba_serve_run(const preba_serve_t* serve, uint32_t* n_batches);
+
+/*
  * Audio path — the paper's second preprocessing pipeline (Table 1 units "Mel spectrogram" and
  * "Normalize"; Sec. 2.3 item 1: a Fourier transform followed by a Mel filterbank;
  * Sec. 4.2: Normalize as three passes, the mean over all samples, the variance from that mean,

@@ -33,7 +33,8 @@ NOALLOC_MAX_BYTES = 64 << 20
 EXPORTS = ("preba_query", "preba_pack", "preba_preprocess", "preba_preprocess_ex",
            "preba_preprocess_antialias", "preba_preprocess_host",
            "preba_preprocess_images",
-           "preba_preprocess_host_noalloc", "preba_preprocess_repeated", "preba_selftest_wait_limit",
+           "preba_preprocess_host_noalloc", "preba_preprocess_repeated", "preba_serve_run",
+           "preba_selftest_wait_limit",
            "preba_strerror",
            "preba_last_cuda_error",
            "preba_batching_params", "preba_batcher_create", "preba_batcher_destroy",
@@ -86,6 +87,24 @@ class PrebaImageBatch(ctypes.Structure):
                 ("dev_pixels_bytes", ctypes.c_uint64), ("dev_table", ctypes.c_void_p),
                 ("dev_out", ctypes.c_void_p), ("dev_status", ctypes.c_void_p),
                 ("dev_scratch", ctypes.c_void_p)]
+
+
+class PrebaServe(ctypes.Structure):
+    _fields_ = [("arrival_ns", ctypes.c_void_p), ("image_index", ctypes.c_void_p),
+                ("n_requests", ctypes.c_uint32), ("pool_size", ctypes.c_uint32),
+                ("pool_images", ctypes.c_void_p), ("pool_h", ctypes.c_void_p),
+                ("pool_w", ctypes.c_void_p), ("batch_max", ctypes.c_uint32),
+                ("n_servers", ctypes.c_uint32), ("time_queue_ns", ctypes.c_uint64),
+                ("out_size", ctypes.c_uint32), ("resize_short", ctypes.c_uint32),
+                ("mean", ctypes.c_float * 3), ("std", ctypes.c_float * 3),
+                ("out_dtype", ctypes.c_int32), ("device", ctypes.c_int32),
+                ("table_host", ctypes.c_void_p), ("out_host", ctypes.c_void_p),
+                ("dev_table", ctypes.c_void_p), ("dev_out", ctypes.c_void_p),
+                ("dev_status", ctypes.c_void_p), ("dev_scratch", ctypes.c_void_p),
+                ("streams", ctypes.c_void_p), ("out_arena", ctypes.c_void_p),
+                ("done_ns", ctypes.c_void_p), ("batch_size", ctypes.c_void_p),
+                ("batch_first", ctypes.c_void_p), ("batch_release_ns", ctypes.c_void_p),
+                ("batch_server", ctypes.c_void_p)]
 
 
 class PrebaAudioSizes(ctypes.Structure):
@@ -151,6 +170,8 @@ def lib() -> ctypes.CDLL:
                                                 ctypes.c_uint32, f32p, f32p, ctypes.c_int,
                                                 ctypes.c_void_p, ctypes.c_uint32, f32p, f32p]
         L.preba_preprocess_repeated.restype = ctypes.c_int
+        L.preba_serve_run.argtypes = [ctypes.POINTER(PrebaServe), ctypes.POINTER(ctypes.c_uint32)]
+        L.preba_serve_run.restype = ctypes.c_int
         L.preba_selftest_wait_limit.argtypes = [ctypes.c_void_p, ctypes.c_void_p]
         L.preba_selftest_wait_limit.restype = ctypes.c_int
         L.preba_preprocess_host_noalloc.argtypes = [
@@ -551,6 +572,74 @@ def preba_preprocess_host_noalloc(packed_host, table_host: np.ndarray, n: int, o
         ctypes.c_void_p(stream))
     if rc != OK:
         raise PrebaError(rc, "preba_preprocess_host_noalloc")
+
+
+def preba_serve_run(arrival_ns, image_index, pool_images, batch_max: int, time_queue_ns: int,
+                    servers, out_size: int, resize_short: int, mean, std, out_dtype: int,
+                    out_arena=None, device: int = 0) -> dict:
+    """``preba_serve_run``: requests ``i`` arriving at ``arrival_ns[i]`` (ns from the start of the
+    run) carry pool image ``image_index[i]``; ``pool_images`` are pinned, 128-byte aligned uint8
+    CPU tensors (h, w, 3); ``servers`` is a list of dicts with the staging of one server each:
+    ``table_host`` (pinned uint8, 16 bytes per image of a full batch), ``out_host`` (pinned),
+    ``dev_table``, ``dev_out``, optional ``dev_status`` and ``dev_scratch`` (CUDA tensors) and
+    ``stream``.  Blocks until every request is served (the interpreter lock is released).
+    Returns the completion time of every request and the record of the batches."""
+    arr = np.ascontiguousarray(np.asarray(arrival_ns, dtype=np.uint64))
+    idx = _u32(image_index)
+    n, k, v = len(arr), len(pool_images), len(servers)
+    ptrs = (ctypes.c_void_p * k)(*[im.data_ptr() for im in pool_images])
+    ph = _u32([im.shape[0] for im in pool_images])
+    pw = _u32([im.shape[1] for im in pool_images])
+
+    def column(name, optional=False):
+        vals = []
+        for sv in servers:
+            t = sv.get(name)
+            if t is None and not optional:
+                raise ValueError(f"server staging lacks {name}")
+            if t is None:
+                vals.append(None)
+            elif name == "stream":
+                vals.append(t.cuda_stream if hasattr(t, "cuda_stream") else int(t))
+            else:
+                vals.append(t.data_ptr())
+        return (ctypes.c_void_p * v)(*vals)
+
+    cols = {name: column(name, name in ("dev_status", "dev_scratch", "out_host"))
+            for name in ("table_host", "out_host", "dev_table", "dev_out", "dev_status",
+                         "dev_scratch", "stream")}
+    done = np.zeros(n, dtype=np.uint64)
+    b_size, b_first = np.zeros(n, dtype=np.uint32), np.zeros(n, dtype=np.uint32)
+    b_release, b_server = np.zeros(n, dtype=np.uint64), np.zeros(n, dtype=np.uint32)
+    sv = PrebaServe()
+    sv.arrival_ns, sv.image_index = arr.ctypes.data, idx.ctypes.data
+    sv.n_requests, sv.pool_size = n, k
+    sv.pool_images = ctypes.cast(ptrs, ctypes.c_void_p)
+    sv.pool_h, sv.pool_w = ph.ctypes.data, pw.ctypes.data
+    sv.batch_max, sv.n_servers, sv.time_queue_ns = batch_max, v, time_queue_ns
+    sv.out_size, sv.resize_short = out_size, resize_short
+    sv.mean = (ctypes.c_float * 3)(*[float(x) for x in _f3(mean)])
+    sv.std = (ctypes.c_float * 3)(*[float(x) for x in _f3(std)])
+    sv.out_dtype, sv.device = out_dtype, device
+    sv.table_host = ctypes.cast(cols["table_host"], ctypes.c_void_p)
+    sv.out_host = ctypes.cast(cols["out_host"], ctypes.c_void_p)
+    sv.dev_table = ctypes.cast(cols["dev_table"], ctypes.c_void_p)
+    sv.dev_out = ctypes.cast(cols["dev_out"], ctypes.c_void_p)
+    sv.dev_status = ctypes.cast(cols["dev_status"], ctypes.c_void_p)
+    sv.dev_scratch = ctypes.cast(cols["dev_scratch"], ctypes.c_void_p)
+    sv.streams = ctypes.cast(cols["stream"], ctypes.c_void_p)
+    sv.out_arena = out_arena.data_ptr() if out_arena is not None else None
+    sv.done_ns = done.ctypes.data
+    sv.batch_size, sv.batch_first = b_size.ctypes.data, b_first.ctypes.data
+    sv.batch_release_ns, sv.batch_server = b_release.ctypes.data, b_server.ctypes.data
+    nb = ctypes.c_uint32()
+    rc = lib().preba_serve_run(ctypes.byref(sv), ctypes.byref(nb))
+    if rc != OK:
+        raise PrebaError(rc, "preba_serve_run")
+    m = nb.value
+    order = np.argsort(b_first[:m], kind="stable")
+    return {"done_ns": done, "batch_size": b_size[:m][order], "batch_first": b_first[:m][order],
+            "batch_release_ns": b_release[:m][order], "batch_server": b_server[:m][order]}
 
 
 def preba_selftest_wait_limit(status, stream=None) -> None:

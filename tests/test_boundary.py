@@ -47,10 +47,11 @@ def test_header_is_plain_c(tmp_path):
     src = tmp_path / "use_header.c"
     src.write_text(
         '#include "preba.h"\n#include <stdio.h>\n'
-        "int main(void) { printf(\"%zu %zu %zu %zu %zu %zu %zu %zu %zu\\n\", sizeof(preba_img_t), "
+        "int main(void) { printf(\"%zu %zu %zu %zu %zu %zu %zu %zu %zu %zu\\n\", sizeof(preba_img_t), "
         "sizeof(preba_sizes_t), sizeof(preba_batch_t), sizeof(preba_host_batch_t), "
         "sizeof(preba_image_batch_t), sizeof(preba_options_t), sizeof(preba_utt_t), "
-        "sizeof(preba_audio_sizes_t), sizeof(preba_audio_batch_t)); return 0; }\n")
+        "sizeof(preba_audio_sizes_t), sizeof(preba_audio_batch_t), sizeof(preba_serve_t)); "
+        "return 0; }\n")
     exe = tmp_path / "use_header"
     subprocess.run(["gcc", "-std=c11", "-Wall", "-Wextra", "-Werror", "-pedantic",
                     "-I", str(ROOT / "include"), "-o", str(exe), str(src)], check=True)
@@ -60,7 +61,7 @@ def test_header_is_plain_c(tmp_path):
                      ctypes.sizeof(pb.PrebaBatch), ctypes.sizeof(pb.PrebaHostBatch),
                      ctypes.sizeof(pb.PrebaImageBatch), ctypes.sizeof(pb.PrebaOptions),
                      pb.UTT_DTYPE.itemsize, ctypes.sizeof(pb.PrebaAudioSizes),
-                     ctypes.sizeof(pb.PrebaAudioBatch)]
+                     ctypes.sizeof(pb.PrebaAudioBatch), ctypes.sizeof(pb.PrebaServe)]
 
 
 def test_struct_layouts_match_header():
