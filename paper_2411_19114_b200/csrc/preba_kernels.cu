@@ -981,8 +981,11 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
   }
 }
 
+// The rounded modes keep integer row state and division constants on top of what the float
+// mode holds: at four CTAs per SM (128 registers) they spill, so they run three per SM.
 template <typename OutT, int MODE, bool CROP>
-__global__ void __launch_bounds__(kThreads, kCtasPerSm) preba_fused_kernel(const Params p) {
+__global__ void __launch_bounds__(kThreads, MODE == kFloat ? kCtasPerSm : kCtasPerSm - 1)
+    preba_fused_kernel(const Params p) {
   __shared__ WarpShared sm[kWarpsPerCta];
   // a following launch that was marked independent of this one may start as soon as
   // resources free up
