@@ -46,6 +46,9 @@ struct Params {
   uint32_t n, C, S;
   uint32_t rows;         // output rows per CTA
   uint32_t smem_floats;  // shared memory the launch carries, in 4-byte units
+  uint32_t mma_rows;     // output rows per CTA of the tensor-core kernel (<= kMmaRows)
+  uint32_t mma_smem;     // bytes of shared memory of the tensor-core kernel's launch; images it
+                         // can take (mma_plan) are left to it by the other kernel.  0: none are
   float mul[3], add[3];  // y = v * mul + add
 };
 
@@ -160,6 +163,67 @@ __host__ __device__ inline uint32_t ring_slots(const Plan& p, uint32_t floats) {
 // Shared memory (4-byte units) for a ring of `slots` rows.
 __host__ __device__ inline uint64_t plan_floats(const Plan& p, uint64_t slots) {
   return p.off_ring + (slots * (p.seg + 8ull) + 3ull) / 4ull;
+}
+
+// ---- which images the tensor-core kernel (further down) takes ------------------------------------
+
+constexpr uint32_t kMmaRows = 256;    // output rows per CTA, at most
+constexpr uint32_t kGroup = 64;       // output columns per CTA (32 tiles of two)
+constexpr uint32_t kTileBytes = 64;   // bytes of an input row one tile multiplies (two k-steps)
+constexpr uint32_t kMaxTapsX = 20;    // horizontal taps of one column, at most
+constexpr uint32_t kMaxTapsY = 24;    // vertical taps of one row, at most
+constexpr uint32_t kHPlane = 66;      // floats between the channel planes of a row of H
+constexpr uint32_t kHPitch = 200;     // floats between rows of H (3 planes and padding: a warp's
+                                      // stores and loads spread over the banks)
+constexpr uint32_t kHFloats = 16u * kHPitch;  // one tile of H; the kernel keeps two
+constexpr uint32_t kMmaThreads = 256;
+
+struct MmaPlan {
+  uint32_t seg;      // bytes of one staged input row in the ring
+  uint32_t slots;    // 16-row slots of the ring
+  uint32_t off_ring; // byte offsets into the dynamic shared memory
+  uint32_t off_h, off_wx, off_xlo, off_xcnt, off_invx, off_wy, off_ylo, off_ycnt, off_bar;
+};
+
+// Whether the tensor-core kernel takes an image, and its shared-memory layout if so.  The same
+// function decides in both kernels and on the host.
+__host__ __device__ inline bool mma_plan(const Axis& ax, const Axis& ay, uint32_t w, uint32_t C,
+                                         uint32_t smem_bytes, MmaPlan* out) {
+  if (smem_bytes == 0 || (w & 3u) != 0) return false;  // rows must start on the same byte phase
+  if (ax.M > 32767u) return false;                      // weights in two bytes
+  const uint32_t step = (ax.n_in + ax.R - 1u) / ax.R;   // first taps of neighbours differ by <= step
+  if (ax.taps > kMaxTapsX || 3u * (ax.taps + step) + 3u > kTileBytes) return false;
+  if (255ull * ax.taps * 2ull * ax.M >= (1ull << 31)) return false;  // 32-bit sums
+  if (ay.taps > kMaxTapsY || ay.M > 32767u) return false;
+  // a warp finishes an output row before the row 32 further down begins: not for enlargements
+  // beyond about six times
+  if (32ull * ay.n_in < 5ull * ay.R) return false;
+  const uint32_t cols = C < kGroup ? C : kGroup;
+  // pixels under a group: first taps at most ceil((cols - 1) n_in / R) + 1 apart, plus one
+  // column's taps
+  const uint64_t px = (static_cast<uint64_t>(cols - 1u) * ax.n_in + ax.R - 1u) / ax.R + ax.taps + 3u;
+  MmaPlan p;
+  // a staged row: up to 15 bytes of skew, the bytes under the group, the overshoot of the last
+  // tile; 16 modulo 128, so that the eight rows a warp reads together lie four banks apart
+  p.seg = static_cast<uint32_t>(((16u + 3u * px + kTileBytes + 111u) & ~127ull) + 16u);
+  uint32_t at = 0;
+  p.off_h = at, at += 2u * kHFloats * 4u;
+  p.off_wx = at, at += kGroup * kMaxTapsX * 2u;
+  p.off_xlo = at, at += kGroup * 4u;
+  p.off_xcnt = at, at += kGroup * 4u;
+  p.off_invx = at, at += kGroup * 4u;
+  p.off_wy = at, at += kMmaRows * kMaxTapsY * 4u;
+  p.off_ylo = at, at += kMmaRows * 4u;
+  p.off_ycnt = at, at += kMmaRows * 4u;
+  p.off_bar = at, at += 64u;
+  at = (at + 15u) & ~15u;
+  p.off_ring = at;
+  if (smem_bytes <= at) return false;
+  const uint64_t room = (smem_bytes - at) / (16ull * p.seg);
+  if (room < 2) return false;
+  p.slots = room > 4 ? 4u : static_cast<uint32_t>(room);
+  if (out) *out = p;
+  return true;
 }
 
 __device__ __forceinline__ void report(int32_t* status, int code) {
@@ -384,6 +448,7 @@ __global__ void __launch_bounds__(kThreads) preba_antialias_kernel(const Params 
     left = (rw - C) / 2;
   }
   const Axis ax = make_axis(e.w, rw), ay = make_axis(e.h, rh);
+  if (mma_plan(ax, ay, e.w, C, p.mma_smem, nullptr)) return;  // the tensor-core kernel's image
   const Plan pl = make_plan(ax, ay, C, p.rows);
   if (pl.off_ring > p.smem_floats) {
     if (tid == 0) report(p.status, PREBA_ERR_TOO_LARGE);
@@ -598,6 +663,339 @@ __global__ void __launch_bounds__(kThreads) preba_antialias_kernel(const Params 
   }
 }
 
+
+// ---- the tensor-core path ---------------------------------------------------------------------------
+//
+// The horizontal pass is a banded matrix product: H[row][(X, ch)] = sum_b p[row][b] W[b][(X, ch)],
+// b the byte position in the input row (b = 3 j + ch), W the integer triangle weight of pixel j
+// for resized pixel X.  It runs as integer matrix instructions (m16n8k32, 8-bit operands, 32-bit
+// sums, exact): 16 input rows by 64 bytes of a row against the weights of two resized pixels
+// times three channels (six of the eight columns), the weights split into their high and low
+// bytes (two instructions per 32 bytes, joined by a shift of the high sums).  The input rows
+// are the A operand exactly as they lie in memory, so no byte is shuffled; the weights are the
+// B operand, built once per warp and kept in registers.  The vertical pass then runs in fp32 on
+// the 16 x 192 tile of H a CTA has just made (shared memory): output row y of the CTA belongs
+// to warp y % 8, a lane has two columns per channel, and a warp adds the tile's rows under the
+// taps of the rows it has in progress; a row whose last tap has passed is normalised and
+// stored.
+//
+// A CTA makes up to kMmaRows output rows by kGroup columns of one image in one sweep over the
+// input rows underneath, sixteen at a time, through a ring of bulk copies.
+
+__device__ __forceinline__ void mma_u8(int32_t (&d)[4], const uint32_t (&a)[4], uint32_t b0,
+                                       uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k32.row.col.s32.u8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+      "{%0,%1,%2,%3};"
+      : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// Taps of resized pixel X on an axis the tensor-core kernel admits (M <= 32767, so every term
+// fits 32 bits): [lo, hi), as tap_range.
+__device__ __forceinline__ void tap_range32(const Axis& a, uint32_t X, uint32_t* lo, uint32_t* hi) {
+  const uint32_t centre = (2u * X + 1u) * a.n_in, m2 = 2u * a.M, r2 = 2u * a.R;
+  const uint32_t first = centre >= m2 + a.R ? (centre - m2 - a.R) / r2 + 1u : 0u;
+  const uint32_t last = (centre + m2 + a.R - 1u) / r2;
+  *lo = first;
+  *hi = last < a.n_in ? last : a.n_in;
+}
+
+__device__ __forceinline__ uint32_t tap_weight32(const Axis& a, uint32_t X, uint32_t j) {
+  const int32_t d = static_cast<int32_t>((2u * j + 1u) * a.R) -
+                    static_cast<int32_t>((2u * X + 1u) * a.n_in);
+  const int32_t w = static_cast<int32_t>(2u * a.M) - (d < 0 ? -d : d);
+  return w > 0 ? static_cast<uint32_t>(w) : 0u;
+}
+
+template <typename OutT>
+__global__ void __launch_bounds__(kMmaThreads, 2) preba_antialias_mma_kernel(const Params p) {
+  extern __shared__ __align__(16) uint8_t smem_b[];
+  const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5, C = p.C;
+  const uint32_t chunks = (C + p.mma_rows - 1) / p.mma_rows, groups = (C + kGroup - 1) / kGroup;
+  const uint32_t img = blockIdx.x / (chunks * groups);
+  const uint32_t rest = blockIdx.x - img * chunks * groups;
+  const uint32_t k0 = (rest / groups) * p.mma_rows, xg0 = (rest % groups) * kGroup;
+  const preba_img_t e = p.table[img];
+  const uint64_t usable = p.pixels_bytes & ~15ull;
+  if (e.h < 1 || e.w < 1 || e.h > PREBA_MAX_DIM || e.w > PREBA_MAX_DIM ||
+      e.offset % PREBA_PACK_ALIGN != 0 || e.offset > usable ||
+      3ull * e.h * e.w > usable - e.offset) {
+    if (tid == 0 && rest == 0) report(p.status, PREBA_ERR_BAD_TABLE);
+    return;
+  }
+  uint32_t rh, rw, top, left;
+  resized_size(e.h, e.w, p.S, &rh, &rw);
+  if (p.crop) {
+    top = p.crop[2 * img];
+    left = p.crop[2 * img + 1];
+    if (static_cast<uint64_t>(top) + C > rh || static_cast<uint64_t>(left) + C > rw) {
+      if (tid == 0 && rest == 0) report(p.status, PREBA_ERR_BAD_CROP);
+      return;
+    }
+  } else {
+    top = (rh - C) / 2;
+    left = (rw - C) / 2;
+  }
+  const Axis ax = make_axis(e.w, rw), ay = make_axis(e.h, rh);
+  MmaPlan pl;
+  if (!mma_plan(ax, ay, e.w, C, p.mma_smem, &pl)) return;  // the other kernel's image
+
+  float* hbuf = reinterpret_cast<float*>(smem_b + pl.off_h);
+  uint16_t* wxi = reinterpret_cast<uint16_t*>(smem_b + pl.off_wx);
+  uint32_t* xlo = reinterpret_cast<uint32_t*>(smem_b + pl.off_xlo);
+  uint32_t* xcnt = reinterpret_cast<uint32_t*>(smem_b + pl.off_xcnt);
+  float* invx = reinterpret_cast<float*>(smem_b + pl.off_invx);
+  float* wyn = reinterpret_cast<float*>(smem_b + pl.off_wy);
+  uint32_t* ylo = reinterpret_cast<uint32_t*>(smem_b + pl.off_ylo);
+  uint32_t* ycnt = reinterpret_cast<uint32_t*>(smem_b + pl.off_ycnt);
+  const uint32_t bars = smem_addr(smem_b + pl.off_bar);
+  const uint32_t ring = smem_addr(smem_b + pl.off_ring);
+  const uint32_t ncols = C - xg0 < kGroup ? C - xg0 : kGroup;
+  const uint32_t nrows = C - k0 < p.mma_rows ? C - k0 : p.mma_rows;
+
+  // tables: a thread per row of the CTA, and per column of the group
+  if (tid < nrows) {
+    const uint32_t Y = top + k0 + tid;
+    uint32_t j0, j1;
+    tap_range32(ay, Y, &j0, &j1);
+    uint32_t sum = 0;
+    for (uint32_t j = j0; j < j1; ++j) sum += tap_weight32(ay, Y, j);
+    const float inv = 1.0f / static_cast<float>(sum);
+    for (uint32_t j = j0; j < j1; ++j)
+      wyn[tid * kMaxTapsY + (j - j0)] = static_cast<float>(tap_weight32(ay, Y, j)) * inv;
+    ylo[tid] = j0;
+    ycnt[tid] = j1 - j0;
+  }
+  if (tid < kGroup) {
+    uint32_t j0 = 0, j1 = 0;
+    float inv = 0.f;
+    if (tid < ncols) {
+      const uint32_t X = left + xg0 + tid;
+      tap_range32(ax, X, &j0, &j1);
+      uint32_t sum = 0;
+      for (uint32_t j = j0; j < j1; ++j) {
+        const uint32_t wgt = tap_weight32(ax, X, j);
+        wxi[tid * kMaxTapsX + (j - j0)] = static_cast<uint16_t>(wgt);
+        sum += wgt;
+      }
+      inv = 1.0f / static_cast<float>(sum);
+    }
+    xlo[tid] = j0;
+    xcnt[tid] = j1 - j0;
+    invx[tid] = inv;
+  }
+  if (tid == 0) {
+    for (uint32_t s = 0; s < pl.slots; ++s) mbar_init(bars + 8u * s, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  // the bytes of an input row under the group, and the input rows under the CTA's output rows
+  const uint32_t rowbyte0 = 3u * xlo[0];
+  const uint32_t rowbytes = 3u * (xlo[ncols - 1] + xcnt[ncols - 1]) - rowbyte0;
+  const uint32_t ya = ylo[0], yb = ylo[nrows - 1] + ycnt[nrows - 1];
+  const uint32_t ntiles16 = (yb - ya + 15u) / 16u;
+  const uint8_t* image = p.pixels + e.offset;
+  const uint8_t* stop = p.pixels + usable;
+  const uint64_t pitch = 3ull * e.w;
+  if (16u + rowbytes + kTileBytes > pl.seg) {  // cannot happen within the plan's bounds
+    if (tid == 0) report(p.status, PREBA_ERR_TOO_LARGE);
+    return;
+  }
+  // rows start on the same byte phase (the pitch is a multiple of 4)
+  const uint32_t skew4 = static_cast<uint32_t>(reinterpret_cast<uintptr_t>(image + rowbyte0)) & 3u;
+
+  // thread 0 asks for the 16 rows of tile m (those the CTA needs)
+  auto issue = [&](uint32_t m) {
+    const uint32_t slot = m % pl.slots, bar = bars + 8u * slot;
+    uint32_t total = 0;
+    const uint32_t r0 = ya + 16u * m;
+    for (uint32_t i = 0; i < 16u && r0 + i < yb; ++i) {
+      const uint8_t* src = image + (r0 + i) * pitch + rowbyte0;
+      const uint32_t skew = static_cast<uint32_t>(reinterpret_cast<uintptr_t>(src)) & 15u;
+      uint32_t bytes = (skew + rowbytes + 15u) & ~15u;
+      if (bytes > static_cast<uint64_t>(stop - (src - skew)))  // only padding is lost
+        bytes = static_cast<uint32_t>(stop - (src - skew));
+      total += bytes;
+    }
+    mbar_arrive_expect_tx(bar, total);
+    for (uint32_t i = 0; i < 16u && r0 + i < yb; ++i) {
+      const uint8_t* src = image + (r0 + i) * pitch + rowbyte0;
+      const uint32_t skew = static_cast<uint32_t>(reinterpret_cast<uintptr_t>(src)) & 15u;
+      uint32_t bytes = (skew + rowbytes + 15u) & ~15u;
+      if (bytes > static_cast<uint64_t>(stop - (src - skew)))
+        bytes = static_cast<uint32_t>(stop - (src - skew));
+      bulk_copy_g2s(ring + (slot * 16u + i) * pl.seg, src - skew, bytes, bar);
+    }
+  };
+  if (tid == 0)
+    for (uint32_t m = 0; m < pl.slots && m < ntiles16; ++m) issue(m);
+
+  // the weights of this warp's four tiles as B operands: for k-step s, register r, byte i the
+  // row position kst + 32 s + 16 r + 4 q + i, for column g = 2 ch + xi the pixel X0 + xi
+  const uint32_t g = lane >> 2, q = lane & 3u;
+  uint32_t bhi[4][2][2], blo[4][2][2];
+  int32_t kst[4];
+#pragma unroll
+  for (uint32_t t = 0; t < 4; ++t) {
+    const uint32_t col0 = 2u * (4u * warp + t);  // first column of the tile in the group
+    int32_t start = 0;
+    if (col0 < ncols) {
+      const int32_t nb = static_cast<int32_t>(3u * xlo[col0] - rowbyte0);
+      start = nb - static_cast<int32_t>((static_cast<uint32_t>(nb) + skew4) & 3u);
+    }
+    kst[t] = start;
+    const uint32_t ch = g >> 1, col = col0 + (g & 1u);
+    const bool live = g < 6u && col < ncols;
+    const uint32_t lo_px = live ? xlo[col] : 0u, n_px = live ? xcnt[col] : 0u;
+#pragma unroll
+    for (uint32_t s2 = 0; s2 < 2; ++s2)
+#pragma unroll
+      for (uint32_t r = 0; r < 2; ++r) {
+        uint32_t hi = 0, lo = 0;
+#pragma unroll
+        for (uint32_t i = 0; i < 4; ++i) {
+          const int32_t b = static_cast<int32_t>(rowbyte0) + start +
+                            static_cast<int32_t>(32u * s2 + 16u * r + 4u * q + i);
+          uint32_t wgt = 0;
+          if (b >= 0) {
+            const uint32_t px = static_cast<uint32_t>(b) / 3u;
+            if (static_cast<uint32_t>(b) - 3u * px == ch && px >= lo_px && px - lo_px < n_px)
+              wgt = wxi[col * kMaxTapsX + (px - lo_px)];
+          }
+          hi |= (wgt >> 8) << (8u * i);
+          lo |= (wgt & 0xffu) << (8u * i);
+        }
+        bhi[t][s2][r] = hi;
+        blo[t][s2][r] = lo;
+      }
+  }
+
+  // the vertical pass's state: the warp's output rows are warp, warp + 8, ...; row number n of
+  // them uses accumulator n % 4 (a row is finished before the row 32 further down begins);
+  // columns lane and lane + 32 of the group, three channels
+  float acc[4][3][2];
+  uint32_t cur[4];
+#pragma unroll
+  for (uint32_t a = 0; a < 4; ++a) {
+    cur[a] = warp + 8u * a;
+#pragma unroll
+    for (uint32_t c = 0; c < 3; ++c) acc[a][c][0] = acc[a][c][1] = 0.f;
+  }
+  OutT* out = static_cast<OutT*>(p.out) + static_cast<uint64_t>(img) * 3u * C * C;
+  const float sx0 = lane < ncols ? invx[lane] : 0.f;
+  const float sx1 = lane + 32u < ncols ? invx[lane + 32u] : 0.f;
+
+  // horizontal pass of tile m: H = rows x weights on the tensor cores, into buffer m % 2
+  auto horizontal = [&](uint32_t m) {
+    const uint32_t slot = m % pl.slots, r0 = ya + 16u * m;
+    float* hb = hbuf + (m & 1u) * kHFloats;
+    // rows g and g + 8 of the tile: where their first needed byte lies in the slot
+    const uint32_t sk0 = static_cast<uint32_t>(
+        reinterpret_cast<uintptr_t>(image + (r0 + g) * pitch + rowbyte0)) & 15u;
+    const uint32_t sk1 = static_cast<uint32_t>(
+        reinterpret_cast<uintptr_t>(image + (r0 + g + 8u) * pitch + rowbyte0)) & 15u;
+    const uint32_t row0 = ring + (slot * 16u + g) * pl.seg + sk0 + 4u * q;
+    const uint32_t row1 = ring + (slot * 16u + g + 8u) * pl.seg + sk1 + 4u * q;
+#pragma unroll
+    for (uint32_t t = 0; t < 4; ++t) {
+      const uint32_t tile = 4u * warp + t;
+      if (2u * tile >= ncols) break;
+      uint32_t a[2][4];
+#pragma unroll
+      for (uint32_t s2 = 0; s2 < 2; ++s2) {
+        const uint32_t at0 = row0 + kst[t] + 32u * s2, at1 = row1 + kst[t] + 32u * s2;
+        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(a[s2][0]) : "r"(at0));
+        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(a[s2][1]) : "r"(at1));
+        asm volatile("ld.shared.u32 %0, [%1+16];" : "=r"(a[s2][2]) : "r"(at0));
+        asm volatile("ld.shared.u32 %0, [%1+16];" : "=r"(a[s2][3]) : "r"(at1));
+      }
+      int32_t d[4] = {0, 0, 0, 0};
+      mma_u8(d, a[0], bhi[t][0][0], bhi[t][0][1]);
+      mma_u8(d, a[1], bhi[t][1][0], bhi[t][1][1]);
+#pragma unroll
+      for (uint32_t i = 0; i < 4; ++i) d[i] <<= 8;
+      mma_u8(d, a[0], blo[t][0][0], blo[t][0][1]);
+      mma_u8(d, a[1], blo[t][1][0], blo[t][1][1]);
+      if (q < 3u) {  // columns 2 q and 2 q + 1: channel q of the tile's two pixels
+        float2* h0 = reinterpret_cast<float2*>(hb + g * kHPitch + q * kHPlane + 2u * tile);
+        float2* h1 = reinterpret_cast<float2*>(hb + (g + 8u) * kHPitch + q * kHPlane + 2u * tile);
+        *h0 = make_float2(static_cast<float>(d[0]), static_cast<float>(d[1]));
+        *h1 = make_float2(static_cast<float>(d[2]), static_cast<float>(d[3]));
+      }
+    }
+  };
+
+  // Tile m + 1 goes through the tensor cores while tile m's H is summed vertically: one CTA-wide
+  // barrier per tile, and the wait for a tile's rows comes a whole step before they are needed.
+  // Only lane 0 of a warp polls the copies' barrier.
+  bool failed = false;
+  auto arrived = [&](uint32_t m) {
+    uint32_t ok = 1u;
+    if (lane == 0) ok = mbar_wait(bars + 8u * (m % pl.slots), (m / pl.slots) & 1u) ? 1u : 0u;
+    return __shfl_sync(0xffffffffu, ok, 0) != 0u;
+  };
+  if (!arrived(0)) failed = true;
+  failed = __syncthreads_or(failed) != 0;
+  if (!failed) horizontal(0);
+  __syncthreads();
+  for (uint32_t m = 0; m < ntiles16 && !failed; ++m) {
+    const uint32_t r0 = ya + 16u * m;
+    if (m + 1 < ntiles16) {
+      if (arrived(m + 1)) horizontal(m + 1);
+      else failed = true;
+    }
+    // ---- vertical pass: the tile's rows under the taps of the warp's rows in progress ----
+    const float* hb = hbuf + (m & 1u) * kHFloats;
+#pragma unroll
+    for (uint32_t a = 0; a < 4; ++a) {
+      for (;;) {
+        const uint32_t yl = cur[a];
+        if (yl >= nrows) break;
+        const uint32_t y0 = ylo[yl], y1 = y0 + ycnt[yl];
+        if (y0 >= r0 + 16u) break;  // begins in a later tile
+        const uint32_t from = y0 > r0 ? y0 : r0, to = y1 < r0 + 16u ? y1 : r0 + 16u;
+        for (uint32_t r = from; r < to; ++r) {
+          const float wgt = wyn[yl * kMaxTapsY + (r - y0)];
+          const float* h = hb + (r - r0) * kHPitch + lane;
+#pragma unroll
+          for (uint32_t c = 0; c < 3; ++c) {
+            acc[a][c][0] = fmaf(wgt, h[c * kHPlane], acc[a][c][0]);
+            acc[a][c][1] = fmaf(wgt, h[c * kHPlane + 32u], acc[a][c][1]);
+          }
+        }
+        if (y1 > r0 + 16u) break;  // goes on in the next tile
+        // the row's last tap has passed: normalise, store, on to the warp's row 32 further down
+#pragma unroll
+        for (uint32_t c = 0; c < 3; ++c) {
+          const uint64_t at = (static_cast<uint64_t>(c) * C + (k0 + yl)) * C + xg0 + lane;
+          if (lane < ncols) out[at] = to_out<OutT>(fmaf(acc[a][c][0] * sx0, p.mul[c], p.add[c]));
+          if (lane + 32u < ncols)
+            out[at + 32u] = to_out<OutT>(fmaf(acc[a][c][1] * sx1, p.mul[c], p.add[c]));
+          acc[a][c][0] = acc[a][c][1] = 0.f;
+        }
+        cur[a] = yl + 32u;
+      }
+    }
+    // tile m + 1's H is complete, tile m's has been read, and so have the staged rows of tile
+    // m + 1: their slot takes the rows of tile m + 1 + slots
+    failed = __syncthreads_or(failed) != 0;
+    if (tid == 0 && !failed && m + 1 + pl.slots < ntiles16) {
+      fence_async_shared();
+      issue(m + 1 + pl.slots);
+    }
+  }
+  if (failed && tid == 0) {
+    report(p.status, PREBA_ERR_TIMEOUT);
+    // copies already asked for may still be landing in the ring: wait for them (bounded)
+    for (uint32_t s = 0; s < pl.slots; ++s) {
+      (void)mbar_wait(bars + 8u * s, 0u);
+      (void)mbar_wait(bars + 8u * s, 1u);
+    }
+  }
+}
+
 }  // namespace aa
 }  // namespace preba
 
@@ -613,6 +1011,16 @@ Kernel kernel_for(int out_dtype) {
                                   : preba::aa::preba_antialias_kernel<__nv_bfloat16>;
 }
 
+Kernel mma_kernel_for(int out_dtype) {
+  return out_dtype == PREBA_F32   ? preba::aa::preba_antialias_mma_kernel<float>
+         : out_dtype == PREBA_F16 ? preba::aa::preba_antialias_mma_kernel<__half>
+                                  : preba::aa::preba_antialias_mma_kernel<__nv_bfloat16>;
+}
+
+// Shared memory of the tensor-core kernel's launch: its tables, a tile of H and a ring of three
+// 16-row slots of 1080p-wide groups fit, and two CTAs share an SM.
+constexpr int kMmaSmemBytes = 108 * 1024;
+
 // Largest dynamic shared memory a CTA may ask for on the current device; the three kernels
 // are opted in to it once per device.
 int shared_memory_limit(cudaError_t* err) {
@@ -627,10 +1035,14 @@ int shared_memory_limit(cudaError_t* err) {
   }
   int optin = 0;
   *err = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
-  for (int dt : {PREBA_F32, PREBA_F16, PREBA_BF16})
+  for (int dt : {PREBA_F32, PREBA_F16, PREBA_BF16}) {
     if (*err == cudaSuccess)
       *err = cudaFuncSetAttribute(kernel_for(dt), cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   optin);
+    if (*err == cudaSuccess)
+      *err = cudaFuncSetAttribute(mma_kernel_for(dt), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  optin < kMmaSmemBytes ? optin : kMmaSmemBytes);
+  }
   if (*err != cudaSuccess) return 0;
   if (dev >= 0 && dev < kMaxDevices) cache[dev].store(optin, std::memory_order_relaxed);
   return optin;
@@ -674,8 +1086,14 @@ extern "C" int preba_preprocess_antialias(const preba_batch_t* batch, const preb
   const uint32_t limit_floats = static_cast<uint32_t>(limit) / 4u;
   uint32_t floats = limit_floats;
   const uint32_t most_rows = C + 1 < kMaxRows ? (C + 1u) & ~1u : kMaxRows;  // no CTA makes more
+  // Two kernels share the batch: the tensor-core kernel takes the images mma_plan admits, the
+  // other one the rest; each skips the other's images.  With the host's copy of the table a
+  // kernel without images is not launched at all.
+  const uint32_t mma_smem = static_cast<uint32_t>(limit < kMmaSmemBytes ? limit : kMmaSmemBytes);
+  bool any_mma = true, any_rest = true;
   if (batch->table_host) {
     uint64_t most = 0;
+    any_mma = any_rest = false;
     for (uint32_t i = 0; i < batch->n; ++i) {
       const preba_img_t& e = batch->table_host[i];
       // as in the kernel: rows are fetched in 16-byte units, so the buffer counts up to its
@@ -690,6 +1108,11 @@ extern "C" int preba_preprocess_antialias(const preba_batch_t* batch, const preb
           (opt->crop_origin_host[2 * i] + static_cast<uint64_t>(C) > rh ||
            opt->crop_origin_host[2 * i + 1] + static_cast<uint64_t>(C) > rw))
         return PREBA_ERR_BAD_CROP;
+      if (mma_plan(make_axis(e.w, rw), make_axis(e.h, rh), e.w, C, mma_smem, nullptr)) {
+        any_mma = true;
+        continue;
+      }
+      any_rest = true;
       const Plan pl = make_plan(make_axis(e.w, rw), make_axis(e.h, rh), C, most_rows);
       if (pl.off_ring > limit_floats) return PREBA_ERR_TOO_LARGE;
       // with a ring of staged rows (one pair's rows and half as many again in flight) when
@@ -699,6 +1122,7 @@ extern "C" int preba_preprocess_antialias(const preba_batch_t* batch, const preb
       if (want > most) most = want;
     }
     if (most < floats) floats = static_cast<uint32_t>(most);
+    if (!any_rest) floats = 0;
   }
   // Rows per CTA: the CTAs of one image are cut so that the batch fills a whole number of
   // rounds of the CTAs the GPU holds at once (a round more than needed would run nearly
@@ -732,14 +1156,39 @@ extern "C" int preba_preprocess_antialias(const preba_batch_t* batch, const preb
   p.S = S;
   p.rows = rows;
   p.smem_floats = floats;
+  p.mma_smem = any_mma ? mma_smem : 0u;
+  // Output rows per CTA of the tensor-core kernel: a CTA builds its weight operands once and
+  // then sweeps, so it takes as many rows as it can (all of them up to kMmaRows) unless the
+  // batch then has fewer CTAs than the GPU holds at once.
+  {
+    const uint64_t groups = (C + kGroup - 1) / kGroup;
+    const uint64_t room = 2ull * sms / (static_cast<uint64_t>(batch->n) * groups);  // chunks that fit at once
+    uint64_t chunks = (C + kMmaRows - 1) / kMmaRows;
+    if (room > chunks) chunks = room;
+    const uint64_t most_chunks = (C + 31u) / 32u;  // no CTA below 32 rows
+    if (chunks > most_chunks) chunks = most_chunks;
+    uint32_t r = static_cast<uint32_t>((C + chunks - 1) / chunks);
+    r = (r + 7u) & ~7u;
+    p.mma_rows = r > kMmaRows ? kMmaRows : r;
+  }
   for (int c = 0; c < 3; ++c) {
     p.mul[c] = static_cast<float>(1.0 / (255.0 * static_cast<double>(opt->std[c])));
     p.add[c] = static_cast<float>(-static_cast<double>(opt->mean[c]) /
                                   static_cast<double>(opt->std[c]));
   }
-  const uint32_t grid = batch->n * ((C + rows - 1) / rows);
-  kernel_for(opt->out_dtype)<<<grid, kThreads, floats * 4u, static_cast<cudaStream_t>(stream)>>>(p);
-  err = cudaGetLastError();
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (any_mma) {
+    const uint64_t ctas = static_cast<uint64_t>(batch->n) * ((C + p.mma_rows - 1) / p.mma_rows) *
+                          ((C + kGroup - 1) / kGroup);
+    if (ctas > 0x7fffffffull) return PREBA_ERR_INVALID_ARG;
+    mma_kernel_for(opt->out_dtype)<<<static_cast<uint32_t>(ctas), kMmaThreads, mma_smem, s>>>(p);
+    err = cudaGetLastError();
+  }
+  if (any_rest && err == cudaSuccess) {
+    const uint32_t grid = batch->n * ((C + rows - 1) / rows);
+    kernel_for(opt->out_dtype)<<<grid, kThreads, floats * 4u, s>>>(p);
+    err = cudaGetLastError();
+  }
   if (err != cudaSuccess) {
     g_last_cuda_error = static_cast<int>(err);
     return PREBA_ERR_CUDA;

@@ -80,6 +80,25 @@ def test_ragged_batch_fp32_centre_crop():
     assert np.all(err <= 1e-5), err
 
 
+# widths that are multiples of 4 (rows start on the same byte phase: the images the
+# tensor-core kernel takes), with row pitches of every residue modulo 16, reduced up to 5 times,
+# not at all, and enlarged
+MMA_SHAPES = [(1080, 1920), (771, 1028), (600, 808), (333, 444), (250, 1000), (900, 400),
+              (256, 256), (1280, 1284), (120, 160), (517, 1372)]
+
+
+@pytest.mark.parametrize("c,s", [(224, 256), (100, 130), (65, 65), (33, 300), (288, 320)])
+def test_images_of_the_tensor_core_kernel(c, s):
+    images = [uniform(150 + i, h, w) for i, (h, w) in enumerate(MMA_SHAPES)]
+    got = run(images, c, s)
+    err = np.max(np.abs(got - want(images, c, s)), axis=(1, 2, 3))
+    assert np.all(err <= 1e-5), err
+    origins = origins_for(images, c, s, 11)
+    got = run(images, c, s, origins=origins, with_host_table=False)
+    err = np.max(np.abs(got - want(images, c, s, origins)), axis=(1, 2, 3))
+    assert np.all(err <= 1e-5), err
+
+
 @pytest.mark.parametrize("c,s", [(224, 256), (96, 96), (17, 40), (1, 1), (299, 342)])
 def test_other_output_sizes(c, s):
     images = [uniform(200 + i, h, w) for i, (h, w) in enumerate(SHAPES[:7])]
@@ -189,11 +208,13 @@ def test_a_window_off_the_grid_is_skipped_and_reported_by_the_kernel():
 
 
 def test_an_image_reduced_beyond_the_working_set_is_refused():
-    """One 11,600 x 11,600 image at out_size = resize_short = 2,320 needs more shared memory
-    than a block can have: refused on the host with the table, reported by the kernel without."""
+    """One 11,601 x 11,601 image at out_size = resize_short = 2,320 needs more shared memory
+    than a block can have (its width is not a multiple of 4, so the tensor-core kernel, which
+    works on column groups and needs far less, does not take it): refused on the host with the
+    table, reported by the kernel without."""
     import torch
 
-    side, c = 11600, 2320
+    side, c = 11601, 2320
     dev = torch.device("cuda:0")
     pix = torch.zeros(3 * side * side + 128, dtype=torch.uint8, device=dev)
     table = np.zeros(1, dtype=pb.TABLE_DTYPE)
@@ -208,3 +229,11 @@ def test_an_image_reduced_beyond_the_working_set_is_refused():
     torch.cuda.synchronize()
     assert int(status.item()) == pb.ERR_TOO_LARGE
     assert bool(torch.all(out == 7.0))
+
+
+def test_a_large_image_of_the_tensor_core_kernel():
+    """11,600 x 2,000 pixels reduced five times to 2,320 x 400, crop 400: column groups and
+    bands beyond the first, rows far apart in memory."""
+    images = [uniform(950, 2000, 11600)]
+    got = run(images, 400, 400)
+    assert np.max(np.abs(got - want(images, 400, 400))) <= 1e-5
