@@ -266,13 +266,18 @@ int preba_preprocess_ex(const preba_batch_t* batch, const preba_options_t* opt, 
  * the two-tap interpolation of preba_preprocess.  Integer taps and weights, fp32 sums.
  * `opt` is read as by preba_preprocess_ex (crop windows included) with flags == 0 and a float
  * out_dtype; batch layout, table checks and status word are those of preba_preprocess;
- * batch->scratch is not used and PREBA_OVERLAP_PREVIOUS has no effect.  One kernel is
- * enqueued on `stream`.
- * A CTA keeps one channel-planar row of the window's footprint and the weight tables in
- * shared memory; with `table_host` the launch carries what the largest image needs and an
- * image that needs more than the device allows is refused (PREBA_ERR_TOO_LARGE: reductions
- * beyond about 40 at out_size 224); without it the launch carries all the device allows and
- * the kernel skips and reports such an image in the status word.
+ * batch->scratch is not used and PREBA_OVERLAP_PREVIOUS has no effect.
+ * Two kernels share the work, each skipping the other's images.  Images whose width is a
+ * multiple of 4 and that are reduced up to about six times (or enlarged up to about six times)
+ * go to a kernel that runs the horizontal pass as integer matrix instructions on the tensor
+ * cores (the input rows as they lie in memory against the integer weights, exact) and the
+ * vertical pass in fp32.  Every other image goes to a kernel in which a CTA keeps one
+ * channel-planar row of the window's footprint and the weight tables in shared memory.  With
+ * `table_host` only the kernels that have images are enqueued on `stream` (one or two), the
+ * second kernel's launch carries what its largest image needs, and an image that needs more
+ * than the device allows is refused (PREBA_ERR_TOO_LARGE: reductions beyond about 40 at
+ * out_size 224); without it both kernels are enqueued, the second carries all the device
+ * allows and skips and reports such an image in the status word.
  * Errors: PREBA_ERR_INVALID_ARG, PREBA_ERR_BUFFER_TOO_SMALL, PREBA_ERR_BAD_TABLE,
  * PREBA_ERR_BAD_CROP, PREBA_ERR_TOO_LARGE, PREBA_ERR_CUDA.
  */

@@ -328,6 +328,10 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
 
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
                : "memory");
@@ -786,7 +790,7 @@ __global__ void __launch_bounds__(kMmaThreads, 2) preba_antialias_mma_kernel(con
     invx[tid] = inv;
   }
   if (tid == 0) {
-    for (uint32_t s = 0; s < pl.slots; ++s) mbar_init(bars + 8u * s, 1);
+    for (uint32_t s = 0; s < pl.slots; ++s) mbar_init(bars + 8u * s, 16);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
@@ -806,30 +810,26 @@ __global__ void __launch_bounds__(kMmaThreads, 2) preba_antialias_mma_kernel(con
   // rows start on the same byte phase (the pitch is a multiple of 4)
   const uint32_t skew4 = static_cast<uint32_t>(reinterpret_cast<uintptr_t>(image + rowbyte0)) & 3u;
 
-  // thread 0 asks for the 16 rows of tile m (those the CTA needs)
+  // Warp 0 asks for the 16 rows of tile m, a lane per row: a row the CTA needs is copied and
+  // its bytes announced to the slot's barrier, the other lanes of the sixteen just arrive.
   auto issue = [&](uint32_t m) {
+    if (lane >= 16u) return;
     const uint32_t slot = m % pl.slots, bar = bars + 8u * slot;
-    uint32_t total = 0;
-    const uint32_t r0 = ya + 16u * m;
-    for (uint32_t i = 0; i < 16u && r0 + i < yb; ++i) {
-      const uint8_t* src = image + (r0 + i) * pitch + rowbyte0;
+    const uint32_t r = ya + 16u * m + lane;
+    if (r < yb) {
+      const uint8_t* src = image + r * pitch + rowbyte0;
       const uint32_t skew = static_cast<uint32_t>(reinterpret_cast<uintptr_t>(src)) & 15u;
       uint32_t bytes = (skew + rowbytes + 15u) & ~15u;
       if (bytes > static_cast<uint64_t>(stop - (src - skew)))  // only padding is lost
         bytes = static_cast<uint32_t>(stop - (src - skew));
-      total += bytes;
-    }
-    mbar_arrive_expect_tx(bar, total);
-    for (uint32_t i = 0; i < 16u && r0 + i < yb; ++i) {
-      const uint8_t* src = image + (r0 + i) * pitch + rowbyte0;
-      const uint32_t skew = static_cast<uint32_t>(reinterpret_cast<uintptr_t>(src)) & 15u;
-      uint32_t bytes = (skew + rowbytes + 15u) & ~15u;
-      if (bytes > static_cast<uint64_t>(stop - (src - skew)))
-        bytes = static_cast<uint32_t>(stop - (src - skew));
-      bulk_copy_g2s(ring + (slot * 16u + i) * pl.seg, src - skew, bytes, bar);
+      fence_async_shared();
+      mbar_arrive_expect_tx(bar, bytes);
+      bulk_copy_g2s(ring + (slot * 16u + lane) * pl.seg, src - skew, bytes, bar);
+    } else {
+      mbar_arrive(bar);
     }
   };
-  if (tid == 0)
+  if (warp == 0)
     for (uint32_t m = 0; m < pl.slots && m < ntiles16; ++m) issue(m);
 
   // the weights of this warp's four tiles as B operands: for k-step s, register r, byte i the
@@ -940,6 +940,7 @@ __global__ void __launch_bounds__(kMmaThreads, 2) preba_antialias_mma_kernel(con
   failed = __syncthreads_or(failed) != 0;
   if (!failed) horizontal(0);
   __syncthreads();
+  if (warp == 0 && !failed && pl.slots < ntiles16) issue(pl.slots);  // tile 0's rows have been read
   for (uint32_t m = 0; m < ntiles16 && !failed; ++m) {
     const uint32_t r0 = ya + 16u * m;
     if (m + 1 < ntiles16) {
@@ -981,10 +982,7 @@ __global__ void __launch_bounds__(kMmaThreads, 2) preba_antialias_mma_kernel(con
     // tile m + 1's H is complete, tile m's has been read, and so have the staged rows of tile
     // m + 1: their slot takes the rows of tile m + 1 + slots
     failed = __syncthreads_or(failed) != 0;
-    if (tid == 0 && !failed && m + 1 + pl.slots < ntiles16) {
-      fence_async_shared();
-      issue(m + 1 + pl.slots);
-    }
+    if (warp == 0 && !failed && m + 1 + pl.slots < ntiles16) issue(m + 1 + pl.slots);
   }
   if (failed && tid == 0) {
     report(p.status, PREBA_ERR_TIMEOUT);
