@@ -688,8 +688,7 @@ __global__ void __launch_bounds__(kThreads) preba_antialias_kernel(const Params 
 
 __device__ __forceinline__ void mma_u8(int32_t (&d)[4], const uint32_t (&a)[4], uint32_t b0,
                                        uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k32.row.col.s32.u8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+  asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
       "{%0,%1,%2,%3};"
       : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
@@ -754,7 +753,8 @@ __global__ void __launch_bounds__(kMmaThreads, 2) preba_antialias_mma_kernel(con
   uint32_t* ylo = reinterpret_cast<uint32_t*>(smem_b + pl.off_ylo);
   uint32_t* ycnt = reinterpret_cast<uint32_t*>(smem_b + pl.off_ycnt);
   const uint32_t bars = smem_addr(smem_b + pl.off_bar);
-  const uint32_t ring = smem_addr(smem_b + pl.off_ring);
+  const uint8_t* ring_p = smem_b + pl.off_ring;
+  const uint32_t ring = smem_addr(ring_p);
   const uint32_t ncols = C - xg0 < kGroup ? C - xg0 : kGroup;
   const uint32_t nrows = C - k0 < p.mma_rows ? C - k0 : p.mma_rows;
 
@@ -876,10 +876,13 @@ __global__ void __launch_bounds__(kMmaThreads, 2) preba_antialias_mma_kernel(con
   // them uses accumulator n % 4 (a row is finished before the row 32 further down begins);
   // columns lane and lane + 32 of the group, three channels
   float acc[4][3][2];
-  uint32_t cur[4];
+  uint32_t cur[4], cur0[4], cur1[4];  // the row of each accumulator and its taps [cur0, cur1)
 #pragma unroll
   for (uint32_t a = 0; a < 4; ++a) {
     cur[a] = warp + 8u * a;
+    const bool have = cur[a] < nrows;
+    cur0[a] = have ? ylo[cur[a]] : 0xffffffffu;  // no row: never begins
+    cur1[a] = have ? cur0[a] + ycnt[cur[a]] : 0xffffffffu;
 #pragma unroll
     for (uint32_t c = 0; c < 3; ++c) acc[a][c][0] = acc[a][c][1] = 0.f;
   }
@@ -896,8 +899,8 @@ __global__ void __launch_bounds__(kMmaThreads, 2) preba_antialias_mma_kernel(con
         reinterpret_cast<uintptr_t>(image + (r0 + g) * pitch + rowbyte0)) & 15u;
     const uint32_t sk1 = static_cast<uint32_t>(
         reinterpret_cast<uintptr_t>(image + (r0 + g + 8u) * pitch + rowbyte0)) & 15u;
-    const uint32_t row0 = ring + (slot * 16u + g) * pl.seg + sk0 + 4u * q;
-    const uint32_t row1 = ring + (slot * 16u + g + 8u) * pl.seg + sk1 + 4u * q;
+    const uint8_t* row0 = ring_p + (slot * 16u + g) * pl.seg + sk0 + 4u * q;
+    const uint8_t* row1 = ring_p + (slot * 16u + g + 8u) * pl.seg + sk1 + 4u * q;
 #pragma unroll
     for (uint32_t t = 0; t < 4; ++t) {
       const uint32_t tile = 4u * warp + t;
@@ -905,11 +908,12 @@ __global__ void __launch_bounds__(kMmaThreads, 2) preba_antialias_mma_kernel(con
       uint32_t a[2][4];
 #pragma unroll
       for (uint32_t s2 = 0; s2 < 2; ++s2) {
-        const uint32_t at0 = row0 + kst[t] + 32u * s2, at1 = row1 + kst[t] + 32u * s2;
-        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(a[s2][0]) : "r"(at0));
-        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(a[s2][1]) : "r"(at1));
-        asm volatile("ld.shared.u32 %0, [%1+16];" : "=r"(a[s2][2]) : "r"(at0));
-        asm volatile("ld.shared.u32 %0, [%1+16];" : "=r"(a[s2][3]) : "r"(at1));
+        const uint32_t* at0 = reinterpret_cast<const uint32_t*>(row0 + kst[t] + 32 * static_cast<int32_t>(s2));
+        const uint32_t* at1 = reinterpret_cast<const uint32_t*>(row1 + kst[t] + 32 * static_cast<int32_t>(s2));
+        a[s2][0] = at0[0];
+        a[s2][1] = at1[0];
+        a[s2][2] = at0[4];
+        a[s2][3] = at1[4];
       }
       int32_t d[4] = {0, 0, 0, 0};
       mma_u8(d, a[0], bhi[t][0][0], bhi[t][0][1]);
@@ -952,14 +956,14 @@ __global__ void __launch_bounds__(kMmaThreads, 2) preba_antialias_mma_kernel(con
 #pragma unroll
     for (uint32_t a = 0; a < 4; ++a) {
       for (;;) {
+        const uint32_t y0 = cur0[a], y1 = cur1[a];
+        if (y0 >= r0 + 16u) break;  // begins in a later tile (or there is no row)
         const uint32_t yl = cur[a];
-        if (yl >= nrows) break;
-        const uint32_t y0 = ylo[yl], y1 = y0 + ycnt[yl];
-        if (y0 >= r0 + 16u) break;  // begins in a later tile
         const uint32_t from = y0 > r0 ? y0 : r0, to = y1 < r0 + 16u ? y1 : r0 + 16u;
-        for (uint32_t r = from; r < to; ++r) {
-          const float wgt = wyn[yl * kMaxTapsY + (r - y0)];
-          const float* h = hb + (r - r0) * kHPitch + lane;
+        const float* wrow = wyn + yl * kMaxTapsY + (from - y0);
+        const float* h = hb + (from - r0) * kHPitch + lane;
+        for (uint32_t r = from; r < to; ++r, ++wrow, h += kHPitch) {
+          const float wgt = *wrow;
 #pragma unroll
           for (uint32_t c = 0; c < 3; ++c) {
             acc[a][c][0] = fmaf(wgt, h[c * kHPlane], acc[a][c][0]);
@@ -977,6 +981,9 @@ __global__ void __launch_bounds__(kMmaThreads, 2) preba_antialias_mma_kernel(con
           acc[a][c][0] = acc[a][c][1] = 0.f;
         }
         cur[a] = yl + 32u;
+        const bool have = yl + 32u < nrows;
+        cur0[a] = have ? ylo[yl + 32u] : 0xffffffffu;
+        cur1[a] = have ? cur0[a] + ycnt[yl + 32u] : 0xffffffffu;
       }
     }
     // tile m + 1's H is complete, tile m's has been read, and so have the staged rows of tile
