@@ -916,9 +916,16 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
     done = [torch.cuda.Event() for _ in range(nbuf)]
     side = [torch.cuda.Stream(device=dev) for _ in range(nbuf)]  # one stream per buffer set
     scr = [torch.zeros(pb.SCRATCH_BYTES // 4, dtype=torch.int32, device=dev) for _ in range(nbuf)]
-    e2e_calls = [pb.PreparedImages(pinned, th[b], oh[b], None, dtab[b], outs[b], C, S, wl.MEAN,
+    # both directions in place: the kernel reads the images from, and writes the result to,
+    # pinned host memory; a step is the table copy and one kernel
+    e2e_calls = [pb.PreparedImages(pinned, th[b], oh[b], None, dtab[b], None, C, S, wl.MEAN,
                                    wl.STD, out_dtype, stream=side[b], dev_status=status,
-                                   dev_scratch=scr[b], in_place=True) for b in range(nbuf)]
+                                   dev_scratch=scr[b], in_place=True, out_in_place=True)
+                 for b in range(nbuf)]
+    # the kernel reads in place, the result is copied back by the copy engine
+    back_calls = [pb.PreparedImages(pinned, th[b], oh[b], None, dtab[b], outs[b], C, S, wl.MEAN,
+                                    wl.STD, out_dtype, stream=side[b], dev_status=status,
+                                    dev_scratch=scr[b], in_place=True) for b in range(nbuf)]
     copy_calls = [pb.PreparedImages(pinned, th[b], oh[b], pix[b], dtab[b], outs[b], C, S, wl.MEAN,
                                     wl.STD, out_dtype, stream=side[b], dev_status=status,
                                     dev_scratch=scr[b]) for b in range(nbuf)]
@@ -952,6 +959,22 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
     assert int(status.item()) == 0
     for b in range(nbuf):                           # the host result is the device result
         assert bool(torch.equal(oh[b], ref.cpu())), "end-to-end result differs"
+
+    for b in range(nbuf):
+        oh[b].zero_()
+
+    def back_step(i):
+        b = i % nbuf
+        done[b].synchronize()
+        t0 = time.perf_counter()
+        back_calls[b]()
+        done[b].record(side[b])
+        return time.perf_counter() - t0
+
+    back_ms, back_host = timed_e2e(back_step, e2e_steps)
+    assert int(status.item()) == 0
+    for b in range(nbuf):
+        assert bool(torch.equal(oh[b], ref.cpu())), "end-to-end result differs (copy back)"
 
     # the same with one copy per image to the device instead of reads in place
     def copy_step(i):
@@ -998,8 +1021,30 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
         barrier()
         link[name + "_gbs"] = 3 * src.numel() / (l_start.elapsed_time(l_stop) * 1e-3) / 1e9
 
-    elapsed_ms, e2e_ms, packed_ms, copied_ms = max_over_ranks(
-        [elapsed_ms, e2e_ms, packed_ms, copied_ms], dist, dev)
+    # ... and both ways at once (two streams): what the link carries when it is used in both
+    # directions, which is what an end-to-end step does
+    src_out = outs[0].view(torch.uint8).reshape(-1)
+    d_start = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    d_stop = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    barrier()
+    for st in side:
+        st.wait_stream(stream)
+    with torch.cuda.stream(side[0]):
+        d_start[0].record(side[0])
+        for _ in range(4):
+            pix[0].copy_(ph[0], non_blocking=True)
+        d_stop[0].record(side[0])
+    with torch.cuda.stream(side[1]):
+        d_start[1].record(side[1])
+        for _ in range(4):
+            big_out.copy_(src_out, non_blocking=True)
+        d_stop[1].record(side[1])
+    barrier()
+    link["both_ways_h2d_gbs"] = 4 * ph[0].numel() / (d_start[0].elapsed_time(d_stop[0]) * 1e-3) / 1e9
+    link["both_ways_d2h_gbs"] = 4 * src_out.numel() / (d_start[1].elapsed_time(d_stop[1]) * 1e-3) / 1e9
+
+    elapsed_ms, e2e_ms, packed_ms, copied_ms, back_ms = max_over_ranks(
+        [elapsed_ms, e2e_ms, packed_ms, copied_ms, back_ms], dist, dev)
 
     if rank == 0:
         peak, peak_src = measured_peak()
@@ -1042,18 +1087,33 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
                              "sample": f"whole batch of {n} images, {len(cpu_times)} passes",
                              "one_thread_value": cpu_one},
             "e2e": {"value": world * n * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT,
-                    "h2d_bytes_per_step": int(sizes.packed_bytes + sizes.table_bytes),
+                    "h2d_bytes_per_step": int(acct["input_sector_bytes"] + sizes.table_bytes),
                     "d2h_bytes_per_step": int(sizes.out_bytes), "steps": e2e_steps,
                     "ms_per_step": e2e_ms / e2e_steps,
                     "host_ms_per_step": 1e3 * t_pack / e2e_steps,
                     "link_plain_copy_gbs": link,
-                    "includes": "preba_preprocess_images, images read in place: the kernel "
-                                "fetches the tapped rows of every image from its own pinned "
-                                "host buffer across the link, then the result is copied to "
-                                "pinned memory; two buffer sets on two streams",
-                    "h2d_bytes_note": "bytes of the images (all of them would cross in a "
-                                      "copy); in place only the tapped sectors cross: "
-                                      f"{acct['input_sector_bytes']}",
+                    "achieved_link_gbs": {
+                        "h2d": (acct["input_sector_bytes"] + sizes.table_bytes) * e2e_steps
+                               / (e2e_ms * 1e-3) / 1e9,
+                        "d2h": sizes.out_bytes * e2e_steps / (e2e_ms * 1e-3) / 1e9},
+                    "link_bound_ms_per_step": 1e3 * max(
+                        (acct["input_sector_bytes"] + sizes.table_bytes)
+                        / (link["both_ways_h2d_gbs"] * 1e9),
+                        sizes.out_bytes / (link["both_ways_d2h_gbs"] * 1e9)),
+                    "link_bound_note": "bytes each way over what a plain pinned copy gets in "
+                                       "that direction while the other direction is busy too",
+                    "includes": "preba_preprocess_images with both directions in place: the "
+                                "kernel fetches the tapped rows of every image from its own "
+                                "pinned host buffer across the link and stores the result "
+                                "straight into pinned host memory (table copy + one kernel per "
+                                "step); two buffer sets on two streams",
+                    "h2d_bytes_note": "the tapped sectors and the table: what crosses the link "
+                                      f"(the images themselves hold {int(sizes.packed_bytes)} "
+                                      "bytes)",
+                    "kernel_reads_result_copied_back": {
+                        "value": world * n * e2e_steps / (back_ms * 1e-3),
+                        "ms_per_step": back_ms / e2e_steps,
+                        "host_ms_per_step": 1e3 * back_host / e2e_steps},
                     "one_copy_per_image": {
                         "value": world * n * e2e_steps / (copied_ms * 1e-3),
                         "ms_per_step": copied_ms / e2e_steps,

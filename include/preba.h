@@ -141,6 +141,13 @@ typedef struct {
                                      16-byte block that holds the image's last byte; the
                                      images must not overlap.  dev_pixels is not used. */
 
+#define PREBA_IMAGES_OUT_IN_PLACE 2u /* the kernel stores the result where it is wanted, in pinned
+                                        host memory, across the link (streaming 128-byte runs):
+                                        no copy is enqueued for it, and with PREBA_IMAGES_IN_PLACE
+                                        one kernel moves both directions of the link at once.
+                                        out_host must then be pinned memory the device can
+                                        address, 16-byte aligned; dev_out is not used. */
+
 /* A batch of separate decoded images in host memory (no packed copy on the host), with the
  * device buffers the call stages it through. */
 typedef struct {
@@ -149,7 +156,7 @@ typedef struct {
   const uint32_t* h;             /* HOST, n entries */
   const uint32_t* w;             /* HOST, n entries */
   uint32_t n;
-  uint32_t flags;                /* 0 or PREBA_IMAGES_IN_PLACE */
+  uint32_t flags;                /* 0, PREBA_IMAGES_IN_PLACE, PREBA_IMAGES_OUT_IN_PLACE or both */
   preba_img_t* table_host;       /* HOST, n entries, WRITTEN by the call (the table preba_pack
                                     would build); pinned; valid until the stream has passed
                                     the call's copies */
@@ -311,7 +318,8 @@ int preba_preprocess_host(const preba_host_batch_t* batch, uint32_t out_size,
  * gives them weight.  n + 1 host-to-device copies, one kernel, one device-to-host copy.
  * With PREBA_IMAGES_IN_PLACE the image copies are dropped: `table_host` receives each
  * image's distance from the lowest image address, and the kernel fetches the tapped rows
- * from host memory itself (table copy, kernel, result copy).
+ * from host memory itself (table copy, kernel, result copy).  With PREBA_IMAGES_OUT_IN_PLACE
+ * the result copy is dropped too: the kernel writes `out_host` itself (table copy, kernel).
  * Errors: PREBA_ERR_INVALID_ARG, PREBA_ERR_BUFFER_TOO_SMALL (dev_pixels_bytes, out_bytes),
  * PREBA_ERR_CUDA.
  */

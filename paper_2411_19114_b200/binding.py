@@ -16,6 +16,7 @@ _LIB_PATH = Path(__file__).resolve().parent / "libpreba.so"
 PACK_ALIGN = 128
 SCRATCH_BYTES = 256
 IMAGES_IN_PLACE = 1
+IMAGES_OUT_IN_PLACE = 2
 EX_ROUND_U8 = 1
 OVERLAP_PREVIOUS = 1
 F32, F16, BF16, U8 = 0, 1, 2, 3
@@ -494,11 +495,13 @@ class PreparedImages:
     ``table_host`` is a pinned CPU tensor of ``16 * n`` bytes that every call rewrites;
     ``out_host`` a (pinned) CPU tensor; ``dev_*`` CUDA tensors used as staging.  With
     ``in_place`` the kernel reads the (pinned, 128-byte aligned) images over the link itself
-    and ``dev_pixels`` may be None."""
+    and ``dev_pixels`` may be None; with ``out_in_place`` it writes the (pinned) ``out_host``
+    itself and ``dev_out`` may be None."""
 
     def __init__(self, images, table_host, out_host, dev_pixels, dev_table, dev_out,
                  out_size: int, resize_short: int, mean, std, out_dtype: int, stream=None,
-                 dev_status=None, dev_scratch=None, in_place: bool = False):
+                 dev_status=None, dev_scratch=None, in_place: bool = False,
+                 out_in_place: bool = False):
         import torch
 
         def haddr(t):
@@ -525,13 +528,17 @@ class PreparedImages:
         b.h, b.w, b.n = self._h.ctypes.data, self._w.ctypes.data, n
         b.table_host = haddr(table_host)
         b.out_host, b.out_bytes = haddr(out_host), hbytes(out_host)
-        b.flags = IMAGES_IN_PLACE if in_place else 0
+        b.flags = (IMAGES_IN_PLACE if in_place else 0) | (IMAGES_OUT_IN_PLACE if out_in_place else 0)
         if dev_pixels is not None:
             b.dev_pixels = dev_pixels.data_ptr()
             b.dev_pixels_bytes = dev_pixels.numel() * dev_pixels.element_size()
-        b.dev_table, b.dev_out = dev_table.data_ptr(), dev_out.data_ptr()
-        if dev_out.numel() * dev_out.element_size() < b.out_bytes:
-            raise PrebaError(ERR_BUFFER_TOO_SMALL, "preba_preprocess_images (dev_out)")
+        b.dev_table = dev_table.data_ptr()
+        if dev_out is not None:
+            b.dev_out = dev_out.data_ptr()
+            if dev_out.numel() * dev_out.element_size() < b.out_bytes:
+                raise PrebaError(ERR_BUFFER_TOO_SMALL, "preba_preprocess_images (dev_out)")
+        elif not out_in_place:
+            raise ValueError("dev_out is needed unless the kernel writes the result in place")
         b.dev_status = dev_status.data_ptr() if dev_status is not None else None
         b.dev_scratch = dev_scratch.data_ptr() if dev_scratch is not None else None
         self._b, self._m, self._s = b, _f3(mean), _f3(std)

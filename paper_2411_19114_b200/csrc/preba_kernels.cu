@@ -1262,9 +1262,12 @@ extern "C" int preba_preprocess_images(const preba_image_batch_t* b, uint32_t ou
                                        const float std[3], int out_dtype, void* stream) {
   using namespace preba;
   if (!b || !b->images || !b->h || !b->w || !b->table_host || !b->out_host || !b->dev_table ||
-      b->n == 0 || (b->flags & ~PREBA_IMAGES_IN_PLACE))
+      b->n == 0 || (b->flags & ~(PREBA_IMAGES_IN_PLACE | PREBA_IMAGES_OUT_IN_PLACE)))
     return PREBA_ERR_INVALID_ARG;
   const bool in_place = (b->flags & PREBA_IMAGES_IN_PLACE) != 0;
+  // the kernel stores the result in (pinned) host memory itself instead of a copy afterwards
+  const bool out_in_place = (b->flags & PREBA_IMAGES_OUT_IN_PLACE) != 0;
+  void* const out = out_in_place ? b->out_host : b->dev_out;
   for (uint32_t i = 0; i < b->n; ++i)
     if (!b->images[i] || !dims_ok(b->h[i], b->w[i])) return PREBA_ERR_INVALID_ARG;
   const uint8_t* pixels = b->dev_pixels;
@@ -1298,7 +1301,7 @@ extern "C" int preba_preprocess_images(const preba_image_batch_t* b, uint32_t ou
     pixels_bytes = at;
     if (b->dev_pixels_bytes < pixels_bytes) return PREBA_ERR_BUFFER_TOO_SMALL;
   }
-  int rc = check_args(pixels, pixels_bytes, b->dev_table, b->n, b->dev_out, b->out_bytes,
+  int rc = check_args(pixels, pixels_bytes, b->dev_table, b->n, out, b->out_bytes,
                       out_size, resize_short, mean, std, out_dtype);
   if (rc != PREBA_OK) return rc;
   if (reinterpret_cast<uintptr_t>(b->dev_scratch) % 16) return PREBA_ERR_INVALID_ARG;
@@ -1306,6 +1309,14 @@ extern "C" int preba_preprocess_images(const preba_image_batch_t* b, uint32_t ou
   const uint64_t need = static_cast<uint64_t>(b->n) * 3ull * out_size * out_size *
                         dtype_bytes(out_dtype);
   cudaError_t err = cudaSuccess;
+  if (out_in_place) {
+    // the device must be able to address the result buffer through the pointer given
+    cudaPointerAttributes attr;
+    err = cudaPointerGetAttributes(&attr, b->out_host);
+    if (err == cudaSuccess && (attr.type == cudaMemoryTypeUnregistered ||
+                               attr.devicePointer != b->out_host))
+      return PREBA_ERR_INVALID_ARG;
+  }
   if (in_place) {
     // the device must be able to address the images through the pointers given
     for (uint32_t i = 0; i < b->n && err == cudaSuccess; ++i) {
@@ -1327,11 +1338,11 @@ extern "C" int preba_preprocess_images(const preba_image_batch_t* b, uint32_t ou
     g_last_cuda_error = static_cast<int>(err);
     return PREBA_ERR_CUDA;
   }
-  const Params p = make_params(pixels, pixels_bytes, b->dev_table, b->n, b->dev_out,
-                               b->dev_status, b->dev_scratch, out_size, resize_short, mean, std);
+  const Params p = make_params(pixels, pixels_bytes, b->dev_table, b->n, out, b->dev_status,
+                               b->dev_scratch, out_size, resize_short, mean, std);
   rc = launch(p, out_dtype, false, s);
   if (rc != PREBA_OK) return rc;
-  err = cudaMemcpyAsync(b->out_host, b->dev_out, need, cudaMemcpyDeviceToHost, s);
+  if (!out_in_place) err = cudaMemcpyAsync(b->out_host, b->dev_out, need, cudaMemcpyDeviceToHost, s);
   if (err != cudaSuccess) {
     g_last_cuda_error = static_cast<int>(err);
     return PREBA_ERR_CUDA;

@@ -493,3 +493,26 @@ def test_images_read_in_place_from_pinned_host_memory():
     with pytest.raises(pb.PrebaError) as exc:
         pageable()
     assert exc.value.code == pb.ERR_INVALID_ARG
+    # the result written in place too: the kernel stores to the pinned result buffer itself
+    oh2 = torch.full((n, 3, 224, 224), float("nan"), dtype=torch.float16).pin_memory()
+    both = pb.PreparedImages(pinned, th, oh2, None, dtab, None, 224, 256, MEAN, STD, pb.F16,
+                             dev_status=status, in_place=True, out_in_place=True)
+    both()
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert np.array_equal(oh2.numpy().view(np.uint16), want.view(np.uint16))
+    # ... and with the images copied but the result in place, in fp32
+    oh3 = torch.full((n, 3, 224, 224), float("nan"), dtype=torch.float32).pin_memory()
+    dpix = torch.empty(pb.preba_query([im.shape[0] for im in imgs], [im.shape[1] for im in imgs],
+                                      224, pb.F32).packed_bytes, dtype=torch.uint8, device=dev)
+    mixed = pb.PreparedImages(pinned, th, oh3, dpix, dtab, None, 224, 256, MEAN, STD, pb.F32,
+                              dev_status=status, out_in_place=True)
+    mixed()
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert_parity(oh3.numpy().copy(), oracle_f64(imgs, 224, 256), pb.F32)
+    # a pageable result buffer is refused
+    with pytest.raises(pb.PrebaError) as exc:
+        pb.PreparedImages(pinned, th, np.zeros((n, 3, 224, 224), dtype=np.float16), None, dtab,
+                          None, 224, 256, MEAN, STD, pb.F16, in_place=True, out_in_place=True)()
+    assert exc.value.code == pb.ERR_INVALID_ARG
