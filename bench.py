@@ -875,6 +875,12 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
     alone.repeated(20)
     lat_us, _ = alone.repeated(max(50, min(args.steps, 1000)))
     assert bool(torch.equal(outs[0], ref)), "an isolated launch changed the result"
+    # the same with fixed shares instead of claimed slabs (no scratch)
+    fixed = pb.PreparedPreprocess(pix[0], tab, n, outs[0], C, S, wl.MEAN, wl.STD, out_dtype,
+                                  stream=stream, status=status)
+    fixed.repeated(20)
+    lat_fixed_us, _ = fixed.repeated(max(50, min(args.steps, 1000)))
+    assert bool(torch.equal(outs[0], ref)), "an isolated launch changed the result"
 
     # ---- the same launch over and over on one buffer set (whatever fits stays in L2) -----------
     warm_steps = max(3, min(args.steps, 2000))
@@ -1126,9 +1132,11 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
                                     "back (preba_preprocess_host)"}},
             "isolated_launch_us": {"p50": iso_p50,
                                    "p99": float(np.percentile(lat_us, 99)),
+                                   "fixed_shares_p50": float(np.percentile(lat_fixed_us, 50)),
                                    "note": "device time of one launch running alone (warps claim "
-                                           "slabs through the scratch counters), events around "
-                                           "every launch, same buffers every time"},
+                                           "slabs through the scratch counters; fixed_shares: "
+                                           "without scratch), events around every launch, same "
+                                           "buffers every time"},
             "warm_l2": {"value": world * n * warm_steps / (warm_ms * 1e-3), "unit": UNIT,
                         "us_per_launch": 1e3 * warm_ms / warm_steps,
                         "note": "one buffer set reused by every launch, launches not marked as "
