@@ -66,6 +66,10 @@ extern "C" {
 #define PREBA_ERR_TOO_LARGE (-6)        /* the batch exceeds PREBA_NOALLOC_MAX_BYTES, or an image is
                                            reduced by more than the antialiased kernel can hold */
 #define PREBA_ERR_BAD_CROP (-7)         /* a crop window does not lie on its image's resized grid */
+#define PREBA_ERR_RANGE (-8)            /* only in the device status word, and only from the checked
+                                           build of the library (compiled with PREBA_CHECKED): a
+                                           shared-memory offset, a table index or a global address
+                                           left its range inside a kernel; the access was skipped */
 
 /* Device memory the library itself carries for preba_preprocess_host_noalloc (64 MiB). */
 #define PREBA_NOALLOC_MAX_BYTES (64u << 20)

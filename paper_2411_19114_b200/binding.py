@@ -7,11 +7,15 @@ the library has not been built the first call raises: there is no fallback.
 from __future__ import annotations
 
 import ctypes
+import os
 from pathlib import Path
 
 import numpy as np
 
-_LIB_PATH = Path(__file__).resolve().parent / "libpreba.so"
+# PREBA_CHECKED_BUILD=1 in the environment loads the build with device-side range checks
+# (libpreba_checked.so) instead: same entry points, slower kernels, for tests
+_LIB_PATH = Path(__file__).resolve().parent / (
+    "libpreba_checked.so" if os.environ.get("PREBA_CHECKED_BUILD") == "1" else "libpreba.so")
 
 PACK_ALIGN = 128
 SCRATCH_BYTES = 256
@@ -29,6 +33,7 @@ ERR_CUDA = -4
 ERR_TIMEOUT = -5
 ERR_TOO_LARGE = -6
 ERR_BAD_CROP = -7
+ERR_RANGE = -8
 NOALLOC_MAX_BYTES = 64 << 20
 
 EXPORTS = ("preba_query", "preba_pack", "preba_preprocess", "preba_preprocess_ex",

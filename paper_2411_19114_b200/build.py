@@ -11,6 +11,9 @@ PKG = Path(__file__).resolve().parent
 ROOT = PKG.parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libpreba.so"
+# the same sources with -DPREBA_CHECKED: device code range-checks its offsets and addresses and
+# reports a violation in the status word (PREBA_ERR_RANGE); for tests, never for measurements
+LIB_CHECKED = PKG / "libpreba_checked.so"
 
 NVCC_FLAGS = [
     "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
@@ -27,10 +30,10 @@ def _inputs() -> list[Path]:
         Path(__file__)]
 
 
-def stale() -> bool:
-    if not LIB.exists():
+def stale(lib: Path = LIB) -> bool:
+    if not lib.exists():
         return True
-    built = LIB.stat().st_mtime
+    built = lib.stat().st_mtime
     return any(p.stat().st_mtime > built for p in _inputs())
 
 
@@ -41,20 +44,24 @@ def nvcc_path() -> str:
     return found
 
 
-def build(force: bool = False, verbose: bool = False) -> Path:
-    """Compile if the library is missing or older than its sources."""
-    if not force and not stale():
-        return LIB
-    tmp = LIB.with_name(f"libpreba.tmp{os.getpid()}.so")
+def build(force: bool = False, verbose: bool = False, checked: bool = False) -> Path:
+    """Compile if the library is missing or older than its sources (``checked``: the build
+    with device-side range checks)."""
+    lib = LIB_CHECKED if checked else LIB
+    if not force and not stale(lib):
+        return lib
+    tmp = lib.with_name(f"{lib.stem}.tmp{os.getpid()}.so")
     cmd = [nvcc_path(), *NVCC_FLAGS, "-I", str(ROOT / "include"), "-I", str(CSRC)]
+    if checked:
+        cmd += ["-DPREBA_CHECKED"]
     if verbose:
         cmd += ["-Xptxas", "-v"]
     cmd += ["-o", str(tmp)] + [str(s) for s in sources()]
     subprocess.run(cmd, check=True)
-    os.replace(tmp, LIB)
-    return LIB
+    os.replace(tmp, lib)
+    return lib
 
 
 if __name__ == "__main__":
-    build(force="--force" in sys.argv, verbose="-v" in sys.argv)
-    print(LIB)
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv,
+                checked="--checked" in sys.argv))

@@ -383,6 +383,7 @@ struct Ring {
   const uint8_t* stop;  // end of the last whole 16-byte unit of the pixel buffer
   uint64_t pitch;       // bytes per image row
   uint32_t b0, bytes;   // first needed byte of a row and the count of needed bytes
+  int32_t* status;      // the launch's status word (for the checked build's reports)
 };
 
 // Thread 0: asks for every row below `limit` that has not been asked for.
@@ -396,8 +397,12 @@ __device__ __forceinline__ void ring_issue(Ring& rg, uint32_t limit) {
     if (bytes > static_cast<uint64_t>(rg.stop - (src - skew)))  // only padding is lost
       bytes = static_cast<uint32_t>(rg.stop - (src - skew));
     const uint32_t bar = rg.bars + 8u * slot;
+    // checked build: the row lies in its slot and in the pixel buffer (a row that does not is
+    // announced with no bytes, so that its wait still ends)
+    if (!PREBA_IN_RANGE(rg.status, bytes <= rg.seg && slot < rg.slots && src - skew + bytes <= rg.stop))
+      bytes = 0;
     mbar_arrive_expect_tx(bar, bytes);
-    bulk_copy_g2s(rg.data + slot * rg.seg, src - skew, bytes, bar);
+    if (bytes) bulk_copy_g2s(rg.data + slot * rg.seg, src - skew, bytes, bar);
   }
 }
 
@@ -479,6 +484,7 @@ __global__ void __launch_bounds__(kThreads) preba_antialias_kernel(const Params 
   rg.bars = rg.data + slots * pl.seg;
   rg.slots = slots;
   rg.seg = pl.seg;
+  rg.status = p.status;
   tabulate(ax, left, C, pl.tx, wx, xlo, xcnt);
   uint2* wi = reinterpret_cast<uint2*>(smem + pl.off_wi);
   float2* inv = reinterpret_cast<float2*>(smem + pl.off_inv);
@@ -616,8 +622,11 @@ __global__ void __launch_bounds__(kThreads) preba_antialias_kernel(const Params 
             const uint32_t byte = b0 + 4u * (w0 + k * kThreads) + t;
             const uint32_t pix = byte / 3u, ch = byte - 3u * pix, rel = pix - p0;
             const uint32_t at = ch * pl.plane + rel + (rel >> 5);
-            va[at] = acc[k][t];
-            vb[at] = acc[k][4 + t];
+            // checked build: the element lies in its channel plane
+            if (PREBA_IN_RANGE(p.status, rel + (rel >> 5) < pl.plane && ch < 3u)) {
+              va[at] = acc[k][t];
+              vb[at] = acc[k][4 + t];
+            }
           }
         }
       }
@@ -636,6 +645,10 @@ __global__ void __launch_bounds__(kThreads) preba_antialias_kernel(const Params 
       const uint32_t rel0 = xlo[X] - p0, nx = xcnt[X];
       const float* w = wx + X * pl.tx;
       float s[6] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+      // checked build: the column's taps lie in the planes and in its row of the weight table
+      if (!PREBA_IN_RANGE(p.status, nx <= pl.tx && rel0 + nx + ((rel0 + nx) >> 5) <= pl.plane &&
+                                        k0 + 2 * r < C))
+        continue;
       for (uint32_t t = 0; t < nx; ++t) {
         uint32_t idx = rel0 + t;
         idx += idx >> 5;
@@ -823,8 +836,14 @@ __global__ void __launch_bounds__(kMmaThreads, 2) preba_antialias_mma_kernel(con
       if (bytes > static_cast<uint64_t>(stop - (src - skew)))  // only padding is lost
         bytes = static_cast<uint32_t>(stop - (src - skew));
       fence_async_shared();
-      mbar_arrive_expect_tx(bar, bytes);
-      bulk_copy_g2s(ring + (slot * 16u + lane) * pl.seg, src - skew, bytes, bar);
+      // checked build: the row lies in its place in the ring and in the pixel buffer
+      if (PREBA_IN_RANGE(p.status, bytes <= pl.seg && src - skew >= p.pixels &&
+                                       src - skew + bytes <= p.pixels + p.pixels_bytes)) {
+        mbar_arrive_expect_tx(bar, bytes);
+        bulk_copy_g2s(ring + (slot * 16u + lane) * pl.seg, src - skew, bytes, bar);
+      } else {
+        mbar_arrive(bar);
+      }
     } else {
       mbar_arrive(bar);
     }
@@ -905,6 +924,15 @@ __global__ void __launch_bounds__(kMmaThreads, 2) preba_antialias_mma_kernel(con
     for (uint32_t t = 0; t < 4; ++t) {
       const uint32_t tile = 4u * warp + t;
       if (2u * tile >= ncols) break;
+      // checked build: the 64 bytes each of the two rows gives to this tile lie in the row's
+      // place in the ring; the tile's columns lie in H
+      if (!PREBA_IN_RANGE(p.status,
+                          static_cast<int32_t>(sk0 + 4u * q) + kst[t] >= 0 &&
+                              static_cast<int32_t>(sk1 + 4u * q) + kst[t] >= 0 &&
+                              static_cast<int32_t>((sk0 > sk1 ? sk0 : sk1) + 4u * q) + kst[t] + 52 <=
+                                  static_cast<int32_t>(pl.seg) &&
+                              slot < pl.slots && 2u * tile + 1u < kGroup))
+        continue;
       uint32_t a[2][4];
 #pragma unroll
       for (uint32_t s2 = 0; s2 < 2; ++s2) {
@@ -962,6 +990,11 @@ __global__ void __launch_bounds__(kMmaThreads, 2) preba_antialias_mma_kernel(con
         const uint32_t from = y0 > r0 ? y0 : r0, to = y1 < r0 + 16u ? y1 : r0 + 16u;
         const float* wrow = wyn + yl * kMaxTapsY + (from - y0);
         const float* h = hb + (from - r0) * kHPitch + lane;
+        // checked build: the taps lie in the row's weights, the rows in the tile of H, the
+        // output row in the crop
+        if (!PREBA_IN_RANGE(p.status, yl < kMmaRows && yl < nrows && y1 - y0 <= kMaxTapsY &&
+                                          from >= r0 && to <= r0 + 16u && k0 + yl < C))
+          break;
         for (uint32_t r = from; r < to; ++r, ++wrow, h += kHPitch) {
           const float wgt = *wrow;
 #pragma unroll

@@ -231,6 +231,7 @@ __device__ __forceinline__ void mel_round(const float* __restrict__ wp, const fl
     e0 = fmaf(wgt, pw.x, e0);
     e1 = fmaf(wgt, pw.y, e1);
   }
+  // (checked build: the caller has tested filter < 80 and t0 + 1 < t_max or the lone frame)
   if (filter != 0xffu) {
     float* __restrict__ o = out + static_cast<size_t>(filter) * t_max + t0;
     o[0] = __logf(e0 + kLogGuard);
@@ -346,6 +347,19 @@ logmel_kernel(const AudioParams p, const MelPlan plan_param) {
     frames = min(u.frames, p.t_max);
     const float* __restrict__ x0 = p.samples + u.offset + static_cast<size_t>(2 * q) * kHop;
     const float* __restrict__ x1 = 2 * q + 1 < frames ? x0 + kHop : x0;
+    // checked build: both frames lie in the utterance and the utterance in the sample buffer
+    if (!PREBA_IN_RANGE(p.status,
+                        utt < p.n && 2 * q < frames &&
+                            static_cast<uint64_t>(2 * q + (2 * q + 1 < frames ? 1 : 0)) * kHop + kWin <=
+                                u.length &&
+                            u.offset + u.length <= p.samples_count)) {
+#pragma unroll
+      for (int c = 0; c < 2; ++c)
+#pragma unroll
+        for (uint32_t n2 = 0; n2 < 6; ++n2) raw[0][c][n2] = raw[1][c][n2] = 0.f;
+      raw6[0] = raw6[1] = 0.f;
+      return;
+    }
 #pragma unroll
     for (int c = 0; c < 2; ++c)
 #pragma unroll
@@ -442,6 +456,19 @@ logmel_kernel(const AudioParams p, const MelPlan plan_param) {
         upairs = pairs_in(p, utt);
       }
       fetch();
+    }
+    // checked build: the Mel rounds read inside the padded power array and write inside the
+    // utterance's rows of the result
+    if (!PREBA_IN_RANGE(p.status,
+                        mel_begin[0] >= 0 && mel_begin[0] + static_cast<int>(kMelIters0) <= static_cast<int>(kPowLen) &&
+                            mel_begin[1] >= 0 && mel_begin[1] + static_cast<int>(kMelIters1) <= static_cast<int>(kPowLen) &&
+                            mel_begin[2] >= 0 && mel_begin[2] + static_cast<int>(kMelIters2) <= static_cast<int>(kPowLen) &&
+                            (mel_filter[0] == 0xffu || mel_filter[0] < kMels) &&
+                            (mel_filter[1] == 0xffu || mel_filter[1] < kMels) &&
+                            (mel_filter[2] == 0xffu || mel_filter[2] < kMels) &&
+                            this_t0 + (have1 ? 1u : 0u) < p.t_max)) {
+      __syncwarp();
+      continue;
     }
     mel_round<kMelIters0>(plan.w + lane, ws.power + mel_begin[0], mel_filter[0], out, p.t_max,
                           this_t0, have1);

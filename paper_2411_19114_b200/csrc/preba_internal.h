@@ -18,4 +18,21 @@ extern thread_local int g_last_cuda_error;
 
 }  // namespace preba
 
+// The checked build (-DPREBA_CHECKED, a second library built from the same sources): device
+// code tests its shared-memory offsets, table indices and global addresses against their
+// ranges before it uses them.  A violation stores PREBA_ERR_RANGE in the status word and the
+// access is skipped; nothing traps.  In the normal build the test is the constant true and
+// costs nothing.  Use: if (PREBA_IN_RANGE(status, index < size)) { ... the access ... }
+#if defined(PREBA_CHECKED) && defined(__CUDACC__)
+namespace preba {
+__device__ __forceinline__ bool range_violation(int32_t* status) {
+  if (status) atomicCAS(status, 0, PREBA_ERR_RANGE);
+  return false;
+}
+}  // namespace preba
+#define PREBA_IN_RANGE(status, cond) ((cond) ? true : ::preba::range_violation(status))
+#else
+#define PREBA_IN_RANGE(status, cond) true
+#endif
+
 #endif  // PREBA_INTERNAL_H_

@@ -772,9 +772,18 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
             const uint32_t bytes = static_cast<uint32_t>(
                 ((s + is.copy_bytes + 15) & ~static_cast<uintptr_t>(15)) - s0);
             fence_async_shared();
-            mbar_arrive_expect_tx(bar, bytes);
-            bulk_copy_g2s(smem_addr(&ws.ring[slot][lane * is.stride]),
-                          reinterpret_cast<const void*>(s0), bytes, bar);
+            // checked build: the row lies in its ring group and in the pixel buffer
+            if (PREBA_IN_RANGE(p.status,
+                               lane * is.stride + bytes <= kGroupBytes &&
+                                   s0 >= reinterpret_cast<uintptr_t>(p.pixels) &&
+                                   s0 - reinterpret_cast<uintptr_t>(p.pixels) + bytes <=
+                                       p.pixels_bytes)) {
+              mbar_arrive_expect_tx(bar, bytes);
+              bulk_copy_g2s(smem_addr(&ws.ring[slot][lane * is.stride]),
+                            reinterpret_cast<const void*>(s0), bytes, bar);
+            } else {
+              mbar_arrive(bar);
+            }
           } else {
             mbar_arrive(bar);
           }
@@ -882,6 +891,16 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
           const Tap ty = axis_tap(ay, cm->k0 + t);
           const uint8_t* r0 = src + ty.i0 * pitch;
           const uint8_t* r1 = src + ty.i1 * pitch;
+#ifdef PREBA_CHECKED
+          {  // both rows and every tap of the lane inside the image, the output row inside the crop
+            bool fits = ty.i0 < h && ty.i1 < h && cm->k0 + t < C && cm->img < p.n &&
+                        cm->src + 3ull * h * w <= p.pixels_bytes;
+#pragma unroll
+            for (int m = 0; m < static_cast<int>(kLaneCols); ++m)
+              fits = fits && 3 * xmin + ln.off[m] + 6 <= 3 * w + (ln.wgt[m] ? 0u : 3u);
+            if (!PREBA_IN_RANGE(p.status, __all_sync(0xffffffffu, fits))) continue;
+          }
+#endif
 #pragma unroll
           for (int m = 0; m < static_cast<int>(kLaneCols); ++m) {
             // the right neighbour is read only where it carries weight (it exists then)
@@ -918,6 +937,27 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
       const uint32_t cnt = min(c_rpg, c_nlist - c_row);
       uint32_t row_addr = smem_addr(&ws.ring[slot][0]);
       for (uint32_t r = 0; r < cnt; ++r, row_addr += c_stride) {
+#ifdef PREBA_CHECKED
+        // every index and offset of this row before it is used: the list entry, the 12 bytes
+        // each column reads from the ring group, the output rows the row completes
+        bool fits = c_row + r < kMaxList;
+        if (fits) {
+          const uint32_t info_c = cm->info[c_row + r];
+          const uint32_t lo = smem_addr(&ws.ring[slot][0]), hi = lo + kGroupBytes;
+          const uint32_t base_c = row_addr + (info_c & 0xffu);
+#pragma unroll
+          for (int m = 0; m < static_cast<int>(kLaneCols); ++m) {
+            const uint32_t at = (base_c + ln.off[m]) & ~3u;
+            fits = fits && at >= lo && at + 12 <= hi;
+          }
+          fits = fits && t_out + (info_c >> 8) <= 32 && cm->k0 + t_out + (info_c >> 8) <= C &&
+                 cm->img < p.n;
+        }
+        if (!PREBA_IN_RANGE(p.status, __all_sync(0xffffffffu, fits))) {
+          par ^= 1u;
+          continue;
+        }
+#endif
         const uint32_t info = cm->info[c_row + r];
         const uint32_t base = row_addr + (info & 0xffu);  // the row's first tapped byte
         uint32_t e = info >> 8;
@@ -983,8 +1023,13 @@ __device__ __forceinline__ void warp_main(const Params& p, WarpShared& ws, uint3
 
 // The rounded modes keep integer row state and division constants on top of what the float
 // mode holds: at four CTAs per SM (128 registers) they spill, so they run three per SM.
+#ifdef PREBA_CHECKED
+#define PREBA_FUSED_CTAS(MODE) ((void)kCtasPerSm, 2)  // the range checks cost registers
+#else
+#define PREBA_FUSED_CTAS(MODE) ((MODE) == kFloat ? kCtasPerSm : kCtasPerSm - 1)
+#endif
 template <typename OutT, int MODE, bool CROP>
-__global__ void __launch_bounds__(kThreads, MODE == kFloat ? kCtasPerSm : kCtasPerSm - 1)
+__global__ void __launch_bounds__(kThreads, PREBA_FUSED_CTAS(MODE))
     preba_fused_kernel(const Params p) {
   __shared__ WarpShared sm[kWarpsPerCta];
   // a following launch that was marked independent of this one may start as soon as

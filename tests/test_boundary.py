@@ -138,8 +138,8 @@ def test_pack_errors():
 
 
 def test_strerror_covers_every_code():
-    texts = {pb.preba_strerror(c) for c in range(0, -8, -1)}
-    assert len(texts) == 8 and "ok" in texts
+    texts = {pb.preba_strerror(c) for c in range(0, -9, -1)}
+    assert len(texts) == 9 and "ok" in texts
     assert "unknown" in pb.preba_strerror(-99)
 
 
@@ -286,7 +286,7 @@ def test_separate_images_entry_point_rejects_bad_arguments_before_any_copy():
     assert call(out_bytes=2 * 3 * 8 * 8 * 4 - 1) == pb.ERR_BUFFER_TOO_SMALL
     assert call(dev_pixels=0x10004) == pb.ERR_INVALID_ARG          # misaligned staging
     assert call(c=9, s=8) == pb.ERR_INVALID_ARG                    # crop larger than resize
-    assert call(flags=2) == pb.ERR_INVALID_ARG                     # unknown flag
+    assert call(flags=4) == pb.ERR_INVALID_ARG                     # unknown flag
     raw = np.zeros(8 * 8 * 3 + 256, dtype=np.uint8)
     odd = raw.ctypes.data + (64 - raw.ctypes.data) % 128           # an address that is 64 mod 128
     assert odd % 128 == 64
