@@ -36,7 +36,7 @@ constexpr uint32_t kFft = PREBA_AUDIO_NFFT;
 constexpr uint32_t kBins = kFft / 2 + 1;
 constexpr uint32_t kMels = PREBA_AUDIO_MELS;
 constexpr int kWarps = 4;            // warps per CTA of the spectrogram kernel
-constexpr int kCtasPerSm = 4;
+constexpr int kCtasPerSm = 3;
 constexpr float kLogGuard = 5.9604644775390625e-08f;  // 2^-24
 constexpr float kStdGuard = 1e-5f;
 
@@ -283,13 +283,17 @@ logmel_kernel(const AudioParams p, const MelPlan plan_param) {
 #pragma unroll
     for (uint32_t n2 = 0; n2 < 6; ++n2) win[c][n2] = window[64 * n2 + lane + 32 * c];
   win6 = window[384 + lane];  // 0 from lane 16 on
-  const uint32_t i6 = lane < 16 ? 384 + lane : lane;  // a sample that exists, for a weight of 0
 #pragma unroll
   for (uint32_t k1 = 1; k1 < 8; ++k1) {
     float sn, cs;
     sincospif(-2.0f * static_cast<float>(n0 * k1) / 64.0f, &sn, &cs);
     tw2[k1 - 1] = make_float2(cs, sn);
   }
+  float2 tw1r[2][7];  // after pass 1: the lane's two columns
+#pragma unroll
+  for (int c = 0; c < 2; ++c)
+#pragma unroll
+    for (uint32_t k0 = 1; k0 < 8; ++k0) tw1r[c][k0 - 1] = tw1[k0 - 1][lane + 32 * c];
   int mel_begin[kMelRounds];
   uint32_t mel_filter[kMelRounds];
 #pragma unroll
@@ -336,39 +340,35 @@ logmel_kernel(const AudioParams p, const MelPlan plan_param) {
     if (!found) g = g_end;  // nothing left for this warp
   }
 
-  // The samples of a pair are fetched one pair ahead, into the registers the transform has
-  // just released: raw[f][c][n2] is sample 64 n2 + lane + 32 c of frame f, raw6[f] sample
-  // 384 + lane.  A pair without a second frame reads the first one twice (the duplicate
-  // spectrum is not written).
-  float raw[2][2][6], raw6[2];
+  // The samples of a pair are fetched one pair ahead, into registers the transform has just
+  // released.  The two frames overlap (the second starts 160 = 5 * 32 samples after the first),
+  // so the pair is one window of 18 slots of 32 samples: slot[k] is sample 32 k + lane of the
+  // first frame, which uses slots 0..12, and the second frame's slot j is slot j + 5.  Samples
+  // the frames do not hold (slot 12 from lane 16 on without a second frame, slot 17 from lane
+  // 16 on, slots 13..17 without a second frame) are replaced by ones that exist; they meet a
+  // window weight of 0 or belong to the duplicate frame whose spectrum is not written.
+  float slot[18];
   uint32_t frames = 0;
   auto fetch = [&]() {
     const preba_utt_t u = p.table[utt];
     frames = min(u.frames, p.t_max);
+    const bool two = 2 * q + 1 < frames;
     const float* __restrict__ x0 = p.samples + u.offset + static_cast<size_t>(2 * q) * kHop;
-    const float* __restrict__ x1 = 2 * q + 1 < frames ? x0 + kHop : x0;
     // checked build: both frames lie in the utterance and the utterance in the sample buffer
     if (!PREBA_IN_RANGE(p.status,
                         utt < p.n && 2 * q < frames &&
-                            static_cast<uint64_t>(2 * q + (2 * q + 1 < frames ? 1 : 0)) * kHop + kWin <=
-                                u.length &&
+                            static_cast<uint64_t>(2 * q + (two ? 1 : 0)) * kHop + kWin <= u.length &&
                             u.offset + u.length <= p.samples_count)) {
 #pragma unroll
-      for (int c = 0; c < 2; ++c)
-#pragma unroll
-        for (uint32_t n2 = 0; n2 < 6; ++n2) raw[0][c][n2] = raw[1][c][n2] = 0.f;
-      raw6[0] = raw6[1] = 0.f;
+      for (int k = 0; k < 18; ++k) slot[k] = 0.f;
       return;
     }
 #pragma unroll
-    for (int c = 0; c < 2; ++c)
+    for (uint32_t k = 0; k < 12; ++k) slot[k] = x0[32 * k + lane];
+    slot[12] = x0[(two || lane < 16) ? 384 + lane : lane];
 #pragma unroll
-      for (uint32_t n2 = 0; n2 < 6; ++n2) {
-        raw[0][c][n2] = x0[64 * n2 + lane + 32 * c];
-        raw[1][c][n2] = x1[64 * n2 + lane + 32 * c];
-      }
-    raw6[0] = x0[i6];
-    raw6[1] = x1[i6];
+    for (uint32_t k = 13; k < 17; ++k) slot[k] = x0[two ? 32 * k + lane : 32 * (k - 13) + lane];
+    slot[17] = x0[(two && lane < 16) ? 544 + lane : lane];
   };
   if (g < g_end) fetch();
 
@@ -385,13 +385,13 @@ logmel_kernel(const AudioParams p, const MelPlan plan_param) {
       const uint32_t pcol = lane + 32 * c;
 #pragma unroll
       for (uint32_t n2 = 0; n2 < 6; ++n2)
-        v[c][n2] = make_float2(raw[0][c][n2] * win[c][n2], raw[1][c][n2] * win[c][n2]);
-      v[c][6] = c == 0 ? make_float2(raw6[0] * win6, raw6[1] * win6) : make_float2(0.f, 0.f);
+        v[c][n2] = make_float2(slot[2 * n2 + c] * win[c][n2], slot[2 * n2 + c + 5] * win[c][n2]);
+      v[c][6] = c == 0 ? make_float2(slot[12] * win6, slot[17] * win6) : make_float2(0.f, 0.f);
       v[c][7] = make_float2(0.f, 0.f);
       fft8(v[c]);
       ws.z[pcol] = v[c][0];
 #pragma unroll
-      for (uint32_t k0 = 1; k0 < 8; ++k0) ws.z[k0 * kPitch1 + pcol] = cmul(v[c][k0], tw1[k0 - 1][pcol]);
+      for (uint32_t k0 = 1; k0 < 8; ++k0) ws.z[k0 * kPitch1 + pcol] = cmul(v[c][k0], tw1r[c][k0 - 1]);
     }
     __syncwarp();
     // Pass 2 (over n1): a lane takes k0 = (lane + 32 c) / 8 and n0 = lane % 8.
