@@ -66,6 +66,9 @@ extern "C" {
 #define PREBA_ERR_TOO_LARGE (-6)        /* the batch exceeds PREBA_NOALLOC_MAX_BYTES, or an image is
                                            reduced by more than the antialiased kernel can hold */
 #define PREBA_ERR_BAD_CROP (-7)         /* a crop window does not lie on its image's resized grid */
+#define PREBA_ERR_UNSUPPORTED (-9)      /* a JPEG stream of a kind the decoder does not take
+                                           (progressive, arithmetic-coded, 12-bit, CMYK, ...) */
+#define PREBA_ERR_BAD_STREAM (-10)      /* a JPEG stream that is malformed or cut short */
 #define PREBA_ERR_RANGE (-8)            /* only in the device status word, and only from the checked
                                            build of the library (compiled with PREBA_CHECKED): a
                                            shared-memory offset, a table index or a global address
@@ -638,6 +641,66 @@ int preba_audio_resample(const float* samples_in, uint64_t samples_in_count,
                          uint64_t samples_out_count, const preba_utt_t* table_out, uint32_t n,
                          uint32_t longest_out, uint32_t rate_in, uint32_t rate_out,
                          int32_t* status, void* stream);
+
+/*
+ * JPEG Decode -- the first unit of the paper's image pipeline (Table 1 "Decode", the largest
+ * image unit of its accelerator; Sec. 2.3 item 1: JPEG to RGB; Sec. 4.2: Decode -> Resize ->
+ * Crop -> Normalize chained in one compute unit).  The paper fixes no numerics; the decoder
+ * follows ITU-T T.81 for baseline sequential DCT streams (SOF0, 8-bit samples, Huffman coding,
+ * one interleaved scan, restart intervals; one component, or three with the luma sampled 1 or 2
+ * times the chroma on each axis).  Readings where the standard leaves a choice: the inverse
+ * DCT of A.3.3 in float64 (separable, horizontal sums first, sums in index order, no fused
+ * operations), level shift, floor(x + 1/2), clamp; chroma enlarged by pixel replication;
+ * YCbCr -> RGB by the JFIF equations in float64 on the 8-bit samples with one more
+ * floor(x + 1/2) and clamp.  Other streams are refused with PREBA_ERR_UNSUPPORTED.
+ *
+ * preba_jpeg_query   reads the headers of n streams (HOST pointers and sizes): writes every
+ *                    image's height and width (h, w: HOST, n entries, or NULL) and the sizes
+ *                    of the buffers preba_jpeg_decode needs.
+ * preba_jpeg_decode  decodes the batch into the packed pixel buffer and {offset, h, w} table
+ *                    that preba_preprocess reads (the layout of preba_pack), so the transform
+ *                    can follow on the same stream.  The host writes one descriptor per image
+ *                    (sizes, tables) and the entropy-coded bytes into `stage_host`; enqueued on
+ *                    `stream`: the copy of the staging buffer and of the table, the clearing of
+ *                    the coefficient buffer, and three kernels (restart markers found per
+ *                    image; a thread per restart interval decodes its Huffman codes into
+ *                    quantised coefficients; a block per MCU dequantises, transforms,
+ *                    converts and stores).  Streams without restart intervals decode on one
+ *                    thread each.  A stream that turns out damaged while decoding (a code that
+ *                    does not exist, restart markers that do not match the header) leaves its
+ *                    remaining blocks grey and PREBA_ERR_BAD_STREAM in `status`.
+ * Ownership: everything is the caller's; stage_host and table_host must stay valid until the
+ * stream has passed the copies (pinned memory for them to be asynchronous).
+ * Errors: PREBA_ERR_INVALID_ARG, PREBA_ERR_BAD_STREAM, PREBA_ERR_UNSUPPORTED,
+ * PREBA_ERR_BUFFER_TOO_SMALL, PREBA_ERR_CUDA.
+ */
+typedef struct {
+  uint64_t stage_bytes;  /* staging, host and device: descriptors, segment tables, scans */
+  uint64_t coef_bytes;   /* device: the int16 coefficients of every block */
+  uint64_t packed_bytes; /* device: the decoded pixels, packed as preba_pack lays them out */
+  uint64_t table_bytes;  /* n * sizeof(preba_img_t) */
+} preba_jpeg_sizes_t;
+
+typedef struct {
+  const uint8_t* const* jpegs; /* HOST array of n HOST pointers: the streams */
+  const uint64_t* bytes;       /* HOST, n entries: their sizes */
+  uint32_t n;                  /* 1 .. 65535 */
+  uint32_t reserved;
+  uint8_t* stage_host;         /* HOST (pinned), stage_bytes, 16-byte aligned: written by the call */
+  uint8_t* stage_dev;          /* DEVICE, stage_bytes, 16-byte aligned */
+  uint64_t stage_bytes;
+  int16_t* coef;               /* DEVICE, coef_bytes, 16-byte aligned */
+  uint64_t coef_bytes;
+  uint8_t* pixels;             /* DEVICE, 16-byte aligned: receives the packed pixels */
+  uint64_t pixels_bytes;
+  preba_img_t* table;          /* DEVICE, n entries: receives the table */
+  preba_img_t* table_host;     /* HOST (pinned), n entries: receives the same table */
+  int32_t* status;             /* DEVICE word or NULL, as preba_batch_t.status */
+} preba_jpeg_batch_t;
+
+int preba_jpeg_query(const uint8_t* const* jpegs, const uint64_t* bytes, uint32_t n, uint32_t* h,
+                     uint32_t* w, preba_jpeg_sizes_t* sizes);
+int preba_jpeg_decode(const preba_jpeg_batch_t* batch, void* stream);
 
 /* Text for a PREBA_* code (static storage, never NULL). */
 const char* preba_strerror(int code);

@@ -34,6 +34,8 @@ ERR_TIMEOUT = -5
 ERR_TOO_LARGE = -6
 ERR_BAD_CROP = -7
 ERR_RANGE = -8
+ERR_UNSUPPORTED = -9
+ERR_BAD_STREAM = -10
 NOALLOC_MAX_BYTES = 64 << 20
 
 EXPORTS = ("preba_query", "preba_pack", "preba_preprocess", "preba_preprocess_ex",
@@ -48,7 +50,8 @@ EXPORTS = ("preba_query", "preba_pack", "preba_preprocess", "preba_preprocess_ex
            "preba_bucket_batcher_create", "preba_bucket_batcher_destroy",
            "preba_bucket_batcher_push", "preba_bucket_batcher_poll",
            "preba_audio_query", "preba_audio_pack", "preba_audio_logmel",
-           "preba_audio_layout", "preba_audio_resample_query", "preba_audio_resample")
+           "preba_audio_layout", "preba_audio_resample_query", "preba_audio_resample",
+           "preba_jpeg_query", "preba_jpeg_decode")
 
 
 class PrebaImg(ctypes.Structure):
@@ -111,6 +114,21 @@ class PrebaServe(ctypes.Structure):
                 ("done_ns", ctypes.c_void_p), ("batch_size", ctypes.c_void_p),
                 ("batch_first", ctypes.c_void_p), ("batch_release_ns", ctypes.c_void_p),
                 ("batch_server", ctypes.c_void_p)]
+
+
+class PrebaJpegSizes(ctypes.Structure):
+    _fields_ = [("stage_bytes", ctypes.c_uint64), ("coef_bytes", ctypes.c_uint64),
+                ("packed_bytes", ctypes.c_uint64), ("table_bytes", ctypes.c_uint64)]
+
+
+class PrebaJpegBatch(ctypes.Structure):
+    _fields_ = [("jpegs", ctypes.c_void_p), ("bytes", ctypes.c_void_p), ("n", ctypes.c_uint32),
+                ("reserved", ctypes.c_uint32), ("stage_host", ctypes.c_void_p),
+                ("stage_dev", ctypes.c_void_p), ("stage_bytes", ctypes.c_uint64),
+                ("coef", ctypes.c_void_p), ("coef_bytes", ctypes.c_uint64),
+                ("pixels", ctypes.c_void_p), ("pixels_bytes", ctypes.c_uint64),
+                ("table", ctypes.c_void_p), ("table_host", ctypes.c_void_p),
+                ("status", ctypes.c_void_p)]
 
 
 class PrebaAudioSizes(ctypes.Structure):
@@ -227,6 +245,11 @@ def lib() -> ctypes.CDLL:
                                            ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32,
                                            ctypes.c_uint32, ctypes.c_void_p, ctypes.c_void_p]
         L.preba_audio_resample.restype = ctypes.c_int
+        L.preba_jpeg_query.argtypes = [ctypes.POINTER(ctypes.c_void_p), u64p, ctypes.c_uint32, u32p,
+                                       u32p, ctypes.POINTER(PrebaJpegSizes)]
+        L.preba_jpeg_query.restype = ctypes.c_int
+        L.preba_jpeg_decode.argtypes = [ctypes.POINTER(PrebaJpegBatch), ctypes.c_void_p]
+        L.preba_jpeg_decode.restype = ctypes.c_int
         L.preba_strerror.argtypes = [ctypes.c_int]
         L.preba_strerror.restype = ctypes.c_char_p
         L.preba_last_cuda_error.argtypes = []
@@ -843,3 +866,61 @@ def preba_audio_resample(samples_in, table_in, samples_out, table_out, n: int, l
                                     ctypes.c_void_p(stream))
     if rc != OK:
         raise PrebaError(rc, "preba_audio_resample")
+
+
+# ---- JPEG Decode ---------------------------------------------------------------------------------------
+
+def _streams(jpegs):
+    """The streams as contiguous uint8 arrays, their pointer array and their sizes."""
+    arrs = [np.frombuffer(j, dtype=np.uint8) if isinstance(j, (bytes, bytearray, memoryview))
+            else np.ascontiguousarray(j, dtype=np.uint8) for j in jpegs]
+    ptrs = (ctypes.c_void_p * len(arrs))(*[a.ctypes.data for a in arrs])
+    sizes = np.ascontiguousarray([a.size for a in arrs], dtype=np.uint64)
+    return arrs, ptrs, sizes
+
+
+def preba_jpeg_query(jpegs):
+    """(heights, widths, PrebaJpegSizes) of a list of JPEG streams (bytes or uint8 arrays)."""
+    arrs, ptrs, sizes = _streams(jpegs)
+    n = len(arrs)
+    h, w = np.zeros(n, dtype=np.uint32), np.zeros(n, dtype=np.uint32)
+    out = PrebaJpegSizes()
+    rc = lib().preba_jpeg_query(ptrs, _p(sizes, ctypes.c_uint64), n, _p(h, ctypes.c_uint32),
+                                _p(w, ctypes.c_uint32), ctypes.byref(out))
+    if rc != OK:
+        raise PrebaError(rc, "preba_jpeg_query")
+    return h, w, out
+
+
+class PreparedJpeg:
+    """The arguments of ``preba_jpeg_decode`` for a fixed list of streams, marshalled once.
+    ``stage_host`` and ``table_host`` are pinned CPU uint8 tensors, ``stage_dev``, ``coef`` (int16),
+    ``pixels`` (uint8), ``table`` (uint8, 16 bytes per image) and ``status`` CUDA tensors, sized
+    by ``preba_jpeg_query``."""
+
+    def __init__(self, jpegs, stage_host, stage_dev, coef, pixels, table, table_host, status=None,
+                 stream=None):
+        import torch
+
+        if stream is None:
+            stream = torch.cuda.current_stream().cuda_stream
+        elif hasattr(stream, "cuda_stream"):
+            stream = stream.cuda_stream
+        self._arrs, self._ptrs, self._sizes = _streams(jpegs)
+        b = PrebaJpegBatch()
+        b.jpegs = ctypes.cast(self._ptrs, ctypes.c_void_p)
+        b.bytes = self._sizes.ctypes.data
+        b.n = len(self._arrs)
+        b.stage_host, b.stage_dev = stage_host.data_ptr(), stage_dev.data_ptr()
+        b.stage_bytes = min(stage_host.numel(), stage_dev.numel())
+        b.coef, b.coef_bytes = coef.data_ptr(), coef.numel() * coef.element_size()
+        b.pixels, b.pixels_bytes = pixels.data_ptr(), pixels.numel() * pixels.element_size()
+        b.table, b.table_host = table.data_ptr(), table_host.data_ptr()
+        b.status = status.data_ptr() if status is not None else None
+        self._keep = (stage_host, stage_dev, coef, pixels, table, table_host, status, b)
+        self._args = (ctypes.byref(b), ctypes.c_void_p(stream))
+
+    def __call__(self) -> None:
+        rc = lib().preba_jpeg_decode(*self._args)
+        if rc != OK:
+            raise PrebaError(rc, "preba_jpeg_decode")

@@ -104,6 +104,8 @@ extern "C" const char* preba_strerror(int code) {
     case PREBA_ERR_TIMEOUT: return "device wait ran out";
     case PREBA_ERR_TOO_LARGE: return "batch exceeds the library's built-in staging space, or an image is reduced by more than the kernel can hold";
     case PREBA_ERR_BAD_CROP: return "crop window outside the resized image";
+    case PREBA_ERR_UNSUPPORTED: return "a JPEG stream of a kind that is not decoded";
+    case PREBA_ERR_BAD_STREAM: return "a malformed or truncated JPEG stream";
     case PREBA_ERR_RANGE: return "an index left its range inside a kernel (checked build)";
     default: return "unknown preba error code";
   }

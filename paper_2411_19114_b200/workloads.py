@@ -136,3 +136,21 @@ def utterances(n: int, seed: int, min_s: float = 1.5, max_s: float = 15.0) -> li
     seqs = np.random.SeedSequence(seed).spawn(n + 1)
     lens = np.random.default_rng(seqs[0]).uniform(min_s, max_s, size=n)
     return [utterance(np.random.default_rng(seqs[i + 1]), float(lens[i])) for i in range(n)]
+
+
+def jpeg_streams(images, quality: int = 90, subsampling: int = 2, restart_rows: int = 1):
+    """The images as baseline JPEG streams written by an image library (the input of the Decode
+    unit): chroma subsampling 0 (4:4:4), 1 (4:2:2) or 2 (4:2:0), a restart marker every
+    ``restart_rows`` rows of MCUs (0: none).  Stand-ins for the compressed files of the paper's
+    image workload; the content is the seeded synthetic images given."""
+    import io
+
+    from PIL import Image
+
+    out = []
+    for im in images:
+        buf = io.BytesIO()
+        extra = {"restart_marker_rows": restart_rows} if restart_rows else {}
+        Image.fromarray(im).save(buf, format="JPEG", quality=quality, subsampling=subsampling, **extra)
+        out.append(buf.getvalue())
+    return out

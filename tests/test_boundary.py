@@ -51,6 +51,7 @@ def test_header_is_plain_c(tmp_path):
         "sizeof(preba_sizes_t), sizeof(preba_batch_t), sizeof(preba_host_batch_t), "
         "sizeof(preba_image_batch_t), sizeof(preba_options_t), sizeof(preba_utt_t), "
         "sizeof(preba_audio_sizes_t), sizeof(preba_audio_batch_t), sizeof(preba_serve_t)); "
+        "printf(\"%zu %zu\\n\", sizeof(preba_jpeg_sizes_t), sizeof(preba_jpeg_batch_t)); "
         "return 0; }\n")
     exe = tmp_path / "use_header"
     subprocess.run(["gcc", "-std=c11", "-Wall", "-Wextra", "-Werror", "-pedantic",
@@ -61,7 +62,8 @@ def test_header_is_plain_c(tmp_path):
                      ctypes.sizeof(pb.PrebaBatch), ctypes.sizeof(pb.PrebaHostBatch),
                      ctypes.sizeof(pb.PrebaImageBatch), ctypes.sizeof(pb.PrebaOptions),
                      pb.UTT_DTYPE.itemsize, ctypes.sizeof(pb.PrebaAudioSizes),
-                     ctypes.sizeof(pb.PrebaAudioBatch), ctypes.sizeof(pb.PrebaServe)]
+                     ctypes.sizeof(pb.PrebaAudioBatch), ctypes.sizeof(pb.PrebaServe),
+                     ctypes.sizeof(pb.PrebaJpegSizes), ctypes.sizeof(pb.PrebaJpegBatch)]
 
 
 def test_struct_layouts_match_header():
@@ -138,8 +140,8 @@ def test_pack_errors():
 
 
 def test_strerror_covers_every_code():
-    texts = {pb.preba_strerror(c) for c in range(0, -9, -1)}
-    assert len(texts) == 9 and "ok" in texts
+    texts = {pb.preba_strerror(c) for c in range(0, -11, -1)}
+    assert len(texts) == 11 and "ok" in texts
     assert "unknown" in pb.preba_strerror(-99)
 
 
