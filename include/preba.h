@@ -648,11 +648,15 @@ int preba_audio_resample(const float* samples_in, uint64_t samples_in_count,
  * Crop -> Normalize chained in one compute unit).  The paper fixes no numerics; the decoder
  * follows ITU-T T.81 for baseline sequential DCT streams (SOF0, 8-bit samples, Huffman coding,
  * one interleaved scan, restart intervals; one component, or three with the luma sampled 1 or 2
- * times the chroma on each axis).  Readings where the standard leaves a choice: the inverse
- * DCT of A.3.3 in float64 (separable, horizontal sums first, sums in index order, no fused
- * operations), level shift, floor(x + 1/2), clamp; chroma enlarged by pixel replication;
- * YCbCr -> RGB by the JFIF equations in float64 on the 8-bit samples with one more
- * floor(x + 1/2) and clamp.  Other streams are refused with PREBA_ERR_UNSUPPORTED.
+ * times the chroma on each axis).  Readings where the standard leaves a choice (it only bounds
+ * the accuracy of the inverse transform): the inverse DCT of A.3.3 in exact integers -- the basis
+ * as round(2^20 (C_u / 2) cos((2x+1) u pi / 16)), dequantised coefficients limited to +-16383,
+ * horizontal sums first, reduced to floor((t + 2^8) / 2^9), vertical sums, level shift and one
+ * rounding floor((s + 128 * 2^31 + 2^30) / 2^31), clamp -- within one of the rounded real-valued
+ * transform; chroma enlarged by pixel replication; YCbCr -> RGB by the JFIF equations on the
+ * 8-bit samples with the coefficients as round(2^16 c) (91881, 22553, 46802, 116130) and one
+ * rounding floor((x + 2^15) / 2^16), clamp.  Every decoder that follows these steps produces the
+ * same bytes.  Other streams are refused with PREBA_ERR_UNSUPPORTED.
  *
  * preba_jpeg_query   reads the headers of n streams (HOST pointers and sizes): writes every
  *                    image's height and width (h, w: HOST, n entries, or NULL) and the sizes

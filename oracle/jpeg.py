@@ -14,18 +14,25 @@ the order of the standard's decoder:
      natural order through the zig-zag sequence (Figure A.6); at a restart marker the bit
      reader moves to the next byte and the predictors return to 0 (F.2.1.3.1, E.2.4);
   4. dequantisation S = Sq * Q (A.3.4);
-  5. the inverse DCT of A.3.3 in float64, separable, horizontal sums first, every sum taken
-     in index order; level shift by 128; one rounding floor(x + 1/2); clamp to 0..255;
+  5. the inverse DCT of A.3.3 in exact integer arithmetic: the basis (C_u / 2) cos((2x+1) u pi/16)
+     as integers B = round(2^20 * basis), the dequantised coefficient limited to +-16383 (a valid
+     stream stays far inside), horizontal sums t = sum_u B[x][u] S[v][u], reduced to
+     t' = floor((t + 2^8) / 2^9), vertical sums s = sum_v B[y][v] t'[v][x] (scale 2^31), level
+     shift and one rounding floor((s + 128 * 2^31 + 2^30) / 2^31), clamp to 0..255;
   6. components with fewer samples are enlarged by pixel replication (the standard leaves
      upsampling open; replication is the reading taken), planes are cut to the frame size;
-  7. YCbCr -> RGB by the JFIF equations in float64 on the 8-bit samples, one more rounding
-     floor(x + 1/2) and clamp; a single component is written to all three channels.
+  7. YCbCr -> RGB by the JFIF equations on the 8-bit samples with the coefficients as integers
+     round(2^16 * c): R = floor((2^16 Y + 91881 Cr' + 2^15) / 2^16), G = floor((2^16 Y -
+     22553 Cb' - 46802 Cr' + 2^15) / 2^16), B = floor((2^16 Y + 116130 Cb' + 2^15) / 2^16),
+     Cb' = Cb - 128, Cr' = Cr - 128, clamped; a single component goes to all three channels.
 
-Readings where the standard is silent or leaves a choice: the arithmetic of step 5 and 7
-(float64, the stated operation order, ties upward), replication in step 6, and what is refused
-(progressive, arithmetic-coded, 12-bit, four-component, multi-scan frames, DNL).  Where a floating
-sum decides an integer both this file and the CUDA path take the decision in float64 with the
-same order of operations, so the decoded bytes are compared bit for bit.
+Readings where the standard is silent or leaves a choice: the arithmetic of steps 5 and 7, which
+the standard only bounds in accuracy (an approximation of the real-valued transform: integers, so
+that every decoder following these steps produces the same bytes; `idct_blocks` below is the
+real-valued definition in float64 and the pins hold the integer steps to it: a sample differs
+from the rounded definition in about one case in a thousand, never by more than one),
+replication in step 6, and what is refused (progressive, arithmetic-coded, 12-bit,
+four-component, multi-scan frames, DNL).  The decoded bytes are compared bit for bit.
 
 Pins (tests/test_jpeg_oracle_pins.py): hand-built blocks (DC only, one AC coefficient against
 the closed form), the inverse transform against scipy's before rounding, an encoder written in
@@ -323,9 +330,9 @@ def entropy_decode(data: bytes, frame: Frame | None = None) -> list[np.ndarray]:
 
 
 def idct_blocks(coef: np.ndarray) -> np.ndarray:
-    """Inverse DCT of A.3.3 for blocks [..., 64] of dequantised coefficients (natural order
-    8 v + u): float64 [..., 8, 8] before the level shift.  Horizontal sums first, every sum in
-    index order, products and sums rounded one by one (no fused operations)."""
+    """The real-valued inverse DCT of A.3.3 for blocks [..., 64] of dequantised coefficients
+    (natural order 8 v + u) in float64: [..., 8, 8] before the level shift.  The definition the
+    integer steps approximate; not used by `decode`."""
     a = idct_basis()
     s = coef.astype(np.float64).reshape(coef.shape[:-1] + (8, 8))   # [.., v, u]
     rows = np.zeros(s.shape, dtype=np.float64)                        # [.., v, x]
@@ -343,26 +350,42 @@ def idct_blocks(coef: np.ndarray) -> np.ndarray:
     return out
 
 
+def integer_basis() -> np.ndarray:
+    """B[x][u] = round(2^20 * (C_u / 2) cos((2x + 1) u pi / 16))."""
+    return np.rint(idct_basis() * float(1 << 20)).astype(np.int64)
+
+
+def idct_blocks_int(deq: np.ndarray) -> np.ndarray:
+    """Step 5's sums for blocks [..., 64] of dequantised coefficients: int64 [..., 8, 8], the
+    samples before the level shift times 2^31."""
+    b = integer_basis()
+    s = np.clip(deq.astype(np.int64), -16383, 16383).reshape(deq.shape[:-1] + (8, 8))  # [.., v, u]
+    t = np.einsum("xu,...vu->...vx", b, s)                     # exact: below 2^38
+    t = (t + (1 << 8)) >> 9                                    # floor division: below 2^29
+    return np.einsum("yv,...vx->...yx", b, t)                  # exact: below 2^52
+
+
 def samples(coef_q: np.ndarray, qtable: list[int]) -> np.ndarray:
     """One component's sample plane (uint8) from its quantised coefficients: dequantise,
-    inverse DCT, level shift, floor(x + 1/2), clamp."""
+    integer inverse DCT, level shift, one rounding, clamp."""
     q = np.asarray(qtable, dtype=np.int64)
-    deq = coef_q.astype(np.int64) * q
-    pix = np.floor((idct_blocks(deq) + 128.0) + 0.5)
-    pix = np.clip(pix, 0.0, 255.0).astype(np.uint8)                   # [by, bx, y, x]
+    total = idct_blocks_int(coef_q.astype(np.int64) * q)
+    pix = (total + (128 << 31) + (1 << 30)) >> 31
+    pix = np.clip(pix, 0, 255).astype(np.uint8)                       # [by, bx, y, x]
     by, bx = pix.shape[0], pix.shape[1]
     return pix.transpose(0, 2, 1, 3).reshape(by * 8, bx * 8)
 
 
 def ycbcr_to_rgb(y: np.ndarray, cb: np.ndarray, cr: np.ndarray) -> np.ndarray:
     """JFIF: R = Y + 1.402 (Cr - 128), G = Y - 0.344136 (Cb - 128) - 0.714136 (Cr - 128),
-    B = Y + 1.772 (Cb - 128); float64, floor(x + 1/2), clamp."""
-    yf = y.astype(np.float64)
-    cbf, crf = cb.astype(np.float64) - 128.0, cr.astype(np.float64) - 128.0
-    r = np.floor((yf + 1.402 * crf) + 0.5)
-    g = np.floor(((yf - 0.344136 * cbf) - 0.714136 * crf) + 0.5)
-    b = np.floor((yf + 1.772 * cbf) + 0.5)
-    return np.clip(np.stack([r, g, b], axis=-1), 0.0, 255.0).astype(np.uint8)
+    B = Y + 1.772 (Cb - 128), the coefficients as integers round(2^16 c), one rounding
+    floor((x + 2^15) / 2^16), clamp."""
+    yi = y.astype(np.int64) << 16
+    cbi, cri = cb.astype(np.int64) - 128, cr.astype(np.int64) - 128
+    r = (yi + 91881 * cri + (1 << 15)) >> 16
+    g = (yi - 22553 * cbi - 46802 * cri + (1 << 15)) >> 16
+    b = (yi + 116130 * cbi + (1 << 15)) >> 16
+    return np.clip(np.stack([r, g, b], axis=-1), 0, 255).astype(np.uint8)
 
 
 def decode(data: bytes) -> np.ndarray:

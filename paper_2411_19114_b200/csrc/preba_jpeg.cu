@@ -12,14 +12,13 @@
 //   decode_segments a thread per restart interval reads its bits (0xFF00 unstuffed), decodes the
 //                   DC differences and AC runs of its MCUs and writes the quantised coefficients
 //                   of every block in natural order (int16);
-//   idct_colour     a block per MCU: dequantisation, the inverse DCT of T.81 A.3.3 in float64
-//                   (separable, horizontal sums first, sums in index order, every product and
-//                   sum rounded on its own), level shift, floor(x + 1/2), clamp; chroma enlarged
-//                   by replication; YCbCr -> RGB by the JFIF equations in float64 with one more
-//                   rounding; the pixels go straight into the packed HWC buffer and the
-//                   {offset, h, w} table that preba_preprocess reads.
-// Where a floating sum decides an integer the order of operations is fixed (no fused
-// multiply-add), so that the decoded bytes are reproducible bit for bit.
+//   idct_colour     a block per MCU: dequantisation, the inverse DCT of T.81 A.3.3 in exact
+//                   integers (the basis times 2^20, horizontal sums first and reduced by 2^9,
+//                   vertical sums at scale 2^31, level shift, one rounding, clamp); chroma
+//                   enlarged by replication; YCbCr -> RGB by the JFIF equations with the
+//                   coefficients times 2^16 and one rounding; the pixels go straight into the
+//                   packed HWC buffer and the {offset, h, w} table that preba_preprocess reads.
+// Integer arithmetic throughout, so the decoded bytes are reproducible bit for bit.
 #include <cuda_runtime.h>
 
 #include <cstdint>
@@ -428,36 +427,29 @@ __global__ void __launch_bounds__(64) decode_segments(const Params p) {
   }
 }
 
-// cos(k pi / 16), k = 0..7, correctly rounded to double.
-__device__ const double kCos16[8] = {1.0,
-                                     0.9807852804032304,
-                                     0.9238795325112867,
-                                     0.8314696123025452,
-                                     0.7071067811865476,
-                                     0.5555702330196022,
-                                     0.3826834323650898,
-                                     0.19509032201612828};
+// round(2^20 * cos(k pi / 16) / 2), k = 0..7.
+__device__ const int32_t kCosFix[8] = {524288, 514214, 484379, 435930, 370728, 291279, 200636, 102284};
 
-// (C_u / 2) cos((2x + 1) u pi / 16) of T.81 A.3.3, from the eight values by symmetry.
-__device__ __forceinline__ double basis(uint32_t x, uint32_t u) {
-  if (u == 0) return 0.5 * kCos16[4];
+// round(2^20 (C_u / 2) cos((2x + 1) u pi / 16)) of T.81 A.3.3, from the eight values by symmetry.
+__device__ __forceinline__ int32_t basis(uint32_t x, uint32_t u) {
+  if (u == 0) return kCosFix[4];
   uint32_t k = ((2 * x + 1) * u) & 31u;
   if (k > 16) k = 32 - k;
-  return k <= 7 ? 0.5 * kCos16[k] : (k == 8 ? 0.0 : -0.5 * kCos16[16 - k]);
+  return k <= 7 ? kCosFix[k] : (k == 8 ? 0 : -kCosFix[16 - k]);
 }
 
-__device__ __forceinline__ uint32_t round_clamp(double x) {
-  const double r = floor(__dadd_rn(x, 0.5));
-  return r <= 0.0 ? 0u : (r >= 255.0 ? 255u : static_cast<uint32_t>(r));
+__device__ __forceinline__ uint32_t clamp255(int64_t v) {
+  return v <= 0 ? 0u : (v >= 255 ? 255u : static_cast<uint32_t>(v));
 }
 
 // A block per MCU (blockIdx.y: image): 64 threads per 8 x 8 block of the MCU transform it, then
-// the threads convert the MCU's pixels and store them.
+// the threads convert the MCU's pixels and store them.  Exact integer arithmetic throughout:
+// the basis times 2^20, the row sums reduced by 2^9, the column sums at scale 2^31.
 constexpr uint32_t kMaxMcuBlocks = 6;
 
 __global__ void __launch_bounds__(64 * kMaxMcuBlocks) idct_colour(const Params p) {
-  __shared__ double a[64];                       // the basis
-  __shared__ double work[kMaxMcuBlocks][64];     // dequantised coefficients, then row sums
+  __shared__ int32_t a[64];                      // the basis
+  __shared__ int32_t work[kMaxMcuBlocks][64];    // dequantised coefficients, then row sums
   __shared__ uint8_t smp[kMaxMcuBlocks][64];     // the samples of the MCU's blocks
   const Desc& d = desc_of(p, blockIdx.y);
   const uint32_t mcus = d.mcu_cols * d.mcu_rows;
@@ -475,29 +467,30 @@ __global__ void __launch_bounds__(64 * kMaxMcuBlocks) idct_colour(const Params p
       ++comp;
     }
     const int16_t* coef = p.coef + (d.coef_off + static_cast<uint64_t>(blockIdx.x) * per_mcu + blk) * 64;
-    // S = Sq * Q (A.3.4): exact in double
-    work[blk][e] = static_cast<double>(static_cast<int32_t>(coef[e]) *
-                                       static_cast<int32_t>(d.qt[comp][e]));
+    // S = Sq * Q (A.3.4), limited to what the sums below hold (a valid stream stays far inside)
+    const int32_t deq = static_cast<int32_t>(coef[e]) * static_cast<int32_t>(d.qt[comp][e]);
+    work[blk][e] = max(-16383, min(16383, deq));
   }
   __syncthreads();
-  double rowsum = 0.0;
+  int32_t rowsum = 0;
   if (live) {
-    // horizontal sums: thread (v, x) of the block; u in index order
+    // horizontal sums: thread (v, x) of the block
     const uint32_t v = e >> 3, x = e & 7u;
-    rowsum = __dmul_rn(a[8 * x], work[blk][8 * v]);
+    int64_t t = 0;
 #pragma unroll
-    for (uint32_t u = 1; u < 8; ++u)
-      rowsum = __dadd_rn(rowsum, __dmul_rn(a[8 * x + u], work[blk][8 * v + u]));
+    for (uint32_t u = 0; u < 8; ++u)
+      t += static_cast<int64_t>(a[8 * x + u]) * work[blk][8 * v + u];
+    rowsum = static_cast<int32_t>((t + (1 << 8)) >> 9);
   }
   __syncthreads();
   if (live) work[blk][e] = rowsum;  // [v][x]
   __syncthreads();
   if (live) {
     const uint32_t y = e >> 3, x = e & 7u;
-    double s = __dmul_rn(a[8 * y], work[blk][x]);
+    int64_t s = 0;
 #pragma unroll
-    for (uint32_t v = 1; v < 8; ++v) s = __dadd_rn(s, __dmul_rn(a[8 * y + v], work[blk][8 * v + x]));
-    smp[blk][e] = static_cast<uint8_t>(round_clamp(__dadd_rn(s, 128.0)));
+    for (uint32_t v = 0; v < 8; ++v) s += static_cast<int64_t>(a[8 * y + v]) * work[blk][8 * v + x];
+    smp[blk][e] = static_cast<uint8_t>(clamp255((s + (128ll << 31) + (1ll << 30)) >> 31));
   }
   __syncthreads();
   // the MCU's pixels: 8 hmax x 8 vmax; a chroma sample serves hmax x vmax of them
@@ -515,12 +508,13 @@ __global__ void __launch_bounds__(64 * kMaxMcuBlocks) idct_colour(const Params p
     if (d.ncomp == 3) {
       const uint32_t cx = px / d.hmax, cy = py / d.vmax;  // chroma sampled once per MCU block
       const uint32_t nluma = d.hs[0] * d.vs[0];
-      const double yf = static_cast<double>(ys);
-      const double cb = static_cast<double>(smp[nluma][8 * cy + cx]) - 128.0;
-      const double cr = static_cast<double>(smp[nluma + 1][8 * cy + cx]) - 128.0;
-      r = round_clamp(__dadd_rn(yf, __dmul_rn(1.402, cr)));
-      g = round_clamp(__dsub_rn(__dsub_rn(yf, __dmul_rn(0.344136, cb)), __dmul_rn(0.714136, cr)));
-      b = round_clamp(__dadd_rn(yf, __dmul_rn(1.772, cb)));
+      const int64_t y16 = static_cast<int64_t>(ys) << 16;
+      const int64_t cb = static_cast<int64_t>(smp[nluma][8 * cy + cx]) - 128;
+      const int64_t cr = static_cast<int64_t>(smp[nluma + 1][8 * cy + cx]) - 128;
+      // the JFIF coefficients as round(2^16 c); one rounding each
+      r = clamp255((y16 + 91881 * cr + (1 << 15)) >> 16);
+      g = clamp255((y16 - 22553 * cb - 46802 * cr + (1 << 15)) >> 16);
+      b = clamp255((y16 + 116130 * cb + (1 << 15)) >> 16);
     }
     uint8_t* out = img + 3ull * (static_cast<uint64_t>(gy) * d.w + gx);
     out[0] = static_cast<uint8_t>(r);

@@ -1,7 +1,7 @@
 """GPU parity of the JPEG Decode unit against its oracle through the C ABI: quantised
-coefficients and decoded RGB bytes bit for bit (integer work; the floating sums that decide a
-byte are taken in float64 in the same order on both sides), the packed layout and table, the
-chain into the transform, and the refusals."""
+coefficients and decoded RGB bytes bit for bit (integer work from the entropy decoder to the
+colour conversion: both sides take the same exact-integer inverse transform), the packed layout
+and table, the chain into the transform, and the refusals."""
 from __future__ import annotations
 
 import ctypes

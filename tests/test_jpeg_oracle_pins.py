@@ -89,6 +89,30 @@ def test_inverse_transform_against_a_library_routine():
     assert np.allclose(oj.idct_blocks(blocks), want, atol=1e-9)
 
 
+def test_integer_transform_against_the_real_valued_definition():
+    """The integer steps reproduce the rounded real-valued transform except near ties: never
+    more than one apart, about one sample in a thousand."""
+    rng = np.random.default_rng(4)
+    # coefficients shaped like those of images: large at low frequencies, small at high ones
+    scale = 600.0 / (1.0 + np.add.outer(np.arange(8), np.arange(8))) ** 1.5
+    deq = np.rint(rng.normal(size=(4000, 8, 8)) * scale).astype(np.int64).reshape(4000, 64)
+    exact = oj.idct_blocks(deq)
+    got = oj.idct_blocks_int(deq)
+    assert float(np.max(np.abs(got / float(1 << 31) - exact))) <= 2e-3   # the sums themselves
+    want = np.clip(np.floor(exact + 128.5), 0, 255)
+    have = np.clip((got + (128 << 31) + (1 << 30)) >> 31, 0, 255)
+    diff = np.abs(have - want)
+    assert int(diff.max()) <= 1 and float((diff != 0).mean()) <= 3e-3
+    # the basis constants: 2^20 times the cosines, rounded
+    b = oj.integer_basis()
+    assert b[0, 0] == 370728 and b[0, 1] == 514214 and b[1, 1] == 435930 and b[0, 7] == 102284
+    assert np.all(np.abs(b / float(1 << 20) - oj.idct_basis()) <= 0.5 / (1 << 20))
+    # coefficients beyond what a valid stream holds are limited, not wrapped
+    huge = np.zeros((1, 64), dtype=np.int64)
+    huge[0, 0] = 10 ** 6
+    assert np.all(oj.idct_blocks_int(huge) == oj.idct_blocks_int(np.minimum(huge, 16383)))
+
+
 def test_samples_round_once_and_clamp():
     q = [1] * 64
     coef = np.zeros((1, 3, 64), dtype=np.int32)
