@@ -39,15 +39,15 @@ FALLBACK_HBM_GBS = 6650.0
 # without cache flushes between launches, divided by the launch count (so the write-back of a
 # launch's result, which happens while later launches run, is inside the window).  Valid only
 # for the kernel sources with this digest (else reported as null).
-NCU_TRAFFIC = {"csrc_sha1": "", "bytes_per_launch": 0}
+NCU_TRAFFIC = {"csrc_sha1": "e32d7677e8894a744d578d45ab02134ed607a9f2", "bytes_per_launch": 75661344 + 76510784}
 TRAFFIC_NOTE = ("dram read + write bytes summed over 8 consecutive launches of this loop (one "
                 "ncu pass, caches not flushed between launches) / 8")
 
 
 # The same for the antialiased kernel: captured on 32 frames of 1080 x 1920 (traffic grows in
 # proportion to the frames, so a launch over n frames is taken as n / 32 of it).
-AA_NCU_TRAFFIC = {"csrc_sha1": "ec70208c7fbcd001aabcdd3ef84bcaec23248a4f", "frames": 32,
-                  "bytes": 91977216 + 4739840}
+AA_NCU_TRAFFIC = {"csrc_sha1": "5c8d3788196ee0d875094ba210cee84d16dc62b8", "frames": 32,
+                  "bytes": 89862400 + 5886720}
 
 
 def csrc_digest(name: str = "preba_kernels.cu") -> str:
@@ -732,6 +732,19 @@ def run_serve(args, local_rank: int) -> None:
     print(json.dumps(line), flush=True)
 
 
+def jpeg_roofline(compressed: int, decoded: int, decode_ms: float) -> dict:
+    """Decode against the memory it has to touch: the compressed bytes in, the pixels out."""
+    peak, source = measured_peak()
+    alg = compressed + decoded
+    achieved = alg / (decode_ms * 1e-3) / 1e9
+    return {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+            "frac": achieved / peak, "traffic": None, "peak_source": source,
+            "algorithmic_bytes_per_launch": alg, "kernel_us": 1e3 * decode_ms,
+            "note": "the three Decode kernels of a step together (device time); Decode is bound "
+                    "by the serial Huffman decoding of a restart interval per thread (latency), "
+                    "far from any memory or pipe limit; see the launch list under profiles/"}
+
+
 def run_jpeg(args, local_rank: int) -> None:
     """Decode in front of the transform (the paper's Decode -> Resize -> Crop -> Normalize chain,
     Sec. 4.2, Table 1): 256 mixed-size synthetic images as baseline JPEG streams (quality 90,
@@ -844,11 +857,8 @@ def run_jpeg(args, local_rank: int) -> None:
         "timing": "wall clock around the loop of steps (host work is part of a step); "
                   "device_ms_per_step from events on the stream",
         "steps_detail": results,
-        "roofline": {"bound": "alu", "achieved": None, "peak": None, "unit": "TFLOP/s",
-                     "frac": None, "traffic": None,
-                     "note": "Decode is bound by the serial Huffman decoding of a restart "
-                             "interval per thread (latency), not by a pipe or by memory; see "
-                             "the launch list under profiles/"},
+        "roofline": jpeg_roofline(comp_bytes, int(sz.packed_bytes),
+                                  results["decode_only"]["device_ms_per_step"]),
         "cpu_baseline": {"value": done_cpu / spent, "unit": UNIT, "cores": 1, "kind": "oracle",
                          "sample": f"{done_cpu} of the {n} streams, decode only (plain Python)"},
         "e2e": {"value": both["images_per_s"], "unit": UNIT,
@@ -990,7 +1000,9 @@ def run_ours(args, rank: int, world: int, local_rank: int) -> None:
         pb.preba_preprocess_ex(pix[0], tab, n, ref, C, S, wl.MEAN, wl.STD, out_dtype,
                                round_u8=True, stream=stream, status=status, scratch=scratch)
     torch.cuda.synchronize()
-    assert all(bool(torch.equal(o, ref)) for o in outs), "overlapped launches changed the result"
+    written = min(sets, n_warm + args.steps)     # a short run does not reach every set
+    assert all(bool(torch.equal(o, ref)) for o in outs[:written]), \
+        "overlapped launches changed the result"
     if args.variant != "plain":
         report_variant(args, rank, world, n, elapsed_ms, acct, desc, dtype, sets, step_bytes, l2,
                        clocks, dist, dev, t_host, launch_note)
