@@ -49,6 +49,8 @@ struct Params {
   uint32_t mma_rows;     // output rows per CTA of the tensor-core kernel (<= kMmaRows)
   uint32_t mma_smem;     // bytes of shared memory of the tensor-core kernel's launch; images it
                          // can take (mma_plan) are left to it by the other kernel.  0: none are
+  uint32_t mm2_rows;     // the same two for the kernel with both passes on the tensor cores
+  uint32_t mm2_smem;     // (mm2_plan), which comes first in the choice
   float mul[3], add[3];  // y = v * mul + add
 };
 
@@ -225,6 +227,80 @@ __host__ __device__ inline bool mma_plan(const Axis& ax, const Axis& ay, uint32_
   if (out) *out = p;
   return true;
 }
+
+// ---- both passes on the tensor cores ----------------------------------------------------------------
+//
+// For images reduced more than 2.5 times vertically the vertical pass is a matrix product too,
+// and chaining it to the horizontal one keeps H out of shared memory altogether.  The
+// horizontal product is taken transposed: the integer weights of five resized pixels x three
+// channels are the A operand (16 rows, one unused; built once per warp, in registers), the
+// bytes of eight input rows the B operand, again exactly as the rows lie in the ring, so a lane
+// ends up with H[(x, ch)][input row] for (x, ch) = g, g + 8 and rows 2q, 2q + 1 of each
+// eight: the layout an A operand has, with the input rows as its k index.  H is below 2^24;
+// its three bytes go through byte permutes into three A operands, the integer weights of the
+// (at most eight) output rows that lie under the sixteen input rows, split into two bytes, are
+// the B operand, and four more matrix instructions add the six byte products into four
+// accumulators, one per power of 256.  Everything up to there is exact integer arithmetic;
+// an output row whose last tap has passed is put together in fp32, normalised and stored.
+// A warp owns its (x, ch) tiles from the ring to the store: there is no CTA-wide barrier after
+// the start, only the ring's full and empty barriers.
+constexpr uint32_t kT2Px = 5;                        // resized pixels of an M-tile
+constexpr uint32_t kT2Tiles = 15;                    // M-tiles of a CTA (warp w owns w and w + 8)
+constexpr uint32_t kT2Group = kT2Px * kT2Tiles;      // output columns per CTA
+constexpr uint32_t kT2MaxSlots = 6;                  // 16-row slots of the ring, at most
+constexpr uint32_t kT2Warps = kMmaThreads / 32;
+
+struct Mm2Plan {
+  uint32_t seg;    // bytes of one staged input row in the ring
+  uint32_t slots;  // 16-row slots of the ring
+  uint32_t ks;     // 32-byte steps of an M-tile's window (3 or 4)
+  uint32_t off_wx, off_xlo, off_xcnt, off_invx, off_ylo, off_yhi, off_invy, off_bar, off_ring;
+};
+
+// Whether the kernel with both passes on the tensor cores takes an image, and its
+// shared-memory layout if so.  The same function decides in every kernel and on the host.
+__host__ __device__ inline bool mm2_plan(const Axis& ax, const Axis& ay, uint32_t w, uint32_t C,
+                                         uint32_t smem_bytes, Mm2Plan* out) {
+  if (smem_bytes == 0 || (w & 3u) != 0) return false;  // rows must start on the same byte phase
+  if (ax.M > 32767u || ay.M > 32767u) return false;    // weights in two bytes, 32-bit tap arithmetic
+  if (ax.taps > kMaxTapsX || ay.taps > 32u) return false;
+  if (255ull * ax.taps * 2ull * ax.M >= (1ull << 24)) return false;  // H in three bytes
+  // at most eight output rows have taps among sixteen input rows: floor(15 R / n_in) + 3 <= 8
+  if (ay.n_in <= ay.R || 15ull * ay.R / ay.n_in + 3ull > 8ull) return false;
+  // the bytes of a row under an M-tile: first taps of its pixels at most ceil(4 n_in / R) + 1
+  // apart, one pixel's taps, three bytes of alignment
+  const uint64_t px_tile = (4ull * ax.n_in + ax.R - 1u) / ax.R + 1u + ax.taps;
+  uint32_t ks = static_cast<uint32_t>((3ull * px_tile + 3u + 31u) / 32u);
+  if (ks > 4u) return false;
+  if (ks < 3u) ks = 3u;
+  const uint32_t cols = C < kT2Group ? C : kT2Group;
+  const uint64_t px = (static_cast<uint64_t>(cols - 1u) * ax.n_in + ax.R - 1u) / ax.R + ax.taps + 3u;
+  Mm2Plan p;
+  p.ks = ks;
+  // a staged row: up to 15 bytes of skew, the bytes under the group, the overshoot of the last
+  // window; 16 modulo 128, so that the eight rows a warp reads together lie four banks apart
+  p.seg = static_cast<uint32_t>(((16u + 3u * px + 32u * ks + 111u) & ~127ull) + 16u);
+  uint32_t at = 0;
+  p.off_wx = at, at += kT2Group * kMaxTapsX * 2u;
+  at = (at + 3u) & ~3u;
+  p.off_xlo = at, at += kT2Group * 4u;
+  p.off_xcnt = at, at += kT2Group * 4u;
+  p.off_invx = at, at += kT2Group * 4u;
+  p.off_ylo = at, at += kMmaRows * 4u;
+  p.off_yhi = at, at += kMmaRows * 4u;
+  p.off_invy = at, at += kMmaRows * 4u;
+  at = (at + 7u) & ~7u;
+  p.off_bar = at, at += 2u * kT2MaxSlots * 8u;
+  at = (at + 15u) & ~15u;
+  p.off_ring = at;
+  if (smem_bytes <= at) return false;
+  const uint64_t room = (smem_bytes - at) / (16ull * p.seg);
+  if (room < 2) return false;
+  p.slots = room > kT2MaxSlots ? kT2MaxSlots : static_cast<uint32_t>(room);
+  if (out) *out = p;
+  return true;
+}
+
 
 __device__ __forceinline__ void report(int32_t* status, int code) {
   if (status) atomicCAS(status, 0, code);
@@ -457,7 +533,9 @@ __global__ void __launch_bounds__(kThreads) preba_antialias_kernel(const Params 
     left = (rw - C) / 2;
   }
   const Axis ax = make_axis(e.w, rw), ay = make_axis(e.h, rh);
-  if (mma_plan(ax, ay, e.w, C, p.mma_smem, nullptr)) return;  // the tensor-core kernel's image
+  if (mm2_plan(ax, ay, e.w, C, p.mm2_smem, nullptr) ||
+      mma_plan(ax, ay, e.w, C, p.mma_smem, nullptr))
+    return;  // a tensor-core kernel's image
   const Plan pl = make_plan(ax, ay, C, p.rows);
   if (pl.off_ring > p.smem_floats) {
     if (tid == 0) report(p.status, PREBA_ERR_TOO_LARGE);
@@ -755,7 +833,8 @@ __global__ void __launch_bounds__(kMmaThreads, 2) preba_antialias_mma_kernel(con
   }
   const Axis ax = make_axis(e.w, rw), ay = make_axis(e.h, rh);
   MmaPlan pl;
-  if (!mma_plan(ax, ay, e.w, C, p.mma_smem, &pl)) return;  // the other kernel's image
+  if (mm2_plan(ax, ay, e.w, C, p.mm2_smem, nullptr)) return;  // the chained kernel's image
+  if (!mma_plan(ax, ay, e.w, C, p.mma_smem, &pl)) return;    // the general kernel's image
 
   float* hbuf = reinterpret_cast<float*>(smem_b + pl.off_h);
   uint16_t* wxi = reinterpret_cast<uint16_t*>(smem_b + pl.off_wx);
@@ -1034,6 +1113,394 @@ __global__ void __launch_bounds__(kMmaThreads, 2) preba_antialias_mma_kernel(con
   }
 }
 
+__device__ __forceinline__ void mma_f16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0,
+                                        uint32_t b1) {
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+      "{%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// Two bytes of x (bytes 0 and 1 if PAIR == 0, bytes 2 and 3 if PAIR == 1) as a pair of binary16
+// numbers, each times a power of two: a byte b under the exponent byte 0x64 is the number
+// 1024 + b, and one fused multiply-add, (1024 + b) * mul - 1024 * mul, leaves b * mul exactly
+// (mul and off are the binary16 patterns of mul and of -1024 * mul).
+template <uint32_t PAIR>
+__device__ __forceinline__ uint32_t expand_bytes(uint32_t x, uint32_t mul, uint32_t off) {
+  const uint32_t biased = __byte_perm(x, 0x64646464u, PAIR == 0 ? 0x4140u : 0x4342u);
+  uint32_t r;
+  const uint32_t mul2 = mul | (mul << 16), off2 = off | (off << 16);
+  asm("fma.rn.f16x2 %0, %1, %2, %3;" : "=r"(r) : "r"(biased), "r"(mul2), "r"(off2));
+  return r;
+}
+
+template <typename OutT, uint32_t KS>
+__global__ void __launch_bounds__(kMmaThreads, 2) preba_antialias_mm2_kernel(const Params p) {
+  extern __shared__ __align__(16) uint8_t smem_b[];
+  const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5, C = p.C;
+  const uint32_t chunks = (C + p.mm2_rows - 1) / p.mm2_rows, groups = (C + kT2Group - 1) / kT2Group;
+  const uint32_t img = blockIdx.x / (chunks * groups);
+  const uint32_t rest = blockIdx.x - img * chunks * groups;
+  const uint32_t k0 = (rest / groups) * p.mm2_rows, xg0 = (rest % groups) * kT2Group;
+  const preba_img_t e = p.table[img];
+  const uint64_t usable = p.pixels_bytes & ~15ull;
+  if (e.h < 1 || e.w < 1 || e.h > PREBA_MAX_DIM || e.w > PREBA_MAX_DIM ||
+      e.offset % PREBA_PACK_ALIGN != 0 || e.offset > usable ||
+      3ull * e.h * e.w > usable - e.offset) {
+    if (tid == 0 && rest == 0 && KS == 3u) report(p.status, PREBA_ERR_BAD_TABLE);
+    return;
+  }
+  uint32_t rh, rw, top, left;
+  resized_size(e.h, e.w, p.S, &rh, &rw);
+  if (p.crop) {
+    top = p.crop[2 * img];
+    left = p.crop[2 * img + 1];
+    if (static_cast<uint64_t>(top) + C > rh || static_cast<uint64_t>(left) + C > rw) {
+      if (tid == 0 && rest == 0 && KS == 3u) report(p.status, PREBA_ERR_BAD_CROP);
+      return;
+    }
+  } else {
+    top = (rh - C) / 2;
+    left = (rw - C) / 2;
+  }
+  const Axis ax = make_axis(e.w, rw), ay = make_axis(e.h, rh);
+  Mm2Plan pl;
+  if (!mm2_plan(ax, ay, e.w, C, p.mm2_smem, &pl) || pl.ks != KS) return;  // another kernel's image
+
+  uint16_t* wxi = reinterpret_cast<uint16_t*>(smem_b + pl.off_wx);
+  uint32_t* xlo = reinterpret_cast<uint32_t*>(smem_b + pl.off_xlo);
+  uint32_t* xcnt = reinterpret_cast<uint32_t*>(smem_b + pl.off_xcnt);
+  float* invx = reinterpret_cast<float*>(smem_b + pl.off_invx);
+  uint32_t* ylo = reinterpret_cast<uint32_t*>(smem_b + pl.off_ylo);
+  uint32_t* yhi = reinterpret_cast<uint32_t*>(smem_b + pl.off_yhi);
+  float* invy = reinterpret_cast<float*>(smem_b + pl.off_invy);
+  const uint32_t full = smem_addr(smem_b + pl.off_bar), empty = full + 8u * kT2MaxSlots;
+  const uint8_t* ring_p = smem_b + pl.off_ring;
+  const uint32_t ring = smem_addr(ring_p);
+  const uint32_t ncols = C - xg0 < kT2Group ? C - xg0 : kT2Group;
+  const uint32_t nrows = C - k0 < p.mm2_rows ? C - k0 : p.mm2_rows;
+
+  // tables: a thread per row of the CTA, and per column of the group
+  if (tid < nrows) {
+    const uint32_t Y = top + k0 + tid;
+    uint32_t j0, j1;
+    tap_range32(ay, Y, &j0, &j1);
+    uint32_t sum = 0;
+    for (uint32_t j = j0; j < j1; ++j) sum += tap_weight32(ay, Y, j);
+    ylo[tid] = j0;
+    yhi[tid] = j1;
+    invy[tid] = 1.0f / static_cast<float>(sum);
+  }
+  if (tid < kT2Group) {
+    uint32_t j0 = 0, j1 = 0;
+    float inv = 0.f;
+    if (tid < ncols) {
+      const uint32_t X = left + xg0 + tid;
+      tap_range32(ax, X, &j0, &j1);
+      uint32_t sum = 0;
+      for (uint32_t j = j0; j < j1; ++j) {
+        const uint32_t wgt = tap_weight32(ax, X, j);
+        wxi[tid * kMaxTapsX + (j - j0)] = static_cast<uint16_t>(wgt);
+        sum += wgt;
+      }
+      inv = 1.0f / static_cast<float>(sum);
+    }
+    xlo[tid] = j0;
+    xcnt[tid] = j1 - j0;
+    invx[tid] = inv;
+  }
+  if (tid == 0) {
+    for (uint32_t s = 0; s < pl.slots; ++s) {
+      mbar_init(full + 8u * s, 16);
+      mbar_init(empty + 8u * s, kT2Warps);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  // the bytes of an input row under the group, and the input rows under the CTA's output rows
+  const uint32_t rowbyte0 = 3u * xlo[0];
+  const uint32_t rowbytes = 3u * (xlo[ncols - 1] + xcnt[ncols - 1]) - rowbyte0;
+  // Tiles of sixteen input rows start at multiples of 16 in the image, whatever rows the CTA
+  // has: the sums of an output row are then grouped alike however the image is cut into CTAs,
+  // and the result does not depend on the cut.
+  const uint32_t ya_need = ylo[0], ya = ya_need & ~15u, yb = yhi[nrows - 1];
+  const uint32_t ntiles16 = (yb - ya + 15u) / 16u;
+  const uint32_t mtiles = (ncols + kT2Px - 1u) / kT2Px;
+  const uint8_t* image = p.pixels + e.offset;
+  const uint8_t* stop = p.pixels + usable;
+  const uint64_t pitch = 3ull * e.w;
+  // rows start on the same byte phase (the pitch is a multiple of 4)
+  const uint32_t skew4 = static_cast<uint32_t>(reinterpret_cast<uintptr_t>(image + rowbyte0)) & 3u;
+  // cannot happen within the plan's bounds: a row longer than its place in the ring, or an
+  // M-tile whose pixels' taps do not fit its window (every thread checks every tile, so the
+  // CTA leaves as one)
+  bool fits = 16u + rowbytes + 32u * KS <= pl.seg;
+  for (uint32_t t = 0; t < mtiles; ++t) {
+    const uint32_t c0 = kT2Px * t, c1 = c0 + kT2Px - 1u < ncols ? c0 + kT2Px - 1u : ncols - 1u;
+    const uint32_t nb = 3u * xlo[c0] - rowbyte0;
+    const uint32_t start_gap = (nb + skew4) & 3u;  // the window starts this far before the first tap
+    if (3u * (xlo[c1] + xcnt[c1]) - rowbyte0 - nb + start_gap > 32u * KS) fits = false;
+  }
+  if (!fits) {
+    if (tid == 0) report(p.status, PREBA_ERR_TOO_LARGE);
+    return;
+  }
+
+  // The last warp asks for the 16 rows of tile m, a lane per row: a row the CTA needs is
+  // copied and its bytes announced to the slot's barrier, the other lanes of the sixteen just
+  // arrive.
+  auto issue = [&](uint32_t m) {
+    if (lane >= 16u) return;
+    const uint32_t slot = m % pl.slots, bar = full + 8u * slot;
+    const uint32_t r = ya + 16u * m + lane;
+    if (r >= ya_need && r < yb) {  // (rows before the first needed one get no weight)
+      const uint8_t* src = image + r * pitch + rowbyte0;
+      const uint32_t skew = static_cast<uint32_t>(reinterpret_cast<uintptr_t>(src)) & 15u;
+      uint32_t bytes = (skew + rowbytes + 15u) & ~15u;
+      if (bytes > static_cast<uint64_t>(stop - (src - skew)))  // only padding is lost
+        bytes = static_cast<uint32_t>(stop - (src - skew));
+      fence_async_shared();
+      // checked build: the row lies in its place in the ring and in the pixel buffer
+      if (PREBA_IN_RANGE(p.status, bytes <= pl.seg && src - skew >= p.pixels &&
+                                       src - skew + bytes <= p.pixels + p.pixels_bytes)) {
+        mbar_arrive_expect_tx(bar, bytes);
+        bulk_copy_g2s(ring + (slot * 16u + lane) * pl.seg, src - skew, bytes, bar);
+      } else {
+        mbar_arrive(bar);
+      }
+    } else {
+      mbar_arrive(bar);
+    }
+  };
+  if (warp == kT2Warps - 1u)
+    for (uint32_t m = 0; m < pl.slots && m < ntiles16; ++m) issue(m);
+
+  // The weights of this warp's M-tiles as A operands.  Row mr of an M-tile is channel mr % 3 of
+  // the tile's pixel mr / 3 (row 15 is unused); register r holds row g (+ 8 if r is odd), bytes
+  // k = 16 (r / 2) + 4 q + i of step s: the row position kst + 32 s + k.
+  const uint32_t g = lane >> 2, q = lane & 3u;
+  uint32_t ahi[2][KS][4], alo[2][KS][4];
+  int32_t kst[2];
+  float scale[2][2];   // per M-tile and row (g, g + 8): 1 / sum of the column's weights, times 1 / (255 std)
+  bool live[2];
+#pragma unroll
+  for (uint32_t t = 0; t < 2; ++t) {
+    const uint32_t mt = warp + kT2Warps * t, col0 = kT2Px * mt;
+    live[t] = mt < mtiles;
+    int32_t start = 0;
+    if (live[t]) {
+      const int32_t nb = static_cast<int32_t>(3u * xlo[col0] - rowbyte0);
+      start = nb - static_cast<int32_t>((static_cast<uint32_t>(nb) + skew4) & 3u);
+    }
+    kst[t] = start;
+#pragma unroll
+    for (uint32_t half = 0; half < 2; ++half) {
+      const uint32_t mr = g + 8u * half, col = col0 + mr / 3u;
+      const uint32_t ch = mr % 3u;
+      const float mul = ch == 0u ? p.mul[0] : (ch == 1u ? p.mul[1] : p.mul[2]);
+      // (the second product leaves 2^-22 times the sum)
+      scale[t][half] = (live[t] && mr < 15u && col < ncols) ? invx[col] * mul * 4194304.f : 0.f;
+    }
+#pragma unroll
+    for (uint32_t s = 0; s < KS; ++s)
+#pragma unroll
+      for (uint32_t r = 0; r < 4; ++r) {
+        const uint32_t mr = g + 8u * (r & 1u), ch = mr % 3u, col = col0 + mr / 3u;
+        const bool on = live[t] && mr < 15u && col < ncols;
+        const uint32_t lo_px = on ? xlo[col] : 0u, n_px = on ? xcnt[col] : 0u;
+        uint32_t hi = 0, lo = 0;
+#pragma unroll
+        for (uint32_t i = 0; i < 4; ++i) {
+          const int32_t b = static_cast<int32_t>(rowbyte0) + start +
+                            static_cast<int32_t>(32u * s + 16u * (r >> 1) + 4u * q + i);
+          uint32_t wgt = 0;
+          if (b >= 0) {
+            const uint32_t px = static_cast<uint32_t>(b) / 3u;
+            if (static_cast<uint32_t>(b) - 3u * px == ch && px >= lo_px && px - lo_px < n_px)
+              wgt = wxi[col * kMaxTapsX + (px - lo_px)];
+          }
+          hi |= (wgt >> 8) << (8u * i);
+          lo |= (wgt & 0xffu) << (8u * i);
+        }
+        ahi[t][s][r] = hi;
+        alo[t][s][r] = lo;
+      }
+  }
+  // where the lane's two rows of an M-tile go: plane of the channel, column of the pixel
+  const uint32_t px_a = g / 3u, px_b = (g + 8u) / 3u;
+  const uint32_t ch_a = g % 3u, ch_b = (g + 8u) % 3u;
+  const float add_a = ch_a == 0u ? p.add[0] : (ch_a == 1u ? p.add[1] : p.add[2]);
+  const float add_b = ch_b == 0u ? p.add[0] : (ch_b == 1u ? p.add[1] : p.add[2]);
+  OutT* out = static_cast<OutT*>(p.out) + static_cast<uint64_t>(img) * 3u * C * C;
+  OutT* out_a = out + static_cast<uint64_t>(ch_a) * C * C + xg0 + px_a;
+  OutT* out_b = out + static_cast<uint64_t>(ch_b) * C * C + xg0 + px_b;
+
+  // The vertical sums: output row yl of the CTA uses column yl % 8 of the second product; a lane
+  // holds columns 2q and 2q + 1 of rows g and g + 8.
+  float acc[2][4];
+#pragma unroll
+  for (uint32_t t = 0; t < 2; ++t)
+#pragma unroll
+    for (uint32_t i = 0; i < 4; ++i) acc[t][i] = 0.f;
+  uint32_t ynext = 0;  // the first output row of the CTA whose last tap has not passed
+  const int32_t two_m = static_cast<int32_t>(2u * ay.M), two_r = static_cast<int32_t>(2u * ay.R);
+  // 16-byte skew of input row r: (base + r * pitch) & 15, in 32 bits
+  const uint32_t skew_base = static_cast<uint32_t>(reinterpret_cast<uintptr_t>(image + rowbyte0)) & 15u;
+  const uint32_t skew_step = static_cast<uint32_t>(pitch & 15u);
+  const uint32_t ring_row0 = g * pl.seg + 4u * q, ring_row1 = (g + 8u) * pl.seg + 4u * q;
+
+  bool failed = false;
+  for (uint32_t m = 0; m < ntiles16 && !failed; ++m) {
+    const uint32_t slot = m % pl.slots, r0 = ya + 16u * m;
+    if (!mbar_wait(full + 8u * slot, (m / pl.slots) & 1u)) failed = true;
+    if (__any_sync(0xffffffffu, failed)) {
+      failed = true;
+      break;
+    }
+    // The weights of the output rows under this tile, as the B operand of the second product
+    // (16 input rows x 8 output rows, binary16): column g is the row with yl % 8 == g among
+    // ynext .. ynext + 7, the lane's k are input rows r0 + {2q, 2q + 1, 8 + 2q, 9 + 2q}.  An
+    // integer weight w < 2^16 goes in as two exact pieces, (w & 255) / 256 and w >> 8.
+    uint32_t wlo[2] = {0u, 0u}, whi[2] = {0u, 0u};
+    {
+      const uint32_t yl = ynext + ((g - ynext) & 7u);
+      uint32_t w4[4] = {0u, 0u, 0u, 0u};
+      if (yl < nrows) {
+        const uint32_t Y = top + k0 + yl, rbase = r0 + 2u * q;
+        const int32_t d = static_cast<int32_t>((2u * rbase + 1u) * ay.R) -
+                          static_cast<int32_t>((2u * Y + 1u) * ay.n_in);
+#pragma unroll
+        for (uint32_t i = 0; i < 4; ++i) {
+          const uint32_t dr = (i & 1u) + 8u * (i >> 1);
+          const int32_t di = d + static_cast<int32_t>(dr) * two_r;
+          int32_t wgt = two_m - (di < 0 ? -di : di);
+          if (wgt < 0 || rbase + dr >= ay.n_in) wgt = 0;
+          w4[i] = static_cast<uint32_t>(wgt);
+        }
+      }
+#pragma unroll
+      for (uint32_t h = 0; h < 2; ++h) {
+        const uint32_t pair = __byte_perm(w4[2 * h], w4[2 * h + 1], 0x5140);  // lo, lo, hi, hi bytes
+        wlo[h] = expand_bytes<0>(pair, 0x1c00u, 0xc400u);   // (1024 + b) / 256 - 4
+        whi[h] = expand_bytes<1>(pair, 0x3c00u, 0xe400u);   // (1024 + b) - 1024
+      }
+    }
+    // rows that are complete after this tile, for the lane's two columns
+    uint32_t done_row[2];
+    float done_inv[2];
+#pragma unroll
+    for (uint32_t c = 0; c < 2; ++c) {
+      const uint32_t yl = ynext + ((2u * q + c - ynext) & 7u);
+      const bool done = yl < nrows && yhi[yl] <= r0 + 16u;
+      done_row[c] = done ? yl : 0xffffffffu;
+      done_inv[c] = done ? invy[yl] : 0.f;
+    }
+    // rows g and g + 8 of the tile: where their first needed byte lies in the slot
+    const uint32_t sk0 = (skew_base + (r0 + g) * skew_step) & 15u;
+    const uint32_t sk1 = (skew_base + (r0 + g + 8u) * skew_step) & 15u;
+    const uint8_t* row0 = ring_p + slot * 16u * pl.seg + ring_row0 + sk0;
+    const uint8_t* row1 = ring_p + slot * 16u * pl.seg + ring_row1 + sk1;
+#pragma unroll
+    for (uint32_t t = 0; t < 2; ++t) {
+      if (!live[t]) continue;
+      // checked build: the window of both rows lies in the row's place in the ring
+      if (!PREBA_IN_RANGE(p.status,
+                          static_cast<int32_t>(sk0 + 4u * q) + kst[t] >= 0 &&
+                              static_cast<int32_t>(sk1 + 4u * q) + kst[t] >= 0 &&
+                              static_cast<int32_t>((sk0 > sk1 ? sk0 : sk1) + 4u * q) + kst[t] +
+                                      static_cast<int32_t>(32u * KS - 12u) <=
+                                  static_cast<int32_t>(pl.seg) &&
+                              slot < pl.slots))
+        continue;
+      // first product, high and low bytes of the weights apart: e = rows 0-7 of the tile,
+      // f = rows 8-15
+      int32_t eh[4] = {0, 0, 0, 0}, el[4] = {0, 0, 0, 0}, fh[4] = {0, 0, 0, 0}, fl[4] = {0, 0, 0, 0};
+      const uint32_t* at0 = reinterpret_cast<const uint32_t*>(row0 + kst[t]);
+      const uint32_t* at1 = reinterpret_cast<const uint32_t*>(row1 + kst[t]);
+#pragma unroll
+      for (uint32_t s = 0; s < KS; ++s) {
+        const uint32_t b00 = at0[8 * s], b01 = at0[8 * s + 4], b10 = at1[8 * s], b11 = at1[8 * s + 4];
+        mma_u8(eh, ahi[t][s], b00, b01);
+        mma_u8(el, alo[t][s], b00, b01);
+        mma_u8(fh, ahi[t][s], b10, b11);
+        mma_u8(fl, alo[t][s], b10, b11);
+      }
+      // H = 256 high + low, below 2^24; register i: row g + 8 (i / 2), input row 2q + i % 2
+      uint32_t he[4], hf[4];
+#pragma unroll
+      for (uint32_t i = 0; i < 4; ++i) {
+        he[i] = (static_cast<uint32_t>(eh[i]) << 8) + static_cast<uint32_t>(el[i]);
+        hf[i] = (static_cast<uint32_t>(fh[i]) << 8) + static_cast<uint32_t>(fl[i]);
+      }
+      // The three bytes of H as binary16 A operands of the second product (16 (x, ch) rows by
+      // 16 input rows): byte 0 scaled by 2^-14, byte 1 by 2^-6, byte 2 by 4, all exact, so
+      // that the sum below is 2^-22 times sum_r w[r] H[r].
+#pragma unroll
+      for (uint32_t pln = 0; pln < 3; ++pln) {
+        uint32_t a[4];
+#pragma unroll
+        for (uint32_t h = 0; h < 2; ++h) {
+          // bytes pln of the four values of row g + 8 h: input rows 2q, 2q + 1 (e), 8 + 2q, 9 + 2q (f)
+          const uint32_t sel = pln == 0 ? 0x0040u : (pln == 1 ? 0x0051u : 0x0062u);
+          const uint32_t pe = __byte_perm(he[2 * h], he[2 * h + 1], sel);
+          const uint32_t pf = __byte_perm(hf[2 * h], hf[2 * h + 1], sel);
+          const uint32_t mul = pln == 0 ? 0x0400u : (pln == 1 ? 0x2400u : 0x4400u);
+          const uint32_t off = pln == 0 ? 0xac00u : (pln == 1 ? 0xcc00u : 0xec00u);
+          a[h] = expand_bytes<0>(pe, mul, off);      // k = 2q, 2q + 1
+          a[2 + h] = expand_bytes<0>(pf, mul, off);  // k = 8 + 2q, 9 + 2q
+        }
+        mma_f16(acc[t], a, wlo[0], wlo[1]);
+        mma_f16(acc[t], a, whi[0], whi[1]);
+      }
+      // rows whose last tap has passed: normalise, store
+      const uint32_t col0 = kT2Px * (warp + kT2Warps * t);
+#pragma unroll
+      for (uint32_t c = 0; c < 2; ++c) {
+        if (done_row[c] == 0xffffffffu) continue;
+        const uint32_t rowoff = (k0 + done_row[c]) * C + col0;
+        // checked build: the row and the columns lie in the crop
+        if (PREBA_IN_RANGE(p.status, k0 + done_row[c] < C &&
+                                         (scale[t][0] == 0.f || xg0 + col0 + px_a < C) &&
+                                         (scale[t][1] == 0.f || xg0 + col0 + px_b < C))) {
+          if (scale[t][0] != 0.f)
+            out_a[rowoff] = to_out<OutT>(fmaf(acc[t][c] * done_inv[c], scale[t][0], add_a));
+          if (scale[t][1] != 0.f)
+            out_b[rowoff] = to_out<OutT>(fmaf(acc[t][2 + c] * done_inv[c], scale[t][1], add_b));
+        }
+        acc[t][c] = acc[t][2 + c] = 0.f;
+      }
+    }
+    // the staged rows of this tile have been read: the warp gives the slot back
+    __syncwarp();
+    if (lane == 0) mbar_arrive(empty + 8u * slot);
+    // the rows that are complete now
+    {
+      const uint32_t yl = ynext + (lane & 7u);
+      const bool done = yl < nrows && yhi[yl] <= r0 + 16u;
+      const uint32_t mask = __ballot_sync(0xffffffffu, done) & 0xffu;
+      ynext += static_cast<uint32_t>(__ffs(static_cast<int>(~mask))) - 1u;
+    }
+    // when every warp has given the slot back it takes the rows of tile m + slots
+    if (warp == kT2Warps - 1u && m + pl.slots < ntiles16) {
+      bool ok = true;
+      if (lane < 16u) ok = mbar_wait(empty + 8u * slot, (m / pl.slots) & 1u);
+      if (__all_sync(0xffffffffu, ok)) issue(m + pl.slots);
+      else failed = true;
+    }
+  }
+  if (failed) {
+    if (lane == 0) report(p.status, PREBA_ERR_TIMEOUT);
+    // copies already asked for may still be landing in the ring: the issuing warp waits for
+    // them (bounded) before the CTA's shared memory is given up
+    if (warp == kT2Warps - 1u && lane == 0)
+      for (uint32_t s = 0; s < pl.slots; ++s) {
+        (void)mbar_wait(full + 8u * s, 0u);
+        (void)mbar_wait(full + 8u * s, 1u);
+      }
+  }
+}
+
 }  // namespace aa
 }  // namespace preba
 
@@ -1047,6 +1514,13 @@ Kernel kernel_for(int out_dtype) {
   return out_dtype == PREBA_F32   ? preba::aa::preba_antialias_kernel<float>
          : out_dtype == PREBA_F16 ? preba::aa::preba_antialias_kernel<__half>
                                   : preba::aa::preba_antialias_kernel<__nv_bfloat16>;
+}
+
+template <uint32_t KS>
+Kernel mm2_kernel_for(int out_dtype) {
+  return out_dtype == PREBA_F32   ? preba::aa::preba_antialias_mm2_kernel<float, KS>
+         : out_dtype == PREBA_F16 ? preba::aa::preba_antialias_mm2_kernel<__half, KS>
+                                  : preba::aa::preba_antialias_mm2_kernel<__nv_bfloat16, KS>;
 }
 
 Kernel mma_kernel_for(int out_dtype) {
@@ -1079,6 +1553,12 @@ int shared_memory_limit(cudaError_t* err) {
                                   optin);
     if (*err == cudaSuccess)
       *err = cudaFuncSetAttribute(mma_kernel_for(dt), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  optin < kMmaSmemBytes ? optin : kMmaSmemBytes);
+    if (*err == cudaSuccess)
+      *err = cudaFuncSetAttribute(mm2_kernel_for<3>(dt), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  optin < kMmaSmemBytes ? optin : kMmaSmemBytes);
+    if (*err == cudaSuccess)
+      *err = cudaFuncSetAttribute(mm2_kernel_for<4>(dt), cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   optin < kMmaSmemBytes ? optin : kMmaSmemBytes);
   }
   if (*err != cudaSuccess) return 0;
@@ -1128,10 +1608,10 @@ extern "C" int preba_preprocess_antialias(const preba_batch_t* batch, const preb
   // other one the rest; each skips the other's images.  With the host's copy of the table a
   // kernel without images is not launched at all.
   const uint32_t mma_smem = static_cast<uint32_t>(limit < kMmaSmemBytes ? limit : kMmaSmemBytes);
-  bool any_mma = true, any_rest = true;
+  bool any_mma = true, any_rest = true, any_mm2[2] = {true, true};  // windows of 3 and 4 steps
   if (batch->table_host) {
     uint64_t most = 0;
-    any_mma = any_rest = false;
+    any_mma = any_rest = any_mm2[0] = any_mm2[1] = false;
     for (uint32_t i = 0; i < batch->n; ++i) {
       const preba_img_t& e = batch->table_host[i];
       // as in the kernel: rows are fetched in 16-byte units, so the buffer counts up to its
@@ -1146,6 +1626,11 @@ extern "C" int preba_preprocess_antialias(const preba_batch_t* batch, const preb
           (opt->crop_origin_host[2 * i] + static_cast<uint64_t>(C) > rh ||
            opt->crop_origin_host[2 * i + 1] + static_cast<uint64_t>(C) > rw))
         return PREBA_ERR_BAD_CROP;
+      preba::aa::Mm2Plan two;
+      if (mm2_plan(make_axis(e.w, rw), make_axis(e.h, rh), e.w, C, mma_smem, &two)) {
+        any_mm2[two.ks - 3u] = true;
+        continue;
+      }
       if (mma_plan(make_axis(e.w, rw), make_axis(e.h, rh), e.w, C, mma_smem, nullptr)) {
         any_mma = true;
         continue;
@@ -1195,6 +1680,25 @@ extern "C" int preba_preprocess_antialias(const preba_batch_t* batch, const preb
   p.rows = rows;
   p.smem_floats = floats;
   p.mma_smem = any_mma ? mma_smem : 0u;
+  p.mm2_smem = (any_mm2[0] || any_mm2[1]) ? mma_smem : 0u;
+  // Output rows per CTA of the chained kernel: the chunking of an image's rows whose CTAs fill
+  // the rounds of what the GPU holds at once (two CTAs per SM) best, fewest chunks first; no
+  // CTA below 32 rows.
+  {
+    const uint64_t groups = (C + preba::aa::kT2Group - 1) / preba::aa::kT2Group;
+    const uint64_t slots = 2ull * sms, least = (C + kMmaRows - 1) / kMmaRows;
+    const uint64_t most_chunks = C >= 64u ? C / 32u : 1u;
+    uint64_t best = least > most_chunks ? least : 0, best_fill = 0;
+    for (uint64_t c = least; c <= most_chunks && c <= least + 15u; ++c) {
+      const uint64_t ctas = static_cast<uint64_t>(batch->n) * groups * c;
+      const uint64_t rounds = (ctas + slots - 1) / slots;
+      const uint64_t fill = ctas * 1000u / (rounds * slots);
+      if (fill > best_fill + 20u) best = c, best_fill = fill;  // a later choice must be clearly better
+    }
+    if (best == 0) best = least;
+    p.mm2_rows = static_cast<uint32_t>((C + best - 1) / best);
+    if (p.mm2_rows > kMmaRows) p.mm2_rows = kMmaRows;
+  }
   // Output rows per CTA of the tensor-core kernel: a CTA builds its weight operands once and
   // then sweeps, so it takes as many rows as it can (all of them up to kMmaRows) unless the
   // batch then has fewer CTAs than the GPU holds at once.
@@ -1215,7 +1719,16 @@ extern "C" int preba_preprocess_antialias(const preba_batch_t* batch, const preb
                                   static_cast<double>(opt->std[c]));
   }
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (any_mma) {
+  for (uint32_t v = 0; v < 2 && err == cudaSuccess; ++v) {
+    if (!any_mm2[v]) continue;
+    const uint64_t ctas = static_cast<uint64_t>(batch->n) * ((C + p.mm2_rows - 1) / p.mm2_rows) *
+                          ((C + preba::aa::kT2Group - 1) / preba::aa::kT2Group);
+    if (ctas > 0x7fffffffull) return PREBA_ERR_INVALID_ARG;
+    (v == 0 ? mm2_kernel_for<3>(opt->out_dtype) : mm2_kernel_for<4>(opt->out_dtype))
+        <<<static_cast<uint32_t>(ctas), kMmaThreads, mma_smem, s>>>(p);
+    err = cudaGetLastError();
+  }
+  if (any_mma && err == cudaSuccess) {
     const uint64_t ctas = static_cast<uint64_t>(batch->n) * ((C + p.mma_rows - 1) / p.mma_rows) *
                           ((C + kGroup - 1) / kGroup);
     if (ctas > 0x7fffffffull) return PREBA_ERR_INVALID_ARG;

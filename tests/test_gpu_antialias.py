@@ -99,6 +99,37 @@ def test_images_of_the_tensor_core_kernel(c, s):
     assert np.all(err <= 1e-5), err
 
 
+# images reduced between 2.5 and about 6.5 times vertically, widths that are multiples of 4: the
+# ones that take both passes on the tensor cores (windows of three and of four steps, groups
+# with a ragged last tile, portrait and landscape), next to some that just miss it
+CHAINED_SHAPES = [(1080, 1920), (700, 1000), (1600, 1600), (650, 2000), (1920, 1080), (1000, 1404),
+                  (1284, 1280), (644, 644), (1700, 1704), (640, 1640)]
+
+
+@pytest.mark.parametrize("c,s", [(224, 256), (256, 256), (75, 240), (76, 250), (33, 300), (1, 200)])
+def test_images_of_the_chained_tensor_core_kernel(c, s):
+    images = [uniform(170 + i, h, w) for i, (h, w) in enumerate(CHAINED_SHAPES)]
+    got = run(images, c, s)
+    err = np.max(np.abs(got - want(images, c, s)), axis=(1, 2, 3))
+    assert np.all(err <= 1e-5), err
+    origins = origins_for(images, c, s, 13)
+    got = run(images, c, s, origins=origins, with_host_table=False)
+    err = np.max(np.abs(got - want(images, c, s, origins)), axis=(1, 2, 3))
+    assert np.all(err <= 1e-5), err
+    # one image alone: its rows are cut into CTAs differently, but the tiles of input rows sit
+    # at the same places of the image, so the sums group their terms alike
+    alone = run(images[:1], c, s)
+    assert np.array_equal(alone[0], run(images, c, s)[0])
+
+
+@pytest.mark.parametrize("out_dtype", [pb.F16, pb.BF16])
+def test_half_precision_outputs_of_the_chained_kernel(out_dtype):
+    images = [wl.smooth_image(np.random.default_rng(470 + i), h, w)
+              for i, (h, w) in enumerate(CHAINED_SHAPES[:5])]
+    got = run(images, 224, 256, out_dtype=out_dtype)
+    assert_parity(got, want(images, 224, 256), out_dtype)
+
+
 @pytest.mark.parametrize("c,s", [(224, 256), (96, 96), (17, 40), (1, 1), (299, 342)])
 def test_other_output_sizes(c, s):
     images = [uniform(200 + i, h, w) for i, (h, w) in enumerate(SHAPES[:7])]
