@@ -236,25 +236,31 @@ __host__ __device__ inline bool mma_plan(const Axis& ax, const Axis& ay, uint32_
 // channels are the A operand (16 rows, one unused; built once per warp, in registers), the
 // bytes of eight input rows the B operand, again exactly as the rows lie in the ring, so a lane
 // ends up with H[(x, ch)][input row] for (x, ch) = g, g + 8 and rows 2q, 2q + 1 of each
-// eight: the layout an A operand has, with the input rows as its k index.  H is below 2^24;
-// its three bytes go through byte permutes into three A operands, the integer weights of the
-// (at most eight) output rows that lie under the sixteen input rows, split into two bytes, are
-// the B operand, and four more matrix instructions add the six byte products into four
-// accumulators, one per power of 256.  Everything up to there is exact integer arithmetic;
-// an output row whose last tap has passed is put together in fp32, normalised and stored.
-// A warp owns its (x, ch) tiles from the ring to the store: there is no CTA-wide barrier after
-// the start, only the ring's full and empty barriers.
+// eight: the layout an A operand has, with the input rows as its k index.  H is an exact
+// integer below 2^24; its three bytes become three binary16 A operands (exact, scaled by
+// powers of two), the integer weights of the (at most eight) output rows that lie under the
+// sixteen input rows, split into two bytes, the binary16 B operands, and six more matrix
+// instructions add the byte products into one fp32 accumulator.  An output row whose last
+// tap has passed is normalised and stored.
+// Fifteen warps each own one tile of five pixels from the ring to the store; the sixteenth
+// feeds them: it issues the copies of a tile's rows and works out what is the same for every
+// warp (the weights of the second product, which rows the tile completes) into the slot's
+// record.  There is no CTA-wide barrier after the start, only the ring's full and empty
+// barriers.
 constexpr uint32_t kT2Px = 5;                        // resized pixels of an M-tile
-constexpr uint32_t kT2Tiles = 15;                    // M-tiles of a CTA (warp w owns w and w + 8)
+constexpr uint32_t kT2Tiles = 15;                    // M-tiles of a CTA, one per consumer warp
 constexpr uint32_t kT2Group = kT2Px * kT2Tiles;      // output columns per CTA
-constexpr uint32_t kT2MaxSlots = 6;                  // 16-row slots of the ring, at most
-constexpr uint32_t kT2Warps = kMmaThreads / 32;
+constexpr uint32_t kT2MaxSlots = 8;                  // 16-row slots of the ring, at most
+constexpr uint32_t kT2Threads = 32 * (kT2Tiles + 1); // the last warp feeds the others
+constexpr uint32_t kT2MetaBytes = 1024;              // per slot: what the feeding warp works out
+                                                     // for a tile (32 bytes per lane)
 
 struct Mm2Plan {
   uint32_t seg;    // bytes of one staged input row in the ring
   uint32_t slots;  // 16-row slots of the ring
   uint32_t ks;     // 32-byte steps of an M-tile's window (3 or 4)
-  uint32_t off_wx, off_xlo, off_xcnt, off_invx, off_ylo, off_yhi, off_invy, off_bar, off_ring;
+  uint32_t off_wx, off_xlo, off_xcnt, off_invx, off_ylo, off_yhi, off_invy, off_bar, off_meta,
+      off_ring;
 };
 
 // Whether the kernel with both passes on the tensor cores takes an image, and its
@@ -292,6 +298,7 @@ __host__ __device__ inline bool mm2_plan(const Axis& ax, const Axis& ay, uint32_
   at = (at + 7u) & ~7u;
   p.off_bar = at, at += 2u * kT2MaxSlots * 8u;
   at = (at + 15u) & ~15u;
+  p.off_meta = at, at += kT2MaxSlots * kT2MetaBytes;
   p.off_ring = at;
   if (smem_bytes <= at) return false;
   const uint64_t room = (smem_bytes - at) / (16ull * p.seg);
@@ -429,6 +436,24 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
   for (uint32_t it = 0; it < kSpinLimit; ++it)
     if (mbar_try_wait(bar, parity)) return true;
+  return false;
+}
+
+// The same, every try with a time hint: a thread whose phase is not complete yet is put aside
+// by the hardware for up to about that long (or until the phase completes) instead of coming
+// back at once, so waiting warps leave the issue slots to the others.
+__device__ __forceinline__ bool mbar_wait_parked(uint32_t bar, uint32_t parity) {
+  for (uint32_t it = 0; it < kSpinLimit; ++it) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(4000u)
+        : "memory");
+    if (ok) return true;
+  }
   return false;
 }
 
@@ -1135,7 +1160,7 @@ __device__ __forceinline__ uint32_t expand_bytes(uint32_t x, uint32_t mul, uint3
 }
 
 template <typename OutT, uint32_t KS>
-__global__ void __launch_bounds__(kMmaThreads, 2) preba_antialias_mm2_kernel(const Params p) {
+__global__ void __launch_bounds__(kT2Threads, 2) preba_antialias_mm2_kernel(const Params p) {
   extern __shared__ __align__(16) uint8_t smem_b[];
   const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5, C = p.C;
   const uint32_t chunks = (C + p.mm2_rows - 1) / p.mm2_rows, groups = (C + kT2Group - 1) / kT2Group;
@@ -1174,6 +1199,7 @@ __global__ void __launch_bounds__(kMmaThreads, 2) preba_antialias_mm2_kernel(con
   uint32_t* ylo = reinterpret_cast<uint32_t*>(smem_b + pl.off_ylo);
   uint32_t* yhi = reinterpret_cast<uint32_t*>(smem_b + pl.off_yhi);
   float* invy = reinterpret_cast<float*>(smem_b + pl.off_invy);
+  uint4* meta = reinterpret_cast<uint4*>(smem_b + pl.off_meta);
   const uint32_t full = smem_addr(smem_b + pl.off_bar), empty = full + 8u * kT2MaxSlots;
   const uint8_t* ring_p = smem_b + pl.off_ring;
   const uint32_t ring = smem_addr(ring_p);
@@ -1191,28 +1217,29 @@ __global__ void __launch_bounds__(kMmaThreads, 2) preba_antialias_mm2_kernel(con
     yhi[tid] = j1;
     invy[tid] = 1.0f / static_cast<float>(sum);
   }
-  if (tid < kT2Group) {
+  if (tid >= 256u && tid - 256u < kT2Group) {
+    const uint32_t col = tid - 256u;
     uint32_t j0 = 0, j1 = 0;
     float inv = 0.f;
-    if (tid < ncols) {
-      const uint32_t X = left + xg0 + tid;
+    if (col < ncols) {
+      const uint32_t X = left + xg0 + col;
       tap_range32(ax, X, &j0, &j1);
       uint32_t sum = 0;
       for (uint32_t j = j0; j < j1; ++j) {
         const uint32_t wgt = tap_weight32(ax, X, j);
-        wxi[tid * kMaxTapsX + (j - j0)] = static_cast<uint16_t>(wgt);
+        wxi[col * kMaxTapsX + (j - j0)] = static_cast<uint16_t>(wgt);
         sum += wgt;
       }
       inv = 1.0f / static_cast<float>(sum);
     }
-    xlo[tid] = j0;
-    xcnt[tid] = j1 - j0;
-    invx[tid] = inv;
+    xlo[col] = j0;
+    xcnt[col] = j1 - j0;
+    invx[col] = inv;
   }
   if (tid == 0) {
     for (uint32_t s = 0; s < pl.slots; ++s) {
       mbar_init(full + 8u * s, 16);
-      mbar_init(empty + 8u * s, kT2Warps);
+      mbar_init(empty + 8u * s, kT2Tiles);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -1232,273 +1259,277 @@ __global__ void __launch_bounds__(kMmaThreads, 2) preba_antialias_mm2_kernel(con
   const uint64_t pitch = 3ull * e.w;
   // rows start on the same byte phase (the pitch is a multiple of 4)
   const uint32_t skew4 = static_cast<uint32_t>(reinterpret_cast<uintptr_t>(image + rowbyte0)) & 3u;
-  // cannot happen within the plan's bounds: a row longer than its place in the ring, or an
-  // M-tile whose pixels' taps do not fit its window (every thread checks every tile, so the
-  // CTA leaves as one)
+  const uint32_t g = lane >> 2, q = lane & 3u;
+
+  // The window of this warp's M-tile.  Cannot happen within the plan's bounds: a row longer
+  // than its place in the ring, or pixels whose taps do not fit the window; the CTA leaves as
+  // one.
+  const bool live = warp < mtiles;
+  const uint32_t col0 = kT2Px * warp;
+  int32_t kst = 0;
   bool fits = 16u + rowbytes + 32u * KS <= pl.seg;
-  for (uint32_t t = 0; t < mtiles; ++t) {
-    const uint32_t c0 = kT2Px * t, c1 = c0 + kT2Px - 1u < ncols ? c0 + kT2Px - 1u : ncols - 1u;
-    const uint32_t nb = 3u * xlo[c0] - rowbyte0;
-    const uint32_t start_gap = (nb + skew4) & 3u;  // the window starts this far before the first tap
-    if (3u * (xlo[c1] + xcnt[c1]) - rowbyte0 - nb + start_gap > 32u * KS) fits = false;
+  if (live) {
+    const uint32_t c1 = col0 + kT2Px - 1u < ncols ? col0 + kT2Px - 1u : ncols - 1u;
+    const uint32_t nb = 3u * xlo[col0] - rowbyte0, gap = (nb + skew4) & 3u;
+    kst = static_cast<int32_t>(nb) - static_cast<int32_t>(gap);
+    if (3u * (xlo[c1] + xcnt[c1]) - rowbyte0 - nb + gap > 32u * KS) fits = false;
   }
-  if (!fits) {
+  if (!__syncthreads_and(fits)) {
     if (tid == 0) report(p.status, PREBA_ERR_TOO_LARGE);
     return;
   }
 
-  // The last warp asks for the 16 rows of tile m, a lane per row: a row the CTA needs is
-  // copied and its bytes announced to the slot's barrier, the other lanes of the sixteen just
-  // arrive.
-  auto issue = [&](uint32_t m) {
-    if (lane >= 16u) return;
-    const uint32_t slot = m % pl.slots, bar = full + 8u * slot;
-    const uint32_t r = ya + 16u * m + lane;
-    if (r >= ya_need && r < yb) {  // (rows before the first needed one get no weight)
-      const uint8_t* src = image + r * pitch + rowbyte0;
-      const uint32_t skew = static_cast<uint32_t>(reinterpret_cast<uintptr_t>(src)) & 15u;
-      uint32_t bytes = (skew + rowbytes + 15u) & ~15u;
-      if (bytes > static_cast<uint64_t>(stop - (src - skew)))  // only padding is lost
-        bytes = static_cast<uint32_t>(stop - (src - skew));
-      fence_async_shared();
-      // checked build: the row lies in its place in the ring and in the pixel buffer
-      if (PREBA_IN_RANGE(p.status, bytes <= pl.seg && src - skew >= p.pixels &&
-                                       src - skew + bytes <= p.pixels + p.pixels_bytes)) {
-        mbar_arrive_expect_tx(bar, bytes);
-        bulk_copy_g2s(ring + (slot * 16u + lane) * pl.seg, src - skew, bytes, bar);
-      } else {
-        mbar_arrive(bar);
+  if (warp == kT2Tiles) {
+    // ---- the feeding warp ----------------------------------------------------------------------
+    const int32_t two_m = static_cast<int32_t>(2u * ay.M), two_r = static_cast<int32_t>(2u * ay.R);
+    uint32_t ynext = 0;  // the first output row of the CTA whose last tap has not passed
+    bool failed = false;
+    for (uint32_t m = 0; m < ntiles16; ++m) {
+      const uint32_t slot = m % pl.slots, r0 = ya + 16u * m, bar = full + 8u * slot;
+      if (m >= pl.slots) {  // every warp has given the slot back
+        if (!mbar_wait_parked(empty + 8u * slot, ((m / pl.slots) - 1u) & 1u)) failed = true;
+        if (__any_sync(0xffffffffu, failed)) {
+          failed = true;
+          break;
+        }
       }
-    } else {
-      mbar_arrive(bar);
+      // The weights of the output rows under this tile, as the B operand of the second
+      // product (16 input rows x 8 output rows, binary16): column g is the row with
+      // yl % 8 == g among ynext .. ynext + 7, the lane's k are input rows
+      // r0 + {2q, 2q + 1, 8 + 2q, 9 + 2q}.  An integer weight w < 2^16 goes in as two exact
+      // pieces, (w & 255) / 256 and w >> 8.
+      uint4 wrec = make_uint4(0u, 0u, 0u, 0u), drec;
+      {
+        const uint32_t yl = ynext + ((g - ynext) & 7u);
+        uint32_t w4[4] = {0u, 0u, 0u, 0u};
+        if (yl < nrows) {
+          const uint32_t Y = top + k0 + yl, rbase = r0 + 2u * q;
+          const int32_t d = static_cast<int32_t>((2u * rbase + 1u) * ay.R) -
+                            static_cast<int32_t>((2u * Y + 1u) * ay.n_in);
+#pragma unroll
+          for (uint32_t i = 0; i < 4; ++i) {
+            const uint32_t dr = (i & 1u) + 8u * (i >> 1);
+            const int32_t di = d + static_cast<int32_t>(dr) * two_r;
+            int32_t wgt = two_m - (di < 0 ? -di : di);
+            if (wgt < 0 || rbase + dr >= ay.n_in) wgt = 0;
+            w4[i] = static_cast<uint32_t>(wgt);
+          }
+        }
+        const uint32_t pair0 = __byte_perm(w4[0], w4[1], 0x5140);  // low, low, high, high bytes
+        const uint32_t pair1 = __byte_perm(w4[2], w4[3], 0x5140);
+        wrec.x = expand_bytes<0>(pair0, 0x1c00u, 0xc400u);  // (1024 + b) / 256 - 4
+        wrec.y = expand_bytes<0>(pair1, 0x1c00u, 0xc400u);
+        wrec.z = expand_bytes<1>(pair0, 0x3c00u, 0xe400u);  // (1024 + b) - 1024
+        wrec.w = expand_bytes<1>(pair1, 0x3c00u, 0xe400u);
+      }
+      // rows that are complete after this tile, for the lane's two columns of the second product
+      {
+        const uint32_t y0 = ynext + ((2u * q - ynext) & 7u), y1 = ynext + ((2u * q + 1u - ynext) & 7u);
+        const bool d0 = y0 < nrows && yhi[y0] <= r0 + 16u, d1 = y1 < nrows && yhi[y1] <= r0 + 16u;
+        drec.x = d0 ? y0 : 0xffffffffu;
+        drec.y = d1 ? y1 : 0xffffffffu;
+        drec.z = __float_as_uint(d0 ? invy[y0] : 0.f);
+        drec.w = __float_as_uint(d1 ? invy[y1] : 0.f);
+      }
+      meta[slot * (kT2MetaBytes / 16u) + lane] = wrec;
+      meta[slot * (kT2MetaBytes / 16u) + 32u + lane] = drec;
+      {
+        const uint32_t yl = ynext + (lane & 7u);
+        const bool done = yl < nrows && yhi[yl] <= r0 + 16u;
+        const uint32_t mask = __ballot_sync(0xffffffffu, done) & 0xffu;
+        ynext += static_cast<uint32_t>(__ffs(static_cast<int>(~mask))) - 1u;
+      }
+      __syncwarp();  // the record is written before any lane announces the tile
+      // the 16 rows of the tile, a lane per row: a row the CTA needs is copied and its bytes
+      // announced to the slot's barrier, the other lanes of the sixteen just arrive
+      if (lane < 16u) {
+        const uint32_t r = r0 + lane;
+        bool copied = false;
+        if (r >= ya_need && r < yb) {  // (rows before the first needed one get no weight)
+          const uint8_t* src = image + r * pitch + rowbyte0;
+          const uint32_t skew = static_cast<uint32_t>(reinterpret_cast<uintptr_t>(src)) & 15u;
+          uint32_t bytes = (skew + rowbytes + 15u) & ~15u;
+          if (bytes > static_cast<uint64_t>(stop - (src - skew)))  // only padding is lost
+            bytes = static_cast<uint32_t>(stop - (src - skew));
+          fence_async_shared();
+          // checked build: the row lies in its place in the ring and in the pixel buffer
+          if (PREBA_IN_RANGE(p.status, bytes <= pl.seg && src - skew >= p.pixels &&
+                                           src - skew + bytes <= p.pixels + p.pixels_bytes)) {
+            mbar_arrive_expect_tx(bar, bytes);
+            bulk_copy_g2s(ring + (slot * 16u + lane) * pl.seg, src - skew, bytes, bar);
+            copied = true;
+          }
+        }
+        if (!copied) mbar_arrive(bar);
+      }
     }
-  };
-  if (warp == kT2Warps - 1u)
-    for (uint32_t m = 0; m < pl.slots && m < ntiles16; ++m) issue(m);
+    if (failed) {
+      if (lane == 0) report(p.status, PREBA_ERR_TIMEOUT);
+      // copies already asked for may still be landing in the ring: wait for them (bounded)
+      // before the CTA's shared memory is given up
+      if (lane == 0)
+        for (uint32_t s = 0; s < pl.slots; ++s) {
+          (void)mbar_wait(full + 8u * s, 0u);
+          (void)mbar_wait(full + 8u * s, 1u);
+        }
+    }
+    return;
+  }
 
-  // The weights of this warp's M-tiles as A operands.  Row mr of an M-tile is channel mr % 3 of
-  // the tile's pixel mr / 3 (row 15 is unused); register r holds row g (+ 8 if r is odd), bytes
+  // ---- the warps that own an M-tile ----------------------------------------------------------------
+  // The weights as A operands.  Row mr of the M-tile is channel mr % 3 of the tile's pixel
+  // mr / 3 (row 15 is unused); register r holds row g (+ 8 if r is odd), bytes
   // k = 16 (r / 2) + 4 q + i of step s: the row position kst + 32 s + k.
-  const uint32_t g = lane >> 2, q = lane & 3u;
-  uint32_t ahi[2][KS][4], alo[2][KS][4];
-  int32_t kst[2];
-  float scale[2][2];   // per M-tile and row (g, g + 8): 1 / sum of the column's weights, times 1 / (255 std)
-  bool live[2];
+  uint32_t ahi[KS][4], alo[KS][4];
+  float scale[2];  // per row (g, g + 8): 2^22 / (sum of the column's weights * 255 std)
 #pragma unroll
-  for (uint32_t t = 0; t < 2; ++t) {
-    const uint32_t mt = warp + kT2Warps * t, col0 = kT2Px * mt;
-    live[t] = mt < mtiles;
-    int32_t start = 0;
-    if (live[t]) {
-      const int32_t nb = static_cast<int32_t>(3u * xlo[col0] - rowbyte0);
-      start = nb - static_cast<int32_t>((static_cast<uint32_t>(nb) + skew4) & 3u);
-    }
-    kst[t] = start;
+  for (uint32_t half = 0; half < 2; ++half) {
+    const uint32_t mr = g + 8u * half, col = col0 + mr / 3u, ch = mr % 3u;
+    const float mul = ch == 0u ? p.mul[0] : (ch == 1u ? p.mul[1] : p.mul[2]);
+    // (the second product leaves 2^-22 times the sum)
+    scale[half] = (live && mr < 15u && col < ncols) ? invx[col] * mul * 4194304.f : 0.f;
+  }
+  {
+    // The lane's first byte of the window as pixel and channel (three bytes further on, so
+    // that the number is not negative), then byte by byte: (rem + o) / 3 for o < 500 is
+    // ((rem + o) * 171) >> 9.
+    const uint32_t first = static_cast<uint32_t>(static_cast<int32_t>(rowbyte0) + kst +
+                                                 static_cast<int32_t>(4u * q) + 3);
+    const uint32_t first_px = first / 3u, first_rem = first - 3u * first_px;
 #pragma unroll
-    for (uint32_t half = 0; half < 2; ++half) {
-      const uint32_t mr = g + 8u * half, col = col0 + mr / 3u;
-      const uint32_t ch = mr % 3u;
-      const float mul = ch == 0u ? p.mul[0] : (ch == 1u ? p.mul[1] : p.mul[2]);
-      // (the second product leaves 2^-22 times the sum)
-      scale[t][half] = (live[t] && mr < 15u && col < ncols) ? invx[col] * mul * 4194304.f : 0.f;
-    }
+    for (uint32_t r = 0; r < 4; ++r) {
+      const uint32_t mr = g + 8u * (r & 1u), ch = mr % 3u, col = col0 + mr / 3u;
+      const bool on = live && mr < 15u && col < ncols;
+      // taps of the column as pixel numbers shifted like first_px; none if the row is unused
+      const uint32_t lo_px = on ? xlo[col] + 1u : 1u, n_px = on ? xcnt[col] : 0u;
+      const uint16_t* wrow = wxi + col * kMaxTapsX;
 #pragma unroll
-    for (uint32_t s = 0; s < KS; ++s)
-#pragma unroll
-      for (uint32_t r = 0; r < 4; ++r) {
-        const uint32_t mr = g + 8u * (r & 1u), ch = mr % 3u, col = col0 + mr / 3u;
-        const bool on = live[t] && mr < 15u && col < ncols;
-        const uint32_t lo_px = on ? xlo[col] : 0u, n_px = on ? xcnt[col] : 0u;
+      for (uint32_t s = 0; s < KS; ++s) {
         uint32_t hi = 0, lo = 0;
 #pragma unroll
         for (uint32_t i = 0; i < 4; ++i) {
-          const int32_t b = static_cast<int32_t>(rowbyte0) + start +
-                            static_cast<int32_t>(32u * s + 16u * (r >> 1) + 4u * q + i);
+          const uint32_t o = first_rem + 32u * s + 16u * (r >> 1) + i;
+          const uint32_t dpx = (o * 171u) >> 9, rem = o - 3u * dpx;
+          const uint32_t tap = first_px + dpx - lo_px;  // wraps below the first tap
           uint32_t wgt = 0;
-          if (b >= 0) {
-            const uint32_t px = static_cast<uint32_t>(b) / 3u;
-            if (static_cast<uint32_t>(b) - 3u * px == ch && px >= lo_px && px - lo_px < n_px)
-              wgt = wxi[col * kMaxTapsX + (px - lo_px)];
-          }
+          if (rem == ch && tap < n_px) wgt = wrow[tap];
           hi |= (wgt >> 8) << (8u * i);
           lo |= (wgt & 0xffu) << (8u * i);
         }
-        ahi[t][s][r] = hi;
-        alo[t][s][r] = lo;
+        ahi[s][r] = hi;
+        alo[s][r] = lo;
       }
+    }
   }
-  // where the lane's two rows of an M-tile go: plane of the channel, column of the pixel
+  // where the lane's two rows of the M-tile go: plane of the channel, column of the pixel
   const uint32_t px_a = g / 3u, px_b = (g + 8u) / 3u;
   const uint32_t ch_a = g % 3u, ch_b = (g + 8u) % 3u;
   const float add_a = ch_a == 0u ? p.add[0] : (ch_a == 1u ? p.add[1] : p.add[2]);
   const float add_b = ch_b == 0u ? p.add[0] : (ch_b == 1u ? p.add[1] : p.add[2]);
   OutT* out = static_cast<OutT*>(p.out) + static_cast<uint64_t>(img) * 3u * C * C;
-  OutT* out_a = out + static_cast<uint64_t>(ch_a) * C * C + xg0 + px_a;
-  OutT* out_b = out + static_cast<uint64_t>(ch_b) * C * C + xg0 + px_b;
+  OutT* out_a = out + static_cast<uint64_t>(ch_a) * C * C + xg0 + col0 + px_a;
+  OutT* out_b = out + static_cast<uint64_t>(ch_b) * C * C + xg0 + col0 + px_b;
 
   // The vertical sums: output row yl of the CTA uses column yl % 8 of the second product; a lane
   // holds columns 2q and 2q + 1 of rows g and g + 8.
-  float acc[2][4];
-#pragma unroll
-  for (uint32_t t = 0; t < 2; ++t)
-#pragma unroll
-    for (uint32_t i = 0; i < 4; ++i) acc[t][i] = 0.f;
-  uint32_t ynext = 0;  // the first output row of the CTA whose last tap has not passed
-  const int32_t two_m = static_cast<int32_t>(2u * ay.M), two_r = static_cast<int32_t>(2u * ay.R);
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
   // 16-byte skew of input row r: (base + r * pitch) & 15, in 32 bits
   const uint32_t skew_base = static_cast<uint32_t>(reinterpret_cast<uintptr_t>(image + rowbyte0)) & 15u;
   const uint32_t skew_step = static_cast<uint32_t>(pitch & 15u);
-  const uint32_t ring_row0 = g * pl.seg + 4u * q, ring_row1 = (g + 8u) * pl.seg + 4u * q;
+  const uint8_t* ring_row0 = ring_p + g * pl.seg + 4u * q + kst;
+  const uint8_t* ring_row1 = ring_row0 + 8u * pl.seg;
 
   bool failed = false;
-  for (uint32_t m = 0; m < ntiles16 && !failed; ++m) {
+  for (uint32_t m = 0; m < ntiles16; ++m) {
     const uint32_t slot = m % pl.slots, r0 = ya + 16u * m;
-    if (!mbar_wait(full + 8u * slot, (m / pl.slots) & 1u)) failed = true;
+    if (!mbar_wait_parked(full + 8u * slot, (m / pl.slots) & 1u)) failed = true;
     if (__any_sync(0xffffffffu, failed)) {
       failed = true;
       break;
     }
-    // The weights of the output rows under this tile, as the B operand of the second product
-    // (16 input rows x 8 output rows, binary16): column g is the row with yl % 8 == g among
-    // ynext .. ynext + 7, the lane's k are input rows r0 + {2q, 2q + 1, 8 + 2q, 9 + 2q}.  An
-    // integer weight w < 2^16 goes in as two exact pieces, (w & 255) / 256 and w >> 8.
-    uint32_t wlo[2] = {0u, 0u}, whi[2] = {0u, 0u};
-    {
-      const uint32_t yl = ynext + ((g - ynext) & 7u);
-      uint32_t w4[4] = {0u, 0u, 0u, 0u};
-      if (yl < nrows) {
-        const uint32_t Y = top + k0 + yl, rbase = r0 + 2u * q;
-        const int32_t d = static_cast<int32_t>((2u * rbase + 1u) * ay.R) -
-                          static_cast<int32_t>((2u * Y + 1u) * ay.n_in);
+    if (live) {
+      const uint4 wrec = meta[slot * (kT2MetaBytes / 16u) + lane];
+      const uint4 drec = meta[slot * (kT2MetaBytes / 16u) + 32u + lane];
+      // rows g and g + 8 of the tile: where their first needed byte lies in the slot
+      const uint32_t sk0 = (skew_base + (r0 + g) * skew_step) & 15u;
+      const uint32_t sk1 = (skew_base + (r0 + g + 8u) * skew_step) & 15u;
+      // checked build: the window of both rows lies in the row's place in the ring
+      if (PREBA_IN_RANGE(p.status,
+                         static_cast<int32_t>(sk0 + 4u * q) + kst >= 0 &&
+                             static_cast<int32_t>(sk1 + 4u * q) + kst >= 0 &&
+                             static_cast<int32_t>((sk0 > sk1 ? sk0 : sk1) + 4u * q) + kst +
+                                     static_cast<int32_t>(32u * KS - 12u) <=
+                                 static_cast<int32_t>(pl.seg) &&
+                             slot < pl.slots)) {
+        // first product, high and low bytes of the weights apart: e = rows 0-7 of the tile,
+        // f = rows 8-15
+        int32_t eh[4] = {0, 0, 0, 0}, el[4] = {0, 0, 0, 0}, fh[4] = {0, 0, 0, 0}, fl[4] = {0, 0, 0, 0};
+        const uint32_t* at0 = reinterpret_cast<const uint32_t*>(ring_row0 + slot * 16u * pl.seg + sk0);
+        const uint32_t* at1 = reinterpret_cast<const uint32_t*>(ring_row1 + slot * 16u * pl.seg + sk1);
+#pragma unroll
+        for (uint32_t s = 0; s < KS; ++s) {
+          const uint32_t b00 = at0[8 * s], b01 = at0[8 * s + 4], b10 = at1[8 * s], b11 = at1[8 * s + 4];
+          mma_u8(eh, ahi[s], b00, b01);
+          mma_u8(el, alo[s], b00, b01);
+          mma_u8(fh, ahi[s], b10, b11);
+          mma_u8(fl, alo[s], b10, b11);
+        }
+        // H = 256 high + low, below 2^24; register i: row g + 8 (i / 2), input row 2q + i % 2
+        uint32_t he[4], hf[4];
 #pragma unroll
         for (uint32_t i = 0; i < 4; ++i) {
-          const uint32_t dr = (i & 1u) + 8u * (i >> 1);
-          const int32_t di = d + static_cast<int32_t>(dr) * two_r;
-          int32_t wgt = two_m - (di < 0 ? -di : di);
-          if (wgt < 0 || rbase + dr >= ay.n_in) wgt = 0;
-          w4[i] = static_cast<uint32_t>(wgt);
+          he[i] = (static_cast<uint32_t>(eh[i]) << 8) + static_cast<uint32_t>(el[i]);
+          hf[i] = (static_cast<uint32_t>(fh[i]) << 8) + static_cast<uint32_t>(fl[i]);
+        }
+        // The three bytes of H as binary16 A operands of the second product (16 (x, ch) rows
+        // by 16 input rows): byte 0 scaled by 2^-14, byte 1 by 2^-6, byte 2 by 4, all exact,
+        // so that the sum is 2^-22 times sum_r w[r] H[r].
+#pragma unroll
+        for (uint32_t pln = 0; pln < 3; ++pln) {
+          uint32_t a[4];
+#pragma unroll
+          for (uint32_t h = 0; h < 2; ++h) {
+            // bytes pln of the four values of row g + 8 h: input rows 2q, 2q + 1 (e),
+            // 8 + 2q, 9 + 2q (f)
+            const uint32_t sel = pln == 0 ? 0x0040u : (pln == 1 ? 0x0051u : 0x0062u);
+            const uint32_t pe = __byte_perm(he[2 * h], he[2 * h + 1], sel);
+            const uint32_t pf = __byte_perm(hf[2 * h], hf[2 * h + 1], sel);
+            const uint32_t mul = pln == 0 ? 0x0400u : (pln == 1 ? 0x2400u : 0x4400u);
+            const uint32_t off = pln == 0 ? 0xac00u : (pln == 1 ? 0xcc00u : 0xec00u);
+            a[h] = expand_bytes<0>(pe, mul, off);      // k = 2q, 2q + 1
+            a[2 + h] = expand_bytes<0>(pf, mul, off);  // k = 8 + 2q, 9 + 2q
+          }
+          mma_f16(acc, a, wrec.x, wrec.y);
+          mma_f16(acc, a, wrec.z, wrec.w);
         }
       }
-#pragma unroll
-      for (uint32_t h = 0; h < 2; ++h) {
-        const uint32_t pair = __byte_perm(w4[2 * h], w4[2 * h + 1], 0x5140);  // lo, lo, hi, hi bytes
-        wlo[h] = expand_bytes<0>(pair, 0x1c00u, 0xc400u);   // (1024 + b) / 256 - 4
-        whi[h] = expand_bytes<1>(pair, 0x3c00u, 0xe400u);   // (1024 + b) - 1024
-      }
-    }
-    // rows that are complete after this tile, for the lane's two columns
-    uint32_t done_row[2];
-    float done_inv[2];
-#pragma unroll
-    for (uint32_t c = 0; c < 2; ++c) {
-      const uint32_t yl = ynext + ((2u * q + c - ynext) & 7u);
-      const bool done = yl < nrows && yhi[yl] <= r0 + 16u;
-      done_row[c] = done ? yl : 0xffffffffu;
-      done_inv[c] = done ? invy[yl] : 0.f;
-    }
-    // rows g and g + 8 of the tile: where their first needed byte lies in the slot
-    const uint32_t sk0 = (skew_base + (r0 + g) * skew_step) & 15u;
-    const uint32_t sk1 = (skew_base + (r0 + g + 8u) * skew_step) & 15u;
-    const uint8_t* row0 = ring_p + slot * 16u * pl.seg + ring_row0 + sk0;
-    const uint8_t* row1 = ring_p + slot * 16u * pl.seg + ring_row1 + sk1;
-#pragma unroll
-    for (uint32_t t = 0; t < 2; ++t) {
-      if (!live[t]) continue;
-      // checked build: the window of both rows lies in the row's place in the ring
-      if (!PREBA_IN_RANGE(p.status,
-                          static_cast<int32_t>(sk0 + 4u * q) + kst[t] >= 0 &&
-                              static_cast<int32_t>(sk1 + 4u * q) + kst[t] >= 0 &&
-                              static_cast<int32_t>((sk0 > sk1 ? sk0 : sk1) + 4u * q) + kst[t] +
-                                      static_cast<int32_t>(32u * KS - 12u) <=
-                                  static_cast<int32_t>(pl.seg) &&
-                              slot < pl.slots))
-        continue;
-      // first product, high and low bytes of the weights apart: e = rows 0-7 of the tile,
-      // f = rows 8-15
-      int32_t eh[4] = {0, 0, 0, 0}, el[4] = {0, 0, 0, 0}, fh[4] = {0, 0, 0, 0}, fl[4] = {0, 0, 0, 0};
-      const uint32_t* at0 = reinterpret_cast<const uint32_t*>(row0 + kst[t]);
-      const uint32_t* at1 = reinterpret_cast<const uint32_t*>(row1 + kst[t]);
-#pragma unroll
-      for (uint32_t s = 0; s < KS; ++s) {
-        const uint32_t b00 = at0[8 * s], b01 = at0[8 * s + 4], b10 = at1[8 * s], b11 = at1[8 * s + 4];
-        mma_u8(eh, ahi[t][s], b00, b01);
-        mma_u8(el, alo[t][s], b00, b01);
-        mma_u8(fh, ahi[t][s], b10, b11);
-        mma_u8(fl, alo[t][s], b10, b11);
-      }
-      // H = 256 high + low, below 2^24; register i: row g + 8 (i / 2), input row 2q + i % 2
-      uint32_t he[4], hf[4];
-#pragma unroll
-      for (uint32_t i = 0; i < 4; ++i) {
-        he[i] = (static_cast<uint32_t>(eh[i]) << 8) + static_cast<uint32_t>(el[i]);
-        hf[i] = (static_cast<uint32_t>(fh[i]) << 8) + static_cast<uint32_t>(fl[i]);
-      }
-      // The three bytes of H as binary16 A operands of the second product (16 (x, ch) rows by
-      // 16 input rows): byte 0 scaled by 2^-14, byte 1 by 2^-6, byte 2 by 4, all exact, so
-      // that the sum below is 2^-22 times sum_r w[r] H[r].
-#pragma unroll
-      for (uint32_t pln = 0; pln < 3; ++pln) {
-        uint32_t a[4];
-#pragma unroll
-        for (uint32_t h = 0; h < 2; ++h) {
-          // bytes pln of the four values of row g + 8 h: input rows 2q, 2q + 1 (e), 8 + 2q, 9 + 2q (f)
-          const uint32_t sel = pln == 0 ? 0x0040u : (pln == 1 ? 0x0051u : 0x0062u);
-          const uint32_t pe = __byte_perm(he[2 * h], he[2 * h + 1], sel);
-          const uint32_t pf = __byte_perm(hf[2 * h], hf[2 * h + 1], sel);
-          const uint32_t mul = pln == 0 ? 0x0400u : (pln == 1 ? 0x2400u : 0x4400u);
-          const uint32_t off = pln == 0 ? 0xac00u : (pln == 1 ? 0xcc00u : 0xec00u);
-          a[h] = expand_bytes<0>(pe, mul, off);      // k = 2q, 2q + 1
-          a[2 + h] = expand_bytes<0>(pf, mul, off);  // k = 8 + 2q, 9 + 2q
+      // rows whose last tap has passed: normalise, store, start the column afresh
+      {
+        const bool dx = drec.x != 0xffffffffu, dy = drec.y != 0xffffffffu;
+        const uint32_t offx = (k0 + drec.x) * C, offy = (k0 + drec.y) * C;
+        const float ix = __uint_as_float(drec.z), iy = __uint_as_float(drec.w);
+        const float vx_a = fmaf(acc[0] * ix, scale[0], add_a), vx_b = fmaf(acc[2] * ix, scale[1], add_b);
+        const float vy_a = fmaf(acc[1] * iy, scale[0], add_a), vy_b = fmaf(acc[3] * iy, scale[1], add_b);
+        // checked build: the rows and the columns lie in the crop
+        if (PREBA_IN_RANGE(p.status, (!dx || k0 + drec.x < C) && (!dy || k0 + drec.y < C) &&
+                                         (scale[0] == 0.f || xg0 + col0 + px_a < C) &&
+                                         (scale[1] == 0.f || xg0 + col0 + px_b < C))) {
+          if (dx && scale[0] != 0.f) out_a[offx] = to_out<OutT>(vx_a);
+          if (dx && scale[1] != 0.f) out_b[offx] = to_out<OutT>(vx_b);
+          if (dy && scale[0] != 0.f) out_a[offy] = to_out<OutT>(vy_a);
+          if (dy && scale[1] != 0.f) out_b[offy] = to_out<OutT>(vy_b);
         }
-        mma_f16(acc[t], a, wlo[0], wlo[1]);
-        mma_f16(acc[t], a, whi[0], whi[1]);
-      }
-      // rows whose last tap has passed: normalise, store
-      const uint32_t col0 = kT2Px * (warp + kT2Warps * t);
-#pragma unroll
-      for (uint32_t c = 0; c < 2; ++c) {
-        if (done_row[c] == 0xffffffffu) continue;
-        const uint32_t rowoff = (k0 + done_row[c]) * C + col0;
-        // checked build: the row and the columns lie in the crop
-        if (PREBA_IN_RANGE(p.status, k0 + done_row[c] < C &&
-                                         (scale[t][0] == 0.f || xg0 + col0 + px_a < C) &&
-                                         (scale[t][1] == 0.f || xg0 + col0 + px_b < C))) {
-          if (scale[t][0] != 0.f)
-            out_a[rowoff] = to_out<OutT>(fmaf(acc[t][c] * done_inv[c], scale[t][0], add_a));
-          if (scale[t][1] != 0.f)
-            out_b[rowoff] = to_out<OutT>(fmaf(acc[t][2 + c] * done_inv[c], scale[t][1], add_b));
-        }
-        acc[t][c] = acc[t][2 + c] = 0.f;
+        acc[0] = dx ? 0.f : acc[0];
+        acc[2] = dx ? 0.f : acc[2];
+        acc[1] = dy ? 0.f : acc[1];
+        acc[3] = dy ? 0.f : acc[3];
       }
     }
-    // the staged rows of this tile have been read: the warp gives the slot back
+    // the staged rows and the record of this tile have been read: the warp gives the slot back
     __syncwarp();
     if (lane == 0) mbar_arrive(empty + 8u * slot);
-    // the rows that are complete now
-    {
-      const uint32_t yl = ynext + (lane & 7u);
-      const bool done = yl < nrows && yhi[yl] <= r0 + 16u;
-      const uint32_t mask = __ballot_sync(0xffffffffu, done) & 0xffu;
-      ynext += static_cast<uint32_t>(__ffs(static_cast<int>(~mask))) - 1u;
-    }
-    // when every warp has given the slot back it takes the rows of tile m + slots
-    if (warp == kT2Warps - 1u && m + pl.slots < ntiles16) {
-      bool ok = true;
-      if (lane < 16u) ok = mbar_wait(empty + 8u * slot, (m / pl.slots) & 1u);
-      if (__all_sync(0xffffffffu, ok)) issue(m + pl.slots);
-      else failed = true;
-    }
   }
-  if (failed) {
-    if (lane == 0) report(p.status, PREBA_ERR_TIMEOUT);
-    // copies already asked for may still be landing in the ring: the issuing warp waits for
-    // them (bounded) before the CTA's shared memory is given up
-    if (warp == kT2Warps - 1u && lane == 0)
-      for (uint32_t s = 0; s < pl.slots; ++s) {
-        (void)mbar_wait(full + 8u * s, 0u);
-        (void)mbar_wait(full + 8u * s, 1u);
-      }
-  }
+  if (failed && lane == 0) report(p.status, PREBA_ERR_TIMEOUT);
 }
 
 }  // namespace aa
@@ -1532,6 +1563,9 @@ Kernel mma_kernel_for(int out_dtype) {
 // Shared memory of the tensor-core kernel's launch: its tables, a tile of H and a ring of three
 // 16-row slots of 1080p-wide groups fit, and two CTAs share an SM.
 constexpr int kMmaSmemBytes = 108 * 1024;
+// Of the kernel with both passes on the tensor cores, two CTAs of sixteen warps per SM: its
+// tables and a ring of five 16-row slots of 1080p-wide groups.
+constexpr int kMm2SmemBytes = 108 * 1024;
 
 // Largest dynamic shared memory a CTA may ask for on the current device; the three kernels
 // are opted in to it once per device.
@@ -1556,10 +1590,10 @@ int shared_memory_limit(cudaError_t* err) {
                                   optin < kMmaSmemBytes ? optin : kMmaSmemBytes);
     if (*err == cudaSuccess)
       *err = cudaFuncSetAttribute(mm2_kernel_for<3>(dt), cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                  optin < kMmaSmemBytes ? optin : kMmaSmemBytes);
+                                  optin < kMm2SmemBytes ? optin : kMm2SmemBytes);
     if (*err == cudaSuccess)
       *err = cudaFuncSetAttribute(mm2_kernel_for<4>(dt), cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                  optin < kMmaSmemBytes ? optin : kMmaSmemBytes);
+                                  optin < kMm2SmemBytes ? optin : kMm2SmemBytes);
   }
   if (*err != cudaSuccess) return 0;
   if (dev >= 0 && dev < kMaxDevices) cache[dev].store(optin, std::memory_order_relaxed);
@@ -1608,6 +1642,7 @@ extern "C" int preba_preprocess_antialias(const preba_batch_t* batch, const preb
   // other one the rest; each skips the other's images.  With the host's copy of the table a
   // kernel without images is not launched at all.
   const uint32_t mma_smem = static_cast<uint32_t>(limit < kMmaSmemBytes ? limit : kMmaSmemBytes);
+  const uint32_t mm2_smem = static_cast<uint32_t>(limit < kMm2SmemBytes ? limit : kMm2SmemBytes);
   bool any_mma = true, any_rest = true, any_mm2[2] = {true, true};  // windows of 3 and 4 steps
   if (batch->table_host) {
     uint64_t most = 0;
@@ -1627,7 +1662,7 @@ extern "C" int preba_preprocess_antialias(const preba_batch_t* batch, const preb
            opt->crop_origin_host[2 * i + 1] + static_cast<uint64_t>(C) > rw))
         return PREBA_ERR_BAD_CROP;
       preba::aa::Mm2Plan two;
-      if (mm2_plan(make_axis(e.w, rw), make_axis(e.h, rh), e.w, C, mma_smem, &two)) {
+      if (mm2_plan(make_axis(e.w, rw), make_axis(e.h, rh), e.w, C, mm2_smem, &two)) {
         any_mm2[two.ks - 3u] = true;
         continue;
       }
@@ -1680,7 +1715,7 @@ extern "C" int preba_preprocess_antialias(const preba_batch_t* batch, const preb
   p.rows = rows;
   p.smem_floats = floats;
   p.mma_smem = any_mma ? mma_smem : 0u;
-  p.mm2_smem = (any_mm2[0] || any_mm2[1]) ? mma_smem : 0u;
+  p.mm2_smem = (any_mm2[0] || any_mm2[1]) ? mm2_smem : 0u;
   // Output rows per CTA of the chained kernel: the chunking of an image's rows whose CTAs fill
   // the rounds of what the GPU holds at once (two CTAs per SM) best, fewest chunks first; no
   // CTA below 32 rows.
@@ -1725,7 +1760,7 @@ extern "C" int preba_preprocess_antialias(const preba_batch_t* batch, const preb
                           ((C + preba::aa::kT2Group - 1) / preba::aa::kT2Group);
     if (ctas > 0x7fffffffull) return PREBA_ERR_INVALID_ARG;
     (v == 0 ? mm2_kernel_for<3>(opt->out_dtype) : mm2_kernel_for<4>(opt->out_dtype))
-        <<<static_cast<uint32_t>(ctas), kMmaThreads, mma_smem, s>>>(p);
+        <<<static_cast<uint32_t>(ctas), preba::aa::kT2Threads, mm2_smem, s>>>(p);
     err = cudaGetLastError();
   }
   if (any_mma && err == cudaSuccess) {
