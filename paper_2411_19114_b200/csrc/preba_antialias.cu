@@ -1150,13 +1150,15 @@ __device__ __forceinline__ void mma_f16(float (&d)[4], const uint32_t (&a)[4], u
 // numbers, each times a power of two: a byte b under the exponent byte 0x64 is the number
 // 1024 + b, and one fused multiply-add, (1024 + b) * mul - 1024 * mul, leaves b * mul exactly
 // (mul and off are the binary16 patterns of mul and of -1024 * mul).
-template <uint32_t PAIR>
-__device__ __forceinline__ uint32_t expand_bytes(uint32_t x, uint32_t mul, uint32_t off) {
-  const uint32_t biased = __byte_perm(x, 0x64646464u, PAIR == 0 ? 0x4140u : 0x4342u);
+__device__ __forceinline__ uint32_t scale_biased(uint32_t biased, uint32_t mul, uint32_t off) {
   uint32_t r;
   const uint32_t mul2 = mul | (mul << 16), off2 = off | (off << 16);
   asm("fma.rn.f16x2 %0, %1, %2, %3;" : "=r"(r) : "r"(biased), "r"(mul2), "r"(off2));
   return r;
+}
+template <uint32_t PAIR>
+__device__ __forceinline__ uint32_t expand_bytes(uint32_t x, uint32_t mul, uint32_t off) {
+  return scale_biased(__byte_perm(x, 0x64646464u, PAIR == 0 ? 0x4140u : 0x4342u), mul, off);
 }
 
 template <typename OutT, uint32_t KS>
@@ -1284,10 +1286,13 @@ __global__ void __launch_bounds__(kT2Threads, 2) preba_antialias_mm2_kernel(cons
     const int32_t two_m = static_cast<int32_t>(2u * ay.M), two_r = static_cast<int32_t>(2u * ay.R);
     uint32_t ynext = 0;  // the first output row of the CTA whose last tap has not passed
     bool failed = false;
-    for (uint32_t m = 0; m < ntiles16; ++m) {
-      const uint32_t slot = m % pl.slots, r0 = ya + 16u * m, bar = full + 8u * slot;
-      if (m >= pl.slots) {  // every warp has given the slot back
-        if (!mbar_wait_parked(empty + 8u * slot, ((m / pl.slots) - 1u) & 1u)) failed = true;
+    // (slot and use of tile m: m % slots and m / slots, counted along)
+    uint32_t slot = 0, use = 0;
+    for (uint32_t m = 0; m < ntiles16; ++m, slot = slot + 1u == pl.slots ? 0u : slot + 1u,
+                  use += slot == 0u ? 1u : 0u) {
+      const uint32_t r0 = ya + 16u * m, bar = full + 8u * slot;
+      if (use > 0u) {  // every warp has given the slot back
+        if (!mbar_wait_parked(empty + 8u * slot, (use - 1u) & 1u)) failed = true;
         if (__any_sync(0xffffffffu, failed)) {
           failed = true;
           break;
@@ -1440,9 +1445,11 @@ __global__ void __launch_bounds__(kT2Threads, 2) preba_antialias_mm2_kernel(cons
   const uint8_t* ring_row1 = ring_row0 + 8u * pl.seg;
 
   bool failed = false;
-  for (uint32_t m = 0; m < ntiles16; ++m) {
-    const uint32_t slot = m % pl.slots, r0 = ya + 16u * m;
-    if (!mbar_wait_parked(full + 8u * slot, (m / pl.slots) & 1u)) failed = true;
+  uint32_t slot = 0, use = 0;  // of tile m: m % slots and m / slots, counted along
+  for (uint32_t m = 0; m < ntiles16; ++m, slot = slot + 1u == pl.slots ? 0u : slot + 1u,
+                use += slot == 0u ? 1u : 0u) {
+    const uint32_t r0 = ya + 16u * m;
+    if (!mbar_wait_parked(full + 8u * slot, use & 1u)) failed = true;
     if (__any_sync(0xffffffffu, failed)) {
       failed = true;
       break;
@@ -1463,7 +1470,11 @@ __global__ void __launch_bounds__(kT2Threads, 2) preba_antialias_mm2_kernel(cons
                              slot < pl.slots)) {
         // first product, high and low bytes of the weights apart: e = rows 0-7 of the tile,
         // f = rows 8-15
-        int32_t eh[4] = {0, 0, 0, 0}, el[4] = {0, 0, 0, 0}, fh[4] = {0, 0, 0, 0}, fl[4] = {0, 0, 0, 0};
+        // (the low sums start at 0x64 in their top byte, which H never reaches: the exponent
+        // byte of the binary16 pieces below comes along for free)
+        constexpr int32_t kTop = 0x64000000;
+        int32_t eh[4] = {0, 0, 0, 0}, el[4] = {kTop, kTop, kTop, kTop}, fh[4] = {0, 0, 0, 0},
+                fl[4] = {kTop, kTop, kTop, kTop};
         const uint32_t* at0 = reinterpret_cast<const uint32_t*>(ring_row0 + slot * 16u * pl.seg + sk0);
         const uint32_t* at1 = reinterpret_cast<const uint32_t*>(ring_row1 + slot * 16u * pl.seg + sk1);
 #pragma unroll
@@ -1474,7 +1485,8 @@ __global__ void __launch_bounds__(kT2Threads, 2) preba_antialias_mm2_kernel(cons
           mma_u8(fh, ahi[s], b10, b11);
           mma_u8(fl, alo[s], b10, b11);
         }
-        // H = 256 high + low, below 2^24; register i: row g + 8 (i / 2), input row 2q + i % 2
+        // H = 256 high + low, below 2^24, under the byte 0x64; register i: row g + 8 (i / 2),
+        // input row 2q + i % 2
         uint32_t he[4], hf[4];
 #pragma unroll
         for (uint32_t i = 0; i < 4; ++i) {
@@ -1491,13 +1503,14 @@ __global__ void __launch_bounds__(kT2Threads, 2) preba_antialias_mm2_kernel(cons
           for (uint32_t h = 0; h < 2; ++h) {
             // bytes pln of the four values of row g + 8 h: input rows 2q, 2q + 1 (e),
             // 8 + 2q, 9 + 2q (f)
-            const uint32_t sel = pln == 0 ? 0x0040u : (pln == 1 ? 0x0051u : 0x0062u);
+            // one permute puts each byte under the exponent byte: the numbers 1024 + byte
+            const uint32_t sel = pln == 0 ? 0x7430u : (pln == 1 ? 0x7531u : 0x7632u);
             const uint32_t pe = __byte_perm(he[2 * h], he[2 * h + 1], sel);
             const uint32_t pf = __byte_perm(hf[2 * h], hf[2 * h + 1], sel);
             const uint32_t mul = pln == 0 ? 0x0400u : (pln == 1 ? 0x2400u : 0x4400u);
             const uint32_t off = pln == 0 ? 0xac00u : (pln == 1 ? 0xcc00u : 0xec00u);
-            a[h] = expand_bytes<0>(pe, mul, off);      // k = 2q, 2q + 1
-            a[2 + h] = expand_bytes<0>(pf, mul, off);  // k = 8 + 2q, 9 + 2q
+            a[h] = scale_biased(pe, mul, off);      // k = 2q, 2q + 1
+            a[2 + h] = scale_biased(pf, mul, off);  // k = 8 + 2q, 9 + 2q
           }
           mma_f16(acc, a, wrec.x, wrec.y);
           mma_f16(acc, a, wrec.z, wrec.w);
