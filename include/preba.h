@@ -281,17 +281,22 @@ int preba_preprocess_ex(const preba_batch_t* batch, const preba_options_t* opt, 
  * `opt` is read as by preba_preprocess_ex (crop windows included) with flags == 0 and a float
  * out_dtype; batch layout, table checks and status word are those of preba_preprocess;
  * batch->scratch is not used and PREBA_OVERLAP_PREVIOUS has no effect.
- * Two kernels share the work, each skipping the other's images.  Images whose width is a
- * multiple of 4 and that are reduced up to about six times (or enlarged up to about six times)
- * go to a kernel that runs the horizontal pass as integer matrix instructions on the tensor
- * cores (the input rows as they lie in memory against the integer weights, exact) and the
- * vertical pass in fp32.  Every other image goes to a kernel in which a CTA keeps one
- * channel-planar row of the window's footprint and the weight tables in shared memory.  With
- * `table_host` only the kernels that have images are enqueued on `stream` (one or two), the
- * second kernel's launch carries what its largest image needs, and an image that needs more
+ * Up to four kernels share the work, each skipping the others' images.  Images whose width is
+ * a multiple of 4 and that are reduced more than 2.5 times vertically (and up to about 6.5
+ * times horizontally) go to a kernel that runs both passes on the tensor cores: the horizontal
+ * one as integer matrix instructions (the input rows as they lie in memory against the integer
+ * weights, exact), the vertical one as binary16 matrix instructions on the exact bytes of the
+ * horizontal sums against the exact bytes of the integer weights, accumulated in fp32 (two
+ * instances: horizontal windows of 96 and of 128 bytes).  Other images whose width is a
+ * multiple of 4 and that are reduced or enlarged up to about six times go to a kernel with
+ * the horizontal pass on the tensor cores and the vertical pass in fp32.  Every other image
+ * goes to a kernel in which a CTA keeps one channel-planar row of the window's footprint and
+ * the weight tables in shared memory.  The result of an image does not depend on the batch it
+ * is in.  With `table_host` only the kernels that have images are enqueued on `stream`, the
+ * last kernel's launch carries what its largest image needs, and an image that needs more
  * than the device allows is refused (PREBA_ERR_TOO_LARGE: reductions beyond about 40 at
- * out_size 224); without it both kernels are enqueued, the second carries all the device
- * allows and skips and reports such an image in the status word.
+ * out_size 224); without it all are enqueued, the last carries all the device allows and
+ * skips and reports such an image in the status word.
  * Errors: PREBA_ERR_INVALID_ARG, PREBA_ERR_BUFFER_TOO_SMALL, PREBA_ERR_BAD_TABLE,
  * PREBA_ERR_BAD_CROP, PREBA_ERR_TOO_LARGE, PREBA_ERR_CUDA.
  */
