@@ -12,8 +12,8 @@
 //   decode_segments a thread per restart interval reads its bits (0xFF00 unstuffed), decodes the
 //                   DC differences and AC runs of its MCUs and writes the quantised coefficients
 //                   of every block in natural order (int16);
-//   idct_colour     a block per MCU: dequantisation, the inverse DCT of T.81 A.3.3 in exact
-//                   integers (the basis times 2^20, horizontal sums first and reduced by 2^9,
+//   idct_colour     eight threads per 8 x 8 block, 32 blocks per CTA: dequantisation, the
+//                   inverse DCT of T.81 A.3.3 in exact integers (the basis times 2^20, horizontal sums first and reduced by 2^9,
 //                   vertical sums at scale 2^31, level shift, one rounding, clamp); chroma
 //                   enlarged by replication; YCbCr -> RGB by the JFIF equations with the
 //                   coefficients times 2^16 and one rounding; the pixels go straight into the
@@ -427,99 +427,136 @@ __global__ void __launch_bounds__(64) decode_segments(const Params p) {
   }
 }
 
-// round(2^20 * cos(k pi / 16) / 2), k = 0..7.
-__device__ const int32_t kCosFix[8] = {524288, 514214, 484379, 435930, 370728, 291279, 200636, 102284};
-
-// round(2^20 (C_u / 2) cos((2x + 1) u pi / 16)) of T.81 A.3.3, from the eight values by symmetry.
-__device__ __forceinline__ int32_t basis(uint32_t x, uint32_t u) {
-  if (u == 0) return kCosFix[4];
+// round(2^20 (C_u / 2) cos((2x + 1) u pi / 16)) of T.81 A.3.3, from round(2^20 cos(k pi / 16) / 2),
+// k = 0..7, by symmetry; a compile-time constant wherever x and u are.
+__host__ __device__ constexpr int32_t cos_fix(uint32_t k) {
+  return k == 0 ? 524288 : k == 1 ? 514214 : k == 2 ? 484379 : k == 3 ? 435930 : k == 4 ? 370728
+         : k == 5 ? 291279 : k == 6 ? 200636 : 102284;
+}
+__host__ __device__ constexpr int32_t basis(uint32_t x, uint32_t u) {
+  if (u == 0) return cos_fix(4);
   uint32_t k = ((2 * x + 1) * u) & 31u;
   if (k > 16) k = 32 - k;
-  return k <= 7 ? kCosFix[k] : (k == 8 ? 0 : -kCosFix[16 - k]);
+  return k <= 7 ? cos_fix(k) : (k == 8 ? 0 : -cos_fix(16 - k));
 }
 
-__device__ __forceinline__ uint32_t clamp255(int64_t v) {
+// The eight sums sum_u basis(x, u) in[u], x = 0..7, exact in 64 bits.  basis(7 - x, u) is
+// basis(x, u) for even u and its negative for odd u, so the even and the odd terms are summed
+// once for x and 7 - x.
+__device__ __forceinline__ void transform8(const int32_t (&in)[8], int64_t (&out)[8]) {
+#pragma unroll
+  for (uint32_t x = 0; x < 4; ++x) {
+    int64_t even = 0, odd = 0;
+#pragma unroll
+    for (uint32_t u = 0; u < 8; u += 2) {
+      even += static_cast<int64_t>(basis(x, u)) * in[u];
+      odd += static_cast<int64_t>(basis(x, u + 1)) * in[u + 1];
+    }
+    out[x] = even + odd;
+    out[7 - x] = even - odd;
+  }
+}
+
+__device__ __forceinline__ uint32_t clamp255(int32_t v) {
   return v <= 0 ? 0u : (v >= 255 ? 255u : static_cast<uint32_t>(v));
 }
 
-// A block per MCU (blockIdx.y: image): 64 threads per 8 x 8 block of the MCU transform it, then
-// the threads convert the MCU's pixels and store them.  Exact integer arithmetic throughout:
-// the basis times 2^20, the row sums reduced by 2^9, the column sums at scale 2^31.
-constexpr uint32_t kMaxMcuBlocks = 6;
+// Eight threads per 8 x 8 block, 32 blocks per CTA: as many whole MCUs as that holds
+// (blockIdx.y: image).  A thread takes a row of the block through the horizontal sums, then,
+// after an exchange through shared memory within its warp, a column through the vertical
+// ones; then all threads convert the MCUs' pixels and store them.  Exact integer arithmetic
+// throughout: the basis times 2^20, the row sums reduced by 2^9, the column sums at scale 2^31.
+constexpr uint32_t kIdctThreads = 256;
+constexpr uint32_t kIdctBlocks = kIdctThreads / 8;
+constexpr uint32_t kTilePitch = 72;  // words between the blocks' tiles: four blocks of a warp
+                                     // read eight words each from different banks
 
-__global__ void __launch_bounds__(64 * kMaxMcuBlocks) idct_colour(const Params p) {
-  __shared__ int32_t a[64];                      // the basis
-  __shared__ int32_t work[kMaxMcuBlocks][64];    // dequantised coefficients, then row sums
-  __shared__ uint8_t smp[kMaxMcuBlocks][64];     // the samples of the MCU's blocks
+__host__ __device__ inline uint32_t mcus_per_cta(uint32_t blocks_per_mcu) {
+  return kIdctBlocks / blocks_per_mcu;
+}
+
+__global__ void __launch_bounds__(kIdctThreads) idct_colour(const Params p) {
+  __shared__ __align__(16) int32_t tile[kIdctBlocks * kTilePitch];  // row sums, [v][x] per block
+  __shared__ uint8_t smp[kIdctBlocks][64];                           // the samples of the blocks
   const Desc& d = desc_of(p, blockIdx.y);
   const uint32_t mcus = d.mcu_cols * d.mcu_rows;
-  if (blockIdx.x >= mcus) return;
   uint32_t per_mcu = 0;
   for (uint32_t c = 0; c < d.ncomp; ++c) per_mcu += d.hs[c] * d.vs[c];
-  const uint32_t tid = threadIdx.x, blk = tid >> 6, e = tid & 63u;
-  if (tid < 64) a[tid] = basis(tid >> 3, tid & 7u);
-  const bool live = blk < per_mcu;
-  uint32_t comp = 0;
+  const uint32_t held = mcus_per_cta(per_mcu), first = blockIdx.x * held;
+  if (first >= mcus) return;
+  const uint32_t tid = threadIdx.x, group = tid >> 3, r = tid & 7u;
+  const uint32_t local = group / per_mcu, blk = group - local * per_mcu, mcu = first + local;
+  const bool live = local < held && mcu < mcus;
   if (live) {
-    uint32_t before = 0;
+    uint32_t comp = 0, before = 0;
     while (comp + 1 < d.ncomp && blk >= before + d.hs[comp] * d.vs[comp]) {
       before += d.hs[comp] * d.vs[comp];
       ++comp;
     }
-    const int16_t* coef = p.coef + (d.coef_off + static_cast<uint64_t>(blockIdx.x) * per_mcu + blk) * 64;
-    // S = Sq * Q (A.3.4), limited to what the sums below hold (a valid stream stays far inside)
-    const int32_t deq = static_cast<int32_t>(coef[e]) * static_cast<int32_t>(d.qt[comp][e]);
-    work[blk][e] = max(-16383, min(16383, deq));
-  }
-  __syncthreads();
-  int32_t rowsum = 0;
-  if (live) {
-    // horizontal sums: thread (v, x) of the block
-    const uint32_t v = e >> 3, x = e & 7u;
-    int64_t t = 0;
+    // row r of the block: S = Sq * Q (A.3.4), limited to what the sums below hold (a valid
+    // stream stays far inside)
+    const int16_t* coef = p.coef + (d.coef_off + static_cast<uint64_t>(mcu) * per_mcu + blk) * 64 + 8u * r;
+    const int4 raw = *reinterpret_cast<const int4*>(coef);
+    const int32_t packed[4] = {raw.x, raw.y, raw.z, raw.w};
+    const uint16_t* q = d.qt[comp] + 8u * r;
+    int32_t in[8];
 #pragma unroll
-    for (uint32_t u = 0; u < 8; ++u)
-      t += static_cast<int64_t>(a[8 * x + u]) * work[blk][8 * v + u];
-    rowsum = static_cast<int32_t>((t + (1 << 8)) >> 9);
-  }
-  __syncthreads();
-  if (live) work[blk][e] = rowsum;  // [v][x]
-  __syncthreads();
-  if (live) {
-    const uint32_t y = e >> 3, x = e & 7u;
-    int64_t s = 0;
+    for (uint32_t u = 0; u < 8; ++u) {
+      const int32_t c16 = static_cast<int16_t>(static_cast<uint32_t>(packed[u >> 1]) >> (16u * (u & 1u)));
+      in[u] = max(-16383, min(16383, c16 * static_cast<int32_t>(q[u])));
+    }
+    int64_t t[8];
+    transform8(in, t);
+    int32_t* row = tile + group * kTilePitch + 8u * r;
 #pragma unroll
-    for (uint32_t v = 0; v < 8; ++v) s += static_cast<int64_t>(a[8 * y + v]) * work[blk][8 * v + x];
-    smp[blk][e] = static_cast<uint8_t>(clamp255((s + (128ll << 31) + (1ll << 30)) >> 31));
+    for (uint32_t x = 0; x < 8; ++x) row[x] = static_cast<int32_t>((t[x] + (1 << 8)) >> 9);
+  }
+  __syncwarp();  // the eight threads of a block are in one warp
+  if (live) {
+    // column r of the block
+    int32_t in[8];
+#pragma unroll
+    for (uint32_t v = 0; v < 8; ++v) in[v] = tile[group * kTilePitch + 8u * v + r];
+    int64_t sum[8];
+    transform8(in, sum);
+#pragma unroll
+    for (uint32_t y = 0; y < 8; ++y)
+      smp[group][8u * y + r] = static_cast<uint8_t>(
+          clamp255(static_cast<int32_t>((sum[y] + (128ll << 31) + (1ll << 30)) >> 31)));
   }
   __syncthreads();
-  // the MCU's pixels: 8 hmax x 8 vmax; a chroma sample serves hmax x vmax of them
-  const uint32_t mw = 8 * d.hmax, mh = 8 * d.vmax;
-  const uint32_t mx = blockIdx.x % d.mcu_cols, my = blockIdx.x / d.mcu_cols;
+  // the MCUs' pixels: 8 hmax x 8 vmax each (hmax, vmax are 1 or 2); a chroma sample serves
+  // hmax x vmax of them
+  const uint32_t xs = d.hmax >> 1, ys_ = d.vmax >> 1;          // shifts: log2 of hmax, vmax
+  const uint32_t mw_log = 3u + xs, px_log = 6u + xs + ys_;       // log2 of the MCU's width, pixels
+  const uint32_t here = min(held, mcus - first);
+  const uint32_t nluma = d.hs[0] * d.vs[0];
   uint8_t* img = p.pixels + d.pix_off;
-  for (uint32_t i = tid; i < mw * mh; i += blockDim.x) {
-    const uint32_t py = i / mw, px = i - py * mw;
-    const uint32_t gy = my * mh + py, gx = mx * mw + px;
+  for (uint32_t i = tid; i < (here << px_log); i += kIdctThreads) {
+    const uint32_t loc = i >> px_log, within = i & ((1u << px_log) - 1u);
+    const uint32_t py = within >> mw_log, px = within & ((1u << mw_log) - 1u);
+    const uint32_t m = first + loc;
+    const uint32_t my = m / d.mcu_cols, mx = m - my * d.mcu_cols;
+    const uint32_t gy = (my << (3u + ys_)) + py, gx = (mx << mw_log) + px;
     if (gy >= d.h || gx >= d.w) continue;
+    const uint32_t base = loc * per_mcu;
     // the luma block that holds the pixel (raster order inside the MCU)
-    const uint32_t yb = (py >> 3) * d.hs[0] + (px >> 3);
-    const uint32_t ys = smp[yb][8 * (py & 7u) + (px & 7u)];
-    uint32_t r = ys, g = ys, b = ys;
+    const uint32_t ys = smp[base + (py >> 3) * d.hs[0] + (px >> 3)][8u * (py & 7u) + (px & 7u)];
+    uint32_t red = ys, green = ys, blue = ys;
     if (d.ncomp == 3) {
-      const uint32_t cx = px / d.hmax, cy = py / d.vmax;  // chroma sampled once per MCU block
-      const uint32_t nluma = d.hs[0] * d.vs[0];
-      const int64_t y16 = static_cast<int64_t>(ys) << 16;
-      const int64_t cb = static_cast<int64_t>(smp[nluma][8 * cy + cx]) - 128;
-      const int64_t cr = static_cast<int64_t>(smp[nluma + 1][8 * cy + cx]) - 128;
+      const uint32_t at = 8u * (py >> ys_) + (px >> xs);  // chroma sampled once per MCU block
+      const int32_t y16 = static_cast<int32_t>(ys << 16) + (1 << 15);
+      const int32_t cb = static_cast<int32_t>(smp[base + nluma][at]) - 128;
+      const int32_t cr = static_cast<int32_t>(smp[base + nluma + 1][at]) - 128;
       // the JFIF coefficients as round(2^16 c); one rounding each
-      r = clamp255((y16 + 91881 * cr + (1 << 15)) >> 16);
-      g = clamp255((y16 - 22553 * cb - 46802 * cr + (1 << 15)) >> 16);
-      b = clamp255((y16 + 116130 * cb + (1 << 15)) >> 16);
+      red = clamp255((y16 + 91881 * cr) >> 16);
+      green = clamp255((y16 - 22553 * cb - 46802 * cr) >> 16);
+      blue = clamp255((y16 + 116130 * cb) >> 16);
     }
     uint8_t* out = img + 3ull * (static_cast<uint64_t>(gy) * d.w + gx);
-    out[0] = static_cast<uint8_t>(r);
-    out[1] = static_cast<uint8_t>(g);
-    out[2] = static_cast<uint8_t>(b);
+    out[0] = static_cast<uint8_t>(red);
+    out[1] = static_cast<uint8_t>(green);
+    out[2] = static_cast<uint8_t>(blue);
   }
 }
 
@@ -616,8 +653,9 @@ extern "C" int preba_jpeg_decode(const preba_jpeg_batch_t* b, void* stream) {
     b->table_host[i].h = p.h;
     b->table_host[i].w = p.w;
     most_seg = l.nseg > most_seg ? l.nseg : most_seg;
-    const uint32_t mcus = l.mcu_cols * l.mcu_rows;
-    most_mcus = mcus > most_mcus ? mcus : most_mcus;
+    // CTAs of the inverse transform: as many whole MCUs each as its 32 blocks hold
+    const uint32_t mcus = l.mcu_cols * l.mcu_rows, held = mcus_per_cta(before);
+    most_mcus = (mcus + held - 1) / held > most_mcus ? (mcus + held - 1) / held : most_mcus;
     at_seg += 2ull * l.nseg;
     at_scan += align_up(p.scan_len, 16);
     at_block += l.blocks;
@@ -639,7 +677,7 @@ extern "C" int preba_jpeg_decode(const preba_jpeg_batch_t* b, void* stream) {
     p.n = b->n;
     find_segments<<<b->n, 256, 0, s>>>(p);
     decode_segments<<<dim3((most_seg + 63) / 64, b->n), 64, 0, s>>>(p);
-    idct_colour<<<dim3(most_mcus, b->n), 64 * kMaxMcuBlocks, 0, s>>>(p);
+    idct_colour<<<dim3(most_mcus, b->n), kIdctThreads, 0, s>>>(p);
     err = cudaGetLastError();
   }
   if (err != cudaSuccess) {
