@@ -600,7 +600,17 @@ int preba_audio_query(const uint32_t* lengths, uint32_t n, preba_audio_sizes_t* 
 int preba_audio_pack(const float* const* utterances, const uint32_t* lengths, uint32_t n,
                      float* packed, uint64_t capacity_samples, preba_utt_t* table);
 
-/* Mel spectrogram (+ Normalize when `normalize` is non-zero) of a device-resident batch:
+/* Bits of the `normalize` argument of preba_audio_logmel.  With PREBA_AUDIO_OVERLAP_PREVIOUS
+ * the spectrogram kernel starts without waiting for the kernels before it on the stream
+ * (programmatic dependent launch: its CTAs move in while the Normalize kernel of the batch
+ * before is still running), under the contract of PREBA_OVERLAP_PREVIOUS: it may run beside
+ * every kernel back to the last operation on the stream that was not marked, so it must share
+ * no buffer with any of them; completion stays in stream order. */
+#define PREBA_AUDIO_NORMALIZE 1
+#define PREBA_AUDIO_OVERLAP_PREVIOUS 2
+
+/* Mel spectrogram (+ Normalize when bit PREBA_AUDIO_NORMALIZE of `normalize` is set) of a
+ * device-resident batch:
  * enqueues one kernel for the log Mel energies (the frame pairs of the batch are shared out
  * evenly over the warps of a grid that fills the GPU once; a warp transforms two frames with
  * one complex 512-point FFT held in registers) and, when normalising, one more for the three
@@ -609,7 +619,8 @@ int preba_audio_pack(const float* const* utterances, const uint32_t* lengths, ui
  * entry that is misaligned, runs past the samples or whose frame count does not follow from
  * its length is refused on the host when `table_host` is given (PREBA_ERR_BAD_TABLE) and
  * skipped and reported by the kernel otherwise.
- * Errors: PREBA_ERR_INVALID_ARG, PREBA_ERR_BUFFER_TOO_SMALL, PREBA_ERR_BAD_TABLE, PREBA_ERR_CUDA. */
+ * Errors: PREBA_ERR_INVALID_ARG (also: bits of `normalize` other than the two above),
+ * PREBA_ERR_BUFFER_TOO_SMALL, PREBA_ERR_BAD_TABLE, PREBA_ERR_CUDA. */
 int preba_audio_logmel(const preba_audio_batch_t* batch, int normalize, void* stream);
 
 /*

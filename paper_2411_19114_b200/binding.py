@@ -765,12 +765,16 @@ def preba_audio_pack(utterances, packed: np.ndarray | None = None,
     return packed, table
 
 
+AUDIO_NORMALIZE, AUDIO_OVERLAP_PREVIOUS = 1, 2
+
+
 class PreparedAudio:
     """The arguments of one ``preba_audio_logmel`` call, marshalled once.  ``samples``, ``table``,
     ``out`` (float32 [n, 80, t_max]) and ``status`` are CUDA tensors."""
 
     def __init__(self, samples, table, n: int, t_max: int, out, normalize: bool = True,
-                 stream=None, table_host: np.ndarray | None = None, status=None):
+                 stream=None, table_host: np.ndarray | None = None, status=None,
+                 overlap_previous: bool = False):
         import torch
 
         if stream is None:
@@ -785,7 +789,8 @@ class PreparedAudio:
         b.out, b.out_bytes = out.data_ptr(), out.numel() * out.element_size()
         b.status = status.data_ptr() if status is not None else None
         self._keep = (samples, table, out, status, table_host, b)
-        self._args = (ctypes.byref(b), int(bool(normalize)), ctypes.c_void_p(stream))
+        bits = (AUDIO_NORMALIZE if normalize else 0) | (AUDIO_OVERLAP_PREVIOUS if overlap_previous else 0)
+        self._args = (ctypes.byref(b), bits, ctypes.c_void_p(stream))
 
     def __call__(self) -> None:
         rc = lib().preba_audio_logmel(*self._args)

@@ -487,6 +487,9 @@ logmel_kernel(const AudioParams p, const MelPlan plan_param) {
     float* __restrict__ o = p.out + row * p.t_max;
     for (uint32_t t = frames + lane; t < p.t_max; t += 32) o[t] = 0.f;
   }
+  // A launch marked as overlapping started without waiting for the kernels before it on the
+  // stream; it does not complete before them (stream order of completion is kept).
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   if (gwarp == 0) {  // refused entries are reported once
     bool bad = false;
     for (uint32_t i = lane; i < p.n; i += 32) bad |= !utt_ok(p.table[i], p.samples_count);
@@ -500,7 +503,10 @@ logmel_kernel(const AudioParams p, const MelPlan plan_param) {
 constexpr int kHold = 48;
 
 __global__ void __launch_bounds__(256) normalize_kernel(const AudioParams p) {
-  // launched as a programmatic dependent of the spectrogram kernel: wait for its results
+  // launched as a programmatic dependent of the spectrogram kernel: let the launch behind
+  // this one be scheduled (a spectrogram marked as overlapping moves in as these CTAs retire),
+  // then wait for the spectrogram's results
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");
   const uint32_t lane = threadIdx.x & 31;
   const uint32_t row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -794,7 +800,8 @@ int resident_ctas(cudaError_t* err) {
 
 extern "C" int preba_audio_logmel(const preba_audio_batch_t* b, int normalize, void* stream) {
   using namespace preba::audio;
-  if (!b || !b->samples || !b->table || !b->out || b->n == 0 || b->n > 65535 || b->t_max == 0)
+  if (!b || !b->samples || !b->table || !b->out || b->n == 0 || b->n > 65535 || b->t_max == 0 ||
+      (normalize & ~(PREBA_AUDIO_NORMALIZE | PREBA_AUDIO_OVERLAP_PREVIOUS)) != 0)
     return PREBA_ERR_INVALID_ARG;
   if (reinterpret_cast<uintptr_t>(b->samples) % 16 || reinterpret_cast<uintptr_t>(b->out) % 4 ||
       reinterpret_cast<uintptr_t>(b->table) % 8)
@@ -831,10 +838,18 @@ extern "C" int preba_audio_logmel(const preba_audio_batch_t* b, int normalize, v
     const uint64_t want = (pairs + 2 * kWarps - 1) / (2 * kWarps);
     const uint32_t blocks = static_cast<uint32_t>(
         std::max<uint64_t>(1, std::min<uint64_t>(want, static_cast<uint64_t>(resident))));
-    logmel_kernel<<<blocks, 32 * kWarps, 0, s>>>(p, mel);
-    err = cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(blocks);
+    cfg.blockDim = dim3(32 * kWarps);
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = (normalize & PREBA_AUDIO_OVERLAP_PREVIOUS) ? 1 : 0;
+    err = cudaLaunchKernelEx(&cfg, logmel_kernel, p, mel);
   }
-  if (err == cudaSuccess && normalize) {
+  if (err == cudaSuccess && (normalize & PREBA_AUDIO_NORMALIZE)) {
     const uint32_t rows = b->n * kMels;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((rows + 7) / 8);

@@ -252,3 +252,46 @@ def test_resample_then_log_mel_end_to_end():
     assert int(status.item()) == 0
     want = oa.preprocess([oa.resample(u, 48000, 16000) for u in utts])
     assert float(np.max(np.abs(feat.cpu().numpy().astype(np.float64) - want[:, :, :t_max]))) <= NORM_TOL
+
+
+@pytest.mark.gpu
+def test_steps_marked_as_overlapping_leave_the_same_bits_and_complete_in_order():
+    """A chain of steps whose spectrogram kernels start without waiting for the step before
+    (each into buffers of its own), then a copy ordered behind them without any device-wide
+    wait: every result is what a step alone leaves."""
+    import torch
+
+    dev = torch.device("cuda:0")
+    utts = wl.utterances(12, seed=901)
+    packed, table = pb.preba_audio_pack(utts)
+    t_max = int(table["frames"].max())
+    n = len(utts)
+    smp = torch.from_numpy(packed).to(dev)
+    tab = torch.from_numpy(table.view(np.uint8)).to(dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    alone = torch.empty((n, 80, t_max), dtype=torch.float32, device=dev)
+    pb.preba_audio_logmel(smp, tab, n, t_max, alone, True, status=status)
+    torch.cuda.synchronize()
+    stream = torch.cuda.Stream(device=dev)
+    outs = [torch.full((n, 80, t_max), float("nan"), dtype=torch.float32, device=dev) for _ in range(5)]
+    host = [torch.empty((n, 80, t_max), dtype=torch.float32).pin_memory() for _ in range(5)]
+    done = torch.cuda.Event()
+    with torch.cuda.stream(stream):
+        for i, o in enumerate(outs):
+            pb.PreparedAudio(smp, tab, n, t_max, o, True, stream=stream, status=status,
+                             overlap_previous=i > 0)()
+        for o, h in zip(outs, host):
+            h.copy_(o, non_blocking=True)
+        done.record(stream)
+    done.synchronize()
+    assert int(status.item()) == 0
+    want = alone.cpu()
+    for h in host:
+        assert torch.equal(h, want)
+
+
+def test_unknown_bits_of_the_normalize_argument_are_refused():
+    import ctypes
+
+    b = pb.PrebaAudioBatch()
+    assert pb.lib().preba_audio_logmel(ctypes.byref(b), 4, None) == pb.ERR_INVALID_ARG
