@@ -371,9 +371,20 @@ __device__ __forceinline__ int32_t receive_extend(BitReader& br, uint32_t n) {
 // A thread per piece of a scan (blockIdx.y: image).  Writes the quantised coefficients of its
 // MCUs' blocks, natural order, into the zeroed coefficient buffer: per MCU the blocks of
 // component 0, then 1, then 2, each in raster order inside the MCU.
-__global__ void __launch_bounds__(64) decode_segments(const Params p) {
+#ifndef PREBA_JPEG_LANES
+#define PREBA_JPEG_LANES 4
+#endif
+// Lanes of a warp that decode (the others idle): lanes in different places of the decoding
+// loops run in turn, so a warp with few of them wastes little, and more warps keep the
+// schedulers busy while each waits for its own chain of dependent instructions.
+constexpr uint32_t kDecodeLanes = PREBA_JPEG_LANES;
+constexpr uint32_t kDecodeThreads = 128;
+constexpr uint32_t kDecodePerBlock = kDecodeThreads / 32 * kDecodeLanes;
+
+__global__ void __launch_bounds__(kDecodeThreads) decode_segments(const Params p) {
   const Desc& d = desc_of(p, blockIdx.y);
-  const uint32_t s = blockIdx.x * blockDim.x + threadIdx.x;
+  if ((threadIdx.x & 31u) >= kDecodeLanes) return;
+  const uint32_t s = blockIdx.x * kDecodePerBlock + (threadIdx.x >> 5) * kDecodeLanes + (threadIdx.x & 31u);
   if (s >= d.nseg) return;
   const uint32_t* seg = reinterpret_cast<const uint32_t*>(p.stage) + d.seg_off;
   const uint32_t lo = seg[s], hi = seg[d.nseg + s];
@@ -676,7 +687,7 @@ extern "C" int preba_jpeg_decode(const preba_jpeg_batch_t* b, void* stream) {
     p.status = b->status;
     p.n = b->n;
     find_segments<<<b->n, 256, 0, s>>>(p);
-    decode_segments<<<dim3((most_seg + 63) / 64, b->n), 64, 0, s>>>(p);
+    decode_segments<<<dim3((most_seg + kDecodePerBlock - 1) / kDecodePerBlock, b->n), kDecodeThreads, 0, s>>>(p);
     idct_colour<<<dim3(most_mcus, b->n), kIdctThreads, 0, s>>>(p);
     err = cudaGetLastError();
   }
