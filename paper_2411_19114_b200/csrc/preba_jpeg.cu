@@ -341,31 +341,40 @@ struct BitReader {
   }
 };
 
-// DECODE (F.2.2.3) with the 8-bit look-up in front; returns 256 on a code that does not exist.
-__device__ __forceinline__ uint32_t decode_symbol(BitReader& br, const Huff& t) {
+// One step of the decoder: DECODE (F.2.2.3, the 8-bit look-up in front) and, for a symbol that
+// announces `size` further bits (all of a DC symbol, the low four bits of an AC symbol),
+// RECEIVE and EXTEND (F.2.2.4, F.2.2.1), out of one 32-bit window of the stream: a code has at
+// most 16 bits and a value at most 15.  Returns the symbol (256: no such code) and the value.
+__device__ __forceinline__ uint32_t decode_step(BitReader& br, const Huff& t, bool dc, int32_t* value) {
   br.fill();
-  const uint32_t fast = t.look[br.peek(8)];
+  const uint32_t w = br.peek(32);
+  uint32_t len, sym;
+  const uint32_t fast = t.look[w >> 24];
   if (fast) {
-    br.skip(fast >> 8);
-    return fast & 0xffu;
-  }
-  const uint32_t bits16 = br.peek(16);
-  for (uint32_t l = 9; l <= 16; ++l) {
-    const int32_t code = static_cast<int32_t>(bits16 >> (16 - l));
-    if (code <= t.maxcode[l]) {
-      br.skip(l);
-      return t.vals[(code + t.valoff[l]) & 255];
+    len = fast >> 8;
+    sym = fast & 0xffu;
+  } else {
+    len = 0;
+    sym = 256u;
+    for (uint32_t l = 9; l <= 16; ++l) {
+      const int32_t code = static_cast<int32_t>(w >> (32 - l));
+      if (code <= t.maxcode[l]) {
+        len = l;
+        sym = t.vals[(code + t.valoff[l]) & 255];
+        break;
+      }
     }
+    if (sym > 255u) return sym;
   }
-  return 256u;
-}
-
-// RECEIVE and EXTEND (F.2.2.4, F.2.2.1) for 1 <= n <= 16 bits.
-__device__ __forceinline__ int32_t receive_extend(BitReader& br, uint32_t n) {
-  br.fill();
-  const int32_t v = static_cast<int32_t>(br.peek(n));
-  br.skip(n);
-  return v < (1 << (n - 1)) ? v - (1 << n) + 1 : v;
+  const uint32_t size = dc ? sym : (sym & 15u);
+  int32_t v = 0;
+  if (size != 0 && size <= 15u) {
+    v = static_cast<int32_t>((w << len) >> (32 - size));
+    if (v < (1 << (size - 1))) v += 1 - (1 << size);
+  }
+  br.skip(len + (size <= 15u ? size : 0u));
+  *value = v;
+  return sym;
 }
 
 // A thread per piece of a scan (blockIdx.y: image).  Writes the quantised coefficients of its
@@ -406,15 +415,16 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_segments(const Params p
       const Huff& dc = d.dc[c];
       const Huff& ac = d.ac[c];
       for (uint32_t b = 0; b < d.hs[c] * d.vs[c]; ++b, block += 64) {
-        const uint32_t t = decode_symbol(br, dc);
+        int32_t v;
+        const uint32_t t = decode_step(br, dc, true, &v);
         if (t > 11) {
           report(p.status, PREBA_ERR_BAD_STREAM);
           return;
         }
-        if (t) pred[c] += receive_extend(br, t);
+        pred[c] += v;
         block[0] = static_cast<int16_t>(pred[c]);
         for (uint32_t k = 1; k < 64;) {
-          const uint32_t rs = decode_symbol(br, ac);
+          const uint32_t rs = decode_step(br, ac, false, &v);
           if (rs > 255) {
             report(p.status, PREBA_ERR_BAD_STREAM);
             return;
@@ -430,7 +440,7 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_segments(const Params p
             report(p.status, PREBA_ERR_BAD_STREAM);
             return;
           }
-          block[kZigzagDev[k]] = static_cast<int16_t>(receive_extend(br, size));
+          block[kZigzagDev[k]] = static_cast<int16_t>(v);
           ++k;
         }
       }
