@@ -46,7 +46,7 @@ TRAFFIC_NOTE = ("dram read + write bytes summed over 8 consecutive launches of t
 
 # The same for the antialiased kernel: captured on 32 frames of 1080 x 1920 (traffic grows in
 # proportion to the frames, so a launch over n frames is taken as n / 32 of it).
-AA_NCU_TRAFFIC = {"csrc_sha1": "eb53a32665be9a6c1728bb1bd54f25d05e5bafc8", "frames": 32,
+AA_NCU_TRAFFIC = {"csrc_sha1": "55e9f17f9e819ba125b9eb1d2077e366cb9c484e", "frames": 32,
                   "bytes": 90032640 + 7090944}
 
 

@@ -7,8 +7,12 @@
 //   W = max(0, 2M - |(2j+1) R - (2X+1) n_in|)        (an integer; the triangle times 2M)
 // so taps and un-normalised weights come from exact integer arithmetic; the sums run in fp32.
 //
-// One CTA produces `rows` consecutive output rows of one image, two at a time (neighbouring
-// rows share about half of their input rows).  Per pair of output rows:
+// Three kernels share a batch, chosen per image by mm2_plan and mma_plan below: one with both
+// passes on the tensor cores (images reduced more than 2.5 times vertically), one with the
+// horizontal pass on them, and the general one described next; each skips the others' images.
+//
+// The general kernel: one CTA produces `rows` consecutive output rows of one image, two at a
+// time (neighbouring rows share about half of their input rows).  Per pair of output rows:
 //   vertical pass   every thread owns up to kWords 4-byte words of the needed byte range of
 //                   the input rows and accumulates them into both rows' sums, all loads of a
 //                   row in flight together; the results go to shared memory, one plane per
