@@ -54,8 +54,11 @@ want8 = oracle.preprocess_ex(imgs[:n], 224, 256, MEAN, STD, oracle.OUT_U8_HWC, c
                              round_u8=True)
 assert np.array_equal(out8.cpu().numpy(), want8)
 
-# antialiased Resize: both kernels (widths that are and are not multiples of 4)
-aa_imgs = [u(1080, 1920), u(600, 808), u(700, 901), u(241, 499), u(100, 150), u(64, 2000)]
+# antialiased Resize: all its kernels (both passes on the tensor cores with windows of three and
+# of four steps, the horizontal pass on them, the general one: widths that are and are not
+# multiples of 4)
+aa_imgs = [u(1080, 1920), u(1600, 1600), u(600, 808), u(700, 901), u(241, 499), u(100, 150),
+           u(64, 2000)]
 pk, tb = pb.preba_pack(aa_imgs)
 out = torch.empty((len(aa_imgs), 3, 224, 224), dtype=torch.float32, device=dev)
 for host in (tb, None):
