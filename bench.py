@@ -39,7 +39,7 @@ FALLBACK_HBM_GBS = 6650.0
 # without cache flushes between launches, divided by the launch count (so the write-back of a
 # launch's result, which happens while later launches run, is inside the window).  Valid only
 # for the kernel sources with this digest (else reported as null).
-NCU_TRAFFIC = {"csrc_sha1": "e32d7677e8894a744d578d45ab02134ed607a9f2", "bytes_per_launch": 75661344 + 76510784}
+NCU_TRAFFIC = {"csrc_sha1": "81497e8b38d1e1376b16577b2c748b1bd37ec458", "bytes_per_launch": 75668384 + 76500544}
 TRAFFIC_NOTE = ("dram read + write bytes summed over 8 consecutive launches of this loop (one "
                 "ncu pass, caches not flushed between launches) / 8")
 

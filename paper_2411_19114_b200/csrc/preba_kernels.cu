@@ -83,8 +83,8 @@ struct Params {
   uint32_t n;
   uint32_t C;           // crop side
   uint32_t S;           // resized shorter side
-  uint32_t slab_rows;   // output rows per task: 32, or 16 / 8 / 4 when a launch that runs alone
-                        // would leave warps without a task
+  uint32_t slab_rows;   // output rows per task: 32, or fewer (down to 4) in a launch that runs
+                        // alone, so that its busiest warp has the least to do
   uint32_t slabs;       // slabs per image
   uint32_t col_blocks;  // column blocks per image
   uint32_t tasks;       // n * slabs * col_blocks
@@ -1143,17 +1143,24 @@ int launch(const Params& given, int out_dtype, bool overlap, cudaStream_t stream
   const int resident = resident_ctas(variant, &err);
   Params p = given;
   if (err == cudaSuccess && !overlap) {
-    // A launch that runs alone is as long as its longest task.  While the batch has fewer
-    // tasks than the GPU has resident warps, halve the slabs (32 -> 16 -> 8 -> 4 output
-    // rows): more warps share the batch and the launch gets shorter, at the price of more
-    // staged halo rows.  The arithmetic per output element, and so the result, does not
-    // depend on the split.  Launches marked as overlapping their predecessor keep 32-row
-    // slabs: there the GPU is kept busy by the neighbouring launches and throughput counts.
+    // A launch that runs alone is as long as the work of its busiest warp: the rounds of tasks
+    // the resident warps need, times a task's rows (plus about four rows' worth of set-up and
+    // halo per task).  The slab height that makes this smallest is taken, between the full 32
+    // rows and kMinSlabRows (ties: the taller slab): 256 images of 224 rows get nine slabs of
+    // 25 rows each, one per warp, instead of fourteen of 16.  The arithmetic per output
+    // element, and so the result, does not depend on the split.  Launches marked as
+    // overlapping their predecessor keep 32-row slabs: there the GPU is kept busy by the
+    // neighbouring launches and throughput counts.
     const uint64_t warps = static_cast<uint64_t>(resident) * kWarpsPerCta;
-    while (p.slab_rows > kMinSlabRows &&
-           static_cast<uint64_t>(p.n) * ((p.C + p.slab_rows - 1) / p.slab_rows) * p.col_blocks <
-               warps)
-      p.slab_rows /= 2;
+    uint64_t best_cost = ~0ull;
+    uint32_t best_rows = p.slab_rows;
+    for (uint32_t r = p.slab_rows; r >= kMinSlabRows; --r) {
+      const uint64_t tasks = static_cast<uint64_t>(p.n) * ((p.C + r - 1) / r) * p.col_blocks;
+      const uint64_t cost = ((tasks + warps - 1) / warps) * (r + 4u);
+      if (cost < best_cost) best_cost = cost, best_rows = r;
+      if (r == 1) break;
+    }
+    p.slab_rows = best_rows;
     p.slabs = (p.C + p.slab_rows - 1) / p.slab_rows;
     p.tasks = static_cast<uint32_t>(static_cast<uint64_t>(p.n) * p.slabs * p.col_blocks);
   }
